@@ -1,0 +1,311 @@
+"""Pins for the oracle's local update step (Sec. 3, Sec. 6): K=1 is back-propagation, the last
+chunk's gradients are back-propagation's, finite differences with the chunk input frozen,
+independence of the chunks, schedule agreement, pipeline data flow."""
+import math
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+import lp_synth
+from oracle.local_step import LocalUpdateOracle
+
+TINY = {
+    "mlp": lp_synth.config("c1", batch=6, d_in=7, chunks=[[6], [5, 4], [6]], classes=5),
+    "lm": lp_synth.config("c3", batch=2, seq_len=5, vocab=11, d_model=8, n_heads=2, d_ffn=12,
+                          blocks_per_chunk=[1, 2, 1]),
+    "resnet": lp_synth.config("c4", batch=3, height=4, width=4, stem_channels=4,
+                              stage_channels=[4, 6], blocks_per_stage=2, classes=3),
+}
+
+
+def one_chunk(cfg):
+    c = lp_synth.config(cfg["name"], **{k: v for k, v in cfg.items() if k not in ("name",)})
+    if cfg["family"] == "mlp":
+        c["chunks"] = [[w for ch in cfg["chunks"] for w in ch]]
+    elif cfg["family"] == "lm":
+        c["blocks_per_chunk"] = [sum(cfg["blocks_per_chunk"])]
+    return c
+
+
+def spread_params(cfg, seed=5):
+    """Initial parameters with every tensor perturbed so that no gradient is trivially zero."""
+    p = lp_synth.init_params(dict(cfg, dtype="fp32"))
+    g = np.random.default_rng(seed)
+    return {n: (a.astype(np.float64) + 0.3 * g.standard_normal(a.shape)) for n, a in p.items()}
+
+
+# ---------------------------------------------------------------- independent reverse mode (torch)
+
+def torch_forward(cfg, P, x, upto=None):
+    """The same networks written with torch's own operators; returns the trunk output after
+    chunk `upto` (default: the last).  P maps oracle parameter names to torch tensors."""
+    fam = cfg["family"]
+    K = lp_synth.num_chunks(cfg)
+    upto = K - 1 if upto is None else upto
+    if fam == "mlp":
+        h = x
+        for k in range(upto + 1):
+            for i in range(len(cfg["chunks"][k])):
+                h = F.relu(F.linear(h, P[f"c{k}.l{i}.W"], P[f"c{k}.l{i}.b"]))
+        return h
+    if fam == "lm":
+        d, H = cfg["d_model"], cfg["n_heads"]
+        B, T = x.shape
+        h = P["c0.tok"][x] + P["c0.pos"][None]
+        blk = 0
+        for k in range(upto + 1):
+            for _ in range(cfg["blocks_per_chunk"][k]):
+                n = f"c{k}.b{blk}"
+                a = F.layer_norm(h, (d,), P[n + ".ln1.g"], P[n + ".ln1.b"], 1e-5)
+                qkv = F.linear(a, P[n + ".Wqkv"], P[n + ".bqkv"])
+                q, kk, v = (t.reshape(B, T, H, d // H).transpose(1, 2) for t in qkv.split(d, dim=-1))
+                o = F.scaled_dot_product_attention(q, kk, v, is_causal=True)
+                h = h + F.linear(o.transpose(1, 2).reshape(B, T, d), P[n + ".Wo"], P[n + ".bo"])
+                a = F.layer_norm(h, (d,), P[n + ".ln2.g"], P[n + ".ln2.b"], 1e-5)
+                h = h + F.linear(F.gelu(F.linear(a, P[n + ".W1"], P[n + ".b1"])), P[n + ".W2"], P[n + ".b2"])
+                blk += 1
+        return h
+    h = x
+    for k in range(upto + 1):
+        if k == 0:
+            h = F.relu(F.batch_norm(F.conv2d(h, P["c0.stem.conv"], padding=1), None, None,
+                                    P["c0.stem.bn.g"], P["c0.stem.bn.b"], True, 0.1, 1e-5))
+        for j in range(cfg["blocks_per_stage"]):
+            n = f"c{k}.r{j}"
+            s = lp_synth.resnet_stage_stride(cfg, k) if j == 0 else 1
+            u = F.conv2d(h, P[n + ".conv1"], stride=s, padding=1)
+            u = F.relu(F.batch_norm(u, None, None, P[n + ".bn1.g"], P[n + ".bn1.b"], True, 0.1, 1e-5))
+            u = F.conv2d(u, P[n + ".conv2"], padding=1)
+            u = F.batch_norm(u, None, None, P[n + ".bn2.g"], P[n + ".bn2.b"], True, 0.1, 1e-5)
+            if n + ".sc.conv" in P:
+                sc = F.conv2d(h, P[n + ".sc.conv"], stride=s)
+                sc = F.batch_norm(sc, None, None, P[n + ".sc.bn.g"], P[n + ".sc.bn.b"], True, 0.1, 1e-5)
+            else:
+                sc = h
+            h = F.relu(u + sc)
+    return h
+
+
+def torch_head_loss(cfg, P, k, h, y):
+    fam = cfg["family"]
+    if fam == "lm":
+        a = F.layer_norm(h, (cfg["d_model"],), P[f"c{k}.head.ln.g"], P[f"c{k}.head.ln.b"], 1e-5)
+        z = F.linear(a, P[f"c{k}.head.W"], P[f"c{k}.head.b"])
+        return F.cross_entropy(z.reshape(-1, z.shape[-1]), y.reshape(-1).long(), ignore_index=-1)
+    if fam == "resnet":
+        h = h.mean(dim=(2, 3))
+    return F.cross_entropy(F.linear(h, P[f"c{k}.head.W"], P[f"c{k}.head.b"]), y.long())
+
+
+def torch_backprop_grads(cfg, params, x, y, head_chunk):
+    """Ordinary full back-propagation of the loss of head `head_chunk` through everything below."""
+    P = {n: torch.tensor(a, dtype=torch.float64, requires_grad=True) for n, a in params.items()}
+    xt = torch.tensor(x) if cfg["family"] == "lm" else torch.tensor(x, dtype=torch.float64)
+    h = torch_forward(cfg, P, xt, upto=head_chunk)
+    loss = torch_head_loss(cfg, P, head_chunk, h, torch.tensor(y))
+    loss.backward()
+    return float(loss.detach()), {n: (None if t.grad is None else t.grad.numpy()) for n, t in P.items()}
+
+
+def rel(a, b):
+    return np.abs(a - b).max() / max(np.abs(b).max(), 1e-30)
+
+
+# ---------------------------------------------------------------- P1: K = 1 is back-propagation
+
+@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+def test_single_chunk_equals_backprop(fam):
+    cfg = TINY[fam]
+    if fam == "resnet":
+        cfg = lp_synth.config("c4", **{k: v for k, v in cfg.items() if k != "name"})
+        cfg["stage_channels"] = [4]
+    else:
+        cfg = one_chunk(cfg)
+    params = spread_params(cfg)
+    x, y = lp_synth.minibatch(cfg, 0)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    loss, _, grads = orc.local_grads(0, orc._cast_input(x), y)
+    tloss, tg = torch_backprop_grads(cfg, params, x, y, 0)
+    assert abs(loss - tloss) < 1e-10 * max(1, abs(tloss))
+    for n in params:
+        assert tg[n] is not None, n
+        assert rel(grads[n], tg[n]) < 1e-9, n
+
+
+# ---------------------------------------------------------------- P2: last chunk = backprop's gradient
+
+@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+def test_last_chunk_gradients_are_backprop_gradients(fam):
+    cfg = TINY[fam]
+    K = lp_synth.num_chunks(cfg)
+    params = spread_params(cfg)
+    x, y = lp_synth.minibatch(cfg, 0)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    orc.cfg = dict(cfg, optim=dict(kind="sgdm", lr=0.0, momentum=0.0, weight_decay=0.0))
+    orc.step(x, y, "sync")
+    _, tg = torch_backprop_grads(cfg, params, x, y, K - 1)
+    for n in orc.names_of_chunk[K - 1]:
+        assert rel(orc.last_grads[n], tg[n]) < 1e-9, n
+    # ... and an earlier chunk's local gradient is NOT the gradient of the last loss (Sec. 1)
+    n0 = orc.names_of_chunk[0][0]
+    assert rel(orc.last_grads[n0], tg[n0]) > 1e-3
+
+
+# ---------------------------------------------------------------- P3: finite differences, input frozen
+
+@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+def test_local_gradients_match_finite_differences(fam):
+    cfg = TINY[fam]
+    K = lp_synth.num_chunks(cfg)
+    params = spread_params(cfg, seed=9)
+    x, y = lp_synth.minibatch(cfg, 0)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    inp = orc._cast_input(x)
+    rng = np.random.default_rng(0)
+    for k in range(K):
+        loss, h, grads = orc.local_grads(k, inp, y)
+        for n in orc.names_of_chunk[k]:
+            w = orc.p[n]
+            flat = w.reshape(-1)
+            for idx in rng.choice(flat.size, size=min(4, flat.size), replace=False):
+                old = flat[idx]
+                eps = 1e-6
+                flat[idx] = old + eps
+                lp = orc.local_grads(k, inp, y)[0]
+                flat[idx] = old - eps
+                lm = orc.local_grads(k, inp, y)[0]
+                flat[idx] = old
+                fd = (lp - lm) / (2 * eps)
+                an = grads[n].reshape(-1)[idx]
+                assert abs(fd - an) <= 2e-6 * max(1.0, abs(fd), np.abs(grads[n]).max()), (n, idx, fd, an)
+        inp = h
+
+
+# ---------------------------------------------------------------- P4: chunks are independent
+
+@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+def test_chunk_update_ignores_other_chunks_heads_and_losses(fam):
+    cfg = TINY[fam]
+    K = lp_synth.num_chunks(cfg)
+    params = spread_params(cfg)
+    x, y = lp_synth.minibatch(cfg, 0)
+    a = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    a.step(x, y, "sync")
+    for k in range(K - 1):
+        p2 = {n: v.copy() for n, v in params.items()}
+        for j in range(k + 1, K):          # later chunks: different heads (hence different losses)
+            p2[f"c{j}.head.W"] = p2[f"c{j}.head.W"] * -3.0 + 1.0
+        b = LocalUpdateOracle(cfg, p2, dtype=np.float64)
+        b.step(x, y, "sync")
+        for n in a.names_of_chunk[k]:
+            assert np.array_equal(a.p[n], b.p[n]), n
+            assert np.array_equal(a.last_grads[n], b.last_grads[n]), n
+
+
+def test_stop_gradient_is_real():
+    """The local gradient of chunk 0 differs from d(sum of all losses)/d(theta_0): later losses do
+    depend on theta_0 through the forward pass, but that path is cut (Sec. 3, greedy)."""
+    cfg = TINY["mlp"]
+    params = spread_params(cfg)
+    x, y = lp_synth.minibatch(cfg, 0)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    orc.cfg = dict(cfg, optim=dict(kind="sgdm", lr=0.0, momentum=0.0, weight_decay=0.0))
+    orc.step(x, y, "sync")
+    n = "c0.l0.W"
+    w = orc.p[n]
+    idx = (1, 2)
+    tot = lambda: float(orc.forward(x, y)[1].sum())
+    old = w[idx]
+    w[idx] = old + 1e-6; fp = tot()
+    w[idx] = old - 1e-6; fm = tot()
+    w[idx] = old
+    fd_total = (fp - fm) / 2e-6
+    first = lambda: float(orc.forward(x, y)[1][0])
+    w[idx] = old + 1e-6; fp = first()
+    w[idx] = old - 1e-6; fm = first()
+    w[idx] = old
+    fd_first = (fp - fm) / 2e-6
+    g = orc.last_grads[n][idx]
+    assert abs(g - fd_first) < 1e-6 * max(1, abs(g))
+    assert abs(g - fd_total) > 1e-3 * max(1e-3, abs(g))
+
+
+# ---------------------------------------------------------------- P5: schedules
+
+@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+def test_sync_and_pipelined_agree_on_step0(fam):
+    cfg = TINY[fam]
+    params = spread_params(cfg)
+    x, y = lp_synth.minibatch(cfg, 0)
+    a = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    b = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    la = a.step(x, y, "sync")
+    lb = b.step(x, y, "pipelined")
+    assert np.array_equal(la, lb)
+    for n in a.p:
+        assert np.array_equal(a.p[n], b.p[n]), n
+
+
+def test_pipelined_chunk_k_sees_minibatch_t_minus_k_with_its_labels():
+    cfg = TINY["mlp"]
+    K = lp_synth.num_chunks(cfg)
+    params = spread_params(cfg)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    orc.cfg = dict(cfg, optim=dict(kind="sgdm", lr=0.0, momentum=0.0, weight_decay=0.0))
+    frozen = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    batches = [lp_synth.minibatch(cfg, t) for t in range(6)]
+    for t, (x, y) in enumerate(batches):
+        losses = orc.step(x, y, "pipelined")
+        for k in range(K):
+            src = max(t - k, 0)                # with frozen weights the loss identifies the batch
+            exp = frozen.forward(*batches[src])[1][k]
+            assert abs(losses[k] - exp) < 1e-12, (t, k)
+
+
+def test_pipelined_idle_rampup():
+    cfg = TINY["mlp"]
+    K = lp_synth.num_chunks(cfg)
+    orc = LocalUpdateOracle(cfg, spread_params(cfg), dtype=np.float64, ramp="idle")
+    for t in range(K + 1):
+        losses = orc.step(*lp_synth.minibatch(cfg, t), "pipelined")
+        assert [bool(np.isfinite(v)) for v in losses] == [k <= t for k in range(K)]
+
+
+def test_forward_chain_uses_start_of_step_weights():
+    """One forward per chunk per step, all with the weights the step began with (App. A.2, greedy:
+    one forward and one backward pass per layer per step)."""
+    cfg = TINY["mlp"]
+    params = spread_params(cfg)
+    x, y = lp_synth.minibatch(cfg, 0)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    before = orc.forward(x, y)[1]
+    losses = orc.step(x, y, "sync")
+    assert np.allclose(losses, before, rtol=0, atol=1e-13)
+
+
+# ---------------------------------------------------------------- P6, P12
+
+def test_initial_lm_loss_is_log_vocab():
+    cfg = lp_synth.config("c3", batch=2, seq_len=16, vocab=512, d_model=32, n_heads=2, d_ffn=64,
+                          blocks_per_chunk=[1, 1])
+    orc = LocalUpdateOracle(cfg, lp_synth.init_params(cfg), dtype=np.float64)
+    losses = orc.forward(*lp_synth.minibatch(cfg, 0))[1]
+    assert np.all(np.abs(losses - math.log(512)) < 5e-2)   # 30 valid rows: sampling noise ~1e-2
+
+
+def test_determinism_and_dtype_modes():
+    cfg = TINY["lm"]
+    outs = []
+    for _ in range(2):
+        orc = LocalUpdateOracle(cfg, lp_synth.init_params(cfg), dtype=np.float32)
+        ls = [orc.step(*lp_synth.minibatch(cfg, t)) for t in range(3)]
+        outs.append((np.array(ls), {n: v.copy() for n, v in orc.p.items()}))
+    assert np.array_equal(outs[0][0], outs[1][0])
+    for n in outs[0][1]:
+        assert np.array_equal(outs[0][1][n], outs[1][1][n])
+        assert outs[0][1][n].dtype == np.float32
+    o64 = LocalUpdateOracle(cfg, lp_synth.init_params(cfg), dtype=np.float64)
+    l64 = np.array([o64.step(*lp_synth.minibatch(cfg, t)) for t in range(3)])
+    assert np.allclose(outs[0][0], l64, rtol=1e-5)
