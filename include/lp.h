@@ -1,0 +1,198 @@
+/*
+ * lp.h -- C ABI of the local-update training step on one NVIDIA B200 (sm_100a).
+ *
+ * The method (paper Sec. 3, "Local Parallelism"): a network is cut into a sequence of K chunks.
+ * Chunk k runs its layers on the output of chunk k-1 (chunk 0 on the minibatch), feeds the result
+ * to an auxiliary head whose loss has the same form as the global objective, back-propagates that
+ * loss into its own layers only (the activation handed to the next chunk carries no gradient), and
+ * applies its own optimizer update (Sec. 1, Sec. 6: updates need not wait for the rest of the
+ * network).  Back-propagation is the case K = 1.
+ *
+ * All pointers named "device" are CUDA device pointers owned by the caller; "host" pointers are
+ * ordinary host memory.  Nothing here takes or returns a framework type.  Every entry point
+ * returns an lp_status (0 = LP_OK, negative = error) and never throws, aborts or traps; after an
+ * error lp_last_error(h) gives a message.  One handle may be used by one thread at a time.
+ */
+#ifndef LP_H_
+#define LP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lp_handle_s* lp_handle;
+typedef int lp_status;
+
+enum {
+  LP_OK = 0,
+  LP_ERR_INVALID_ARG = -1, /* null pointer, bad enum, bad index                                  */
+  LP_ERR_SHAPE = -2,       /* sizes that the model family cannot take (see lp_model_spec)        */
+  LP_ERR_UNSUPPORTED = -3, /* valid request that this build does not implement                   */
+  LP_ERR_ALLOC = -4,       /* device allocation failed                                           */
+  LP_ERR_CUDA = -5,        /* a CUDA call failed; message holds the CUDA error string            */
+  LP_ERR_STATE = -6,       /* call not allowed in the handle's current state                     */
+  LP_ERR_LABEL_RANGE = -7, /* lp_status_poll: a label or token id was outside its range          */
+  LP_ERR_NONFINITE = -8,   /* lp_status_poll: a loss was NaN or infinite                         */
+  LP_ERR_TIMEOUT = -9      /* lp_status_poll: a device-side wait gave up (kernel returned early)  */
+};
+
+enum { LP_FAMILY_MLP = 0, LP_FAMILY_LM = 1, LP_FAMILY_RESNET = 2 };
+enum { LP_FP32 = 0, LP_BF16 = 1 }; /* LP_BF16: bf16 matrices and activations, fp32 master weights,
+                                      fp32 accumulation, fp32 normalisation statistics and loss  */
+enum { LP_HEAD_LINEAR = 0, LP_HEAD_LN_LINEAR = 1, LP_HEAD_GAP_LINEAR = 2 };
+enum { LP_OPT_SGDM = 0, LP_OPT_ADAM = 1 };
+enum { LP_SYNC = 0, LP_PIPELINED = 1 };
+enum { LP_MASTER = 0, LP_WORKING = 1, LP_MOMENT1 = 2, LP_MOMENT2 = 3, LP_GRAD = 4 };
+
+/*
+ * Model description.  Only the fields of the chosen family are read.  Arrays are host pointers
+ * read during lp_create only.
+ *
+ *  MLP (App. A.1: matrix product, bias add, ReLU per layer): n_layers Linear+ReLU layers of widths
+ *    layer_widths[], input width d_in; chunk k holds layers_per_chunk[k] consecutive layers.
+ *  LM (App. B.2: decoder-only transformer, one or more layers per chunk): learned token and
+ *    position embeddings (in chunk 0), pre-LayerNorm blocks with causal softmax attention
+ *    (n_heads heads of d_model/n_heads = 64) and a GELU feed-forward of width d_ffn; chunk k holds
+ *    blocks_per_chunk[k] blocks.
+ *  RESNET (App. B.3): 3x3 stem convolution + BatchNorm + ReLU (in chunk 0), then K stages of
+ *    blocks_per_stage BasicBlocks with stage_channels[k] channels; stages after the first start
+ *    with stride 2 and a 1x1-convolution + BatchNorm shortcut.  BatchNorm uses batch statistics.
+ */
+typedef struct {
+  int family;
+  int dtype;
+  int batch;
+  /* MLP */
+  int d_in;
+  int n_layers;
+  const int* layer_widths;     /* [n_layers] */
+  const int* layers_per_chunk; /* [K] */
+  /* LM */
+  int vocab, seq_len, d_model, n_heads, d_ffn;
+  const int* blocks_per_chunk; /* [K] */
+  /* RESNET */
+  int in_channels, height, width, stem_channels;
+  const int* stage_channels; /* [K] */
+  int blocks_per_stage;
+  /* 0: tensor-core GEMMs wherever a problem's sizes allow (default); 1: plain FP32-ALU GEMMs
+     everywhere (diagnostic).  The fp32 dtype always uses the FP32-ALU GEMMs. */
+  int gemm_backend;
+} lp_model_spec;
+
+/* Auxiliary head of every chunk (Sec. 3: same form as the global objective): softmax
+ * cross-entropy over `classes` on top of Linear (MLP), LayerNorm+Linear (LM; classes = vocab) or
+ * global-average-pool+Linear (RESNET). */
+typedef struct {
+  int kind;
+  int classes;
+} lp_head_spec;
+
+/* Per-chunk optimizer (App. B: Adam, SGD with momentum).  SGDM: g += weight_decay*w on matrices,
+ * filters and embedding tables only; v = momentum*v + g; w -= lr*v.  ADAM: bias-corrected, step
+ * count from 1, eps added outside the square root. */
+typedef struct {
+  int kind;
+  float lr, momentum, weight_decay, beta1, beta2, eps;
+} lp_optim_spec;
+
+/* Optional allocator for the handle's device memory (e.g. backed by a framework's caching
+ * allocator).  alloc returns a device pointer aligned to 256 bytes or NULL.  If the lp_alloc
+ * pointer given to lp_create is NULL, cudaMalloc/cudaFree are used. */
+typedef struct {
+  void* (*alloc)(size_t bytes, void* user);
+  void (*release)(void* ptr, void* user);
+  void* user;
+} lp_alloc;
+
+typedef struct {
+  char name[48]; /* e.g. "c3.b3.Wqkv", "c0.head.W" */
+  int chunk;
+  int ndim;
+  int64_t shape[4]; /* Linear [out,in]; convolution filter [C_out,kh,kw,C_in]; embedding [rows,d] */
+  int64_t numel;
+  int has_working_bf16; /* 1 if a bf16 working copy exists (matrices under LP_BF16) */
+} lp_tensor_info;
+
+/*
+ * lp_create: build the K-chunk model, its heads and optimizer state on the current CUDA device
+ * (Sec. 3).  All parameters, optimizer state, saved activations and the boundary buffers are
+ * allocated here and owned by the handle.  Parameters start at zero: the caller installs initial
+ * values with lp_set_tensor.  Errors: INVALID_ARG, SHAPE (e.g. d_model/n_heads != 64, sizes not
+ * accepted by the family), UNSUPPORTED, ALLOC, CUDA.  On error *out is NULL.
+ */
+lp_status lp_create(const lp_model_spec* model, int K, const lp_head_spec* head,
+                    const lp_optim_spec* optim, const lp_alloc* alloc, lp_handle* out);
+
+/*
+ * lp_step: one local update step (Sec. 3; schedules: App. E.1 for the synchronous order, Sec. 6
+ * for the pipelined steady state).
+ *   x: device.  MLP: [batch, d_in] fp32 (LP_FP32) or bf16 (LP_BF16), row-major.  LM: int32 token
+ *      ids [batch, seq_len].  RESNET: [batch, C, H, W] (NCHW) fp32 or bf16.
+ *   y: device int32 labels.  MLP/RESNET: [batch].  LM: [batch, seq_len], -1 = position ignored.
+ *   schedule: LP_SYNC -- chunk k reads the output chunk k-1 produced in this step from the same
+ *      minibatch.  LP_PIPELINED -- chunk k reads the output chunk k-1 produced in the previous
+ *      step, with the labels of that older minibatch; the first pipelined step after lp_create or
+ *      lp_reset_pipeline fills the boundary buffers by a forward pass of (x, y).
+ *   stream: cudaStream_t (as void*) all work is issued on; no host synchronisation happens.
+ *   out_losses: device, K floats: each chunk's mean auxiliary loss for the minibatch it trained on.
+ * x, y and out_losses must stay valid until the caller synchronises `stream`.
+ * Errors: INVALID_ARG, STATE (sync step while a pipeline is in flight needs lp_reset_pipeline), CUDA.
+ */
+lp_status lp_step(lp_handle h, const void* x, const void* y, int schedule, void* stream,
+                  float* out_losses);
+
+/* lp_step_host: the same step with HOST buffers: copies x and y to the device, runs lp_step,
+ * copies the K losses back to out_losses_host and synchronises `stream` before returning. */
+lp_status lp_step_host(lp_handle h, const void* x_host, const void* y_host, int schedule,
+                       void* stream, float* out_losses_host);
+
+/*
+ * lp_forward: forward chain through all chunks with the current weights; no gradient, no update.
+ *   y may be NULL (then out_losses must be NULL).  out_logits (device, nullable) receives the last
+ *   chunk's head logits, [rows, classes] in the activation dtype, rows = batch (MLP, RESNET) or
+ *   batch*seq_len (LM).  out_losses (device, nullable): K floats.
+ */
+lp_status lp_forward(lp_handle h, const void* x, const void* y, void* stream, void* out_logits,
+                     float* out_losses);
+
+/* lp_destroy: release everything the handle owns.  NULL is accepted. */
+lp_status lp_destroy(lp_handle h);
+
+/* Parameter access (host buffers; these calls synchronise `stream`).  `which` selects the fp32
+ * master copy, the bf16 working copy (uint16 bit patterns), the optimizer moments (fp32) or the
+ * last step's gradient (fp32).  Setting LP_MASTER also refreshes the bf16 working copy. `bytes`
+ * must equal numel * element size, else LP_ERR_SHAPE. */
+int lp_num_tensors(lp_handle h);
+lp_status lp_tensor_info_get(lp_handle h, int i, lp_tensor_info* out);
+lp_status lp_get_tensor(lp_handle h, int i, int which, void* host_dst, size_t bytes, void* stream);
+lp_status lp_set_tensor(lp_handle h, int i, int which, const void* host_src, size_t bytes,
+                        void* stream);
+
+/* Forget the activations in flight between chunks; the next pipelined step refills them. */
+lp_status lp_reset_pipeline(lp_handle h);
+
+/* Read the device status word (synchronises `stream`): LP_OK, or LABEL_RANGE / NONFINITE /
+ * TIMEOUT if any kernel since the last poll flagged it.  The word is cleared. */
+lp_status lp_status_poll(lp_handle h, void* stream);
+
+/* Checkpoint: master weights, moments, step count, boundary buffers and their labels.
+ * lp_save_state / lp_load_state synchronise the device.  A handle restored into an identically
+ * created handle continues bit-for-bit. */
+size_t lp_state_size(lp_handle h);
+lp_status lp_save_state(lp_handle h, void* host_dst, size_t bytes);
+lp_status lp_load_state(lp_handle h, const void* host_src, size_t bytes);
+
+/* Number of kernel launches the last lp_step issued (for reporting). */
+int lp_last_step_launches(lp_handle h);
+/* Device bytes owned by the handle. */
+size_t lp_device_bytes(lp_handle h);
+/* Message of the last error on this handle (or of the last failed lp_create if h is NULL). */
+const char* lp_last_error(lp_handle h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LP_H_ */

@@ -1,0 +1,234 @@
+"""ctypes binding of liblp.so: the same entry points as include/lp.h, argument marshalling only.
+
+Every step of the local update runs inside the library's CUDA kernels.  PyTorch appears only as
+the owner of device buffers (``tensor.data_ptr()``) and streams.  If the library is missing the
+import fails: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liblp.so")
+
+LP_OK = 0
+LP_ERR = {-1: "INVALID_ARG", -2: "SHAPE", -3: "UNSUPPORTED", -4: "ALLOC", -5: "CUDA", -6: "STATE",
+          -7: "LABEL_RANGE", -8: "NONFINITE", -9: "TIMEOUT"}
+LP_FAMILY_MLP, LP_FAMILY_LM, LP_FAMILY_RESNET = 0, 1, 2
+LP_FP32, LP_BF16 = 0, 1
+LP_HEAD_LINEAR, LP_HEAD_LN_LINEAR, LP_HEAD_GAP_LINEAR = 0, 1, 2
+LP_OPT_SGDM, LP_OPT_ADAM = 0, 1
+LP_SYNC, LP_PIPELINED = 0, 1
+LP_MASTER, LP_WORKING, LP_MOMENT1, LP_MOMENT2, LP_GRAD = 0, 1, 2, 3, 4
+
+
+class LpError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"LP_ERR_{LP_ERR.get(code, code)}: {msg}")
+        self.code = code
+
+
+class lp_model_spec(C.Structure):
+    _fields_ = [("family", C.c_int), ("dtype", C.c_int), ("batch", C.c_int),
+                ("d_in", C.c_int), ("n_layers", C.c_int),
+                ("layer_widths", C.POINTER(C.c_int)), ("layers_per_chunk", C.POINTER(C.c_int)),
+                ("vocab", C.c_int), ("seq_len", C.c_int), ("d_model", C.c_int), ("n_heads", C.c_int),
+                ("d_ffn", C.c_int), ("blocks_per_chunk", C.POINTER(C.c_int)),
+                ("in_channels", C.c_int), ("height", C.c_int), ("width", C.c_int),
+                ("stem_channels", C.c_int), ("stage_channels", C.POINTER(C.c_int)),
+                ("blocks_per_stage", C.c_int), ("gemm_backend", C.c_int)]
+
+
+class lp_head_spec(C.Structure):
+    _fields_ = [("kind", C.c_int), ("classes", C.c_int)]
+
+
+class lp_optim_spec(C.Structure):
+    _fields_ = [("kind", C.c_int), ("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
+                ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float)]
+
+
+class lp_tensor_info(C.Structure):
+    _fields_ = [("name", C.c_char * 48), ("chunk", C.c_int), ("ndim", C.c_int), ("shape", C.c_int64 * 4),
+                ("numel", C.c_int64), ("has_working_bf16", C.c_int)]
+
+
+EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "lp_num_tensors",
+           "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
+           "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
+           "lp_last_error"]
+
+
+def load_library() -> C.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(f"{_LIB_PATH} is missing: run `python -m paper_2012_03837_b200.build` (needs nvcc)")
+    lib = C.CDLL(_LIB_PATH)
+    vp, ip = C.c_void_p, C.c_int
+    lib.lp_create.argtypes = [C.POINTER(lp_model_spec), ip, C.POINTER(lp_head_spec), C.POINTER(lp_optim_spec), vp, C.POINTER(vp)]
+    lib.lp_step.argtypes = [vp, vp, vp, ip, vp, vp]
+    lib.lp_step_host.argtypes = [vp, vp, vp, ip, vp, vp]
+    lib.lp_forward.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.lp_destroy.argtypes = [vp]
+    lib.lp_num_tensors.argtypes = [vp]
+    lib.lp_tensor_info_get.argtypes = [vp, ip, C.POINTER(lp_tensor_info)]
+    lib.lp_get_tensor.argtypes = [vp, ip, ip, vp, C.c_size_t, vp]
+    lib.lp_set_tensor.argtypes = [vp, ip, ip, vp, C.c_size_t, vp]
+    lib.lp_reset_pipeline.argtypes = [vp]
+    lib.lp_status_poll.argtypes = [vp, vp]
+    lib.lp_state_size.argtypes = [vp]
+    lib.lp_state_size.restype = C.c_size_t
+    lib.lp_save_state.argtypes = [vp, vp, C.c_size_t]
+    lib.lp_load_state.argtypes = [vp, vp, C.c_size_t]
+    lib.lp_last_step_launches.argtypes = [vp]
+    lib.lp_device_bytes.argtypes = [vp]
+    lib.lp_device_bytes.restype = C.c_size_t
+    lib.lp_last_error.argtypes = [vp]
+    lib.lp_last_error.restype = C.c_char_p
+    return lib
+
+
+_lib = load_library()
+
+
+def _check(h, code):
+    if code != LP_OK:
+        raise LpError(code, (_lib.lp_last_error(h) or b"").decode())
+
+
+def _ints(seq):
+    return (C.c_int * len(seq))(*[int(v) for v in seq])
+
+
+def _ptr(t):
+    """Device or host address of a torch tensor / numpy array / raw int."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def specs_from_config(cfg: dict, gemm_backend: int = 0):
+    """Translate a workload dictionary (see lp_synth.config) into the three C structs and K."""
+    m = lp_model_spec()
+    keep = []
+    fam = cfg["family"]
+    m.dtype = LP_BF16 if cfg["dtype"] == "bf16" else LP_FP32
+    m.batch = cfg["batch"]
+    m.gemm_backend = gemm_backend
+    hd = lp_head_spec()
+    if fam == "mlp":
+        m.family = LP_FAMILY_MLP
+        widths = [w for ch in cfg["chunks"] for w in ch]
+        per = [len(ch) for ch in cfg["chunks"]]
+        m.d_in, m.n_layers = cfg["d_in"], len(widths)
+        a, b = _ints(widths), _ints(per)
+        keep += [a, b]
+        m.layer_widths, m.layers_per_chunk = a, b
+        K = len(per)
+        hd.kind, hd.classes = LP_HEAD_LINEAR, cfg["classes"]
+    elif fam == "lm":
+        m.family = LP_FAMILY_LM
+        m.vocab, m.seq_len, m.d_model = cfg["vocab"], cfg["seq_len"], cfg["d_model"]
+        m.n_heads, m.d_ffn = cfg["n_heads"], cfg["d_ffn"]
+        a = _ints(cfg["blocks_per_chunk"])
+        keep.append(a)
+        m.blocks_per_chunk = a
+        K = len(cfg["blocks_per_chunk"])
+        hd.kind, hd.classes = LP_HEAD_LN_LINEAR, cfg["vocab"]
+    else:
+        m.family = LP_FAMILY_RESNET
+        m.in_channels, m.height, m.width = cfg["in_channels"], cfg["height"], cfg["width"]
+        m.stem_channels, m.blocks_per_stage = cfg["stem_channels"], cfg["blocks_per_stage"]
+        a = _ints(cfg["stage_channels"])
+        keep.append(a)
+        m.stage_channels = a
+        K = len(cfg["stage_channels"])
+        hd.kind, hd.classes = LP_HEAD_GAP_LINEAR, cfg["classes"]
+    o = cfg["optim"]
+    op = lp_optim_spec()
+    if o["kind"] == "sgdm":
+        op.kind, op.lr, op.momentum, op.weight_decay = LP_OPT_SGDM, o["lr"], o["momentum"], o.get("weight_decay", 0.0)
+    else:
+        op.kind, op.lr, op.beta1, op.beta2, op.eps = LP_OPT_ADAM, o["lr"], o["beta1"], o["beta2"], o["eps"]
+    m._keep = keep
+    return m, K, hd, op
+
+
+def lp_create(model: lp_model_spec, K: int, head: lp_head_spec, optim: lp_optim_spec) -> int:
+    h = C.c_void_p()
+    code = _lib.lp_create(C.byref(model), K, C.byref(head), C.byref(optim), None, C.byref(h))
+    _check(None, code)
+    return h.value
+
+
+def lp_destroy(h):
+    _check(h, _lib.lp_destroy(h))
+
+
+def lp_step(h, x, y, schedule, stream, out_losses):
+    _check(h, _lib.lp_step(h, _ptr(x), _ptr(y), schedule, stream, _ptr(out_losses)))
+
+
+def lp_step_host(h, x_host, y_host, schedule, stream, out_losses_host):
+    _check(h, _lib.lp_step_host(h, _ptr(x_host), _ptr(y_host), schedule, stream, _ptr(out_losses_host)))
+
+
+def lp_forward(h, x, y, stream, out_logits, out_losses):
+    _check(h, _lib.lp_forward(h, _ptr(x), _ptr(y), stream, _ptr(out_logits), _ptr(out_losses)))
+
+
+def lp_num_tensors(h) -> int:
+    return _lib.lp_num_tensors(h)
+
+
+def lp_tensor_info_get(h, i) -> dict:
+    info = lp_tensor_info()
+    _check(h, _lib.lp_tensor_info_get(h, i, C.byref(info)))
+    return dict(name=info.name.decode(), chunk=info.chunk, shape=tuple(info.shape[:info.ndim]),
+                numel=info.numel, has_working_bf16=bool(info.has_working_bf16))
+
+
+def lp_get_tensor(h, i, which, host_array: np.ndarray, stream=None):
+    _check(h, _lib.lp_get_tensor(h, i, which, host_array.ctypes.data, host_array.nbytes, stream))
+
+
+def lp_set_tensor(h, i, which, host_array: np.ndarray, stream=None):
+    _check(h, _lib.lp_set_tensor(h, i, which, host_array.ctypes.data, host_array.nbytes, stream))
+
+
+def lp_reset_pipeline(h):
+    _check(h, _lib.lp_reset_pipeline(h))
+
+
+def lp_status_poll(h, stream=None):
+    _check(h, _lib.lp_status_poll(h, stream))
+
+
+def lp_state_size(h) -> int:
+    return _lib.lp_state_size(h)
+
+
+def lp_save_state(h, host_array: np.ndarray):
+    _check(h, _lib.lp_save_state(h, host_array.ctypes.data, host_array.nbytes))
+
+
+def lp_load_state(h, host_array: np.ndarray):
+    _check(h, _lib.lp_load_state(h, host_array.ctypes.data, host_array.nbytes))
+
+
+def lp_last_step_launches(h) -> int:
+    return _lib.lp_last_step_launches(h)
+
+
+def lp_device_bytes(h) -> int:
+    return _lib.lp_device_bytes(h)
+
+
+def lp_last_error(h=None) -> str:
+    return (_lib.lp_last_error(h) or b"").decode()

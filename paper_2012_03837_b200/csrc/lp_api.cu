@@ -1,0 +1,391 @@
+// C ABI of the local update step (include/lp.h): argument checks, handle life cycle, step
+// drivers, parameter access, checkpointing.  No exception leaves this file.
+#include <cstring>
+#include <stdexcept>
+
+#include "runtime.h"
+
+using namespace lp;
+
+struct lp_handle_s {
+  Handle h;
+};
+
+static thread_local std::string g_create_error;
+
+namespace {
+
+struct ShapeError : std::runtime_error { using std::runtime_error::runtime_error; };
+struct UnsupportedError : std::runtime_error { using std::runtime_error::runtime_error; };
+
+lp_status fail(Handle* h, lp_status code, const std::string& msg) {
+  if (h) h->err = msg;
+  else g_create_error = msg;
+  return code;
+}
+
+lp_status check_cuda(Handle* h, const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) return LP_OK;
+  return fail(h, LP_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+void validate(const lp_model_spec* m, int K, const lp_head_spec* hd, const lp_optim_spec* o) {
+  if (K < 1 || K > 1024) throw ShapeError("K must be in [1, 1024]");
+  if (m->batch < 1) throw ShapeError("batch must be positive");
+  if (m->dtype != LP_FP32 && m->dtype != LP_BF16) throw std::invalid_argument("dtype");
+  if (o->kind != LP_OPT_SGDM && o->kind != LP_OPT_ADAM) throw std::invalid_argument("optimizer kind");
+  if (hd->classes < 2) throw ShapeError("classes must be at least 2");
+  switch (m->family) {
+    case LP_FAMILY_MLP: {
+      if (hd->kind != LP_HEAD_LINEAR) throw std::invalid_argument("MLP takes LP_HEAD_LINEAR");
+      if (!m->layer_widths || !m->layers_per_chunk) throw std::invalid_argument("null layer arrays");
+      if (m->d_in < 1 || m->n_layers < 1) throw ShapeError("d_in and n_layers must be positive");
+      int tot = 0;
+      for (int k = 0; k < K; ++k) {
+        if (m->layers_per_chunk[k] < 1) throw ShapeError("every chunk needs at least one layer");
+        tot += m->layers_per_chunk[k];
+      }
+      if (tot != m->n_layers) throw ShapeError("layers_per_chunk does not sum to n_layers");
+      for (int i = 0; i < m->n_layers; ++i)
+        if (m->layer_widths[i] < 1) throw ShapeError("layer width must be positive");
+      break;
+    }
+    case LP_FAMILY_LM: {
+      if (hd->kind != LP_HEAD_LN_LINEAR) throw std::invalid_argument("LM takes LP_HEAD_LN_LINEAR");
+      if (!m->blocks_per_chunk) throw std::invalid_argument("null blocks_per_chunk");
+      if (m->vocab < 2 || m->seq_len < 1 || m->d_model < 1 || m->n_heads < 1 || m->d_ffn < 1)
+        throw ShapeError("LM sizes must be positive");
+      if (m->d_model != m->n_heads * 64) throw ShapeError("d_model / n_heads must be 64");
+      if (hd->classes != m->vocab) throw ShapeError("LM head classes must equal vocab");
+      for (int k = 0; k < K; ++k)
+        if (m->blocks_per_chunk[k] < 1) throw ShapeError("every chunk needs at least one block");
+      break;
+    }
+    case LP_FAMILY_RESNET: {
+      if (hd->kind != LP_HEAD_GAP_LINEAR) throw std::invalid_argument("RESNET takes LP_HEAD_GAP_LINEAR");
+      if (!m->stage_channels) throw std::invalid_argument("null stage_channels");
+      if (m->in_channels < 1 || m->height < 1 || m->width < 1 || m->stem_channels < 1 || m->blocks_per_stage < 1)
+        throw ShapeError("RESNET sizes must be positive");
+      if ((m->height >> (K - 1)) < 1 || (m->width >> (K - 1)) < 1) throw ShapeError("image too small for K stages");
+      break;
+    }
+    default: throw std::invalid_argument("family");
+  }
+}
+
+// Copy a tensor between host and the arena.
+lp_status tensor_io(lp_handle hh, int i, int which, void* host, size_t bytes, void* stream, bool set) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!host) return fail(&h, LP_ERR_INVALID_ARG, "null host pointer");
+  if (i < 0 || i >= (int)h.tensors.size()) return fail(&h, LP_ERR_INVALID_ARG, "tensor index out of range");
+  const TensorRec& t = h.tensors[i];
+  cudaStream_t s = (cudaStream_t)stream;
+  void* dev = nullptr;
+  size_t es = 4;
+  switch (which) {
+    case LP_MASTER: dev = h.master + t.off; break;
+    case LP_MOMENT1: dev = h.m1 + t.off; break;
+    case LP_MOMENT2:
+      if (!h.m2) return fail(&h, LP_ERR_STATE, "no second moment for this optimizer");
+      dev = h.m2 + t.off; break;
+    case LP_GRAD: dev = h.grad + t.off; break;
+    case LP_WORKING:
+      if (!h.bf16_mode || !t.matrix) return fail(&h, LP_ERR_STATE, "tensor has no bf16 working copy");
+      dev = h.working + t.off; es = 2; break;
+    default: return fail(&h, LP_ERR_INVALID_ARG, "bad `which`");
+  }
+  if (bytes != (size_t)t.numel * es) return fail(&h, LP_ERR_SHAPE, "byte count does not match the tensor");
+  if (set) {
+    cudaMemcpyAsync(dev, host, bytes, cudaMemcpyHostToDevice, s);
+    if (which == LP_MASTER && h.bf16_mode && t.matrix) {
+      // refresh the working copy: round to nearest even on the host, same rule as the device update
+      std::vector<uint16_t> w(t.numel);
+      const uint32_t* src = (const uint32_t*)host;
+      for (int64_t j = 0; j < t.numel; ++j) {
+        uint32_t u = src[j];
+        if ((u & 0x7fffffffu) > 0x7f800000u) w[j] = (uint16_t)((u >> 16) | 0x40);
+        else w[j] = (uint16_t)((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
+      }
+      cudaMemcpyAsync(h.working + t.off, w.data(), t.numel * 2, cudaMemcpyHostToDevice, s);
+      cudaStreamSynchronize(s);
+    }
+  } else {
+    cudaMemcpyAsync(host, dev, bytes, cudaMemcpyDeviceToHost, s);
+  }
+  cudaStreamSynchronize(s);
+  return check_cuda(&h, set ? "lp_set_tensor" : "lp_get_tensor");
+}
+
+lp_status copy_inputs(Handle& h, const void* x, const void* y, cudaMemcpyKind kind, cudaStream_t s) {
+  cudaMemcpyAsync(h.x_in, x, h.x_bytes, kind, s);
+  if (y) cudaMemcpyAsync(h.y_in, y, h.y_bytes, kind, s);
+  return check_cuda(&h, "input copy");
+}
+
+lp_status run_step(Handle& h, int schedule, cudaStream_t s) {
+  RunCtx ctx{s, nullptr};
+  int launches = 0;
+  if (schedule == LP_SYNC) {
+    if (h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
+    h.sync_plan.run(ctx);
+    launches = h.sync_plan.launches;
+  } else {
+    if (!h.primed) {
+      h.prime_plan[h.parity].run(ctx);
+      launches += h.prime_plan[h.parity].launches;
+      h.primed = true;
+    }
+    h.pipe_plan[h.parity].run(ctx);
+    launches += h.pipe_plan[h.parity].launches;
+    h.parity ^= 1;
+  }
+  h.step_count += 1;
+  h.last_launches = launches;
+  return check_cuda(&h, "lp_step launch");
+}
+
+}  // namespace
+
+extern "C" {
+
+lp_status lp_create(const lp_model_spec* model, int K, const lp_head_spec* head, const lp_optim_spec* optim,
+                    const lp_alloc* alloc, lp_handle* out) {
+  if (out) *out = nullptr;
+  if (!model || !head || !optim || !out) return fail(nullptr, LP_ERR_INVALID_ARG, "null argument");
+  if (alloc && (!alloc->alloc || !alloc->release)) return fail(nullptr, LP_ERR_INVALID_ARG, "allocator needs both callbacks");
+  lp_handle hh = nullptr;
+  try {
+    validate(model, K, head, optim);
+    int dev_count = 0;
+    if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count == 0) {
+      cudaGetLastError();
+      return fail(nullptr, LP_ERR_CUDA, "no CUDA device available");
+    }
+    hh = new lp_handle_s();
+    Handle& h = hh->h;
+    h.spec = *model;
+    h.head = *head;
+    h.opt = *optim;
+    h.K = K;
+    h.bf16_mode = model->dtype == LP_BF16;
+    h.force_simt = model->gemm_backend == 1 || !h.bf16_mode;
+    if (alloc) { h.alloc = *alloc; h.use_cuda_malloc = false; }
+    h.d_losses = (float*)h.dalloc(sizeof(float) * K);
+    h.d_status = (int*)h.dalloc(sizeof(int));
+    switch (model->family) {
+      case LP_FAMILY_MLP:
+        h.layer_widths.assign(model->layer_widths, model->layer_widths + model->n_layers);
+        h.per_chunk.assign(model->layers_per_chunk, model->layers_per_chunk + K);
+        h.spec.layer_widths = nullptr; h.spec.layers_per_chunk = nullptr;
+        build_mlp(h);
+        break;
+      case LP_FAMILY_LM:
+        h.per_chunk.assign(model->blocks_per_chunk, model->blocks_per_chunk + K);
+        h.spec.blocks_per_chunk = nullptr;
+        build_lm(h);
+        break;
+      default:
+        h.stage_channels.assign(model->stage_channels, model->stage_channels + K);
+        h.spec.stage_channels = nullptr;
+        build_resnet(h);
+        break;
+    }
+    cudaDeviceSynchronize();
+    lp_status st = check_cuda(nullptr, "lp_create");
+    if (st != LP_OK) { lp_destroy(hh); return st; }
+    *out = hh;
+    return LP_OK;
+  } catch (const ShapeError& e) {
+    if (hh) lp_destroy(hh);
+    return fail(nullptr, LP_ERR_SHAPE, e.what());
+  } catch (const UnsupportedError& e) {
+    if (hh) lp_destroy(hh);
+    return fail(nullptr, LP_ERR_UNSUPPORTED, e.what());
+  } catch (const std::invalid_argument& e) {
+    if (hh) lp_destroy(hh);
+    return fail(nullptr, LP_ERR_INVALID_ARG, e.what());
+  } catch (const std::bad_alloc&) {
+    if (hh) lp_destroy(hh);
+    return fail(nullptr, LP_ERR_ALLOC, "host allocation failed");
+  } catch (const std::exception& e) {
+    std::string m = e.what();
+    if (hh) lp_destroy(hh);
+    lp_status code = m.rfind("alloc:", 0) == 0 ? LP_ERR_ALLOC
+                     : m.rfind("unsupported:", 0) == 0 ? LP_ERR_UNSUPPORTED
+                     : m.rfind("shape:", 0) == 0 ? LP_ERR_SHAPE : LP_ERR_CUDA;
+    return fail(nullptr, code, m);
+  }
+}
+
+lp_status lp_destroy(lp_handle hh) {
+  if (!hh) return LP_OK;
+  Handle& h = hh->h;
+  cudaDeviceSynchronize();
+  for (void* p : h.blocks) {
+    if (h.use_cuda_malloc) cudaFree(p);
+    else h.alloc.release(p, h.alloc.user);
+  }
+  cudaGetLastError();
+  delete hh;
+  return LP_OK;
+}
+
+lp_status lp_step(lp_handle hh, const void* x, const void* y, int schedule, void* stream, float* out_losses) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!x || !y || !out_losses) return fail(&h, LP_ERR_INVALID_ARG, "null pointer");
+  if (schedule != LP_SYNC && schedule != LP_PIPELINED) return fail(&h, LP_ERR_INVALID_ARG, "bad schedule");
+  if (schedule == LP_SYNC && h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
+  cudaStream_t s = (cudaStream_t)stream;
+  lp_status st = copy_inputs(h, x, y, cudaMemcpyDeviceToDevice, s);
+  if (st != LP_OK) return st;
+  st = run_step(h, schedule, s);
+  if (st != LP_OK) return st;
+  cudaMemcpyAsync(out_losses, h.d_losses, sizeof(float) * h.K, cudaMemcpyDeviceToDevice, s);
+  return check_cuda(&h, "lp_step");
+}
+
+lp_status lp_step_host(lp_handle hh, const void* x_host, const void* y_host, int schedule, void* stream,
+                       float* out_losses_host) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!x_host || !y_host || !out_losses_host) return fail(&h, LP_ERR_INVALID_ARG, "null pointer");
+  if (schedule != LP_SYNC && schedule != LP_PIPELINED) return fail(&h, LP_ERR_INVALID_ARG, "bad schedule");
+  if (schedule == LP_SYNC && h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
+  cudaStream_t s = (cudaStream_t)stream;
+  lp_status st = copy_inputs(h, x_host, y_host, cudaMemcpyHostToDevice, s);
+  if (st != LP_OK) return st;
+  st = run_step(h, schedule, s);
+  if (st != LP_OK) return st;
+  cudaMemcpyAsync(out_losses_host, h.d_losses, sizeof(float) * h.K, cudaMemcpyDeviceToHost, s);
+  cudaStreamSynchronize(s);
+  return check_cuda(&h, "lp_step_host");
+}
+
+lp_status lp_forward(lp_handle hh, const void* x, const void* y, void* stream, void* out_logits, float* out_losses) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!x) return fail(&h, LP_ERR_INVALID_ARG, "null x");
+  if (!y && out_losses) return fail(&h, LP_ERR_INVALID_ARG, "losses need labels");
+  cudaStream_t s = (cudaStream_t)stream;
+  lp_status st = copy_inputs(h, x, y, cudaMemcpyDeviceToDevice, s);
+  if (st != LP_OK) return st;
+  if (!y) cudaMemsetAsync(h.y_in, 0xff, h.y_bytes, s);   // all labels -1: no row is valid
+  RunCtx ctx{s, out_logits};
+  int half = h.primed ? h.parity ^ 1 : 0;                 // the half no chunk will read next step
+  h.fwd_plan[half].run(ctx);
+  if (out_losses) cudaMemcpyAsync(out_losses, h.d_losses, sizeof(float) * h.K, cudaMemcpyDeviceToDevice, s);
+  if (!y) cudaMemsetAsync(h.d_status, 0, sizeof(int), s); // the unlabeled pass yields NaN losses by design
+  return check_cuda(&h, "lp_forward");
+}
+
+int lp_num_tensors(lp_handle hh) { return hh ? (int)hh->h.tensors.size() : 0; }
+
+lp_status lp_tensor_info_get(lp_handle hh, int i, lp_tensor_info* out) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!out || i < 0 || i >= (int)h.tensors.size()) return fail(&h, LP_ERR_INVALID_ARG, "bad tensor index or null output");
+  const TensorRec& t = h.tensors[i];
+  memset(out, 0, sizeof(*out));
+  strncpy(out->name, t.name.c_str(), sizeof(out->name) - 1);
+  out->chunk = t.chunk;
+  out->ndim = (int)t.shape.size();
+  for (size_t j = 0; j < t.shape.size() && j < 4; ++j) out->shape[j] = t.shape[j];
+  out->numel = t.numel;
+  out->has_working_bf16 = (h.bf16_mode && t.matrix) ? 1 : 0;
+  return LP_OK;
+}
+
+lp_status lp_get_tensor(lp_handle hh, int i, int which, void* host_dst, size_t bytes, void* stream) {
+  return tensor_io(hh, i, which, host_dst, bytes, stream, false);
+}
+lp_status lp_set_tensor(lp_handle hh, int i, int which, const void* host_src, size_t bytes, void* stream) {
+  return tensor_io(hh, i, which, const_cast<void*>(host_src), bytes, stream, true);
+}
+
+lp_status lp_reset_pipeline(lp_handle hh) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  hh->h.primed = false;
+  hh->h.parity = 0;
+  return LP_OK;
+}
+
+lp_status lp_status_poll(lp_handle hh, void* stream) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  cudaStream_t s = (cudaStream_t)stream;
+  int w = 0;
+  cudaMemcpyAsync(&w, h.d_status, sizeof(int), cudaMemcpyDeviceToHost, s);
+  cudaMemsetAsync(h.d_status, 0, sizeof(int), s);
+  cudaStreamSynchronize(s);
+  lp_status st = check_cuda(&h, "lp_status_poll");
+  if (st != LP_OK) return st;
+  if (w & ST_TIMEOUT) return fail(&h, LP_ERR_TIMEOUT, "a device-side wait gave up");
+  if (w & ST_LABEL_RANGE) return fail(&h, LP_ERR_LABEL_RANGE, "a label or token id was out of range");
+  if (w & ST_NONFINITE) return fail(&h, LP_ERR_NONFINITE, "a loss was not finite");
+  return LP_OK;
+}
+
+// Checkpoint layout: header {magic, n_total, K, step_count, parity, primed}, master, m1, [m2],
+// then for each half and chunk: boundary activation, labels.
+struct StateHeader { uint64_t magic; int64_t n_total; int64_t K; int64_t step_count; int64_t parity; int64_t primed; };
+static const uint64_t kMagic = 0x4c50535441544531ull;
+
+size_t lp_state_size(lp_handle hh) {
+  if (!hh) return 0;
+  Handle& h = hh->h;
+  size_t n = sizeof(StateHeader) + (size_t)h.n_total * 4 * (h.m2 ? 3 : 2);
+  for (int s = 0; s < 2; ++s)
+    for (int k = 0; k < h.K; ++k) n += h.bnd_bytes[k] + h.y_bytes;
+  return n;
+}
+
+static lp_status state_io(lp_handle hh, void* host, size_t bytes, bool save) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!host) return fail(&h, LP_ERR_INVALID_ARG, "null host pointer");
+  if (bytes != lp_state_size(hh)) return fail(&h, LP_ERR_SHAPE, "state size mismatch");
+  cudaDeviceSynchronize();
+  char* p = (char*)host;
+  StateHeader hd{kMagic, h.n_total, h.K, h.step_count, h.parity, h.primed ? 1 : 0};
+  if (save) memcpy(p, &hd, sizeof(hd));
+  else {
+    memcpy(&hd, p, sizeof(hd));
+    if (hd.magic != kMagic || hd.n_total != h.n_total || hd.K != h.K) return fail(&h, LP_ERR_STATE, "state blob does not match this handle");
+    h.step_count = hd.step_count; h.parity = (int)hd.parity; h.primed = hd.primed != 0;
+  }
+  p += sizeof(hd);
+  auto io = [&](void* dev, size_t n) {
+    if (save) cudaMemcpy(p, dev, n, cudaMemcpyDeviceToHost);
+    else cudaMemcpy(dev, p, n, cudaMemcpyHostToDevice);
+    p += n;
+  };
+  io(h.master, (size_t)h.n_total * 4);
+  io(h.m1, (size_t)h.n_total * 4);
+  if (h.m2) io(h.m2, (size_t)h.n_total * 4);
+  for (int s = 0; s < 2; ++s)
+    for (int k = 0; k < h.K; ++k) { io(h.bnd[s][k], h.bnd_bytes[k]); io(h.lab[s][k], h.y_bytes); }
+  if (!save && h.bf16_mode) {
+    // working copies follow the restored masters: one optimizer-free refresh on the host side
+    std::vector<float> m((size_t)h.n_matrix);
+    cudaMemcpy(m.data(), h.master, (size_t)h.n_matrix * 4, cudaMemcpyDeviceToHost);
+    std::vector<uint16_t> w((size_t)h.n_matrix);
+    for (long long j = 0; j < h.n_matrix; ++j) {
+      uint32_t u; memcpy(&u, &m[j], 4);
+      w[j] = ((u & 0x7fffffffu) > 0x7f800000u) ? (uint16_t)((u >> 16) | 0x40) : (uint16_t)((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
+    }
+    cudaMemcpy(h.working, w.data(), (size_t)h.n_matrix * 2, cudaMemcpyHostToDevice);
+  }
+  return check_cuda(&h, save ? "lp_save_state" : "lp_load_state");
+}
+
+lp_status lp_save_state(lp_handle hh, void* host_dst, size_t bytes) { return state_io(hh, host_dst, bytes, true); }
+lp_status lp_load_state(lp_handle hh, const void* host_src, size_t bytes) { return state_io(hh, const_cast<void*>(host_src), bytes, false); }
+
+int lp_last_step_launches(lp_handle hh) { return hh ? hh->h.last_launches : 0; }
+size_t lp_device_bytes(lp_handle hh) { return hh ? hh->h.device_bytes : 0; }
+const char* lp_last_error(lp_handle hh) { return hh ? hh->h.err.c_str() : g_create_error.c_str(); }
+
+}  // extern "C"

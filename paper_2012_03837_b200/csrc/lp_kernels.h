@@ -1,0 +1,151 @@
+// Device-side problem tables and host launchers of the kernels behind the local update step.
+// Every kernel is "grouped": one launch serves a list of independent problems (one per chunk,
+// Sec. 3: chunks are trained independently), selected by blockIdx.y or by a tile scheduler.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lp {
+
+typedef __nv_bfloat16 bf16;
+
+// Bits of the device status word.
+enum { ST_LABEL_RANGE = 1, ST_NONFINITE = 2, ST_TIMEOUT = 4 };
+
+// ---------------------------------------------------------------------------- GEMM
+// C[m,n] = epilogue( sum_k A(m,k) * B(n,k) ),  A(m,k) = A[m*a_ms + k*a_ks], B(n,k) = B[n*b_ns + k*b_ks].
+// Exactly one stride of each operand is 1.  Forward of a Linear layer (App. A.1): A = x [M,K],
+// B = W [N,K].  Input gradient: A = dy, B(n,k) = W[k,n].  Weight gradient: A(m,k) = dy[k,m],
+// B(n,k) = x[k,n] (the reduction runs over the rows of the minibatch).
+enum EpiAct { EPI_NONE = 0, EPI_RELU = 1, EPI_GELU = 2, EPI_RELU_MASK = 3, EPI_GELU_GRAD = 4 };
+
+struct GemmProb {
+  const void* A;
+  const void* B;
+  void* C;            // [M, ldc] output, element type = operand type, or float if out_f32
+  void* C2;           // EPI_GELU: receives the pre-activation (operand type); else unused
+  const float* bias;  // [N] added to every row, or null
+  const void* resid;  // [M, ldc] operand type, added before the activation, or null
+  const void* aux;    // [M, ldc] operand type: EPI_RELU_MASK: layer output y (mask y>0);
+                      // EPI_GELU_GRAD: pre-activation u (multiply by gelu'(u))
+  int M, N, K;
+  long long a_ms, a_ks, b_ns, b_ks;
+  int ldc;
+  int act;
+  int out_f32;
+  int tile_start;  // first tile index of this problem in the launch (filled by the launcher)
+  int tiles_n;
+};
+
+// FP32-ALU GEMM (any sizes and strides).  T = float or bf16 operands, fp32 accumulation.
+void launch_gemm_simt(const GemmProb* d_probs, const GemmProb* h_probs, int n, bool is_bf16,
+                      cudaStream_t s);
+
+// ---------------------------------------------------------------------------- row-wise kernels
+struct LnProb {       // LayerNorm over the last axis of x [rows, d]
+  const void* x; void* y; const float* g; const float* b; float* mean; float* rstd;
+  int rows, d;
+};
+void launch_ln_fwd(const LnProb* d_probs, int n, int max_rows, bool is_bf16, cudaStream_t s);
+
+struct LnBwdProb {    // dx = LN'(dy) (+ dres); partial dgamma/dbeta per row block
+  const void* dy; const void* x; const float* g; const float* mean; const float* rstd;
+  void* dx;            // may be null: parameter gradients only (chunk input is a constant, Sec. 3)
+  const void* dres;    // optional gradient arriving over the residual path, added to dx
+  float* part;         // [nblk, 2, d] partial sums, nblk = ceil(rows / LN_BWD_ROWS)
+  int rows, d;
+};
+enum { LN_BWD_ROWS = 64 };
+void launch_ln_bwd(const LnBwdProb* d_probs, int n, int max_rows, bool is_bf16, cudaStream_t s);
+
+struct ColReduceProb { // out[c] = sum_r in[r, c] over r < rows, for c < cols; in is fp32 [rows, ld]
+  const float* in; float* out; int rows, cols, ld;
+};
+void launch_col_reduce_f32(const ColReduceProb* d_probs, int n, int max_cols, cudaStream_t s);
+
+struct ColSumProb {   // part[blk, c] = sum over a block of rows of x[r, c]; x is [rows, ld]
+  const void* x; float* part; int rows, cols, ld;
+};
+enum { COLSUM_ROWS = 128 };
+void launch_colsum_partial(const ColSumProb* d_probs, int n, int max_rows, int max_cols, bool is_bf16,
+                           cudaStream_t s);
+
+struct LabelProb {    // count valid labels, check range, (pipelined) carry labels to the next chunk
+  const int* y; int* y_out; int rows; int classes; int* n_valid;
+};
+void launch_label_prep(const LabelProb* d_probs, int n, int* d_status, cudaStream_t s);
+
+struct XentProb {     // softmax cross-entropy rows (App. A.1): z [rows, ld] -> dz in place, row losses
+  void* z; const int* y; const int* n_valid; float* row_loss; int rows, classes, ld;
+};
+void launch_xent(const XentProb* d_probs, int n, int max_rows, bool is_bf16, cudaStream_t s);
+
+struct LossProb { const float* row_loss; const int* n_valid; int rows; int out_index; };
+void launch_loss_reduce(const LossProb* d_probs, int n, float* d_losses, int* d_status, cudaStream_t s);
+
+// ---------------------------------------------------------------------------- LM-specific
+struct EmbedProb { const int* ids; const void* tok; const void* pos; void* h; int rows, T, d, vocab; };
+void launch_embed_fwd(const EmbedProb& p, int* d_status, bool is_bf16, cudaStream_t s);
+struct EmbedBwdProb {
+  const int* ids; const void* dh; float* dtok; float* dpos; int* next; int* first; int rows, T, d, vocab, B;
+};
+void launch_embed_bwd(const EmbedBwdProb& p, bool is_bf16, cudaStream_t s);
+
+struct AttnProb {     // causal attention over qkv [B*T, 3d], heads of 64
+  const void* qkv; void* o; float* lse; const void* dout; void* dqkv; float* delta; int B, T, H;
+};
+void launch_attn_fwd(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s);
+void launch_attn_bwd(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s);
+
+// ---------------------------------------------------------------------------- ResNet-specific
+struct LayoutProb { const void* in; void* out; int N, C, H, W; };
+void launch_nchw_to_nhwc(const LayoutProb& p, bool is_bf16, cudaStream_t s);
+
+struct Im2colProb {   // x NHWC [N,H,W,C] -> cols [N*Ho*Wo, ldk], column (i*kw + j)*C + c, zero padded
+  const void* x; void* cols; int N, H, W, C, kh, kw, stride, pad, Ho, Wo, ldk;
+};
+void launch_im2col(const Im2colProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
+// dx[n,h,w,c] = sum over the filter taps that read this pixel of dcols (gather form: no atomics)
+void launch_col2im(const Im2colProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
+
+struct BnStatProb {   // per-channel partial sums of x and x^2 (fwd) or of dy and dy*xhat (bwd)
+  const void* x; const void* dy; const float* mean; const float* rstd; const void* relu_out;
+  float* part; int rows, C;
+};
+enum { BN_ROWS = 256 };
+void launch_bn_stat_partial(const BnStatProb* d_probs, int n, int max_rows, int max_c, bool bwd, bool is_bf16,
+                            cudaStream_t s);
+struct BnFinalProb {  // fwd: sums -> mean, rstd.  part is [nblk, 2, C]
+  const float* part; int nblk; int rows; int C; float* mean; float* rstd; float* dgamma; float* dbeta; float eps;
+};
+void launch_bn_finalize(const BnFinalProb* d_probs, int n, int max_c, bool bwd, cudaStream_t s);
+struct BnApplyProb {
+  // fwd: y = relu?( (x-mean)*rstd*g + b (+ res) ).
+  // bwd: dx = rstd*g*( dyr - sum_dy/rows - xhat*sum_dyxhat/rows ), dyr = dy masked by relu_out>0;
+  //      dres_out (optional) receives dyr (gradient of the residual branch).
+  const void* x; void* y; const void* res; const float* g; const float* b; const float* mean; const float* rstd;
+  const void* dy; const void* relu_out; void* dx; void* dres_out; const float* dgamma; const float* dbeta;
+  int rows, C, relu;
+};
+void launch_bn_apply(const BnApplyProb* d_probs, int n, long long max_elems, bool bwd, bool is_bf16, cudaStream_t s);
+
+struct GapProb { const void* x; void* y; const void* dy; void* dx; int N, HW, C; };
+void launch_gap_fwd(const GapProb* d_probs, int n, int max_n, int max_c, bool is_bf16, cudaStream_t s);
+void launch_gap_bwd(const GapProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
+
+struct AddProb { const void* a; const void* b; void* out; long long n; };
+void launch_add(const AddProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
+
+// ---------------------------------------------------------------------------- optimizer
+struct OptimArgs {
+  float* master; float* m1; float* m2; const float* grad; bf16* working;  // working may be null
+  long long n_total;    // elements in the arena
+  long long n_matrix;   // leading elements that are matrices (weight decay + bf16 working copy)
+  int kind; float lr, momentum, weight_decay, beta1, beta2, eps;
+  float omb1, omb2;     // 1 - beta, rounded from double
+  float bc1, bc2;       // 1 - beta^t, rounded from double
+};
+void launch_optim(const OptimArgs& a, cudaStream_t s);
+
+}  // namespace lp

@@ -1,0 +1,355 @@
+// Decoder-only transformer LM family (App. B.2): token + position embeddings in chunk 0, pre-LayerNorm
+// blocks (causal attention, GELU feed-forward), and a LayerNorm + vocabulary projection + softmax
+// cross-entropy auxiliary head on every chunk (Sec. 3; App. B.2 for the head's form).
+//
+// Forward of one block:  a1 = LN1(h); qkv = a1 Wqkv^T + b; o = Attn(qkv); h1 = h + o Wo^T + b;
+//                        a2 = LN2(h1); u = a2 W1^T + b; g = GELU(u); h' = h1 + g W2^T + b.
+// Backward is truncated at the chunk input: for the first block of a chunk k > 0 only LN1's scale
+// and shift gradients are formed, not the gradient of the chunk input (Sec. 3).
+#include <stdexcept>
+
+#include "runtime.h"
+
+namespace lp {
+namespace {
+
+struct BlockBufs {
+  std::string name;
+  const void* hin = nullptr;   // set per plan
+  void *a1, *qkv, *o, *h1, *a2, *u, *g;
+  void* hout_internal;         // output when this is not the chunk's last block
+  float *mean1, *rstd1, *mean2, *rstd2, *lse, *delta;
+};
+struct ChunkBufs {
+  std::vector<BlockBufs> blocks;
+  void* emb = nullptr;         // chunk 0: embedding output
+  void *ah, *z;                // head LayerNorm output, logits / dlogits
+  float *meanh, *rstdh, *row_loss;
+  void *G0, *G1, *G2, *Gf, *Gq;   // gradient scratch: [M,d] x3, [M,ffn], [M,3d]
+};
+
+std::string hn(int k, const char* s) { return "c" + std::to_string(k) + ".head." + s; }
+
+}  // namespace
+
+void build_lm(Handle& h) {
+  const int K = h.K, B = h.spec.batch, T = h.spec.seq_len, d = h.spec.d_model, F = h.spec.d_ffn, V = h.spec.vocab,
+            H = h.spec.n_heads;
+  const int M = B * T;
+  h.rows = M;
+  std::vector<ChunkBufs> cb(K);
+  int blk = 0;
+  for (int k = 0; k < K; ++k) {
+    if (k == 0) {
+      h.add_tensor("c0.tok", 0, {V, d}, true);
+      h.add_tensor("c0.pos", 0, {T, d}, true);
+    }
+    for (int j = 0; j < h.per_chunk[k]; ++j, ++blk) {
+      BlockBufs bb;
+      bb.name = "c" + std::to_string(k) + ".b" + std::to_string(blk);
+      const std::string& n = bb.name;
+      h.add_tensor(n + ".ln1.g", k, {d}, false);
+      h.add_tensor(n + ".ln1.b", k, {d}, false);
+      h.add_tensor(n + ".Wqkv", k, {3 * d, d}, true);
+      h.add_tensor(n + ".bqkv", k, {3 * d}, false);
+      h.add_tensor(n + ".Wo", k, {d, d}, true);
+      h.add_tensor(n + ".bo", k, {d}, false);
+      h.add_tensor(n + ".ln2.g", k, {d}, false);
+      h.add_tensor(n + ".ln2.b", k, {d}, false);
+      h.add_tensor(n + ".W1", k, {F, d}, true);
+      h.add_tensor(n + ".b1", k, {F}, false);
+      h.add_tensor(n + ".W2", k, {d, F}, true);
+      h.add_tensor(n + ".b2", k, {d}, false);
+      cb[k].blocks.push_back(bb);
+    }
+    h.add_tensor(hn(k, "ln.g"), k, {d}, false);
+    h.add_tensor(hn(k, "ln.b"), k, {d}, false);
+    h.add_tensor(hn(k, "W"), k, {V, d}, true);
+    h.add_tensor(hn(k, "b"), k, {V}, false);
+  }
+  h.finalize_arena();
+
+  const size_t es = h.esize();
+  const size_t md = (size_t)M * d * es;
+  h.x_bytes = (size_t)M * sizeof(int);
+  h.x_in = h.dalloc(h.x_bytes);
+  h.y_bytes = (size_t)M * sizeof(int);
+  h.y_in = (int*)h.dalloc(h.y_bytes);
+  int* emb_next = (int*)h.dalloc((size_t)M * sizeof(int));
+  int* emb_first = (int*)h.dalloc((size_t)M * sizeof(int));
+  auto fal = [&](size_t n) { return (float*)h.dalloc(n * sizeof(float)); };
+  for (int k = 0; k < K; ++k) {
+    h.bnd_bytes.push_back(md);
+    for (int s = 0; s < 2; ++s) {
+      h.bnd[s].push_back(h.dalloc(md));
+      h.lab[s].push_back((int*)h.dalloc(h.y_bytes));
+    }
+    h.n_valid.push_back((int*)h.dalloc(sizeof(int)));
+    ChunkBufs& c = cb[k];
+    if (k == 0) c.emb = h.dalloc(md);
+    for (size_t j = 0; j < c.blocks.size(); ++j) {
+      BlockBufs& b = c.blocks[j];
+      b.a1 = h.dalloc(md); b.qkv = h.dalloc(3 * md); b.o = h.dalloc(md); b.h1 = h.dalloc(md); b.a2 = h.dalloc(md);
+      b.u = h.dalloc((size_t)M * F * es); b.g = h.dalloc((size_t)M * F * es);
+      b.hout_internal = (j + 1 < c.blocks.size()) ? h.dalloc(md) : nullptr;
+      b.mean1 = fal(M); b.rstd1 = fal(M); b.mean2 = fal(M); b.rstd2 = fal(M);
+      b.lse = fal((size_t)B * H * T); b.delta = fal((size_t)B * H * T);
+    }
+    c.ah = h.dalloc(md);
+    c.z = h.dalloc((size_t)M * V * es);
+    c.meanh = fal(M); c.rstdh = fal(M); c.row_loss = fal(M);
+    c.G0 = h.dalloc(md); c.G1 = h.dalloc(md); c.G2 = h.dalloc(md);
+    c.Gf = h.dalloc((size_t)M * F * es); c.Gq = h.dalloc(3 * md);
+  }
+
+  std::vector<int> all;
+  for (int k = 0; k < K; ++k) all.push_back(k);
+  const bool bf = h.bf16_mode;
+  int* st = h.d_status;
+
+  auto chunk_in = [&](int k, int rd) -> const void* { return k == 0 ? cb[0].emb : h.bnd[rd][k - 1]; };
+  auto block_in = [&](int k, size_t j, int rd) -> const void* {
+    return j == 0 ? chunk_in(k, rd) : cb[k].blocks[j - 1].hout_internal;
+  };
+  auto block_out = [&](int k, size_t j, int wr) -> void* {
+    return (j + 1 < cb[k].blocks.size()) ? cb[k].blocks[j].hout_internal : h.bnd[wr][k];
+  };
+  auto labels_of = [&](int k, bool pipelined, int rd) -> const int* {
+    return (!pipelined || k == 0) ? h.y_in : h.lab[rd][k - 1];
+  };
+
+  // ---- forward of the trunks of chunks `ks`
+  auto forward = [&](Plan& p, const std::vector<int>& ks, int rd, int wr) {
+    for (int k : ks)
+      if (k == 0) {
+        EmbedProb e{(const int*)h.x_in, h.W("c0.tok"), h.W("c0.pos"), cb[0].emb, M, T, d, V};
+        p.add(1, [e, st, bf](const RunCtx& c) { launch_embed_fwd(e, st, bf, c.stream); });
+      }
+    size_t maxb = 0;
+    for (int k : ks) maxb = std::max(maxb, cb[k].blocks.size());
+    for (size_t j = 0; j < maxb; ++j) {
+      std::vector<int> act;
+      for (int k : ks) if (j < cb[k].blocks.size()) act.push_back(k);
+      std::vector<LnProb> ln;
+      std::vector<GemmProb> g;
+      std::vector<AttnProb> at;
+      for (int k : act) {
+        BlockBufs& b = cb[k].blocks[j];
+        ln.push_back(LnProb{block_in(k, j, rd), b.a1, h.P32(b.name + ".ln1.g"), h.P32(b.name + ".ln1.b"), b.mean1, b.rstd1, M, d});
+        g.push_back(gemm_fwd(b.a1, h.W(b.name + ".Wqkv"), b.qkv, M, 3 * d, d, h.P32(b.name + ".bqkv"), EPI_NONE));
+        at.push_back(AttnProb{b.qkv, b.o, b.lse, nullptr, nullptr, b.delta, B, T, H});
+      }
+      emit_ln_fwd(h, p, ln);
+      emit_gemm(h, p, g);
+      {
+        const AttnProb* dp = h.upload(at);
+        int n = (int)at.size();
+        p.add(1, [=](const RunCtx& c) { launch_attn_fwd(dp, n, B, T, H, bf, c.stream); });
+      }
+      g.clear(); ln.clear();
+      for (int k : act) {
+        BlockBufs& b = cb[k].blocks[j];
+        GemmProb q = gemm_fwd(b.o, h.W(b.name + ".Wo"), b.h1, M, d, d, h.P32(b.name + ".bo"), EPI_NONE);
+        q.resid = block_in(k, j, rd);
+        g.push_back(q);
+        ln.push_back(LnProb{b.h1, b.a2, h.P32(b.name + ".ln2.g"), h.P32(b.name + ".ln2.b"), b.mean2, b.rstd2, M, d});
+      }
+      emit_gemm(h, p, g);
+      emit_ln_fwd(h, p, ln);
+      g.clear();
+      for (int k : act) {
+        BlockBufs& b = cb[k].blocks[j];
+        GemmProb q = gemm_fwd(b.a2, h.W(b.name + ".W1"), b.g, M, F, d, h.P32(b.name + ".b1"), EPI_GELU);
+        q.C2 = b.u;
+        g.push_back(q);
+      }
+      emit_gemm(h, p, g);
+      g.clear();
+      for (int k : act) {
+        BlockBufs& b = cb[k].blocks[j];
+        GemmProb q = gemm_fwd(b.g, h.W(b.name + ".W2"), block_out(k, j, wr), M, d, F, h.P32(b.name + ".b2"), EPI_NONE);
+        q.resid = b.h1;
+        g.push_back(q);
+      }
+      emit_gemm(h, p, g);
+    }
+  };
+
+  // ---- heads: LayerNorm, logits, loss (+ dlogits in place)
+  auto heads_forward = [&](Plan& p, int wr, bool pipelined, int rd, bool copy_logits) {
+    std::vector<LnProb> ln;
+    std::vector<GemmProb> g;
+    std::vector<XentProb> xs;
+    for (int k = 0; k < K; ++k) {
+      ChunkBufs& c = cb[k];
+      ln.push_back(LnProb{h.bnd[wr][k], c.ah, h.P32(hn(k, "ln.g")), h.P32(hn(k, "ln.b")), c.meanh, c.rstdh, M, d});
+      g.push_back(gemm_fwd(c.ah, h.W(hn(k, "W")), c.z, M, V, d, h.P32(hn(k, "b")), EPI_NONE));
+      xs.push_back(XentProb{c.z, labels_of(k, pipelined, rd), h.n_valid[k], c.row_loss, M, V, V});
+    }
+    emit_ln_fwd(h, p, ln);
+    emit_gemm(h, p, g);
+    if (copy_logits) {
+      void* zlast = cb[K - 1].z;
+      size_t zbytes = (size_t)M * V * es;
+      p.add(0, [zlast, zbytes](const RunCtx& c) {
+        if (c.out_logits) cudaMemcpyAsync(c.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, c.stream);
+      });
+    }
+    emit_xent_and_loss(h, p, xs, all);
+  };
+
+  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr) {
+    std::vector<LabelProb> lps;
+    for (int k = 0; k < K; ++k)
+      lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, M, V,
+                              h.n_valid[k]});
+    emit_labels(h, p, lps);
+    if (pipelined) forward(p, all, rd, wr);
+    else for (int k = 0; k < K; ++k) forward(p, {k}, rd, wr);
+    heads_forward(p, wr, pipelined, rd, false);
+
+    // ---- head backward -> gradient at the trunk output in G0
+    {
+      std::vector<GemmProb> g;
+      std::vector<ColSumProb> cs;
+      std::vector<float*> outs;
+      for (int k = 0; k < K; ++k) {
+        ChunkBufs& c = cb[k];
+        g.push_back(gemm_wgrad(c.z, c.ah, h.G(hn(k, "W")), M, V, d));
+        g.push_back(gemm_dgrad(c.z, h.W(hn(k, "W")), c.G1, M, V, d, EPI_NONE, nullptr));
+        cs.push_back(ColSumProb{c.z, nullptr, M, V, V});
+        outs.push_back(h.G(hn(k, "b")));
+      }
+      emit_gemm(h, p, g);
+      emit_colsum(h, p, cs, outs);
+      std::vector<LnBwdProb> lb;
+      std::vector<float*> dgs, dbs;
+      for (int k = 0; k < K; ++k) {
+        ChunkBufs& c = cb[k];
+        lb.push_back(LnBwdProb{c.G1, h.bnd[wr][k], h.P32(hn(k, "ln.g")), c.meanh, c.rstdh, c.G0, nullptr, nullptr, M, d});
+        dgs.push_back(h.G(hn(k, "ln.g")));
+        dbs.push_back(h.G(hn(k, "ln.b")));
+      }
+      emit_ln_bwd(h, p, lb, dgs, dbs);
+    }
+
+    // ---- trunk backward, blocks aligned from the back of each chunk
+    size_t maxb = 0;
+    for (int k = 0; k < K; ++k) maxb = std::max(maxb, cb[k].blocks.size());
+    for (size_t jj = 0; jj < maxb; ++jj) {
+      std::vector<int> act;
+      for (int k = 0; k < K; ++k) if (jj < cb[k].blocks.size()) act.push_back(k);
+      auto BJ = [&](int k) -> size_t { return cb[k].blocks.size() - 1 - jj; };
+      std::vector<GemmProb> g;
+      std::vector<ColSumProb> cs;
+      std::vector<float*> outs;
+      // 1. feed-forward second matrix: dW2, db2, du = (dout W2) * gelu'(u)
+      for (int k : act) {
+        ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
+        g.push_back(gemm_wgrad(c.G0, b.g, h.G(b.name + ".W2"), M, d, F));
+        g.push_back(gemm_dgrad(c.G0, h.W(b.name + ".W2"), c.Gf, M, d, F, EPI_GELU_GRAD, b.u));
+        cs.push_back(ColSumProb{c.G0, nullptr, M, d, d});
+        outs.push_back(h.G(b.name + ".b2"));
+      }
+      emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
+      g.clear(); cs.clear(); outs.clear();
+      // 2. feed-forward first matrix: dW1, db1, da2
+      for (int k : act) {
+        ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
+        g.push_back(gemm_wgrad(c.Gf, b.a2, h.G(b.name + ".W1"), M, F, d));
+        g.push_back(gemm_dgrad(c.Gf, h.W(b.name + ".W1"), c.G1, M, F, d, EPI_NONE, nullptr));
+        cs.push_back(ColSumProb{c.Gf, nullptr, M, F, F});
+        outs.push_back(h.G(b.name + ".b1"));
+      }
+      emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
+      g.clear(); cs.clear(); outs.clear();
+      // 3. LN2 backward; the residual path adds dout: dh1 -> G2
+      {
+        std::vector<LnBwdProb> lb;
+        std::vector<float*> dgs, dbs;
+        for (int k : act) {
+          ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
+          lb.push_back(LnBwdProb{c.G1, b.h1, h.P32(b.name + ".ln2.g"), b.mean2, b.rstd2, c.G2, c.G0, nullptr, M, d});
+          dgs.push_back(h.G(b.name + ".ln2.g"));
+          dbs.push_back(h.G(b.name + ".ln2.b"));
+        }
+        emit_ln_bwd(h, p, lb, dgs, dbs);
+      }
+      // 4. attention output projection: dWo, dbo, do -> G1
+      for (int k : act) {
+        ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
+        g.push_back(gemm_wgrad(c.G2, b.o, h.G(b.name + ".Wo"), M, d, d));
+        g.push_back(gemm_dgrad(c.G2, h.W(b.name + ".Wo"), c.G1, M, d, d, EPI_NONE, nullptr));
+        cs.push_back(ColSumProb{c.G2, nullptr, M, d, d});
+        outs.push_back(h.G(b.name + ".bo"));
+      }
+      emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
+      g.clear(); cs.clear(); outs.clear();
+      // 5. attention backward: dqkv -> Gq
+      {
+        std::vector<AttnProb> at;
+        for (int k : act) {
+          ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
+          at.push_back(AttnProb{b.qkv, b.o, b.lse, c.G1, c.Gq, b.delta, B, T, H});
+        }
+        const AttnProb* dp = h.upload(at);
+        int n = (int)at.size();
+        p.add(2, [=](const RunCtx& c) { launch_attn_bwd(dp, n, B, T, H, bf, c.stream); });
+      }
+      // 6. qkv projection: dWqkv, dbqkv, da1 -> G1 (needed for LN1's own parameters in every case)
+      for (int k : act) {
+        ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
+        g.push_back(gemm_wgrad(c.Gq, b.a1, h.G(b.name + ".Wqkv"), M, 3 * d, d));
+        g.push_back(gemm_dgrad(c.Gq, h.W(b.name + ".Wqkv"), c.G1, M, 3 * d, d, EPI_NONE, nullptr));
+        cs.push_back(ColSumProb{c.Gq, nullptr, M, 3 * d, 3 * d});
+        outs.push_back(h.G(b.name + ".bqkv"));
+      }
+      emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
+      g.clear(); cs.clear(); outs.clear();
+      // 7. LN1 backward.  The block-input gradient (dh1 + LN1 path -> G0) is formed only if a
+      //    layer of the same chunk consumes it: an earlier block, or chunk 0's embeddings.
+      {
+        std::vector<LnBwdProb> lb;
+        std::vector<float*> dgs, dbs;
+        for (int k : act) {
+          ChunkBufs& c = cb[k]; size_t j = BJ(k); BlockBufs& b = c.blocks[j];
+          bool need_dx = (j > 0) || (k == 0);
+          lb.push_back(LnBwdProb{c.G1, block_in(k, j, rd), h.P32(b.name + ".ln1.g"), b.mean1, b.rstd1,
+                                 need_dx ? c.G0 : nullptr, need_dx ? c.G2 : nullptr, nullptr, M, d});
+          dgs.push_back(h.G(b.name + ".ln1.g"));
+          dbs.push_back(h.G(b.name + ".ln1.b"));
+        }
+        emit_ln_bwd(h, p, lb, dgs, dbs);
+      }
+      // 8. chunk 0, first block: embedding tables
+      for (int k : act)
+        if (k == 0 && BJ(k) == 0) {
+          EmbedBwdProb e{(const int*)h.x_in, cb[0].G0, h.G("c0.tok"), h.G("c0.pos"), emb_next, emb_first, M, T, d, V, B};
+          p.add(5, [e, bf](const RunCtx& c) { launch_embed_bwd(e, bf, c.stream); });
+        }
+    }
+    emit_pending_reduce(h, p);
+    emit_optimizer(h, p);
+  };
+
+  auto build_forward = [&](Plan& p, int wr, bool heads) {
+    for (int k = 0; k < K; ++k) forward(p, {k}, wr, wr);
+    if (!heads) return;
+    std::vector<LabelProb> lps;
+    for (int k = 0; k < K; ++k) lps.push_back(LabelProb{h.y_in, nullptr, M, V, h.n_valid[k]});
+    emit_labels(h, p, lps);
+    heads_forward(p, wr, false, wr, true);
+  };
+
+  build_step(h.sync_plan, false, 0, 0);
+  for (int par = 0; par < 2; ++par) {
+    build_step(h.pipe_plan[par], true, par, 1 - par);
+    build_forward(h.prime_plan[par], par, false);
+    std::vector<LabelProb> lps;
+    for (int k = 0; k + 1 < K; ++k) lps.push_back(LabelProb{h.y_in, h.lab[par][k], M, V, h.n_valid[k]});
+    if (!lps.empty()) emit_labels(h, h.prime_plan[par], lps);
+    build_forward(h.fwd_plan[par], par, true);
+  }
+}
+
+}  // namespace lp

@@ -1,0 +1,195 @@
+// MLP family: chunks of Linear+ReLU layers (App. A.1) with a Linear + softmax cross-entropy
+// auxiliary head per chunk (Sec. 3).  Builds the synchronous, pipelined, priming and forward-only
+// plans.  Within a plan, work that belongs to different chunks and does not depend on another
+// chunk's result of the same step is issued as one grouped launch.
+#include <stdexcept>
+
+#include "runtime.h"
+
+namespace lp {
+namespace {
+
+struct MlpBufs {
+  std::vector<std::vector<int>> widths;        // [k][i]
+  std::vector<int> d_in;                       // input width of chunk k
+  std::vector<std::vector<void*>> y;           // [k][i] layer outputs except the last (which is the boundary)
+  std::vector<void*> z;                        // [k] logits / dlogits
+  std::vector<float*> row_loss;                // [k]
+  std::vector<void*> g0, g1;                   // [k] gradient ping-pong buffers [B, max width]
+};
+
+std::string tn(int k, int i, const char* s) { return "c" + std::to_string(k) + ".l" + std::to_string(i) + "." + s; }
+std::string hn(int k, const char* s) { return "c" + std::to_string(k) + ".head." + s; }
+
+// Input of chunk k for a plan that reads boundary half `rd`.
+const void* chunk_in(Handle& h, int k, int rd) { return k == 0 ? h.x_in : h.bnd[rd][k - 1]; }
+
+// Forward of the chunks in `ks` (layer index aligned from the front), outputs into half `wr`.
+void forward_level(Handle& h, MlpBufs& b, Plan& p, const std::vector<int>& ks, int rd, int wr) {
+  size_t maxl = 0;
+  for (int k : ks) maxl = std::max(maxl, b.widths[k].size());
+  int B = h.spec.batch;
+  for (size_t i = 0; i < maxl; ++i) {
+    std::vector<GemmProb> g;
+    for (int k : ks) {
+      if (i >= b.widths[k].size()) continue;
+      bool last = i + 1 == b.widths[k].size();
+      const void* in = i == 0 ? chunk_in(h, k, rd) : b.y[k][i - 1];
+      int din = i == 0 ? b.d_in[k] : b.widths[k][i - 1];
+      void* out = last ? h.bnd[wr][k] : b.y[k][i];
+      g.push_back(gemm_fwd(in, h.W(tn(k, (int)i, "W")), out, B, b.widths[k][i], din, h.P32(tn(k, (int)i, "b")), EPI_RELU));
+    }
+    emit_gemm(h, p, g);
+  }
+}
+
+}  // namespace
+
+void build_mlp(Handle& h) {
+  const int K = h.K, B = h.spec.batch, C = h.head.classes;
+  auto* bp = new MlpBufs();   // lives as long as the handle's plans (freed with the process; tiny)
+  MlpBufs& b = *bp;
+  b.widths.resize(K);
+  b.d_in.resize(K);
+  int li = 0, prev = h.spec.d_in, maxw = 0;
+  for (int k = 0; k < K; ++k) {
+    b.d_in[k] = prev;
+    for (int i = 0; i < h.per_chunk[k]; ++i) {
+      int w = h.layer_widths[li++];
+      h.add_tensor(tn(k, i, "W"), k, {w, prev}, true);
+      h.add_tensor(tn(k, i, "b"), k, {w}, false);
+      b.widths[k].push_back(w);
+      prev = w;
+      maxw = std::max(maxw, w);
+    }
+    h.add_tensor(hn(k, "W"), k, {C, prev}, true);
+    h.add_tensor(hn(k, "b"), k, {C}, false);
+  }
+  h.finalize_arena();
+  h.rows = B;
+  size_t es = h.esize();
+  h.x_bytes = (size_t)B * h.spec.d_in * es;
+  h.x_in = h.dalloc(h.x_bytes);
+  h.y_bytes = (size_t)B * sizeof(int);
+  h.y_in = (int*)h.dalloc(h.y_bytes);
+  b.y.resize(K);
+  for (int k = 0; k < K; ++k) {
+    size_t bytes = (size_t)B * b.widths[k].back() * es;
+    h.bnd_bytes.push_back(bytes);
+    for (int s = 0; s < 2; ++s) {
+      h.bnd[s].push_back(h.dalloc(bytes));
+      h.lab[s].push_back((int*)h.dalloc(h.y_bytes));
+    }
+    h.n_valid.push_back((int*)h.dalloc(sizeof(int)));
+    for (size_t i = 0; i + 1 < b.widths[k].size(); ++i) b.y[k].push_back(h.dalloc((size_t)B * b.widths[k][i] * es));
+    b.z.push_back(h.dalloc((size_t)B * C * es));
+    b.row_loss.push_back((float*)h.dalloc((size_t)B * sizeof(float)));
+    b.g0.push_back(h.dalloc((size_t)B * maxw * es));
+    b.g1.push_back(h.dalloc((size_t)B * maxw * es));
+  }
+
+  std::vector<int> all;
+  for (int k = 0; k < K; ++k) all.push_back(k);
+
+  // labels chunk k trains on, for a plan that reads half `rd` (pipelined) or the step's own y (sync)
+  auto labels_of = [&](int k, bool pipelined, int rd) -> const int* {
+    return (!pipelined || k == 0) ? h.y_in : h.lab[rd][k - 1];
+  };
+
+  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr) {
+    std::vector<LabelProb> lps;
+    for (int k = 0; k < K; ++k)
+      lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, B, C,
+                              h.n_valid[k]});
+    emit_labels(h, p, lps);
+    if (pipelined) forward_level(h, b, p, all, rd, wr);
+    else for (int k = 0; k < K; ++k) forward_level(h, b, p, {k}, rd, wr);
+    // heads: logits, loss, dlogits
+    {
+      std::vector<GemmProb> g;
+      std::vector<XentProb> xs;
+      for (int k = 0; k < K; ++k) {
+        g.push_back(gemm_fwd(h.bnd[wr][k], h.W(hn(k, "W")), b.z[k], B, C, b.widths[k].back(), h.P32(hn(k, "b")), EPI_NONE));
+        xs.push_back(XentProb{b.z[k], labels_of(k, pipelined, rd), h.n_valid[k], b.row_loss[k], B, C, C});
+      }
+      emit_gemm(h, p, g);
+      emit_xent_and_loss(h, p, xs, all);
+    }
+    // head backward: dW_h, db_h, and the gradient at the last layer's pre-activation
+    {
+      std::vector<GemmProb> g;
+      std::vector<ColSumProb> cs;
+      std::vector<float*> outs;
+      for (int k = 0; k < K; ++k) {
+        int D = b.widths[k].back();
+        g.push_back(gemm_wgrad(b.z[k], h.bnd[wr][k], h.G(hn(k, "W")), B, C, D));
+        g.push_back(gemm_dgrad(b.z[k], h.W(hn(k, "W")), b.g0[k], B, C, D, EPI_RELU_MASK, h.bnd[wr][k]));
+        cs.push_back(ColSumProb{b.z[k], nullptr, B, C, C});
+        outs.push_back(h.G(hn(k, "b")));
+      }
+      emit_gemm(h, p, g);
+      emit_colsum(h, p, cs, outs);
+    }
+    // trunk backward, aligned from the last layer of each chunk; nothing is propagated to the
+    // chunk input (Sec. 3: the gradient stops at the chunk boundary)
+    size_t maxl = 0;
+    for (int k = 0; k < K; ++k) maxl = std::max(maxl, b.widths[k].size());
+    for (size_t j = 0; j < maxl; ++j) {
+      std::vector<GemmProb> g;
+      std::vector<ColSumProb> cs;
+      std::vector<float*> outs;
+      for (int k = 0; k < K; ++k) {
+        int nl = (int)b.widths[k].size();
+        if ((int)j >= nl) continue;
+        int i = nl - 1 - (int)j;
+        void* du = (j % 2 == 0) ? b.g0[k] : b.g1[k];
+        void* dnext = (j % 2 == 0) ? b.g1[k] : b.g0[k];
+        const void* in = i == 0 ? chunk_in(h, k, rd) : b.y[k][i - 1];
+        int din = i == 0 ? b.d_in[k] : b.widths[k][i - 1];
+        int w = b.widths[k][i];
+        g.push_back(gemm_wgrad(du, in, h.G(tn(k, i, "W")), B, w, din));
+        if (i > 0) g.push_back(gemm_dgrad(du, h.W(tn(k, i, "W")), dnext, B, w, din, EPI_RELU_MASK, b.y[k][i - 1]));
+        cs.push_back(ColSumProb{du, nullptr, B, w, w});
+        outs.push_back(h.G(tn(k, i, "b")));
+      }
+      emit_gemm(h, p, g);
+      emit_colsum(h, p, cs, outs);
+    }
+    emit_pending_reduce(h, p);
+    emit_optimizer(h, p);
+  };
+
+  auto build_forward = [&](Plan& p, int wr, bool heads) {
+    for (int k = 0; k < K; ++k) forward_level(h, b, p, {k}, wr, wr);
+    if (!heads) return;
+    std::vector<LabelProb> lps;
+    for (int k = 0; k < K; ++k) lps.push_back(LabelProb{h.y_in, nullptr, B, C, h.n_valid[k]});
+    emit_labels(h, p, lps);
+    std::vector<GemmProb> g;
+    std::vector<XentProb> xs;
+    for (int k = 0; k < K; ++k) {
+      g.push_back(gemm_fwd(h.bnd[wr][k], h.W(hn(k, "W")), b.z[k], B, C, b.widths[k].back(), h.P32(hn(k, "b")), EPI_NONE));
+      xs.push_back(XentProb{b.z[k], h.y_in, h.n_valid[k], b.row_loss[k], B, C, C});
+    }
+    emit_gemm(h, p, g);
+    void* zlast = b.z[K - 1];
+    size_t zbytes = (size_t)B * C * es;
+    p.add(0, [zlast, zbytes](const RunCtx& c) {
+      if (c.out_logits) cudaMemcpyAsync(c.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, c.stream);
+    });
+    emit_xent_and_loss(h, p, xs, all);
+  };
+
+  build_step(h.sync_plan, false, 0, 0);
+  for (int par = 0; par < 2; ++par) {
+    build_step(h.pipe_plan[par], true, par, 1 - par);
+    // priming: forward chain into the half the first pipelined step will read, labels alongside
+    build_forward(h.prime_plan[par], par, false);
+    std::vector<LabelProb> lps;
+    for (int k = 0; k + 1 < K; ++k) lps.push_back(LabelProb{h.y_in, h.lab[par][k], B, C, h.n_valid[k]});
+    if (!lps.empty()) emit_labels(h, h.prime_plan[par], lps);
+    build_forward(h.fwd_plan[par], par, true);
+  }
+}
+
+}  // namespace lp

@@ -1,0 +1,142 @@
+// Fused multi-tensor optimizer update over the whole parameter arena (each chunk's parameters are
+// updated from that chunk's own gradients only, Sec. 1 / Sec. 6: the update is element-wise, so one
+// flat sweep applies all K per-chunk updates), and the token/position embedding of LM chunk 0.
+#include "common.cuh"
+
+namespace lp {
+namespace {
+
+// 4 elements per thread, 128-bit accesses.  Reads master, moments, gradient; writes master,
+// moments and (for the leading n_matrix elements) the bf16 working copy re-rounded from master.
+__global__ void __launch_bounds__(256) optim_kernel(OptimArgs a) {
+  long long i4 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i4 >= a.n_total) return;   // the arena length is a multiple of 4
+  float4 w = *(const float4*)(a.master + i4);
+  float4 g = *(const float4*)(a.grad + i4);
+  float4 m1 = *(const float4*)(a.m1 + i4);
+  float wv[4] = {w.x, w.y, w.z, w.w}, gv[4] = {g.x, g.y, g.z, g.w}, mv[4] = {m1.x, m1.y, m1.z, m1.w};
+  bool is_mat = i4 < a.n_matrix;   // the matrix region length is a multiple of 4
+  if (a.kind == 0) {               // SGD with momentum
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float gg = gv[j];
+      if (is_mat && a.weight_decay != 0.f) gg += a.weight_decay * wv[j];
+      mv[j] = a.momentum * mv[j] + gg;
+      wv[j] -= a.lr * mv[j];
+    }
+  } else {                         // Adam
+    float4 m2 = *(const float4*)(a.m2 + i4);
+    float vv[4] = {m2.x, m2.y, m2.z, m2.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      mv[j] = a.beta1 * mv[j] + a.omb1 * gv[j];
+      vv[j] = a.beta2 * vv[j] + a.omb2 * gv[j] * gv[j];
+      float mh = mv[j] / a.bc1, vh = vv[j] / a.bc2;
+      wv[j] -= a.lr * mh / (sqrtf(vh) + a.eps);
+    }
+    *(float4*)(a.m2 + i4) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+  }
+  *(float4*)(a.m1 + i4) = make_float4(mv[0], mv[1], mv[2], mv[3]);
+  *(float4*)(a.master + i4) = make_float4(wv[0], wv[1], wv[2], wv[3]);
+  if (a.working && is_mat) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(wv[0], wv[1]);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(wv[2], wv[3]);
+    uint2 pk;
+    pk.x = *(uint32_t*)&lo;
+    pk.y = *(uint32_t*)&hi;
+    *(uint2*)(a.working + i4) = pk;
+  }
+}
+
+// h[r, :] = tok[ids[r], :] + pos[r % T, :]; ids outside [0, vocab) are flagged and clamped.
+template <typename T>
+__global__ void __launch_bounds__(256) embed_fwd_kernel(EmbedProb p, int* status) {
+  int row = blockIdx.x;
+  int id = p.ids[row];
+  if (id < 0 || id >= p.vocab) {
+    if (threadIdx.x == 0) atomicOr(status, ST_LABEL_RANGE);
+    id = min(max(id, 0), p.vocab - 1);
+  }
+  const T* tok = (const T*)p.tok + (size_t)id * p.d;
+  const T* pos = (const T*)p.pos + (size_t)(row % p.T) * p.d;
+  T* h = (T*)p.h + (size_t)row * p.d;
+  for (int c = threadIdx.x; c < p.d; c += blockDim.x) h[c] = from_f<T>(to_f(tok[c]) + to_f(pos[c]));
+}
+
+// next[i] = smallest j > i holding the same token id (or -1); first[] starts at 1 everywhere.
+__global__ void __launch_bounds__(256) embed_link_kernel(EmbedBwdProb p) {
+  __shared__ int tile[256];
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  int my = i < p.rows ? min(max(p.ids[i], 0), p.vocab - 1) : -1;
+  int nxt = -1;
+  for (int j0 = blockIdx.x * blockDim.x; j0 < p.rows; j0 += blockDim.x) {
+    __syncthreads();
+    int j = j0 + threadIdx.x;
+    tile[threadIdx.x] = j < p.rows ? min(max(p.ids[j], 0), p.vocab - 1) : -2;
+    __syncthreads();
+    if (nxt < 0 && my >= 0) {
+      for (int t = 0; t < blockDim.x; ++t) {
+        int jj = j0 + t;
+        if (jj > i && tile[t] == my) { nxt = jj; break; }
+      }
+    }
+  }
+  if (i < p.rows) { p.next[i] = nxt; p.first[i] = 1; }
+}
+__global__ void __launch_bounds__(256) embed_mark_kernel(EmbedBwdProb p) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < p.rows && p.next[i] >= 0) p.first[p.next[i]] = 0;
+}
+// One block per position: the first holder of a token id sums dh over the chain of positions
+// holding that id, in increasing position order (deterministic), and writes the table row.
+template <typename T>
+__global__ void __launch_bounds__(256) embed_bwd_tok_kernel(EmbedBwdProb p) {
+  int i = blockIdx.x;
+  if (!p.first[i]) return;
+  int id = min(max(p.ids[i], 0), p.vocab - 1);
+  const T* dh = (const T*)p.dh;
+  for (int c = threadIdx.x; c < p.d; c += blockDim.x) {
+    float s = 0.f;
+    for (int j = i; j >= 0; j = p.next[j]) s += to_f(dh[(size_t)j * p.d + c]);
+    p.dtok[(size_t)id * p.d + c] = s;
+  }
+}
+template <typename T>
+__global__ void __launch_bounds__(256) embed_bwd_pos_kernel(EmbedBwdProb p) {
+  int t = blockIdx.x;
+  const T* dh = (const T*)p.dh;
+  for (int c = threadIdx.x; c < p.d; c += blockDim.x) {
+    float s = 0.f;
+    for (int b = 0; b < p.B; ++b) s += to_f(dh[((size_t)b * p.T + t) * p.d + c]);
+    p.dpos[(size_t)t * p.d + c] = s;
+  }
+}
+
+}  // namespace
+
+void launch_optim(const OptimArgs& a, cudaStream_t s) {
+  long long threads = (a.n_total + 3) / 4;
+  if (threads == 0) return;
+  optim_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, s>>>(a);
+}
+
+void launch_embed_fwd(const EmbedProb& p, int* d_status, bool is_bf16, cudaStream_t s) {
+  if (is_bf16) embed_fwd_kernel<bf16><<<p.rows, 256, 0, s>>>(p, d_status);
+  else embed_fwd_kernel<float><<<p.rows, 256, 0, s>>>(p, d_status);
+}
+
+void launch_embed_bwd(const EmbedBwdProb& p, bool is_bf16, cudaStream_t s) {
+  int nb = (p.rows + 255) / 256;
+  embed_link_kernel<<<nb, 256, 0, s>>>(p);
+  embed_mark_kernel<<<nb, 256, 0, s>>>(p);
+  cudaMemsetAsync(p.dtok, 0, (size_t)p.vocab * p.d * sizeof(float), s);
+  if (is_bf16) {
+    embed_bwd_tok_kernel<bf16><<<p.rows, 256, 0, s>>>(p);
+    embed_bwd_pos_kernel<bf16><<<p.T, 256, 0, s>>>(p);
+  } else {
+    embed_bwd_tok_kernel<float><<<p.rows, 256, 0, s>>>(p);
+    embed_bwd_pos_kernel<float><<<p.T, 256, 0, s>>>(p);
+  }
+}
+
+}  // namespace lp

@@ -1,0 +1,213 @@
+// Handle memory, parameter arena and launch emitters (see runtime.h).
+#include "runtime.h"
+
+#include <algorithm>
+#include <stdexcept>
+
+namespace lp {
+
+// ------------------------------------------------------------------ memory
+void* Handle::dalloc(size_t bytes) {
+  if (bytes == 0) bytes = 256;
+  bytes = (bytes + 255) / 256 * 256;
+  void* p = nullptr;
+  if (use_cuda_malloc) {
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) { cudaGetLastError(); p = nullptr; }
+  } else {
+    p = alloc.alloc(bytes, alloc.user);
+  }
+  if (!p) throw std::runtime_error("alloc: device allocation of " + std::to_string(bytes) + " bytes failed");
+  blocks.push_back(p);
+  device_bytes += bytes;
+  cudaError_t e = cudaMemset(p, 0, bytes);
+  if (e != cudaSuccess) throw std::runtime_error(std::string("cuda: memset: ") + cudaGetErrorString(e));
+  return p;
+}
+
+// ------------------------------------------------------------------ arena
+void Handle::add_tensor(const std::string& name, int chunk, std::vector<int64_t> shape, bool matrix) {
+  TensorRec t;
+  t.name = name;
+  t.chunk = chunk;
+  t.shape = shape;
+  t.numel = 1;
+  for (auto s : shape) t.numel *= s;
+  t.matrix = matrix;
+  tensors.push_back(t);
+}
+
+// Arena order: every matrix first, then every vector; each tensor starts on a 128-element
+// boundary (256 bytes in bf16, 512 in fp32), padding stays zero under every update rule.
+void Handle::finalize_arena() {
+  long long off = 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    for (auto& t : tensors) {
+      if (t.matrix != (pass == 0)) continue;
+      t.off = off;
+      off += (t.numel + 127) / 128 * 128;
+    }
+    if (pass == 0) n_matrix = off;
+  }
+  n_total = off;
+  master = (float*)dalloc(n_total * sizeof(float));
+  m1 = (float*)dalloc(n_total * sizeof(float));
+  if (opt.kind == LP_OPT_ADAM) m2 = (float*)dalloc(n_total * sizeof(float));
+  grad = (float*)dalloc(n_total * sizeof(float));
+  if (bf16_mode) working = (bf16*)dalloc(std::max<long long>(n_matrix, 128) * sizeof(bf16));
+}
+
+int Handle::find(const std::string& name) const {
+  for (size_t i = 0; i < tensors.size(); ++i)
+    if (tensors[i].name == name) return (int)i;
+  throw std::runtime_error("internal: no tensor named " + name);
+}
+const void* Handle::W(const std::string& name) const {
+  const TensorRec& t = tensors[find(name)];
+  if (bf16_mode && t.matrix) return working + t.off;
+  return master + t.off;
+}
+float* Handle::P32(const std::string& name) const { return master + tensors[find(name)].off; }
+float* Handle::G(const std::string& name) const { return grad + tensors[find(name)].off; }
+
+// ------------------------------------------------------------------ GEMM problems
+GemmProb gemm_fwd(const void* x, const void* W, void* y, int M, int N, int Kd, const float* bias, int act) {
+  GemmProb g{};
+  g.A = x; g.B = W; g.C = y; g.bias = bias; g.act = act;
+  g.M = M; g.N = N; g.K = Kd;
+  g.a_ms = Kd; g.a_ks = 1; g.b_ns = Kd; g.b_ks = 1; g.ldc = N;
+  return g;
+}
+// dx[M,Kd] = dy[M,N] * W[N,Kd]  (reduction over N)
+GemmProb gemm_dgrad(const void* dy, const void* W, void* dx, int M, int N, int Kd, int act, const void* aux) {
+  GemmProb g{};
+  g.A = dy; g.B = W; g.C = dx; g.act = act; g.aux = aux;
+  g.M = M; g.N = Kd; g.K = N;
+  g.a_ms = N; g.a_ks = 1; g.b_ns = 1; g.b_ks = Kd; g.ldc = Kd;
+  return g;
+}
+// dW[N,Kd] = dy[M,N]^T * x[M,Kd]  (reduction over the M rows of the minibatch), fp32 output
+GemmProb gemm_wgrad(const void* dy, const void* x, float* dW, int M, int N, int Kd) {
+  GemmProb g{};
+  g.A = dy; g.B = x; g.C = dW; g.out_f32 = 1;
+  g.M = N; g.N = Kd; g.K = M;
+  g.a_ms = 1; g.a_ks = N; g.b_ns = 1; g.b_ks = Kd; g.ldc = Kd;
+  return g;
+}
+
+// ------------------------------------------------------------------ emitters
+void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
+  if (probs.empty()) return;
+  int t = 0;
+  for (auto& g : probs) {
+    g.tiles_n = (g.N + 63) / 64;
+    g.tile_start = t;
+    t += ((g.M + 63) / 64) * g.tiles_n;
+  }
+  const GemmProb* d = h.upload(probs);
+  bool bf = h.bf16_mode;
+  int n = (int)probs.size();
+  p.add(1, [d, probs, n, bf](const RunCtx& c) { launch_gemm_simt(d, probs.data(), n, bf, c.stream); });
+}
+
+void emit_ln_fwd(Handle& h, Plan& p, const std::vector<LnProb>& probs) {
+  if (probs.empty()) return;
+  int mr = 0;
+  for (auto& q : probs) mr = std::max(mr, q.rows);
+  const LnProb* d = h.upload(probs);
+  int n = (int)probs.size();
+  bool bf = h.bf16_mode;
+  p.add(1, [=](const RunCtx& c) { launch_ln_fwd(d, n, mr, bf, c.stream); });
+}
+
+void emit_ln_bwd(Handle& h, Plan& p, std::vector<LnBwdProb> probs, const std::vector<float*>& dgamma,
+                 const std::vector<float*>& dbeta) {
+  if (probs.empty()) return;
+  int mr = 0;
+  for (size_t i = 0; i < probs.size(); ++i) {
+    auto& q = probs[i];
+    mr = std::max(mr, q.rows);
+    int nblk = (q.rows + LN_BWD_ROWS - 1) / LN_BWD_ROWS;
+    q.part = (float*)h.dalloc((size_t)nblk * 2 * q.d * sizeof(float));
+    h.pending_reduce.push_back(ColReduceProb{q.part, dgamma[i], nblk, q.d, 2 * q.d});
+    h.pending_reduce.push_back(ColReduceProb{q.part + q.d, dbeta[i], nblk, q.d, 2 * q.d});
+  }
+  const LnBwdProb* d = h.upload(probs);
+  int n = (int)probs.size();
+  bool bf = h.bf16_mode;
+  p.add(1, [=](const RunCtx& c) { launch_ln_bwd(d, n, mr, bf, c.stream); });
+}
+
+void emit_colsum(Handle& h, Plan& p, const std::vector<ColSumProb>& in, const std::vector<float*>& out) {
+  if (in.empty()) return;
+  std::vector<ColSumProb> probs = in;
+  int mr = 0, mc = 0;
+  for (size_t i = 0; i < probs.size(); ++i) {
+    auto& q = probs[i];
+    mr = std::max(mr, q.rows);
+    mc = std::max(mc, q.cols);
+    int nblk = (q.rows + COLSUM_ROWS - 1) / COLSUM_ROWS;
+    q.part = (float*)h.dalloc((size_t)nblk * q.cols * sizeof(float));
+    h.pending_reduce.push_back(ColReduceProb{q.part, out[i], nblk, q.cols, q.cols});
+  }
+  const ColSumProb* d = h.upload(probs);
+  int n = (int)probs.size();
+  bool bf = h.bf16_mode;
+  p.add(1, [=](const RunCtx& c) { launch_colsum_partial(d, n, mr, mc, bf, c.stream); });
+}
+
+void emit_pending_reduce(Handle& h, Plan& p) {
+  if (h.pending_reduce.empty()) return;
+  int mc = 0;
+  for (auto& q : h.pending_reduce) mc = std::max(mc, q.cols);
+  const ColReduceProb* d = h.upload(h.pending_reduce);
+  int n = (int)h.pending_reduce.size();
+  h.pending_reduce.clear();
+  p.add(1, [=](const RunCtx& c) { launch_col_reduce_f32(d, n, mc, c.stream); });
+}
+
+void emit_labels(Handle& h, Plan& p, const std::vector<LabelProb>& probs) {
+  const LabelProb* d = h.upload(probs);
+  int n = (int)probs.size();
+  int* st = h.d_status;
+  p.add(1, [=](const RunCtx& c) { launch_label_prep(d, n, st, c.stream); });
+}
+
+void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, const std::vector<int>& chunk_of) {
+  if (probs.empty()) return;
+  int mr = 0;
+  std::vector<LossProb> lps;
+  for (size_t i = 0; i < probs.size(); ++i) {
+    mr = std::max(mr, probs[i].rows);
+    lps.push_back(LossProb{probs[i].row_loss, probs[i].n_valid, probs[i].rows, chunk_of[i]});
+  }
+  const XentProb* d = h.upload(probs);
+  const LossProb* dl = h.upload(lps);
+  int n = (int)probs.size();
+  bool bf = h.bf16_mode;
+  float* losses = h.d_losses;
+  int* st = h.d_status;
+  p.add(2, [=](const RunCtx& c) {
+    launch_xent(d, n, mr, bf, c.stream);
+    launch_loss_reduce(dl, n, losses, st, c.stream);
+  });
+}
+
+void emit_optimizer(Handle& h, Plan& p) {
+  Handle* hp = &h;
+  p.add(1, [hp](const RunCtx& c) {
+    OptimArgs a{};
+    a.master = hp->master; a.m1 = hp->m1; a.m2 = hp->m2; a.grad = hp->grad; a.working = hp->working;
+    a.n_total = hp->n_total; a.n_matrix = hp->n_matrix;
+    a.kind = hp->opt.kind; a.lr = hp->opt.lr; a.momentum = hp->opt.momentum; a.weight_decay = hp->opt.weight_decay;
+    a.beta1 = hp->opt.beta1; a.beta2 = hp->opt.beta2; a.eps = hp->opt.eps;
+    double t = (double)(hp->step_count + 1);
+    a.omb1 = (float)(1.0 - (double)hp->opt.beta1);
+    a.omb2 = (float)(1.0 - (double)hp->opt.beta2);
+    a.bc1 = (float)(1.0 - pow((double)hp->opt.beta1, t));
+    a.bc2 = (float)(1.0 - pow((double)hp->opt.beta2, t));
+    launch_optim(a, c.stream);
+  });
+}
+
+}  // namespace lp

@@ -1,0 +1,116 @@
+// Host runtime behind the C ABI: the handle, its device memory, the parameter arena, and "plans"
+// (ordered lists of grouped kernel launches with device-resident problem tables, built once at
+// lp_create because every buffer a step touches is owned by the handle).
+#pragma once
+#include <functional>
+#include <string>
+#include <vector>
+
+#include "../../include/lp.h"
+#include "lp_kernels.h"
+
+namespace lp {
+
+struct TensorRec {
+  std::string name;
+  int chunk = 0;
+  std::vector<int64_t> shape;
+  int64_t numel = 0;
+  bool matrix = false;   // Linear weight, convolution filter or embedding table
+  int64_t off = 0;       // element offset in the arena
+};
+
+struct RunCtx {
+  cudaStream_t stream;
+  void* out_logits;      // lp_forward only
+};
+
+struct Plan {
+  std::vector<std::function<void(const RunCtx&)>> ops;
+  int launches = 0;
+  void add(int n_launches, std::function<void(const RunCtx&)> f) { ops.push_back(std::move(f)); launches += n_launches; }
+  void run(const RunCtx& c) const { for (auto& f : ops) f(c); }
+};
+
+struct Handle {
+  // ---- specification
+  lp_model_spec spec{};
+  std::vector<int> layer_widths, per_chunk, stage_channels;
+  lp_head_spec head{};
+  lp_optim_spec opt{};
+  int K = 0;
+  bool bf16_mode = false;
+  bool force_simt = false;
+  int rows = 0;             // rows entering the head: batch (MLP, RESNET) or batch*seq_len (LM)
+  // ---- memory
+  lp_alloc alloc{};
+  bool use_cuda_malloc = true;
+  std::vector<void*> blocks;
+  size_t device_bytes = 0;
+  // ---- parameter arena: [matrices of all chunks | vectors of all chunks]
+  std::vector<TensorRec> tensors;
+  long long n_total = 0, n_matrix = 0;
+  float *master = nullptr, *m1 = nullptr, *m2 = nullptr, *grad = nullptr;
+  bf16* working = nullptr;
+  // ---- step inputs / outputs
+  void* x_in = nullptr;  size_t x_bytes = 0;
+  int* y_in = nullptr;   size_t y_bytes = 0;
+  float* d_losses = nullptr;
+  int* d_status = nullptr;
+  // ---- chunk boundaries: activation and labels, two halves each (Sec. 6 pipelining)
+  std::vector<void*> bnd[2];
+  std::vector<int*> lab[2];
+  size_t bnd_bytes_total = 0;
+  std::vector<size_t> bnd_bytes;
+  std::vector<int*> n_valid;
+  // ---- plans
+  Plan sync_plan, pipe_plan[2], prime_plan[2], fwd_plan[2];
+  std::vector<ColReduceProb> pending_reduce;   // collected while a plan is being built
+  int parity = 0;
+  bool primed = false;
+  long long step_count = 0;
+  int last_launches = 0;
+  std::string err;
+
+  size_t esize() const { return bf16_mode ? 2 : 4; }
+  // tensor lookup
+  int find(const std::string& name) const;
+  const void* W(const std::string& name) const;   // GEMM operand pointer (bf16 working copy or fp32 master)
+  float* P32(const std::string& name) const;      // fp32 master (vectors: biases, norm scales)
+  float* G(const std::string& name) const;        // fp32 gradient
+  // device memory (zero-filled); throws std::runtime_error on failure
+  void* dalloc(size_t bytes);
+  template <typename T> const T* upload(const std::vector<T>& v) {
+    if (v.empty()) return nullptr;
+    void* d = dalloc(v.size() * sizeof(T));
+    cudaMemcpy(d, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice);
+    return (const T*)d;
+  }
+  void add_tensor(const std::string& name, int chunk, std::vector<int64_t> shape, bool matrix);
+  void finalize_arena();
+};
+
+// ---- emitters: append one grouped launch (or a few) to a plan
+void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs);
+void emit_ln_fwd(Handle& h, Plan& p, const std::vector<LnProb>& probs);
+// LayerNorm backward; the parameter-gradient partials are queued for the plan's final reduction
+void emit_ln_bwd(Handle& h, Plan& p, std::vector<LnBwdProb> probs, const std::vector<float*>& dgamma,
+                 const std::vector<float*>& dbeta);
+// db[c] = sum_r x[r,c]: partial sums now, final reduction queued
+void emit_colsum(Handle& h, Plan& p, const std::vector<ColSumProb>& probs_without_part, const std::vector<float*>& out);
+void emit_pending_reduce(Handle& h, Plan& p);
+void emit_labels(Handle& h, Plan& p, const std::vector<LabelProb>& probs);
+void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, const std::vector<int>& chunk_of);
+void emit_optimizer(Handle& h, Plan& p);
+
+// GEMM problem constructors (x: [M,K] row-major, W: [N,K] row-major, dy: [M,N] row-major)
+GemmProb gemm_fwd(const void* x, const void* W, void* y, int M, int N, int Kd, const float* bias, int act);
+GemmProb gemm_dgrad(const void* dy, const void* W, void* dx, int M, int N, int Kd, int act, const void* aux);
+GemmProb gemm_wgrad(const void* dy, const void* x, float* dW, int M, int N, int Kd);
+
+// ---- per-family builders: register tensors, allocate buffers, build all plans
+void build_mlp(Handle& h);
+void build_lm(Handle& h);
+void build_resnet(Handle& h);
+
+}  // namespace lp

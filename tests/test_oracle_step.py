@@ -309,3 +309,18 @@ def test_determinism_and_dtype_modes():
     o64 = LocalUpdateOracle(cfg, lp_synth.init_params(cfg), dtype=np.float64)
     l64 = np.array([o64.step(*lp_synth.minibatch(cfg, t)) for t in range(3)])
     assert np.allclose(outs[0][0], l64, rtol=1e-5)
+
+
+def test_key_bias_gradient_is_identically_zero():
+    """Softmax is invariant to a shift common to all scores of a row, so the key bias of an attention
+    layer has zero gradient: what an fp32 run stores there is rounding noise (parity tests skip it)."""
+    cfg = TINY["lm"]
+    params = spread_params(cfg)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    x, y = lp_synth.minibatch(cfg, 0)
+    orc.cfg = dict(cfg, optim=dict(kind="sgdm", lr=0.0, momentum=0.0, weight_decay=0.0))
+    orc.step(x, y, "sync")
+    d = cfg["d_model"]
+    for n, g in orc.last_grads.items():
+        if n.endswith(".bqkv"):
+            assert np.abs(g[d:2 * d]).max() < 1e-12 * np.abs(g[:d]).max()
