@@ -185,6 +185,26 @@ size_t lp_state_size(lp_handle h);
 lp_status lp_save_state(lp_handle h, void* host_dst, size_t bytes);
 lp_status lp_load_state(lp_handle h, const void* host_src, size_t bytes);
 
+/*
+ * Kernel-level entry for tests and profiling: one grouped launch of n bf16 GEMM problems
+ *   C[m,n] = epilogue( sum_k A(m,k) * B(n,k) ),  A(m,k) = A[m*a_ms + k*a_ks], B(n,k) = B[n*b_ns + k*b_ks]
+ * (the products of a Linear layer, App. A.1, in forward, input-gradient and weight-gradient form).
+ * All pointers inside the descriptors are device pointers; `probs` itself is a host array.
+ * Exactly one stride of each operand must be 1.  act: 0 none, 1 ReLU, 2 GELU (C2 receives the
+ * pre-activation), 3 multiply by [aux > 0], 4 multiply by GELU'(aux).  out_f32: C is float, else bf16.
+ * backend: 0 = tensor cores where the sizes allow, 1 = FP32 ALUs.  *used_tensor_cores (nullable)
+ * receives how many of the problems ran on the tensor-core kernel.  Asynchronous on `stream`
+ * except for the upload of the descriptor table.  Errors: INVALID_ARG, ALLOC, CUDA.
+ */
+typedef struct {
+  const void* A; const void* B; void* C; void* C2;
+  const float* bias; const void* resid; const void* aux;
+  int M, N, K;
+  long long a_ms, a_ks, b_ns, b_ks;
+  int ldc, act, out_f32;
+} lp_gemm_desc;
+lp_status lp_gemm_bf16(int n, const lp_gemm_desc* probs, int backend, void* stream, int* used_tensor_cores);
+
 /* Number of kernel launches the last lp_step issued (for reporting). */
 int lp_last_step_launches(lp_handle h);
 /* Device bytes owned by the handle. */

@@ -59,7 +59,7 @@ class lp_tensor_info(C.Structure):
 EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "lp_num_tensors",
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
-           "lp_last_error"]
+           "lp_last_error", "lp_gemm_bf16"]
 
 
 def load_library() -> C.CDLL:
@@ -232,3 +232,26 @@ def lp_device_bytes(h) -> int:
 
 def lp_last_error(h=None) -> str:
     return (_lib.lp_last_error(h) or b"").decode()
+
+
+class lp_gemm_desc(C.Structure):
+    _fields_ = [("A", C.c_void_p), ("B", C.c_void_p), ("C", C.c_void_p), ("C2", C.c_void_p),
+                ("bias", C.c_void_p), ("resid", C.c_void_p), ("aux", C.c_void_p),
+                ("M", C.c_int), ("N", C.c_int), ("K", C.c_int),
+                ("a_ms", C.c_longlong), ("a_ks", C.c_longlong), ("b_ns", C.c_longlong), ("b_ks", C.c_longlong),
+                ("ldc", C.c_int), ("act", C.c_int), ("out_f32", C.c_int)]
+
+
+_lib.lp_gemm_bf16.argtypes = [C.c_int, C.POINTER(lp_gemm_desc), C.c_int, C.c_void_p, C.POINTER(C.c_int)]
+
+
+def lp_gemm_bf16(descs: list, backend: int = 0, stream=None) -> int:
+    """One grouped launch of bf16 GEMM problems (list of dicts with the fields of lp_gemm_desc;
+    pointers may be torch tensors).  Returns how many problems ran on the tensor-core kernel."""
+    arr = (lp_gemm_desc * len(descs))()
+    for d, q in zip(arr, descs):
+        for k, v in q.items():
+            setattr(d, k, _ptr(v) if k in ("A", "B", "C", "C2", "bias", "resid", "aux") else int(v))
+    used = C.c_int(0)
+    _check(None, _lib.lp_gemm_bf16(len(descs), arr, backend, stream, C.byref(used)))
+    return used.value

@@ -1,0 +1,434 @@
+// Grouped bf16 GEMM on the 5th-generation tensor cores (tcgen05) for sm_100a.
+//
+// One persistent CTA per SM walks a flat list of 128x256 output tiles that spans every problem of
+// the launch (all chunks' forward, input-gradient and weight-gradient products of one phase:
+// Sec. 3 makes them independent).  Per tile, 64-deep k slices of A and B are brought into a
+// 4-stage shared-memory ring by TMA (128-byte swizzle; out-of-range rows/columns read as zero, so
+// ragged M, N, K need no special case), one elected thread issues tcgen05.mma (M=128, N=256, K=16,
+// bf16 x bf16 -> fp32) into one of two 256-column TMEM accumulators, and four epilogue warps read
+// the finished accumulator back with tcgen05.ld, apply the fused epilogue (bias, residual,
+// ReLU/GELU, ReLU mask, GELU') and store bf16 or fp32 while the next tile's main loop already
+// runs on the other accumulator.
+//
+// Operands may be K-major (reduction index contiguous) or MN-major (row/column index contiguous),
+// per problem: forward uses K/K, the input gradient K/MN, the weight gradient MN/MN, so no
+// transposed copy of a weight or an activation is ever materialised.
+//
+// Every wait on an mbarrier is bounded (about two seconds): on expiry the thread raises the
+// TIMEOUT bit of the status word, all roles leave their loops, TMEM is freed and the kernel returns.
+// No TMA load uses cluster multicast.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "gemm_tc.h"
+
+namespace lp {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;              // 16 KB
+constexpr int B_BYTES = BN * BK * 2;              // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;    // 48 KB
+constexpr int NTHREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+struct __align__(8) Shared {
+  uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long gtime_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the wait gave up or another role already did.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
+  if (mbar_try(bar, parity)) return true;
+  unsigned long long t0 = gtime_ns();
+  int spins = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spins & 255) == 0) {
+      if (*(volatile int*)&sh->abort_flag) return false;
+      if (gtime_ns() - t0 > WAIT_LIMIT_NS) {
+        *(volatile int*)&sh->abort_flag = 1;
+        atomicOr(status, ST_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 1024-byte atoms (8 rows of 128 bytes).
+//   K-major : rows of 64 k-elements; next 8-row group 1024 B further (stride field); leading field unused.
+//   MN-major: rows of 64 m/n-elements, one row per k; next 8-k group 1024 B further (stride field);
+//             next 64-element m/n block BK*128 B further (leading field).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(mn_major ? ((BK * 128) >> 4) : 1) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  return d;
+}
+
+// Epilogue for 32 consecutive columns of one row held in registers.
+template <bool VEC>
+__device__ __forceinline__ void store_row32(const GemmProb& p, int m, int n0, const uint32_t* acc) {
+  float v[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
+  size_t off = (size_t)m * p.ldc + n0;
+  int nvalid = min(32, p.N - n0);
+  if (p.bias) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) if (VEC || j < nvalid) v[j] += p.bias[n0 + j];
+  }
+  auto load32 = [&](const void* base, float* o) {
+    const bf16* src = (const bf16*)base + off;
+    if (VEC) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint4 u = *(const uint4*)(src + q * 8);
+        const __nv_bfloat162* h = (const __nv_bfloat162*)&u;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { float2 f = __bfloat1622float2(h[t]); o[q * 8 + 2 * t] = f.x; o[q * 8 + 2 * t + 1] = f.y; }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) o[j] = j < nvalid ? __bfloat162float(src[j]) : 0.f;
+    }
+  };
+  auto store32 = [&](void* base, const float* o) {
+    bf16* dst = (bf16*)base + off;
+    if (VEC) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint4 u;
+        __nv_bfloat162* h = (__nv_bfloat162*)&u;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(o[q * 8 + 2 * t], o[q * 8 + 2 * t + 1]);
+        *(uint4*)(dst + q * 8) = u;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = __float2bfloat16_rn(o[j]);
+    }
+  };
+  float t[32];
+  if (p.resid) {
+    load32(p.resid, t);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] += t[j];
+  }
+  switch (p.act) {
+    case EPI_RELU:
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+      break;
+    case EPI_GELU:
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = __bfloat162float(__float2bfloat16_rn(v[j]));
+      store32(p.C2, v);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = gelu_f(v[j]);
+      break;
+    case EPI_RELU_MASK:
+      load32(p.aux, t);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = t[j] > 0.f ? v[j] : 0.f;
+      break;
+    case EPI_GELU_GRAD:
+      load32(p.aux, t);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_f(t[j]);
+      break;
+    default: break;
+  }
+  if (p.out_f32) {
+    float* dst = (float*)p.C + off;
+    if (VEC) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) *(float4*)(dst + q * 4) = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
+    }
+  } else {
+    store32(p.C, v);
+  }
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict__ maps, int nprob, int total_tiles,
+               int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  Shared* sh = (Shared*)(tiles + STAGES * STAGE_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh->tmem_full[a], 1); mbar_init(&sh->tmem_empty[a], 4); }
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *(volatile uint32_t*)&sh->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int pi = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
+        const GemmProb& p = probs[pi];
+        const CUtensorMap* mapA = maps + 2 * pi;
+        const CUtensorMap* mapB = mapA + 1;
+        int t = tile - p.tile_start;
+        int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * BN;
+        bool a_mn = p.a_ms == 1, b_mn = p.b_ns == 1;
+        int kb_n = (p.K + BK - 1) / BK;
+        for (int kb = 0; kb < kb_n; ++kb) {
+          if (!(ok = mbar_wait(&sh->empty[stage], phase ^ 1, sh, status))) break;
+          uint8_t* a_dst = tiles + stage * STAGE_BYTES;
+          uint8_t* b_dst = a_dst + A_BYTES;
+          mbar_expect_tx(&sh->full[stage], STAGE_BYTES);
+          int k0 = kb * BK;
+          if (a_mn) {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, &sh->full[stage]);
+          } else {
+            tma_load_2d(a_dst, mapA, k0, m0, &sh->full[stage]);
+          }
+          if (b_mn) {
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, &sh->full[stage]);
+          } else {
+            tma_load_2d(b_dst, mapB, k0, n0, &sh->full[stage]);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        // copies already issued still land in this CTA's shared memory: give them a bounded time
+        unsigned long long t0 = gtime_ns();
+        while (gtime_ns() - t0 < 2000000ull) { }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int pi = 0, it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+        while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
+        const GemmProb& p = probs[pi];
+        bool a_mn = p.a_ms == 1, b_mn = p.b_ns == 1;
+        uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+                         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        int ab = it & 1;
+        uint32_t use = (uint32_t)(it >> 1);
+        if (!(ok = mbar_wait(&sh->tmem_empty[ab], (use & 1) ^ 1, sh, status))) break;
+        tc_fence_after();
+        uint32_t d_tmem = tmem_base + ab * BN;
+        int kb_n = (p.K + BK - 1) / BK;
+        for (int kb = 0; kb < kb_n; ++kb) {
+          if (!(ok = mbar_wait(&sh->full[stage], phase, sh, status))) break;
+          tc_fence_after();
+          uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
+          uint32_t b_addr = a_addr + A_BYTES;
+          uint64_t adesc = make_desc(a_addr, a_mn), bdesc = make_desc(b_addr, b_mn);
+          uint32_t a_step = a_mn ? (16 * 128) >> 4 : 32 >> 4;
+          uint32_t b_step = b_mn ? (16 * 128) >> 4 : 32 >> 4;
+#pragma unroll
+          for (int k4 = 0; k4 < BK / 16; ++k4)
+            tc_mma(d_tmem, adesc + (uint64_t)(k4 * a_step), bdesc + (uint64_t)(k4 * b_step), idesc, (kb | k4) != 0);
+          tc_commit(&sh->empty[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) tc_commit(&sh->tmem_full[ab]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int quarter = warp & 3;            // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
+    int pi = 0, it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
+      const GemmProb p = probs[pi];
+      int t = tile - p.tile_start;
+      int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * BN;
+      int ab = it & 1;
+      uint32_t use = (uint32_t)(it >> 1);
+      ok = mbar_wait(&sh->tmem_full[ab], use & 1, sh, status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      int m = m0 + quarter * 32 + lane;
+      size_t esz = p.out_f32 ? 4 : 2;
+      bool vec_ok = (p.ldc % 8 == 0) && (((uintptr_t)p.C & 15) == 0) && (!p.C2 || ((uintptr_t)p.C2 & 15) == 0) &&
+                    (!p.resid || ((uintptr_t)p.resid & 15) == 0) && (!p.aux || ((uintptr_t)p.aux & 15) == 0);
+      (void)esz;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t acc[32];
+        uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + c * 32);
+        tc_ld32(taddr, acc);
+        tc_wait_ld();
+        int nc = n0 + c * 32;
+        if (m < p.M && nc < p.N) {
+          if (vec_ok && nc + 32 <= p.N) store_row32<true>(p, m, nc, acc);
+          else store_row32<false>(p, m, nc, acc);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->tmem_empty[ab]);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode() {
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = (EncodeFn)p;
+  }
+  return fn;
+}
+
+// 2-D bf16 tensor map: inner extent `inner` (contiguous), outer extent `outer` with a row pitch of
+// `pitch` elements, box = 64 x box_outer, 128-byte swizzle, zero fill outside the tensor.
+bool encode_map(CUtensorMap* out, const void* base, long long inner, long long outer, long long pitch, int box_outer) {
+  EncodeFn fn = get_encode();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+  cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_outer};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool gemm_tc_eligible(const GemmProb& g) {
+  if (g.M < 1 || g.N < 1 || g.K < 1) return false;
+  if ((long long)g.M * g.N < 64 * 64 || g.K < 32) return false;          // too small to pay for a 128x256 tile
+  if (((uintptr_t)g.A & 15) || ((uintptr_t)g.B & 15)) return false;
+  long long a_pitch = g.a_ms == 1 ? g.a_ks : g.a_ms, b_pitch = g.b_ns == 1 ? g.b_ks : g.b_ns;
+  if (a_pitch % 8 || b_pitch % 8) return false;                          // TMA: pitches are multiples of 16 bytes
+  if (g.a_ms != 1 && g.a_ks != 1) return false;
+  if (g.b_ns != 1 && g.b_ks != 1) return false;
+  return get_encode() != nullptr;
+}
+
+int gemm_tc_tiles(GemmProb& g, int tile_start) {
+  g.tile_start = tile_start;
+  g.tiles_n = (g.N + BN - 1) / BN;
+  return ((g.M + BM - 1) / BM) * g.tiles_n;
+}
+
+bool gemm_tc_encode(const GemmProb& g, void* mapA, void* mapB) {
+  bool okA, okB;
+  if (g.a_ms == 1) okA = encode_map((CUtensorMap*)mapA, g.A, g.M, g.K, g.a_ks, BK);       // MN-major: rows are k
+  else okA = encode_map((CUtensorMap*)mapA, g.A, g.K, g.M, g.a_ms, BM);
+  if (g.b_ns == 1) okB = encode_map((CUtensorMap*)mapB, g.B, g.N, g.K, g.b_ks, BK);
+  else okB = encode_map((CUtensorMap*)mapB, g.B, g.K, g.N, g.b_ns, BN);
+  return okA && okB;
+}
+
+cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int nprob, int total_tiles, int* d_status,
+                           int num_sms, cudaStream_t s) {
+  static bool attr_set = false;
+  size_t smem = STAGES * STAGE_BYTES + 1024 + sizeof(Shared);
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  if (total_tiles == 0) return cudaSuccess;
+  int grid = total_tiles < num_sms ? total_tiles : num_sms;
+  gemm_tc_kernel<<<grid, NTHREADS, smem, s>>>(d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
+  return cudaGetLastError();
+}
+
+}  // namespace lp

@@ -1,0 +1,18 @@
+// Host interface of the tcgen05 grouped GEMM (gemm_tc.cu).
+#pragma once
+#include "lp_kernels.h"
+
+namespace lp {
+
+// True if the problem can run on the tensor-core kernel: bf16 operands, 16-byte aligned bases,
+// pitches that are multiples of 8 elements, and enough work to fill a 128x256 tile.
+bool gemm_tc_eligible(const GemmProb& g);
+// Fill tile_start / tiles_n for 128x256 tiles; returns the number of tiles of this problem.
+int gemm_tc_tiles(GemmProb& g, int tile_start);
+// Encode the two TMA tensor maps (128 bytes each, 64-byte aligned host memory) of a problem.
+bool gemm_tc_encode(const GemmProb& g, void* mapA, void* mapB);
+// d_maps: device array of 2*nprob tensor maps, [A0, B0, A1, B1, ...].
+cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int nprob, int total_tiles, int* d_status,
+                           int num_sms, cudaStream_t s);
+
+}  // namespace lp

@@ -4,6 +4,7 @@
 #include <stdexcept>
 
 #include "runtime.h"
+#include "gemm_tc.h"
 
 using namespace lp;
 
@@ -172,6 +173,11 @@ lp_status lp_create(const lp_model_spec* model, int K, const lp_head_spec* head,
     h.bf16_mode = model->dtype == LP_BF16;
     h.force_simt = model->gemm_backend == 1 || !h.bf16_mode;
     if (alloc) { h.alloc = *alloc; h.use_cuda_malloc = false; }
+    {
+      int dev = 0;
+      cudaGetDevice(&dev);
+      cudaDeviceGetAttribute(&h.num_sms, cudaDevAttrMultiProcessorCount, dev);
+    }
     h.d_losses = (float*)h.dalloc(sizeof(float) * K);
     h.d_status = (int*)h.dalloc(sizeof(int));
     switch (model->family) {
@@ -383,6 +389,68 @@ static lp_status state_io(lp_handle hh, void* host, size_t bytes, bool save) {
 
 lp_status lp_save_state(lp_handle hh, void* host_dst, size_t bytes) { return state_io(hh, host_dst, bytes, true); }
 lp_status lp_load_state(lp_handle hh, const void* host_src, size_t bytes) { return state_io(hh, const_cast<void*>(host_src), bytes, false); }
+
+lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream, int* used_tc) {
+  if (n < 1 || !in) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_gemm_bf16: no problems");
+  cudaStream_t s = (cudaStream_t)stream;
+  static int* d_status = nullptr;
+  static int num_sms = 0;
+  if (!d_status) {
+    if (cudaMalloc(&d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, LP_ERR_ALLOC, "status word"); }
+    cudaMemset(d_status, 0, sizeof(int));
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  std::vector<GemmProb> tc, simt;
+  for (int i = 0; i < n; ++i) {
+    const lp_gemm_desc& q = in[i];
+    if (!q.A || !q.B || !q.C || q.M < 1 || q.N < 1 || q.K < 1) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_gemm_bf16: bad problem");
+    if ((q.a_ms != 1 && q.a_ks != 1) || (q.b_ns != 1 && q.b_ks != 1)) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_gemm_bf16: one stride per operand must be 1");
+    GemmProb g{};
+    g.A = q.A; g.B = q.B; g.C = q.C; g.C2 = q.C2; g.bias = q.bias; g.resid = q.resid; g.aux = q.aux;
+    g.M = q.M; g.N = q.N; g.K = q.K; g.a_ms = q.a_ms; g.a_ks = q.a_ks; g.b_ns = q.b_ns; g.b_ks = q.b_ks;
+    g.ldc = q.ldc; g.act = q.act; g.out_f32 = q.out_f32;
+    if (backend == 0 && gemm_tc_eligible(g)) tc.push_back(g);
+    else simt.push_back(g);
+  }
+  if (used_tc) *used_tc = (int)tc.size();
+  // descriptor tables live in a per-process scratch buffer that grows on demand
+  static void* d_tab = nullptr;
+  static size_t d_cap = 0;
+  struct alignas(64) Map { unsigned char b[128]; };
+  size_t need = 256 + tc.size() * sizeof(GemmProb) + 256 + 2 * tc.size() * sizeof(Map) + simt.size() * sizeof(GemmProb) + 256;
+  if (need > d_cap) {
+    cudaStreamSynchronize(s);
+    if (d_tab) cudaFree(d_tab);
+    if (cudaMalloc(&d_tab, need * 2) != cudaSuccess) { cudaGetLastError(); d_tab = nullptr; d_cap = 0; return fail(nullptr, LP_ERR_ALLOC, "descriptor table"); }
+    d_cap = need * 2;
+  }
+  char* cur = (char*)d_tab;
+  auto take = [&](size_t bytes) { char* r = cur; cur += (bytes + 255) / 256 * 256; return r; };
+  if (!tc.empty()) {
+    int total = 0;
+    for (auto& g : tc) total += gemm_tc_tiles(g, total);
+    std::vector<Map> maps(2 * tc.size());
+    for (size_t i = 0; i < tc.size(); ++i)
+      if (!gemm_tc_encode(tc[i], &maps[2 * i], &maps[2 * i + 1])) return fail(nullptr, LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+    GemmProb* dp = (GemmProb*)take(tc.size() * sizeof(GemmProb));
+    Map* dm = (Map*)take(maps.size() * sizeof(Map));
+    cudaMemcpyAsync(dp, tc.data(), tc.size() * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
+    cudaMemcpyAsync(dm, maps.data(), maps.size() * sizeof(Map), cudaMemcpyHostToDevice, s);
+    cudaStreamSynchronize(s);
+    launch_gemm_tc(dp, dm, (int)tc.size(), total, d_status, num_sms, s);
+  }
+  if (!simt.empty()) {
+    int t = 0;
+    for (auto& g : simt) { g.tiles_n = (g.N + 63) / 64; g.tile_start = t; t += ((g.M + 63) / 64) * g.tiles_n; }
+    GemmProb* dp = (GemmProb*)take(simt.size() * sizeof(GemmProb));
+    cudaMemcpyAsync(dp, simt.data(), simt.size() * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
+    cudaStreamSynchronize(s);
+    launch_gemm_simt(dp, simt.data(), (int)simt.size(), true, s);
+  }
+  return check_cuda(nullptr, "lp_gemm_bf16");
+}
 
 int lp_last_step_launches(lp_handle hh) { return hh ? hh->h.last_launches : 0; }
 size_t lp_device_bytes(lp_handle hh) { return hh ? hh->h.device_bytes : 0; }

@@ -1,5 +1,6 @@
 // Handle memory, parameter arena and launch emitters (see runtime.h).
 #include "runtime.h"
+#include "gemm_tc.h"
 
 #include <algorithm>
 #include <stdexcept>
@@ -98,16 +99,38 @@ GemmProb gemm_wgrad(const void* dy, const void* x, float* dW, int M, int N, int 
 // ------------------------------------------------------------------ emitters
 void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
   if (probs.empty()) return;
-  int t = 0;
+  // Problems the tensor-core kernel takes go into one grouped launch, the rest into another.
+  std::vector<GemmProb> tc, simt;
   for (auto& g : probs) {
-    g.tiles_n = (g.N + 63) / 64;
-    g.tile_start = t;
-    t += ((g.M + 63) / 64) * g.tiles_n;
+    if (!h.force_simt && gemm_tc_eligible(g)) tc.push_back(g);
+    else simt.push_back(g);
   }
-  const GemmProb* d = h.upload(probs);
-  bool bf = h.bf16_mode;
-  int n = (int)probs.size();
-  p.add(1, [d, probs, n, bf](const RunCtx& c) { launch_gemm_simt(d, probs.data(), n, bf, c.stream); });
+  if (!tc.empty()) {
+    int total = 0;
+    for (auto& g : tc) total += gemm_tc_tiles(g, total);
+    struct alignas(64) Map { unsigned char b[128]; };
+    std::vector<Map> maps(2 * tc.size());
+    for (size_t i = 0; i < tc.size(); ++i)
+      if (!gemm_tc_encode(tc[i], &maps[2 * i], &maps[2 * i + 1])) throw std::runtime_error("cuda: cuTensorMapEncodeTiled failed");
+    const GemmProb* d = h.upload(tc);
+    const void* dm = h.upload(maps);
+    int n = (int)tc.size();
+    int* st = h.d_status;
+    int sms = h.num_sms;
+    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream); });
+  }
+  if (!simt.empty()) {
+    int t = 0;
+    for (auto& g : simt) {
+      g.tiles_n = (g.N + 63) / 64;
+      g.tile_start = t;
+      t += ((g.M + 63) / 64) * g.tiles_n;
+    }
+    const GemmProb* d = h.upload(simt);
+    bool bf = h.bf16_mode;
+    int n = (int)simt.size();
+    p.add(1, [d, simt, n, bf](const RunCtx& c) { launch_gemm_simt(d, simt.data(), n, bf, c.stream); });
+  }
 }
 
 void emit_ln_fwd(Handle& h, Plan& p, const std::vector<LnProb>& probs) {

@@ -41,6 +41,7 @@ struct Handle {
   int K = 0;
   bool bf16_mode = false;
   bool force_simt = false;
+  int num_sms = 148;
   int rows = 0;             // rows entering the head: batch (MLP, RESNET) or batch*seq_len (LM)
   // ---- memory
   lp_alloc alloc{};

@@ -1,0 +1,93 @@
+"""The grouped bf16 GEMM kernels against the oracle's Linear layer (forward, input gradient,
+weight gradient), on ragged sizes that span several 128x256 tiles and a partial tail."""
+import numpy as np
+import pytest
+import torch
+
+import lp_synth
+from oracle import layers as L
+from paper_2012_03837_b200 import binding as lp
+
+pytestmark = pytest.mark.gpu
+
+
+def bf(a):
+    return torch.from_numpy(lp_synth.bf16_round(a)).to("cuda").to(torch.bfloat16).contiguous()
+
+
+def problems(M, N, K, rng):
+    """Forward, dgrad and wgrad problems of one Linear layer y = x W^T + b with their oracle results."""
+    x = lp_synth.bf16_round(rng.standard_normal((M, K)).astype(np.float32))
+    W = lp_synth.bf16_round((rng.standard_normal((N, K)) / np.sqrt(K)).astype(np.float32))
+    b = rng.standard_normal(N).astype(np.float32)
+    dy = lp_synth.bf16_round(rng.standard_normal((M, N)).astype(np.float32))
+    y, cache = L.linear_fwd(x.astype(np.float64), W.astype(np.float64), b.astype(np.float64))
+    dx, dW, _ = L.linear_bwd(dy.astype(np.float64), cache)
+    t = dict(x=bf(x), W=bf(W), dy=bf(dy), b=torch.from_numpy(b).cuda(),
+             y=torch.zeros(M, N, dtype=torch.bfloat16, device="cuda"),
+             dx=torch.zeros(M, K, dtype=torch.bfloat16, device="cuda"),
+             dW=torch.zeros(N, K, dtype=torch.float32, device="cuda"))
+    descs = [
+        dict(A=t["x"], B=t["W"], C=t["y"], bias=t["b"], M=M, N=N, K=K, a_ms=K, a_ks=1, b_ns=K, b_ks=1, ldc=N),
+        dict(A=t["dy"], B=t["W"], C=t["dx"], M=M, N=K, K=N, a_ms=N, a_ks=1, b_ns=1, b_ks=K, ldc=K),
+        dict(A=t["dy"], B=t["x"], C=t["dW"], M=N, N=K, K=M, a_ms=1, a_ks=N, b_ns=1, b_ks=K, ldc=K, out_f32=1),
+    ]
+    return t, descs, dict(y=y, dx=dx, dW=dW)
+
+
+def check(t, ref, tag):
+    for name in ("y", "dx", "dW"):
+        got = t[name].float().cpu().numpy().astype(np.float64)
+        scale = np.abs(ref[name]).max()
+        err = np.abs(got - ref[name]).max() / scale
+        tol = 1e-2 if name != "dW" else 1e-4     # bf16 outputs carry one rounding (2^-9); fp32 output does not
+        assert err < tol, (tag, name, err)
+
+
+@pytest.mark.parametrize("backend", [1, 0])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 128), (200, 264, 72), (1000, 520, 328), (136, 1000, 2048)])
+def test_linear_products(M, N, K, backend):
+    rng = np.random.default_rng(M + N + K)
+    t, descs, ref = problems(M, N, K, rng)
+    used = 0
+    for d in descs:                      # one launch per product
+        used += lp.lp_gemm_bf16([d], backend)
+    torch.cuda.synchronize()
+    assert used == (0 if backend else 3)
+    check(t, ref, (M, N, K, backend))
+
+
+def test_grouped_launch_of_mixed_problems():
+    rng = np.random.default_rng(7)
+    sets = [problems(*s, rng) for s in [(256, 256, 128), (200, 264, 72), (384, 1000, 256)]]
+    descs = [d for _, ds, _ in sets for d in ds]
+    assert lp.lp_gemm_bf16(descs, 0) == len(descs)
+    torch.cuda.synchronize()
+    for i, (t, _, ref) in enumerate(sets):
+        check(t, ref, i)
+
+
+def test_epilogues_match_between_backends():
+    """Bias + residual + GELU (two outputs), ReLU mask and GELU' epilogues: tensor-core kernel vs FP32-ALU kernel."""
+    rng = np.random.default_rng(3)
+    M, N, K = 264, 520, 136
+    x, W = bf(rng.standard_normal((M, K)).astype(np.float32)), bf((rng.standard_normal((N, K)) / 12).astype(np.float32))
+    b = torch.from_numpy(rng.standard_normal(N).astype(np.float32)).cuda()
+    r = bf(rng.standard_normal((M, N)).astype(np.float32))
+    aux = bf(rng.standard_normal((M, N)).astype(np.float32))
+    outs = {}
+    for backend in (1, 0):
+        res = []
+        for act in (1, 2, 3, 4):
+            c = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+            c2 = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+            d = dict(A=x, B=W, C=c, C2=c2, bias=b, resid=r, aux=aux, M=M, N=N, K=K, a_ms=K, a_ks=1, b_ns=K, b_ks=1, ldc=N, act=act)
+            lp.lp_gemm_bf16([d], backend)
+            res += [c, c2]
+        torch.cuda.synchronize()
+        outs[backend] = [t.float().cpu().numpy() for t in res]
+    for a, b_ in zip(outs[0], outs[1]):
+        assert np.abs(a - b_).max() <= 2e-2 * max(1.0, np.abs(b_).max())
+    # and the FP32-ALU GELU output equals the oracle's GELU of its own stored pre-activation
+    u, g = outs[1][3], outs[1][2]
+    assert np.abs(lp_synth.bf16_round(L.gelu_fwd(u.astype(np.float64))[0].astype(np.float32)) - g).max() < 1e-2
