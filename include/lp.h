@@ -205,6 +205,21 @@ typedef struct {
 } lp_gemm_desc;
 lp_status lp_gemm_bf16(int n, const lp_gemm_desc* probs, int backend, void* stream, int* used_tensor_cores);
 
+/*
+ * Per-kernel-class timing for benchmarks.  While enabled, every grouped launch of lp_step is
+ * bracketed by a pair of CUDA events on the caller's stream.  lp_profile_read synchronises the
+ * device and returns, for each class and summed over the steps since the last read: device
+ * milliseconds, algorithmic work (FLOPs for the GEMM and attention classes, bytes for the others)
+ * and kernel launches.  Each output array has LP_KIND_COUNT entries.
+ */
+enum {
+  LP_KIND_OTHER = 0, LP_KIND_GEMM_TC = 1, LP_KIND_GEMM_ALU = 2, LP_KIND_NORM = 3, LP_KIND_XENT = 4,
+  LP_KIND_ATTN = 5, LP_KIND_OPTIM = 6, LP_KIND_REDUCE = 7, LP_KIND_EMBED = 8, LP_KIND_CONV_AUX = 9,
+  LP_KIND_COUNT = 10
+};
+lp_status lp_profile_enable(lp_handle h, int on);
+lp_status lp_profile_read(lp_handle h, double* ms, double* work, int* launches);
+
 /* Number of kernel launches the last lp_step issued (for reporting). */
 int lp_last_step_launches(lp_handle h);
 /* Device bytes owned by the handle. */

@@ -59,7 +59,8 @@ class lp_tensor_info(C.Structure):
 EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "lp_num_tensors",
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
-           "lp_last_error", "lp_gemm_bf16"]
+           "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read"]
+LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
 
 def load_library() -> C.CDLL:
@@ -220,6 +221,20 @@ def lp_save_state(h, host_array: np.ndarray):
 
 def lp_load_state(h, host_array: np.ndarray):
     _check(h, _lib.lp_load_state(h, host_array.ctypes.data, host_array.nbytes))
+
+
+def lp_profile_enable(h, on: bool):
+    _lib.lp_profile_enable.argtypes = [C.c_void_p, C.c_int]
+    _check(h, _lib.lp_profile_enable(h, 1 if on else 0))
+
+
+def lp_profile_read(h) -> dict:
+    """{class name: (milliseconds, algorithmic work, launches)} accumulated since the last read."""
+    n = len(LP_KIND_NAMES)
+    ms, work, launches = (C.c_double * n)(), (C.c_double * n)(), (C.c_int * n)()
+    _lib.lp_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int)]
+    _check(h, _lib.lp_profile_read(h, ms, work, launches))
+    return {LP_KIND_NAMES[i]: (ms[i], work[i], launches[i]) for i in range(n)}
 
 
 def lp_last_step_launches(h) -> int:

@@ -126,7 +126,7 @@ lp_status copy_inputs(Handle& h, const void* x, const void* y, cudaMemcpyKind ki
 }
 
 lp_status run_step(Handle& h, int schedule, cudaStream_t s) {
-  RunCtx ctx{s, nullptr};
+  RunCtx ctx{s, nullptr, h.profiling ? &h.prof : nullptr};
   int launches = 0;
   if (schedule == LP_SYNC) {
     if (h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
@@ -450,6 +450,30 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream,
     launch_gemm_simt(dp, simt.data(), (int)simt.size(), true, s);
   }
   return check_cuda(nullptr, "lp_gemm_bf16");
+}
+
+lp_status lp_profile_enable(lp_handle hh, int on) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  hh->h.profiling = on != 0;
+  return LP_OK;
+}
+
+lp_status lp_profile_read(lp_handle hh, double* ms, double* work, int* launches) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!ms || !work || !launches) return fail(&h, LP_ERR_INVALID_ARG, "null output");
+  cudaDeviceSynchronize();
+  for (int k = 0; k < LP_KIND_COUNT; ++k) { ms[k] = 0; work[k] = 0; launches[k] = 0; }
+  for (auto& r : h.prof) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.e0, r.e1) == cudaSuccess && r.kind >= 0 && r.kind < LP_KIND_COUNT) {
+      ms[r.kind] += t; work[r.kind] += r.work; launches[r.kind] += r.launches;
+    }
+    cudaEventDestroy(r.e0);
+    cudaEventDestroy(r.e1);
+  }
+  h.prof.clear();
+  return check_cuda(&h, "lp_profile_read");
 }
 
 int lp_last_step_launches(lp_handle hh) { return hh ? hh->h.last_launches : 0; }

@@ -123,7 +123,7 @@ void build_lm(Handle& h) {
     for (int k : ks)
       if (k == 0) {
         EmbedProb e{(const int*)h.x_in, h.W("c0.tok"), h.W("c0.pos"), cb[0].emb, M, T, d, V};
-        p.add(1, [e, st, bf](const RunCtx& c) { launch_embed_fwd(e, st, bf, c.stream); });
+        p.add(1, [e, st, bf](const RunCtx& c) { launch_embed_fwd(e, st, bf, c.stream); }, KIND_EMBED, 3.0 * M * d * es);
       }
     size_t maxb = 0;
     for (int k : ks) maxb = std::max(maxb, cb[k].blocks.size());
@@ -144,7 +144,8 @@ void build_lm(Handle& h) {
       {
         const AttnProb* dp = h.upload(at);
         int n = (int)at.size();
-        p.add(1, [=](const RunCtx& c) { launch_attn_fwd(dp, n, B, T, H, bf, c.stream); });
+        p.add(1, [=](const RunCtx& c) { launch_attn_fwd(dp, n, B, T, H, bf, c.stream); }, KIND_ATTN,
+              (double)n * 4.0 * B * H * 64.0 * T * (T + 1) / 2);
       }
       g.clear(); ln.clear();
       for (int k : act) {
@@ -294,7 +295,8 @@ void build_lm(Handle& h) {
         }
         const AttnProb* dp = h.upload(at);
         int n = (int)at.size();
-        p.add(2, [=](const RunCtx& c) { launch_attn_bwd(dp, n, B, T, H, bf, c.stream); });
+        p.add(2, [=](const RunCtx& c) { launch_attn_bwd(dp, n, B, T, H, bf, c.stream); }, KIND_ATTN,
+              (double)n * 10.0 * B * H * 64.0 * T * (T + 1) / 2);
       }
       // 6. qkv projection: dWqkv, dbqkv, da1 -> G1 (needed for LN1's own parameters in every case)
       for (int k : act) {
@@ -325,7 +327,7 @@ void build_lm(Handle& h) {
       for (int k : act)
         if (k == 0 && BJ(k) == 0) {
           EmbedBwdProb e{(const int*)h.x_in, cb[0].G0, h.G("c0.tok"), h.G("c0.pos"), emb_next, emb_first, M, T, d, V, B};
-          p.add(5, [e, bf](const RunCtx& c) { launch_embed_bwd(e, bf, c.stream); });
+          p.add(5, [e, bf](const RunCtx& c) { launch_embed_bwd(e, bf, c.stream); }, KIND_EMBED, (double)M * d * es + 4.0 * V * d);
         }
     }
     emit_pending_reduce(h, p);

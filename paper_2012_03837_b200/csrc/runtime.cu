@@ -117,7 +117,9 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
     int n = (int)tc.size();
     int* st = h.d_status;
     int sms = h.num_sms;
-    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream); });
+    double fl = 0;
+    for (auto& g : tc) fl += 2.0 * g.M * g.N * g.K;
+    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream); }, KIND_GEMM_TC, fl);
   }
   if (!simt.empty()) {
     int t = 0;
@@ -129,7 +131,9 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
     const GemmProb* d = h.upload(simt);
     bool bf = h.bf16_mode;
     int n = (int)simt.size();
-    p.add(1, [d, simt, n, bf](const RunCtx& c) { launch_gemm_simt(d, simt.data(), n, bf, c.stream); });
+    double fl = 0;
+    for (auto& g : simt) fl += 2.0 * g.M * g.N * g.K;
+    p.add(1, [d, simt, n, bf](const RunCtx& c) { launch_gemm_simt(d, simt.data(), n, bf, c.stream); }, KIND_GEMM_ALU, fl);
   }
 }
 
@@ -140,7 +144,9 @@ void emit_ln_fwd(Handle& h, Plan& p, const std::vector<LnProb>& probs) {
   const LnProb* d = h.upload(probs);
   int n = (int)probs.size();
   bool bf = h.bf16_mode;
-  p.add(1, [=](const RunCtx& c) { launch_ln_fwd(d, n, mr, bf, c.stream); });
+  double by = 0;
+  for (auto& q : probs) by += 2.0 * q.rows * q.d * h.esize();
+  p.add(1, [=](const RunCtx& c) { launch_ln_fwd(d, n, mr, bf, c.stream); }, KIND_NORM, by);
 }
 
 void emit_ln_bwd(Handle& h, Plan& p, std::vector<LnBwdProb> probs, const std::vector<float*>& dgamma,
@@ -158,7 +164,9 @@ void emit_ln_bwd(Handle& h, Plan& p, std::vector<LnBwdProb> probs, const std::ve
   const LnBwdProb* d = h.upload(probs);
   int n = (int)probs.size();
   bool bf = h.bf16_mode;
-  p.add(1, [=](const RunCtx& c) { launch_ln_bwd(d, n, mr, bf, c.stream); });
+  double by = 0;
+  for (auto& q : probs) by += (double)q.rows * q.d * h.esize() * (2 + (q.dx ? 1 : 0) + (q.dres ? 1 : 0));
+  p.add(1, [=](const RunCtx& c) { launch_ln_bwd(d, n, mr, bf, c.stream); }, KIND_NORM, by);
 }
 
 void emit_colsum(Handle& h, Plan& p, const std::vector<ColSumProb>& in, const std::vector<float*>& out) {
@@ -176,7 +184,9 @@ void emit_colsum(Handle& h, Plan& p, const std::vector<ColSumProb>& in, const st
   const ColSumProb* d = h.upload(probs);
   int n = (int)probs.size();
   bool bf = h.bf16_mode;
-  p.add(1, [=](const RunCtx& c) { launch_colsum_partial(d, n, mr, mc, bf, c.stream); });
+  double by = 0;
+  for (auto& q : probs) by += (double)q.rows * q.cols * h.esize();
+  p.add(1, [=](const RunCtx& c) { launch_colsum_partial(d, n, mr, mc, bf, c.stream); }, KIND_REDUCE, by);
 }
 
 void emit_pending_reduce(Handle& h, Plan& p) {
@@ -185,8 +195,10 @@ void emit_pending_reduce(Handle& h, Plan& p) {
   for (auto& q : h.pending_reduce) mc = std::max(mc, q.cols);
   const ColReduceProb* d = h.upload(h.pending_reduce);
   int n = (int)h.pending_reduce.size();
+  double by = 0;
+  for (auto& q : h.pending_reduce) by += (double)q.rows * q.cols * 4;
   h.pending_reduce.clear();
-  p.add(1, [=](const RunCtx& c) { launch_col_reduce_f32(d, n, mc, c.stream); });
+  p.add(1, [=](const RunCtx& c) { launch_col_reduce_f32(d, n, mc, c.stream); }, KIND_REDUCE, by);
 }
 
 void emit_labels(Handle& h, Plan& p, const std::vector<LabelProb>& probs) {
@@ -204,6 +216,8 @@ void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, 
     mr = std::max(mr, probs[i].rows);
     lps.push_back(LossProb{probs[i].row_loss, probs[i].n_valid, probs[i].rows, chunk_of[i]});
   }
+  double by = 0;
+  for (auto& q : probs) by += 2.0 * q.rows * q.classes * h.esize();
   const XentProb* d = h.upload(probs);
   const LossProb* dl = h.upload(lps);
   int n = (int)probs.size();
@@ -213,7 +227,7 @@ void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, 
   p.add(2, [=](const RunCtx& c) {
     launch_xent(d, n, mr, bf, c.stream);
     launch_loss_reduce(dl, n, losses, st, c.stream);
-  });
+  }, KIND_XENT, by);
 }
 
 void emit_optimizer(Handle& h, Plan& p) {
@@ -230,7 +244,7 @@ void emit_optimizer(Handle& h, Plan& p) {
     a.bc1 = (float)(1.0 - pow((double)hp->opt.beta1, t));
     a.bc2 = (float)(1.0 - pow((double)hp->opt.beta2, t));
     launch_optim(a, c.stream);
-  });
+  }, KIND_OPTIM, (double)h.n_total * (h.opt.kind == LP_OPT_ADAM ? 28.0 : 20.0) + (h.bf16_mode ? 2.0 * h.n_matrix : 0.0));
 }
 
 }  // namespace lp

@@ -20,16 +20,46 @@ struct TensorRec {
   int64_t off = 0;       // element offset in the arena
 };
 
+// Kernel classes for the optional per-class timing (lp_profile_*): values of LP_KIND_* in lp.h.
+enum { KIND_OTHER = 0, KIND_GEMM_TC = 1, KIND_GEMM_ALU = 2, KIND_NORM = 3, KIND_XENT = 4, KIND_ATTN = 5,
+       KIND_OPTIM = 6, KIND_REDUCE = 7, KIND_EMBED = 8, KIND_CONV_AUX = 9, KIND_COUNT = 10 };
+
+struct ProfRecord { int kind; int launches; double work; cudaEvent_t e0, e1; };
+
 struct RunCtx {
   cudaStream_t stream;
-  void* out_logits;      // lp_forward only
+  void* out_logits;                      // lp_forward only
+  std::vector<ProfRecord>* prof;         // non-null: bracket every op with events
+};
+
+struct PlanOp {
+  std::function<void(const RunCtx&)> fn;
+  int kind, launches;
+  double work;                           // algorithmic FLOPs (GEMM, attention) or bytes (the rest)
 };
 
 struct Plan {
-  std::vector<std::function<void(const RunCtx&)>> ops;
+  std::vector<PlanOp> ops;
   int launches = 0;
-  void add(int n_launches, std::function<void(const RunCtx&)> f) { ops.push_back(std::move(f)); launches += n_launches; }
-  void run(const RunCtx& c) const { for (auto& f : ops) f(c); }
+  void add(int n_launches, std::function<void(const RunCtx&)> f, int kind = KIND_OTHER, double work = 0) {
+    ops.push_back(PlanOp{std::move(f), kind, n_launches, work});
+    launches += n_launches;
+  }
+  void run(const RunCtx& c) const {
+    for (auto& op : ops) {
+      if (c.prof && op.launches > 0) {
+        ProfRecord r{op.kind, op.launches, op.work, nullptr, nullptr};
+        cudaEventCreate(&r.e0);
+        cudaEventCreate(&r.e1);
+        cudaEventRecord(r.e0, c.stream);
+        op.fn(c);
+        cudaEventRecord(r.e1, c.stream);
+        c.prof->push_back(r);
+      } else {
+        op.fn(c);
+      }
+    }
+  }
 };
 
 struct Handle {
@@ -71,6 +101,8 @@ struct Handle {
   bool primed = false;
   long long step_count = 0;
   int last_launches = 0;
+  bool profiling = false;
+  std::vector<ProfRecord> prof;
   std::string err;
 
   size_t esize() const { return bf16_mode ? 2 : 4; }
