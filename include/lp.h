@@ -206,6 +206,35 @@ typedef struct {
 lp_status lp_gemm_bf16(int n, const lp_gemm_desc* probs, int backend, void* stream, int* used_tensor_cores);
 
 /*
+ * lp_gemm_bf16_static: lp_gemm_bf16 for callers that cannot allocate device memory.  (The paper
+ * has no counterpart to this entry point; it exists for the library's users.)
+ *
+ * Who needs it: code that may not call cudaMalloc at the point where it launches work -- a thread
+ * recording a CUDA graph, a real-time or serving loop that must never take the driver's allocator
+ * lock, an embedding into a host whose device-memory budget was handed out up front.  lp_gemm_bf16
+ * keeps its problem table, its TMA tensor maps and its status word in a cudaMalloc'ed buffer that
+ * grows on demand; this variant keeps them in a fixed array that is part of the library image
+ * (about 41 KB of device memory on every GPU that loads the library, held until the process exits)
+ * and calls no cudaMalloc, cudaFree or any other allocating routine.
+ *
+ *   n: 1 .. LP_GEMM_STATIC_MAX problems; more is rejected with LP_ERR_SHAPE and nothing is launched.
+ *   probs: host array, same meaning as for lp_gemm_bf16 (device pointers inside).  Each problem runs
+ *     on the tensor-core kernel if its sizes allow, otherwise on the FP32-ALU kernel.
+ *   stream: the problems are uploaded and launched on this stream, asynchronously.
+ *
+ * The first call on a device looks up the array's device address (one-time set-up, with that
+ * device current); make that first call before any stream capture begins.  All calls on a device
+ * share the one array, which keeps the previous call's contents: each call clears the status word
+ * and overwrites the table entries it uses.  Two calls whose work may overlap on the GPU (different
+ * streams without an ordering between them) race on the array; calls on one stream are ordered.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED (device ordinal above 63), CUDA; the message is returned
+ * by lp_gemm_static_last_error().
+ */
+#define LP_GEMM_STATIC_MAX 64
+lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* probs, void* stream);
+const char* lp_gemm_static_last_error(void);
+
+/*
  * Per-kernel-class timing for benchmarks.  While enabled, every grouped launch of lp_step is
  * bracketed by a pair of CUDA events on the caller's stream.  lp_profile_read synchronises the
  * device and returns, for each class and summed over the steps since the last read: device

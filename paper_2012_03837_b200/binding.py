@@ -59,7 +59,8 @@ class lp_tensor_info(C.Structure):
 EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "lp_num_tensors",
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
-           "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read"]
+           "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
+           "lp_gemm_bf16_static", "lp_gemm_static_last_error"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
 
@@ -270,3 +271,23 @@ def lp_gemm_bf16(descs: list, backend: int = 0, stream=None) -> int:
     used = C.c_int(0)
     _check(None, _lib.lp_gemm_bf16(len(descs), arr, backend, stream, C.byref(used)))
     return used.value
+
+
+LP_GEMM_STATIC_MAX = 64
+_lib.lp_gemm_bf16_static.argtypes = [C.c_int, C.POINTER(lp_gemm_desc), C.c_void_p]
+_lib.lp_gemm_static_last_error.restype = C.c_char_p
+
+
+def lp_gemm_bf16_static(descs: list, stream=None) -> None:
+    """lp_gemm_bf16 for callers that must not allocate device memory (a thread recording a CUDA
+    graph, a serving loop that may not take the allocator lock): the problem table lives in a
+    fixed array inside the library, at most LP_GEMM_STATIC_MAX problems per call.  Same descriptor
+    dictionaries as lp_gemm_bf16.  Calls on one stream are ordered; calls that could overlap on
+    the GPU share that array and race."""
+    arr = (lp_gemm_desc * len(descs))()
+    for d, q in zip(arr, descs):
+        for k, v in q.items():
+            setattr(d, k, _ptr(v) if k in ("A", "B", "C", "C2", "bias", "resid", "aux") else int(v))
+    code = _lib.lp_gemm_bf16_static(len(descs), arr, stream)
+    if code != LP_OK:
+        raise LpError(code, (_lib.lp_gemm_static_last_error() or b"").decode())

@@ -19,6 +19,8 @@
 // No TMA load uses cluster multicast.
 #include <cuda.h>
 
+#include <cstdio>
+
 #include "common.cuh"
 #include "gemm_tc.h"
 
@@ -432,3 +434,111 @@ cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int npro
 }
 
 }  // namespace lp
+
+// ---------------------------------------------------------------------------------------------
+// lp_gemm_bf16_static: the grouped GEMM for callers that must not allocate device memory.
+//
+// The grouped kernels read their problem table (and, for the tensor-core kernel, two TMA tensor
+// maps per problem and a status word) from global memory.  lp_gemm_bf16 keeps that table in a
+// cudaMalloc'ed buffer that grows on demand.  Some callers cannot afford that: code that runs
+// while a CUDA graph is being captured or inside a memory-pool-managed region, real-time loops
+// that must not take the driver's allocation lock, and hosts whose memory budget is fixed up
+// front.  This variant keeps the table in the file-scope array below instead: a fixed
+// LP_GEMM_STATIC_MAX problems, about 41 KB that every GPU loading this library holds until the
+// process exits.
+// ---------------------------------------------------------------------------------------------
+#include "../../include/lp.h"
+
+namespace {
+using namespace lp;
+
+struct alignas(64) TMap { unsigned char b[128]; };
+struct StaticLayout {
+  int status;                                   // cleared at the start of every call
+  int pad[63];
+  GemmProb tc[LP_GEMM_STATIC_MAX];
+  GemmProb alu[LP_GEMM_STATIC_MAX];
+  alignas(64) TMap maps[2 * LP_GEMM_STATIC_MAX];
+};
+
+// In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticLayout)];
+
+constexpr int MAX_DEVICES = 64;
+StaticLayout* g_static_ptr[MAX_DEVICES] = {};
+int g_static_sms[MAX_DEVICES] = {};
+thread_local char g_static_err[256] = "";
+
+lp_status static_fail(lp_status code, const char* msg, cudaError_t e = cudaSuccess) {
+  if (e != cudaSuccess) snprintf(g_static_err, sizeof(g_static_err), "%s: %s", msg, cudaGetErrorString(e));
+  else snprintf(g_static_err, sizeof(g_static_err), "%s", msg);
+  return code;
+}
+}  // namespace
+
+extern "C" const char* lp_gemm_static_last_error(void) { return g_static_err; }
+
+extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* stream) {
+  if (n < 1 || !in) return static_fail(LP_ERR_INVALID_ARG, "lp_gemm_bf16_static: no problems");
+  if (n > LP_GEMM_STATIC_MAX) return static_fail(LP_ERR_SHAPE, "lp_gemm_bf16_static: more than LP_GEMM_STATIC_MAX (64) problems in one call");
+  cudaStream_t s = (cudaStream_t)stream;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "cudaGetDevice", e);
+  if (dev < 0 || dev >= MAX_DEVICES) return static_fail(LP_ERR_UNSUPPORTED, "lp_gemm_bf16_static: device ordinal above 63");
+  if (!g_static_ptr[dev]) {
+    // set-up, once per device, with that device current: resolve the array's device address
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess || !p) return static_fail(LP_ERR_CUDA, "cudaGetSymbolAddress", e);
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "cudaDeviceGetAttribute", e);
+    g_static_sms[dev] = sms;
+    g_static_ptr[dev] = (StaticLayout*)p;
+  }
+  StaticLayout* sc = g_static_ptr[dev];
+
+  GemmProb tc[LP_GEMM_STATIC_MAX], alu[LP_GEMM_STATIC_MAX];
+  TMap maps[2 * LP_GEMM_STATIC_MAX];
+  int ntc = 0, nalu = 0, tc_tiles = 0, alu_tiles = 0;
+  for (int i = 0; i < n; ++i) {
+    const lp_gemm_desc& q = in[i];
+    if (!q.A || !q.B || !q.C || q.M < 1 || q.N < 1 || q.K < 1) return static_fail(LP_ERR_INVALID_ARG, "lp_gemm_bf16_static: bad problem");
+    if ((q.a_ms != 1 && q.a_ks != 1) || (q.b_ns != 1 && q.b_ks != 1))
+      return static_fail(LP_ERR_INVALID_ARG, "lp_gemm_bf16_static: one stride per operand must be 1");
+    GemmProb g{};
+    g.A = q.A; g.B = q.B; g.C = q.C; g.C2 = q.C2; g.bias = q.bias; g.resid = q.resid; g.aux = q.aux;
+    g.M = q.M; g.N = q.N; g.K = q.K; g.a_ms = q.a_ms; g.a_ks = q.a_ks; g.b_ns = q.b_ns; g.b_ks = q.b_ks;
+    g.ldc = q.ldc; g.act = q.act; g.out_f32 = q.out_f32;
+    if (gemm_tc_eligible(g)) {
+      tc_tiles += gemm_tc_tiles(g, tc_tiles);
+      if (!gemm_tc_encode(g, &maps[2 * ntc], &maps[2 * ntc + 1])) return static_fail(LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+      tc[ntc++] = g;
+    } else {
+      g.tiles_n = (g.N + 63) / 64;
+      g.tile_start = alu_tiles;
+      alu_tiles += ((g.M + 63) / 64) * g.tiles_n;
+      alu[nalu++] = g;
+    }
+  }
+  // The array keeps whatever the previous call left: the status word must start at zero, the
+  // tables are overwritten for the entries this call uses.  Copies from pageable host memory are
+  // staged before cudaMemcpyAsync returns, so the stack arrays above may go out of scope.
+  e = cudaMemsetAsync(&sc->status, 0, sizeof(int), s);
+  if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "cudaMemsetAsync", e);
+  if (ntc) {
+    e = cudaMemcpyAsync(sc->tc, tc, ntc * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sc->maps, maps, 2 * ntc * sizeof(TMap), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = launch_gemm_tc(sc->tc, sc->maps, ntc, tc_tiles, &sc->status, g_static_sms[dev], s);
+    if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "tensor-core launch", e);
+  }
+  if (nalu) {
+    e = cudaMemcpyAsync(sc->alu, alu, nalu * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "cudaMemcpyAsync", e);
+    launch_gemm_simt(sc->alu, alu, nalu, true, s);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "FP32-ALU launch", e);
+  }
+  return LP_OK;
+}
