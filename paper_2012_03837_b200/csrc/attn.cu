@@ -1,8 +1,9 @@
 // Causal multi-head softmax attention (App. B.2's transformer layers), heads of 64, forward and
 // backward, flash-style: keys/values are streamed through shared memory in tiles of 64 with an
 // online softmax, the T x T score matrix is never stored; backward recomputes the probabilities
-// from Q, K and the saved log-sum-exp.  FP32-ALU version: one thread per query row (forward, dQ),
-// two threads per key row (dK, dV).  All sums run in a fixed order (no atomics).
+// from Q, K and the saved log-sum-exp.  FP32-ALU version for fp32 activations: one thread per query
+// row (forward, dQ), two threads per key row (dK, dV).  All sums run in a fixed order (no atomics).
+// bf16 activations take the tensor-core kernels of attn_tc.cu.
 //
 // qkv is [B*T, 3*H*64]: columns [0, d) queries, [d, 2d) keys, [2d, 3d) values, head h at h*64.
 #include "common.cuh"
@@ -199,19 +200,15 @@ __global__ void __launch_bounds__(128) attn_bwd_dkv_kernel(const AttnProb* __res
 
 void launch_attn_fwd(const AttnProb* d, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s) {
   dim3 grid((maxT + TILE - 1) / TILE, maxB * maxH, n);
-  if (is_bf16) attn_fwd_kernel<bf16><<<grid, 64, 0, s>>>(d);
-  else attn_fwd_kernel<float><<<grid, 64, 0, s>>>(d);
+  if (is_bf16) { launch_attn_fwd_tc(d, n, maxB, maxT, maxH, s); return; }
+  attn_fwd_kernel<float><<<grid, 64, 0, s>>>(d);
 }
 
 void launch_attn_bwd(const AttnProb* d, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s) {
   dim3 grid((maxT + TILE - 1) / TILE, maxB * maxH, n);
-  if (is_bf16) {
-    attn_bwd_dq_kernel<bf16><<<grid, 64, 0, s>>>(d);
-    attn_bwd_dkv_kernel<bf16><<<grid, 128, 0, s>>>(d);
-  } else {
-    attn_bwd_dq_kernel<float><<<grid, 64, 0, s>>>(d);
-    attn_bwd_dkv_kernel<float><<<grid, 128, 0, s>>>(d);
-  }
+  if (is_bf16) { launch_attn_bwd_tc(d, n, maxB, maxT, maxH, s); return; }
+  attn_bwd_dq_kernel<float><<<grid, 64, 0, s>>>(d);
+  attn_bwd_dkv_kernel<float><<<grid, 128, 0, s>>>(d);
 }
 
 }  // namespace lp

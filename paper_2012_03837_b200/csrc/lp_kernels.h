@@ -97,6 +97,8 @@ struct AttnProb {     // causal attention over qkv [B*T, 3d], heads of 64
 };
 void launch_attn_fwd(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s);
 void launch_attn_bwd(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s);
+void launch_attn_fwd_tc(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, cudaStream_t s);
+void launch_attn_bwd_tc(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, cudaStream_t s);
 
 // ---------------------------------------------------------------------------- ResNet-specific
 struct LayoutProb { const void* in; void* out; int N, C, H, W; };
