@@ -81,6 +81,11 @@ struct XentProb {     // softmax cross-entropy rows (App. A.1): z [rows, ld] -> 
 };
 void launch_xent(const XentProb* d_probs, int n, int max_rows, bool is_bf16, cudaStream_t s);
 
+// 128-bit vectorised bf16 variants (rowwise_vec.cu); nv = compile-time vectors per lane / thread.
+void launch_ln_fwd_vec(const LnProb* d_probs, int n, int max_rows, int nv, cudaStream_t s);
+void launch_ln_bwd_vec(const LnBwdProb* d_probs, int n, int max_rows, int nv, cudaStream_t s);
+void launch_xent_vec(const XentProb* d_probs, int n, int max_rows, int nv, cudaStream_t s);
+
 struct LossProb { const float* row_loss; const int* n_valid; int rows; int out_index; };
 void launch_loss_reduce(const LossProb* d_probs, int n, float* d_losses, int* d_status, cudaStream_t s);
 

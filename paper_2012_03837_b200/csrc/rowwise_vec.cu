@@ -1,0 +1,244 @@
+// 128-bit vectorised bf16 versions of the HBM-bound row kernels (LayerNorm forward/backward,
+// softmax cross-entropy with in-place dlogits).  Each row is read from HBM exactly once and kept in
+// registers; outputs are written once.  Used when every row is 16-byte aligned and its length fits
+// the register budget; otherwise the generic kernels of rowwise.cu run.  Fixed reduction orders.
+#include "common.cuh"
+
+namespace lp {
+namespace {
+
+__device__ __forceinline__ void unpack8(const uint4& u, float* f) {
+  const __nv_bfloat162* h = (const __nv_bfloat162*)&u;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) { float2 v = __bfloat1622float2(h[t]); f[2 * t] = v.x; f[2 * t + 1] = v.y; }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  uint4 u;
+  __nv_bfloat162* h = (__nv_bfloat162*)&u;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(f[2 * t], f[2 * t + 1]);
+  return u;
+}
+
+// ------------------------------------------------------------------ LayerNorm forward
+// Warp per row; lane owns the 8-element vectors j*32 + lane, j < NV (d = NV * 256).
+template <int NV>
+__global__ void __launch_bounds__(256) ln_fwd_vec_kernel(const LnProb* __restrict__ probs) {
+  const LnProb p = probs[blockIdx.y];
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  int row = blockIdx.x * 8 + w;
+  if (row >= p.rows) return;
+  const uint4* x = (const uint4*)((const bf16*)p.x + (size_t)row * p.d);
+  float v[NV][8];
+  float s = 0.f;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    unpack8(x[j * 32 + lane], v[j]);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) s += v[j][t];
+  }
+  float mu = warp_sum(s) / p.d;
+  float q = 0.f;
+#pragma unroll
+  for (int j = 0; j < NV; ++j)
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { float c = v[j][t] - mu; q += c * c; }
+  float rstd = rsqrtf(warp_sum(q) / p.d + 1e-5f);
+  uint4* y = (uint4*)((bf16*)p.y + (size_t)row * p.d);
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int c0 = (j * 32 + lane) * 8;
+    float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
+    float4 b0 = *(const float4*)(p.b + c0), b1 = *(const float4*)(p.b + c0 + 4);
+    float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+    float o[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) o[t] = (v[j][t] - mu) * rstd * g[t] + b[t];
+    y[j * 32 + lane] = pack8(o);
+  }
+  if (lane == 0) { p.mean[row] = mu; p.rstd[row] = rstd; }
+}
+
+// ------------------------------------------------------------------ LayerNorm backward
+// Block = 8 warps over LN_BWD_ROWS rows (warp w takes rows w, w+8, ...).  Each lane accumulates
+// the scale/shift gradient of its own columns over the warp's rows in registers; the 8 warps are
+// then summed through shared memory in warp order and the block writes one partial row.
+template <int NV>
+__global__ void __launch_bounds__(256) ln_bwd_vec_kernel(const LnBwdProb* __restrict__ probs) {
+  extern __shared__ float red[];   // [8][2][d]
+  const LnBwdProb p = probs[blockIdx.y];
+  int r0 = blockIdx.x * LN_BWD_ROWS;
+  if (r0 >= p.rows) return;
+  int r1 = min(r0 + LN_BWD_ROWS, p.rows);
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  float ag[NV][8], ab[NV][8], g[NV][8];
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int c0 = (j * 32 + lane) * 8;
+    float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
+    g[j][0] = g0.x; g[j][1] = g0.y; g[j][2] = g0.z; g[j][3] = g0.w;
+    g[j][4] = g1.x; g[j][5] = g1.y; g[j][6] = g1.z; g[j][7] = g1.w;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { ag[j][t] = 0.f; ab[j][t] = 0.f; }
+  }
+  for (int row = r0 + w; row < r1; row += 8) {
+    const uint4* dy = (const uint4*)((const bf16*)p.dy + (size_t)row * p.d);
+    const uint4* x = (const uint4*)((const bf16*)p.x + (size_t)row * p.d);
+    float mu = p.mean[row], rs = p.rstd[row];
+    float xh[NV][8], dv[NV][8];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      unpack8(x[j * 32 + lane], xh[j]);
+      unpack8(dy[j * 32 + lane], dv[j]);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        xh[j][t] = (xh[j][t] - mu) * rs;
+        ag[j][t] += dv[j][t] * xh[j][t];
+        ab[j][t] += dv[j][t];
+        float dxh = dv[j][t] * g[j][t];
+        s1 += dxh;
+        s2 += dxh * xh[j][t];
+      }
+    }
+    if (p.dx) {
+      s1 = warp_sum(s1) / p.d;
+      s2 = warp_sum(s2) / p.d;
+      uint4* dx = (uint4*)((bf16*)p.dx + (size_t)row * p.d);
+      const uint4* dres = p.dres ? (const uint4*)((const bf16*)p.dres + (size_t)row * p.d) : nullptr;
+#pragma unroll
+      for (int j = 0; j < NV; ++j) {
+        float o[8], r[8];
+        if (dres) unpack8(dres[j * 32 + lane], r);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          o[t] = rs * (dv[j][t] * g[j][t] - s1 - xh[j][t] * s2);
+          if (dres) o[t] += r[t];
+        }
+        dx[j * 32 + lane] = pack8(o);
+      }
+    }
+  }
+  const int d = p.d;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int c0 = (j * 32 + lane) * 8;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      red[(w * 2 + 0) * d + c0 + t] = ag[j][t];
+      red[(w * 2 + 1) * d + c0 + t] = ab[j][t];
+    }
+  }
+  __syncthreads();
+  float* part = p.part + (size_t)blockIdx.x * 2 * d;
+  for (int c = threadIdx.x; c < 2 * d; c += blockDim.x) {
+    float s = 0.f;
+#pragma unroll
+    for (int ww = 0; ww < 8; ++ww) s += red[ww * 2 * d + c];
+    part[c] = s;
+  }
+}
+
+// ------------------------------------------------------------------ softmax cross-entropy
+// Block (NT threads) per row; thread owns vectors j*NT + tid, j < NV.  Long rows use 1024 threads
+// with few vectors each, so that two blocks fit an SM and one block's loads overlap the other's math.
+template <int NV, int NT>
+__global__ void __launch_bounds__(NT) xent_vec_kernel(const XentProb* __restrict__ probs) {
+  __shared__ float red[33];
+  const XentProb p = probs[blockIdx.y];
+  int row = blockIdx.x;
+  if (row >= p.rows) return;
+  uint4* z = (uint4*)((bf16*)p.z + (size_t)row * p.ld);
+  const int nvec = p.classes >> 3;
+  int y = p.y[row];
+  bool valid = (y >= 0 && y < p.classes);
+  if (!valid) {
+    for (int i = threadIdx.x; i < nvec; i += NT) z[i] = make_uint4(0, 0, 0, 0);
+    if (threadIdx.x == 0) p.row_loss[row] = 0.f;
+    return;
+  }
+  uint4 raw[NV];
+  float m = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int i = j * NT + threadIdx.x;
+    if (i < nvec) {
+      raw[j] = z[i];
+      float f[8];
+      unpack8(raw[j], f);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) m = fmaxf(m, f[t]);
+    }
+  }
+  float M = block_max(m, red);
+  float s = 0.f;
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int i = j * NT + threadIdx.x;
+    if (i < nvec) {
+      float f[8];
+      unpack8(raw[j], f);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) s += __expf(f[t] - M);
+    }
+  }
+  float S = block_sum(s, red);
+  float lse = M + logf(S);
+  float inv = 1.0f / (float)(*p.n_valid);
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int i = j * NT + threadIdx.x;
+    if (i < nvec) {
+      float f[8], o[8];
+      unpack8(raw[j], f);
+      int c0 = i * 8;
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        if (c0 + t == y) p.row_loss[row] = lse - f[t];
+        o[t] = (__expf(f[t] - lse) - (c0 + t == y ? 1.f : 0.f)) * inv;
+      }
+      z[i] = pack8(o);
+    }
+  }
+}
+
+}  // namespace
+
+// d must equal nv*256 with nv in {1, 2, 4}; rows, scale and shift 16-byte aligned.
+void launch_ln_fwd_vec(const LnProb* d, int n, int max_rows, int nv, cudaStream_t s) {
+  dim3 grid((max_rows + 7) / 8, n);
+  switch (nv) {
+    case 1: ln_fwd_vec_kernel<1><<<grid, 256, 0, s>>>(d); break;
+    case 2: ln_fwd_vec_kernel<2><<<grid, 256, 0, s>>>(d); break;
+    default: ln_fwd_vec_kernel<4><<<grid, 256, 0, s>>>(d); break;
+  }
+}
+void launch_ln_bwd_vec(const LnBwdProb* d, int n, int max_rows, int nv, cudaStream_t s) {
+  dim3 grid((max_rows + LN_BWD_ROWS - 1) / LN_BWD_ROWS, n);
+  size_t smem = (size_t)8 * 2 * nv * 256 * sizeof(float);
+  static bool set = false;
+  if (!set) {
+    cudaFuncSetAttribute(ln_bwd_vec_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 2 * 4 * 256 * 4);
+    set = true;
+  }
+  switch (nv) {
+    case 1: ln_bwd_vec_kernel<1><<<grid, 256, smem, s>>>(d); break;
+    case 2: ln_bwd_vec_kernel<2><<<grid, 256, smem, s>>>(d); break;
+    default: ln_bwd_vec_kernel<4><<<grid, 256, smem, s>>>(d); break;
+  }
+}
+// classes and ld multiples of 8, z 16-byte aligned, classes <= nv*2048, nv in {1,2,4,8,16}
+// (nv*2048 elements are covered either by 256 threads x nv vectors or by 1024 threads x nv/4).
+void launch_xent_vec(const XentProb* d, int n, int max_rows, int nv, cudaStream_t s) {
+  dim3 grid(max_rows, n);
+  switch (nv) {
+    case 1: xent_vec_kernel<1, 256><<<grid, 256, 0, s>>>(d); break;
+    case 2: xent_vec_kernel<2, 256><<<grid, 256, 0, s>>>(d); break;
+    case 4: xent_vec_kernel<1, 1024><<<grid, 1024, 0, s>>>(d); break;
+    case 8: xent_vec_kernel<2, 1024><<<grid, 1024, 0, s>>>(d); break;
+    default: xent_vec_kernel<4, 1024><<<grid, 1024, 0, s>>>(d); break;
+  }
+}
+
+}  // namespace lp

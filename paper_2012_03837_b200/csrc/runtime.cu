@@ -137,6 +137,12 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
   }
 }
 
+// Vectors per lane for the register-resident LayerNorm kernels (rows of 256, 512 or 1024 bf16), else 0.
+static int ln_vec_width(const Handle& h, int d) {
+  if (!h.bf16_mode) return 0;
+  return d == 256 ? 1 : d == 512 ? 2 : d == 1024 ? 4 : 0;
+}
+
 void emit_ln_fwd(Handle& h, Plan& p, const std::vector<LnProb>& probs) {
   if (probs.empty()) return;
   int mr = 0;
@@ -146,7 +152,10 @@ void emit_ln_fwd(Handle& h, Plan& p, const std::vector<LnProb>& probs) {
   bool bf = h.bf16_mode;
   double by = 0;
   for (auto& q : probs) by += 2.0 * q.rows * q.d * h.esize();
-  p.add(1, [=](const RunCtx& c) { launch_ln_fwd(d, n, mr, bf, c.stream); }, KIND_NORM, by);
+  int nv = ln_vec_width(h, probs[0].d);
+  for (auto& q : probs) if (q.d != probs[0].d) nv = 0;
+  if (nv) p.add(1, [=](const RunCtx& c) { launch_ln_fwd_vec(d, n, mr, nv, c.stream); }, KIND_NORM, by);
+  else p.add(1, [=](const RunCtx& c) { launch_ln_fwd(d, n, mr, bf, c.stream); }, KIND_NORM, by);
 }
 
 void emit_ln_bwd(Handle& h, Plan& p, std::vector<LnBwdProb> probs, const std::vector<float*>& dgamma,
@@ -166,7 +175,10 @@ void emit_ln_bwd(Handle& h, Plan& p, std::vector<LnBwdProb> probs, const std::ve
   bool bf = h.bf16_mode;
   double by = 0;
   for (auto& q : probs) by += (double)q.rows * q.d * h.esize() * (2 + (q.dx ? 1 : 0) + (q.dres ? 1 : 0));
-  p.add(1, [=](const RunCtx& c) { launch_ln_bwd(d, n, mr, bf, c.stream); }, KIND_NORM, by);
+  int nv = ln_vec_width(h, probs[0].d);
+  for (auto& q : probs) if (q.d != probs[0].d) nv = 0;
+  if (nv) p.add(1, [=](const RunCtx& c) { launch_ln_bwd_vec(d, n, mr, nv, c.stream); }, KIND_NORM, by);
+  else p.add(1, [=](const RunCtx& c) { launch_ln_bwd(d, n, mr, bf, c.stream); }, KIND_NORM, by);
 }
 
 void emit_colsum(Handle& h, Plan& p, const std::vector<ColSumProb>& in, const std::vector<float*>& out) {
@@ -224,8 +236,16 @@ void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, 
   bool bf = h.bf16_mode;
   float* losses = h.d_losses;
   int* st = h.d_status;
+  int nv = 0;
+  if (bf && probs[0].classes % 8 == 0 && probs[0].classes <= 32768) {
+    nv = 1;
+    while (nv * 2048 < probs[0].classes) nv *= 2;
+    for (auto& q : probs)
+      if (q.classes != probs[0].classes || q.ld % 8 != 0 || ((uintptr_t)q.z & 15)) nv = 0;
+  }
   p.add(2, [=](const RunCtx& c) {
-    launch_xent(d, n, mr, bf, c.stream);
+    if (nv) launch_xent_vec(d, n, mr, nv, c.stream);
+    else launch_xent(d, n, mr, bf, c.stream);
     launch_loss_reduce(dl, n, losses, st, c.stream);
   }, KIND_XENT, by);
 }

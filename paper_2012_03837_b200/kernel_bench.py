@@ -1,0 +1,83 @@
+"""Micro-benchmark of the grouped bf16 GEMM through the C ABI (lp_gemm_bf16): the Linear-layer
+products of the transformer workloads in forward, input-gradient and weight-gradient form.
+
+    python -m paper_2012_03837_b200.kernel_bench [--shape qkv|out|ffn1|ffn2|head|all] [--form fwd|dgrad|wgrad|all]
+                                                 [--d 1024] [--rows 8192] [--vocab 32768] [--groups 4] [--reps 10]
+
+Prints one JSON line per (shape, form): milliseconds per launch and TFLOP/s (2*M*N*K per problem).
+Inputs are larger than the L2 cache in total, so every launch streams its operands from HBM.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as lp
+
+
+def shapes(d, ffn, vocab):
+    return {"qkv": (3 * d, d), "out": (d, d), "ffn1": (ffn, d), "ffn2": (d, ffn), "head": (vocab, d)}
+
+
+def descs(form, rows, n_out, n_in, groups):
+    """`groups` independent Linear layers y = x W^T with x [rows, n_in], W [n_out, n_in]."""
+    out, keep = [], []
+    bf = dict(dtype=torch.bfloat16, device="cuda")
+    for _ in range(groups):
+        x = torch.randn(rows, n_in, **bf)
+        W = torch.randn(n_out, n_in, **bf) * 0.02
+        dy = torch.randn(rows, n_out, **bf)
+        if form == "fwd":
+            c = torch.empty(rows, n_out, **bf)
+            out.append(dict(A=x, B=W, C=c, M=rows, N=n_out, K=n_in, a_ms=n_in, a_ks=1, b_ns=n_in, b_ks=1, ldc=n_out))
+        elif form == "dgrad":
+            c = torch.empty(rows, n_in, **bf)
+            out.append(dict(A=dy, B=W, C=c, M=rows, N=n_in, K=n_out, a_ms=n_out, a_ks=1, b_ns=1, b_ks=n_in, ldc=n_in))
+        else:
+            c = torch.empty(n_out, n_in, dtype=torch.float32, device="cuda")
+            out.append(dict(A=dy, B=x, C=c, M=n_out, N=n_in, K=rows, a_ms=1, a_ks=n_out, b_ns=1, b_ks=n_in, ldc=n_in, out_f32=1))
+        keep += [x, W, dy, c]
+    return out, keep
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--shape", default="all")
+    ap.add_argument("--form", default="all")
+    ap.add_argument("--d", type=int, default=1024)
+    ap.add_argument("--rows", type=int, default=8192)
+    ap.add_argument("--vocab", type=int, default=32768)
+    ap.add_argument("--groups", type=int, default=4)
+    ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--backend", type=int, default=0)
+    a = ap.parse_args()
+    sh = shapes(a.d, 4 * a.d, a.vocab)
+    names = list(sh) if a.shape == "all" else [a.shape]
+    forms = ["fwd", "dgrad", "wgrad"] if a.form == "all" else [a.form]
+    stream = torch.cuda.current_stream().cuda_stream
+    for name in names:
+        n_out, n_in = sh[name]
+        groups = max(1, a.groups // 4) if name == "head" else a.groups
+        for form in forms:
+            ds, keep = descs(form, a.rows, n_out, n_in, groups)
+            for _ in range(3):
+                used = lp.lp_gemm_bf16(ds, a.backend, stream)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(a.reps):
+                lp.lp_gemm_bf16(ds, a.backend, stream)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / a.reps
+            flops = 2.0 * a.rows * n_out * n_in * groups
+            print(json.dumps(dict(shape=name, form=form, rows=a.rows, n_out=n_out, n_in=n_in, groups=groups,
+                                  tensor_core_problems=used, ms_per_launch=ms, tflops=flops / ms / 1e9)))
+            del ds, keep
+            torch.cuda.empty_cache()
+
+
+if __name__ == "__main__":
+    main()

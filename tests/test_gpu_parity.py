@@ -77,6 +77,13 @@ def test_lm_bf16_small(backend):
     check(cfg, gemm_backend=backend)
 
 
+def test_lm_bf16_wide_rows_sync():
+    """d_model 256 and a vocabulary of 2056: the register-resident LayerNorm / cross-entropy kernels."""
+    cfg = lp_synth.config("c3", batch=2, seq_len=200, vocab=2056, d_model=256, n_heads=4, d_ffn=512,
+                          blocks_per_chunk=[2, 1], schedule="sync")
+    check(cfg)
+
+
 def test_sync_and_pipelined_agree_on_step0():
     cfg = lp_synth.config("c1")
     x, y = lp_synth.minibatch(cfg, 0)
