@@ -1,0 +1,418 @@
+// HBM-bound kernels around the convolution GEMMs of the ResNet family (App. B.3): layout change,
+// im2col / col2im (gather form, no atomics), train-mode BatchNorm (statistics, apply, backward) with
+// fp32 statistics, global average pool.  Activations are NHWC: [N*H*W, C] row-major, so a
+// convolution is the GEMM  y[M, C_out] = cols[M, kh*kw*C_in] * W[C_out, kh*kw*C_in]^T.
+// blockIdx.y selects the problem.  All reductions have a fixed order.
+#include "common.cuh"
+
+namespace lp {
+namespace {
+
+template <typename T>
+__global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(LayoutProb p) {
+  long long total = (long long)p.N * p.C * p.H * p.W;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    int c = (int)(i % p.C);
+    long long r = i / p.C;
+    int w = (int)(r % p.W); r /= p.W;
+    int h = (int)(r % p.H);
+    int n = (int)(r / p.H);
+    ((T*)p.out)[i] = ((const T*)p.in)[(((long long)n * p.C + c) * p.H + h) * p.W + w];
+  }
+}
+
+// cols[(n,ho,wo), (i*kw+j)*C + c] = x[n, ho*s+i-pad, wo*s+j-pad, c] (0 outside the image)
+template <typename T>
+__global__ void __launch_bounds__(256) im2col_kernel(const Im2colProb* __restrict__ probs) {
+  const Im2colProb p = probs[blockIdx.y];
+  const int K = p.kh * p.kw * p.C;
+  long long total = (long long)p.N * p.Ho * p.Wo * K;
+  const T* x = (const T*)p.x;
+  T* cols = (T*)p.cols;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    int kk = (int)(e % K);
+    long long m = e / K;
+    int c = kk % p.C, tap = kk / p.C;
+    int i = tap / p.kw, j = tap % p.kw;
+    int wo = (int)(m % p.Wo);
+    long long r = m / p.Wo;
+    int ho = (int)(r % p.Ho);
+    int n = (int)(r / p.Ho);
+    int h = ho * p.stride + i - p.pad, w = wo * p.stride + j - p.pad;
+    T v = from_f<T>(0.f);
+    if (h >= 0 && h < p.H && w >= 0 && w < p.W) v = x[(((long long)n * p.H + h) * p.W + w) * p.C + c];
+    cols[m * p.ldk + kk] = v;
+  }
+}
+
+// dx[n,h,w,c] = sum over taps (i,j) with h = ho*s+i-pad, w = wo*s+j-pad of dcols[(n,ho,wo), (i*kw+j)*C+c]
+template <typename T>
+__global__ void __launch_bounds__(256) col2im_kernel(const Im2colProb* __restrict__ probs) {
+  const Im2colProb p = probs[blockIdx.y];
+  long long total = (long long)p.N * p.H * p.W * p.C;
+  const T* cols = (const T*)p.cols;
+  T* dx = (T*)p.x;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    int c = (int)(e % p.C);
+    long long r = e / p.C;
+    int w = (int)(r % p.W); r /= p.W;
+    int h = (int)(r % p.H);
+    int n = (int)(r / p.H);
+    float s = 0.f;
+    for (int i = 0; i < p.kh; ++i) {
+      int hh = h + p.pad - i;
+      if (hh < 0 || hh % p.stride) continue;
+      int ho = hh / p.stride;
+      if (ho >= p.Ho) continue;
+      for (int j = 0; j < p.kw; ++j) {
+        int ww = w + p.pad - j;
+        if (ww < 0 || ww % p.stride) continue;
+        int wo = ww / p.stride;
+        if (wo >= p.Wo) continue;
+        long long m = ((long long)n * p.Ho + ho) * p.Wo + wo;
+        s += to_f(cols[m * p.ldk + (i * p.kw + j) * p.C + c]);
+      }
+    }
+    dx[e] = from_f<T>(s);
+  }
+}
+
+// Per-channel partial sums over a block of BN_ROWS rows.
+//   forward : part[blk][0][c] = sum x,   part[blk][1][c] = sum x^2
+//   backward: part[blk][0][c] = sum dyr * xhat, part[blk][1][c] = sum dyr, dyr = dy * [relu_out > 0]
+template <typename T, bool BWD>
+__global__ void __launch_bounds__(256) bn_stat_kernel(const BnStatProb* __restrict__ probs) {
+  const BnStatProb p = probs[blockIdx.z];
+  int r0 = blockIdx.y * BN_ROWS;
+  if (r0 >= p.rows) return;
+  int r1 = min(r0 + BN_ROWS, p.rows);
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= p.C) return;
+  const T* x = (const T*)p.x;
+  float a = 0.f, b = 0.f;
+  if (BWD) {
+    const T* dy = (const T*)p.dy;
+    const T* ro = (const T*)p.relu_out;
+    float mu = p.mean[c], rs = p.rstd[c];
+    for (int r = r0; r < r1; ++r) {
+      size_t off = (size_t)r * p.C + c;
+      float g = to_f(dy[off]);
+      if (ro && !(to_f(ro[off]) > 0.f)) g = 0.f;
+      a += g * (to_f(x[off]) - mu) * rs;
+      b += g;
+    }
+  } else {
+    for (int r = r0; r < r1; ++r) {
+      float v = to_f(x[(size_t)r * p.C + c]);
+      a += v;
+      b += v * v;
+    }
+  }
+  float* part = p.part + (size_t)blockIdx.y * 2 * p.C;
+  part[c] = a;
+  part[p.C + c] = b;
+}
+
+// forward: mean and 1/sqrt(biased variance + eps); backward: dgamma, dbeta.  One warp per channel:
+// lane l sums partial blocks l, l+32, ... in double, then a fixed shuffle tree combines the lanes.
+template <bool BWD>
+__global__ void __launch_bounds__(256) bn_finalize_kernel(const BnFinalProb* __restrict__ probs) {
+  const BnFinalProb p = probs[blockIdx.y];
+  int lane = threadIdx.x & 31;
+  int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (c >= p.C) return;
+  double a = 0.0, b = 0.0;
+  for (int k = lane; k < p.nblk; k += 32) {
+    a += (double)p.part[(size_t)k * 2 * p.C + c];
+    b += (double)p.part[(size_t)k * 2 * p.C + p.C + c];
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a += __shfl_xor_sync(0xffffffffu, a, o);
+    b += __shfl_xor_sync(0xffffffffu, b, o);
+  }
+  if (lane != 0) return;
+  if (BWD) {
+    p.dgamma[c] = (float)a;
+    p.dbeta[c] = (float)b;
+  } else {
+    double mu = a / p.rows;
+    double var = b / p.rows - mu * mu;
+    if (var < 0.0) var = 0.0;
+    p.mean[c] = (float)mu;
+    p.rstd[c] = (float)(1.0 / sqrt(var + (double)p.eps));
+  }
+}
+
+template <typename T, bool BWD>
+__global__ void __launch_bounds__(256) bn_apply_kernel(const BnApplyProb* __restrict__ probs) {
+  const BnApplyProb p = probs[blockIdx.y];
+  long long total = (long long)p.rows * p.C;
+  const T* x = (const T*)p.x;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    int c = (int)(e % p.C);
+    float xh = (to_f(x[e]) - p.mean[c]) * p.rstd[c];
+    if (!BWD) {
+      float v = xh * p.g[c] + p.b[c];
+      if (p.res) v += to_f(((const T*)p.res)[e]);
+      if (p.relu) v = fmaxf(v, 0.f);
+      ((T*)p.y)[e] = from_f<T>(v);
+    } else {
+      float g = to_f(((const T*)p.dy)[e]);
+      if (p.relu_out && !(to_f(((const T*)p.relu_out)[e]) > 0.f)) g = 0.f;
+      if (p.dres_out) ((T*)p.dres_out)[e] = from_f<T>(g);
+      float inv = 1.0f / (float)p.rows;
+      float v = p.rstd[c] * p.g[c] * (g - p.dbeta[c] * inv - xh * p.dgamma[c] * inv);
+      ((T*)p.dx)[e] = from_f<T>(v);
+    }
+  }
+}
+
+// y[n, c] = mean over hw of x[n, hw, c]
+template <typename T>
+__global__ void __launch_bounds__(256) gap_fwd_kernel(const GapProb* __restrict__ probs) {
+  const GapProb p = probs[blockIdx.z];
+  int n = blockIdx.y;
+  int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= p.N || c >= p.C) return;
+  const T* x = (const T*)p.x + (size_t)n * p.HW * p.C;
+  float s = 0.f;
+  for (int i = 0; i < p.HW; ++i) s += to_f(x[(size_t)i * p.C + c]);
+  ((T*)p.y)[(size_t)n * p.C + c] = from_f<T>(s / p.HW);
+}
+template <typename T>
+__global__ void __launch_bounds__(256) gap_bwd_kernel(const GapProb* __restrict__ probs) {
+  const GapProb p = probs[blockIdx.y];
+  long long total = (long long)p.N * p.HW * p.C;
+  float inv = 1.0f / p.HW;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    int c = (int)(e % p.C);
+    int n = (int)(e / ((long long)p.HW * p.C));
+    ((T*)p.dx)[e] = from_f<T>(to_f(((const T*)p.dy)[(size_t)n * p.C + c]) * inv);
+  }
+}
+
+// ------------------------------------------------------------------ 128-bit bf16 variants (C % 8 == 0)
+__device__ __forceinline__ void unpack8(const uint4& u, float* f) {
+  const __nv_bfloat162* h = (const __nv_bfloat162*)&u;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) { float2 v = __bfloat1622float2(h[t]); f[2 * t] = v.x; f[2 * t + 1] = v.y; }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+  uint4 u;
+  __nv_bfloat162* h = (__nv_bfloat162*)&u;
+#pragma unroll
+  for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(f[2 * t], f[2 * t + 1]);
+  return u;
+}
+
+__global__ void __launch_bounds__(256) im2col_vec_kernel(const Im2colProb* __restrict__ probs) {
+  const Im2colProb p = probs[blockIdx.y];
+  const int cv = p.C >> 3, taps = p.kh * p.kw;
+  long long total = (long long)p.N * p.Ho * p.Wo * taps * cv;
+  const bf16* x = (const bf16*)p.x;
+  bf16* cols = (bf16*)p.cols;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    int c8 = (int)(e % cv);
+    long long r = e / cv;
+    int tap = (int)(r % taps);
+    long long m = r / taps;
+    int i = tap / p.kw, j = tap % p.kw;
+    int wo = (int)(m % p.Wo);
+    long long q = m / p.Wo;
+    int ho = (int)(q % p.Ho);
+    int n = (int)(q / p.Ho);
+    int h = ho * p.stride + i - p.pad, w = wo * p.stride + j - p.pad;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (h >= 0 && h < p.H && w >= 0 && w < p.W) v = *(const uint4*)(x + (((long long)n * p.H + h) * p.W + w) * p.C + c8 * 8);
+    *(uint4*)(cols + m * p.ldk + tap * p.C + c8 * 8) = v;
+  }
+}
+
+__global__ void __launch_bounds__(256) col2im_vec_kernel(const Im2colProb* __restrict__ probs) {
+  const Im2colProb p = probs[blockIdx.y];
+  const int cv = p.C >> 3;
+  long long total = (long long)p.N * p.H * p.W * cv;
+  const bf16* cols = (const bf16*)p.cols;
+  bf16* dx = (bf16*)p.x;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    int c8 = (int)(e % cv);
+    long long r = e / cv;
+    int w = (int)(r % p.W); r /= p.W;
+    int h = (int)(r % p.H);
+    int n = (int)(r / p.H);
+    float s[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int i = 0; i < p.kh; ++i) {
+      int hh = h + p.pad - i;
+      if (hh < 0 || hh % p.stride) continue;
+      int ho = hh / p.stride;
+      if (ho >= p.Ho) continue;
+      for (int j = 0; j < p.kw; ++j) {
+        int ww = w + p.pad - j;
+        if (ww < 0 || ww % p.stride) continue;
+        int wo = ww / p.stride;
+        if (wo >= p.Wo) continue;
+        long long m = ((long long)n * p.Ho + ho) * p.Wo + wo;
+        float f[8];
+        unpack8(*(const uint4*)(cols + m * p.ldk + (i * p.kw + j) * p.C + c8 * 8), f);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) s[t] += f[t];
+      }
+    }
+    *(uint4*)(dx + e * 8) = pack8(s);
+  }
+}
+
+// Block of 256 threads = (C/8 channel vectors) x (256 / (C/8) row lanes) over BN_ROWS rows; the row
+// lanes are summed through shared memory in lane order.  Requires C % 8 == 0 and C/8 <= 256.
+template <bool BWD>
+__global__ void __launch_bounds__(256) bn_stat_vec_kernel(const BnStatProb* __restrict__ probs) {
+  __shared__ float red[256 * 16];
+  const BnStatProb p = probs[blockIdx.z];
+  int r0 = blockIdx.y * BN_ROWS;
+  if (r0 >= p.rows) return;
+  int r1 = min(r0 + BN_ROWS, p.rows);
+  const int cv = p.C >> 3, ny = 256 / cv;
+  const int tx = threadIdx.x % cv, ty = threadIdx.x / cv;
+  float a[8], b[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) { a[t] = 0.f; b[t] = 0.f; }
+  if (ty < ny) {
+    const bf16* x = (const bf16*)p.x;
+    float mu[8], rs[8];
+    if (BWD) {
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { mu[t] = p.mean[tx * 8 + t]; rs[t] = p.rstd[tx * 8 + t]; }
+    }
+    for (int r = r0 + ty; r < r1; r += ny) {
+      size_t off = (size_t)r * p.C + tx * 8;
+      float xv[8];
+      unpack8(*(const uint4*)(x + off), xv);
+      if (BWD) {
+        float g[8];
+        unpack8(*(const uint4*)((const bf16*)p.dy + off), g);
+        if (p.relu_out) {
+          float ro[8];
+          unpack8(*(const uint4*)((const bf16*)p.relu_out + off), ro);
+#pragma unroll
+          for (int t = 0; t < 8; ++t) if (!(ro[t] > 0.f)) g[t] = 0.f;
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) { a[t] += g[t] * (xv[t] - mu[t]) * rs[t]; b[t] += g[t]; }
+      } else {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) { a[t] += xv[t]; b[t] += xv[t] * xv[t]; }
+      }
+    }
+  }
+#pragma unroll
+  for (int t = 0; t < 8; ++t) { red[threadIdx.x * 16 + t] = a[t]; red[threadIdx.x * 16 + 8 + t] = b[t]; }
+  __syncthreads();
+  // thread (c, which) sums lane 0..ny-1 for channel c
+  for (int idx = threadIdx.x; idx < 2 * p.C; idx += 256) {
+    int which = idx / p.C, c = idx % p.C;
+    float s = 0.f;
+    for (int l = 0; l < ny; ++l) s += red[(l * cv + (c >> 3)) * 16 + which * 8 + (c & 7)];
+    p.part[(size_t)blockIdx.y * 2 * p.C + which * p.C + c] = s;
+  }
+}
+
+template <bool BWD>
+__global__ void __launch_bounds__(256) bn_apply_vec_kernel(const BnApplyProb* __restrict__ probs) {
+  const BnApplyProb p = probs[blockIdx.y];
+  const int cv = p.C >> 3;
+  long long total = (long long)p.rows * cv;
+  const bf16* x = (const bf16*)p.x;
+  const float inv = 1.0f / (float)p.rows;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    int c0 = (int)(e % cv) * 8;
+    float xv[8], o[8];
+    unpack8(*(const uint4*)(x + e * 8), xv);
+    if (!BWD) {
+      float r[8];
+      if (p.res) unpack8(*(const uint4*)((const bf16*)p.res + e * 8), r);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        float v = (xv[t] - p.mean[c0 + t]) * p.rstd[c0 + t] * p.g[c0 + t] + p.b[c0 + t];
+        if (p.res) v += r[t];
+        o[t] = p.relu ? fmaxf(v, 0.f) : v;
+      }
+      *(uint4*)((bf16*)p.y + e * 8) = pack8(o);
+    } else {
+      float g[8];
+      unpack8(*(const uint4*)((const bf16*)p.dy + e * 8), g);
+      if (p.relu_out) {
+        float ro[8];
+        unpack8(*(const uint4*)((const bf16*)p.relu_out + e * 8), ro);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) if (!(ro[t] > 0.f)) g[t] = 0.f;
+      }
+      if (p.dres_out) *(uint4*)((bf16*)p.dres_out + e * 8) = pack8(g);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) {
+        float xh = (xv[t] - p.mean[c0 + t]) * p.rstd[c0 + t];
+        o[t] = p.rstd[c0 + t] * p.g[c0 + t] * (g[t] - p.dbeta[c0 + t] * inv - xh * p.dgamma[c0 + t] * inv);
+      }
+      *(uint4*)((bf16*)p.dx + e * 8) = pack8(o);
+    }
+  }
+}
+
+unsigned grid_for(long long elems) {
+  long long b = (elems + 255) / 256;
+  long long cap = 148LL * 32;
+  return (unsigned)(b < 1 ? 1 : (b > cap ? cap : b));
+}
+
+}  // namespace
+
+void launch_nchw_to_nhwc(const LayoutProb& p, bool is_bf16, cudaStream_t s) {
+  unsigned g = grid_for((long long)p.N * p.C * p.H * p.W);
+  if (is_bf16) nchw_to_nhwc_kernel<bf16><<<g, 256, 0, s>>>(p);
+  else nchw_to_nhwc_kernel<float><<<g, 256, 0, s>>>(p);
+}
+void launch_im2col(const Im2colProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8) {
+  dim3 grid(grid_for(vec8 ? max_elems / 8 : max_elems), n);
+  if (vec8) im2col_vec_kernel<<<grid, 256, 0, s>>>(d);
+  else if (is_bf16) im2col_kernel<bf16><<<grid, 256, 0, s>>>(d);
+  else im2col_kernel<float><<<grid, 256, 0, s>>>(d);
+}
+void launch_col2im(const Im2colProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8) {
+  dim3 grid(grid_for(vec8 ? max_elems / 8 : max_elems), n);
+  if (vec8) col2im_vec_kernel<<<grid, 256, 0, s>>>(d);
+  else if (is_bf16) col2im_kernel<bf16><<<grid, 256, 0, s>>>(d);
+  else col2im_kernel<float><<<grid, 256, 0, s>>>(d);
+}
+void launch_bn_stat_partial(const BnStatProb* d, int n, int max_rows, int max_c, bool bwd, bool is_bf16, cudaStream_t s,
+                            bool vec8) {
+  dim3 grid((max_c + 255) / 256, (max_rows + BN_ROWS - 1) / BN_ROWS, n);
+  if (vec8) {
+    grid.x = 1;
+    if (bwd) bn_stat_vec_kernel<true><<<grid, 256, 0, s>>>(d); else bn_stat_vec_kernel<false><<<grid, 256, 0, s>>>(d);
+  } else if (is_bf16) { if (bwd) bn_stat_kernel<bf16, true><<<grid, 256, 0, s>>>(d); else bn_stat_kernel<bf16, false><<<grid, 256, 0, s>>>(d); }
+  else { if (bwd) bn_stat_kernel<float, true><<<grid, 256, 0, s>>>(d); else bn_stat_kernel<float, false><<<grid, 256, 0, s>>>(d); }
+}
+void launch_bn_finalize(const BnFinalProb* d, int n, int max_c, bool bwd, cudaStream_t s) {
+  dim3 grid((max_c + 7) / 8, n);
+  if (bwd) bn_finalize_kernel<true><<<grid, 256, 0, s>>>(d);
+  else bn_finalize_kernel<false><<<grid, 256, 0, s>>>(d);
+}
+void launch_bn_apply(const BnApplyProb* d, int n, long long max_elems, bool bwd, bool is_bf16, cudaStream_t s, bool vec8) {
+  dim3 grid(grid_for(vec8 ? max_elems / 8 : max_elems), n);
+  if (vec8) {
+    if (bwd) bn_apply_vec_kernel<true><<<grid, 256, 0, s>>>(d); else bn_apply_vec_kernel<false><<<grid, 256, 0, s>>>(d);
+  } else if (is_bf16) { if (bwd) bn_apply_kernel<bf16, true><<<grid, 256, 0, s>>>(d); else bn_apply_kernel<bf16, false><<<grid, 256, 0, s>>>(d); }
+  else { if (bwd) bn_apply_kernel<float, true><<<grid, 256, 0, s>>>(d); else bn_apply_kernel<float, false><<<grid, 256, 0, s>>>(d); }
+}
+void launch_gap_fwd(const GapProb* d, int n, int max_n, int max_c, bool is_bf16, cudaStream_t s) {
+  dim3 grid((max_c + 255) / 256, max_n, n);
+  if (is_bf16) gap_fwd_kernel<bf16><<<grid, 256, 0, s>>>(d);
+  else gap_fwd_kernel<float><<<grid, 256, 0, s>>>(d);
+}
+void launch_gap_bwd(const GapProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s) {
+  dim3 grid(grid_for(max_elems), n);
+  if (is_bf16) gap_bwd_kernel<bf16><<<grid, 256, 0, s>>>(d);
+  else gap_bwd_kernel<float><<<grid, 256, 0, s>>>(d);
+}
+
+}  // namespace lp

@@ -112,9 +112,10 @@ void launch_nchw_to_nhwc(const LayoutProb& p, bool is_bf16, cudaStream_t s);
 struct Im2colProb {   // x NHWC [N,H,W,C] -> cols [N*Ho*Wo, ldk], column (i*kw + j)*C + c, zero padded
   const void* x; void* cols; int N, H, W, C, kh, kw, stride, pad, Ho, Wo, ldk;
 };
-void launch_im2col(const Im2colProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
+// vec8: bf16 with channel counts that are multiples of 8 (128-bit accesses)
+void launch_im2col(const Im2colProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8 = false);
 // dx[n,h,w,c] = sum over the filter taps that read this pixel of dcols (gather form: no atomics)
-void launch_col2im(const Im2colProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
+void launch_col2im(const Im2colProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8 = false);
 
 struct BnStatProb {   // per-channel partial sums of x and x^2 (fwd) or of dy and dy*xhat (bwd)
   const void* x; const void* dy; const float* mean; const float* rstd; const void* relu_out;
@@ -122,7 +123,7 @@ struct BnStatProb {   // per-channel partial sums of x and x^2 (fwd) or of dy an
 };
 enum { BN_ROWS = 256 };
 void launch_bn_stat_partial(const BnStatProb* d_probs, int n, int max_rows, int max_c, bool bwd, bool is_bf16,
-                            cudaStream_t s);
+                            cudaStream_t s, bool vec8 = false);
 struct BnFinalProb {  // fwd: sums -> mean, rstd.  part is [nblk, 2, C]
   const float* part; int nblk; int rows; int C; float* mean; float* rstd; float* dgamma; float* dbeta; float eps;
 };
@@ -135,7 +136,7 @@ struct BnApplyProb {
   const void* dy; const void* relu_out; void* dx; void* dres_out; const float* dgamma; const float* dbeta;
   int rows, C, relu;
 };
-void launch_bn_apply(const BnApplyProb* d_probs, int n, long long max_elems, bool bwd, bool is_bf16, cudaStream_t s);
+void launch_bn_apply(const BnApplyProb* d_probs, int n, long long max_elems, bool bwd, bool is_bf16, cudaStream_t s, bool vec8 = false);
 
 struct GapProb { const void* x; void* y; const void* dy; void* dx; int N, HW, C; };
 void launch_gap_fwd(const GapProb* d_probs, int n, int max_n, int max_c, bool is_bf16, cudaStream_t s);

@@ -1,8 +1,362 @@
-// ResNet family (App. B.3): not built yet in this file; lp_create reports LP_ERR_UNSUPPORTED.
+// ResNet family (App. B.3): a 3x3 stem convolution + BatchNorm + ReLU in chunk 0, then one stage of
+// BasicBlocks per chunk (conv3x3-BN-ReLU-conv3x3-BN, identity or 1x1-stride-2 conv+BN shortcut, ReLU),
+// BatchNorm with batch statistics, and a global-average-pool + Linear + softmax cross-entropy
+// auxiliary head per chunk (Sec. 3).  Activations are NHWC; a convolution is im2col + GEMM
+// (cols are kept for the weight gradient), its input gradient a GEMM + col2im gather.
+//
+// Backward is truncated at the chunk input (Sec. 3): the first block of a stage k > 0 forms no input
+// gradient (no dgrad for its first convolution and its shortcut convolution), nor does the stem.
+// The synchronous schedule is the natural one here; the pipelined plans are built too.
 #include <stdexcept>
 
 #include "runtime.h"
 
 namespace lp {
-void build_resnet(Handle&) { throw std::runtime_error("unsupported: the RESNET family is not implemented yet"); }
+namespace {
+
+struct Conv {
+  std::string w;
+  int Cin, Cout, k, stride, pad, H, W, Ho, Wo, N;
+  long long M;   // N*Ho*Wo
+  int K;         // k*k*Cin
+  int ldk;       // pitch of the cols matrix: K rounded up to 8 elements (16 bytes for bf16), pad columns stay zero
+  void* cols = nullptr;
+  void* y = nullptr;
+};
+struct Bn {
+  std::string g, b;
+  int C;
+  long long rows;
+  float *mean, *rstd;
+};
+struct Block {
+  Conv c1, c2, cs;
+  Bn b1, b2, bs;
+  bool has_sc = false;
+  void *a1 = nullptr, *sc = nullptr, *out = nullptr;   // out is null for the chunk's last block (boundary buffer)
+};
+struct Chunk {
+  bool has_stem = false;
+  Conv stem;
+  Bn stem_bn;
+  void *x_nhwc = nullptr, *stem_out = nullptr;
+  std::vector<Block> blocks;
+  int C, Hout, Wout;
+  void *pool, *z, *dpool;
+  float* row_loss;
+  void* G[4];
+  void* dcols;
+};
+
+Conv make_conv(const std::string& w, int N, int H, int W, int Cin, int Cout, int k, int stride) {
+  Conv c;
+  c.w = w; c.N = N; c.H = H; c.W = W; c.Cin = Cin; c.Cout = Cout; c.k = k; c.stride = stride; c.pad = k / 2;
+  c.Ho = (H + 2 * c.pad - k) / stride + 1;
+  c.Wo = (W + 2 * c.pad - k) / stride + 1;
+  c.M = (long long)N * c.Ho * c.Wo;
+  c.K = k * k * Cin;
+  c.ldk = (c.K + 7) / 8 * 8;
+  return c;
+}
+
+}  // namespace
+
+void build_resnet(Handle& h) {
+  const int K = h.K, B = h.spec.batch, NC = h.head.classes;
+  const bool bf = h.bf16_mode;
+  const size_t es = h.esize();
+  std::vector<Chunk> ch(K);
+  int H = h.spec.height, W = h.spec.width, cprev = h.spec.stem_channels;
+  for (int k = 0; k < K; ++k) {
+    Chunk& c = ch[k];
+    const std::string ck = "c" + std::to_string(k);
+    if (k == 0) {
+      c.has_stem = true;
+      c.stem = make_conv("c0.stem.conv", B, H, W, h.spec.in_channels, cprev, 3, 1);
+      h.add_tensor("c0.stem.conv", 0, {cprev, 3, 3, h.spec.in_channels}, true);
+      h.add_tensor("c0.stem.bn.g", 0, {cprev}, false);
+      h.add_tensor("c0.stem.bn.b", 0, {cprev}, false);
+      c.stem_bn = Bn{"c0.stem.bn.g", "c0.stem.bn.b", cprev, c.stem.M, nullptr, nullptr};
+    }
+    int cout = h.stage_channels[k];
+    for (int j = 0; j < h.spec.blocks_per_stage; ++j) {
+      Block b;
+      const std::string p = ck + ".r" + std::to_string(j);
+      int stride = (j == 0 && k > 0) ? 2 : 1;
+      int cin = j == 0 ? cprev : cout;
+      b.c1 = make_conv(p + ".conv1", B, H, W, cin, cout, 3, stride);
+      h.add_tensor(p + ".conv1", k, {cout, 3, 3, cin}, true);
+      h.add_tensor(p + ".bn1.g", k, {cout}, false);
+      h.add_tensor(p + ".bn1.b", k, {cout}, false);
+      b.b1 = Bn{p + ".bn1.g", p + ".bn1.b", cout, b.c1.M, nullptr, nullptr};
+      b.c2 = make_conv(p + ".conv2", B, b.c1.Ho, b.c1.Wo, cout, cout, 3, 1);
+      h.add_tensor(p + ".conv2", k, {cout, 3, 3, cout}, true);
+      h.add_tensor(p + ".bn2.g", k, {cout}, false);
+      h.add_tensor(p + ".bn2.b", k, {cout}, false);
+      b.b2 = Bn{p + ".bn2.g", p + ".bn2.b", cout, b.c2.M, nullptr, nullptr};
+      b.has_sc = j == 0 && (stride != 1 || cin != cout);
+      if (b.has_sc) {
+        b.cs = make_conv(p + ".sc.conv", B, H, W, cin, cout, 1, stride);
+        h.add_tensor(p + ".sc.conv", k, {cout, 1, 1, cin}, true);
+        h.add_tensor(p + ".sc.bn.g", k, {cout}, false);
+        h.add_tensor(p + ".sc.bn.b", k, {cout}, false);
+        b.bs = Bn{p + ".sc.bn.g", p + ".sc.bn.b", cout, b.cs.M, nullptr, nullptr};
+      }
+      H = b.c1.Ho; W = b.c1.Wo;
+      c.blocks.push_back(b);
+    }
+    cprev = cout;
+    c.C = cout; c.Hout = H; c.Wout = W;
+    h.add_tensor(ck + ".head.W", k, {NC, cout}, true);
+    h.add_tensor(ck + ".head.b", k, {NC}, false);
+  }
+  h.finalize_arena();
+  h.rows = B;
+
+  // ---- buffers
+  const size_t in_elems = (size_t)B * h.spec.in_channels * h.spec.height * h.spec.width;
+  h.x_bytes = in_elems * es;
+  h.x_in = h.dalloc(h.x_bytes);
+  h.y_bytes = (size_t)B * sizeof(int);
+  h.y_in = (int*)h.dalloc(h.y_bytes);
+  auto fal = [&](size_t n) { return (float*)h.dalloc(n * sizeof(float)); };
+  auto alloc_conv = [&](Conv& c) {
+    c.cols = h.dalloc((size_t)c.M * c.ldk * es);
+    c.y = h.dalloc((size_t)c.M * c.Cout * es);
+  };
+  auto alloc_bn = [&](Bn& b) { b.mean = fal(b.C); b.rstd = fal(b.C); };
+  for (int k = 0; k < K; ++k) {
+    Chunk& c = ch[k];
+    size_t out_bytes = (size_t)B * c.Hout * c.Wout * c.C * es;
+    h.bnd_bytes.push_back(out_bytes);
+    for (int s = 0; s < 2; ++s) {
+      h.bnd[s].push_back(h.dalloc(out_bytes));
+      h.lab[s].push_back((int*)h.dalloc(h.y_bytes));
+    }
+    h.n_valid.push_back((int*)h.dalloc(sizeof(int)));
+    size_t max_act = 0, max_cols = 0;
+    auto track = [&](const Conv& cv) {
+      max_act = std::max(max_act, (size_t)cv.M * cv.Cout);
+      max_act = std::max(max_act, (size_t)cv.N * cv.H * cv.W * cv.Cin);
+      max_cols = std::max(max_cols, (size_t)cv.M * cv.ldk);
+    };
+    if (c.has_stem) {
+      c.x_nhwc = h.dalloc(in_elems * es);
+      alloc_conv(c.stem); alloc_bn(c.stem_bn); track(c.stem);
+      c.stem_out = h.dalloc((size_t)c.stem.M * c.stem.Cout * es);
+    }
+    for (size_t j = 0; j < c.blocks.size(); ++j) {
+      Block& b = c.blocks[j];
+      alloc_conv(b.c1); alloc_bn(b.b1); track(b.c1);
+      alloc_conv(b.c2); alloc_bn(b.b2); track(b.c2);
+      b.a1 = h.dalloc((size_t)b.c1.M * b.c1.Cout * es);
+      if (b.has_sc) { alloc_conv(b.cs); alloc_bn(b.bs); track(b.cs); b.sc = h.dalloc((size_t)b.cs.M * b.cs.Cout * es); }
+      if (j + 1 < c.blocks.size()) b.out = h.dalloc((size_t)b.c2.M * b.c2.Cout * es);
+    }
+    c.pool = h.dalloc((size_t)B * c.C * es);
+    c.dpool = h.dalloc((size_t)B * c.C * es);
+    c.z = h.dalloc((size_t)B * NC * es);
+    c.row_loss = fal(B);
+    for (int i = 0; i < 4; ++i) c.G[i] = h.dalloc(max_act * es);
+    c.dcols = h.dalloc(max_cols * es);
+  }
+
+  // ---- op emitters (one problem per launch: the stages differ in every size)
+  auto conv_fwd = [&](Plan& p, const Conv& c, const void* x) {
+    Im2colProb ip{x, c.cols, c.N, c.H, c.W, c.Cin, c.k, c.k, c.stride, c.pad, c.Ho, c.Wo, c.ldk};
+    const Im2colProb* d = h.upload(std::vector<Im2colProb>{ip});
+    long long elems = c.M * c.K;
+    bool v8 = bf && c.Cin % 8 == 0;
+    p.add(1, [=](const RunCtx& r) { launch_im2col(d, 1, elems, bf, r.stream, v8); }, KIND_CONV_AUX, (double)elems * es * (1.0 + 1.0 / (c.k * c.k)));
+    GemmProb g = gemm_fwd(c.cols, h.W(c.w), c.y, (int)c.M, c.Cout, c.K, nullptr, EPI_NONE);
+    g.a_ms = c.ldk;
+    emit_gemm(h, p, {g});
+  };
+  auto conv_wgrad = [&](Plan& p, const Conv& c, const void* dy) {
+    GemmProb g = gemm_wgrad(dy, c.cols, h.G(c.w), (int)c.M, c.Cout, c.K);
+    g.b_ks = c.ldk;
+    emit_gemm(h, p, {g});
+  };
+  auto conv_dgrad = [&](Plan& p, const Conv& c, const void* dy, void* dx, void* dcols) {
+    GemmProb g = gemm_dgrad(dy, h.W(c.w), dcols, (int)c.M, c.Cout, c.K, EPI_NONE, nullptr);
+    g.ldc = c.ldk;
+    emit_gemm(h, p, {g});
+    Im2colProb ip{dx, dcols, c.N, c.H, c.W, c.Cin, c.k, c.k, c.stride, c.pad, c.Ho, c.Wo, c.ldk};
+    const Im2colProb* d = h.upload(std::vector<Im2colProb>{ip});
+    long long elems = (long long)c.N * c.H * c.W * c.Cin;
+    bool v8 = bf && c.Cin % 8 == 0;
+    p.add(1, [=](const RunCtx& r) { launch_col2im(d, 1, elems, bf, r.stream, v8); }, KIND_CONV_AUX, (double)(elems + c.M * c.K) * es);
+  };
+  auto bn_fwd = [&](Plan& p, const Bn& b, const void* x, void* y, const void* res, bool relu) {
+    int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
+    float* part = fal((size_t)nblk * 2 * b.C);
+    BnStatProb sp{x, nullptr, nullptr, nullptr, nullptr, part, (int)b.rows, b.C};
+    BnFinalProb fp{part, nblk, (int)b.rows, b.C, b.mean, b.rstd, nullptr, nullptr, 1e-5f};
+    BnApplyProb ap{x, y, res, h.P32(b.g), h.P32(b.b), b.mean, b.rstd, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                   (int)b.rows, b.C, relu ? 1 : 0};
+    const BnStatProb* ds = h.upload(std::vector<BnStatProb>{sp});
+    const BnFinalProb* df = h.upload(std::vector<BnFinalProb>{fp});
+    const BnApplyProb* da = h.upload(std::vector<BnApplyProb>{ap});
+    int rows = (int)b.rows, C = b.C;
+    bool v8 = bf && C % 8 == 0 && C / 8 <= 256;
+    long long elems = b.rows * b.C;
+    p.add(3, [=](const RunCtx& r) {
+      launch_bn_stat_partial(ds, 1, rows, C, false, bf, r.stream, v8);
+      launch_bn_finalize(df, 1, C, false, r.stream);
+      launch_bn_apply(da, 1, elems, false, bf, r.stream, v8);
+    }, KIND_NORM, (double)elems * es * (3 + (res ? 1 : 0)));
+  };
+  // dx = BN'(dy masked by relu_out > 0); dres (optional) receives the masked dy
+  auto bn_bwd = [&](Plan& p, const Bn& b, const void* x, const void* dy, const void* relu_out, void* dx, void* dres) {
+    int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
+    float* part = fal((size_t)nblk * 2 * b.C);
+    BnStatProb sp{x, dy, b.mean, b.rstd, relu_out, part, (int)b.rows, b.C};
+    BnFinalProb fp{part, nblk, (int)b.rows, b.C, nullptr, nullptr, h.G(b.g), h.G(b.b), 1e-5f};
+    BnApplyProb ap{x, nullptr, nullptr, h.P32(b.g), h.P32(b.b), b.mean, b.rstd, dy, relu_out, dx, dres, h.G(b.g), h.G(b.b),
+                   (int)b.rows, b.C, 0};
+    const BnStatProb* ds = h.upload(std::vector<BnStatProb>{sp});
+    const BnFinalProb* df = h.upload(std::vector<BnFinalProb>{fp});
+    const BnApplyProb* da = h.upload(std::vector<BnApplyProb>{ap});
+    int rows = (int)b.rows, C = b.C;
+    bool v8 = bf && C % 8 == 0 && C / 8 <= 256;
+    long long elems = b.rows * b.C;
+    p.add(3, [=](const RunCtx& r) {
+      launch_bn_stat_partial(ds, 1, rows, C, true, bf, r.stream, v8);
+      launch_bn_finalize(df, 1, C, true, r.stream);
+      launch_bn_apply(da, 1, elems, true, bf, r.stream, v8);
+    }, KIND_NORM, (double)elems * es * (5 + (relu_out ? 2 : 0) + (dres ? 1 : 0)));
+  };
+  auto add_into = [&](Plan& p, void* acc, const void* other, long long n) {
+    const AddProb* d = h.upload(std::vector<AddProb>{AddProb{acc, other, acc, n}});
+    p.add(1, [=](const RunCtx& r) { launch_add(d, 1, n, bf, r.stream); }, KIND_CONV_AUX, 3.0 * n * es);
+  };
+
+  auto chunk_in = [&](int k, int rd) -> const void* { return k == 0 ? ch[0].stem_out : h.bnd[rd][k - 1]; };
+  auto labels_of = [&](int k, bool pipelined, int rd) -> const int* {
+    return (!pipelined || k == 0) ? h.y_in : h.lab[rd][k - 1];
+  };
+
+  auto forward_chunk = [&](Plan& p, int k, int rd, int wr) {
+    Chunk& c = ch[k];
+    if (c.has_stem) {
+      LayoutProb lp{h.x_in, c.x_nhwc, B, h.spec.in_channels, h.spec.height, h.spec.width};
+      p.add(1, [=](const RunCtx& r) { launch_nchw_to_nhwc(lp, bf, r.stream); }, KIND_CONV_AUX, 2.0 * in_elems * es);
+      conv_fwd(p, c.stem, c.x_nhwc);
+      bn_fwd(p, c.stem_bn, c.stem.y, c.stem_out, nullptr, true);
+    }
+    const void* x = chunk_in(k, rd);
+    for (size_t j = 0; j < c.blocks.size(); ++j) {
+      Block& b = c.blocks[j];
+      void* out = b.out ? b.out : h.bnd[wr][k];
+      conv_fwd(p, b.c1, x);
+      bn_fwd(p, b.b1, b.c1.y, b.a1, nullptr, true);
+      conv_fwd(p, b.c2, b.a1);
+      const void* res = x;
+      if (b.has_sc) {
+        conv_fwd(p, b.cs, x);
+        bn_fwd(p, b.bs, b.cs.y, b.sc, nullptr, false);
+        res = b.sc;
+      }
+      bn_fwd(p, b.b2, b.c2.y, out, res, true);
+      x = out;
+    }
+  };
+
+  auto head_forward = [&](Plan& p, int k, int wr, const int* labels, bool copy_logits) {
+    Chunk& c = ch[k];
+    const std::string ck = "c" + std::to_string(k);
+    GapProb gp{h.bnd[wr][k], c.pool, nullptr, nullptr, B, c.Hout * c.Wout, c.C};
+    const GapProb* dg = h.upload(std::vector<GapProb>{gp});
+    int C = c.C;
+    p.add(1, [=](const RunCtx& r) { launch_gap_fwd(dg, 1, B, C, bf, r.stream); }, KIND_CONV_AUX, (double)B * c.Hout * c.Wout * c.C * es);
+    emit_gemm(h, p, {gemm_fwd(c.pool, h.W(ck + ".head.W"), c.z, B, NC, c.C, h.P32(ck + ".head.b"), EPI_NONE)});
+    if (copy_logits && k == K - 1) {
+      void* zlast = c.z;
+      size_t zbytes = (size_t)B * NC * es;
+      p.add(0, [zlast, zbytes](const RunCtx& r) {
+        if (r.out_logits) cudaMemcpyAsync(r.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, r.stream);
+      });
+    }
+    emit_xent_and_loss(h, p, {XentProb{c.z, labels, h.n_valid[k], c.row_loss, B, NC, NC}}, {k});
+  };
+
+  auto backward_chunk = [&](Plan& p, int k, int rd, int wr) {
+    Chunk& c = ch[k];
+    const std::string ck = "c" + std::to_string(k);
+    // head: dW_h, db_h, d(pool), then the pool's gradient spread over H*W -> G[0]
+    emit_gemm(h, p, {gemm_wgrad(c.z, c.pool, h.G(ck + ".head.W"), B, NC, c.C),
+                     gemm_dgrad(c.z, h.W(ck + ".head.W"), c.dpool, B, NC, c.C, EPI_NONE, nullptr)});
+    emit_colsum(h, p, {ColSumProb{c.z, nullptr, B, NC, NC}}, {h.G(ck + ".head.b")});
+    {
+      GapProb gp{nullptr, nullptr, c.dpool, c.G[0], B, c.Hout * c.Wout, c.C};
+      const GapProb* dg = h.upload(std::vector<GapProb>{gp});
+      long long elems = (long long)B * c.Hout * c.Wout * c.C;
+      p.add(1, [=](const RunCtx& r) { launch_gap_bwd(dg, 1, elems, bf, r.stream); }, KIND_CONV_AUX, (double)elems * es);
+    }
+    void *gin = c.G[0], *ga = c.G[1], *gb = c.G[2], *gc = c.G[3];
+    for (int j = (int)c.blocks.size() - 1; j >= 0; --j) {
+      Block& b = c.blocks[j];
+      const void* x = j == 0 ? chunk_in(k, rd) : c.blocks[j - 1].out;
+      const void* out = b.out ? b.out : h.bnd[wr][k];
+      bool need_dx = (j > 0) || c.has_stem;
+      // out = relu(bn2(c2) + shortcut): ga <- d(c2), gb <- gradient of the shortcut branch
+      bn_bwd(p, b.b2, b.c2.y, gin, out, ga, gb);
+      conv_wgrad(p, b.c2, ga);
+      conv_dgrad(p, b.c2, ga, gc, c.dcols);                 // gc <- d(a1)
+      bn_bwd(p, b.b1, b.c1.y, gc, b.a1, ga, nullptr);       // ga <- d(c1)
+      conv_wgrad(p, b.c1, ga);
+      long long in_elems_blk = (long long)b.c1.N * b.c1.H * b.c1.W * b.c1.Cin;
+      if (need_dx) conv_dgrad(p, b.c1, ga, gc, c.dcols);    // gc <- d(x) through the main branch
+      if (b.has_sc) {
+        bn_bwd(p, b.bs, b.cs.y, gb, nullptr, ga, nullptr);  // ga <- d(cs)
+        conv_wgrad(p, b.cs, ga);
+        if (need_dx) {
+          conv_dgrad(p, b.cs, ga, gin, c.dcols);            // gin <- d(x) through the shortcut
+          add_into(p, gc, gin, in_elems_blk);
+        }
+      } else if (need_dx) {
+        add_into(p, gc, gb, in_elems_blk);
+      }
+      std::swap(gin, gc);                                   // the block-input gradient feeds the next (earlier) block
+    }
+    if (c.has_stem) {
+      bn_bwd(p, c.stem_bn, c.stem.y, gin, c.stem_out, ga, nullptr);
+      conv_wgrad(p, c.stem, ga);
+    }
+  };
+
+  std::vector<int> all;
+  for (int k = 0; k < K; ++k) all.push_back(k);
+
+  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr) {
+    std::vector<LabelProb> lps;
+    for (int k = 0; k < K; ++k)
+      lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, B, NC, h.n_valid[k]});
+    emit_labels(h, p, lps);
+    for (int k = 0; k < K; ++k) forward_chunk(p, k, rd, wr);
+    for (int k = 0; k < K; ++k) head_forward(p, k, wr, labels_of(k, pipelined, rd), false);
+    for (int k = 0; k < K; ++k) backward_chunk(p, k, rd, wr);
+    emit_pending_reduce(h, p);
+    emit_optimizer(h, p);
+  };
+  auto build_forward = [&](Plan& p, int wr, bool heads) {
+    for (int k = 0; k < K; ++k) forward_chunk(p, k, wr, wr);
+    if (!heads) return;
+    std::vector<LabelProb> lps;
+    for (int k = 0; k < K; ++k) lps.push_back(LabelProb{h.y_in, nullptr, B, NC, h.n_valid[k]});
+    emit_labels(h, p, lps);
+    for (int k = 0; k < K; ++k) head_forward(p, k, wr, h.y_in, true);
+  };
+
+  build_step(h.sync_plan, false, 0, 0);
+  for (int par = 0; par < 2; ++par) {
+    build_step(h.pipe_plan[par], true, par, 1 - par);
+    build_forward(h.prime_plan[par], par, false);
+    std::vector<LabelProb> lps;
+    for (int k = 0; k + 1 < K; ++k) lps.push_back(LabelProb{h.y_in, h.lab[par][k], B, NC, h.n_valid[k]});
+    if (!lps.empty()) emit_labels(h, h.prime_plan[par], lps);
+    build_forward(h.fwd_plan[par], par, true);
+  }
+}
+
 }  // namespace lp

@@ -99,6 +99,35 @@ GemmProb gemm_wgrad(const void* dy, const void* x, float* dW, int M, int N, int 
 // ------------------------------------------------------------------ emitters
 void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
   if (probs.empty()) return;
+  // Weight gradients whose output is a handful of tiles but whose reduction runs over very many
+  // rows (first-stage convolutions, the stem) would keep only a few SMs busy: split the reduction
+  // into slices that write fp32 partial outputs, summed in slice order by the plan's final
+  // column reduction (deterministic; no atomics).
+  {
+    std::vector<GemmProb> expanded;
+    const size_t es = h.esize();
+    for (auto& g : probs) {
+      bool plain = g.out_f32 && g.act == EPI_NONE && !g.bias && !g.resid && g.ldc == g.N;
+      long long tiles = (long long)((g.M + 127) / 128) * ((g.N + 255) / 256);
+      long long S = 1;
+      if (plain && g.K >= 8192 && tiles * 2 <= h.num_sms) S = std::max(1LL, std::min<long long>({h.num_sms / tiles, g.K / 2048LL, 64LL}));
+      if (S == 1) { expanded.push_back(g); continue; }
+      size_t mn = (size_t)g.M * g.N;
+      float* part = (float*)h.dalloc((size_t)S * mn * sizeof(float));
+      int kc = (int)(((g.K + S - 1) / S + 63) / 64 * 64);
+      int made = 0;
+      for (int k0 = 0; k0 < g.K; k0 += kc, ++made) {
+        GemmProb q = g;
+        q.K = std::min(kc, g.K - k0);
+        q.A = (const char*)g.A + (size_t)k0 * g.a_ks * es;
+        q.B = (const char*)g.B + (size_t)k0 * g.b_ks * es;
+        q.C = part + (size_t)made * mn;
+        expanded.push_back(q);
+      }
+      h.pending_reduce.push_back(ColReduceProb{part, (float*)g.C, made, (int)mn, (int)mn});
+    }
+    probs.swap(expanded);
+  }
   // Problems the tensor-core kernel takes go into one grouped launch, the rest into another.
   std::vector<GemmProb> tc, simt;
   for (auto& g : probs) {
