@@ -172,33 +172,45 @@ __global__ void __launch_bounds__(NT) xent_vec_kernel(const XentProb* __restrict
     }
   }
   float M = block_max(m, red);
-  float s = 0.f;
+  // One exponential per logit: e = exp(z - max) is summed in fp32 and kept (as bf16, the precision
+  // the stored dlogits have anyway) in the registers that held z; the label's logit is saved first.
+  float s = 0.f, zy = 0.f;
+  const float ML2 = M * 1.4426950408889634f;
 #pragma unroll
   for (int j = 0; j < NV; ++j) {
     int i = j * NT + threadIdx.x;
     if (i < nvec) {
       float f[8];
       unpack8(raw[j], f);
+      int c0 = i * 8;
+      if (y >= c0 && y < c0 + 8) {
 #pragma unroll
-      for (int t = 0; t < 8; ++t) s += __expf(f[t] - M);
+        for (int t = 0; t < 8; ++t) if (c0 + t == y) zy = f[t];
+      }
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { f[t] = exp2f(fmaf(f[t], 1.4426950408889634f, -ML2)); s += f[t]; }
+      raw[j] = pack8(f);
     }
   }
   float S = block_sum(s, red);
   float lse = M + logf(S);
   float inv = 1.0f / (float)(*p.n_valid);
+  float scale = inv / S;
 #pragma unroll
   for (int j = 0; j < NV; ++j) {
     int i = j * NT + threadIdx.x;
     if (i < nvec) {
-      float f[8], o[8];
+      float f[8];
       unpack8(raw[j], f);
       int c0 = i * 8;
 #pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        if (c0 + t == y) p.row_loss[row] = lse - f[t];
-        o[t] = (__expf(f[t] - lse) - (c0 + t == y ? 1.f : 0.f)) * inv;
+      for (int t = 0; t < 8; ++t) f[t] *= scale;
+      if (y >= c0 && y < c0 + 8) {
+        p.row_loss[row] = lse - zy;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) if (c0 + t == y) f[t] -= inv;
       }
-      z[i] = pack8(o);
+      z[i] = pack8(f);
     }
   }
 }
