@@ -5,7 +5,7 @@
 // Sec. 3 makes them independent).  Per tile, 64-deep k slices of A and B are brought into a
 // 4-stage shared-memory ring by TMA (128-byte swizzle; out-of-range rows/columns read as zero, so
 // ragged M, N, K need no special case), one elected thread issues tcgen05.mma (M=128, N=256, K=16,
-// bf16 x bf16 -> fp32) into one of two 256-column TMEM accumulators, and four epilogue warps read
+// bf16 x bf16 -> fp32) into one of two 256-column TMEM accumulators, and eight epilogue warps read
 // the finished accumulator back with tcgen05.ld, apply the fused epilogue (bias, residual,
 // ReLU/GELU, ReLU mask, GELU') and store bf16 or fp32 while the next tile's main loop already
 // runs on the other accumulator.
@@ -31,7 +31,8 @@ constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;              // 16 KB
 constexpr int B_BYTES = BN * BK * 2;              // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;    // 48 KB
-constexpr int NTHREADS = 192;
+constexpr int EPI_WARPS = 8;                      // two warps per TMEM lane quarter, each takes half of the 256 columns
+constexpr int NTHREADS = 64 + 32 * EPI_WARPS;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
@@ -223,7 +224,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&sh->tmem_full[a], 1); mbar_init(&sh->tmem_empty[a], 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh->tmem_full[a], 1); mbar_init(&sh->tmem_empty[a], EPI_WARPS); }
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -329,22 +330,30 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      int m = m0 + quarter * 32 + lane;
-      size_t esz = p.out_f32 ? 4 : 2;
-      bool vec_ok = (p.ldc % 8 == 0) && (((uintptr_t)p.C & 15) == 0) && (!p.C2 || ((uintptr_t)p.C2 & 15) == 0) &&
-                    (!p.resid || ((uintptr_t)p.resid & 15) == 0) && (!p.aux || ((uintptr_t)p.aux & 15) == 0);
-      (void)esz;
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t acc[32];
-        uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + c * 32);
-        tc_ld32(taddr, acc);
-        tc_wait_ld();
-        int nc = n0 + c * 32;
+      // Each thread owns one accumulator row and walks this warp's half of the columns 32 at a time;
+      // the TMEM load of the next 32 columns is in flight while the current ones are stored.
+      const int m = m0 + quarter * 32 + lane;
+      const int col0 = ((warp - 2) >> 2) * (BN / 2);
+      const bool vec_ok = (p.ldc % 8 == 0) && (((uintptr_t)p.C & 15) == 0) && (!p.C2 || ((uintptr_t)p.C2 & 15) == 0) &&
+                          (!p.resid || ((uintptr_t)p.resid & 15) == 0) && (!p.aux || ((uintptr_t)p.aux & 15) == 0);
+      const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + col0);
+      auto emit = [&](const uint32_t* a, int c) {
+        const int nc = n0 + col0 + c * 32;
         if (m < p.M && nc < p.N) {
-          if (vec_ok && nc + 32 <= p.N) store_row32<true>(p, m, nc, acc);
-          else store_row32<false>(p, m, nc, acc);
+          if (vec_ok && nc + 32 <= p.N) store_row32<true>(p, m, nc, a);
+          else store_row32<false>(p, m, nc, a);
         }
+      };
+      uint32_t acc0[32], acc1[32];
+      tc_ld32(trow, acc0);
+#pragma unroll 1
+      for (int c = 0; c < BN / 64; c += 2) {
+        tc_wait_ld();
+        tc_ld32(trow + (c + 1) * 32, acc1);
+        emit(acc0, c);
+        tc_wait_ld();
+        if (c + 2 < BN / 64) tc_ld32(trow + (c + 2) * 32, acc0);
+        emit(acc1, c + 1);
       }
       tc_fence_before();
       __syncwarp();
