@@ -20,6 +20,7 @@
 #include <cuda.h>
 
 #include <cstdio>
+#include <cstdlib>
 
 #include "common.cuh"
 #include "gemm_tc.h"
@@ -27,17 +28,26 @@
 namespace lp {
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2;              // 16 KB
-constexpr int B_BYTES = BN * BK * 2;              // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;    // 48 KB
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int A_BYTES = BM * BK * 2;              // 16 KB of A per CTA and stage
+// CG = 1: one CTA per 128x256 tile, B tile 256x64 (32 KB), 4 stages of 48 KB.
+// CG = 2: a pair of CTAs (cluster of 2, tcgen05 cta_group::2) per 256x256 tile; each CTA holds its own
+//         128 rows of A and HALF of the B tile (128x64, 16 KB), so every SM pulls a third fewer bytes per
+//         FLOP through its L2 port and the ring is 6 stages of 32 KB.
+template <int CG> struct Cfg {
+  static constexpr int BNL = BN / CG;                       // rows of B this CTA loads
+  static constexpr int B_BYTES = BNL * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = CG == 1 ? 4 : 6;
+};
+constexpr int MAX_STAGES = 6;
 constexpr int EPI_WARPS = 8;                      // two warps per TMEM lane quarter, each takes half of the 256 columns
 constexpr int NTHREADS = 64 + 32 * EPI_WARPS;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 struct __align__(8) Shared {
-  uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+  uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -214,61 +224,130 @@ __device__ __forceinline__ void store_row32(const GemmProb& p, int m, int n0, co
   }
 }
 
+// ---- cluster helpers (CG = 2)
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {   // same offset in CTA `rank` of the cluster
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t bar_caddr, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_caddr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_caddr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_caddr) : "memory");
+}
+// TMA load whose completion is signalled on a barrier given by cluster address (the pair leader's).
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, int x, int y, uint32_t bar_caddr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_caddr) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {   // arrives on this barrier in both CTAs of the pair
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+template <int CG>
 __global__ void __launch_bounds__(NTHREADS, 1)
 gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict__ maps, int nprob, int total_tiles,
                int* status) {
+  using C = Cfg<CG>;
+  constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, BNL = C::BNL;
+  constexpr int TILE_M = BM * CG;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   Shared* sh = (Shared*)(tiles + STAGES * STAGE_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = CG == 2 ? cluster_rank() : 0;          // 0 = the CTA that issues the pair's MMAs
+  const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&sh->tmem_full[a], 1); mbar_init(&sh->tmem_empty[a], EPI_WARPS); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh->full[s], CG); mbar_init(&sh->empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh->tmem_full[a], 1); mbar_init(&sh->tmem_empty[a], CG * EPI_WARPS); }
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CG == 1) {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();             // the partner's barriers exist before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *(volatile uint32_t*)&sh->tmem_base;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer (one per CTA)
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       int pi = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
         while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
         const GemmProb& p = probs[pi];
         const CUtensorMap* mapA = maps + 2 * pi;
         const CUtensorMap* mapB = mapA + 1;
         int t = tile - p.tile_start;
-        int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * BN;
+        int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN + (int)rank * BNL;
         bool a_mn = p.a_ms == 1, b_mn = p.b_ns == 1;
         int kb_n = (p.K + BK - 1) / BK;
         for (int kb = 0; kb < kb_n; ++kb) {
           if (!(ok = mbar_wait(&sh->empty[stage], phase ^ 1, sh, status))) break;
           uint8_t* a_dst = tiles + stage * STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_BYTES;
-          mbar_expect_tx(&sh->full[stage], STAGE_BYTES);
           int k0 = kb * BK;
-          if (a_mn) {
+          if (CG == 1) {
+            uint64_t* bar = &sh->full[stage];
+            mbar_expect_tx(bar, STAGE_BYTES);
+            if (a_mn) {
 #pragma unroll
-            for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, &sh->full[stage]);
-          } else {
-            tma_load_2d(a_dst, mapA, k0, m0, &sh->full[stage]);
-          }
-          if (b_mn) {
+              for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, bar);
+            } else {
+              tma_load_2d(a_dst, mapA, k0, m0, bar);
+            }
+            if (b_mn) {
 #pragma unroll
-            for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, &sh->full[stage]);
+              for (int i = 0; i < BNL / 64; ++i) tma_load_2d(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, bar);
+            } else {
+              tma_load_2d(b_dst, mapB, k0, n0, bar);
+            }
           } else {
-            tma_load_2d(b_dst, mapB, k0, n0, &sh->full[stage]);
+            // both CTAs' bytes are counted on the leader's barrier
+            uint32_t bar = map_to_rank(smem_u32(&sh->full[stage]), 0);
+            mbar_expect_tx_cluster(bar, STAGE_BYTES);
+            if (a_mn) {
+#pragma unroll
+              for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, bar);
+            } else {
+              tma_load_2d_pair(a_dst, mapA, k0, m0, bar);
+            }
+            if (b_mn) {
+#pragma unroll
+              for (int i = 0; i < BNL / 64; ++i) tma_load_2d_pair(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, bar);
+            } else {
+              tma_load_2d_pair(b_dst, mapB, k0, n0, bar);
+            }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -280,17 +359,17 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (the pair's leader only)
+    if (lane == 0 && rank == 0) {
       int stage = 0; uint32_t phase = 0;
       int pi = 0, it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
         while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
         const GemmProb& p = probs[pi];
         bool a_mn = p.a_ms == 1, b_mn = p.b_ns == 1;
         uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-                         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
         int ab = it & 1;
         uint32_t use = (uint32_t)(it >> 1);
         if (!(ok = mbar_wait(&sh->tmem_empty[ab], (use & 1) ^ 1, sh, status))) break;
@@ -306,12 +385,14 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
           uint32_t a_step = a_mn ? (16 * 128) >> 4 : 32 >> 4;
           uint32_t b_step = b_mn ? (16 * 128) >> 4 : 32 >> 4;
 #pragma unroll
-          for (int k4 = 0; k4 < BK / 16; ++k4)
-            tc_mma(d_tmem, adesc + (uint64_t)(k4 * a_step), bdesc + (uint64_t)(k4 * b_step), idesc, (kb | k4) != 0);
-          tc_commit(&sh->empty[stage]);
+          for (int k4 = 0; k4 < BK / 16; ++k4) {
+            if (CG == 1) tc_mma(d_tmem, adesc + (uint64_t)(k4 * a_step), bdesc + (uint64_t)(k4 * b_step), idesc, (kb | k4) != 0);
+            else tc_mma_pair(d_tmem, adesc + (uint64_t)(k4 * a_step), bdesc + (uint64_t)(k4 * b_step), idesc, (kb | k4) != 0);
+          }
+          if (CG == 1) tc_commit(&sh->empty[stage]); else tc_commit_pair(&sh->empty[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
-        if (ok) tc_commit(&sh->tmem_full[ab]);
+        if (ok) { if (CG == 1) tc_commit(&sh->tmem_full[ab]); else tc_commit_pair(&sh->tmem_full[ab]); }
       }
     }
   } else {
@@ -319,11 +400,11 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
     const int quarter = warp & 3;            // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
     int pi = 0, it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+    for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
       while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
       const GemmProb p = probs[pi];
       int t = tile - p.tile_start;
-      int m0 = (t / p.tiles_n) * BM, n0 = (t % p.tiles_n) * BN;
+      int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN;
       int ab = it & 1;
       uint32_t use = (uint32_t)(it >> 1);
       ok = mbar_wait(&sh->tmem_full[ab], use & 1, sh, status);
@@ -357,15 +438,20 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->tmem_empty[ab]);
+      if (lane == 0) {
+        if (CG == 1) mbar_arrive(&sh->tmem_empty[ab]);
+        else mbar_arrive_cluster(map_to_rank(smem_u32(&sh->tmem_empty[ab]), 0));   // the leader's MMA warp waits for both CTAs
+      }
     }
   }
 
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();             // neither CTA frees TMEM or exits while the partner may still touch it
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    if (CG == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -412,34 +498,64 @@ bool gemm_tc_eligible(const GemmProb& g) {
   return get_encode() != nullptr;
 }
 
-int gemm_tc_tiles(GemmProb& g, int tile_start) {
-  g.tile_start = tile_start;
-  g.tiles_n = (g.N + BN - 1) / BN;
-  return ((g.M + BM - 1) / BM) * g.tiles_n;
+int gemm_tc_choose_cg(const GemmProb* probs, int n) {
+  static int forced = -1;
+  if (forced < 0) {
+    const char* e = getenv("LP_GEMM_CG");      // diagnostic override: 1 or 2
+    forced = e ? atoi(e) : 0;
+  }
+  if (forced == 1 || forced == 2) return forced;
+  for (int i = 0; i < n; ++i)
+    if (probs[i].M <= BM) return 1;            // a 256-row pair tile would be half empty
+  return 2;
 }
 
-bool gemm_tc_encode(const GemmProb& g, void* mapA, void* mapB) {
+int gemm_tc_tiles(GemmProb& g, int tile_start, int cg) {
+  g.tile_start = tile_start;
+  g.tiles_n = (g.N + BN - 1) / BN;
+  return ((g.M + BM * cg - 1) / (BM * cg)) * g.tiles_n;
+}
+
+bool gemm_tc_encode(const GemmProb& g, void* mapA, void* mapB, int cg) {
   bool okA, okB;
   if (g.a_ms == 1) okA = encode_map((CUtensorMap*)mapA, g.A, g.M, g.K, g.a_ks, BK);       // MN-major: rows are k
   else okA = encode_map((CUtensorMap*)mapA, g.A, g.K, g.M, g.a_ms, BM);
   if (g.b_ns == 1) okB = encode_map((CUtensorMap*)mapB, g.B, g.N, g.K, g.b_ks, BK);
-  else okB = encode_map((CUtensorMap*)mapB, g.B, g.K, g.N, g.b_ns, BN);
+  else okB = encode_map((CUtensorMap*)mapB, g.B, g.K, g.N, g.b_ns, BN / cg);
   return okA && okB;
 }
 
 cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int nprob, int total_tiles, int* d_status,
-                           int num_sms, cudaStream_t s) {
-  static bool attr_set = false;
-  size_t smem = STAGES * STAGE_BYTES + 1024 + sizeof(Shared);
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                           int num_sms, cudaStream_t s, int cg) {
+  static bool attr_set[3] = {false, false, false};
+  size_t smem = (cg == 2 ? Cfg<2>::STAGES * Cfg<2>::STAGE_BYTES : Cfg<1>::STAGES * Cfg<1>::STAGE_BYTES) + 1024 + sizeof(Shared);
+  if (!attr_set[cg]) {
+    cudaError_t e = cg == 2 ? cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                            : cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[cg] = true;
   }
   if (total_tiles == 0) return cudaSuccess;
-  int grid = total_tiles < num_sms ? total_tiles : num_sms;
-  gemm_tc_kernel<<<grid, NTHREADS, smem, s>>>(d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
-  return cudaGetLastError();
+  if (cg == 1) {
+    int grid = total_tiles < num_sms ? total_tiles : num_sms;
+    gemm_tc_kernel<1><<<grid, NTHREADS, smem, s>>>(d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
+    return cudaGetLastError();
+  }
+  int pairs = num_sms / 2;
+  if (total_tiles < pairs) pairs = total_tiles;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(NTHREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
 }
 
 }  // namespace lp

@@ -430,16 +430,17 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream,
   auto take = [&](size_t bytes) { char* r = cur; cur += (bytes + 255) / 256 * 256; return r; };
   if (!tc.empty()) {
     int total = 0;
-    for (auto& g : tc) total += gemm_tc_tiles(g, total);
+    const int cg = gemm_tc_choose_cg(tc.data(), (int)tc.size());
+    for (auto& g : tc) total += gemm_tc_tiles(g, total, cg);
     std::vector<Map> maps(2 * tc.size());
     for (size_t i = 0; i < tc.size(); ++i)
-      if (!gemm_tc_encode(tc[i], &maps[2 * i], &maps[2 * i + 1])) return fail(nullptr, LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+      if (!gemm_tc_encode(tc[i], &maps[2 * i], &maps[2 * i + 1], cg)) return fail(nullptr, LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
     GemmProb* dp = (GemmProb*)take(tc.size() * sizeof(GemmProb));
     Map* dm = (Map*)take(maps.size() * sizeof(Map));
     cudaMemcpyAsync(dp, tc.data(), tc.size() * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
     cudaMemcpyAsync(dm, maps.data(), maps.size() * sizeof(Map), cudaMemcpyHostToDevice, s);
     cudaStreamSynchronize(s);
-    launch_gemm_tc(dp, dm, (int)tc.size(), total, d_status, num_sms, s);
+    launch_gemm_tc(dp, dm, (int)tc.size(), total, d_status, num_sms, s, cg);
   }
   if (!simt.empty()) {
     int t = 0;

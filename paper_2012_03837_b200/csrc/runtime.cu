@@ -136,11 +136,12 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
   }
   if (!tc.empty()) {
     int total = 0;
-    for (auto& g : tc) total += gemm_tc_tiles(g, total);
+    const int cg = gemm_tc_choose_cg(tc.data(), (int)tc.size());
+    for (auto& g : tc) total += gemm_tc_tiles(g, total, cg);
     struct alignas(64) Map { unsigned char b[128]; };
     std::vector<Map> maps(2 * tc.size());
     for (size_t i = 0; i < tc.size(); ++i)
-      if (!gemm_tc_encode(tc[i], &maps[2 * i], &maps[2 * i + 1])) throw std::runtime_error("cuda: cuTensorMapEncodeTiled failed");
+      if (!gemm_tc_encode(tc[i], &maps[2 * i], &maps[2 * i + 1], cg)) throw std::runtime_error("cuda: cuTensorMapEncodeTiled failed");
     const GemmProb* d = h.upload(tc);
     const void* dm = h.upload(maps);
     int n = (int)tc.size();
@@ -148,7 +149,7 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
     int sms = h.num_sms;
     double fl = 0;
     for (auto& g : tc) fl += 2.0 * g.M * g.N * g.K;
-    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream); }, KIND_GEMM_TC, fl);
+    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream, cg); }, KIND_GEMM_TC, fl);
   }
   if (!simt.empty()) {
     int t = 0;
