@@ -214,7 +214,7 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* probs, int backend, void* stre
  * lock, an embedding into a host whose device-memory budget was handed out up front.  lp_gemm_bf16
  * keeps its problem table, its TMA tensor maps and its status word in a cudaMalloc'ed buffer that
  * grows on demand; this variant keeps them in a fixed array that is part of the library image
- * (about 41 KB of device memory on every GPU that loads the library, held until the process exits)
+ * (about 58 KB of device memory on every GPU that loads the library, held until the process exits)
  * and calls no cudaMalloc, cudaFree or any other allocating routine.
  *
  *   n: 1 .. LP_GEMM_STATIC_MAX problems; more is rejected with LP_ERR_SHAPE and nothing is launched.

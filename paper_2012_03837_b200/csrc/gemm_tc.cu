@@ -76,13 +76,16 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false if the wait gave up or another role already did.
+// Bounded wait.  Returns false if the wait gave up or another role already did.  The clock is only
+// consulted after a first batch of polls (each poll already blocks in hardware for a short while).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
-  if (mbar_try(bar, parity)) return true;
+#pragma unroll 1
+  for (int i = 0; i < 64; ++i)
+    if (mbar_try(bar, parity)) return true;
   unsigned long long t0 = gtime_ns();
   int spins = 0;
   while (!mbar_try(bar, parity)) {
-    if ((++spins & 255) == 0) {
+    if ((++spins & 63) == 0) {
       if (*(volatile int*)&sh->abort_flag) return false;
       if (gtime_ns() - t0 > WAIT_LIMIT_NS) {
         *(volatile int*)&sh->abort_flag = 1;
@@ -137,21 +140,35 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
   return d;
 }
 
-// Epilogue for 32 consecutive columns of one row held in registers.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src)) : "memory");
+}
+
+// Fused epilogue for 32 consecutive columns (n0 ..) of one accumulator row (row m, held by this lane).
+// Output path: if `stg` is non-null the warp's 32x32 block is written to a 4 KB shared-memory staging
+// buffer in the swizzled layout of the output tensor map and leaves through ONE TMA store (full-line
+// writes, clipped at the matrix edge by the hardware); otherwise every lane stores its own row.
+// VEC: all 32 columns exist and resid / aux / C are 16-byte aligned (128-bit accesses).
 template <bool VEC>
-__device__ __forceinline__ void store_row32(const GemmProb& p, int m, int n0, const uint32_t* acc) {
+__device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensorMap* mapC, const CUtensorMap* mapC2,
+                                               uint8_t* stg, int m, int m_warp0, int n0, const uint32_t* acc, int lane) {
   float v[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
-  size_t off = (size_t)m * p.ldc + n0;
-  int nvalid = min(32, p.N - n0);
+  const bool row_ok = m < p.M;
+  const size_t off = (size_t)m * p.ldc + n0;
+  const int nvalid = min(32, p.N - n0);
   if (p.bias) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) if (VEC || j < nvalid) v[j] += p.bias[n0 + j];
   }
   auto load32 = [&](const void* base, float* o) {
     const bf16* src = (const bf16*)base + off;
-    if (VEC) {
+    if (!row_ok) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) o[j] = 0.f;
+    } else if (VEC) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         uint4 u = *(const uint4*)(src + q * 8);
@@ -164,20 +181,57 @@ __device__ __forceinline__ void store_row32(const GemmProb& p, int m, int n0, co
       for (int j = 0; j < 32; ++j) o[j] = j < nvalid ? __bfloat162float(src[j]) : 0.f;
     }
   };
-  auto store32 = [&](void* base, const float* o) {
-    bf16* dst = (bf16*)base + off;
-    if (VEC) {
+  // one output block (bf16 or fp32) of this warp
+  auto put = [&](void* base, const CUtensorMap* map, const float* o, bool f32) {
+    if (stg) {
+      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging buffer free again
+      __syncwarp();
+      if (f32) {
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint4 u;
-        __nv_bfloat162* h = (__nv_bfloat162*)&u;
+        for (int q = 0; q < 8; ++q)
+          *(float4*)(stg + lane * 128 + ((q ^ (lane & 7)) << 4)) = make_float4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+      } else {
 #pragma unroll
-        for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(o[q * 8 + 2 * t], o[q * 8 + 2 * t + 1]);
-        *(uint4*)(dst + q * 8) = u;
+        for (int q = 0; q < 4; ++q) {
+          uint4 u;
+          __nv_bfloat162* h = (__nv_bfloat162*)&u;
+#pragma unroll
+          for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(o[q * 8 + 2 * t], o[q * 8 + 2 * t + 1]);
+          *(uint4*)(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) = u;
+        }
       }
-    } else {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_2d(map, n0, m_warp0, stg);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+      }
+    } else if (row_ok) {
+      if (f32) {
+        float* dst = (float*)base + off;
+        if (VEC) {
 #pragma unroll
-      for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = __float2bfloat16_rn(o[j]);
+          for (int q = 0; q < 8; ++q) *(float4*)(dst + q * 4) = make_float4(o[q * 4], o[q * 4 + 1], o[q * 4 + 2], o[q * 4 + 3]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = o[j];
+        }
+      } else {
+        bf16* dst = (bf16*)base + off;
+        if (VEC) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint4 u;
+            __nv_bfloat162* h = (__nv_bfloat162*)&u;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(o[q * 8 + 2 * t], o[q * 8 + 2 * t + 1]);
+            *(uint4*)(dst + q * 8) = u;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = __float2bfloat16_rn(o[j]);
+        }
+      }
     }
   };
   float t[32];
@@ -194,7 +248,7 @@ __device__ __forceinline__ void store_row32(const GemmProb& p, int m, int n0, co
     case EPI_GELU:
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] = __bfloat162float(__float2bfloat16_rn(v[j]));
-      store32(p.C2, v);
+      put(p.C2, mapC2, v, false);
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] = gelu_f(v[j]);
       break;
@@ -210,18 +264,7 @@ __device__ __forceinline__ void store_row32(const GemmProb& p, int m, int n0, co
       break;
     default: break;
   }
-  if (p.out_f32) {
-    float* dst = (float*)p.C + off;
-    if (VEC) {
-#pragma unroll
-      for (int q = 0; q < 8; ++q) *(float4*)(dst + q * 4) = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
-    } else {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = v[j];
-    }
-  } else {
-    store32(p.C, v);
-  }
+  put(p.C, mapC, v, p.out_f32 != 0);
 }
 
 // ---- cluster helpers (CG = 2)
@@ -271,7 +314,8 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
   constexpr int TILE_M = BM * CG;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  Shared* sh = (Shared*)(tiles + STAGES * STAGE_BYTES);
+  uint8_t* staging = tiles + STAGES * STAGE_BYTES;                     // EPI_WARPS x 4 KB, 1024-byte aligned
+  Shared* sh = (Shared*)(staging + EPI_WARPS * 4096);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = CG == 2 ? cluster_rank() : 0;          // 0 = the CTA that issues the pair's MMAs
   const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
@@ -306,7 +350,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
         while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
         const GemmProb& p = probs[pi];
-        const CUtensorMap* mapA = maps + 2 * pi;
+        const CUtensorMap* mapA = maps + 4 * pi;
         const CUtensorMap* mapB = mapA + 1;
         int t = tile - p.tile_start;
         int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN + (int)rank * BNL;
@@ -407,7 +451,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN;
       int ab = it & 1;
       uint32_t use = (uint32_t)(it >> 1);
-      ok = mbar_wait(&sh->tmem_full[ab], use & 1, sh, status);
+      ok = lane == 0 ? mbar_wait(&sh->tmem_full[ab], use & 1, sh, status) : true;   // one poller per warp
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -418,12 +462,14 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       const bool vec_ok = (p.ldc % 8 == 0) && (((uintptr_t)p.C & 15) == 0) && (!p.C2 || ((uintptr_t)p.C2 & 15) == 0) &&
                           (!p.resid || ((uintptr_t)p.resid & 15) == 0) && (!p.aux || ((uintptr_t)p.aux & 15) == 0);
       const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + col0);
+      const CUtensorMap* mapC = maps + 4 * pi + 2;
+      uint8_t* stg = p.store_tma ? staging + (warp - 2) * 4096 : nullptr;
+      const int m_warp0 = m0 + quarter * 32;
       auto emit = [&](const uint32_t* a, int c) {
         const int nc = n0 + col0 + c * 32;
-        if (m < p.M && nc < p.N) {
-          if (vec_ok && nc + 32 <= p.N) store_row32<true>(p, m, nc, a);
-          else store_row32<false>(p, m, nc, a);
-        }
+        if (nc >= p.N || m_warp0 >= p.M) return;            // warp-uniform
+        if (vec_ok && nc + 32 <= p.N) epilogue_row32<true>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane);
+        else epilogue_row32<false>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane);
       };
       uint32_t acc0[32], acc1[32];
       tc_ld32(trow, acc0);
@@ -445,6 +491,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
     }
   }
 
+  if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's TMA stores are done
   tc_fence_before();
   __syncthreads();
   if (CG == 2) cluster_sync_all();             // neither CTA frees TMEM or exits while the partner may still touch it
@@ -516,19 +563,45 @@ int gemm_tc_tiles(GemmProb& g, int tile_start, int cg) {
   return ((g.M + BM * cg - 1) / (BM * cg)) * g.tiles_n;
 }
 
-bool gemm_tc_encode(const GemmProb& g, void* mapA, void* mapB, int cg) {
+// Output map: [M, N] with a pitch of ldc elements, 32x32 boxes, swizzled like the epilogue's staging buffer
+// (64-byte rows for bf16, 128-byte rows for fp32).
+bool encode_out_map(CUtensorMap* out, const void* base, long long N, long long M, long long ldc, bool f32) {
+  EncodeFn fn = get_encode();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  cuuint64_t strides[1] = {(cuuint64_t)ldc * (f32 ? 4 : 2)};
+  cuuint32_t box[2] = {32u, 32u};
+  cuuint32_t estr[2] = {1u, 1u};
+  CUresult r = fn(out, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// maps: 4 consecutive 128-byte tensor maps [A, B, C, C2].  Sets g.store_tma.
+bool gemm_tc_encode(GemmProb& g, void* maps, int cg) {
+  CUtensorMap* mapA = (CUtensorMap*)maps;
+  CUtensorMap* mapB = mapA + 1;
+  const long long esz = g.out_f32 ? 4 : 2;
+  g.store_tma = ((g.ldc * esz) % 16 == 0) && (((uintptr_t)g.C & 15) == 0) &&
+                (g.act != EPI_GELU || (((uintptr_t)g.C2 & 15) == 0 && (g.ldc * 2) % 16 == 0));
+  if (g.store_tma) {
+    bool ok = encode_out_map(mapA + 2, g.C, g.N, g.M, g.ldc, g.out_f32 != 0);
+    if (ok && g.act == EPI_GELU) ok = encode_out_map(mapA + 3, g.C2, g.N, g.M, g.ldc, false);
+    if (!ok) g.store_tma = 0;
+  }
   bool okA, okB;
-  if (g.a_ms == 1) okA = encode_map((CUtensorMap*)mapA, g.A, g.M, g.K, g.a_ks, BK);       // MN-major: rows are k
-  else okA = encode_map((CUtensorMap*)mapA, g.A, g.K, g.M, g.a_ms, BM);
-  if (g.b_ns == 1) okB = encode_map((CUtensorMap*)mapB, g.B, g.N, g.K, g.b_ks, BK);
-  else okB = encode_map((CUtensorMap*)mapB, g.B, g.K, g.N, g.b_ns, BN / cg);
+  if (g.a_ms == 1) okA = encode_map(mapA, g.A, g.M, g.K, g.a_ks, BK);       // MN-major: rows are k
+  else okA = encode_map(mapA, g.A, g.K, g.M, g.a_ms, BM);
+  if (g.b_ns == 1) okB = encode_map(mapB, g.B, g.N, g.K, g.b_ks, BK);
+  else okB = encode_map(mapB, g.B, g.K, g.N, g.b_ns, BN / cg);
   return okA && okB;
 }
 
 cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int nprob, int total_tiles, int* d_status,
                            int num_sms, cudaStream_t s, int cg) {
   static bool attr_set[3] = {false, false, false};
-  size_t smem = (cg == 2 ? Cfg<2>::STAGES * Cfg<2>::STAGE_BYTES : Cfg<1>::STAGES * Cfg<1>::STAGE_BYTES) + 1024 + sizeof(Shared);
+  size_t smem = (cg == 2 ? Cfg<2>::STAGES * Cfg<2>::STAGE_BYTES : Cfg<1>::STAGES * Cfg<1>::STAGE_BYTES) + EPI_WARPS * 4096 + 1024 + sizeof(Shared);
   if (!attr_set[cg]) {
     cudaError_t e = cg == 2 ? cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
                             : cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -569,7 +642,7 @@ cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int npro
 // while a CUDA graph is being captured or inside a memory-pool-managed region, real-time loops
 // that must not take the driver's allocation lock, and hosts whose memory budget is fixed up
 // front.  This variant keeps the table in the file-scope array below instead: a fixed
-// LP_GEMM_STATIC_MAX problems, about 41 KB that every GPU loading this library holds until the
+// LP_GEMM_STATIC_MAX problems, about 58 KB that every GPU loading this library holds until the
 // process exits.
 // ---------------------------------------------------------------------------------------------
 #include "../../include/lp.h"
@@ -583,7 +656,7 @@ struct StaticLayout {
   int pad[63];
   GemmProb tc[LP_GEMM_STATIC_MAX];
   GemmProb alu[LP_GEMM_STATIC_MAX];
-  alignas(64) TMap maps[2 * LP_GEMM_STATIC_MAX];
+  alignas(64) TMap maps[4 * LP_GEMM_STATIC_MAX];
 };
 
 // In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
@@ -625,7 +698,7 @@ extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* st
   StaticLayout* sc = g_static_ptr[dev];
 
   GemmProb tc[LP_GEMM_STATIC_MAX], alu[LP_GEMM_STATIC_MAX];
-  TMap maps[2 * LP_GEMM_STATIC_MAX];
+  TMap maps[4 * LP_GEMM_STATIC_MAX];
   int ntc = 0, nalu = 0, tc_tiles = 0, alu_tiles = 0;
   for (int i = 0; i < n; ++i) {
     const lp_gemm_desc& q = in[i];
@@ -638,7 +711,7 @@ extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* st
     g.ldc = q.ldc; g.act = q.act; g.out_f32 = q.out_f32;
     if (gemm_tc_eligible(g)) {
       tc_tiles += gemm_tc_tiles(g, tc_tiles);
-      if (!gemm_tc_encode(g, &maps[2 * ntc], &maps[2 * ntc + 1])) return static_fail(LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+      if (!gemm_tc_encode(g, &maps[4 * ntc], 1)) return static_fail(LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
       tc[ntc++] = g;
     } else {
       g.tiles_n = (g.N + 63) / 64;
@@ -654,7 +727,7 @@ extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* st
   if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "cudaMemsetAsync", e);
   if (ntc) {
     e = cudaMemcpyAsync(sc->tc, tc, ntc * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(sc->maps, maps, 2 * ntc * sizeof(TMap), cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sc->maps, maps, 4 * ntc * sizeof(TMap), cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = launch_gemm_tc(sc->tc, sc->maps, ntc, tc_tiles, &sc->status, g_static_sms[dev], s);
     if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "tensor-core launch", e);
   }

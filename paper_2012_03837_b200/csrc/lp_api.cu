@@ -419,7 +419,7 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream,
   static void* d_tab = nullptr;
   static size_t d_cap = 0;
   struct alignas(64) Map { unsigned char b[128]; };
-  size_t need = 256 + tc.size() * sizeof(GemmProb) + 256 + 2 * tc.size() * sizeof(Map) + simt.size() * sizeof(GemmProb) + 256;
+  size_t need = 256 + tc.size() * sizeof(GemmProb) + 256 + 4 * tc.size() * sizeof(Map) + simt.size() * sizeof(GemmProb) + 256;
   if (need > d_cap) {
     cudaStreamSynchronize(s);
     if (d_tab) cudaFree(d_tab);
@@ -432,9 +432,9 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream,
     int total = 0;
     const int cg = gemm_tc_choose_cg(tc.data(), (int)tc.size());
     for (auto& g : tc) total += gemm_tc_tiles(g, total, cg);
-    std::vector<Map> maps(2 * tc.size());
+    std::vector<Map> maps(4 * tc.size());
     for (size_t i = 0; i < tc.size(); ++i)
-      if (!gemm_tc_encode(tc[i], &maps[2 * i], &maps[2 * i + 1], cg)) return fail(nullptr, LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+      if (!gemm_tc_encode(tc[i], &maps[4 * i], cg)) return fail(nullptr, LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
     GemmProb* dp = (GemmProb*)take(tc.size() * sizeof(GemmProb));
     Map* dm = (Map*)take(maps.size() * sizeof(Map));
     cudaMemcpyAsync(dp, tc.data(), tc.size() * sizeof(GemmProb), cudaMemcpyHostToDevice, s);

@@ -36,6 +36,7 @@ struct GemmProb {
   int out_f32;
   int tile_start;  // first tile index of this problem in the launch (filled by the launcher)
   int tiles_n;
+  int store_tma;   // tensor-core kernel: outputs leave through TMA stores (set by the launcher when C's pitch allows)
 };
 
 // FP32-ALU GEMM (any sizes and strides).  T = float or bf16 operands, fp32 accumulation.

@@ -139,9 +139,9 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
     const int cg = gemm_tc_choose_cg(tc.data(), (int)tc.size());
     for (auto& g : tc) total += gemm_tc_tiles(g, total, cg);
     struct alignas(64) Map { unsigned char b[128]; };
-    std::vector<Map> maps(2 * tc.size());
+    std::vector<Map> maps(4 * tc.size());
     for (size_t i = 0; i < tc.size(); ++i)
-      if (!gemm_tc_encode(tc[i], &maps[2 * i], &maps[2 * i + 1], cg)) throw std::runtime_error("cuda: cuTensorMapEncodeTiled failed");
+      if (!gemm_tc_encode(tc[i], &maps[4 * i], cg)) throw std::runtime_error("cuda: cuTensorMapEncodeTiled failed");
     const GemmProb* d = h.upload(tc);
     const void* dm = h.upload(maps);
     int n = (int)tc.size();
