@@ -79,13 +79,17 @@ void launch_label_prep(const LabelProb* d_probs, int n, int* d_status, cudaStrea
 
 struct XentProb {     // softmax cross-entropy rows (App. A.1): z [rows, ld] -> dz in place, row losses
   void* z; const int* y; const int* n_valid; float* row_loss; int rows, classes, ld;
+  float* colsum_part;   // optional [ceil(rows / XENT_ROWS), classes]: per-row-block column sums of dz (bias gradient)
 };
+enum { XENT_ROWS = 64 };
 void launch_xent(const XentProb* d_probs, int n, int max_rows, bool is_bf16, cudaStream_t s);
 
 // 128-bit vectorised bf16 variants (rowwise_vec.cu); nv = compile-time vectors per lane / thread.
 void launch_ln_fwd_vec(const LnProb* d_probs, int n, int max_rows, int nv, cudaStream_t s);
 void launch_ln_bwd_vec(const LnBwdProb* d_probs, int n, int max_rows, int nv, cudaStream_t s);
 void launch_xent_vec(const XentProb* d_probs, int n, int max_rows, int nv, cudaStream_t s);
+// Blocks of XENT_ROWS rows, dlogits in place plus per-block column sums; classes % 8 == 0, classes <= 32768.
+void launch_xent_rows(const XentProb* d_probs, int n, int max_rows, int classes, cudaStream_t s);
 
 struct LossProb { const float* row_loss; const int* n_valid; int rows; int out_index; };
 void launch_loss_reduce(const LossProb* d_probs, int n, float* d_losses, int* d_status, cudaStream_t s);

@@ -177,7 +177,8 @@ void build_lm(Handle& h) {
   };
 
   // ---- heads: LayerNorm, logits, loss (+ dlogits in place)
-  auto heads_forward = [&](Plan& p, int wr, bool pipelined, int rd, bool copy_logits) {
+  bool head_bias_done = false;   // the cross-entropy kernel already produced the head bias gradients
+  auto heads_forward = [&](Plan& p, int wr, bool pipelined, int rd, bool copy_logits, bool train) {
     std::vector<LnProb> ln;
     std::vector<GemmProb> g;
     std::vector<XentProb> xs;
@@ -185,7 +186,7 @@ void build_lm(Handle& h) {
       ChunkBufs& c = cb[k];
       ln.push_back(LnProb{h.bnd[wr][k], c.ah, h.P32(hn(k, "ln.g")), h.P32(hn(k, "ln.b")), c.meanh, c.rstdh, M, d});
       g.push_back(gemm_fwd(c.ah, h.W(hn(k, "W")), c.z, M, V, d, h.P32(hn(k, "b")), EPI_NONE));
-      xs.push_back(XentProb{c.z, labels_of(k, pipelined, rd), h.n_valid[k], c.row_loss, M, V, V});
+      xs.push_back(XentProb{c.z, labels_of(k, pipelined, rd), h.n_valid[k], c.row_loss, M, V, V, nullptr});
     }
     emit_ln_fwd(h, p, ln);
     emit_gemm(h, p, g);
@@ -196,7 +197,9 @@ void build_lm(Handle& h) {
         if (c.out_logits) cudaMemcpyAsync(c.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, c.stream);
       });
     }
-    emit_xent_and_loss(h, p, xs, all);
+    std::vector<float*> bgs;
+    for (int k = 0; k < K; ++k) bgs.push_back(h.G(hn(k, "b")));
+    head_bias_done = emit_xent_and_loss(h, p, xs, all, train ? &bgs : nullptr);
   };
 
   auto build_step = [&](Plan& p, bool pipelined, int rd, int wr) {
@@ -207,7 +210,7 @@ void build_lm(Handle& h) {
     emit_labels(h, p, lps);
     if (pipelined) forward(p, all, rd, wr);
     else for (int k = 0; k < K; ++k) forward(p, {k}, rd, wr);
-    heads_forward(p, wr, pipelined, rd, false);
+    heads_forward(p, wr, pipelined, rd, false, true);
 
     // ---- head backward -> gradient at the trunk output in G0
     {
@@ -218,8 +221,10 @@ void build_lm(Handle& h) {
         ChunkBufs& c = cb[k];
         g.push_back(gemm_wgrad(c.z, c.ah, h.G(hn(k, "W")), M, V, d));
         g.push_back(gemm_dgrad(c.z, h.W(hn(k, "W")), c.G1, M, V, d, EPI_NONE, nullptr));
-        cs.push_back(ColSumProb{c.z, nullptr, M, V, V});
-        outs.push_back(h.G(hn(k, "b")));
+        if (!head_bias_done) {
+          cs.push_back(ColSumProb{c.z, nullptr, M, V, V});
+          outs.push_back(h.G(hn(k, "b")));
+        }
       }
       emit_gemm(h, p, g);
       emit_colsum(h, p, cs, outs);
@@ -340,7 +345,7 @@ void build_lm(Handle& h) {
     std::vector<LabelProb> lps;
     for (int k = 0; k < K; ++k) lps.push_back(LabelProb{h.y_in, nullptr, M, V, h.n_valid[k]});
     emit_labels(h, p, lps);
-    heads_forward(p, wr, false, wr, true);
+    heads_forward(p, wr, false, wr, true, false);
   };
 
   build_step(h.sync_plan, false, 0, 0);

@@ -110,7 +110,7 @@ void build_mlp(Handle& h) {
       std::vector<XentProb> xs;
       for (int k = 0; k < K; ++k) {
         g.push_back(gemm_fwd(h.bnd[wr][k], h.W(hn(k, "W")), b.z[k], B, C, b.widths[k].back(), h.P32(hn(k, "b")), EPI_NONE));
-        xs.push_back(XentProb{b.z[k], labels_of(k, pipelined, rd), h.n_valid[k], b.row_loss[k], B, C, C});
+        xs.push_back(XentProb{b.z[k], labels_of(k, pipelined, rd), h.n_valid[k], b.row_loss[k], B, C, C, nullptr});
       }
       emit_gemm(h, p, g);
       emit_xent_and_loss(h, p, xs, all);
@@ -169,7 +169,7 @@ void build_mlp(Handle& h) {
     std::vector<XentProb> xs;
     for (int k = 0; k < K; ++k) {
       g.push_back(gemm_fwd(h.bnd[wr][k], h.W(hn(k, "W")), b.z[k], B, C, b.widths[k].back(), h.P32(hn(k, "b")), EPI_NONE));
-      xs.push_back(XentProb{b.z[k], h.y_in, h.n_valid[k], b.row_loss[k], B, C, C});
+      xs.push_back(XentProb{b.z[k], h.y_in, h.n_valid[k], b.row_loss[k], B, C, C, nullptr});
     }
     emit_gemm(h, p, g);
     void* zlast = b.z[K - 1];

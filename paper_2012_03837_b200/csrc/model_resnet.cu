@@ -277,7 +277,7 @@ void build_resnet(Handle& h) {
         if (r.out_logits) cudaMemcpyAsync(r.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, r.stream);
       });
     }
-    emit_xent_and_loss(h, p, {XentProb{c.z, labels, h.n_valid[k], c.row_loss, B, NC, NC}}, {k});
+    emit_xent_and_loss(h, p, {XentProb{c.z, labels, h.n_valid[k], c.row_loss, B, NC, NC, nullptr}}, {k});
   };
 
   auto backward_chunk = [&](Plan& p, int k, int rd, int wr) {

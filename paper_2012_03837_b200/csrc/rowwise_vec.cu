@@ -215,6 +215,117 @@ __global__ void __launch_bounds__(NT) xent_vec_kernel(const XentProb* __restrict
   }
 }
 
+// ------------------------------------------------------------------ cross-entropy over blocks of rows
+// One block of 512 threads walks XENT_ROWS consecutive rows; thread t owns the 8-column vectors
+// j*512 + t.  While the current row goes through its two block reductions, the next row is already
+// being loaded.  The column sums of the written dlogits (the head's bias gradient) are accumulated
+// on the way in shared memory (each thread only ever touches its own columns) and written once per
+// block, so the logits are read from HBM exactly once and written exactly once per step.
+template <int NV>
+__global__ void __launch_bounds__(512) xent_rows_kernel(const XentProb* __restrict__ probs) {
+  extern __shared__ float csum[];            // [classes]
+  __shared__ float red[33];
+  const XentProb p = probs[blockIdx.y];
+  const int r0 = blockIdx.x * XENT_ROWS;
+  if (r0 >= p.rows) return;
+  const int r1 = min(r0 + XENT_ROWS, p.rows);
+  const int nvec = p.classes >> 3;
+  const float inv = 1.0f / (float)(*p.n_valid);
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int i = j * 512 + threadIdx.x;
+    if (i < nvec) { *(float4*)(csum + i * 8) = make_float4(0, 0, 0, 0); *(float4*)(csum + i * 8 + 4) = make_float4(0, 0, 0, 0); }
+  }
+  uint4 nxt[NV];
+  {
+    const uint4* z = (const uint4*)((const bf16*)p.z + (size_t)r0 * p.ld);
+#pragma unroll
+    for (int j = 0; j < NV; ++j) { int i = j * 512 + threadIdx.x; if (i < nvec) nxt[j] = z[i]; }
+  }
+  for (int row = r0; row < r1; ++row) {
+    uint4 raw[NV];
+#pragma unroll
+    for (int j = 0; j < NV; ++j) raw[j] = nxt[j];
+    if (row + 1 < r1) {
+      const uint4* zn = (const uint4*)((const bf16*)p.z + (size_t)(row + 1) * p.ld);
+#pragma unroll
+      for (int j = 0; j < NV; ++j) { int i = j * 512 + threadIdx.x; if (i < nvec) nxt[j] = zn[i]; }
+    }
+    uint4* z = (uint4*)((bf16*)p.z + (size_t)row * p.ld);
+    const int y = p.y[row];
+    if (!(y >= 0 && y < p.classes)) {          // ignored row: no loss, zero gradient (uniform over the block)
+#pragma unroll
+      for (int j = 0; j < NV; ++j) { int i = j * 512 + threadIdx.x; if (i < nvec) z[i] = make_uint4(0, 0, 0, 0); }
+      if (threadIdx.x == 0) p.row_loss[row] = 0.f;
+      continue;
+    }
+    float m = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      int i = j * 512 + threadIdx.x;
+      if (i < nvec) {
+        float f[8];
+        unpack8(raw[j], f);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) m = fmaxf(m, f[t]);
+      }
+    }
+    const float M = block_max(m, red);
+    const float ML2 = M * 1.4426950408889634f;
+    float s = 0.f, zy = 0.f;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      int i = j * 512 + threadIdx.x;
+      if (i < nvec) {
+        float f[8];
+        unpack8(raw[j], f);
+        int c0 = i * 8;
+        if (y >= c0 && y < c0 + 8) {
+#pragma unroll
+          for (int t = 0; t < 8; ++t) if (c0 + t == y) zy = f[t];
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t) { f[t] = exp2f(fmaf(f[t], 1.4426950408889634f, -ML2)); s += f[t]; }
+        raw[j] = pack8(f);
+      }
+    }
+    const float S = block_sum(s, red);
+    const float lse = M + logf(S);
+    const float scale = inv / S;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      int i = j * 512 + threadIdx.x;
+      if (i < nvec) {
+        float f[8];
+        unpack8(raw[j], f);
+        int c0 = i * 8;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) f[t] *= scale;
+        if (y >= c0 && y < c0 + 8) {
+          p.row_loss[row] = lse - zy;
+#pragma unroll
+          for (int t = 0; t < 8; ++t) if (c0 + t == y) f[t] -= inv;
+        }
+        z[i] = pack8(f);
+        if (p.colsum_part) {
+          float4 a = *(float4*)(csum + c0), b = *(float4*)(csum + c0 + 4);
+          a.x += f[0]; a.y += f[1]; a.z += f[2]; a.w += f[3];
+          b.x += f[4]; b.y += f[5]; b.z += f[6]; b.w += f[7];
+          *(float4*)(csum + c0) = a; *(float4*)(csum + c0 + 4) = b;
+        }
+      }
+    }
+  }
+  if (p.colsum_part) {
+    float* part = p.colsum_part + (size_t)blockIdx.x * p.classes;
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      int i = j * 512 + threadIdx.x;
+      if (i < nvec) { *(float4*)(part + i * 8) = *(float4*)(csum + i * 8); *(float4*)(part + i * 8 + 4) = *(float4*)(csum + i * 8 + 4); }
+    }
+  }
+}
+
 }  // namespace
 
 // d must equal nv*256 with nv in {1, 2, 4}; rows, scale and shift 16-byte aligned.
@@ -251,6 +362,22 @@ void launch_xent_vec(const XentProb* d, int n, int max_rows, int nv, cudaStream_
     case 8: xent_vec_kernel<2, 1024><<<grid, 1024, 0, s>>>(d); break;
     default: xent_vec_kernel<4, 1024><<<grid, 1024, 0, s>>>(d); break;
   }
+}
+
+void launch_xent_rows(const XentProb* d, int n, int max_rows, int classes, cudaStream_t s) {
+  dim3 grid((max_rows + XENT_ROWS - 1) / XENT_ROWS, n);
+  size_t smem = (size_t)classes * sizeof(float);
+  static bool set = false;
+  if (!set) {
+    cudaFuncSetAttribute(xent_rows_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
+    cudaFuncSetAttribute(xent_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * 4);
+    set = true;
+  }
+  int nv = (classes / 8 + 511) / 512;
+  if (nv <= 1) xent_rows_kernel<1><<<grid, 512, smem, s>>>(d);
+  else if (nv <= 2) xent_rows_kernel<2><<<grid, 512, smem, s>>>(d);
+  else if (nv <= 4) xent_rows_kernel<4><<<grid, 512, smem, s>>>(d);
+  else xent_rows_kernel<8><<<grid, 512, smem, s>>>(d);
 }
 
 }  // namespace lp

@@ -250,8 +250,9 @@ void emit_labels(Handle& h, Plan& p, const std::vector<LabelProb>& probs) {
   p.add(1, [=](const RunCtx& c) { launch_label_prep(d, n, st, c.stream); });
 }
 
-void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, const std::vector<int>& chunk_of) {
-  if (probs.empty()) return;
+bool emit_xent_and_loss(Handle& h, Plan& p, std::vector<XentProb> probs, const std::vector<int>& chunk_of,
+                        const std::vector<float*>* bias_grads) {
+  if (probs.empty()) return false;
   int mr = 0;
   std::vector<LossProb> lps;
   for (size_t i = 0; i < probs.size(); ++i) {
@@ -260,12 +261,7 @@ void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, 
   }
   double by = 0;
   for (auto& q : probs) by += 2.0 * q.rows * q.classes * h.esize();
-  const XentProb* d = h.upload(probs);
-  const LossProb* dl = h.upload(lps);
-  int n = (int)probs.size();
   bool bf = h.bf16_mode;
-  float* losses = h.d_losses;
-  int* st = h.d_status;
   int nv = 0;
   if (bf && probs[0].classes % 8 == 0 && probs[0].classes <= 32768) {
     nv = 1;
@@ -273,11 +269,28 @@ void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, 
     for (auto& q : probs)
       if (q.classes != probs[0].classes || q.ld % 8 != 0 || ((uintptr_t)q.z & 15)) nv = 0;
   }
+  // Long rows: blocks of XENT_ROWS rows with the next row prefetched, and the bias gradient on the way.
+  const bool rows_kernel = nv != 0 && probs[0].classes >= 2048;
+  const int classes = probs[0].classes;
+  if (rows_kernel && bias_grads) {
+    for (size_t i = 0; i < probs.size(); ++i) {
+      int nblk = (probs[i].rows + XENT_ROWS - 1) / XENT_ROWS;
+      probs[i].colsum_part = (float*)h.dalloc((size_t)nblk * classes * sizeof(float));
+      h.pending_reduce.push_back(ColReduceProb{probs[i].colsum_part, (*bias_grads)[i], nblk, classes, classes});
+    }
+  }
+  const XentProb* d = h.upload(probs);
+  const LossProb* dl = h.upload(lps);
+  int n = (int)probs.size();
+  float* losses = h.d_losses;
+  int* st = h.d_status;
   p.add(2, [=](const RunCtx& c) {
-    if (nv) launch_xent_vec(d, n, mr, nv, c.stream);
+    if (rows_kernel) launch_xent_rows(d, n, mr, classes, c.stream);
+    else if (nv) launch_xent_vec(d, n, mr, nv, c.stream);
     else launch_xent(d, n, mr, bf, c.stream);
     launch_loss_reduce(dl, n, losses, st, c.stream);
   }, KIND_XENT, by);
+  return rows_kernel && bias_grads;
 }
 
 void emit_optimizer(Handle& h, Plan& p) {

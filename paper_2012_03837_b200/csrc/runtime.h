@@ -133,7 +133,10 @@ void emit_ln_bwd(Handle& h, Plan& p, std::vector<LnBwdProb> probs, const std::ve
 void emit_colsum(Handle& h, Plan& p, const std::vector<ColSumProb>& probs_without_part, const std::vector<float*>& out);
 void emit_pending_reduce(Handle& h, Plan& p);
 void emit_labels(Handle& h, Plan& p, const std::vector<LabelProb>& probs);
-void emit_xent_and_loss(Handle& h, Plan& p, const std::vector<XentProb>& probs, const std::vector<int>& chunk_of);
+// bias_grads (optional, one pointer per problem): where the column sums of dlogits go.  Returns true if the
+// cross-entropy kernel produces them itself (then the caller needs no separate column-sum pass).
+bool emit_xent_and_loss(Handle& h, Plan& p, std::vector<XentProb> probs, const std::vector<int>& chunk_of,
+                        const std::vector<float*>* bias_grads = nullptr);
 void emit_optimizer(Handle& h, Plan& p);
 
 // GEMM problem constructors (x: [M,K] row-major, W: [N,K] row-major, dy: [M,N] row-major)
