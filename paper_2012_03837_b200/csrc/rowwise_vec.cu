@@ -216,32 +216,68 @@ __global__ void __launch_bounds__(NT) xent_vec_kernel(const XentProb* __restrict
 }
 
 // ------------------------------------------------------------------ cross-entropy over blocks of rows
-// One block of 512 threads walks XENT_ROWS consecutive rows; thread t owns the 8-column vectors
-// j*512 + t.  While the current row goes through its two block reductions, the next row is already
-// being loaded.  The column sums of the written dlogits (the head's bias gradient) are accumulated
-// on the way in shared memory (each thread only ever touches its own columns) and written once per
-// block, so the logits are read from HBM exactly once and written exactly once per step.
-template <int NV>
-__global__ void __launch_bounds__(512) xent_rows_kernel(const XentProb* __restrict__ probs) {
-  extern __shared__ float csum[];            // [classes]
-  __shared__ float red[33];
+// One block of NT threads walks XENT_ROWS consecutive rows; thread t owns the 8-column vectors
+// j*NT + t.  Per row: packed bf16 max over the thread's logits and a shuffle max over the warp; then
+// e = exp(z - warp max) (one exponential per logit; kept as bf16 in the registers that held z) and
+// its sum; the per-warp (max, sum) pairs are merged over the block through double-buffered shared
+// memory, so a row costs a single block barrier.  The next row is loaded while the current one is
+// reduced; labels and the logits at the labels are fetched once per block.  The label's "- 1/n" is
+// applied by the one thread that owns that column after the vector stores, which keeps the inner
+// loops free of label tests.  The column sums of the written dlogits (the head's bias gradient)
+// accumulate in shared memory (each thread only touches its own columns) and are written once per
+// block: the logits are read once and written once per step.
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float warp_max_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+template <int NV, int NT>
+__global__ void __launch_bounds__(NT) xent_rows_kernel(const XentProb* __restrict__ probs) {
+  // column sums, two planes of float4 per 8-column vector (conflict-free 16-byte lane stride):
+  // plane 0 = columns 8i..8i+3 at csum4[i], plane 1 = columns 8i+4..8i+7 at csum4[nvec + i]
+  extern __shared__ float4 csum4[];
+  __shared__ float2 wred[2][32];             // per-warp (max, sum), double-buffered by row parity
+  __shared__ int ys[XENT_ROWS];
+  __shared__ float zys[XENT_ROWS];
+  const float L2E = 1.4426950408889634f;
   const XentProb p = probs[blockIdx.y];
   const int r0 = blockIdx.x * XENT_ROWS;
   if (r0 >= p.rows) return;
   const int r1 = min(r0 + XENT_ROWS, p.rows);
   const int nvec = p.classes >> 3;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int NW = NT / 32;
   const float inv = 1.0f / (float)(*p.n_valid);
 #pragma unroll
   for (int j = 0; j < NV; ++j) {
-    int i = j * 512 + threadIdx.x;
-    if (i < nvec) { *(float4*)(csum + i * 8) = make_float4(0, 0, 0, 0); *(float4*)(csum + i * 8 + 4) = make_float4(0, 0, 0, 0); }
+    int i = j * NT + threadIdx.x;
+    if (i < nvec) { csum4[i] = make_float4(0, 0, 0, 0); csum4[nvec + i] = make_float4(0, 0, 0, 0); }
   }
   uint4 nxt[NV];
   {
     const uint4* z = (const uint4*)((const bf16*)p.z + (size_t)r0 * p.ld);
 #pragma unroll
-    for (int j = 0; j < NV; ++j) { int i = j * 512 + threadIdx.x; if (i < nvec) nxt[j] = z[i]; }
+    for (int j = 0; j < NV; ++j) { int i = j * NT + threadIdx.x; if (i < nvec) nxt[j] = z[i]; }
   }
+  if (threadIdx.x < r1 - r0) {
+    int y = p.y[r0 + threadIdx.x];
+    bool ok = y >= 0 && y < p.classes;
+    ys[threadIdx.x] = ok ? y : -1;
+    zys[threadIdx.x] = ok ? __bfloat162float(((const bf16*)p.z)[(size_t)(r0 + threadIdx.x) * p.ld + y]) : 0.f;
+  }
+  __syncthreads();
+  int par = 0;
   for (int row = r0; row < r1; ++row) {
     uint4 raw[NV];
 #pragma unroll
@@ -249,79 +285,83 @@ __global__ void __launch_bounds__(512) xent_rows_kernel(const XentProb* __restri
     if (row + 1 < r1) {
       const uint4* zn = (const uint4*)((const bf16*)p.z + (size_t)(row + 1) * p.ld);
 #pragma unroll
-      for (int j = 0; j < NV; ++j) { int i = j * 512 + threadIdx.x; if (i < nvec) nxt[j] = zn[i]; }
+      for (int j = 0; j < NV; ++j) { int i = j * NT + threadIdx.x; if (i < nvec) nxt[j] = zn[i]; }
     }
     uint4* z = (uint4*)((bf16*)p.z + (size_t)row * p.ld);
-    const int y = p.y[row];
-    if (!(y >= 0 && y < p.classes)) {          // ignored row: no loss, zero gradient (uniform over the block)
+    const int y = ys[row - r0];
+    if (y < 0) {                               // ignored row: no loss, zero gradient (uniform over the block)
 #pragma unroll
-      for (int j = 0; j < NV; ++j) { int i = j * 512 + threadIdx.x; if (i < nvec) z[i] = make_uint4(0, 0, 0, 0); }
+      for (int j = 0; j < NV; ++j) { int i = j * NT + threadIdx.x; if (i < nvec) z[i] = make_uint4(0, 0, 0, 0); }
       if (threadIdx.x == 0) p.row_loss[row] = 0.f;
       continue;
     }
-    float m = -INFINITY;
+    const float zy = zys[row - r0];
+    // max: packed bf16 over the thread's vectors, then over the warp
+    __nv_bfloat162 mx2 = __float2bfloat162_rn(-INFINITY);
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      int i = j * 512 + threadIdx.x;
+      int i = j * NT + threadIdx.x;
       if (i < nvec) {
-        float f[8];
-        unpack8(raw[j], f);
-#pragma unroll
-        for (int t = 0; t < 8; ++t) m = fmaxf(m, f[t]);
+        const __nv_bfloat162* h2 = (const __nv_bfloat162*)&raw[j];
+        mx2 = __hmax2(mx2, __hmax2(__hmax2(h2[0], h2[1]), __hmax2(h2[2], h2[3])));
       }
     }
-    const float M = block_max(m, red);
-    const float ML2 = M * 1.4426950408889634f;
-    float s = 0.f, zy = 0.f;
+    const float wm = warp_max_f(fmaxf(__low2float(mx2), __high2float(mx2)));   // -inf only for a warp without columns
+    const float wml = wm * L2E;
+    float st = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      int i = j * 512 + threadIdx.x;
+      int i = j * NT + threadIdx.x;
       if (i < nvec) {
         float f[8];
         unpack8(raw[j], f);
-        int c0 = i * 8;
-        if (y >= c0 && y < c0 + 8) {
 #pragma unroll
-          for (int t = 0; t < 8; ++t) if (c0 + t == y) zy = f[t];
-        }
-#pragma unroll
-        for (int t = 0; t < 8; ++t) { f[t] = exp2f(fmaf(f[t], 1.4426950408889634f, -ML2)); s += f[t]; }
+        for (int t = 0; t < 8; ++t) { f[t] = fast_exp2(fmaf(f[t], L2E, -wml)); st += f[t]; }
         raw[j] = pack8(f);
       }
     }
-    const float S = block_sum(s, red);
+    st = warp_sum_f(st);
+    if (lane == 0) wred[par][warp] = make_float2(wm, st);
+    __syncthreads();
+    const float2 v = lane < NW ? wred[par][lane] : make_float2(-INFINITY, 0.f);
+    par ^= 1;
+    const float M = warp_max_f(v.x);
+    const float S = warp_sum_f(v.x == -INFINITY ? 0.f : v.y * fast_exp2((v.x - M) * L2E));
     const float lse = M + logf(S);
-    const float scale = inv / S;
+    const float scale = wm == -INFINITY ? 0.f : fast_exp2((wm - M) * L2E) * inv / S;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      int i = j * 512 + threadIdx.x;
+      int i = j * NT + threadIdx.x;
       if (i < nvec) {
         float f[8];
         unpack8(raw[j], f);
-        int c0 = i * 8;
 #pragma unroll
         for (int t = 0; t < 8; ++t) f[t] *= scale;
-        if (y >= c0 && y < c0 + 8) {
-          p.row_loss[row] = lse - zy;
-#pragma unroll
-          for (int t = 0; t < 8; ++t) if (c0 + t == y) f[t] -= inv;
-        }
         z[i] = pack8(f);
         if (p.colsum_part) {
-          float4 a = *(float4*)(csum + c0), b = *(float4*)(csum + c0 + 4);
+          float4 a = csum4[i], b = csum4[nvec + i];
           a.x += f[0]; a.y += f[1]; a.z += f[2]; a.w += f[3];
           b.x += f[4]; b.y += f[5]; b.z += f[6]; b.w += f[7];
-          *(float4*)(csum + c0) = a; *(float4*)(csum + c0 + 4) = b;
+          csum4[i] = a; csum4[nvec + i] = b;
         }
       }
     }
+    if (threadIdx.x == ((y >> 3) % NT)) {      // the thread that owns the label's column
+      float ey = __bfloat162float(__float2bfloat16(fast_exp2(fmaf(zy, L2E, -wml))));
+      ((bf16*)z)[y] = __float2bfloat16(ey * scale - inv);
+      if (p.colsum_part) {
+        float* c = (float*)csum4 + (((y >> 2) & 1) ? (size_t)(nvec + (y >> 3)) * 4 : (size_t)(y >> 3) * 4) + (y & 3);
+        *c -= inv;
+      }
+    }
+    if (threadIdx.x == 0) p.row_loss[row] = lse - zy;
   }
   if (p.colsum_part) {
     float* part = p.colsum_part + (size_t)blockIdx.x * p.classes;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      int i = j * 512 + threadIdx.x;
-      if (i < nvec) { *(float4*)(part + i * 8) = *(float4*)(csum + i * 8); *(float4*)(part + i * 8 + 4) = *(float4*)(csum + i * 8 + 4); }
+      int i = j * NT + threadIdx.x;
+      if (i < nvec) { *(float4*)(part + i * 8) = csum4[i]; *(float4*)(part + i * 8 + 4) = csum4[nvec + i]; }
     }
   }
 }
@@ -369,15 +409,15 @@ void launch_xent_rows(const XentProb* d, int n, int max_rows, int classes, cudaS
   size_t smem = (size_t)classes * sizeof(float);
   static bool set = false;
   if (!set) {
-    cudaFuncSetAttribute(xent_rows_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
-    cudaFuncSetAttribute(xent_rows_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * 4);
+    cudaFuncSetAttribute(xent_rows_kernel<4, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
+    cudaFuncSetAttribute(xent_rows_kernel<2, 1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * 4);
     set = true;
   }
-  int nv = (classes / 8 + 511) / 512;
-  if (nv <= 1) xent_rows_kernel<1><<<grid, 512, smem, s>>>(d);
-  else if (nv <= 2) xent_rows_kernel<2><<<grid, 512, smem, s>>>(d);
-  else if (nv <= 4) xent_rows_kernel<4><<<grid, 512, smem, s>>>(d);
-  else xent_rows_kernel<8><<<grid, 512, smem, s>>>(d);
+  int nvec = classes / 8;
+  if (nvec <= 512) xent_rows_kernel<1, 512><<<grid, 512, smem, s>>>(d);
+  else if (nvec <= 1024) xent_rows_kernel<1, 1024><<<grid, 1024, smem, s>>>(d);
+  else if (nvec <= 2048) xent_rows_kernel<2, 1024><<<grid, 1024, smem, s>>>(d);
+  else xent_rows_kernel<4, 1024><<<grid, 1024, smem, s>>>(d);
 }
 
 }  // namespace lp
