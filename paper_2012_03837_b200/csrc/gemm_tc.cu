@@ -140,9 +140,34 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
   return d;
 }
 
+constexpr int RASTER = 8;   // row tiles per band of the tile walk
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+// Outputs are streamed: they leave with an evict-first L2 policy so that they do not push the
+// operand panels (re-read by the neighbouring tiles) out of the cache.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-               ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src)) : "memory");
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
+               ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src)), "l"(policy_evict_first()) : "memory");
+}
+// Tile t of a problem -> (row tile, column tile).  Tiles are walked in bands of RASTER row tiles,
+// row tile fastest inside a band, so that the tiles in flight at any time share a few operand
+// panels of each kind instead of one row panel and all column panels.
+__device__ __forceinline__ void tile_coords(const GemmProb& p, int t, int tile_m, int& mt, int& nt) {
+  const int tiles_m = (p.M + tile_m - 1) / tile_m;
+  const int band = t / (RASTER * p.tiles_n);
+  const int m_base = band * RASTER;
+  const int gm = min(RASTER, tiles_m - m_base);
+  const int r = t - band * (RASTER * p.tiles_n);
+  nt = r / gm;
+  mt = m_base + r - nt * gm;
 }
 
 // Fused epilogue for 32 consecutive columns (n0 ..) of one accumulator row (row m, held by this lane).
@@ -289,9 +314,10 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_caddr) {
 }
 // TMA load whose completion is signalled on a barrier given by cluster address (the pair leader's).
 __device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, int x, int y, uint32_t bar_caddr) {
+  // operand panels are re-read by the neighbouring tiles: keep them in L2 ahead of the streamed outputs
   asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_caddr) : "memory");
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_caddr), "l"(policy_evict_last()) : "memory");
 }
 __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {   // arrives on this barrier in both CTAs of the pair
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -352,8 +378,9 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
         const GemmProb& p = probs[pi];
         const CUtensorMap* mapA = maps + 4 * pi;
         const CUtensorMap* mapB = mapA + 1;
-        int t = tile - p.tile_start;
-        int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN + (int)rank * BNL;
+        int mt, nt;
+        tile_coords(p, tile - p.tile_start, TILE_M, mt, nt);
+        int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN + (int)rank * BNL;
         bool a_mn = p.a_ms == 1, b_mn = p.b_ns == 1;
         int kb_n = (p.K + BK - 1) / BK;
         for (int kb = 0; kb < kb_n; ++kb) {
@@ -447,8 +474,9 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
     for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
       while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
       const GemmProb p = probs[pi];
-      int t = tile - p.tile_start;
-      int m0 = (t / p.tiles_n) * TILE_M + (int)rank * BM, n0 = (t % p.tiles_n) * BN;
+      int mt, nt;
+      tile_coords(p, tile - p.tile_start, TILE_M, mt, nt);
+      int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN;
       int ab = it & 1;
       uint32_t use = (uint32_t)(it >> 1);
       ok = lane == 0 ? mbar_wait(&sh->tmem_full[ab], use & 1, sh, status) : true;   // one poller per warp

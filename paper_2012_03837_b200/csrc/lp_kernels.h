@@ -63,14 +63,16 @@ void launch_ln_bwd(const LnBwdProb* d_probs, int n, int max_rows, bool is_bf16, 
 struct ColReduceProb { // out[c] = sum_r in[r, c] over r < rows, for c < cols; in is fp32 [rows, ld]
   const float* in; float* out; int rows, cols, ld;
 };
-void launch_col_reduce_f32(const ColReduceProb* d_probs, int n, int max_cols, cudaStream_t s);
+// d_blocks[i] = (problem, block of 128 columns inside it): one thread block each
+void launch_col_reduce_f32(const ColReduceProb* d_probs, const int2* d_blocks, int n_blocks, cudaStream_t s);
 
 struct ColSumProb {   // part[blk, c] = sum over a block of rows of x[r, c]; x is [rows, ld]
   const void* x; float* part; int rows, cols, ld;
 };
 enum { COLSUM_ROWS = 128 };
+// vec8: bf16 with cols % 8 == 0, ld % 8 == 0 and 16-byte aligned x in every problem (128-bit loads)
 void launch_colsum_partial(const ColSumProb* d_probs, int n, int max_rows, int max_cols, bool is_bf16,
-                           cudaStream_t s);
+                           cudaStream_t s, bool vec8 = false);
 
 struct LabelProb {    // count valid labels, check range, (pipelined) carry labels to the next chunk
   const int* y; int* y_out; int rows; int classes; int* n_valid;

@@ -332,7 +332,7 @@ void build_lm(Handle& h) {
       for (int k : act)
         if (k == 0 && BJ(k) == 0) {
           EmbedBwdProb e{(const int*)h.x_in, cb[0].G0, h.G("c0.tok"), h.G("c0.pos"), emb_next, emb_first, M, T, d, V, B};
-          p.add(5, [e, bf](const RunCtx& c) { launch_embed_bwd(e, bf, c.stream); }, KIND_EMBED, (double)M * d * es + 4.0 * V * d);
+          p.add(6, [e, bf](const RunCtx& c) { launch_embed_bwd(e, bf, c.stream); }, KIND_EMBED, (double)M * d * es + 4.0 * V * d);
         }
     }
     emit_pending_reduce(h, p);

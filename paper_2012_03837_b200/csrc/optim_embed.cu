@@ -1,6 +1,8 @@
 // Fused multi-tensor optimizer update over the whole parameter arena (each chunk's parameters are
 // updated from that chunk's own gradients only, Sec. 1 / Sec. 6: the update is element-wise, so one
 // flat sweep applies all K per-chunk updates), and the token/position embedding of LM chunk 0.
+#include <climits>
+
 #include "common.cuh"
 
 namespace lp {
@@ -63,29 +65,33 @@ __global__ void __launch_bounds__(256) embed_fwd_kernel(EmbedProb p, int* status
   for (int c = threadIdx.x; c < p.d; c += blockDim.x) h[c] = from_f<T>(to_f(tok[c]) + to_f(pos[c]));
 }
 
-// next[i] = smallest j > i holding the same token id (or -1); first[] starts at 1 everywhere.
+// next[i] = smallest j > i holding the same token id (or -1); first[i] = 1 unless some earlier
+// position holds the same id.  Three steps: reset, one block per (tile of i, later tile of j) that
+// takes an atomic minimum over the matches it finds (a minimum does not depend on the order of
+// its arguments, so the result is deterministic), then the successors are marked.
+__global__ void __launch_bounds__(256) embed_link_init_kernel(EmbedBwdProb p) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < p.rows) { p.next[i] = INT_MAX; p.first[i] = 1; }
+}
 __global__ void __launch_bounds__(256) embed_link_kernel(EmbedBwdProb p) {
   __shared__ int tile[256];
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  int my = i < p.rows ? min(max(p.ids[i], 0), p.vocab - 1) : -1;
-  int nxt = -1;
-  for (int j0 = blockIdx.x * blockDim.x; j0 < p.rows; j0 += blockDim.x) {
-    __syncthreads();
-    int j = j0 + threadIdx.x;
-    tile[threadIdx.x] = j < p.rows ? min(max(p.ids[j], 0), p.vocab - 1) : -2;
-    __syncthreads();
-    if (nxt < 0 && my >= 0) {
-      for (int t = 0; t < blockDim.x; ++t) {
-        int jj = j0 + t;
-        if (jj > i && tile[t] == my) { nxt = jj; break; }
-      }
-    }
+  if (blockIdx.x < blockIdx.y) return;         // only tiles of j at or after the tile of i
+  const int i = blockIdx.y * 256 + threadIdx.x, j0 = blockIdx.x * 256;
+  const int j = j0 + threadIdx.x;
+  tile[threadIdx.x] = j < p.rows ? min(max(p.ids[j], 0), p.vocab - 1) : -2;
+  const int my = i < p.rows ? min(max(p.ids[i], 0), p.vocab - 1) : -1;
+  __syncthreads();
+  if (my < 0) return;
+  for (int t = 0; t < 256; ++t) {
+    if (tile[t] == my && j0 + t > i) { atomicMin(&p.next[i], j0 + t); break; }
   }
-  if (i < p.rows) { p.next[i] = nxt; p.first[i] = 1; }
 }
 __global__ void __launch_bounds__(256) embed_mark_kernel(EmbedBwdProb p) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < p.rows && p.next[i] >= 0) p.first[p.next[i]] = 0;
+  if (i >= p.rows) return;
+  int n = p.next[i];
+  if (n == INT_MAX) p.next[i] = -1;
+  else p.first[n] = 0;
 }
 // One block per position: the first holder of a token id sums dh over the chain of positions
 // holding that id, in increasing position order (deterministic), and writes the table row.
@@ -127,7 +133,8 @@ void launch_embed_fwd(const EmbedProb& p, int* d_status, bool is_bf16, cudaStrea
 
 void launch_embed_bwd(const EmbedBwdProb& p, bool is_bf16, cudaStream_t s) {
   int nb = (p.rows + 255) / 256;
-  embed_link_kernel<<<nb, 256, 0, s>>>(p);
+  embed_link_init_kernel<<<nb, 256, 0, s>>>(p);
+  embed_link_kernel<<<dim3(nb, nb), 256, 0, s>>>(p);
   embed_mark_kernel<<<nb, 256, 0, s>>>(p);
   cudaMemsetAsync(p.dtok, 0, (size_t)p.vocab * p.d * sizeof(float), s);
   if (is_bf16) {

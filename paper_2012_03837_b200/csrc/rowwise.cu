@@ -75,13 +75,53 @@ __global__ void __launch_bounds__(256) ln_bwd_kernel(const LnBwdProb* __restrict
 }
 
 // ------------------------------------------------------------------ column reductions
-__global__ void __launch_bounds__(256) col_reduce_kernel(const ColReduceProb* __restrict__ probs) {
-  const ColReduceProb p = probs[blockIdx.y];
-  int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= p.cols) return;
-  float s = 0.f;
-  for (int r = 0; r < p.rows; ++r) s += p.in[(size_t)r * p.ld + c];
-  p.out[c] = s;
+// Block = 32 column lanes x 8 row lanes.  A row lane sums every 8th row with four independent
+// loads in flight; the 8 row lanes are then added in lane order through shared memory, so the sum
+// of a column always has the same order.  A column lane covers 4 (fp32) or 8 (bf16) adjacent
+// columns with one 128-bit load when the matrix allows it, one column otherwise.
+__global__ void __launch_bounds__(256) col_reduce_kernel(const ColReduceProb* __restrict__ probs, const int2* __restrict__ blocks) {
+  __shared__ float4 red[8][32];
+  const int2 blk = blocks[blockIdx.x];
+  const ColReduceProb p = probs[blk.x];
+  const int bx = blk.y;
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const bool vec = (p.cols % 4 == 0) && (p.ld % 4 == 0) && (((uintptr_t)p.in & 15) == 0);
+  if (vec) {
+    const int c = (bx * 32 + cx) * 4;
+    float4 s = make_float4(0, 0, 0, 0);
+    if (c < p.cols) {
+      const float* base = p.in + c;
+      int r = ry;
+      for (; r + 24 < p.rows; r += 32) {
+        float4 a0 = *(const float4*)(base + (size_t)r * p.ld), a1 = *(const float4*)(base + (size_t)(r + 8) * p.ld);
+        float4 a2 = *(const float4*)(base + (size_t)(r + 16) * p.ld), a3 = *(const float4*)(base + (size_t)(r + 24) * p.ld);
+        s.x += a0.x; s.y += a0.y; s.z += a0.z; s.w += a0.w;
+        s.x += a1.x; s.y += a1.y; s.z += a1.z; s.w += a1.w;
+        s.x += a2.x; s.y += a2.y; s.z += a2.z; s.w += a2.w;
+        s.x += a3.x; s.y += a3.y; s.z += a3.z; s.w += a3.w;
+      }
+      for (; r < p.rows; r += 8) {
+        float4 a0 = *(const float4*)(base + (size_t)r * p.ld);
+        s.x += a0.x; s.y += a0.y; s.z += a0.z; s.w += a0.w;
+      }
+    }
+    red[ry][cx] = s;
+    __syncthreads();
+    if (ry == 0 && c < p.cols) {
+#pragma unroll
+      for (int k = 1; k < 8; ++k) { float4 a = red[k][cx]; s.x += a.x; s.y += a.y; s.z += a.z; s.w += a.w; }
+      if (((uintptr_t)p.out & 15) == 0) *(float4*)(p.out + c) = s;
+      else { p.out[c] = s.x; p.out[c + 1] = s.y; p.out[c + 2] = s.z; p.out[c + 3] = s.w; }
+    }
+  } else {
+    // one column per thread, 128 columns per block
+    if (threadIdx.x >= 128) return;
+    const int c = bx * 128 + threadIdx.x;
+    if (c >= p.cols) return;
+    float s = 0.f;
+    for (int r = 0; r < p.rows; ++r) s += p.in[(size_t)r * p.ld + c];
+    p.out[c] = s;
+  }
 }
 
 template <typename T>
@@ -96,6 +136,46 @@ __global__ void __launch_bounds__(256) colsum_partial_kernel(const ColSumProb* _
   float s = 0.f;
   for (int r = r0; r < r1; ++r) s += to_f(x[(size_t)r * p.ld + c]);
   p.part[(size_t)blockIdx.y * p.cols + c] = s;
+}
+
+// bf16, cols % 8 == 0, ld % 8 == 0, 16-byte aligned x: 256 columns x COLSUM_ROWS rows per block
+__global__ void __launch_bounds__(256) colsum_partial_vec_kernel(const ColSumProb* __restrict__ probs) {
+  __shared__ float red[8][32][9];
+  const ColSumProb p = probs[blockIdx.z];
+  const int r0 = blockIdx.y * COLSUM_ROWS;
+  if (r0 >= p.rows || (int)blockIdx.x * 256 >= p.cols) return;
+  const int r1 = min(r0 + COLSUM_ROWS, p.rows);
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int c = (blockIdx.x * 32 + cx) * 8;
+  float s[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) s[t] = 0.f;
+  auto acc = [&](uint4 u) {
+    const __nv_bfloat162* h = (const __nv_bfloat162*)&u;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) { float2 f = __bfloat1622float2(h[t]); s[2 * t] += f.x; s[2 * t + 1] += f.y; }
+  };
+  if (c < p.cols) {
+    const bf16* base = (const bf16*)p.x + c;
+    int r = r0 + ry;
+    for (; r + 24 < r1; r += 32) {
+      uint4 a0 = *(const uint4*)(base + (size_t)r * p.ld), a1 = *(const uint4*)(base + (size_t)(r + 8) * p.ld);
+      uint4 a2 = *(const uint4*)(base + (size_t)(r + 16) * p.ld), a3 = *(const uint4*)(base + (size_t)(r + 24) * p.ld);
+      acc(a0); acc(a1); acc(a2); acc(a3);
+    }
+    for (; r < r1; r += 8) acc(*(const uint4*)(base + (size_t)r * p.ld));
+  }
+#pragma unroll
+  for (int t = 0; t < 8; ++t) red[ry][cx][t] = s[t];
+  __syncthreads();
+  // thread -> one column of the block's 256: add the 8 row lanes in order
+  const int col = threadIdx.x, gc = blockIdx.x * 256 + col;
+  if (gc < p.cols) {
+    float v = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v += red[k][col >> 3][col & 7];
+    p.part[(size_t)blockIdx.y * p.cols + gc] = v;
+  }
 }
 
 // ------------------------------------------------------------------ labels
@@ -187,13 +267,13 @@ void launch_ln_bwd(const LnBwdProb* d, int n, int max_rows, bool is_bf16, cudaSt
   dim3 grid((max_rows + LN_BWD_ROWS - 1) / LN_BWD_ROWS, n);
   DISPATCH_T(is_bf16, ln_bwd_kernel, grid, 256, s, d);
 }
-void launch_col_reduce_f32(const ColReduceProb* d, int n, int max_cols, cudaStream_t s) {
-  dim3 grid((max_cols + 255) / 256, n);
-  col_reduce_kernel<<<grid, 256, 0, s>>>(d);
+void launch_col_reduce_f32(const ColReduceProb* d, const int2* blocks, int n_blocks, cudaStream_t s) {
+  if (n_blocks > 0) col_reduce_kernel<<<n_blocks, 256, 0, s>>>(d, blocks);
 }
-void launch_colsum_partial(const ColSumProb* d, int n, int max_rows, int max_cols, bool is_bf16, cudaStream_t s) {
+void launch_colsum_partial(const ColSumProb* d, int n, int max_rows, int max_cols, bool is_bf16, cudaStream_t s, bool vec8) {
   dim3 grid((max_cols + 255) / 256, (max_rows + COLSUM_ROWS - 1) / COLSUM_ROWS, n);
-  DISPATCH_T(is_bf16, colsum_partial_kernel, grid, 256, s, d);
+  if (is_bf16 && vec8) colsum_partial_vec_kernel<<<grid, 256, 0, s>>>(d);
+  else DISPATCH_T(is_bf16, colsum_partial_kernel, grid, 256, s, d);
 }
 void launch_label_prep(const LabelProb* d, int n, int* d_status, cudaStream_t s) {
   label_prep_kernel<<<n, 256, 0, s>>>(d, d_status);

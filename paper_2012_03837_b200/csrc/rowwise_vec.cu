@@ -21,121 +21,171 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 }
 
 // ------------------------------------------------------------------ LayerNorm forward
-// Warp per row; lane owns the 8-element vectors j*32 + lane, j < NV (d = NV * 256).
+// Block = 8 warps over LN_FWD_ROWS rows (warp w takes rows w, w+8, ...); a lane owns the 8-element
+// vectors j*32 + lane, j < NV (d = NV * 256).  The warp's next row is loaded while the current one
+// is normalised.
+enum { LN_FWD_ROWS = 32 };
 template <int NV>
 __global__ void __launch_bounds__(256) ln_fwd_vec_kernel(const LnProb* __restrict__ probs) {
   const LnProb p = probs[blockIdx.y];
-  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  int row = blockIdx.x * 8 + w;
-  if (row >= p.rows) return;
-  const uint4* x = (const uint4*)((const bf16*)p.x + (size_t)row * p.d);
-  float v[NV][8];
-  float s = 0.f;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int r0 = blockIdx.x * LN_FWD_ROWS;
+  if (r0 >= p.rows) return;
+  const int r1 = min(r0 + LN_FWD_ROWS, p.rows);
+  const float inv_d = 1.0f / p.d;
+  uint4 nxt[NV];
+  if (r0 + w < r1) {
+    const uint4* x = (const uint4*)((const bf16*)p.x + (size_t)(r0 + w) * p.d);
 #pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    unpack8(x[j * 32 + lane], v[j]);
-#pragma unroll
-    for (int t = 0; t < 8; ++t) s += v[j][t];
+    for (int j = 0; j < NV; ++j) nxt[j] = x[j * 32 + lane];
   }
-  float mu = warp_sum(s) / p.d;
-  float q = 0.f;
+  for (int row = r0 + w; row < r1; row += 8) {
+    float v[NV][8];
+    float s = 0.f;
 #pragma unroll
-  for (int j = 0; j < NV; ++j)
+    for (int j = 0; j < NV; ++j) {
+      unpack8(nxt[j], v[j]);
 #pragma unroll
-    for (int t = 0; t < 8; ++t) { float c = v[j][t] - mu; q += c * c; }
-  float rstd = rsqrtf(warp_sum(q) / p.d + 1e-5f);
-  uint4* y = (uint4*)((bf16*)p.y + (size_t)row * p.d);
+      for (int t = 0; t < 8; ++t) s += v[j][t];
+    }
+    if (row + 8 < r1) {
+      const uint4* x = (const uint4*)((const bf16*)p.x + (size_t)(row + 8) * p.d);
 #pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    int c0 = (j * 32 + lane) * 8;
-    float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
-    float4 b0 = *(const float4*)(p.b + c0), b1 = *(const float4*)(p.b + c0 + 4);
-    float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-    float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-    float o[8];
+      for (int j = 0; j < NV; ++j) nxt[j] = x[j * 32 + lane];
+    }
+    float mu = warp_sum(s) * inv_d;
+    float q = 0.f;
 #pragma unroll
-    for (int t = 0; t < 8; ++t) o[t] = (v[j][t] - mu) * rstd * g[t] + b[t];
-    y[j * 32 + lane] = pack8(o);
+    for (int j = 0; j < NV; ++j)
+#pragma unroll
+      for (int t = 0; t < 8; ++t) { float c = v[j][t] - mu; q += c * c; }
+    float rstd = rsqrtf(warp_sum(q) * inv_d + 1e-5f);
+    uint4* y = (uint4*)((bf16*)p.y + (size_t)row * p.d);
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+      int c0 = (j * 32 + lane) * 8;
+      float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
+      float4 b0 = *(const float4*)(p.b + c0), b1 = *(const float4*)(p.b + c0 + 4);
+      float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+      float o[8];
+#pragma unroll
+      for (int t = 0; t < 8; ++t) o[t] = (v[j][t] - mu) * rstd * g[t] + b[t];
+      y[j * 32 + lane] = pack8(o);
+    }
+    if (lane == 0) { p.mean[row] = mu; p.rstd[row] = rstd; }
   }
-  if (lane == 0) { p.mean[row] = mu; p.rstd[row] = rstd; }
 }
 
 // ------------------------------------------------------------------ LayerNorm backward
-// Block = 8 warps over LN_BWD_ROWS rows (warp w takes rows w, w+8, ...).  Each lane accumulates
-// the scale/shift gradient of its own columns over the warp's rows in registers; the 8 warps are
-// then summed through shared memory in warp order and the block writes one partial row.
+// Block = 8 warps over LN_BWD_ROWS rows (warp w takes rows w, w+8, ...).  Each warp streams its
+// rows of x and dy (and of the residual-path gradient) through its own three-deep ring of
+// shared-memory buffers filled by cp.async, so two rows are in flight while one is reduced.  Each
+// lane accumulates the scale/shift gradient of its own columns over the warp's rows in registers;
+// the 8 warps are then summed through shared memory in warp order and the block writes one
+// partial row.
+enum { LN_RING = 3 };
+__device__ __forceinline__ void cp_async_16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src));
+}
 template <int NV>
 __global__ void __launch_bounds__(256) ln_bwd_vec_kernel(const LnBwdProb* __restrict__ probs) {
-  extern __shared__ float red[];   // [8][2][d]
+  extern __shared__ __align__(16) float red[];   // [8][2][d] floats, then the rings: [8 warps][LN_RING][3][d] bf16
   const LnBwdProb p = probs[blockIdx.y];
   int r0 = blockIdx.x * LN_BWD_ROWS;
   if (r0 >= p.rows) return;
   int r1 = min(r0 + LN_BWD_ROWS, p.rows);
   int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  float ag[NV][8], ab[NV][8], g[NV][8];
+  constexpr int D = NV * 256;
+  uint4* ring = (uint4*)(red + 8 * 2 * D) + (size_t)w * LN_RING * 3 * (D / 8);
+  const bool has_res = p.dx && p.dres;
+  auto fetch = [&](int row, int slot) {
+    if (row < r1) {
+      const uint4* x = (const uint4*)((const bf16*)p.x + (size_t)row * D);
+      const uint4* dy = (const uint4*)((const bf16*)p.dy + (size_t)row * D);
+      uint4* dst = ring + (size_t)slot * 3 * (D / 8);
 #pragma unroll
-  for (int j = 0; j < NV; ++j) {
-    int c0 = (j * 32 + lane) * 8;
-    float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
-    g[j][0] = g0.x; g[j][1] = g0.y; g[j][2] = g0.z; g[j][3] = g0.w;
-    g[j][4] = g1.x; g[j][5] = g1.y; g[j][6] = g1.z; g[j][7] = g1.w;
+      for (int j = 0; j < NV; ++j) {
+        cp_async_16(dst + j * 32 + lane, x + j * 32 + lane);
+        cp_async_16(dst + D / 8 + j * 32 + lane, dy + j * 32 + lane);
+      }
+      if (has_res) {
+        const uint4* dr = (const uint4*)((const bf16*)p.dres + (size_t)row * D);
+#pragma unroll
+        for (int j = 0; j < NV; ++j) cp_async_16(dst + 2 * (D / 8) + j * 32 + lane, dr + j * 32 + lane);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  float ag[NV][8], ab[NV][8];
+#pragma unroll
+  for (int j = 0; j < NV; ++j)
 #pragma unroll
     for (int t = 0; t < 8; ++t) { ag[j][t] = 0.f; ab[j][t] = 0.f; }
-  }
+  fetch(r0 + w, 0);
+  fetch(r0 + w + 8, 1);
+  int slot = 0;
+  const float inv_d = 1.0f / D;
   for (int row = r0 + w; row < r1; row += 8) {
-    const uint4* dy = (const uint4*)((const bf16*)p.dy + (size_t)row * p.d);
-    const uint4* x = (const uint4*)((const bf16*)p.x + (size_t)row * p.d);
+    fetch(row + 16, slot == 0 ? 2 : slot - 1);      // the slot freed by the previous row
+    asm volatile("cp.async.wait_group 2;" ::: "memory");
+    __syncwarp();
+    const uint4* buf = ring + (size_t)slot * 3 * (D / 8);
     float mu = p.mean[row], rs = p.rstd[row];
     float xh[NV][8], dv[NV][8];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      unpack8(x[j * 32 + lane], xh[j]);
-      unpack8(dy[j * 32 + lane], dv[j]);
+      int c0 = (j * 32 + lane) * 8;
+      float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
+      float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      unpack8(buf[j * 32 + lane], xh[j]);
+      unpack8(buf[D / 8 + j * 32 + lane], dv[j]);
 #pragma unroll
       for (int t = 0; t < 8; ++t) {
         xh[j][t] = (xh[j][t] - mu) * rs;
         ag[j][t] += dv[j][t] * xh[j][t];
         ab[j][t] += dv[j][t];
-        float dxh = dv[j][t] * g[j][t];
-        s1 += dxh;
-        s2 += dxh * xh[j][t];
+        dv[j][t] *= g[t];                             // from here on: gradient w.r.t. the normalised value
+        s1 += dv[j][t];
+        s2 += dv[j][t] * xh[j][t];
       }
     }
     if (p.dx) {
-      s1 = warp_sum(s1) / p.d;
-      s2 = warp_sum(s2) / p.d;
-      uint4* dx = (uint4*)((bf16*)p.dx + (size_t)row * p.d);
-      const uint4* dres = p.dres ? (const uint4*)((const bf16*)p.dres + (size_t)row * p.d) : nullptr;
+      s1 = warp_sum(s1) * inv_d;
+      s2 = warp_sum(s2) * inv_d;
+      uint4* dx = (uint4*)((bf16*)p.dx + (size_t)row * D);
 #pragma unroll
       for (int j = 0; j < NV; ++j) {
         float o[8], r[8];
-        if (dres) unpack8(dres[j * 32 + lane], r);
+        if (has_res) unpack8(buf[2 * (D / 8) + j * 32 + lane], r);
 #pragma unroll
         for (int t = 0; t < 8; ++t) {
-          o[t] = rs * (dv[j][t] * g[j][t] - s1 - xh[j][t] * s2);
-          if (dres) o[t] += r[t];
+          o[t] = rs * (dv[j][t] - s1 - xh[j][t] * s2);
+          if (has_res) o[t] += r[t];
         }
         dx[j * 32 + lane] = pack8(o);
       }
     }
+    __syncwarp();                                     // all lanes are done with this slot before it is refilled
+    slot = slot == LN_RING - 1 ? 0 : slot + 1;
   }
-  const int d = p.d;
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
   for (int j = 0; j < NV; ++j) {
     int c0 = (j * 32 + lane) * 8;
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
-      red[(w * 2 + 0) * d + c0 + t] = ag[j][t];
-      red[(w * 2 + 1) * d + c0 + t] = ab[j][t];
+      red[(w * 2 + 0) * D + c0 + t] = ag[j][t];
+      red[(w * 2 + 1) * D + c0 + t] = ab[j][t];
     }
   }
   __syncthreads();
-  float* part = p.part + (size_t)blockIdx.x * 2 * d;
-  for (int c = threadIdx.x; c < 2 * d; c += blockDim.x) {
+  float* part = p.part + (size_t)blockIdx.x * 2 * D;
+  for (int c = threadIdx.x; c < 2 * D; c += blockDim.x) {
     float s = 0.f;
 #pragma unroll
-    for (int ww = 0; ww < 8; ++ww) s += red[ww * 2 * d + c];
+    for (int ww = 0; ww < 8; ++ww) s += red[ww * 2 * D + c];
     part[c] = s;
   }
 }
@@ -370,7 +420,7 @@ __global__ void __launch_bounds__(NT) xent_rows_kernel(const XentProb* __restric
 
 // d must equal nv*256 with nv in {1, 2, 4}; rows, scale and shift 16-byte aligned.
 void launch_ln_fwd_vec(const LnProb* d, int n, int max_rows, int nv, cudaStream_t s) {
-  dim3 grid((max_rows + 7) / 8, n);
+  dim3 grid((max_rows + LN_FWD_ROWS - 1) / LN_FWD_ROWS, n);
   switch (nv) {
     case 1: ln_fwd_vec_kernel<1><<<grid, 256, 0, s>>>(d); break;
     case 2: ln_fwd_vec_kernel<2><<<grid, 256, 0, s>>>(d); break;
@@ -379,10 +429,14 @@ void launch_ln_fwd_vec(const LnProb* d, int n, int max_rows, int nv, cudaStream_
 }
 void launch_ln_bwd_vec(const LnBwdProb* d, int n, int max_rows, int nv, cudaStream_t s) {
   dim3 grid((max_rows + LN_BWD_ROWS - 1) / LN_BWD_ROWS, n);
-  size_t smem = (size_t)8 * 2 * nv * 256 * sizeof(float);
+  // [8][2][d] fp32 for the final reduction + 8 warps x LN_RING slots x 3 rows of d bf16
+  auto bytes = [](int v) { return (size_t)8 * 2 * v * 256 * sizeof(float) + (size_t)8 * LN_RING * 3 * v * 256 * 2; };
+  size_t smem = bytes(nv == 1 || nv == 2 ? nv : 4);
   static bool set = false;
   if (!set) {
-    cudaFuncSetAttribute(ln_bwd_vec_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 2 * 4 * 256 * 4);
+    cudaFuncSetAttribute(ln_bwd_vec_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes(1));
+    cudaFuncSetAttribute(ln_bwd_vec_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes(2));
+    cudaFuncSetAttribute(ln_bwd_vec_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes(4));
     set = true;
   }
   switch (nv) {

@@ -106,11 +106,13 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
   {
     std::vector<GemmProb> expanded;
     const size_t es = h.esize();
+    long long launch_tiles = 0;   // of the whole grouped launch: the other problems keep the SMs busy too
+    for (auto& g : probs) launch_tiles += (long long)((g.M + 127) / 128) * ((g.N + 255) / 256);
     for (auto& g : probs) {
       bool plain = g.out_f32 && g.act == EPI_NONE && !g.bias && !g.resid && g.ldc == g.N;
-      long long tiles = (long long)((g.M + 127) / 128) * ((g.N + 255) / 256);
       long long S = 1;
-      if (plain && g.K >= 8192 && tiles * 2 <= h.num_sms) S = std::max(1LL, std::min<long long>({h.num_sms / tiles, g.K / 2048LL, 64LL}));
+      if (plain && g.K >= 8192 && launch_tiles * 2 <= h.num_sms)
+        S = std::max(1LL, std::min<long long>({h.num_sms / launch_tiles, g.K / 2048LL, 64LL}));
       if (S == 1) { expanded.push_back(g); continue; }
       size_t mn = (size_t)g.M * g.N;
       float* part = (float*)h.dalloc((size_t)S * mn * sizeof(float));
@@ -227,20 +229,27 @@ void emit_colsum(Handle& h, Plan& p, const std::vector<ColSumProb>& in, const st
   int n = (int)probs.size();
   bool bf = h.bf16_mode;
   double by = 0;
-  for (auto& q : probs) by += (double)q.rows * q.cols * h.esize();
-  p.add(1, [=](const RunCtx& c) { launch_colsum_partial(d, n, mr, mc, bf, c.stream); }, KIND_REDUCE, by);
+  bool vec8 = bf;
+  for (auto& q : probs) {
+    by += (double)q.rows * q.cols * h.esize();
+    if (q.cols % 8 || q.ld % 8 || ((uintptr_t)q.x & 15)) vec8 = false;
+  }
+  p.add(1, [=](const RunCtx& c) { launch_colsum_partial(d, n, mr, mc, bf, c.stream, vec8); }, KIND_REDUCE, by);
 }
 
 void emit_pending_reduce(Handle& h, Plan& p) {
   if (h.pending_reduce.empty()) return;
-  int mc = 0;
-  for (auto& q : h.pending_reduce) mc = std::max(mc, q.cols);
+  // flat list of blocks: (problem, block of 128 columns inside it)
+  std::vector<int2> blocks;
+  for (size_t i = 0; i < h.pending_reduce.size(); ++i)
+    for (int b = 0; b * 128 < h.pending_reduce[i].cols; ++b) blocks.push_back(make_int2((int)i, b));
   const ColReduceProb* d = h.upload(h.pending_reduce);
-  int n = (int)h.pending_reduce.size();
+  const int2* db = h.upload(blocks);
+  int nb = (int)blocks.size();
   double by = 0;
   for (auto& q : h.pending_reduce) by += (double)q.rows * q.cols * 4;
   h.pending_reduce.clear();
-  p.add(1, [=](const RunCtx& c) { launch_col_reduce_f32(d, n, mc, c.stream); }, KIND_REDUCE, by);
+  p.add(1, [=](const RunCtx& c) { launch_col_reduce_f32(d, db, nb, c.stream); }, KIND_REDUCE, by);
 }
 
 void emit_labels(Handle& h, Plan& p, const std::vector<LabelProb>& probs) {
