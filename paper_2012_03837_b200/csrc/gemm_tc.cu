@@ -177,7 +177,8 @@ __device__ __forceinline__ void tile_coords(const GemmProb& p, int t, int tile_m
 // VEC: all 32 columns exist and resid / aux / C are 16-byte aligned (128-bit accesses).
 template <bool VEC>
 __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensorMap* mapC, const CUtensorMap* mapC2,
-                                               uint8_t* stg, int m, int m_warp0, int n0, const uint32_t* acc, int lane) {
+                                               uint8_t* stg, int m, int m_warp0, int n0, const uint32_t* acc, int lane,
+                                               int chunk) {
   float v[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
@@ -208,7 +209,31 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
   };
   // one output block (bf16 or fp32) of this warp
   auto put = [&](void* base, const CUtensorMap* map, const float* o, bool f32) {
-    if (stg) {
+    if (stg && p.store_tma == 2) {
+      // bf16, two neighbouring 32-column blocks share one store of 128-byte rows: the even block
+      // fills 16-byte units 0-3 of every row, the odd one units 4-7 (128-byte swizzle)
+      const int half = chunk & 1;
+      if (half == 0) {
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint4 u;
+        __nv_bfloat162* h = (__nv_bfloat162*)&u;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(o[q * 8 + 2 * t], o[q * 8 + 2 * t + 1]);
+        *(uint4*)(stg + lane * 128 + (((half * 4 + q) ^ (lane & 7)) << 4)) = u;
+      }
+      if (half == 1 || n0 + 32 >= p.N) {          // the pair is complete (or has no second block)
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(map, n0 - half * 32, m_warp0, stg);
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+      }
+    } else if (stg) {
       if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging buffer free again
       __syncwarp();
       if (f32) {
@@ -496,8 +521,8 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       auto emit = [&](const uint32_t* a, int c) {
         const int nc = n0 + col0 + c * 32;
         if (nc >= p.N || m_warp0 >= p.M) return;            // warp-uniform
-        if (vec_ok && nc + 32 <= p.N) epilogue_row32<true>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane);
-        else epilogue_row32<false>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane);
+        if (vec_ok && nc + 32 <= p.N) epilogue_row32<true>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c);
+        else epilogue_row32<false>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c);
       };
       uint32_t acc0[32], acc1[32];
       tc_ld32(trow, acc0);
@@ -593,15 +618,17 @@ int gemm_tc_tiles(GemmProb& g, int tile_start, int cg) {
 
 // Output map: [M, N] with a pitch of ldc elements, 32x32 boxes, swizzled like the epilogue's staging buffer
 // (64-byte rows for bf16, 128-byte rows for fp32).
-bool encode_out_map(CUtensorMap* out, const void* base, long long N, long long M, long long ldc, bool f32) {
+// `wide`: bf16 boxes of 64 columns (128-byte rows, 128-byte swizzle) filled by two neighbouring column blocks.
+bool encode_out_map(CUtensorMap* out, const void* base, long long N, long long M, long long ldc, bool f32, bool wide) {
   EncodeFn fn = get_encode();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
   cuuint64_t strides[1] = {(cuuint64_t)ldc * (f32 ? 4 : 2)};
-  cuuint32_t box[2] = {32u, 32u};
+  cuuint32_t box[2] = {wide ? 64u : 32u, 32u};
   cuuint32_t estr[2] = {1u, 1u};
   CUresult r = fn(out, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
-                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  (f32 || wide) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -614,9 +641,11 @@ bool gemm_tc_encode(GemmProb& g, void* maps, int cg) {
   g.store_tma = ((g.ldc * esz) % 16 == 0) && (((uintptr_t)g.C & 15) == 0) &&
                 (g.act != EPI_GELU || (((uintptr_t)g.C2 & 15) == 0 && (g.ldc * 2) % 16 == 0));
   if (g.store_tma) {
-    bool ok = encode_out_map(mapA + 2, g.C, g.N, g.M, g.ldc, g.out_f32 != 0);
-    if (ok && g.act == EPI_GELU) ok = encode_out_map(mapA + 3, g.C2, g.N, g.M, g.ldc, false);
-    if (!ok) g.store_tma = 0;
+    // one bf16 output: pairs of column blocks leave in one store of full 128-byte rows (mode 2)
+    const bool wide = !g.out_f32 && g.act != EPI_GELU;
+    bool ok = encode_out_map(mapA + 2, g.C, g.N, g.M, g.ldc, g.out_f32 != 0, wide);
+    if (ok && g.act == EPI_GELU) ok = encode_out_map(mapA + 3, g.C2, g.N, g.M, g.ldc, false, false);
+    g.store_tma = ok ? (wide ? 2 : 1) : 0;
   }
   bool okA, okB;
   if (g.a_ms == 1) okA = encode_map(mapA, g.A, g.M, g.K, g.a_ks, BK);       // MN-major: rows are k

@@ -281,15 +281,19 @@ __device__ __forceinline__ float fast_exp2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Warp reductions in one instruction each.  The maximum is the hardware's fp32 reduction; the sum
+// goes through fixed point (integer adds: exact and order-free), `scale` being a power of two that
+// keeps the warp's total below 2^32.  A non-finite addend makes the result NaN.
 __device__ __forceinline__ float warp_max_f(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
+  float m;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(m) : "f"(v));
+  return m;
 }
-__device__ __forceinline__ float warp_sum_f(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
+__device__ __forceinline__ float warp_sum_fixed(float v, float scale, float inv_scale) {
+  unsigned q = __float2uint_rn(v * scale), bad = (v >= 0.f && v <= 3.0e38f) ? 0u : 1u, s, b;
+  asm volatile("redux.sync.add.u32 %0, %1, 0xffffffff;" : "=r"(s) : "r"(q));
+  asm volatile("redux.sync.or.b32 %0, %1, 0xffffffff;" : "=r"(b) : "r"(bad));
+  return b ? __int_as_float(0x7fc00000) : (float)s * inv_scale;
 }
 
 template <int NV, int NT>
@@ -370,13 +374,13 @@ __global__ void __launch_bounds__(NT) xent_rows_kernel(const XentProb* __restric
         raw[j] = pack8(f);
       }
     }
-    st = warp_sum_f(st);
+    st = warp_sum_fixed(st, 2097152.f, 1.f / 2097152.f);          // <= 32 lanes x 32 terms <= 1 each, x 2^21
     if (lane == 0) wred[par][warp] = make_float2(wm, st);
     __syncthreads();
     const float2 v = lane < NW ? wred[par][lane] : make_float2(-INFINITY, 0.f);
     par ^= 1;
     const float M = warp_max_f(v.x);
-    const float S = warp_sum_f(v.x == -INFINITY ? 0.f : v.y * fast_exp2((v.x - M) * L2E));
+    const float S = warp_sum_fixed(v.x == -INFINITY ? 0.f : v.y * fast_exp2((v.x - M) * L2E), 65536.f, 1.f / 65536.f);   // <= 32 x 1024, x 2^16
     const float lse = M + logf(S);
     const float scale = wm == -INFINITY ? 0.f : fast_exp2((wm - M) * L2E) * inv / S;
 #pragma unroll
