@@ -175,10 +175,15 @@ __device__ __forceinline__ void tile_coords(const GemmProb& p, int t, int tile_m
 // buffer in the swizzled layout of the output tensor map and leaves through ONE TMA store (full-line
 // writes, clipped at the matrix edge by the hardware); otherwise every lane stores its own row.
 // VEC: all 32 columns exist and resid / aux / C are 16-byte aligned (128-bit accesses).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 template <bool VEC>
 __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensorMap* mapC, const CUtensorMap* mapC2,
                                                uint8_t* stg, int m, int m_warp0, int n0, const uint32_t* acc, int lane,
-                                               int chunk) {
+                                               int chunk, float2& run) {
   float v[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
@@ -312,6 +317,23 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_f(t[j]);
       break;
+    case EPI_LOGIT_STATS: {
+      // running (max, sum of exp(z - max)) of this row over the warp's columns, on the values as stored
+      const float L2E = 1.4426950408889634f;
+      float cm = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        v[j] = __bfloat162float(__float2bfloat16_rn(v[j]));
+        if (VEC || j < nvalid) cm = fmaxf(cm, v[j]);
+      }
+      const float nm = fmaxf(run.x, cm), nml = nm * L2E;
+      float cs = 0.f;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (VEC || j < nvalid) cs += ex2_approx(fmaf(v[j], L2E, -nml));
+      run.y = (run.x == -INFINITY ? 0.f : run.y * ex2_approx((run.x - nm) * L2E)) + cs;
+      run.x = nm;
+      break;
+    }
     default: break;
   }
   put(p.C, mapC, v, p.out_f32 != 0);
@@ -518,11 +540,12 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       const CUtensorMap* mapC = maps + 4 * pi + 2;
       uint8_t* stg = p.store_tma ? staging + (warp - 2) * 4096 : nullptr;
       const int m_warp0 = m0 + quarter * 32;
+      float2 run = make_float2(-INFINITY, 0.f);          // EPI_LOGIT_STATS: this row's statistics over the warp's columns
       auto emit = [&](const uint32_t* a, int c) {
         const int nc = n0 + col0 + c * 32;
         if (nc >= p.N || m_warp0 >= p.M) return;            // warp-uniform
-        if (vec_ok && nc + 32 <= p.N) epilogue_row32<true>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c);
-        else epilogue_row32<false>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c);
+        if (vec_ok && nc + 32 <= p.N) epilogue_row32<true>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c, run);
+        else epilogue_row32<false>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c, run);
       };
       uint32_t acc0[32], acc1[32];
       tc_ld32(trow, acc0);
@@ -535,6 +558,8 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
         if (c + 2 < BN / 64) tc_ld32(trow + (c + 2) * 32, acc0);
         emit(acc1, c + 1);
       }
+      if (p.act == EPI_LOGIT_STATS && m < p.M && n0 + col0 < p.N)
+        ((float2*)p.C2)[(size_t)m * ((p.N + 127) >> 7) + ((n0 + col0) >> 7)] = run;
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {

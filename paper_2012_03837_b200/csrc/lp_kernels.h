@@ -18,7 +18,11 @@ enum { ST_LABEL_RANGE = 1, ST_NONFINITE = 2, ST_TIMEOUT = 4 };
 // Exactly one stride of each operand is 1.  Forward of a Linear layer (App. A.1): A = x [M,K],
 // B = W [N,K].  Input gradient: A = dy, B(n,k) = W[k,n].  Weight gradient: A(m,k) = dy[k,m],
 // B(n,k) = x[k,n] (the reduction runs over the rows of the minibatch).
-enum EpiAct { EPI_NONE = 0, EPI_RELU = 1, EPI_GELU = 2, EPI_RELU_MASK = 3, EPI_GELU_GRAD = 4 };
+// EPI_LOGIT_STATS (tensor-core kernel only): no activation; besides C (bf16 logits), C2 receives, as
+// float2 [M, ceil(N/128)], the maximum and the sum of exp(z - max) over every group of 128 columns of
+// the stored (rounded) logits: the first pass of the softmax cross-entropy (App. A.1) done where the
+// logits are produced.
+enum EpiAct { EPI_NONE = 0, EPI_RELU = 1, EPI_GELU = 2, EPI_RELU_MASK = 3, EPI_GELU_GRAD = 4, EPI_LOGIT_STATS = 5 };
 
 struct GemmProb {
   const void* A;
@@ -92,6 +96,17 @@ void launch_ln_bwd_vec(const LnBwdProb* d_probs, int n, int max_rows, int nv, cu
 void launch_xent_vec(const XentProb* d_probs, int n, int max_rows, int nv, cudaStream_t s);
 // Blocks of XENT_ROWS rows, dlogits in place plus per-block column sums; classes % 8 == 0, classes <= 32768.
 void launch_xent_rows(const XentProb* d_probs, int n, int max_rows, int classes, cudaStream_t s);
+
+// Cross-entropy from per-group softmax statistics (EPI_LOGIT_STATS): a merge kernel turns the groups
+// of a row into its log-sum-exp and loss, then dlogits = softmax/n - onehot/n are written in place by
+// column strips with no reduction left inside a row; the strips' column sums (bias gradient) go to
+// colsum_part [ceil(rows / XENT_APPLY_ROWS), classes] when it is non-null.
+struct XentStatsProb {
+  void* z; const int* y; const int* n_valid; float* row_loss; const float2* stats; float* row_c;
+  float* colsum_part; int rows, classes, ld, groups;
+};
+enum { XENT_APPLY_ROWS = 256 };
+void launch_xent_from_stats(const XentStatsProb* d_probs, int n, int max_rows, int classes, cudaStream_t s);
 
 struct LossProb { const float* row_loss; const int* n_valid; int rows; int out_index; };
 void launch_loss_reduce(const LossProb* d_probs, int n, float* d_losses, int* d_status, cudaStream_t s);

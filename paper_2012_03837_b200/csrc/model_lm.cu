@@ -8,6 +8,7 @@
 // and shift gradients are formed, not the gradient of the chunk input (Sec. 3).
 #include <stdexcept>
 
+#include "gemm_tc.h"
 #include "runtime.h"
 
 namespace lp {
@@ -25,6 +26,7 @@ struct ChunkBufs {
   void* emb = nullptr;         // chunk 0: embedding output
   void *ah, *z;                // head LayerNorm output, logits / dlogits
   float *meanh, *rstdh, *row_loss;
+  float2* zstats = nullptr;    // per-row softmax statistics of the logits' column groups (training, tensor-core path)
   void *G0, *G1, *G2, *Gf, *Gq;   // gradient scratch: [M,d] x3, [M,ffn], [M,3d]
 };
 
@@ -182,11 +184,27 @@ void build_lm(Handle& h) {
     std::vector<LnProb> ln;
     std::vector<GemmProb> g;
     std::vector<XentProb> xs;
+    std::vector<XentStatsProb> xst;
+    // Training steps on the tensor-core path: the head GEMM leaves per-group softmax statistics next
+    // to the logits, so the cross-entropy needs no reduction pass over the logits of its own.
+    bool fused = train && h.bf16_mode && !h.force_simt && V % 8 == 0;
+    for (int k = 0; k < K && fused; ++k) {
+      GemmProb probe = gemm_fwd(cb[k].ah, h.W(hn(k, "W")), cb[k].z, M, V, d, h.P32(hn(k, "b")), EPI_LOGIT_STATS);
+      fused = gemm_tc_eligible(probe) && (((uintptr_t)cb[k].z & 15) == 0);
+    }
+    const int groups = (V + 127) / 128;
     for (int k = 0; k < K; ++k) {
       ChunkBufs& c = cb[k];
       ln.push_back(LnProb{h.bnd[wr][k], c.ah, h.P32(hn(k, "ln.g")), h.P32(hn(k, "ln.b")), c.meanh, c.rstdh, M, d});
-      g.push_back(gemm_fwd(c.ah, h.W(hn(k, "W")), c.z, M, V, d, h.P32(hn(k, "b")), EPI_NONE));
-      xs.push_back(XentProb{c.z, labels_of(k, pipelined, rd), h.n_valid[k], c.row_loss, M, V, V, nullptr});
+      g.push_back(gemm_fwd(c.ah, h.W(hn(k, "W")), c.z, M, V, d, h.P32(hn(k, "b")), fused ? EPI_LOGIT_STATS : EPI_NONE));
+      if (fused) {
+        if (!c.zstats) c.zstats = (float2*)h.dalloc((size_t)M * groups * sizeof(float2));
+        g.back().C2 = c.zstats;
+        xst.push_back(XentStatsProb{c.z, labels_of(k, pipelined, rd), h.n_valid[k], c.row_loss, c.zstats, nullptr, nullptr,
+                                    M, V, V, groups});
+      } else {
+        xs.push_back(XentProb{c.z, labels_of(k, pipelined, rd), h.n_valid[k], c.row_loss, M, V, V, nullptr});
+      }
     }
     emit_ln_fwd(h, p, ln);
     emit_gemm(h, p, g);
@@ -199,7 +217,12 @@ void build_lm(Handle& h) {
     }
     std::vector<float*> bgs;
     for (int k = 0; k < K; ++k) bgs.push_back(h.G(hn(k, "b")));
-    head_bias_done = emit_xent_and_loss(h, p, xs, all, train ? &bgs : nullptr);
+    if (fused) {
+      emit_xent_from_stats(h, p, xst, all, &bgs);
+      head_bias_done = true;
+    } else {
+      head_bias_done = emit_xent_and_loss(h, p, xs, all, train ? &bgs : nullptr);
+    }
   };
 
   auto build_step = [&](Plan& p, bool pipelined, int rd, int wr) {

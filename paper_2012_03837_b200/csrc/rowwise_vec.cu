@@ -420,6 +420,110 @@ __global__ void __launch_bounds__(NT) xent_rows_kernel(const XentProb* __restric
   }
 }
 
+// ------------------------------------------------------------------ cross-entropy from GEMM-side statistics
+// Warp per row: merge the (max, sum-exp) pairs of the row's column groups; row_c is the base-2 constant
+// with exp2(z*log2(e) - row_c) = softmax(z) / n_valid (+inf for ignored rows: zero gradient).
+__global__ void __launch_bounds__(256) xent_merge_kernel(const XentStatsProb* __restrict__ probs) {
+  const float L2E = 1.4426950408889634f;
+  const XentStatsProb p = probs[blockIdx.y];
+  const int lane = threadIdx.x & 31, row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= p.rows) return;
+  const int y = p.y[row];
+  if (!(y >= 0 && y < p.classes)) {
+    if (lane == 0) { p.row_loss[row] = 0.f; p.row_c[row] = INFINITY; }
+    return;
+  }
+  const float2* st = p.stats + (size_t)row * p.groups;
+  float m = -INFINITY;
+  for (int g = lane; g < p.groups; g += 32) m = fmaxf(m, st[g].x);
+  m = warp_max_f(m);
+  float s = 0.f;
+  for (int g = lane; g < p.groups; g += 32) { float2 v = st[g]; s += v.y * fast_exp2((v.x - m) * L2E); }
+  s = warp_sum(s);
+  if (lane == 0) {
+    float lse = m + logf(s);
+    float zy = __bfloat162float(((const bf16*)p.z)[(size_t)row * p.ld + y]);
+    p.row_loss[row] = lse - zy;
+    p.row_c[row] = lse * L2E + log2f((float)(*p.n_valid));
+  }
+}
+
+__device__ __forceinline__ void xent_apply_row(uint4 raw, float c, int y, int vec, float inv, bool col_ok, float (&cs)[8],
+                                               bf16* out) {
+  const float L2E = 1.4426950408889634f;
+  float f[8];
+  unpack8(raw, f);
+#pragma unroll
+  for (int t = 0; t < 8; ++t) f[t] = fast_exp2(fmaf(f[t], L2E, -c));
+  if ((y >> 3) == vec && c != INFINITY) {
+    const int ty = y & 7;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) f[t] -= (t == ty) ? inv : 0.f;
+  }
+  if (col_ok) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) cs[t] += f[t];
+    *(uint4*)out = pack8(f);
+  }
+}
+
+// Block = 32 column lanes (8 columns each: a strip of 256 columns) x 8 row lanes over XENT_APPLY_ROWS
+// rows; four rows per row lane in flight.  A thread keeps the column sums of its 8 columns in
+// registers; the 8 row lanes are added in order at the end.
+__global__ void __launch_bounds__(256) xent_apply_kernel(const XentStatsProb* __restrict__ probs) {
+  __shared__ float red[8][32][9];
+  const float L2E = 1.4426950408889634f;
+  const XentStatsProb p = probs[blockIdx.z];
+  const int r0 = blockIdx.y * XENT_APPLY_ROWS;
+  if (r0 >= p.rows || (int)blockIdx.x * 256 >= p.classes) return;
+  const int r1 = min(r0 + XENT_APPLY_ROWS, p.rows);
+  const int cx = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int vec = blockIdx.x * 32 + cx, c0 = vec * 8;
+  const bool col_ok = c0 < p.classes;
+  const float inv = 1.0f / (float)(*p.n_valid);
+  float cs[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) cs[t] = 0.f;
+  // the warp's rows are r0 + ry + 8*k, k < 32: lane k fetches row k's constant and label once, the
+  // loop broadcasts them with shuffles (no per-element loads besides the logits themselves)
+  static_assert(XENT_APPLY_ROWS == 256, "one row per lane of each of the 8 row-lane warps");
+  float c_mine = INFINITY;
+  int y_mine = -1;
+  {
+    int r = r0 + ry + 8 * cx;
+    if (r < r1) { c_mine = p.row_c[r]; y_mine = p.y[r]; }
+  }
+  auto one = [&](uint4 raw, int r, int k) {
+    xent_apply_row(raw, __shfl_sync(0xffffffffu, c_mine, k), __shfl_sync(0xffffffffu, y_mine, k), vec, inv, col_ok, cs,
+                   (bf16*)p.z + (size_t)r * p.ld + c0);
+  };
+  {
+    const bf16* base = (const bf16*)p.z + (col_ok ? c0 : 0);
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    int r = r0 + ry, k = 0;
+    for (; r + 24 < r1; r += 32, k += 4) {
+      uint4 a0 = zero, a1 = zero, a2 = zero, a3 = zero;
+      if (col_ok) {
+        a0 = *(const uint4*)(base + (size_t)r * p.ld); a1 = *(const uint4*)(base + (size_t)(r + 8) * p.ld);
+        a2 = *(const uint4*)(base + (size_t)(r + 16) * p.ld); a3 = *(const uint4*)(base + (size_t)(r + 24) * p.ld);
+      }
+      one(a0, r, k); one(a1, r + 8, k + 1); one(a2, r + 16, k + 2); one(a3, r + 24, k + 3);
+    }
+    for (; r < r1; r += 8, ++k) one(col_ok ? *(const uint4*)(base + (size_t)r * p.ld) : zero, r, k);
+  }
+  if (!p.colsum_part) return;
+#pragma unroll
+  for (int t = 0; t < 8; ++t) red[ry][cx][t] = cs[t];
+  __syncthreads();
+  const int col = threadIdx.x, gc = blockIdx.x * 256 + col;
+  if (gc < p.classes) {
+    float v = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v += red[k][col >> 3][col & 7];
+    p.colsum_part[(size_t)blockIdx.y * p.classes + gc] = v;
+  }
+}
+
 }  // namespace
 
 // d must equal nv*256 with nv in {1, 2, 4}; rows, scale and shift 16-byte aligned.
@@ -476,6 +580,13 @@ void launch_xent_rows(const XentProb* d, int n, int max_rows, int classes, cudaS
   else if (nvec <= 1024) xent_rows_kernel<1, 1024><<<grid, 1024, smem, s>>>(d);
   else if (nvec <= 2048) xent_rows_kernel<2, 1024><<<grid, 1024, smem, s>>>(d);
   else xent_rows_kernel<4, 1024><<<grid, 1024, smem, s>>>(d);
+}
+
+// classes and ld multiples of 8, z 16-byte aligned
+void launch_xent_from_stats(const XentStatsProb* d, int n, int max_rows, int classes, cudaStream_t s) {
+  xent_merge_kernel<<<dim3((max_rows + 7) / 8, n), 256, 0, s>>>(d);
+  dim3 grid((classes + 255) / 256, (max_rows + XENT_APPLY_ROWS - 1) / XENT_APPLY_ROWS, n);
+  xent_apply_kernel<<<grid, 256, 0, s>>>(d);
 }
 
 }  // namespace lp

@@ -302,6 +302,36 @@ bool emit_xent_and_loss(Handle& h, Plan& p, std::vector<XentProb> probs, const s
   return rows_kernel && bias_grads;
 }
 
+void emit_xent_from_stats(Handle& h, Plan& p, std::vector<XentStatsProb> probs, const std::vector<int>& chunk_of,
+                          const std::vector<float*>* bias_grads) {
+  if (probs.empty()) return;
+  int mr = 0;
+  const int classes = probs[0].classes;
+  std::vector<LossProb> lps;
+  double by = 0;
+  for (size_t i = 0; i < probs.size(); ++i) {
+    auto& q = probs[i];
+    mr = std::max(mr, q.rows);
+    lps.push_back(LossProb{q.row_loss, q.n_valid, q.rows, chunk_of[i]});
+    by += 2.0 * q.rows * q.classes * h.esize();
+    q.row_c = (float*)h.dalloc((size_t)q.rows * sizeof(float));
+    if (bias_grads) {
+      int nblk = (q.rows + XENT_APPLY_ROWS - 1) / XENT_APPLY_ROWS;
+      q.colsum_part = (float*)h.dalloc((size_t)nblk * classes * sizeof(float));
+      h.pending_reduce.push_back(ColReduceProb{q.colsum_part, (*bias_grads)[i], nblk, classes, classes});
+    }
+  }
+  const XentStatsProb* d = h.upload(probs);
+  const LossProb* dl = h.upload(lps);
+  int n = (int)probs.size();
+  float* losses = h.d_losses;
+  int* st = h.d_status;
+  p.add(3, [=](const RunCtx& c) {
+    launch_xent_from_stats(d, n, mr, classes, c.stream);
+    launch_loss_reduce(dl, n, losses, st, c.stream);
+  }, KIND_XENT, by);
+}
+
 void emit_optimizer(Handle& h, Plan& p) {
   Handle* hp = &h;
   p.add(1, [hp](const RunCtx& c) {

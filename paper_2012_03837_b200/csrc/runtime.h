@@ -137,6 +137,10 @@ void emit_labels(Handle& h, Plan& p, const std::vector<LabelProb>& probs);
 // cross-entropy kernel produces them itself (then the caller needs no separate column-sum pass).
 bool emit_xent_and_loss(Handle& h, Plan& p, std::vector<XentProb> probs, const std::vector<int>& chunk_of,
                         const std::vector<float*>* bias_grads = nullptr);
+// Cross-entropy whose per-group softmax statistics were left by the head GEMM (EPI_LOGIT_STATS); classes of
+// all problems equal.  The column sums of dlogits are queued for bias_grads when it is given.
+void emit_xent_from_stats(Handle& h, Plan& p, std::vector<XentStatsProb> probs, const std::vector<int>& chunk_of,
+                          const std::vector<float*>* bias_grads);
 void emit_optimizer(Handle& h, Plan& p);
 
 // GEMM problem constructors (x: [M,K] row-major, W: [N,K] row-major, dy: [M,N] row-major)
