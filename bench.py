@@ -174,6 +174,29 @@ class ClockSampler:
         return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(np.max(mx)), reasons=sorted(reasons), samples=len(sm))
 
 
+# ----------------------------------------------------------------------------- N > 1: independent replicas
+
+def replica_config(cfg, rank):
+    """Every replica draws its own weights and data: the path has no exchange step, so N GPUs run N
+    independent copies of the local update step (weak scaling)."""
+    return dict(cfg, seed=cfg["seed"] + rank)
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of `values` over all ranks (the slowest replica sets the job's time)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    tt = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return tt.tolist()
+
+
+def whole_job_rate(world, units_per_step, ms_per_step):
+    """Units all replicas processed per second, given the slowest replica's step time."""
+    return world * units_per_step / (ms_per_step * 1e-3)
+
+
 # ----------------------------------------------------------------------------- the GPU arm
 
 def run_ours(args, cfg):
@@ -200,7 +223,7 @@ def run_ours(args, cfg):
         info = lp.lp_tensor_info_get(h, i)
         names[info["name"]] = (i, info)
     stream = torch.cuda.current_stream().cuda_stream
-    cfg_r = dict(cfg, seed=cfg["seed"] + rank)          # every replica draws its own weights and data
+    cfg_r = replica_config(cfg, rank)
     for n, a in lp_synth.init_params(cfg_r).items():
         if a.ndim == 4:
             a = np.ascontiguousarray(a.transpose(0, 2, 3, 1))
@@ -271,14 +294,11 @@ def run_ours(args, cfg):
     barrier()
     ms_e2e = e0.elapsed_time(e1) / e2e_steps
 
-    if dist is not None:
-        tt = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = tt.tolist()
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, dev)
     units = lp_synth.units_per_step(cfg)
     ms_step = ms_total / args.steps
-    value = world * units / (ms_step * 1e-3)
-    e2e_value = world * units / (ms_e2e * 1e-3)
+    value = whole_job_rate(world, units, ms_step)
+    e2e_value = whole_job_rate(world, units, ms_e2e)
 
     if rank == 0:
         metric, unit = metric_of(cfg)

@@ -1,14 +1,20 @@
 // Grouped bf16 GEMM on the 5th-generation tensor cores (tcgen05) for sm_100a.
 //
-// One persistent CTA per SM walks a flat list of 128x256 output tiles that spans every problem of
-// the launch (all chunks' forward, input-gradient and weight-gradient products of one phase:
-// Sec. 3 makes them independent).  Per tile, 64-deep k slices of A and B are brought into a
-// 4-stage shared-memory ring by TMA (128-byte swizzle; out-of-range rows/columns read as zero, so
-// ragged M, N, K need no special case), one elected thread issues tcgen05.mma (M=128, N=256, K=16,
-// bf16 x bf16 -> fp32) into one of two 256-column TMEM accumulators, and eight epilogue warps read
-// the finished accumulator back with tcgen05.ld, apply the fused epilogue (bias, residual,
-// ReLU/GELU, ReLU mask, GELU') and store bf16 or fp32 while the next tile's main loop already
-// runs on the other accumulator.
+// Persistent CTAs walk a flat list of output tiles that spans every problem of the launch (all
+// chunks' forward, input-gradient and weight-gradient products of one phase: Sec. 3 makes them
+// independent).  Two variants of one kernel template:
+//   CG = 2 (default): a cluster of two CTAs on neighbouring SMs owns a 256x256 tile
+//          (tcgen05 cta_group::2, M = 256, N = 256, K = 16 per instruction, issued by the leader);
+//   CG = 1: one CTA per 128x256 tile (launches that hold a problem with M <= 128).
+// Per tile, 64-deep k slices of A and B are brought into a shared-memory ring (6 stages of 32 KB,
+// or 4 of 48 KB) by TMA (128-byte swizzle; out-of-range rows/columns read as zero, so ragged M, N,
+// K need no special case; operand panels carry an evict-last L2 hint), one elected thread issues
+// the MMAs into one of two 256-column TMEM accumulators, and eight epilogue warps read the finished
+// accumulator back with tcgen05.ld, apply the fused epilogue (bias, residual, ReLU/GELU, ReLU mask,
+// GELU', softmax statistics of the logits) and hand bf16 or fp32 blocks, staged in swizzled shared
+// memory, to TMA stores (evict-first) while the next tile's main loop already runs on the other
+// accumulator.  Tiles of a problem are walked in bands of 8 row tiles so that the tiles in flight
+// share operand panels in L2.
 //
 // Operands may be K-major (reduction index contiguous) or MN-major (row/column index contiguous),
 // per problem: forward uses K/K, the input gradient K/MN, the weight gradient MN/MN, so no
