@@ -24,9 +24,9 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 // Block = 8 warps over LN_FWD_ROWS rows (warp w takes rows w, w+8, ...); a lane owns the 8-element
 // vectors j*32 + lane, j < NV (d = NV * 256).  The warp's next row is loaded while the current one
 // is normalised.
-enum { LN_FWD_ROWS = 32 };
+enum { LN_FWD_ROWS = 64 };
 template <int NV>
-__global__ void __launch_bounds__(256) ln_fwd_vec_kernel(const LnProb* __restrict__ probs) {
+__global__ void __launch_bounds__(256, 2) ln_fwd_vec_kernel(const LnProb* __restrict__ probs) {
   const LnProb p = probs[blockIdx.y];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const int r0 = blockIdx.x * LN_FWD_ROWS;
@@ -38,6 +38,16 @@ __global__ void __launch_bounds__(256) ln_fwd_vec_kernel(const LnProb* __restric
     const uint4* x = (const uint4*)((const bf16*)p.x + (size_t)(r0 + w) * p.d);
 #pragma unroll
     for (int j = 0; j < NV; ++j) nxt[j] = x[j * 32 + lane];
+  }
+  // scale and shift of this lane's columns stay in registers for all rows of the warp
+  float g[NV][8], b[NV][8];
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    int c0 = (j * 32 + lane) * 8;
+    float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
+    float4 b0 = *(const float4*)(p.b + c0), b1 = *(const float4*)(p.b + c0 + 4);
+    g[j][0] = g0.x; g[j][1] = g0.y; g[j][2] = g0.z; g[j][3] = g0.w; g[j][4] = g1.x; g[j][5] = g1.y; g[j][6] = g1.z; g[j][7] = g1.w;
+    b[j][0] = b0.x; b[j][1] = b0.y; b[j][2] = b0.z; b[j][3] = b0.w; b[j][4] = b1.x; b[j][5] = b1.y; b[j][6] = b1.z; b[j][7] = b1.w;
   }
   for (int row = r0 + w; row < r1; row += 8) {
     float v[NV][8];
@@ -58,19 +68,14 @@ __global__ void __launch_bounds__(256) ln_fwd_vec_kernel(const LnProb* __restric
 #pragma unroll
     for (int j = 0; j < NV; ++j)
 #pragma unroll
-      for (int t = 0; t < 8; ++t) { float c = v[j][t] - mu; q += c * c; }
+      for (int t = 0; t < 8; ++t) { v[j][t] -= mu; q += v[j][t] * v[j][t]; }
     float rstd = rsqrtf(warp_sum(q) * inv_d + 1e-5f);
     uint4* y = (uint4*)((bf16*)p.y + (size_t)row * p.d);
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      int c0 = (j * 32 + lane) * 8;
-      float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
-      float4 b0 = *(const float4*)(p.b + c0), b1 = *(const float4*)(p.b + c0 + 4);
-      float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-      float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
       float o[8];
 #pragma unroll
-      for (int t = 0; t < 8; ++t) o[t] = (v[j][t] - mu) * rstd * g[t] + b[t];
+      for (int t = 0; t < 8; ++t) o[t] = v[j][t] * rstd * g[j][t] + b[j][t];
       y[j * 32 + lane] = pack8(o);
     }
     if (lane == 0) { p.mean[row] = mu; p.rstd[row] = rstd; }
@@ -117,28 +122,33 @@ __global__ void __launch_bounds__(256) ln_bwd_vec_kernel(const LnBwdProb* __rest
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  float ag[NV][8], ab[NV][8];
+  float ag[NV][8], ab[NV][8], g[NV][8];
 #pragma unroll
-  for (int j = 0; j < NV; ++j)
+  for (int j = 0; j < NV; ++j) {
+    int c0 = (j * 32 + lane) * 8;
+    float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
+    g[j][0] = g0.x; g[j][1] = g0.y; g[j][2] = g0.z; g[j][3] = g0.w; g[j][4] = g1.x; g[j][5] = g1.y; g[j][6] = g1.z; g[j][7] = g1.w;
 #pragma unroll
     for (int t = 0; t < 8; ++t) { ag[j][t] = 0.f; ab[j][t] = 0.f; }
+  }
   fetch(r0 + w, 0);
   fetch(r0 + w + 8, 1);
-  int slot = 0;
+  // lane k holds the statistics of the warp's k-th row (rows r0 + w + 8k, k < LN_BWD_ROWS / 8 <= 32)
+  static_assert(LN_BWD_ROWS / 8 <= 32, "one row per lane");
+  float mu_mine = 0.f, rs_mine = 0.f;
+  if (r0 + w + 8 * lane < r1) { mu_mine = p.mean[r0 + w + 8 * lane]; rs_mine = p.rstd[r0 + w + 8 * lane]; }
+  int slot = 0, kk = 0;
   const float inv_d = 1.0f / D;
-  for (int row = r0 + w; row < r1; row += 8) {
+  for (int row = r0 + w; row < r1; row += 8, ++kk) {
     fetch(row + 16, slot == 0 ? 2 : slot - 1);      // the slot freed by the previous row
     asm volatile("cp.async.wait_group 2;" ::: "memory");
     __syncwarp();
     const uint4* buf = ring + (size_t)slot * 3 * (D / 8);
-    float mu = p.mean[row], rs = p.rstd[row];
+    const float mu = __shfl_sync(0xffffffffu, mu_mine, kk), rs = __shfl_sync(0xffffffffu, rs_mine, kk);
     float xh[NV][8], dv[NV][8];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int j = 0; j < NV; ++j) {
-      int c0 = (j * 32 + lane) * 8;
-      float4 g0 = *(const float4*)(p.g + c0), g1 = *(const float4*)(p.g + c0 + 4);
-      float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
       unpack8(buf[j * 32 + lane], xh[j]);
       unpack8(buf[D / 8 + j * 32 + lane], dv[j]);
 #pragma unroll
@@ -146,7 +156,7 @@ __global__ void __launch_bounds__(256) ln_bwd_vec_kernel(const LnBwdProb* __rest
         xh[j][t] = (xh[j][t] - mu) * rs;
         ag[j][t] += dv[j][t] * xh[j][t];
         ab[j][t] += dv[j][t];
-        dv[j][t] *= g[t];                             // from here on: gradient w.r.t. the normalised value
+        dv[j][t] *= g[j][t];                          // from here on: gradient w.r.t. the normalised value
         s1 += dv[j][t];
         s2 += dv[j][t] * xh[j][t];
       }
