@@ -48,7 +48,14 @@ template <int CG> struct Cfg {
 };
 constexpr int MAX_STAGES = 6;
 constexpr int EPI_WARPS = 8;                      // two warps per TMEM lane quarter, each takes half of the 256 columns
-constexpr int NTHREADS = 64 + 32 * EPI_WARPS;
+// Warps 0-3 form the control warpgroup (0: TMA producer, 1: MMA issuer, 2-3: idle); warps 4-11 are
+// the two epilogue warpgroups.  After set-up the control warpgroup hands most of its registers to
+// the epilogue warpgroups (setmaxnreg), whose threads each hold 64 accumulator values, the prefetched
+// side input and the converted outputs.
+constexpr int EPI_FIRST = 4;
+constexpr int NTHREADS = 32 * (EPI_FIRST + EPI_WARPS);
+// The pool that setmaxnreg redistributes is what the launch allocated: 384 threads x 168 registers.
+constexpr int CTRL_REGS = 56, EPI_REGS = 224;     // 128 * 56 + 256 * 224 = 384 * 168
 constexpr uint32_t TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
@@ -186,10 +193,33 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// GELU x*Phi(x) and its derivative Phi(x) + x*phi(x) for the epilogue, where 128 values per thread
+// and tile have to fit under the tile's main loop: Phi through the rational approximation of erfc
+// of Abramowitz & Stegun 7.1.26 (absolute error of erf below 1.5e-7), whose exp(-x^2/2) is shared
+// with phi; one ex2 and one rcp per value.
+__device__ __forceinline__ void phi_parts(float x, float& cdf, float& e) {
+  const float ax = fabsf(x) * 0.70710678118654752f;
+  e = ex2_approx(x * x * -0.72134752044448170f);            // exp(-x^2 / 2)
+  float t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, ax, 1.0f)));
+  float poly = fmaf(fmaf(fmaf(fmaf(1.061405429f, t, -1.453152027f), t, 1.421413741f), t, -0.284496736f), t, 0.254829592f) * t;
+  const float half_erfc = 0.5f * poly * e;                  // 0.5 * erfc(|x| / sqrt 2)
+  cdf = x >= 0.f ? 1.0f - half_erfc : half_erfc;
+}
+__device__ __forceinline__ float gelu_fast(float x) {
+  float cdf, e;
+  phi_parts(x, cdf, e);
+  return x * cdf;
+}
+__device__ __forceinline__ float gelu_grad_fast(float x) {
+  float cdf, e;
+  phi_parts(x, cdf, e);
+  return fmaf(x * 0.39894228040143268f, e, cdf);
+}
 template <bool VEC>
 __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensorMap* mapC, const CUtensorMap* mapC2,
                                                uint8_t* stg, int m, int m_warp0, int n0, const uint32_t* acc, int lane,
-                                               int chunk, float2& run) {
+                                               int chunk, float2& run, const void* side, const uint4* side_pre) {
   float v[32];
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(acc[j]);
@@ -197,9 +227,18 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
   const size_t off = (size_t)m * p.ldc + n0;
   const int nvalid = min(32, p.N - n0);
   if (p.bias) {
+    if (VEC && (((uintptr_t)p.bias & 15) == 0)) {
 #pragma unroll
-    for (int j = 0; j < 32; ++j) if (VEC || j < nvalid) v[j] += p.bias[n0 + j];
+      for (int q = 0; q < 8; ++q) {
+        float4 b4 = *(const float4*)(p.bias + n0 + 4 * q);
+        v[4 * q] += b4.x; v[4 * q + 1] += b4.y; v[4 * q + 2] += b4.z; v[4 * q + 3] += b4.w;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (VEC || j < nvalid) v[j] += p.bias[n0 + j];
+    }
   }
+  // `side` (resid or aux, when only one of them is set) arrives already loaded in side_pre on the 128-bit path
   auto load32 = [&](const void* base, float* o) {
     const bf16* src = (const bf16*)base + off;
     if (!row_ok) {
@@ -208,7 +247,7 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
     } else if (VEC) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        uint4 u = *(const uint4*)(src + q * 8);
+        uint4 u = (side_pre && base == side) ? side_pre[q] : *(const uint4*)(src + q * 8);
         const __nv_bfloat162* h = (const __nv_bfloat162*)&u;
 #pragma unroll
         for (int t = 0; t < 4; ++t) { float2 f = __bfloat1622float2(h[t]); o[q * 8 + 2 * t] = f.x; o[q * 8 + 2 * t + 1] = f.y; }
@@ -311,7 +350,7 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
       for (int j = 0; j < 32; ++j) v[j] = __bfloat162float(__float2bfloat16_rn(v[j]));
       put(p.C2, mapC2, v, false);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = gelu_f(v[j]);
+      for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
       break;
     case EPI_RELU_MASK:
       load32(p.aux, t);
@@ -321,7 +360,7 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
     case EPI_GELU_GRAD:
       load32(p.aux, t);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_f(t[j]);
+      for (int j = 0; j < 32; ++j) v[j] *= gelu_grad_fast(t[j]);
       break;
     case EPI_LOGIT_STATS: {
       // running (max, sum of exp(z - max)) of this row over the warp's columns, on the values as stored
@@ -420,6 +459,8 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
   tc_fence_after();
   const uint32_t tmem_base = *(volatile uint32_t*)&sh->tmem_base;
 
+  if (warp < EPI_FIRST) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(CTRL_REGS));
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (one per CTA)
     if (lane == 0) {
@@ -519,7 +560,9 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
         if (ok) { if (CG == 1) tc_commit(&sh->tmem_full[ab]); else tc_commit_pair(&sh->tmem_full[ab]); }
       }
     }
+  }
   } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(EPI_REGS));
     // ------------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;            // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
     int pi = 0, it = 0;
@@ -532,26 +575,38 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN;
       int ab = it & 1;
       uint32_t use = (uint32_t)(it >> 1);
+      // Each thread owns one accumulator row and walks this warp's half of the columns 32 at a time;
+      // the TMEM load of the next 32 columns and the global load of the next block of the side input
+      // (residual or activation-derivative operand) are in flight while the current block is stored.
+      const int m = m0 + quarter * 32 + lane;
+      const int col0 = ((warp - EPI_FIRST) >> 2) * (BN / 2);
+      const bool vec_ok = (p.ldc % 8 == 0) && (((uintptr_t)p.C & 15) == 0) && (!p.C2 || ((uintptr_t)p.C2 & 15) == 0) &&
+                          (!p.resid || ((uintptr_t)p.resid & 15) == 0) && (!p.aux || ((uintptr_t)p.aux & 15) == 0);
+      const void* side = (p.resid && !p.aux) ? p.resid : (p.aux && !p.resid) ? p.aux : nullptr;
+      uint4 side0[4], side1[4];
+      auto fetch_side = [&](uint4* dst, int c) {
+        const int nc = n0 + col0 + c * 32;
+        if (side && vec_ok && m < p.M && nc + 32 <= p.N) {
+          const uint4* src = (const uint4*)((const bf16*)side + (size_t)m * p.ldc + nc);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) dst[q] = src[q];
+        }
+      };
+      fetch_side(side0, 0);                    // on its way while the accumulator is still being produced
       ok = lane == 0 ? mbar_wait(&sh->tmem_full[ab], use & 1, sh, status) : true;   // one poller per warp
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      // Each thread owns one accumulator row and walks this warp's half of the columns 32 at a time;
-      // the TMEM load of the next 32 columns is in flight while the current ones are stored.
-      const int m = m0 + quarter * 32 + lane;
-      const int col0 = ((warp - 2) >> 2) * (BN / 2);
-      const bool vec_ok = (p.ldc % 8 == 0) && (((uintptr_t)p.C & 15) == 0) && (!p.C2 || ((uintptr_t)p.C2 & 15) == 0) &&
-                          (!p.resid || ((uintptr_t)p.resid & 15) == 0) && (!p.aux || ((uintptr_t)p.aux & 15) == 0);
       const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(ab * BN + col0);
       const CUtensorMap* mapC = maps + 4 * pi + 2;
-      uint8_t* stg = p.store_tma ? staging + (warp - 2) * 4096 : nullptr;
+      uint8_t* stg = p.store_tma ? staging + (warp - EPI_FIRST) * 4096 : nullptr;
       const int m_warp0 = m0 + quarter * 32;
       float2 run = make_float2(-INFINITY, 0.f);          // EPI_LOGIT_STATS: this row's statistics over the warp's columns
-      auto emit = [&](const uint32_t* a, int c) {
+      auto emit = [&](const uint32_t* a, int c, const uint4* sp) {
         const int nc = n0 + col0 + c * 32;
         if (nc >= p.N || m_warp0 >= p.M) return;            // warp-uniform
-        if (vec_ok && nc + 32 <= p.N) epilogue_row32<true>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c, run);
-        else epilogue_row32<false>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c, run);
+        if (vec_ok && nc + 32 <= p.N) epilogue_row32<true>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c, run, side, side ? sp : nullptr);
+        else epilogue_row32<false>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c, run, nullptr, nullptr);
       };
       uint32_t acc0[32], acc1[32];
       tc_ld32(trow, acc0);
@@ -559,10 +614,11 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       for (int c = 0; c < BN / 64; c += 2) {
         tc_wait_ld();
         tc_ld32(trow + (c + 1) * 32, acc1);
-        emit(acc0, c);
+        fetch_side(side1, c + 1);
+        emit(acc0, c, side0);
         tc_wait_ld();
-        if (c + 2 < BN / 64) tc_ld32(trow + (c + 2) * 32, acc0);
-        emit(acc1, c + 1);
+        if (c + 2 < BN / 64) { tc_ld32(trow + (c + 2) * 32, acc0); fetch_side(side0, c + 2); }
+        emit(acc1, c + 1, side1);
       }
       if (p.act == EPI_LOGIT_STATS && m < p.M && n0 + col0 < p.N)
         ((float2*)p.C2)[(size_t)m * ((p.N + 127) >> 7) + ((n0 + col0) >> 7)] = run;
@@ -575,7 +631,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
     }
   }
 
-  if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's TMA stores are done
+  if (warp >= EPI_FIRST && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's TMA stores are done
   tc_fence_before();
   __syncthreads();
   if (CG == 2) cluster_sync_all();             // neither CTA frees TMEM or exits while the partner may still touch it
@@ -694,6 +750,12 @@ cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int npro
     cudaError_t e = cg == 2 ? cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
                             : cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    // The epilogue warpgroups' register increase must fit into what the launch allocates (threads x
+    // compiled register count); otherwise it would wait forever.  Refuse to launch instead.
+    cudaFuncAttributes fa;
+    e = cg == 2 ? cudaFuncGetAttributes(&fa, gemm_tc_kernel<2>) : cudaFuncGetAttributes(&fa, gemm_tc_kernel<1>);
+    if (e != cudaSuccess) return e;
+    if (32 * EPI_FIRST * CTRL_REGS + 32 * EPI_WARPS * EPI_REGS > NTHREADS * fa.numRegs) return cudaErrorLaunchOutOfResources;
     attr_set[cg] = true;
   }
   if (total_tiles == 0) return cudaSuccess;

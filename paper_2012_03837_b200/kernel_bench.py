@@ -3,6 +3,7 @@ products of the transformer workloads in forward, input-gradient and weight-grad
 
     python -m paper_2012_03837_b200.kernel_bench [--shape qkv|out|ffn1|ffn2|head|all] [--form fwd|dgrad|wgrad|all]
                                                  [--d 1024] [--rows 8192] [--vocab 32768] [--groups 4] [--reps 10]
+                                                 [--epilogue none|model]
 
 Prints one JSON line per (shape, form): milliseconds per launch and TFLOP/s (2*M*N*K per problem).
 Inputs are larger than the L2 cache in total, so every launch streams its operands from HBM.
@@ -21,20 +22,40 @@ def shapes(d, ffn, vocab):
     return {"qkv": (3 * d, d), "out": (d, d), "ffn1": (ffn, d), "ffn2": (d, ffn), "head": (vocab, d)}
 
 
-def descs(form, rows, n_out, n_in, groups):
+# fused epilogue of each product in the transformer block (--epilogue model): (bias, residual, activation)
+EPI_NONE, EPI_GELU, EPI_GELU_GRAD = 0, 2, 4
+MODEL_EPILOGUE = {("qkv", "fwd"): (True, False, EPI_NONE), ("out", "fwd"): (True, True, EPI_NONE),
+                  ("ffn1", "fwd"): (True, False, EPI_GELU), ("ffn2", "fwd"): (True, True, EPI_NONE),
+                  ("head", "fwd"): (True, False, EPI_NONE), ("ffn2", "dgrad"): (False, False, EPI_GELU_GRAD)}
+
+
+def descs(form, rows, n_out, n_in, groups, epilogue=(False, False, EPI_NONE)):
     """`groups` independent Linear layers y = x W^T with x [rows, n_in], W [n_out, n_in]."""
     out, keep = [], []
     bf = dict(dtype=torch.bfloat16, device="cuda")
+    bias, resid, act = epilogue
     for _ in range(groups):
         x = torch.randn(rows, n_in, **bf)
         W = torch.randn(n_out, n_in, **bf) * 0.02
         dy = torch.randn(rows, n_out, **bf)
         if form == "fwd":
             c = torch.empty(rows, n_out, **bf)
-            out.append(dict(A=x, B=W, C=c, M=rows, N=n_out, K=n_in, a_ms=n_in, a_ks=1, b_ns=n_in, b_ks=1, ldc=n_out))
+            d = dict(A=x, B=W, C=c, M=rows, N=n_out, K=n_in, a_ms=n_in, a_ks=1, b_ns=n_in, b_ks=1, ldc=n_out, act=act)
+            if bias:
+                d["bias"] = torch.randn(n_out, dtype=torch.float32, device="cuda")
+            if resid:
+                d["resid"] = torch.randn(rows, n_out, **bf)
+            if act == EPI_GELU:
+                d["C2"] = torch.empty(rows, n_out, **bf)
+            keep += [v for v in d.values() if torch.is_tensor(v)]
+            out.append(d)
         elif form == "dgrad":
             c = torch.empty(rows, n_in, **bf)
-            out.append(dict(A=dy, B=W, C=c, M=rows, N=n_in, K=n_out, a_ms=n_out, a_ks=1, b_ns=1, b_ks=n_in, ldc=n_in))
+            d = dict(A=dy, B=W, C=c, M=rows, N=n_in, K=n_out, a_ms=n_out, a_ks=1, b_ns=1, b_ks=n_in, ldc=n_in, act=act)
+            if act == EPI_GELU_GRAD:
+                d["aux"] = torch.randn(rows, n_in, **bf)
+                keep.append(d["aux"])
+            out.append(d)
         else:
             c = torch.empty(n_out, n_in, dtype=torch.float32, device="cuda")
             out.append(dict(A=dy, B=x, C=c, M=n_out, N=n_in, K=rows, a_ms=1, a_ks=n_out, b_ns=1, b_ks=n_in, ldc=n_in, out_f32=1))
@@ -52,6 +73,8 @@ def main():
     ap.add_argument("--groups", type=int, default=4)
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--backend", type=int, default=0)
+    ap.add_argument("--epilogue", default="none", choices=["none", "model"],
+                    help="model: the bias / residual / GELU / GELU' epilogue that product has in the transformer block")
     a = ap.parse_args()
     sh = shapes(a.d, 4 * a.d, a.vocab)
     names = list(sh) if a.shape == "all" else [a.shape]
@@ -61,7 +84,8 @@ def main():
         n_out, n_in = sh[name]
         groups = max(1, a.groups // 4) if name == "head" else a.groups
         for form in forms:
-            ds, keep = descs(form, a.rows, n_out, n_in, groups)
+            epi = MODEL_EPILOGUE.get((name, form), (False, False, EPI_NONE)) if a.epilogue == "model" else (False, False, EPI_NONE)
+            ds, keep = descs(form, a.rows, n_out, n_in, groups, epi)
             for _ in range(3):
                 used = lp.lp_gemm_bf16(ds, a.backend, stream)
             torch.cuda.synchronize()
