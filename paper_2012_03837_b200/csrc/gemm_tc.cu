@@ -25,6 +25,7 @@
 // No TMA load uses cluster multicast.
 #include <cuda.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 
@@ -153,7 +154,6 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
   return d;
 }
 
-constexpr int RASTER = 8;   // row tiles per band of the tile walk
 __device__ __forceinline__ uint64_t policy_evict_first() {
   uint64_t pol;
   asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
@@ -170,15 +170,16 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int 
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
                ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src)), "l"(policy_evict_first()) : "memory");
 }
-// Tile t of a problem -> (row tile, column tile).  Tiles are walked in bands of RASTER row tiles,
+// Tile t of a problem -> (row tile, column tile).  Tiles are walked in bands of p.raster row tiles,
 // row tile fastest inside a band, so that the tiles in flight at any time share a few operand
-// panels of each kind instead of one row panel and all column panels.
+// panels of each kind instead of one row panel and all column panels; the band is as high as
+// lets its row panels stay in L2 while the column panels stream past once.
 __device__ __forceinline__ void tile_coords(const GemmProb& p, int t, int tile_m, int& mt, int& nt) {
   const int tiles_m = (p.M + tile_m - 1) / tile_m;
-  const int band = t / (RASTER * p.tiles_n);
-  const int m_base = band * RASTER;
-  const int gm = min(RASTER, tiles_m - m_base);
-  const int r = t - band * (RASTER * p.tiles_n);
+  const int band = t / (p.raster * p.tiles_n);
+  const int m_base = band * p.raster;
+  const int gm = min(p.raster, tiles_m - m_base);
+  const int r = t - band * (p.raster * p.tiles_n);
   nt = r / gm;
   mt = m_base + r - nt * gm;
 }
@@ -700,6 +701,9 @@ int gemm_tc_choose_cg(const GemmProb* probs, int n) {
 int gemm_tc_tiles(GemmProb& g, int tile_start, int cg) {
   g.tile_start = tile_start;
   g.tiles_n = (g.N + BN - 1) / BN;
+  // band height: at least 8 row tiles, more while the band's row panels (tile rows x K) stay within ~32 MB of L2
+  const long long panel = (long long)BM * cg * g.K * 2;
+  g.raster = (int)std::max(8LL, std::min(4096LL, (32LL << 20) / std::max(panel, 1LL)));
   return ((g.M + BM * cg - 1) / (BM * cg)) * g.tiles_n;
 }
 

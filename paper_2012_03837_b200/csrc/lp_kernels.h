@@ -41,6 +41,7 @@ struct GemmProb {
   int tile_start;  // first tile index of this problem in the launch (filled by the launcher)
   int tiles_n;
   int store_tma;   // tensor-core kernel: outputs leave through TMA stores (set by the launcher when C's pitch allows)
+  int raster;      // tensor-core kernel: row tiles per band of the tile walk (set by the launcher)
 };
 
 // FP32-ALU GEMM (any sizes and strides).  T = float or bf16 operands, fp32 accumulation.

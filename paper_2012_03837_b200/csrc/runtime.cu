@@ -137,6 +137,10 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
     else simt.push_back(g);
   }
   if (!tc.empty()) {
+    // Longest tiles (largest K) first: the persistent CTAs take tiles in list order, so the long ones do not
+    // end up in the tail, and products that walk the same operand in different directions (a weight
+    // gradient and an input gradient reading the same dy) are not interleaved in the cache.
+    std::stable_sort(tc.begin(), tc.end(), [](const GemmProb& a, const GemmProb& b) { return a.K > b.K; });
     int total = 0;
     const int cg = gemm_tc_choose_cg(tc.data(), (int)tc.size());
     for (auto& g : tc) total += gemm_tc_tiles(g, total, cg);
