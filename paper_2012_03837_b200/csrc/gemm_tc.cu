@@ -170,19 +170,43 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int 
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
                ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src)), "l"(policy_evict_first()) : "memory");
 }
-// Tile t of a problem -> (row tile, column tile).  Tiles are walked in bands of p.raster row tiles,
+// Which problem a tile of the launch's flat tile list belongs to.  Tiles are visited in increasing
+// order, so the cursor only moves forward; seek() touches global memory only when the problem changes.
+struct ProbCursor {
+  const GemmProb* probs;
+  int nprob, pi, next_start;
+  __device__ __forceinline__ ProbCursor(const GemmProb* pr, int n) : probs(pr), nprob(n), pi(-1), next_start(0) {}
+  // Moves to the problem holding `tile`; true if the problem changed (always on the first call).
+  __device__ __forceinline__ bool seek(int tile) {
+    if (tile < next_start) return false;
+    do {
+      ++pi;
+      next_start = pi + 1 < nprob ? probs[pi + 1].tile_start : 0x7fffffff;
+    } while (tile >= next_start);                 // problems without tiles are stepped over
+    return true;
+  }
+};
+// Tile t of a problem -> (row tile, column tile).  Tiles are walked in bands of `raster` row tiles,
 // row tile fastest inside a band, so that the tiles in flight at any time share a few operand
 // panels of each kind instead of one row panel and all column panels; the band is as high as
 // lets its row panels stay in L2 while the column panels stream past once.
-__device__ __forceinline__ void tile_coords(const GemmProb& p, int t, int tile_m, int& mt, int& nt) {
-  const int tiles_m = (p.M + tile_m - 1) / tile_m;
-  const int band = t / (p.raster * p.tiles_n);
-  const int m_base = band * p.raster;
-  const int gm = min(p.raster, tiles_m - m_base);
-  const int r = t - band * (p.raster * p.tiles_n);
-  nt = r / gm;
-  mt = m_base + r - nt * gm;
-}
+struct TileWalk {
+  int tile_start, tiles_m, tiles_n, raster;
+  __device__ __forceinline__ void set(const GemmProb& p, int tile_m) {
+    tile_start = p.tile_start; tiles_n = p.tiles_n; raster = p.raster;
+    tiles_m = (p.M + tile_m - 1) / tile_m;
+  }
+  __device__ __forceinline__ void coords(int tile, int& mt, int& nt) const {
+    const int t = tile - tile_start;
+    const int per_band = raster * tiles_n;
+    const int band = t / per_band;
+    const int m_base = band * raster;
+    const int gm = min(raster, tiles_m - m_base);
+    const int r = t - band * per_band;
+    nt = r / gm;
+    mt = m_base + r - nt * gm;
+  }
+};
 
 // Fused epilogue for 32 consecutive columns (n0 ..) of one accumulator row (row m, held by this lane).
 // Output path: if `stg` is non-null the warp's 32x32 block is written to a 4 KB shared-memory staging
@@ -194,28 +218,32 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// GELU x*Phi(x) and its derivative Phi(x) + x*phi(x) for the epilogue, where 128 values per thread
-// and tile have to fit under the tile's main loop: Phi through the rational approximation of erfc
-// of Abramowitz & Stegun 7.1.26 (absolute error of erf below 1.5e-7), whose exp(-x^2/2) is shared
-// with phi; one ex2 and one rcp per value.
-__device__ __forceinline__ void phi_parts(float x, float& cdf, float& e) {
-  const float ax = fabsf(x) * 0.70710678118654752f;
-  e = ex2_approx(x * x * -0.72134752044448170f);            // exp(-x^2 / 2)
-  float t;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, ax, 1.0f)));
-  float poly = fmaf(fmaf(fmaf(fmaf(1.061405429f, t, -1.453152027f), t, 1.421413741f), t, -0.284496736f), t, 0.254829592f) * t;
-  const float half_erfc = 0.5f * poly * e;                  // 0.5 * erfc(|x| / sqrt 2)
-  cdf = x >= 0.f ? 1.0f - half_erfc : half_erfc;
+// GELU x*Phi(x) and its derivative for the epilogue, where 128 values per thread and tile have to
+// fit under the tile's main loop (16 k-slices for the feed-forward products).  Phi is evaluated as
+// the logistic function of an odd quintic:  Phi(x) ~ 1 / (1 + 2^(-z)),  z = x (k0 + k1 s + k2 s^2),
+// s = min(x^2, 64), fitted to 2 log2(e) atanh(erf(x / sqrt 2)) on |x| <= 8 (beyond it z keeps growing
+// linearly and Phi is 0 or 1 to fp32 precision).  Largest deviation from the erf form: 6e-5 in Phi,
+// 3e-5 in GELU, 1e-4 in GELU' -- below the bf16 rounding step (2^-9 relative) of the values the
+// epilogue stores.  One ex2, one rcp and five FMA-class operations per value; the derivative
+// d/dx [x Phi] = Phi + x Phi (1 - Phi) z'(x) ln 2 reuses Phi and needs no further special function.
+constexpr float GELU_K0 = 2.30104886f, GELU_K1 = 0.106717206f, GELU_K2 = -1.00029423e-3f;   // 2 log2(e) * (c0, c1, c2)
+__device__ __forceinline__ float phi_logistic(float x, float& s) {
+  s = fminf(x * x, 64.f);
+  const float z = x * fmaf(fmaf(GELU_K2, s, GELU_K1), s, GELU_K0);
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + ex2_approx(-z)));
+  return r;
 }
 __device__ __forceinline__ float gelu_fast(float x) {
-  float cdf, e;
-  phi_parts(x, cdf, e);
-  return x * cdf;
+  float s;
+  return x * phi_logistic(x, s);
 }
 __device__ __forceinline__ float gelu_grad_fast(float x) {
-  float cdf, e;
-  phi_parts(x, cdf, e);
-  return fmaf(x * 0.39894228040143268f, e, cdf);
+  float s;
+  const float cdf = phi_logistic(x, s);
+  // z'(x) ln 2 = ln 2 (k0 + 3 k1 s + 5 k2 s^2); the clamp of s only acts where Phi (1 - Phi) has vanished
+  const float dz = fmaf(fmaf(5.f * 0.69314718f * GELU_K2, s, 3.f * 0.69314718f * GELU_K1), s, 0.69314718f * GELU_K0);
+  return fmaf(x * fmaf(-cdf, cdf, cdf), dz, cdf);
 }
 template <bool VEC>
 __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensorMap* mapC, const CUtensorMap* mapC2,
@@ -258,8 +286,23 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
       for (int j = 0; j < 32; ++j) o[j] = j < nvalid ? __bfloat162float(src[j]) : 0.f;
     }
   };
-  // one output block (bf16 or fp32) of this warp
-  auto put = [&](void* base, const CUtensorMap* map, const float* o, bool f32) {
+  // 32 values -> 16 packed bf16 pairs (round to nearest even), and the values as stored
+  auto pack32 = [](const float* o, uint32_t* pk) {
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(o[2 * t], o[2 * t + 1]);
+      pk[t] = *(uint32_t*)&h;
+    }
+  };
+  auto unpack32 = [](const uint32_t* pk, float* o) {
+#pragma unroll
+    for (int t = 0; t < 16; ++t) { o[2 * t] = __uint_as_float(pk[t] << 16); o[2 * t + 1] = __uint_as_float(pk[t] & 0xffff0000u); }
+  };
+  // One output block of this warp: 32 rows x 32 columns, bf16 (pk: 16 packed pairs per lane) or fp32 (o).
+  // With TMA stores the block is staged in this warp's 4 KB buffer.  `slot` selects the 2 KB half a
+  // narrow bf16 block uses; only a block in slot 0 waits for the buffer's previous stores to have been
+  // read, so the two outputs of the GELU epilogue are in flight together.
+  auto put = [&](void* base, const CUtensorMap* map, const uint32_t* pk, const float* o, bool f32, int slot) {
     if (stg && p.store_tma == 2) {
       // bf16, two neighbouring 32-column blocks share one store of 128-byte rows: the even block
       // fills 16-byte units 0-3 of every row, the odd one units 4-7 (128-byte swizzle)
@@ -269,13 +312,8 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
         __syncwarp();
       }
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint4 u;
-        __nv_bfloat162* h = (__nv_bfloat162*)&u;
-#pragma unroll
-        for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(o[q * 8 + 2 * t], o[q * 8 + 2 * t + 1]);
-        *(uint4*)(stg + lane * 128 + (((half * 4 + q) ^ (lane & 7)) << 4)) = u;
-      }
+      for (int q = 0; q < 4; ++q)
+        *(uint4*)(stg + lane * 128 + (((half * 4 + q) ^ (lane & 7)) << 4)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
       if (half == 1 || n0 + 32 >= p.N) {          // the pair is complete (or has no second block)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
@@ -285,26 +323,24 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
         }
       }
     } else if (stg) {
-      if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging buffer free again
-      __syncwarp();
+      if (slot == 0) {
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging buffer free again
+        __syncwarp();
+      }
+      uint8_t* dst = stg + slot * 2048;
       if (f32) {
 #pragma unroll
         for (int q = 0; q < 8; ++q)
-          *(float4*)(stg + lane * 128 + ((q ^ (lane & 7)) << 4)) = make_float4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
+          *(float4*)(dst + lane * 128 + ((q ^ (lane & 7)) << 4)) = make_float4(o[4 * q], o[4 * q + 1], o[4 * q + 2], o[4 * q + 3]);
       } else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint4 u;
-          __nv_bfloat162* h = (__nv_bfloat162*)&u;
-#pragma unroll
-          for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(o[q * 8 + 2 * t], o[q * 8 + 2 * t + 1]);
-          *(uint4*)(stg + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) = u;
-        }
+        for (int q = 0; q < 4; ++q)
+          *(uint4*)(dst + lane * 64 + ((q ^ ((lane >> 1) & 3)) << 4)) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) {
-        tma_store_2d(map, n0, m_warp0, stg);
+        tma_store_2d(map, n0, m_warp0, dst);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
     } else if (row_ok) {
@@ -321,21 +357,17 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
         bf16* dst = (bf16*)base + off;
         if (VEC) {
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint4 u;
-            __nv_bfloat162* h = (__nv_bfloat162*)&u;
-#pragma unroll
-            for (int t = 0; t < 4; ++t) h[t] = __floats2bfloat162_rn(o[q * 8 + 2 * t], o[q * 8 + 2 * t + 1]);
-            *(uint4*)(dst + q * 8) = u;
-          }
+          for (int q = 0; q < 4; ++q) *(uint4*)(dst + q * 8) = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
         } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) if (j < nvalid) dst[j] = __float2bfloat16_rn(o[j]);
+          for (int j = 0; j < 32; ++j)
+            if (j < nvalid) ((uint16_t*)dst)[j] = (uint16_t)((j & 1) ? (pk[j >> 1] >> 16) : (pk[j >> 1] & 0xffffu));
         }
       }
     }
   };
   float t[32];
+  uint32_t pk[16];
   if (p.resid) {
     load32(p.resid, t);
 #pragma unroll
@@ -347,12 +379,15 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
       for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
       break;
     case EPI_GELU:
-#pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = __bfloat162float(__float2bfloat16_rn(v[j]));
-      put(p.C2, mapC2, v, false);
+      // the pre-activation is stored (C2) and the activation is taken of the value as stored
+      pack32(v, pk);
+      unpack32(pk, v);
+      put(p.C2, mapC2, pk, nullptr, false, 0);
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
-      break;
+      pack32(v, pk);
+      put(p.C, mapC, pk, nullptr, false, 1);
+      return;
     case EPI_RELU_MASK:
       load32(p.aux, t);
 #pragma unroll
@@ -366,23 +401,29 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
     case EPI_LOGIT_STATS: {
       // running (max, sum of exp(z - max)) of this row over the warp's columns, on the values as stored
       const float L2E = 1.4426950408889634f;
+      pack32(v, pk);
+      unpack32(pk, v);
       float cm = -INFINITY;
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        v[j] = __bfloat162float(__float2bfloat16_rn(v[j]));
+      for (int j = 0; j < 32; ++j)
         if (VEC || j < nvalid) cm = fmaxf(cm, v[j]);
-      }
       const float nm = fmaxf(run.x, cm), nml = nm * L2E;
       float cs = 0.f;
 #pragma unroll
       for (int j = 0; j < 32; ++j) if (VEC || j < nvalid) cs += ex2_approx(fmaf(v[j], L2E, -nml));
       run.y = (run.x == -INFINITY ? 0.f : run.y * ex2_approx((run.x - nm) * L2E)) + cs;
       run.x = nm;
-      break;
+      put(p.C, mapC, pk, nullptr, false, 0);
+      return;
     }
     default: break;
   }
-  put(p.C, mapC, v, p.out_f32 != 0);
+  if (p.out_f32) {
+    put(p.C, mapC, nullptr, v, true, 0);
+  } else {
+    pack32(v, pk);
+    put(p.C, mapC, pk, nullptr, false, 0);
+  }
 }
 
 // ---- cluster helpers (CG = 2)
@@ -466,18 +507,23 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
     // ------------------------------------------------------------------ TMA producer (one per CTA)
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
-      int pi = 0;
       bool ok = true;
+      ProbCursor cur(probs, nprob);
+      TileWalk walk;
+      bool a_mn = false, b_mn = false;
+      int kb_n = 0;
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
-        while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
-        const GemmProb& p = probs[pi];
-        const CUtensorMap* mapA = maps + 4 * pi;
+        if (cur.seek(tile)) {                        // problem changed: re-read its fields (once per problem, not per tile)
+          const GemmProb& p = probs[cur.pi];
+          walk.set(p, TILE_M);
+          a_mn = p.a_ms == 1; b_mn = p.b_ns == 1;
+          kb_n = (p.K + BK - 1) / BK;
+        }
+        const CUtensorMap* mapA = maps + 4 * cur.pi;
         const CUtensorMap* mapB = mapA + 1;
         int mt, nt;
-        tile_coords(p, tile - p.tile_start, TILE_M, mt, nt);
+        walk.coords(tile, mt, nt);
         int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN + (int)rank * BNL;
-        bool a_mn = p.a_ms == 1, b_mn = p.b_ns == 1;
-        int kb_n = (p.K + BK - 1) / BK;
         for (int kb = 0; kb < kb_n; ++kb) {
           if (!(ok = mbar_wait(&sh->empty[stage], phase ^ 1, sh, status))) break;
           uint8_t* a_dst = tiles + stage * STAGE_BYTES;
@@ -528,20 +574,27 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
     // ------------------------------------------------------------------ MMA issuer (the pair's leader only)
     if (lane == 0 && rank == 0) {
       int stage = 0; uint32_t phase = 0;
-      int pi = 0, it = 0;
+      int it = 0;
       bool ok = true;
+      // The issuer runs only a few k-slices ahead of the tensor pipe, so whatever it does between two tiles
+      // must be short: the problem's fields stay in registers and are re-read only when the problem changes.
+      ProbCursor cur(probs, nprob);
+      bool a_mn = false, b_mn = false;
+      int kb_n = 0;
+      uint32_t idesc = 0;
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
-        while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
-        const GemmProb& p = probs[pi];
-        bool a_mn = p.a_ms == 1, b_mn = p.b_ns == 1;
-        uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-                         ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+        if (cur.seek(tile)) {
+          const GemmProb& p = probs[cur.pi];
+          a_mn = p.a_ms == 1; b_mn = p.b_ns == 1;
+          kb_n = (p.K + BK - 1) / BK;
+          idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+                  ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+        }
         int ab = it & 1;
         uint32_t use = (uint32_t)(it >> 1);
         if (!(ok = mbar_wait(&sh->tmem_empty[ab], (use & 1) ^ 1, sh, status))) break;
         tc_fence_after();
         uint32_t d_tmem = tmem_base + ab * BN;
-        int kb_n = (p.K + BK - 1) / BK;
         for (int kb = 0; kb < kb_n; ++kb) {
           if (!(ok = mbar_wait(&sh->full[stage], phase, sh, status))) break;
           tc_fence_after();
@@ -566,13 +619,16 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(EPI_REGS));
     // ------------------------------------------------------------------ epilogue warps
     const int quarter = warp & 3;            // TMEM lanes [32*quarter, 32*quarter + 32) belong to this warp
-    int pi = 0, it = 0;
+    int it = 0;
     bool ok = true;
+    ProbCursor cur(probs, nprob);
+    TileWalk walk;
     for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
-      while (pi + 1 < nprob && probs[pi + 1].tile_start <= tile) ++pi;
-      const GemmProb p = probs[pi];
+      if (cur.seek(tile)) walk.set(probs[cur.pi], TILE_M);
+      const int pi = cur.pi;
+      const GemmProb p = probs[pi];          // read-only table: fields are fetched where they are used
       int mt, nt;
-      tile_coords(p, tile - p.tile_start, TILE_M, mt, nt);
+      walk.coords(tile, mt, nt);
       int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN;
       int ab = it & 1;
       uint32_t use = (uint32_t)(it >> 1);
