@@ -206,6 +206,24 @@ typedef struct {
 lp_status lp_gemm_bf16(int n, const lp_gemm_desc* probs, int backend, void* stream, int* used_tensor_cores);
 
 /*
+ * lp_conv3x3_bf16: kernel-level entry for tests and profiling: one 3x3 convolution, stride 1, zero padding 1,
+ * no bias, over bf16 NHWC activations (the residual blocks of App. B.3), as an implicit GEMM on the tensor
+ * cores: the activation tensor itself is the GEMM operand, fetched as one shifted box per filter tap; no
+ * im2col matrix exists.  All pointers are device pointers.
+ *   LP_CONV_FORWARD:     act = x  [n,h,w,c_in],  other = filters [c_out,3,3,c_in] bf16, out = y  [n,h,w,c_out] bf16
+ *                        y[n,p,q,o] = sum_{i,j,c} x[n,p+i-1,q+j-1,c] * filters[o,i,j,c]
+ *   LP_CONV_INPUT_GRAD:  act = dy [n,h,w,c_out], other = filters,                     out = dx [n,h,w,c_in]  bf16
+ *   LP_CONV_FILTER_GRAD: act = x  [n,h,w,c_in],  other = dy [n,h,w,c_out] bf16,       out = dW [c_out,3,3,c_in] fp32
+ * Accepted sizes: the channel count of `act` a multiple of 64, the other channel count a multiple of 8,
+ * w a divisor of 64, h*w a divisor or a multiple of 128, 16-byte aligned tensors; otherwise
+ * LP_ERR_UNSUPPORTED and nothing is launched.  Asynchronous on `stream` except for the upload of the
+ * descriptor table.  Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALLOC, CUDA (message: lp_last_error(NULL)).
+ */
+enum { LP_CONV_FORWARD = 0, LP_CONV_INPUT_GRAD = 1, LP_CONV_FILTER_GRAD = 2 };
+lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* out, int n, int h, int w,
+                          int c_in, int c_out, void* stream);
+
+/*
  * lp_gemm_bf16_static: lp_gemm_bf16 for callers that cannot allocate device memory.  (The paper
  * has no counterpart to this entry point; it exists for the library's users.)
  *

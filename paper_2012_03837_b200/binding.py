@@ -60,7 +60,7 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
-           "lp_gemm_bf16_static", "lp_gemm_static_last_error"]
+           "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
 
@@ -274,6 +274,17 @@ def lp_gemm_bf16(descs: list, backend: int = 0, stream=None) -> int:
 
 
 LP_GEMM_STATIC_MAX = 64
+LP_CONV_FORWARD, LP_CONV_INPUT_GRAD, LP_CONV_FILTER_GRAD = 0, 1, 2
+_lib.lp_conv3x3_bf16.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                 C.c_void_p]
+
+
+def lp_conv3x3_bf16(form: int, act, other, out, n: int, h: int, w: int, c_in: int, c_out: int, stream=None) -> None:
+    """One implicit-GEMM 3x3 convolution (stride 1, padding 1) over bf16 NHWC tensors: forward, input
+    gradient or filter gradient (see lp.h).  Tensors may be torch tensors or raw device pointers."""
+    _check(None, _lib.lp_conv3x3_bf16(form, _ptr(act), _ptr(other), _ptr(out), n, h, w, c_in, c_out, stream))
+
+
 _lib.lp_gemm_bf16_static.argtypes = [C.c_int, C.POINTER(lp_gemm_desc), C.c_void_p]
 _lib.lp_gemm_static_last_error.restype = C.c_char_p
 

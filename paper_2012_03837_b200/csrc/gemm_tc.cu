@@ -115,6 +115,13 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// 4-D tiled load (implicit convolution: channel, column, row, image); coordinates may lie outside the
+// tensor in every dimension but the first, the box then reads as zero there.
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
@@ -453,6 +460,11 @@ __device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* m
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
       ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(bar_caddr), "l"(policy_evict_last()) : "memory");
 }
+__device__ __forceinline__ void tma_load_4d_pair(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar_caddr) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar_caddr), "l"(policy_evict_last()) : "memory");
+}
 __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {   // arrives on this barrier in both CTAs of the pair
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
@@ -512,54 +524,74 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       TileWalk walk;
       bool a_mn = false, b_mn = false;
       int kb_n = 0;
+      int conv = 0, cv_c = 64, cv_w = 1, cv_hw = 1, cv_n = 0, cv_k0 = 0, p_n = 0;
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
         if (cur.seek(tile)) {                        // problem changed: re-read its fields (once per problem, not per tile)
           const GemmProb& p = probs[cur.pi];
           walk.set(p, TILE_M);
           a_mn = p.a_ms == 1; b_mn = p.b_ns == 1;
           kb_n = (p.K + BK - 1) / BK;
+          conv = p.conv;
+          if (conv) { cv_c = p.conv_c; cv_w = p.conv_w; cv_hw = p.conv_h * p.conv_w; cv_n = p.conv_n; cv_k0 = p.conv_k0; p_n = p.N; }
         }
         const CUtensorMap* mapA = maps + 4 * cur.pi;
         const CUtensorMap* mapB = mapA + 1;
         int mt, nt;
         walk.coords(tile, mt, nt);
         int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN + (int)rank * BNL;
+        // implicit convolution: this CTA's 128 output pixels start at row a_h0 of image a_img (whole rows)
+        int a_img = 0, a_h0 = 0;
+        if (conv == CONV_FWD || conv == CONV_DGRAD) { a_img = m0 / cv_hw; a_h0 = (m0 - a_img * cv_hw) / cv_w; }
         for (int kb = 0; kb < kb_n; ++kb) {
           if (!(ok = mbar_wait(&sh->empty[stage], phase ^ 1, sh, status))) break;
           uint8_t* a_dst = tiles + stage * STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_BYTES;
           int k0 = kb * BK;
-          if (CG == 1) {
-            uint64_t* bar = &sh->full[stage];
-            mbar_expect_tx(bar, STAGE_BYTES);
-            if (a_mn) {
+          // both CTAs' bytes of a pair are counted on the leader's barrier
+          uint64_t* bar1 = &sh->full[stage];
+          uint32_t bar2 = 0;
+          if (CG == 1) mbar_expect_tx(bar1, STAGE_BYTES);
+          else { bar2 = map_to_rank(smem_u32(bar1), 0); mbar_expect_tx_cluster(bar2, STAGE_BYTES); }
+          auto ld2 = [&](void* dst, const CUtensorMap* map, int x, int y) {
+            if (CG == 1) tma_load_2d(dst, map, x, y, bar1); else tma_load_2d_pair(dst, map, x, y, bar2);
+          };
+          auto ld4 = [&](void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3) {
+            if (CG == 1) tma_load_4d(dst, map, c0, c1, c2, c3, bar1); else tma_load_4d_pair(dst, map, c0, c1, c2, c3, bar2);
+          };
+          // filter tap and channel block of this k-slice (CONV_FWD / CONV_DGRAD: k = tap * conv_c + channel)
+          int tap = 0, ch0 = 0;
+          if (conv == CONV_FWD || conv == CONV_DGRAD) { const int cb = cv_c >> 6; tap = kb / cb; ch0 = (kb - tap * cb) << 6; }
+          // ---- A
+          if (conv == CONV_FWD || conv == CONV_DGRAD) {
+            int di = tap / 3 - 1, dj = tap - (tap / 3) * 3 - 1;
+            if (conv == CONV_DGRAD) { di = -di; dj = -dj; }
+            ld4(a_dst, mapA, ch0, dj, a_h0 + di, a_img);
+          } else if (a_mn) {
 #pragma unroll
-              for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, bar);
-            } else {
-              tma_load_2d(a_dst, mapA, k0, m0, bar);
-            }
-            if (b_mn) {
-#pragma unroll
-              for (int i = 0; i < BNL / 64; ++i) tma_load_2d(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, bar);
-            } else {
-              tma_load_2d(b_dst, mapB, k0, n0, bar);
-            }
+            for (int i = 0; i < BM / 64; ++i) ld2(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0);
           } else {
-            // both CTAs' bytes are counted on the leader's barrier
-            uint32_t bar = map_to_rank(smem_u32(&sh->full[stage]), 0);
-            mbar_expect_tx_cluster(bar, STAGE_BYTES);
-            if (a_mn) {
+            ld2(a_dst, mapA, k0, m0);
+          }
+          // ---- B
+          if (conv == CONV_WGRAD) {
+            const int kp = cv_k0 + k0;               // first pixel of this k-slice (whole rows, 64 pixels)
+            const int img = kp / cv_hw, h0 = (kp - img * cv_hw) / cv_w;
 #pragma unroll
-              for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, bar);
-            } else {
-              tma_load_2d_pair(a_dst, mapA, k0, m0, bar);
+            for (int i = 0; i < BNL / 64; ++i) {
+              const int col = n0 + i * 64;           // column block -> (tap, channel block)
+              const int t = col / cv_c, c0 = col - t * cv_c;
+              if (t < 9) ld4(b_dst + i * (BK * 128), mapB, c0, t - (t / 3) * 3 - 1, h0 + t / 3 - 1, img);
+              else ld4(b_dst + i * (BK * 128), mapB, 0, 0, 0, cv_n);        // beyond the last tap: an all-zero box
             }
-            if (b_mn) {
+          } else if (conv == CONV_DGRAD) {
+            // filters [conv_c, 3, 3, N] read in place: rows = output channel (the reduction), columns (tap, n)
 #pragma unroll
-              for (int i = 0; i < BNL / 64; ++i) tma_load_2d_pair(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, bar);
-            } else {
-              tma_load_2d_pair(b_dst, mapB, k0, n0, bar);
-            }
+            for (int i = 0; i < BNL / 64; ++i) ld2(b_dst + i * (BK * 128), mapB, tap * p_n + n0 + i * 64, ch0);
+          } else if (b_mn) {
+#pragma unroll
+            for (int i = 0; i < BNL / 64; ++i) ld2(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0);
+          } else {
+            ld2(b_dst, mapB, k0, n0);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -729,10 +761,43 @@ bool encode_map(CUtensorMap* out, const void* base, long long inner, long long o
   return r == CUDA_SUCCESS;
 }
 
+// 4-D bf16 tensor map of an NHWC activation tensor [n, h, w, c] for the implicit convolution: boxes of
+// 64 channels x whole image rows that hold `pixels` pixels (128: a K-major A tile; 64: one k-slice of an
+// MN-major B tile), i.e. (w, pixels / w, 1) inside an image or (w, h, pixels / (h w)) across small images.
+// 128-byte swizzle; everything outside the tensor (the padding ring of the convolution) reads as zero.
+bool encode_map4(CUtensorMap* out, const void* base, int n, int h, int w, int c, int pixels) {
+  EncodeFn fn = get_encode();
+  if (!fn) return false;
+  const long long hw = (long long)h * w;
+  cuuint32_t bw = (cuuint32_t)w, bh, bn;
+  if (hw >= pixels) { bh = (cuuint32_t)(pixels / w); bn = 1; }
+  else { bh = (cuuint32_t)h; bn = (cuuint32_t)(pixels / hw); }
+  cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+  cuuint64_t strides[3] = {(cuuint64_t)c * 2, (cuuint64_t)w * c * 2, (cuuint64_t)hw * c * 2};
+  cuuint32_t box[4] = {64u, bw, bh, bn};
+  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool gemm_tc_eligible(const GemmProb& g) {
   if (g.M < 1 || g.N < 1 || g.K < 1) return false;
+  if (g.conv != CONV_NONE) {
+    // implicit 3x3 convolution: whole-row boxes, 64-channel k-slices, filters with 16-byte pitches
+    if (g.conv_c < 64 || g.conv_c % 64 || g.conv_n < 1 || !conv_boxes_ok(g.conv_h, g.conv_w)) return false;
+    if (((uintptr_t)g.A & 15) || ((uintptr_t)g.B & 15)) return false;
+    const long long pixels = (long long)g.conv_n * g.conv_h * g.conv_w;
+    if (g.conv == CONV_FWD) return g.K == 9 * g.conv_c && g.M == pixels && g.b_ks == 1 && g.b_ns % 8 == 0 && get_encode() != nullptr;
+    if (g.conv == CONV_DGRAD) return g.K == 9 * g.conv_c && g.M == pixels && g.N % 8 == 0 && get_encode() != nullptr;
+    if (g.conv == CONV_WGRAD)
+      return g.N == 9 * g.conv_c && g.a_ms == 1 && g.a_ks % 8 == 0 && g.conv_k0 % 64 == 0 && g.conv_k0 + g.K <= pixels &&
+             get_encode() != nullptr;
+    return false;
+  }
   if ((long long)g.M * g.N < 64 * 64 || g.K < 32) return false;          // too small to pay for a 128x256 tile
   if (((uintptr_t)g.A & 15) || ((uintptr_t)g.B & 15)) return false;
   long long a_pitch = g.a_ms == 1 ? g.a_ks : g.a_ms, b_pitch = g.b_ns == 1 ? g.b_ks : g.b_ns;
@@ -795,9 +860,12 @@ bool gemm_tc_encode(GemmProb& g, void* maps, int cg) {
     g.store_tma = ok ? (wide ? 2 : 1) : 0;
   }
   bool okA, okB;
-  if (g.a_ms == 1) okA = encode_map(mapA, g.A, g.M, g.K, g.a_ks, BK);       // MN-major: rows are k
+  if (g.conv == CONV_FWD || g.conv == CONV_DGRAD) okA = encode_map4(mapA, g.A, g.conv_n, g.conv_h, g.conv_w, g.conv_c, BM);
+  else if (g.a_ms == 1) okA = encode_map(mapA, g.A, g.M, g.K, g.a_ks, BK);       // MN-major: rows are k
   else okA = encode_map(mapA, g.A, g.K, g.M, g.a_ms, BM);
-  if (g.b_ns == 1) okB = encode_map(mapB, g.B, g.N, g.K, g.b_ks, BK);
+  if (g.conv == CONV_WGRAD) okB = encode_map4(mapB, g.B, g.conv_n, g.conv_h, g.conv_w, g.conv_c, BK);
+  else if (g.conv == CONV_DGRAD) okB = encode_map(mapB, g.B, 9LL * g.N, g.conv_c, 9LL * g.N, BK);   // rows: output channel
+  else if (g.b_ns == 1) okB = encode_map(mapB, g.B, g.N, g.K, g.b_ks, BK);
   else okB = encode_map(mapB, g.B, g.K, g.N, g.b_ns, BN / cg);
   return okA && okB;
 }

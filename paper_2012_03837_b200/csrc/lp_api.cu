@@ -453,6 +453,61 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream,
   return check_cuda(nullptr, "lp_gemm_bf16");
 }
 
+lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* out, int n, int hgt, int wid, int c_in,
+                          int c_out, void* stream) {
+  if (!act || !other || !out) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_conv3x3_bf16: null pointer");
+  if (n < 1 || hgt < 1 || wid < 1 || c_in < 1 || c_out < 1) return fail(nullptr, LP_ERR_SHAPE, "lp_conv3x3_bf16: sizes must be positive");
+  const long long pixels = (long long)n * hgt * wid;
+  if (pixels > 0x7fffffffLL) return fail(nullptr, LP_ERR_SHAPE, "lp_conv3x3_bf16: too many pixels");
+  GemmProb g{};
+  g.conv_n = n; g.conv_h = hgt; g.conv_w = wid;
+  switch (form) {
+    case LP_CONV_FORWARD:        // act = x [n,h,w,c_in], other = filters [c_out,3,3,c_in], out = y [n,h,w,c_out]
+      g.A = act; g.B = other; g.C = out; g.M = (int)pixels; g.N = c_out; g.K = 9 * c_in;
+      g.a_ms = c_in; g.a_ks = 1; g.b_ns = 9LL * c_in; g.b_ks = 1; g.ldc = c_out;
+      g.conv = CONV_FWD; g.conv_c = c_in;
+      break;
+    case LP_CONV_INPUT_GRAD:     // act = dy [n,h,w,c_out], other = filters, out = dx [n,h,w,c_in]
+      g.A = act; g.B = other; g.C = out; g.M = (int)pixels; g.N = c_in; g.K = 9 * c_out;
+      g.a_ms = c_out; g.a_ks = 1; g.b_ns = 1; g.b_ks = 9LL * c_in; g.ldc = c_in;
+      g.conv = CONV_DGRAD; g.conv_c = c_out;
+      break;
+    case LP_CONV_FILTER_GRAD:    // act = x [n,h,w,c_in], other = dy [n,h,w,c_out], out = dW [c_out,3,3,c_in] fp32
+      g.A = other; g.B = act; g.C = out; g.M = c_out; g.N = 9 * c_in; g.K = (int)pixels;
+      g.a_ms = 1; g.a_ks = c_out; g.b_ns = 1; g.b_ks = c_in; g.ldc = 9 * c_in; g.out_f32 = 1;
+      g.conv = CONV_WGRAD; g.conv_c = c_in;
+      break;
+    default: return fail(nullptr, LP_ERR_INVALID_ARG, "lp_conv3x3_bf16: unknown form");
+  }
+  if (!gemm_tc_eligible(g))
+    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_conv3x3_bf16: needs 16-byte aligned tensors, the shifted operand's channels a multiple of 64, "
+                                             "the other channel count a multiple of 8, a width dividing 64 and h*w dividing or divisible by 128");
+  cudaStream_t s = (cudaStream_t)stream;
+  static int* d_status = nullptr;
+  static void* d_tab = nullptr;
+  static int num_sms = 0;
+  struct alignas(64) Map { unsigned char b[128]; };
+  if (!d_tab) {
+    if (cudaMalloc(&d_tab, 1024 + 4 * sizeof(Map)) != cudaSuccess) { cudaGetLastError(); d_tab = nullptr; return fail(nullptr, LP_ERR_ALLOC, "descriptor table"); }
+    d_status = (int*)d_tab;
+    cudaMemset(d_status, 0, sizeof(int));
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  const int cg = gemm_tc_choose_cg(&g, 1);
+  const int total = gemm_tc_tiles(g, 0, cg);
+  Map maps[4];
+  if (!gemm_tc_encode(g, maps, cg)) return fail(nullptr, LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+  GemmProb* dp = (GemmProb*)((char*)d_tab + 256);
+  Map* dm = (Map*)((char*)d_tab + 1024);
+  cudaMemcpyAsync(dp, &g, sizeof(GemmProb), cudaMemcpyHostToDevice, s);
+  cudaMemcpyAsync(dm, maps, sizeof(maps), cudaMemcpyHostToDevice, s);
+  cudaStreamSynchronize(s);                      // the tables above are host stack memory
+  launch_gemm_tc(dp, dm, 1, total, d_status, num_sms, s, cg);
+  return check_cuda(nullptr, "lp_conv3x3_bf16");
+}
+
 lp_status lp_profile_enable(lp_handle hh, int on) {
   if (!hh) return LP_ERR_INVALID_ARG;
   hh->h.profiling = on != 0;

@@ -42,7 +42,27 @@ struct GemmProb {
   int tiles_n;
   int store_tma;   // tensor-core kernel: outputs leave through TMA stores (set by the launcher when C's pitch allows)
   int raster;      // tensor-core kernel: row tiles per band of the tile walk (set by the launcher)
+  // Implicit 3x3 convolution, stride 1, padding 1, over NHWC activations (tensor-core kernel only; App. B.3's
+  // residual blocks).  One operand is never materialised as a matrix: its tiles are fetched as shifted boxes
+  // of the activation tensor [conv_n, conv_h, conv_w, conv_c], one shift per filter tap (i, j), rows and
+  // columns outside the image reading as zero.
+  //   CONV_FWD   : A(m, k) = x[pixel m shifted by (i-1, j-1)][c],  k = (3i + j) conv_c + c;  K = 9 conv_c;
+  //                B = filters [N, 9 conv_c] (reduction index contiguous).
+  //   CONV_DGRAD : A(m, k) = dy[pixel m shifted by (1-i, 1-j)][co], k = (3i + j) conv_c + co; K = 9 conv_c;
+  //                B(n, k) = filters[co][(3i + j) N + n]  (the filter tensor [conv_c, 3, 3, N] read in place).
+  //   CONV_WGRAD : B(n, k) = x[pixel conv_k0 + k shifted by (i-1, j-1)][ci], n = (3i + j) conv_c + ci;
+  //                N = 9 conv_c; A(m, k) = dy[pixel k][m] as an ordinary MN-major operand; K = pixels.
+  // A is the activation tensor for CONV_FWD / CONV_DGRAD, B for CONV_WGRAD.
+  int conv;
+  int conv_n, conv_h, conv_w, conv_c;
+  int conv_k0;     // CONV_WGRAD: first pixel of this slice of the reduction (split-K)
 };
+enum { CONV_NONE = 0, CONV_FWD = 1, CONV_DGRAD = 2, CONV_WGRAD = 3 };
+// True if an image of h x w pixels can be walked in whole-row boxes of 128 and of 64 pixels.
+inline bool conv_boxes_ok(int h, int w) {
+  const long long hw = (long long)h * w;
+  return w >= 1 && 64 % w == 0 && (hw % 128 == 0 || 128 % hw == 0);
+}
 
 // FP32-ALU GEMM (any sizes and strides).  T = float or bf16 operands, fp32 accumulation.
 void launch_gemm_simt(const GemmProb* d_probs, const GemmProb* h_probs, int n, bool is_bf16,

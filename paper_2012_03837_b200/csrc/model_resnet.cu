@@ -22,6 +22,8 @@ struct Conv {
   int ldk;       // pitch of the cols matrix: K rounded up to 8 elements (16 bytes for bf16), pad columns stay zero
   void* cols = nullptr;
   void* y = nullptr;
+  // implicit GEMM on the tensor-core kernel (no im2col / col2im): forward and weight gradient, input gradient
+  bool imp_fwd = false, imp_dgrad = false;
 };
 struct Bn {
   std::string g, b;
@@ -120,8 +122,16 @@ void build_resnet(Handle& h) {
   h.y_bytes = (size_t)B * sizeof(int);
   h.y_in = (int*)h.dalloc(h.y_bytes);
   auto fal = [&](size_t n) { return (float*)h.dalloc(n * sizeof(float)); };
+  // 3x3 stride-1 convolutions whose channel counts are multiples of 64 run as implicit GEMMs: the activation
+  // tensor itself is the operand (shifted TMA boxes per filter tap), nothing 9 times its size is written.
+  auto set_implicit = [&](Conv& c) {
+    const bool base = bf && !h.force_simt && c.k == 3 && c.stride == 1 && conv_boxes_ok(c.H, c.W);
+    c.imp_fwd = base && c.Cin % 64 == 0 && c.Cout % 8 == 0;
+    c.imp_dgrad = base && c.Cout % 64 == 0 && c.Cin % 8 == 0;
+  };
   auto alloc_conv = [&](Conv& c) {
-    c.cols = h.dalloc((size_t)c.M * c.ldk * es);
+    set_implicit(c);
+    if (!c.imp_fwd) c.cols = h.dalloc((size_t)c.M * c.ldk * es);
     c.y = h.dalloc((size_t)c.M * c.Cout * es);
   };
   auto alloc_bn = [&](Bn& b) { b.mean = fal(b.C); b.rstd = fal(b.C); };
@@ -138,7 +148,7 @@ void build_resnet(Handle& h) {
     auto track = [&](const Conv& cv) {
       max_act = std::max(max_act, (size_t)cv.M * cv.Cout);
       max_act = std::max(max_act, (size_t)cv.N * cv.H * cv.W * cv.Cin);
-      max_cols = std::max(max_cols, (size_t)cv.M * cv.ldk);
+      if (!cv.imp_dgrad) max_cols = std::max(max_cols, (size_t)cv.M * cv.ldk);
     };
     if (c.has_stem) {
       c.x_nhwc = h.dalloc(in_elems * es);
@@ -158,11 +168,21 @@ void build_resnet(Handle& h) {
     c.z = h.dalloc((size_t)B * NC * es);
     c.row_loss = fal(B);
     for (int i = 0; i < 4; ++i) c.G[i] = h.dalloc(max_act * es);
-    c.dcols = h.dalloc(max_cols * es);
+    c.dcols = max_cols ? h.dalloc(max_cols * es) : nullptr;
   }
 
   // ---- op emitters (one problem per launch: the stages differ in every size)
+  auto conv_fields = [&](GemmProb& g, const Conv& c, int mode, int channels) {
+    g.conv = mode; g.conv_n = c.N; g.conv_h = c.H; g.conv_w = c.W; g.conv_c = channels; g.conv_k0 = 0;
+  };
   auto conv_fwd = [&](Plan& p, const Conv& c, const void* x) {
+    if (c.imp_fwd) {
+      GemmProb g = gemm_fwd(x, h.W(c.w), c.y, (int)c.M, c.Cout, c.K, nullptr, EPI_NONE);
+      g.a_ms = c.Cin;
+      conv_fields(g, c, CONV_FWD, c.Cin);
+      emit_gemm(h, p, {g});
+      return;
+    }
     Im2colProb ip{x, c.cols, c.N, c.H, c.W, c.Cin, c.k, c.k, c.stride, c.pad, c.Ho, c.Wo, c.ldk};
     const Im2colProb* d = h.upload(std::vector<Im2colProb>{ip});
     long long elems = c.M * c.K;
@@ -172,12 +192,30 @@ void build_resnet(Handle& h) {
     g.a_ms = c.ldk;
     emit_gemm(h, p, {g});
   };
-  auto conv_wgrad = [&](Plan& p, const Conv& c, const void* dy) {
+  // x: the convolution's input in this plan (the operand of the implicit form; the explicit form reads c.cols)
+  auto conv_wgrad = [&](Plan& p, const Conv& c, const void* dy, const void* x) {
+    if (c.imp_fwd) {
+      GemmProb g = gemm_wgrad(dy, x, h.G(c.w), (int)c.M, c.Cout, c.K);
+      g.b_ks = c.Cin;
+      conv_fields(g, c, CONV_WGRAD, c.Cin);
+      emit_gemm(h, p, {g});
+      return;
+    }
     GemmProb g = gemm_wgrad(dy, c.cols, h.G(c.w), (int)c.M, c.Cout, c.K);
     g.b_ks = c.ldk;
     emit_gemm(h, p, {g});
   };
   auto conv_dgrad = [&](Plan& p, const Conv& c, const void* dy, void* dx, void* dcols) {
+    if (c.imp_dgrad) {
+      // dx[pixel, ci] = sum over taps and output channels of dy[pixel shifted back by the tap][co] * W[co][tap][ci]
+      GemmProb g{};
+      g.A = dy; g.B = h.W(c.w); g.C = dx;
+      g.M = (int)c.M; g.N = c.Cin; g.K = 9 * c.Cout;
+      g.a_ms = c.Cout; g.a_ks = 1; g.b_ns = 1; g.b_ks = 9LL * c.Cin; g.ldc = c.Cin;
+      conv_fields(g, c, CONV_DGRAD, c.Cout);
+      emit_gemm(h, p, {g});
+      return;
+    }
     GemmProb g = gemm_dgrad(dy, h.W(c.w), dcols, (int)c.M, c.Cout, c.K, EPI_NONE, nullptr);
     g.ldc = c.ldk;
     emit_gemm(h, p, {g});
@@ -301,15 +339,15 @@ void build_resnet(Handle& h) {
       bool need_dx = (j > 0) || c.has_stem;
       // out = relu(bn2(c2) + shortcut): ga <- d(c2), gb <- gradient of the shortcut branch
       bn_bwd(p, b.b2, b.c2.y, gin, out, ga, gb);
-      conv_wgrad(p, b.c2, ga);
+      conv_wgrad(p, b.c2, ga, b.a1);
       conv_dgrad(p, b.c2, ga, gc, c.dcols);                 // gc <- d(a1)
       bn_bwd(p, b.b1, b.c1.y, gc, b.a1, ga, nullptr);       // ga <- d(c1)
-      conv_wgrad(p, b.c1, ga);
+      conv_wgrad(p, b.c1, ga, x);
       long long in_elems_blk = (long long)b.c1.N * b.c1.H * b.c1.W * b.c1.Cin;
       if (need_dx) conv_dgrad(p, b.c1, ga, gc, c.dcols);    // gc <- d(x) through the main branch
       if (b.has_sc) {
         bn_bwd(p, b.bs, b.cs.y, gb, nullptr, ga, nullptr);  // ga <- d(cs)
-        conv_wgrad(p, b.cs, ga);
+        conv_wgrad(p, b.cs, ga, x);
         if (need_dx) {
           conv_dgrad(p, b.cs, ga, gin, c.dcols);            // gin <- d(x) through the shortcut
           add_into(p, gc, gin, in_elems_blk);
@@ -321,7 +359,7 @@ void build_resnet(Handle& h) {
     }
     if (c.has_stem) {
       bn_bwd(p, c.stem_bn, c.stem.y, gin, c.stem_out, ga, nullptr);
-      conv_wgrad(p, c.stem, ga);
+      conv_wgrad(p, c.stem, ga, c.x_nhwc);
     }
   };
 

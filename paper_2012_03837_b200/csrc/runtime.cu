@@ -122,7 +122,8 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
         GemmProb q = g;
         q.K = std::min(kc, g.K - k0);
         q.A = (const char*)g.A + (size_t)k0 * g.a_ks * es;
-        q.B = (const char*)g.B + (size_t)k0 * g.b_ks * es;
+        if (g.conv == CONV_WGRAD) q.conv_k0 = g.conv_k0 + k0;     // the implicit operand is addressed by pixel, not by pointer
+        else q.B = (const char*)g.B + (size_t)k0 * g.b_ks * es;
         q.C = part + (size_t)made * mn;
         expanded.push_back(q);
       }
@@ -134,6 +135,7 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
   std::vector<GemmProb> tc, simt;
   for (auto& g : probs) {
     if (!h.force_simt && gemm_tc_eligible(g)) tc.push_back(g);
+    else if (g.conv != CONV_NONE) throw std::runtime_error("internal: implicit convolution problem not accepted by the tensor-core kernel");
     else simt.push_back(g);
   }
   if (!tc.empty()) {

@@ -91,3 +91,52 @@ def test_epilogues_match_between_backends():
     # and the FP32-ALU GELU output equals the oracle's GELU of its own stored pre-activation
     u, g = outs[1][3], outs[1][2]
     assert np.abs(lp_synth.bf16_round(L.gelu_fwd(u.astype(np.float64))[0].astype(np.float32)) - g).max() < 1e-2
+
+
+# ------------------------------------------------------------------ implicit-GEMM 3x3 convolution
+
+@pytest.mark.parametrize("n,h,w,c_in,c_out", [
+    (3, 16, 16, 64, 128),     # boxes of 8 (4) rows inside an image; 768 pixels = three 256-row tiles
+    (5, 8, 8, 128, 64),       # 128-pixel boxes span two images; 320 pixels: ragged last tile, box past the last image
+    (9, 4, 4, 64, 64),        # boxes of eight (four) whole images; 144 pixels
+    (2, 32, 32, 64, 72),      # four (two) rows of a 32 x 32 image per box; output channels not a multiple of 64
+])
+def test_implicit_convolution_against_the_oracle(n, h, w, c_in, c_out):
+    """Forward, input gradient and filter gradient of a 3x3 stride-1 convolution (App. B.3's residual blocks)
+    through lp_conv3x3_bf16 against the oracle's convolution, element by element."""
+    rng = np.random.default_rng(n * 1000 + h * 10 + c_in)
+    x = lp_synth.bf16_round(rng.standard_normal((n, c_in, h, w)).astype(np.float32))                   # NCHW (oracle layout)
+    W = lp_synth.bf16_round((rng.standard_normal((c_out, c_in, 3, 3)) / np.sqrt(9 * c_in)).astype(np.float32))
+    dy = lp_synth.bf16_round(rng.standard_normal((n, c_out, h, w)).astype(np.float32))
+    y_ref, cache = L.conv2d_fwd(x.astype(np.float64), W.astype(np.float64), 1, 1)
+    dx_ref, dW_ref = L.conv2d_bwd(dy.astype(np.float64), cache)
+    nhwc = lambda a: np.ascontiguousarray(a.transpose(0, 2, 3, 1))
+    xd, dyd = bf(nhwc(x)), bf(nhwc(dy))
+    Wd = bf(np.ascontiguousarray(W.transpose(0, 2, 3, 1)))                                             # [c_out, 3, 3, c_in]
+    y = torch.zeros(n, h, w, c_out, dtype=torch.bfloat16, device="cuda")
+    dx = torch.zeros(n, h, w, c_in, dtype=torch.bfloat16, device="cuda")
+    dW = torch.zeros(c_out, 3, 3, c_in, dtype=torch.float32, device="cuda")
+    lp.lp_conv3x3_bf16(lp.LP_CONV_FORWARD, xd, Wd, y, n, h, w, c_in, c_out)
+    if c_out % 64 == 0:
+        lp.lp_conv3x3_bf16(lp.LP_CONV_INPUT_GRAD, dyd, Wd, dx, n, h, w, c_in, c_out)
+    lp.lp_conv3x3_bf16(lp.LP_CONV_FILTER_GRAD, xd, dyd, dW, n, h, w, c_in, c_out)
+    torch.cuda.synchronize()
+    got = dict(y=y.float().cpu().numpy().transpose(0, 3, 1, 2), dW=dW.cpu().numpy().transpose(0, 3, 1, 2))
+    ref = dict(y=y_ref, dW=dW_ref)
+    if c_out % 64 == 0:
+        got["dx"], ref["dx"] = dx.float().cpu().numpy().transpose(0, 3, 1, 2), dx_ref
+    for name in got:
+        err = np.abs(got[name].astype(np.float64) - ref[name]).max() / np.abs(ref[name]).max()
+        tol = 1e-2 if name != "dW" else 1e-4     # bf16 outputs carry one rounding (2^-9); the fp32 output does not
+        assert err < tol, (name, err)
+
+
+def test_implicit_convolution_rejects_what_it_cannot_tile():
+    t = torch.zeros(1 << 16, dtype=torch.bfloat16, device="cuda")
+    for form, args in [(lp.LP_CONV_FORWARD, (2, 12, 12, 64, 64)),       # width does not divide 64
+                       (lp.LP_CONV_FORWARD, (2, 16, 16, 32, 64)),       # shifted operand's channels not a multiple of 64
+                       (lp.LP_CONV_FORWARD, (3, 12, 16, 64, 64)),       # h*w = 192 neither divides nor is divided by 128
+                       (lp.LP_CONV_INPUT_GRAD, (2, 16, 16, 60, 64))]:   # filter columns not 16-byte aligned per tap
+        with pytest.raises(lp.LpError) as e:
+            lp.lp_conv3x3_bf16(form, t, t, t, *args)
+        assert lp.LP_ERR[e.value.code] == "UNSUPPORTED"

@@ -104,6 +104,16 @@ def test_resnet_bf16_small(backend):
     check(cfg, gemm_backend=backend, v_tol=0.3)
 
 
+@pytest.mark.parametrize("size,schedule", [(16, "sync"), (8, "pipelined")])
+def test_resnet_bf16_implicit_convolutions(size, schedule):
+    """Channel counts that are multiples of 64 on 16x16, 8x8 and 4x4 images: the 3x3 stride-1 convolutions run
+    as implicit GEMMs (forward, input gradient, weight gradient; boxes inside one image, of whole images, and
+    across several images), next to the stride-2 and 1x1 convolutions in their explicit form."""
+    cfg = lp_synth.config("c4", batch=32, height=size, width=size, stem_channels=64,
+                          stage_channels=[64, 128], blocks_per_stage=2, classes=10, schedule=schedule)
+    check(cfg, v_tol=0.3)
+
+
 def test_sync_and_pipelined_agree_on_step0():
     cfg = lp_synth.config("c1")
     x, y = lp_synth.minibatch(cfg, 0)
