@@ -50,6 +50,27 @@ def describe(cfg):
     return d
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ and scaled to the launches of a full step.  A figure is only
+# valid for the kernel source it was captured on: it is dropped when that file has changed since.
+TRAFFIC = {
+    "c5": dict(bytes_per_launch=None, kernel_file="paper_2012_03837_b200/csrc/gemm_tc.cu", kernel_sha256=""),
+}
+
+
+def measured_traffic(workload):
+    rec = TRAFFIC.get(workload)
+    if not rec or rec["bytes_per_launch"] is None:
+        return None
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, rec["kernel_file"]), "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return rec["bytes_per_launch"] if sha == rec["kernel_sha256"] else None
+
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -327,7 +348,7 @@ def run_ours(args, cfg):
             achieved = gflop / (gms * 1e-3) / 1e12
             roof = dict(bound="tensor", kernel="gemm_tc_kernel (grouped tcgen05 bf16 GEMM)", achieved=achieved,
                         peak=pk["tensor_sustained"], unit="TFLOP/s", frac=achieved / pk["tensor_sustained"],
-                        peak_source=pk["source"] + " sustained cuBLAS bf16", traffic=None,
+                        peak_source=pk["source"] + " sustained cuBLAS bf16", traffic=measured_traffic(cfg["name"]),
                         launches=gl, ms_per_launch=gms / gl, share_of_step=gms / ms_profiled)
         else:
             ams, aflop, al = prof["gemm_alu"]

@@ -171,8 +171,23 @@ lp_status lp_get_tensor(lp_handle h, int i, int which, void* host_dst, size_t by
 lp_status lp_set_tensor(lp_handle h, int i, int which, const void* host_src, size_t bytes,
                         void* stream);
 
-/* Forget the activations in flight between chunks; the next pipelined step refills them. */
+/* Forget the activations in flight between chunks; the next pipelined step starts the ramp-up again. */
 lp_status lp_reset_pipeline(lp_handle h);
+
+/*
+ * lp_set_ramp: how the pipelined schedule starts after lp_create or lp_reset_pipeline (Sec. 6 speaks only
+ * of "an initial ramp-up phase"; both readings are offered).
+ *   LP_RAMP_PRIME (default): the first pipelined step fills every boundary buffer by a forward pass of its
+ *     own minibatch; every chunk then trains in every step, and that first step equals a synchronous step.
+ *   LP_RAMP_IDLE: nothing is filled.  In the s-th pipelined step after the reset (s = 0, 1, ...) only chunks
+ *     0..s train: chunk k waits until an activation produced from real data reaches it, as a pipeline of K
+ *     processors would.  An idle chunk's parameters, optimizer state and step count do not change, and its
+ *     entry of out_losses is NaN.  (Idle chunks still execute, on stale buffer contents; the cost of a step
+ *     is the same.)
+ * Allowed only while no pipeline is in flight.  Errors: INVALID_ARG, STATE.
+ */
+enum { LP_RAMP_PRIME = 0, LP_RAMP_IDLE = 1 };
+lp_status lp_set_ramp(lp_handle h, int ramp);
 
 /* Read the device status word (synchronises `stream`): LP_OK, or LABEL_RANGE / NONFINITE /
  * TIMEOUT if any kernel since the last poll flagged it.  The word is cleared. */

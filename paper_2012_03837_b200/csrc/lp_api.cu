@@ -1,5 +1,7 @@
 // C ABI of the local update step (include/lp.h): argument checks, handle life cycle, step
 // drivers, parameter access, checkpointing.  No exception leaves this file.
+#include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <stdexcept>
 
@@ -125,23 +127,75 @@ lp_status copy_inputs(Handle& h, const void* x, const void* y, cudaMemcpyKind ki
   return check_cuda(&h, "input copy");
 }
 
+// Arena segments for the optimizer's per-chunk mode: one per tensor, in arena order; a tensor's
+// alignment padding belongs to it (its gradient there is zero).
+void build_segments(Handle& h) {
+  std::vector<const TensorRec*> order;
+  for (auto& t : h.tensors) order.push_back(&t);
+  std::sort(order.begin(), order.end(), [](const TensorRec* a, const TensorRec* b) { return a->off < b->off; });
+  std::vector<long long> ends;
+  std::vector<int> chunks;
+  for (size_t i = 0; i < order.size(); ++i) {
+    ends.push_back(i + 1 < order.size() ? (long long)order[i + 1]->off : h.n_total);
+    chunks.push_back(order[i]->chunk);
+  }
+  h.d_seg_end = h.upload(ends);
+  h.d_seg_chunk = h.upload(chunks);
+  h.n_seg = (int)ends.size();
+  h.d_chunk_tab = (float4*)h.dalloc(sizeof(float4) * h.K);
+  h.updates.assign(h.K, 0);
+}
+
+// Which chunks take part in this step (Sec. 6: with the idle ramp-up, chunk k waits until the k-th
+// pipelined step after a reset has brought it an activation), and the per-chunk optimizer table when
+// the chunks' step counts differ.  Returns true if some chunk idles.
+bool prepare_chunks(Handle& h, int schedule, cudaStream_t s, std::vector<char>& active) {
+  const int K = h.K;
+  active.assign(K, 1);
+  bool any_idle = false, differ = false;
+  if (schedule == LP_PIPELINED && h.ramp == LP_RAMP_IDLE)
+    for (int k = 0; k < K; ++k)
+      if (k > h.pipe_steps) { active[k] = 0; any_idle = true; }
+  for (int k = 1; k < K; ++k) differ |= h.updates[k] != h.updates[0];
+  h.per_chunk_counts = any_idle || differ;
+  if (h.per_chunk_counts) {
+    std::vector<float4> tab(K);
+    for (int k = 0; k < K; ++k) {
+      const double t = (double)(h.updates[k] + 1);
+      tab[k] = make_float4(active[k] ? 1.f : 0.f, (float)(1.0 - pow((double)h.opt.beta1, t)),
+                           (float)(1.0 - pow((double)h.opt.beta2, t)), 0.f);
+    }
+    // pageable source: the runtime stages it before the call returns, so the vector may go out of scope
+    cudaMemcpyAsync(h.d_chunk_tab, tab.data(), sizeof(float4) * K, cudaMemcpyHostToDevice, s);
+  }
+  return any_idle;
+}
+
 lp_status run_step(Handle& h, int schedule, cudaStream_t s) {
   RunCtx ctx{s, nullptr, h.profiling ? &h.prof : nullptr};
   int launches = 0;
+  std::vector<char> active;
+  const bool any_idle = prepare_chunks(h, schedule, s, active);
   if (schedule == LP_SYNC) {
     if (h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
     h.sync_plan.run(ctx);
     launches = h.sync_plan.launches;
   } else {
-    if (!h.primed) {
+    if (!h.primed && h.ramp == LP_RAMP_PRIME) {
       h.prime_plan[h.parity].run(ctx);
       launches += h.prime_plan[h.parity].launches;
-      h.primed = true;
     }
+    h.primed = true;
+    // Idle chunks run through the plan as well, on whatever their boundary buffer holds (finite values:
+    // zeros after lp_create); the optimizer leaves their parameters alone, their losses read NaN, and
+    // what they publish is overwritten before an active chunk reads it.
     h.pipe_plan[h.parity].run(ctx);
     launches += h.pipe_plan[h.parity].launches;
+    if (any_idle) { launch_mask_losses(h.d_losses, h.d_chunk_tab, h.K, s); launches += 1; }
     h.parity ^= 1;
+    h.pipe_steps += 1;
   }
+  for (int k = 0; k < h.K; ++k) h.updates[k] += active[k] ? 1 : 0;
   h.step_count += 1;
   h.last_launches = launches;
   return check_cuda(&h, "lp_step launch");
@@ -198,6 +252,7 @@ lp_status lp_create(const lp_model_spec* model, int K, const lp_head_spec* head,
         build_resnet(h);
         break;
     }
+    build_segments(h);
     cudaDeviceSynchronize();
     lp_status st = check_cuda(nullptr, "lp_create");
     if (st != LP_OK) { lp_destroy(hh); return st; }
@@ -315,6 +370,16 @@ lp_status lp_reset_pipeline(lp_handle hh) {
   if (!hh) return LP_ERR_INVALID_ARG;
   hh->h.primed = false;
   hh->h.parity = 0;
+  hh->h.pipe_steps = 0;
+  return LP_OK;
+}
+
+lp_status lp_set_ramp(lp_handle hh, int ramp) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (ramp != LP_RAMP_PRIME && ramp != LP_RAMP_IDLE) return fail(&h, LP_ERR_INVALID_ARG, "bad ramp mode");
+  if (h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before changing the ramp-up");
+  h.ramp = ramp;
   return LP_OK;
 }
 
@@ -334,15 +399,18 @@ lp_status lp_status_poll(lp_handle hh, void* stream) {
   return LP_OK;
 }
 
-// Checkpoint layout: header {magic, n_total, K, step_count, parity, primed}, master, m1, [m2],
-// then for each half and chunk: boundary activation, labels.
-struct StateHeader { uint64_t magic; int64_t n_total; int64_t K; int64_t step_count; int64_t parity; int64_t primed; };
-static const uint64_t kMagic = 0x4c50535441544531ull;
+// Checkpoint layout: header {magic, n_total, K, step_count, parity, primed, ramp, pipe_steps}, the K per-chunk
+// update counts, master, m1, [m2], then for each half and chunk: boundary activation, labels.
+struct StateHeader {
+  uint64_t magic; int64_t n_total; int64_t K; int64_t step_count; int64_t parity; int64_t primed;
+  int64_t ramp; int64_t pipe_steps;
+};
+static const uint64_t kMagic = 0x4c50535441544532ull;
 
 size_t lp_state_size(lp_handle hh) {
   if (!hh) return 0;
   Handle& h = hh->h;
-  size_t n = sizeof(StateHeader) + (size_t)h.n_total * 4 * (h.m2 ? 3 : 2);
+  size_t n = sizeof(StateHeader) + sizeof(int64_t) * h.K + (size_t)h.n_total * 4 * (h.m2 ? 3 : 2);
   for (int s = 0; s < 2; ++s)
     for (int k = 0; k < h.K; ++k) n += h.bnd_bytes[k] + h.y_bytes;
   return n;
@@ -355,14 +423,21 @@ static lp_status state_io(lp_handle hh, void* host, size_t bytes, bool save) {
   if (bytes != lp_state_size(hh)) return fail(&h, LP_ERR_SHAPE, "state size mismatch");
   cudaDeviceSynchronize();
   char* p = (char*)host;
-  StateHeader hd{kMagic, h.n_total, h.K, h.step_count, h.parity, h.primed ? 1 : 0};
+  StateHeader hd{kMagic, h.n_total, h.K, h.step_count, h.parity, h.primed ? 1 : 0, h.ramp, h.pipe_steps};
   if (save) memcpy(p, &hd, sizeof(hd));
   else {
     memcpy(&hd, p, sizeof(hd));
     if (hd.magic != kMagic || hd.n_total != h.n_total || hd.K != h.K) return fail(&h, LP_ERR_STATE, "state blob does not match this handle");
     h.step_count = hd.step_count; h.parity = (int)hd.parity; h.primed = hd.primed != 0;
+    h.ramp = (int)hd.ramp; h.pipe_steps = hd.pipe_steps;
   }
   p += sizeof(hd);
+  for (int k = 0; k < h.K; ++k) {
+    int64_t u = h.updates[k];
+    if (save) memcpy(p, &u, sizeof(u));
+    else { memcpy(&u, p, sizeof(u)); h.updates[k] = u; }
+    p += sizeof(u);
+  }
   auto io = [&](void* dev, size_t n) {
     if (save) cudaMemcpy(p, dev, n, cudaMemcpyDeviceToHost);
     else cudaMemcpy(dev, p, n, cudaMemcpyHostToDevice);

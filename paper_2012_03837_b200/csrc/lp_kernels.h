@@ -196,7 +196,15 @@ struct OptimArgs {
   int kind; float lr, momentum, weight_decay, beta1, beta2, eps;
   float omb1, omb2;     // 1 - beta, rounded from double
   float bc1, bc2;       // 1 - beta^t, rounded from double
+  // Per-chunk mode (idle ramp-up of the pipelined schedule, Sec. 6: a chunk that no minibatch has reached
+  // yet makes no update, so the chunks' step counts differ).  seg_end[i] = one past the last arena element
+  // of segment i (segments in arena order), seg_chunk[i] = its chunk, chunk_tab[k] = (active ? 1 : 0,
+  // 1 - beta1^t_k, 1 - beta2^t_k, unused).  Null seg_end: all chunks share bc1 / bc2 and are updated.
+  const long long* seg_end; const int* seg_chunk; int n_seg;
+  const float4* chunk_tab;
 };
 void launch_optim(const OptimArgs& a, cudaStream_t s);
+// losses[k] = NaN for the chunks whose chunk_tab entry is inactive
+void launch_mask_losses(float* losses, const float4* chunk_tab, int K, cudaStream_t s);
 
 }  // namespace lp

@@ -10,9 +10,21 @@ namespace {
 
 // 4 elements per thread, 128-bit accesses.  Reads master, moments, gradient; writes master,
 // moments and (for the leading n_matrix elements) the bf16 working copy re-rounded from master.
+template <bool PER_CHUNK>
 __global__ void __launch_bounds__(256) optim_kernel(OptimArgs a) {
   long long i4 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i4 >= a.n_total) return;   // the arena length is a multiple of 4
+  if (PER_CHUNK) {
+    // segment holding element i4 (segments start on multiples of 4, so the four elements share it)
+    int lo = 0, hi = a.n_seg - 1;
+    while (lo < hi) {
+      int mid = (lo + hi) >> 1;
+      if (i4 < a.seg_end[mid]) hi = mid; else lo = mid + 1;
+    }
+    const float4 tab = a.chunk_tab[a.seg_chunk[lo]];
+    if (tab.x == 0.f) return;    // idle chunk: parameters, moments and working copy stay as they are
+    a.bc1 = tab.y; a.bc2 = tab.z;
+  }
   float4 w = *(const float4*)(a.master + i4);
   float4 g = *(const float4*)(a.grad + i4);
   float4 m1 = *(const float4*)(a.m1 + i4);
@@ -48,6 +60,11 @@ __global__ void __launch_bounds__(256) optim_kernel(OptimArgs a) {
     pk.y = *(uint32_t*)&hi;
     *(uint2*)(a.working + i4) = pk;
   }
+}
+
+__global__ void __launch_bounds__(256) mask_losses_kernel(float* losses, const float4* chunk_tab, int K) {
+  int k = blockIdx.x * blockDim.x + threadIdx.x;
+  if (k < K && chunk_tab[k].x == 0.f) losses[k] = __int_as_float(0x7fc00000);
 }
 
 // h[r, :] = tok[ids[r], :] + pos[r % T, :]; ids outside [0, vocab) are flagged and clamped.
@@ -123,7 +140,12 @@ __global__ void __launch_bounds__(256) embed_bwd_pos_kernel(EmbedBwdProb p) {
 void launch_optim(const OptimArgs& a, cudaStream_t s) {
   long long threads = (a.n_total + 3) / 4;
   if (threads == 0) return;
-  optim_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, s>>>(a);
+  if (a.seg_end) optim_kernel<true><<<(unsigned)((threads + 255) / 256), 256, 0, s>>>(a);
+  else optim_kernel<false><<<(unsigned)((threads + 255) / 256), 256, 0, s>>>(a);
+}
+
+void launch_mask_losses(float* losses, const float4* chunk_tab, int K, cudaStream_t s) {
+  mask_losses_kernel<<<(K + 255) / 256, 256, 0, s>>>(losses, chunk_tab, K);
 }
 
 void launch_embed_fwd(const EmbedProb& p, int* d_status, bool is_bf16, cudaStream_t s) {

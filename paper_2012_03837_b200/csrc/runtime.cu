@@ -346,11 +346,15 @@ void emit_optimizer(Handle& h, Plan& p) {
     a.n_total = hp->n_total; a.n_matrix = hp->n_matrix;
     a.kind = hp->opt.kind; a.lr = hp->opt.lr; a.momentum = hp->opt.momentum; a.weight_decay = hp->opt.weight_decay;
     a.beta1 = hp->opt.beta1; a.beta2 = hp->opt.beta2; a.eps = hp->opt.eps;
-    double t = (double)(hp->step_count + 1);
+    // all chunks share one step count here (otherwise the per-chunk table below carries theirs)
+    double t = (double)((hp->updates.empty() ? hp->step_count : hp->updates[0]) + 1);
     a.omb1 = (float)(1.0 - (double)hp->opt.beta1);
     a.omb2 = (float)(1.0 - (double)hp->opt.beta2);
     a.bc1 = (float)(1.0 - pow((double)hp->opt.beta1, t));
     a.bc2 = (float)(1.0 - pow((double)hp->opt.beta2, t));
+    if (hp->per_chunk_counts) {   // the step driver has filled d_chunk_tab for this step
+      a.seg_end = hp->d_seg_end; a.seg_chunk = hp->d_seg_chunk; a.n_seg = hp->n_seg; a.chunk_tab = hp->d_chunk_tab;
+    }
     launch_optim(a, c.stream);
   }, KIND_OPTIM, (double)h.n_total * (h.opt.kind == LP_OPT_ADAM ? 28.0 : 20.0) + (h.bf16_mode ? 2.0 * h.n_matrix : 0.0));
 }

@@ -100,6 +100,16 @@ struct Handle {
   int parity = 0;
   bool primed = false;
   long long step_count = 0;
+  // ---- ramp-up of the pipelined schedule (Sec. 6): LP_RAMP_PRIME fills the boundary buffers by a forward
+  // pass; LP_RAMP_IDLE lets chunk k idle until the k-th pipelined step after a reset
+  int ramp = 0;
+  long long pipe_steps = 0;                    // pipelined steps since create / reset
+  std::vector<long long> updates;              // per chunk: optimizer updates made so far
+  bool per_chunk_counts = false;               // some chunk has idled: the chunks' step counts differ
+  const long long* d_seg_end = nullptr;        // arena segments (see OptimArgs), built on first use
+  const int* d_seg_chunk = nullptr;
+  int n_seg = 0;
+  float4* d_chunk_tab = nullptr;
   int last_launches = 0;
   bool profiling = false;
   std::vector<ProfRecord> prof;

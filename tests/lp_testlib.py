@@ -18,7 +18,7 @@ def to_abi_layout(name: str, a: np.ndarray) -> np.ndarray:
 
 
 class GpuModel:
-    def __init__(self, cfg: dict, params: dict | None = None, gemm_backend: int = 0):
+    def __init__(self, cfg: dict, params: dict | None = None, gemm_backend: int = 0, ramp: str = "prime"):
         self.cfg = cfg
         m, K, hd, op = lp.specs_from_config(cfg, gemm_backend)
         self._specs = (m, hd, op)
@@ -32,6 +32,8 @@ class GpuModel:
         self.losses = torch.zeros(K, dtype=torch.float32, device=self.dev)
         self.stream = torch.cuda.current_stream().cuda_stream
         self.set_params(params if params is not None else lp_synth.init_params(cfg))
+        if ramp == "idle":
+            lp.lp_set_ramp(self.h, lp.LP_RAMP_IDLE)
 
     def close(self):
         if self.h:
@@ -95,11 +97,11 @@ def tensor_rel_err(a: np.ndarray, b: np.ndarray) -> float:
     return float(np.abs(a.astype(np.float64) - b.astype(np.float64)).max() / max(np.abs(b).max(), 1e-30))
 
 
-def run_both(cfg: dict, steps: int, gemm_backend: int = 0, params: dict | None = None):
+def run_both(cfg: dict, steps: int, gemm_backend: int = 0, params: dict | None = None, ramp: str = "prime"):
     """Run `steps` steps on both sides.  Returns (gpu_losses [steps,K], oracle_losses, gpu model, oracle)."""
     params = params if params is not None else lp_synth.init_params(cfg)
-    gm = GpuModel(cfg, params, gemm_backend)
-    orc = LocalUpdateOracle(cfg, params, dtype=np.float32)
+    gm = GpuModel(cfg, params, gemm_backend, ramp)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float32, ramp=ramp)
     gl, ol = [], []
     for t in range(steps):
         x, y = lp_synth.minibatch(cfg, t)

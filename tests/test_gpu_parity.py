@@ -140,3 +140,77 @@ def test_run_to_run_bit_reproducible():
     assert np.array_equal(outs[0][0], outs[1][0])
     for n in outs[0][1]:
         assert np.array_equal(outs[0][1][n], outs[1][1][n]), n
+
+
+# ------------------------------------------------------------------ idle ramp-up of the pipelined schedule
+
+def check_idle(cfg, steps=10):
+    """Pipelined steps with the idle ramp-up (chunk k waits until the k-th step brings it real data) against the
+    oracle run with ramp="idle": the same chunks idle (NaN loss, bit-exact pattern), the others agree."""
+    dt = cfg["dtype"]
+    gl, ol, gm, orc = T.run_both(cfg, steps, ramp="idle")
+    K = gl.shape[1]
+    assert np.array_equal(np.isnan(gl), np.isnan(ol)), (gl, ol)
+    for t in range(steps):
+        assert np.array_equal(np.isnan(gl[t]), np.arange(K) > t), gl[t]
+    fin = ~np.isnan(ol)
+    lerr = np.abs(gl[fin] - ol[fin]) / np.abs(ol[fin])
+    werr = T.compare_weights(gm, orc, lp_synth.init_params(cfg))
+    gm.close()
+    worst = {kind: max((e, n) for n, (kd, e) in werr.items() if kd == kind) for kind in ("matrix", "vector", "chunk")}
+    print("idle ramp-up: loss rel err max", f"{lerr.max():.2e}", "weights worst", {k: (f"{e:.2e}", n) for k, (e, n) in worst.items()})
+    assert lerr.max() <= LOSS_TOL[dt]
+    assert worst["matrix"][0] <= W_TOL[dt] and worst["chunk"][0] <= W_TOL[dt], worst
+    assert worst["vector"][0] <= V_TOL[dt], worst
+
+
+def test_idle_ramp_up_mlp_fp32():
+    check_idle(lp_synth.config("c1", schedule="pipelined"))
+
+
+def test_idle_ramp_up_mlp_fp32_adam():
+    """Adam's bias correction follows each chunk's own step count (chunk k has made k fewer updates)."""
+    cfg = lp_synth.config("c1", schedule="pipelined", batch=48, d_in=40, chunks=[[64], [48, 56], [32], [72]], classes=6)
+    cfg["optim"] = dict(kind="adam", lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+    check_idle(cfg)
+
+
+def test_idle_ramp_up_lm_bf16():
+    cfg = lp_synth.config("c3", batch=3, seq_len=136, vocab=1000, d_model=128, n_heads=2, d_ffn=320,
+                          blocks_per_chunk=[1, 1, 1, 1], schedule="pipelined")
+    check_idle(cfg, steps=8)
+
+
+def test_idle_ramp_up_reset_and_checkpoint():
+    """A reset sends the later chunks back to idling while their step counts stay behind; a checkpoint taken in
+    the middle of a ramp-up continues bit for bit in a fresh handle."""
+    from paper_2012_03837_b200 import binding as lp
+    cfg = lp_synth.config("c1", schedule="pipelined")
+    cfg["optim"] = dict(kind="adam", lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+    params = lp_synth.init_params(cfg)
+    from oracle.local_step import LocalUpdateOracle
+    gm = T.GpuModel(cfg, params, ramp="idle")
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float32, ramp="idle")
+    for t in range(3):
+        gl, ol = gm.step(*lp_synth.minibatch(cfg, t)), orc.step(*lp_synth.minibatch(cfg, t))
+    lp.lp_reset_pipeline(gm.h)
+    orc.reset_pipeline()
+    for t in range(3, 5):
+        gl, ol = gm.step(*lp_synth.minibatch(cfg, t)), orc.step(*lp_synth.minibatch(cfg, t))
+        assert np.array_equal(np.isnan(gl), np.isnan(ol)) and np.array_equal(np.isnan(gl), np.arange(4) > t - 3)
+        assert np.nanmax(np.abs(gl - ol) / np.abs(ol)) <= 1e-4
+    blob = np.empty(lp.lp_state_size(gm.h), dtype=np.uint8)
+    lp.lp_save_state(gm.h, blob)
+    gm2 = T.GpuModel(cfg, params, ramp="idle")
+    lp.lp_load_state(gm2.h, blob)
+    for t in range(5, 8):
+        a, b = gm.step(*lp_synth.minibatch(cfg, t)), gm2.step(*lp_synth.minibatch(cfg, t))
+        assert np.array_equal(a, b, equal_nan=True)
+        o = orc.step(*lp_synth.minibatch(cfg, t))
+        assert np.nanmax(np.abs(a - o) / np.abs(o)) <= 1e-4
+    wa, wb = gm.get(), gm2.get()
+    for n in wa:
+        assert np.array_equal(wa[n], wb[n]), n
+    werr = T.compare_weights(gm, orc, params)
+    assert max(e for _, e in werr.values()) <= 1e-3, werr
+    gm.close(); gm2.close()
