@@ -524,7 +524,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       TileWalk walk;
       bool a_mn = false, b_mn = false;
       int kb_n = 0;
-      int conv = 0, cv_c = 64, cv_w = 1, cv_hw = 1, cv_n = 0, cv_k0 = 0, p_n = 0;
+      int conv = 0;
       for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
         if (cur.seek(tile)) {                        // problem changed: re-read its fields (once per problem, not per tile)
           const GemmProb& p = probs[cur.pi];
@@ -532,22 +532,66 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
           a_mn = p.a_ms == 1; b_mn = p.b_ns == 1;
           kb_n = (p.K + BK - 1) / BK;
           conv = p.conv;
-          if (conv) { cv_c = p.conv_c; cv_w = p.conv_w; cv_hw = p.conv_h * p.conv_w; cv_n = p.conv_n; cv_k0 = p.conv_k0; p_n = p.N; }
         }
         const CUtensorMap* mapA = maps + 4 * cur.pi;
         const CUtensorMap* mapB = mapA + 1;
         int mt, nt;
         walk.coords(tile, mt, nt);
         int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN + (int)rank * BNL;
-        // implicit convolution: this CTA's 128 output pixels start at row a_h0 of image a_img (whole rows)
+        if (conv == CONV_NONE) {
+          // ---- ordinary operands: 2-D boxes of the A and B matrices
+          for (int kb = 0; kb < kb_n; ++kb) {
+            if (!(ok = mbar_wait(&sh->empty[stage], phase ^ 1, sh, status))) break;
+            uint8_t* a_dst = tiles + stage * STAGE_BYTES;
+            uint8_t* b_dst = a_dst + A_BYTES;
+            int k0 = kb * BK;
+            if (CG == 1) {
+              uint64_t* bar = &sh->full[stage];
+              mbar_expect_tx(bar, STAGE_BYTES);
+              if (a_mn) {
+#pragma unroll
+                for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, bar);
+              } else {
+                tma_load_2d(a_dst, mapA, k0, m0, bar);
+              }
+              if (b_mn) {
+#pragma unroll
+                for (int i = 0; i < BNL / 64; ++i) tma_load_2d(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, bar);
+              } else {
+                tma_load_2d(b_dst, mapB, k0, n0, bar);
+              }
+            } else {
+              // both CTAs' bytes are counted on the leader's barrier
+              uint32_t bar = map_to_rank(smem_u32(&sh->full[stage]), 0);
+              mbar_expect_tx_cluster(bar, STAGE_BYTES);
+              if (a_mn) {
+#pragma unroll
+                for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, bar);
+              } else {
+                tma_load_2d_pair(a_dst, mapA, k0, m0, bar);
+              }
+              if (b_mn) {
+#pragma unroll
+                for (int i = 0; i < BNL / 64; ++i) tma_load_2d_pair(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, bar);
+              } else {
+                tma_load_2d_pair(b_dst, mapB, k0, n0, bar);
+              }
+            }
+            if (++stage == STAGES) { stage = 0; phase ^= 1; }
+          }
+          continue;
+        }
+        // ---- implicit convolution: one operand is fetched as shifted boxes of the activation tensor
+        const GemmProb& p = probs[cur.pi];
+        const int cv_c = p.conv_c, cv_w = p.conv_w, cv_hw = p.conv_h * p.conv_w, cv_n = p.conv_n, cv_k0 = p.conv_k0, p_n = p.N;
+        // this CTA's 128 output pixels start at row a_h0 of image a_img (whole rows)
         int a_img = 0, a_h0 = 0;
-        if (conv == CONV_FWD || conv == CONV_DGRAD) { a_img = m0 / cv_hw; a_h0 = (m0 - a_img * cv_hw) / cv_w; }
+        if (conv != CONV_WGRAD) { a_img = m0 / cv_hw; a_h0 = (m0 - a_img * cv_hw) / cv_w; }
         for (int kb = 0; kb < kb_n; ++kb) {
           if (!(ok = mbar_wait(&sh->empty[stage], phase ^ 1, sh, status))) break;
           uint8_t* a_dst = tiles + stage * STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_BYTES;
           int k0 = kb * BK;
-          // both CTAs' bytes of a pair are counted on the leader's barrier
           uint64_t* bar1 = &sh->full[stage];
           uint32_t bar2 = 0;
           if (CG == 1) mbar_expect_tx(bar1, STAGE_BYTES);
@@ -558,40 +602,33 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
           auto ld4 = [&](void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3) {
             if (CG == 1) tma_load_4d(dst, map, c0, c1, c2, c3, bar1); else tma_load_4d_pair(dst, map, c0, c1, c2, c3, bar2);
           };
-          // filter tap and channel block of this k-slice (CONV_FWD / CONV_DGRAD: k = tap * conv_c + channel)
-          int tap = 0, ch0 = 0;
-          if (conv == CONV_FWD || conv == CONV_DGRAD) { const int cb = cv_c >> 6; tap = kb / cb; ch0 = (kb - tap * cb) << 6; }
-          // ---- A
-          if (conv == CONV_FWD || conv == CONV_DGRAD) {
-            int di = tap / 3 - 1, dj = tap - (tap / 3) * 3 - 1;
-            if (conv == CONV_DGRAD) { di = -di; dj = -dj; }
-            ld4(a_dst, mapA, ch0, dj, a_h0 + di, a_img);
-          } else if (a_mn) {
+          if (conv == CONV_WGRAD) {
+            // A: dy as an ordinary MN-major operand; B: 64 pixels (whole rows) of x per 64-column block, each
+            // column block with the shift of its own filter tap
 #pragma unroll
             for (int i = 0; i < BM / 64; ++i) ld2(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0);
-          } else {
-            ld2(a_dst, mapA, k0, m0);
-          }
-          // ---- B
-          if (conv == CONV_WGRAD) {
-            const int kp = cv_k0 + k0;               // first pixel of this k-slice (whole rows, 64 pixels)
+            const int kp = cv_k0 + k0;
             const int img = kp / cv_hw, h0 = (kp - img * cv_hw) / cv_w;
 #pragma unroll
             for (int i = 0; i < BNL / 64; ++i) {
-              const int col = n0 + i * 64;           // column block -> (tap, channel block)
+              const int col = n0 + i * 64;
               const int t = col / cv_c, c0 = col - t * cv_c;
               if (t < 9) ld4(b_dst + i * (BK * 128), mapB, c0, t - (t / 3) * 3 - 1, h0 + t / 3 - 1, img);
               else ld4(b_dst + i * (BK * 128), mapB, 0, 0, 0, cv_n);        // beyond the last tap: an all-zero box
             }
-          } else if (conv == CONV_DGRAD) {
-            // filters [conv_c, 3, 3, N] read in place: rows = output channel (the reduction), columns (tap, n)
-#pragma unroll
-            for (int i = 0; i < BNL / 64; ++i) ld2(b_dst + i * (BK * 128), mapB, tap * p_n + n0 + i * 64, ch0);
-          } else if (b_mn) {
-#pragma unroll
-            for (int i = 0; i < BNL / 64; ++i) ld2(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0);
           } else {
-            ld2(b_dst, mapB, k0, n0);
+            // k-slice -> (filter tap, channel block); A: 128 pixels shifted by the tap (mirrored for the input gradient)
+            const int cb = cv_c >> 6, tap = kb / cb, ch0 = (kb - tap * cb) << 6;
+            int di = tap / 3 - 1, dj = tap - (tap / 3) * 3 - 1;
+            if (conv == CONV_DGRAD) { di = -di; dj = -dj; }
+            ld4(a_dst, mapA, ch0, dj, a_h0 + di, a_img);
+            if (conv == CONV_FWD) {
+              ld2(b_dst, mapB, k0, n0);                  // filters [N, 9 conv_c], reduction index contiguous
+            } else {
+              // filters [conv_c, 3, 3, N] read in place: rows = output channel (the reduction), columns (tap, n)
+#pragma unroll
+              for (int i = 0; i < BNL / 64; ++i) ld2(b_dst + i * (BK * 128), mapB, tap * p_n + n0 + i * 64, ch0);
+            }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }

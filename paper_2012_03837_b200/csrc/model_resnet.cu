@@ -50,6 +50,21 @@ struct Chunk {
   void* dcols;
 };
 
+// Backward passes of the chunks are independent of one another (Sec. 3): each chunk records its backward
+// as a list of ops, and the lists are emitted in lockstep, ops of the same kind at the same position
+// sharing one grouped launch.
+enum OpKind { OP_NOP = 0, OP_GEMM, OP_COLSUM, OP_GAP_BWD, OP_BN_BWD, OP_ADD, OP_RAW };
+struct Op {
+  OpKind kind = OP_NOP;
+  std::vector<GemmProb> gemms;                       // OP_GEMM
+  ColSumProb colsum{}; float* colsum_out = nullptr;  // OP_COLSUM
+  GapProb gap{}; long long elems = 0;                // OP_GAP_BWD (elems also: OP_BN_BWD, OP_ADD)
+  BnStatProb bn_stat{}; BnFinalProb bn_final{}; BnApplyProb bn_apply{}; bool v8 = false; double work = 0;  // OP_BN_BWD
+  AddProb add{};                                     // OP_ADD
+  std::function<void(Plan&)> raw;                    // OP_RAW: emitted on its own
+};
+typedef std::vector<Op> OpList;
+
 Conv make_conv(const std::string& w, int N, int H, int W, int Cin, int Cout, int k, int stride) {
   Conv c;
   c.w = w; c.N = N; c.H = H; c.W = W; c.Cin = Cin; c.Cout = Cout; c.k = k; c.stride = stride; c.pad = k / 2;
@@ -192,39 +207,6 @@ void build_resnet(Handle& h) {
     g.a_ms = c.ldk;
     emit_gemm(h, p, {g});
   };
-  // x: the convolution's input in this plan (the operand of the implicit form; the explicit form reads c.cols)
-  auto conv_wgrad = [&](Plan& p, const Conv& c, const void* dy, const void* x) {
-    if (c.imp_fwd) {
-      GemmProb g = gemm_wgrad(dy, x, h.G(c.w), (int)c.M, c.Cout, c.K);
-      g.b_ks = c.Cin;
-      conv_fields(g, c, CONV_WGRAD, c.Cin);
-      emit_gemm(h, p, {g});
-      return;
-    }
-    GemmProb g = gemm_wgrad(dy, c.cols, h.G(c.w), (int)c.M, c.Cout, c.K);
-    g.b_ks = c.ldk;
-    emit_gemm(h, p, {g});
-  };
-  auto conv_dgrad = [&](Plan& p, const Conv& c, const void* dy, void* dx, void* dcols) {
-    if (c.imp_dgrad) {
-      // dx[pixel, ci] = sum over taps and output channels of dy[pixel shifted back by the tap][co] * W[co][tap][ci]
-      GemmProb g{};
-      g.A = dy; g.B = h.W(c.w); g.C = dx;
-      g.M = (int)c.M; g.N = c.Cin; g.K = 9 * c.Cout;
-      g.a_ms = c.Cout; g.a_ks = 1; g.b_ns = 1; g.b_ks = 9LL * c.Cin; g.ldc = c.Cin;
-      conv_fields(g, c, CONV_DGRAD, c.Cout);
-      emit_gemm(h, p, {g});
-      return;
-    }
-    GemmProb g = gemm_dgrad(dy, h.W(c.w), dcols, (int)c.M, c.Cout, c.K, EPI_NONE, nullptr);
-    g.ldc = c.ldk;
-    emit_gemm(h, p, {g});
-    Im2colProb ip{dx, dcols, c.N, c.H, c.W, c.Cin, c.k, c.k, c.stride, c.pad, c.Ho, c.Wo, c.ldk};
-    const Im2colProb* d = h.upload(std::vector<Im2colProb>{ip});
-    long long elems = (long long)c.N * c.H * c.W * c.Cin;
-    bool v8 = bf && c.Cin % 8 == 0;
-    p.add(1, [=](const RunCtx& r) { launch_col2im(d, 1, elems, bf, r.stream, v8); }, KIND_CONV_AUX, (double)(elems + c.M * c.K) * es);
-  };
   auto bn_fwd = [&](Plan& p, const Bn& b, const void* x, void* y, const void* res, bool relu) {
     int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
     float* part = fal((size_t)nblk * 2 * b.C);
@@ -243,30 +225,6 @@ void build_resnet(Handle& h) {
       launch_bn_finalize(df, 1, C, false, r.stream);
       launch_bn_apply(da, 1, elems, false, bf, r.stream, v8);
     }, KIND_NORM, (double)elems * es * (3 + (res ? 1 : 0)));
-  };
-  // dx = BN'(dy masked by relu_out > 0); dres (optional) receives the masked dy
-  auto bn_bwd = [&](Plan& p, const Bn& b, const void* x, const void* dy, const void* relu_out, void* dx, void* dres) {
-    int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
-    float* part = fal((size_t)nblk * 2 * b.C);
-    BnStatProb sp{x, dy, b.mean, b.rstd, relu_out, part, (int)b.rows, b.C};
-    BnFinalProb fp{part, nblk, (int)b.rows, b.C, nullptr, nullptr, h.G(b.g), h.G(b.b), 1e-5f};
-    BnApplyProb ap{x, nullptr, nullptr, h.P32(b.g), h.P32(b.b), b.mean, b.rstd, dy, relu_out, dx, dres, h.G(b.g), h.G(b.b),
-                   (int)b.rows, b.C, 0};
-    const BnStatProb* ds = h.upload(std::vector<BnStatProb>{sp});
-    const BnFinalProb* df = h.upload(std::vector<BnFinalProb>{fp});
-    const BnApplyProb* da = h.upload(std::vector<BnApplyProb>{ap});
-    int rows = (int)b.rows, C = b.C;
-    bool v8 = bf && C % 8 == 0 && C / 8 <= 256;
-    long long elems = b.rows * b.C;
-    p.add(3, [=](const RunCtx& r) {
-      launch_bn_stat_partial(ds, 1, rows, C, true, bf, r.stream, v8);
-      launch_bn_finalize(df, 1, C, true, r.stream);
-      launch_bn_apply(da, 1, elems, true, bf, r.stream, v8);
-    }, KIND_NORM, (double)elems * es * (5 + (relu_out ? 2 : 0) + (dres ? 1 : 0)));
-  };
-  auto add_into = [&](Plan& p, void* acc, const void* other, long long n) {
-    const AddProb* d = h.upload(std::vector<AddProb>{AddProb{acc, other, acc, n}});
-    p.add(1, [=](const RunCtx& r) { launch_add(d, 1, n, bf, r.stream); }, KIND_CONV_AUX, 3.0 * n * es);
   };
 
   auto chunk_in = [&](int k, int rd) -> const void* { return k == 0 ? ch[0].stem_out : h.bnd[rd][k - 1]; };
@@ -318,48 +276,177 @@ void build_resnet(Handle& h) {
     emit_xent_and_loss(h, p, {XentProb{c.z, labels, h.n_valid[k], c.row_loss, B, NC, NC, nullptr}}, {k});
   };
 
-  auto backward_chunk = [&](Plan& p, int k, int rd, int wr) {
+  // ---- backward, recorded per chunk and emitted in lockstep
+  auto wgrad_prob = [&](const Conv& c, const void* dy, const void* x) {
+    if (c.imp_fwd) {
+      GemmProb g = gemm_wgrad(dy, x, h.G(c.w), (int)c.M, c.Cout, c.K);
+      g.b_ks = c.Cin;
+      conv_fields(g, c, CONV_WGRAD, c.Cin);
+      return g;
+    }
+    GemmProb g = gemm_wgrad(dy, c.cols, h.G(c.w), (int)c.M, c.Cout, c.K);
+    g.b_ks = c.ldk;
+    return g;
+  };
+  // the input gradient of a convolution: its GEMM problem and, for the explicit form, the col2im gather after it
+  auto dgrad_prob = [&](const Conv& c, const void* dy, void* dx, void* dcols, Op& gather) {
+    gather = Op{};
+    if (c.imp_dgrad) {
+      GemmProb g{};
+      g.A = dy; g.B = h.W(c.w); g.C = dx;
+      g.M = (int)c.M; g.N = c.Cin; g.K = 9 * c.Cout;
+      g.a_ms = c.Cout; g.a_ks = 1; g.b_ns = 1; g.b_ks = 9LL * c.Cin; g.ldc = c.Cin;
+      conv_fields(g, c, CONV_DGRAD, c.Cout);
+      return g;
+    }
+    GemmProb g = gemm_dgrad(dy, h.W(c.w), dcols, (int)c.M, c.Cout, c.K, EPI_NONE, nullptr);
+    g.ldc = c.ldk;
+    Im2colProb ip{dx, dcols, c.N, c.H, c.W, c.Cin, c.k, c.k, c.stride, c.pad, c.Ho, c.Wo, c.ldk};
+    long long elems = (long long)c.N * c.H * c.W * c.Cin;
+    bool v8 = bf && c.Cin % 8 == 0;
+    double work = (double)(elems + c.M * c.K) * es;
+    gather.kind = OP_RAW;
+    gather.raw = [=, &h](Plan& p) {
+      const Im2colProb* d = h.upload(std::vector<Im2colProb>{ip});
+      p.add(1, [=](const RunCtx& r) { launch_col2im(d, 1, elems, bf, r.stream, v8); }, KIND_CONV_AUX, work);
+    };
+    return g;
+  };
+  auto rec_gemm = [&](OpList& L, std::vector<GemmProb> g) {
+    Op o; o.kind = OP_GEMM; o.gemms = std::move(g); L.push_back(std::move(o));
+  };
+  auto rec_nop = [&](OpList& L, int n = 1) { for (int i = 0; i < n; ++i) L.push_back(Op{}); };
+  // dx = BN'(dy masked by relu_out > 0); dres (optional) receives the masked dy
+  auto rec_bn_bwd = [&](OpList& L, const Bn& b, const void* x, const void* dy, const void* relu_out, void* dx, void* dres) {
+    int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
+    float* part = fal((size_t)nblk * 2 * b.C);
+    Op o; o.kind = OP_BN_BWD;
+    o.bn_stat = BnStatProb{x, dy, b.mean, b.rstd, relu_out, part, (int)b.rows, b.C};
+    o.bn_final = BnFinalProb{part, nblk, (int)b.rows, b.C, nullptr, nullptr, h.G(b.g), h.G(b.b), 1e-5f};
+    o.bn_apply = BnApplyProb{x, nullptr, nullptr, h.P32(b.g), h.P32(b.b), b.mean, b.rstd, dy, relu_out, dx, dres, h.G(b.g), h.G(b.b),
+                             (int)b.rows, b.C, 0};
+    o.v8 = bf && b.C % 8 == 0 && b.C / 8 <= 256;
+    o.elems = b.rows * b.C;
+    o.work = (double)o.elems * es * (5 + (relu_out ? 2 : 0) + (dres ? 1 : 0));
+    L.push_back(std::move(o));
+  };
+  auto rec_add = [&](OpList& L, void* acc, const void* other, long long n) {
+    Op o; o.kind = OP_ADD; o.add = AddProb{acc, other, acc, n}; o.elems = n; L.push_back(std::move(o));
+  };
+
+  // Every chunk's list has the same length and the same kind (or a gap) at every position.
+  auto record_backward = [&](OpList& L, int k, int rd, int wr) {
     Chunk& c = ch[k];
     const std::string ck = "c" + std::to_string(k);
     // head: dW_h, db_h, d(pool), then the pool's gradient spread over H*W -> G[0]
-    emit_gemm(h, p, {gemm_wgrad(c.z, c.pool, h.G(ck + ".head.W"), B, NC, c.C),
-                     gemm_dgrad(c.z, h.W(ck + ".head.W"), c.dpool, B, NC, c.C, EPI_NONE, nullptr)});
-    emit_colsum(h, p, {ColSumProb{c.z, nullptr, B, NC, NC}}, {h.G(ck + ".head.b")});
-    {
-      GapProb gp{nullptr, nullptr, c.dpool, c.G[0], B, c.Hout * c.Wout, c.C};
-      const GapProb* dg = h.upload(std::vector<GapProb>{gp});
-      long long elems = (long long)B * c.Hout * c.Wout * c.C;
-      p.add(1, [=](const RunCtx& r) { launch_gap_bwd(dg, 1, elems, bf, r.stream); }, KIND_CONV_AUX, (double)elems * es);
-    }
+    rec_gemm(L, {gemm_wgrad(c.z, c.pool, h.G(ck + ".head.W"), B, NC, c.C),
+                 gemm_dgrad(c.z, h.W(ck + ".head.W"), c.dpool, B, NC, c.C, EPI_NONE, nullptr)});
+    { Op o; o.kind = OP_COLSUM; o.colsum = ColSumProb{c.z, nullptr, B, NC, NC}; o.colsum_out = h.G(ck + ".head.b"); L.push_back(std::move(o)); }
+    { Op o; o.kind = OP_GAP_BWD; o.gap = GapProb{nullptr, nullptr, c.dpool, c.G[0], B, c.Hout * c.Wout, c.C};
+      o.elems = (long long)B * c.Hout * c.Wout * c.C; L.push_back(std::move(o)); }
     void *gin = c.G[0], *ga = c.G[1], *gb = c.G[2], *gc = c.G[3];
     for (int j = (int)c.blocks.size() - 1; j >= 0; --j) {
       Block& b = c.blocks[j];
       const void* x = j == 0 ? chunk_in(k, rd) : c.blocks[j - 1].out;
       const void* out = b.out ? b.out : h.bnd[wr][k];
       bool need_dx = (j > 0) || c.has_stem;
-      // out = relu(bn2(c2) + shortcut): ga <- d(c2), gb <- gradient of the shortcut branch
-      bn_bwd(p, b.b2, b.c2.y, gin, out, ga, gb);
-      conv_wgrad(p, b.c2, ga, b.a1);
-      conv_dgrad(p, b.c2, ga, gc, c.dcols);                 // gc <- d(a1)
-      bn_bwd(p, b.b1, b.c1.y, gc, b.a1, ga, nullptr);       // ga <- d(c1)
-      conv_wgrad(p, b.c1, ga, x);
       long long in_elems_blk = (long long)b.c1.N * b.c1.H * b.c1.W * b.c1.Cin;
-      if (need_dx) conv_dgrad(p, b.c1, ga, gc, c.dcols);    // gc <- d(x) through the main branch
+      Op gather;
+      // out = relu(bn2(c2) + shortcut): ga <- d(c2), gb <- gradient of the shortcut branch
+      rec_bn_bwd(L, b.b2, b.c2.y, gin, out, ga, gb);
+      {                                                     // dW(c2) and gc <- d(a1) read the same ga: one launch
+        GemmProb dg = dgrad_prob(b.c2, ga, gc, c.dcols, gather);
+        rec_gemm(L, {wgrad_prob(b.c2, ga, b.a1), dg});
+        L.push_back(gather);
+      }
+      rec_bn_bwd(L, b.b1, b.c1.y, gc, b.a1, ga, nullptr);   // ga <- d(c1)
+      if (need_dx) {                                        // gc <- d(x) through the main branch
+        GemmProb dg = dgrad_prob(b.c1, ga, gc, c.dcols, gather);
+        rec_gemm(L, {wgrad_prob(b.c1, ga, x), dg});
+        L.push_back(gather);
+      } else {
+        rec_gemm(L, {wgrad_prob(b.c1, ga, x)});
+        rec_nop(L);
+      }
       if (b.has_sc) {
-        bn_bwd(p, b.bs, b.cs.y, gb, nullptr, ga, nullptr);  // ga <- d(cs)
-        conv_wgrad(p, b.cs, ga, x);
+        rec_bn_bwd(L, b.bs, b.cs.y, gb, nullptr, ga, nullptr);   // ga <- d(cs)
         if (need_dx) {
-          conv_dgrad(p, b.cs, ga, gin, c.dcols);            // gin <- d(x) through the shortcut
-          add_into(p, gc, gin, in_elems_blk);
+          GemmProb dg = dgrad_prob(b.cs, ga, gin, c.dcols, gather);   // gin <- d(x) through the shortcut
+          rec_gemm(L, {wgrad_prob(b.cs, ga, x), dg});
+          L.push_back(gather);
+          rec_add(L, gc, gin, in_elems_blk);
+        } else {
+          rec_gemm(L, {wgrad_prob(b.cs, ga, x)});
+          rec_nop(L, 2);
         }
-      } else if (need_dx) {
-        add_into(p, gc, gb, in_elems_blk);
+      } else {
+        rec_nop(L, 3);
+        if (need_dx) rec_add(L, gc, gb, in_elems_blk); else rec_nop(L);
       }
       std::swap(gin, gc);                                   // the block-input gradient feeds the next (earlier) block
     }
     if (c.has_stem) {
-      bn_bwd(p, c.stem_bn, c.stem.y, gin, c.stem_out, ga, nullptr);
-      conv_wgrad(p, c.stem, ga, c.x_nhwc);
+      rec_bn_bwd(L, c.stem_bn, c.stem.y, gin, c.stem_out, ga, nullptr);
+      rec_gemm(L, {wgrad_prob(c.stem, ga, c.x_nhwc)});
+    } else {
+      rec_nop(L, 2);
+    }
+  };
+
+  // Emit the recorded lists position by position; at a position, ops of one kind from all chunks form one
+  // grouped launch (BatchNorm ops with different vector widths stay apart).  A chunk's own order is kept.
+  auto flush_ops = [&](Plan& p, std::vector<OpList>& lists) {
+    size_t len = 0;
+    for (auto& L : lists) len = std::max(len, L.size());
+    for (size_t i = 0; i < len; ++i) {
+      std::vector<Op*> at;
+      for (auto& L : lists) if (i < L.size() && L[i].kind != OP_NOP) at.push_back(&L[i]);
+      std::vector<GemmProb> gemms;
+      std::vector<ColSumProb> cs; std::vector<float*> cs_out;
+      std::vector<GapProb> gaps; long long gap_max = 0; double gap_work = 0;
+      std::vector<AddProb> adds; long long add_max = 0; double add_work = 0;
+      for (Op* o : at) {
+        switch (o->kind) {
+          case OP_GEMM: gemms.insert(gemms.end(), o->gemms.begin(), o->gemms.end()); break;
+          case OP_COLSUM: cs.push_back(o->colsum); cs_out.push_back(o->colsum_out); break;
+          case OP_GAP_BWD: gaps.push_back(o->gap); gap_max = std::max(gap_max, o->elems); gap_work += (double)o->elems * es; break;
+          case OP_ADD: adds.push_back(o->add); add_max = std::max(add_max, o->elems); add_work += 3.0 * o->elems * es; break;
+          default: break;
+        }
+      }
+      if (!gemms.empty()) emit_gemm(h, p, gemms);
+      if (!cs.empty()) emit_colsum(h, p, cs, cs_out);
+      if (!gaps.empty()) {
+        const GapProb* dg = h.upload(gaps);
+        int n = (int)gaps.size();
+        p.add(1, [=](const RunCtx& r) { launch_gap_bwd(dg, n, gap_max, bf, r.stream); }, KIND_CONV_AUX, gap_work);
+      }
+      for (int v8 = 0; v8 < 2; ++v8) {
+        std::vector<BnStatProb> st; std::vector<BnFinalProb> fi; std::vector<BnApplyProb> ap;
+        int rows = 0, C = 0; long long elems = 0; double work = 0;
+        for (Op* o : at)
+          if (o->kind == OP_BN_BWD && (int)o->v8 == v8) {
+            st.push_back(o->bn_stat); fi.push_back(o->bn_final); ap.push_back(o->bn_apply);
+            rows = std::max(rows, o->bn_stat.rows); C = std::max(C, o->bn_stat.C); elems = std::max(elems, o->elems); work += o->work;
+          }
+        if (st.empty()) continue;
+        const BnStatProb* ds = h.upload(st);
+        const BnFinalProb* df = h.upload(fi);
+        const BnApplyProb* da = h.upload(ap);
+        int n = (int)st.size();
+        bool vec = v8 != 0;
+        p.add(3, [=](const RunCtx& r) {
+          launch_bn_stat_partial(ds, n, rows, C, true, bf, r.stream, vec);
+          launch_bn_finalize(df, n, C, true, r.stream);
+          launch_bn_apply(da, n, elems, true, bf, r.stream, vec);
+        }, KIND_NORM, work);
+      }
+      if (!adds.empty()) {
+        const AddProb* d = h.upload(adds);
+        int n = (int)adds.size();
+        p.add(1, [=](const RunCtx& r) { launch_add(d, n, add_max, bf, r.stream); }, KIND_CONV_AUX, add_work);
+      }
+      for (Op* o : at) if (o->kind == OP_RAW) o->raw(p);
     }
   };
 
@@ -373,7 +460,9 @@ void build_resnet(Handle& h) {
     emit_labels(h, p, lps);
     for (int k = 0; k < K; ++k) forward_chunk(p, k, rd, wr);
     for (int k = 0; k < K; ++k) head_forward(p, k, wr, labels_of(k, pipelined, rd), false);
-    for (int k = 0; k < K; ++k) backward_chunk(p, k, rd, wr);
+    std::vector<OpList> lists(K);
+    for (int k = 0; k < K; ++k) record_backward(lists[k], k, rd, wr);
+    flush_ops(p, lists);
     emit_pending_reduce(h, p);
     emit_optimizer(h, p);
   };

@@ -3,6 +3,7 @@
 #include "gemm_tc.h"
 
 #include <algorithm>
+#include <cmath>
 #include <stdexcept>
 
 namespace lp {
@@ -106,13 +107,16 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
   {
     std::vector<GemmProb> expanded;
     const size_t es = h.esize();
-    long long launch_tiles = 0;   // of the whole grouped launch: the other problems keep the SMs busy too
-    for (auto& g : probs) launch_tiles += (long long)((g.M + 127) / 128) * ((g.N + 255) / 256);
+    // Work of the whole grouped launch in k-slices (tiles x 64-deep slices per tile) and what one SM gets if
+    // it is spread evenly: a problem whose single tile is longer than that share would be the launch's tail.
+    double launch_slices = 0;
+    for (auto& g : probs) launch_slices += (double)((g.M + 127) / 128) * ((g.N + 255) / 256) * ((g.K + 63) / 64);
+    const double share = std::max(32.0, launch_slices / h.num_sms);
     for (auto& g : probs) {
       bool plain = g.out_f32 && g.act == EPI_NONE && !g.bias && !g.resid && g.ldc == g.N;
       long long S = 1;
-      if (plain && g.K >= 8192 && launch_tiles * 2 <= h.num_sms)
-        S = std::max(1LL, std::min<long long>({h.num_sms / launch_tiles, g.K / 2048LL, 64LL}));
+      if (plain && g.K >= 8192 && (g.K + 63) / 64 > share)
+        S = std::max(1LL, std::min<long long>({(long long)std::ceil(((g.K + 63) / 64) / share), g.K / 2048LL, 64LL}));
       if (S == 1) { expanded.push_back(g); continue; }
       size_t mn = (size_t)g.M * g.N;
       float* part = (float*)h.dalloc((size_t)S * mn * sizeof(float));
