@@ -158,6 +158,21 @@ lp_status lp_step_host(lp_handle h, const void* x_host, const void* y_host, int 
 lp_status lp_forward(lp_handle h, const void* x, const void* y, void* stream, void* out_logits,
                      float* out_losses);
 
+/*
+ * lp_evaluate: the forward chain of lp_forward on a labelled minibatch, reporting how well every chunk's
+ * auxiliary head predicts it (Sec. 3: each block is trained to predict the target on its own; the last
+ * chunk's head is the network's output).  No gradient, no update.
+ *   out_losses  (device, nullable): K floats, each chunk's mean auxiliary loss.
+ *   out_correct (device, nullable): K int32, the number of rows whose prediction equals the label.
+ *   out_pred    (device, nullable): K x rows int32 (rows = batch, or batch*seq_len for LM), the predicted
+ *     class of every row: the index of its largest logit, the lowest index among equal logits, taken on
+ *     the logits as the head stores them (activation dtype).  Rows with label -1 get a prediction but
+ *     are not counted in out_correct.
+ * BatchNorm (RESNET) uses the statistics of this minibatch, as in training.  Errors: INVALID_ARG, CUDA.
+ */
+lp_status lp_evaluate(lp_handle h, const void* x, const void* y, void* stream, float* out_losses,
+                      int* out_correct, int* out_pred);
+
 /* lp_destroy: release everything the handle owns.  NULL is accepted. */
 lp_status lp_destroy(lp_handle h);
 

@@ -286,5 +286,21 @@ class LocalUpdateOracle:
                     losses[k] = loss
         return z, losses
 
+    def evaluate(self, x, y):
+        """Forward chain with the current weights on a labelled minibatch: per chunk the auxiliary loss,
+        the logits [rows, classes], the predicted class of every row (largest logit, lowest index among
+        equal ones) and the number of rows predicted correctly (rows labelled -1 are not counted).  Every
+        chunk's head is trained to predict the target on its own (Sec. 3)."""
+        h = self._cast_input(x)
+        out = []
+        for k in range(self.K):
+            h, _ = self.chunk_forward(k, h)
+            loss, z, _, _ = self.head(k, h, y)
+            z2 = z.reshape(-1, z.shape[-1])
+            pred = np.argmax(z2, axis=1).astype(np.int32)
+            lab = np.asarray(y).reshape(-1)
+            out.append(dict(loss=float(loss), logits=z2, pred=pred, correct=int(np.sum((lab >= 0) & (pred == lab)))))
+        return out
+
     def _head_rows(self, h):
         return h.shape[:2] if self.cfg["family"] == "lm" else h.shape[0]

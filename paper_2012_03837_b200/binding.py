@@ -60,7 +60,7 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
-           "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp"]
+           "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
 
@@ -73,6 +73,7 @@ def load_library() -> C.CDLL:
     lib.lp_step.argtypes = [vp, vp, vp, ip, vp, vp]
     lib.lp_step_host.argtypes = [vp, vp, vp, ip, vp, vp]
     lib.lp_forward.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.lp_evaluate.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.lp_destroy.argtypes = [vp]
     lib.lp_num_tensors.argtypes = [vp]
     lib.lp_tensor_info_get.argtypes = [vp, ip, C.POINTER(lp_tensor_info)]
@@ -184,6 +185,10 @@ def lp_step_host(h, x_host, y_host, schedule, stream, out_losses_host):
 
 def lp_forward(h, x, y, stream, out_logits, out_losses):
     _check(h, _lib.lp_forward(h, _ptr(x), _ptr(y), stream, _ptr(out_logits), _ptr(out_losses)))
+
+
+def lp_evaluate(h, x, y, stream, out_losses=None, out_correct=None, out_pred=None):
+    _check(h, _lib.lp_evaluate(h, _ptr(x), _ptr(y), stream, _ptr(out_losses), _ptr(out_correct), _ptr(out_pred)))
 
 
 def lp_num_tensors(h) -> int:

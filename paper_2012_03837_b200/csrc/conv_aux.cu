@@ -358,6 +358,106 @@ __global__ void __launch_bounds__(256) bn_apply_vec_kernel(const BnApplyProb* __
   }
 }
 
+// ------------------------------------------------------------------ few-channel 3x3 convolution (the stem)
+// Forward: Cout / 8 threads per pixel, 8 output channels each; filters transposed to [k][Cout] in shared
+// memory (a pixel's threads read consecutive 32-byte pieces, threads of different pixels the same ones).
+template <typename T, typename WT>
+__global__ void __launch_bounds__(256) small_conv_fwd_kernel(SmallConvProb p) {
+  extern __shared__ float ws[];                       // [9 * Cin][Cout]
+  const int K = 9 * p.Cin;
+  for (int i = threadIdx.x; i < K * p.Cout; i += blockDim.x) {
+    int co = i / K, k = i - co * K;
+    ws[k * p.Cout + co] = to_f(((const WT*)p.w)[i]);
+  }
+  __syncthreads();
+  const int groups = p.Cout >> 3, ppb = blockDim.x / groups;
+  const int g = threadIdx.x % groups, pl = threadIdx.x / groups;
+  const long long total = (long long)p.N * p.H * p.W;
+  const long long pix = (long long)blockIdx.x * ppb + pl;
+  if (pl >= ppb || pix >= total) return;
+  const int w0 = (int)(pix % p.W), h0 = (int)((pix / p.W) % p.H);
+  const long long img = pix / ((long long)p.W * p.H);
+  float acc[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) acc[t] = 0.f;
+  const T* x = (const T*)p.x;
+  for (int i = 0; i < 3; ++i) {
+    const int hh = h0 + i - 1;
+    if (hh < 0 || hh >= p.H) continue;
+    for (int j = 0; j < 3; ++j) {
+      const int ww = w0 + j - 1;
+      if (ww < 0 || ww >= p.W) continue;
+      const T* xp = x + ((img * p.H + hh) * p.W + ww) * p.Cin;
+      for (int c = 0; c < p.Cin; ++c) {
+        const float xv = to_f(xp[c]);
+        const float4* wr = (const float4*)(ws + ((i * 3 + j) * p.Cin + c) * p.Cout + g * 8);
+        const float4 w0v = wr[0], w1v = wr[1];
+        acc[0] = fmaf(xv, w0v.x, acc[0]); acc[1] = fmaf(xv, w0v.y, acc[1]); acc[2] = fmaf(xv, w0v.z, acc[2]); acc[3] = fmaf(xv, w0v.w, acc[3]);
+        acc[4] = fmaf(xv, w1v.x, acc[4]); acc[5] = fmaf(xv, w1v.y, acc[5]); acc[6] = fmaf(xv, w1v.z, acc[6]); acc[7] = fmaf(xv, w1v.w, acc[7]);
+      }
+    }
+  }
+  T* y = (T*)p.y + pix * p.Cout + g * 8;
+#pragma unroll
+  for (int t = 0; t < 8; ++t) y[t] = from_f<T>(acc[t]);
+}
+
+// Filter gradient: thread (co, part) owns the taps/channels k = part, part + parts, ... of output channel co
+// (parts = 256 / Cout); a block walks its pixels in groups of 32 staged in shared memory: the 9*Cin input
+// values around each pixel and its Cout output gradients.
+template <typename T>
+__global__ void __launch_bounds__(256) small_conv_wgrad_kernel(SmallConvProb p) {
+  __shared__ float patch[32][33];
+  extern __shared__ float dys[];                      // [32][Cout]
+  const int K = 9 * p.Cin, parts = blockDim.x / p.Cout;
+  const int co = threadIdx.x % p.Cout, part = threadIdx.x / p.Cout;
+  const long long total = (long long)p.N * p.H * p.W;
+  const long long p0 = (long long)blockIdx.x * SMALLCONV_PIXELS;
+  float acc[8];                                       // ceil(32 / parts) <= 8 for parts >= 4
+#pragma unroll
+  for (int t = 0; t < 8; ++t) acc[t] = 0.f;
+  const T* x = (const T*)p.x;
+  const T* dy = (const T*)p.dy;
+  for (long long base = p0; base < p0 + SMALLCONV_PIXELS && base < total; base += 32) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < 32 * K; i += blockDim.x) {
+      const int pl = i / K, k = i - pl * K;
+      const long long pix = base + pl;
+      float v = 0.f;
+      if (pix < total) {
+        const int tap = k / p.Cin, c = k - tap * p.Cin;
+        const int ww = (int)(pix % p.W) + tap % 3 - 1, hh = (int)((pix / p.W) % p.H) + tap / 3 - 1;
+        if (hh >= 0 && hh < p.H && ww >= 0 && ww < p.W)
+          v = to_f(x[((pix / ((long long)p.W * p.H) * p.H + hh) * p.W + ww) * p.Cin + c]);
+      }
+      patch[pl][k] = v;
+    }
+    for (int i = threadIdx.x; i < 32 * p.Cout; i += blockDim.x) {
+      const long long pix = base + i / p.Cout;
+      dys[i] = pix < total ? to_f(dy[pix * p.Cout + i % p.Cout]) : 0.f;
+    }
+    __syncthreads();
+    if (part < parts) {
+      for (int pl = 0; pl < 32; ++pl) {
+        const float d = dys[pl * p.Cout + co];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const int k = part + t * parts;
+          if (k < K) acc[t] = fmaf(d, patch[pl][k], acc[t]);
+        }
+      }
+    }
+  }
+  if (part < parts) {
+    float* out = p.part + (size_t)blockIdx.x * p.Cout * K + (size_t)co * K;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      const int k = part + t * parts;
+      if (k < K) out[k] = acc[t];
+    }
+  }
+}
+
 unsigned grid_for(long long elems) {
   long long b = (elems + 255) / 256;
   long long cap = 148LL * 32;
@@ -408,6 +508,25 @@ void launch_gap_fwd(const GapProb* d, int n, int max_n, int max_c, bool is_bf16,
   dim3 grid((max_c + 255) / 256, max_n, n);
   if (is_bf16) gap_fwd_kernel<bf16><<<grid, 256, 0, s>>>(d);
   else gap_fwd_kernel<float><<<grid, 256, 0, s>>>(d);
+}
+void launch_small_conv_fwd(const SmallConvProb& p, bool w_is_bf16, bool is_bf16, cudaStream_t s) {
+  const int groups = p.Cout / 8, ppb = 256 / groups;
+  const long long total = (long long)p.N * p.H * p.W;
+  const unsigned grid = (unsigned)((total + ppb - 1) / ppb);
+  const size_t smem = (size_t)9 * p.Cin * p.Cout * sizeof(float);
+  if (is_bf16) {
+    if (w_is_bf16) small_conv_fwd_kernel<bf16, bf16><<<grid, 256, smem, s>>>(p);
+    else small_conv_fwd_kernel<bf16, float><<<grid, 256, smem, s>>>(p);
+  } else {
+    small_conv_fwd_kernel<float, float><<<grid, 256, smem, s>>>(p);
+  }
+}
+void launch_small_conv_wgrad(const SmallConvProb& p, bool is_bf16, cudaStream_t s) {
+  const long long total = (long long)p.N * p.H * p.W;
+  const unsigned grid = (unsigned)((total + SMALLCONV_PIXELS - 1) / SMALLCONV_PIXELS);
+  const size_t smem = (size_t)32 * p.Cout * sizeof(float);
+  if (is_bf16) small_conv_wgrad_kernel<bf16><<<grid, 256, smem, s>>>(p);
+  else small_conv_wgrad_kernel<float><<<grid, 256, smem, s>>>(p);
 }
 void launch_gap_bwd(const GapProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s) {
   dim3 grid(grid_for(max_elems), n);

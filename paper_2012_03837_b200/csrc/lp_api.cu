@@ -342,6 +342,25 @@ lp_status lp_forward(lp_handle hh, const void* x, const void* y, void* stream, v
   return check_cuda(&h, "lp_forward");
 }
 
+lp_status lp_evaluate(lp_handle hh, const void* x, const void* y, void* stream, float* out_losses, int* out_correct,
+                      int* out_pred) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!x || !y) return fail(&h, LP_ERR_INVALID_ARG, "null x or y");
+  if (!out_losses && !out_correct && !out_pred) return fail(&h, LP_ERR_INVALID_ARG, "no output requested");
+  cudaStream_t s = (cudaStream_t)stream;
+  lp_status st = copy_inputs(h, x, y, cudaMemcpyDeviceToDevice, s);
+  if (st != LP_OK) return st;
+  if (out_correct) cudaMemsetAsync(out_correct, 0, sizeof(int) * h.K, s);
+  RunCtx ctx{s, nullptr, nullptr};
+  ctx.out_pred = out_pred;
+  ctx.out_correct = out_correct;
+  int half = h.primed ? h.parity ^ 1 : 0;                 // the half no chunk will read next step
+  h.fwd_plan[half].run(ctx);
+  if (out_losses) cudaMemcpyAsync(out_losses, h.d_losses, sizeof(float) * h.K, cudaMemcpyDeviceToDevice, s);
+  return check_cuda(&h, "lp_evaluate");
+}
+
 int lp_num_tensors(lp_handle hh) { return hh ? (int)hh->h.tensors.size() : 0; }
 
 lp_status lp_tensor_info_get(lp_handle hh, int i, lp_tensor_info* out) {

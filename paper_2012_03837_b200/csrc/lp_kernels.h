@@ -129,6 +129,13 @@ struct XentStatsProb {
 enum { XENT_APPLY_ROWS = 256 };
 void launch_xent_from_stats(const XentStatsProb* d_probs, int n, int max_rows, int classes, cudaStream_t s);
 
+// Prediction of every row: the index of its largest logit, the lowest index among equal values (an
+// integer result: exact).  pred[chunk * pred_stride + r] receives it; correct[chunk] counts the rows
+// whose prediction equals the label (rows with a negative label are not counted).  Either may be null.
+struct ArgmaxProb { const void* z; const int* y; int rows, classes, ld, chunk; };
+void launch_argmax(const ArgmaxProb* d_probs, int n, int max_rows, bool is_bf16, int* pred, int pred_stride,
+                   int* correct, cudaStream_t s);
+
 struct LossProb { const float* row_loss; const int* n_valid; int rows; int out_index; };
 void launch_loss_reduce(const LossProb* d_probs, int n, float* d_losses, int* d_status, cudaStream_t s);
 
@@ -180,6 +187,18 @@ struct BnApplyProb {
   int rows, C, relu;
 };
 void launch_bn_apply(const BnApplyProb* d_probs, int n, long long max_elems, bool bwd, bool is_bf16, cudaStream_t s, bool vec8 = false);
+
+// 3x3 stride-1 convolution of an image with very few channels (9 * Cin <= 32: the stem of App. B.3's
+// networks, which a 64-deep tensor-core k-slice would leave mostly empty), on the FP32 ALUs with fp32
+// accumulation.  x [N,H,W,Cin] NHWC, filters w [Cout,3,3,Cin], y / dy [N,H,W,Cout]; Cout % 8 == 0.
+//   forward: y = conv(x, w).
+//   filter gradient: part[blk][co*9*Cin + k] = sum over block blk's SMALLCONV_PIXELS pixels of
+//     dy[pixel, co] * x[pixel shifted by tap(k), channel(k)]  (needs 256 % Cout == 0); the blocks'
+//     partial sums are added up in block order by the caller's column reduction.
+struct SmallConvProb { const void* x; const void* w; void* y; const void* dy; float* part; int N, H, W, Cin, Cout; };
+enum { SMALLCONV_PIXELS = 512 };
+void launch_small_conv_fwd(const SmallConvProb& p, bool w_is_bf16, bool is_bf16, cudaStream_t s);
+void launch_small_conv_wgrad(const SmallConvProb& p, bool is_bf16, cudaStream_t s);
 
 struct GapProb { const void* x; void* y; const void* dy; void* dx; int N, HW, C; };
 void launch_gap_fwd(const GapProb* d_probs, int n, int max_n, int max_c, bool is_bf16, cudaStream_t s);

@@ -214,6 +214,9 @@ void build_lm(Handle& h) {
       p.add(0, [zlast, zbytes](const RunCtx& c) {
         if (c.out_logits) cudaMemcpyAsync(c.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, c.stream);
       });
+      std::vector<ArgmaxProb> am;
+      for (int k = 0; k < K; ++k) am.push_back(ArgmaxProb{cb[k].z, labels_of(k, pipelined, rd), M, V, V, k});
+      emit_argmax(h, p, am);
     }
     std::vector<float*> bgs;
     for (int k = 0; k < K; ++k) bgs.push_back(h.G(hn(k, "b")));

@@ -177,6 +177,9 @@ void build_mlp(Handle& h) {
     p.add(0, [zlast, zbytes](const RunCtx& c) {
       if (c.out_logits) cudaMemcpyAsync(c.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, c.stream);
     });
+    std::vector<ArgmaxProb> am;
+    for (int k = 0; k < K; ++k) am.push_back(ArgmaxProb{b.z[k], h.y_in, B, C, C, k});
+    emit_argmax(h, p, am);
     emit_xent_and_loss(h, p, xs, all);
   };
 

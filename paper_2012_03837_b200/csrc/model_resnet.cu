@@ -24,6 +24,8 @@ struct Conv {
   void* y = nullptr;
   // implicit GEMM on the tensor-core kernel (no im2col / col2im): forward and weight gradient, input gradient
   bool imp_fwd = false, imp_dgrad = false;
+  // few-channel direct convolution on the FP32 ALUs (the stem): forward and filter gradient, no im2col
+  bool small = false;
 };
 struct Bn {
   std::string g, b;
@@ -146,7 +148,7 @@ void build_resnet(Handle& h) {
   };
   auto alloc_conv = [&](Conv& c) {
     set_implicit(c);
-    if (!c.imp_fwd) c.cols = h.dalloc((size_t)c.M * c.ldk * es);
+    if (!c.imp_fwd && !c.small) c.cols = h.dalloc((size_t)c.M * c.ldk * es);
     c.y = h.dalloc((size_t)c.M * c.Cout * es);
   };
   auto alloc_bn = [&](Bn& b) { b.mean = fal(b.C); b.rstd = fal(b.C); };
@@ -167,6 +169,8 @@ void build_resnet(Handle& h) {
     };
     if (c.has_stem) {
       c.x_nhwc = h.dalloc(in_elems * es);
+      c.stem.small = c.stem.k == 3 && c.stem.stride == 1 && 9 * c.stem.Cin <= 32 && c.stem.Cout % 8 == 0 &&
+                     c.stem.Cout <= 64 && 256 % c.stem.Cout == 0;
       alloc_conv(c.stem); alloc_bn(c.stem_bn); track(c.stem);
       c.stem_out = h.dalloc((size_t)c.stem.M * c.stem.Cout * es);
     }
@@ -191,6 +195,11 @@ void build_resnet(Handle& h) {
     g.conv = mode; g.conv_n = c.N; g.conv_h = c.H; g.conv_w = c.W; g.conv_c = channels; g.conv_k0 = 0;
   };
   auto conv_fwd = [&](Plan& p, const Conv& c, const void* x) {
+    if (c.small) {
+      SmallConvProb sp{x, h.W(c.w), c.y, nullptr, nullptr, c.N, c.H, c.W, c.Cin, c.Cout};
+      p.add(1, [=](const RunCtx& r) { launch_small_conv_fwd(sp, bf, bf, r.stream); }, KIND_GEMM_ALU, 2.0 * c.M * c.Cout * c.K);
+      return;
+    }
     if (c.imp_fwd) {
       GemmProb g = gemm_fwd(x, h.W(c.w), c.y, (int)c.M, c.Cout, c.K, nullptr, EPI_NONE);
       g.a_ms = c.Cin;
@@ -273,6 +282,7 @@ void build_resnet(Handle& h) {
         if (r.out_logits) cudaMemcpyAsync(r.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, r.stream);
       });
     }
+    if (copy_logits) emit_argmax(h, p, {ArgmaxProb{c.z, labels, B, NC, NC, k}});
     emit_xent_and_loss(h, p, {XentProb{c.z, labels, h.n_valid[k], c.row_loss, B, NC, NC, nullptr}}, {k});
   };
 
@@ -387,7 +397,19 @@ void build_resnet(Handle& h) {
     }
     if (c.has_stem) {
       rec_bn_bwd(L, c.stem_bn, c.stem.y, gin, c.stem_out, ga, nullptr);
-      rec_gemm(L, {wgrad_prob(c.stem, ga, c.x_nhwc)});
+      if (c.stem.small) {
+        const Conv& cv = c.stem;
+        const int nblk = (int)((cv.M + SMALLCONV_PIXELS - 1) / SMALLCONV_PIXELS), cols = cv.Cout * cv.K;
+        float* part = fal((size_t)nblk * cols);
+        h.pending_reduce.push_back(ColReduceProb{part, h.G(cv.w), nblk, cols, cols});
+        SmallConvProb sp{c.x_nhwc, nullptr, nullptr, ga, part, cv.N, cv.H, cv.W, cv.Cin, cv.Cout};
+        const double work = 2.0 * cv.M * cv.Cout * cv.K;
+        Op o; o.kind = OP_RAW;
+        o.raw = [=](Plan& p) { p.add(1, [=](const RunCtx& r) { launch_small_conv_wgrad(sp, bf, r.stream); }, KIND_GEMM_ALU, work); };
+        L.push_back(std::move(o));
+      } else {
+        rec_gemm(L, {wgrad_prob(c.stem, ga, c.x_nhwc)});
+      }
     } else {
       rec_nop(L, 2);
     }

@@ -244,6 +244,41 @@ __global__ void __launch_bounds__(256) loss_reduce_kernel(const LossProb* __rest
   }
 }
 
+// One block per row.  A candidate (value, index) beats another if its value is larger, or equal with a
+// smaller index; threads scan their columns in increasing order, so "strictly larger" keeps the first.
+template <typename T>
+__global__ void __launch_bounds__(256) argmax_kernel(const ArgmaxProb* __restrict__ probs, int* pred, int pred_stride,
+                                                     int* correct) {
+  __shared__ float sv[8];
+  __shared__ int si[8];
+  const ArgmaxProb p = probs[blockIdx.y];
+  const int r = blockIdx.x;
+  if (r >= p.rows) return;
+  const T* z = (const T*)p.z + (size_t)r * p.ld;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int c = threadIdx.x; c < p.classes; c += blockDim.x) {
+    float v = to_f(z[c]);
+    if (v > best) { best = v; bi = c; }
+  }
+  auto merge = [](float& v, int& i, float ov, int oi) {
+    if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+  };
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) merge(best, bi, __shfl_xor_sync(0xffffffffu, best, o), __shfl_xor_sync(0xffffffffu, bi, o));
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = best; si[threadIdx.x >> 5] = bi; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) merge(best, bi, sv[w], si[w]);
+    if (bi == 0x7fffffff) bi = 0;              // no finite value in the row
+    if (pred) pred[(size_t)p.chunk * pred_stride + r] = bi;
+    if (correct) {
+      const int lab = p.y[r];
+      if (lab >= 0 && lab == bi) atomicAdd(&correct[p.chunk], 1);   // integer sum: order does not matter
+    }
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) add_kernel(const AddProb* __restrict__ probs) {
   const AddProb p = probs[blockIdx.y];
@@ -284,6 +319,12 @@ void launch_xent(const XentProb* d, int n, int max_rows, bool is_bf16, cudaStrea
 }
 void launch_loss_reduce(const LossProb* d, int n, float* d_losses, int* d_status, cudaStream_t s) {
   loss_reduce_kernel<<<n, 256, 0, s>>>(d, d_losses, d_status);
+}
+void launch_argmax(const ArgmaxProb* d, int n, int max_rows, bool is_bf16, int* pred, int pred_stride, int* correct,
+                   cudaStream_t s) {
+  if (n < 1 || max_rows < 1) return;
+  dim3 grid(max_rows, n);
+  DISPATCH_T(is_bf16, argmax_kernel, grid, 256, s, d, pred, pred_stride, correct);
 }
 void launch_add(const AddProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s) {
   long long blocks = (max_elems + 255) / 256;

@@ -342,6 +342,17 @@ void emit_xent_from_stats(Handle& h, Plan& p, std::vector<XentStatsProb> probs, 
   }, KIND_XENT, by);
 }
 
+void emit_argmax(Handle& h, Plan& p, const std::vector<ArgmaxProb>& probs) {
+  if (probs.empty()) return;
+  const ArgmaxProb* d = h.upload(probs);
+  int n = (int)probs.size(), mr = 0, stride = h.rows;
+  for (auto& q : probs) mr = std::max(mr, q.rows);
+  bool bf = h.bf16_mode;
+  p.add(0, [=](const RunCtx& c) {
+    if (c.out_pred || c.out_correct) launch_argmax(d, n, mr, bf, c.out_pred, stride, c.out_correct, c.stream);
+  });
+}
+
 void emit_optimizer(Handle& h, Plan& p) {
   Handle* hp = &h;
   p.add(1, [hp](const RunCtx& c) {

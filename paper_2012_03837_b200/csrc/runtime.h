@@ -30,6 +30,8 @@ struct RunCtx {
   cudaStream_t stream;
   void* out_logits;                      // lp_forward only
   std::vector<ProfRecord>* prof;         // non-null: bracket every op with events
+  int* out_pred = nullptr;               // lp_evaluate only: per-row predictions [K, rows]
+  int* out_correct = nullptr;            // lp_evaluate only: per-chunk count of correct predictions
 };
 
 struct PlanOp {
@@ -152,6 +154,8 @@ bool emit_xent_and_loss(Handle& h, Plan& p, std::vector<XentProb> probs, const s
 void emit_xent_from_stats(Handle& h, Plan& p, std::vector<XentStatsProb> probs, const std::vector<int>& chunk_of,
                           const std::vector<float*>* bias_grads);
 void emit_optimizer(Handle& h, Plan& p);
+// Predictions of the heads' logits (before the cross-entropy overwrites them); runs only under lp_evaluate
+void emit_argmax(Handle& h, Plan& p, const std::vector<ArgmaxProb>& probs);
 
 // GEMM problem constructors (x: [M,K] row-major, W: [N,K] row-major, dy: [M,N] row-major)
 GemmProb gemm_fwd(const void* x, const void* W, void* y, int M, int N, int Kd, const float* bias, int act);

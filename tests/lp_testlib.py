@@ -92,6 +92,18 @@ class GpuModel:
         return logits.float().cpu().numpy(), self.losses.cpu().numpy().astype(np.float64)
 
 
+def gpu_evaluate(gm: GpuModel, x, y):
+    """lp_evaluate on (x, y): (losses [K], correct [K], predictions [K, rows])."""
+    xt, yt = gm.device_batch(x, y)
+    rows = lp_synth.units_per_step(gm.cfg)
+    correct = torch.full((gm.K,), -1, dtype=torch.int32, device=gm.dev)
+    pred = torch.full((gm.K, rows), -1, dtype=torch.int32, device=gm.dev)
+    lp.lp_evaluate(gm.h, xt, yt, gm.stream, gm.losses, correct, pred)
+    torch.cuda.synchronize()
+    lp.lp_status_poll(gm.h, gm.stream)
+    return gm.losses.cpu().numpy().astype(np.float64), correct.cpu().numpy(), pred.cpu().numpy()
+
+
 def tensor_rel_err(a: np.ndarray, b: np.ndarray) -> float:
     """max |a - b| / max |b| over one tensor (the oracle's tensor is b)."""
     return float(np.abs(a.astype(np.float64) - b.astype(np.float64)).max() / max(np.abs(b).max(), 1e-30))

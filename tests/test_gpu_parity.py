@@ -214,3 +214,57 @@ def test_idle_ramp_up_reset_and_checkpoint():
     werr = T.compare_weights(gm, orc, params)
     assert max(e for _, e in werr.values()) <= 1e-3, werr
     gm.close(); gm2.close()
+
+
+# ------------------------------------------------------------------ predictions (integer work: exact)
+
+def check_evaluate(cfg, steps=3, margin=None):
+    """lp_evaluate after a few training steps against the oracle's evaluate().  The argmax is an integer
+    decision taken on floating-point logits, so it is compared where it is unique at the kernel's precision:
+    rows whose two best oracle logits differ by more than the rounding of the stored logits must match
+    exactly, every other row must pick a class within that margin of the best, and the last chunk's
+    predictions must equal the argmax (lowest index on ties) of the logits lp_forward returns, bit for bit.
+    The counts must equal what the library's own predictions give."""
+    dt = cfg["dtype"]
+    gl, ol, gm, orc = T.run_both(cfg, steps)
+    x, y = lp_synth.minibatch(cfg, steps)
+    losses, correct, pred = T.gpu_evaluate(gm, x, y)
+    ref = orc.evaluate(x, y)
+    lab = np.asarray(y).reshape(-1)
+    margin = margin if margin is not None else (2e-2 if dt == "bf16" else 1e-4)
+    for k, r in enumerate(ref):
+        assert abs(losses[k] - r["loss"]) <= LOSS_TOL[dt] * abs(r["loss"]), (k, losses[k], r["loss"])
+        z = r["logits"].astype(np.float64)
+        top = z.max(axis=1)
+        scale = np.abs(z).max()
+        z_sorted = np.sort(z, axis=1)
+        clear = (z_sorted[:, -1] - z_sorted[:, -2]) > margin * scale
+        assert np.array_equal(pred[k][clear], r["pred"][clear]), (k, int(np.sum(pred[k][clear] != r["pred"][clear])))
+        picked = z[np.arange(z.shape[0]), pred[k]]
+        assert np.all(top - picked <= margin * scale), k
+        assert correct[k] == int(np.sum((lab >= 0) & (pred[k] == lab))), (k, correct[k])
+    logits, _ = gm.forward(x, y)
+    assert np.array_equal(pred[-1], np.argmax(logits, axis=1).astype(np.int32))
+    print("evaluate: correct per chunk", correct.tolist(), "oracle", [r["correct"] for r in ref],
+          "rows decided within the margin:", [int(np.sum(~((np.sort(r["logits"], axis=1)[:, -1] - np.sort(r["logits"], axis=1)[:, -2]) > margin * np.abs(r["logits"]).max()))) for r in ref])
+    gm.close()
+
+
+def test_evaluate_mlp_fp32():
+    check_evaluate(lp_synth.config("c1"))
+
+
+def test_evaluate_mlp_bf16_many_classes():
+    check_evaluate(lp_synth.config("c2", batch=192, d_in=160, chunks=[[256, 192], [320, 256], [128, 256]], classes=200))
+
+
+def test_evaluate_lm_bf16_ignored_positions():
+    cfg = lp_synth.config("c3", batch=3, seq_len=136, vocab=1000, d_model=128, n_heads=2, d_ffn=320,
+                          blocks_per_chunk=[1, 2, 1], schedule="pipelined")
+    check_evaluate(cfg)
+
+
+def test_evaluate_resnet_bf16():
+    cfg = lp_synth.config("c4", batch=32, height=16, width=16, stem_channels=64,
+                          stage_channels=[64, 128], blocks_per_stage=2, classes=10)
+    check_evaluate(cfg, margin=5e-2)

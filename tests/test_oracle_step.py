@@ -324,3 +324,25 @@ def test_key_bias_gradient_is_identically_zero():
     for n, g in orc.last_grads.items():
         if n.endswith(".bqkv"):
             assert np.abs(g[d:2 * d]).max() < 1e-12 * np.abs(g[:d]).max()
+
+
+def test_evaluate_counts_follow_the_logits_and_ties_take_the_lowest_index():
+    """evaluate(): the prediction is the first largest logit; labels of -1 are not counted; the losses equal
+    forward()'s.  A head with all-zero weights makes every logit equal, so every row predicts class 0."""
+    cfg = lp_synth.config("c3", dtype="fp32", batch=2, seq_len=12, vocab=17, d_model=64, n_heads=1, d_ffn=32,
+                          blocks_per_chunk=[1, 1])
+    params = lp_synth.init_params(cfg)
+    params["c1.head.W"] = np.zeros_like(params["c1.head.W"])
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    x, y = lp_synth.minibatch(cfg, 0)
+    ev = orc.evaluate(x, y)
+    _, losses = orc.forward(x, y)
+    lab = y.reshape(-1)
+    assert (lab == -1).sum() == cfg["batch"]                       # the last position of every sequence
+    for k, r in enumerate(ev):
+        assert abs(r["loss"] - losses[k]) < 1e-12
+        brute = np.array([max(range(17), key=lambda c: (row[c], -c)) for row in r["logits"]])
+        assert np.array_equal(r["pred"], brute)
+        assert r["correct"] == sum(int(p == t) for p, t in zip(r["pred"], lab) if t >= 0)
+    assert np.all(ev[1]["pred"] == 0)
+    assert ev[1]["correct"] == int(np.sum(lab == 0))
