@@ -59,7 +59,8 @@ enum { LP_MASTER = 0, LP_WORKING = 1, LP_MOMENT1 = 2, LP_MOMENT2 = 3, LP_GRAD = 
  *    blocks_per_chunk[k] blocks.
  *  RESNET (App. B.3): 3x3 stem convolution + BatchNorm + ReLU (in chunk 0), then K stages of
  *    blocks_per_stage BasicBlocks with stage_channels[k] channels; stages after the first start
- *    with stride 2 and a 1x1-convolution + BatchNorm shortcut.  BatchNorm uses batch statistics.
+ *    with stride 2 and a 1x1-convolution + BatchNorm shortcut.  BatchNorm uses batch statistics
+ *    (and keeps running statistics, which lp_evaluate can use).
  */
 typedef struct {
   int family;
@@ -168,9 +169,15 @@ lp_status lp_forward(lp_handle h, const void* x, const void* y, void* stream, vo
  *     class of every row: the index of its largest logit, the lowest index among equal logits, taken on
  *     the logits as the head stores them (activation dtype).  Rows with label -1 get a prediction but
  *     are not counted in out_correct.
- * BatchNorm (RESNET) uses the statistics of this minibatch, as in training.  Errors: INVALID_ARG, CUDA.
+ *   bn_mode: what BatchNorm (RESNET) normalises with.  LP_BN_BATCH: the statistics of this minibatch, as in
+ *     training.  LP_BN_RUNNING: its running mean and variance -- exponential averages (momentum 0.1) of the
+ *     batch mean and the unbiased batch variance that every training step of a chunk updates (tensors
+ *     "<bn>.rm" and "<bn>.rv", starting from 0 and 1; the optimizer never changes them).  Ignored by the
+ *     other families.
+ * Errors: INVALID_ARG, CUDA.
  */
-lp_status lp_evaluate(lp_handle h, const void* x, const void* y, void* stream, float* out_losses,
+enum { LP_BN_BATCH = 0, LP_BN_RUNNING = 1 };
+lp_status lp_evaluate(lp_handle h, const void* x, const void* y, void* stream, int bn_mode, float* out_losses,
                       int* out_correct, int* out_pred);
 
 /* lp_destroy: release everything the handle owns.  NULL is accepted. */

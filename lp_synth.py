@@ -109,14 +109,16 @@ def param_table(cfg: dict) -> list[dict]:
     "ones"), and whether weight decay applies (matrices and filters only).
 
     Layouts: Linear weights are [out, in]; convolution filters are [C_out, C_in, kh, kw];
-    embedding tables are [rows, d_model].
+    embedding tables are [rows, d_model].  Entries marked buffer=True are state that no gradient
+    reaches (BatchNorm running mean ".rm" and variance ".rv"); they come last so that the other
+    tensors keep their random streams.
     """
     fam = cfg["family"]
     out: list[dict] = []
 
-    def add(name, chunk, shape, init, std=0.0, decay=False):
+    def add(name, chunk, shape, init, std=0.0, decay=False, buffer=False):
         out.append(dict(name=name, chunk=chunk, shape=tuple(int(s) for s in shape), init=init,
-                        std=float(std), decay=bool(decay)))
+                        std=float(std), decay=bool(decay), buffer=bool(buffer)))
 
     if fam == "mlp":
         d_prev = cfg["d_in"]
@@ -178,6 +180,10 @@ def param_table(cfg: dict) -> list[dict]:
             c_prev = c
             add(f"c{k}.head.W", k, (cfg["classes"], c), "normal", np.sqrt(1.0 / c), True)
             add(f"c{k}.head.b", k, (cfg["classes"],), "zeros")
+        for t in [t for t in out if t["name"].endswith(".g") and ".bn" in t["name"]]:
+            stem = t["name"][:-2]
+            add(stem + ".rm", t["chunk"], t["shape"], "zeros", buffer=True)
+            add(stem + ".rv", t["chunk"], t["shape"], "ones", buffer=True)
     else:
         raise ValueError(fam)
     return out

@@ -89,6 +89,20 @@ def batchnorm_fwd(x, g, b, eps=1e-5):
     return y, (xhat, rstd, g, mu.reshape(-1), var.reshape(-1))
 
 
+def batchnorm_running_update(run_mean, run_var, cache, n, momentum=0.1):
+    """Running statistics after a train-mode pass over n values per channel: exponential averages of the
+    batch mean and of the unbiased batch variance (n / (n - 1) times the biased one)."""
+    mu, var = cache[3], cache[4]
+    unbiased = var * (n / max(n - 1, 1))
+    return (1 - momentum) * run_mean + momentum * mu, (1 - momentum) * run_var + momentum * unbiased
+
+
+def batchnorm_eval(x, g, b, run_mean, run_var, eps=1e-5):
+    """Evaluation-mode BatchNorm over [N, C, H, W]: normalises with the running statistics."""
+    sh = (1, -1, 1, 1)
+    return (x - run_mean.reshape(sh)) / np.sqrt(run_var.reshape(sh) + eps) * g.reshape(sh) + b.reshape(sh)
+
+
 def batchnorm_bwd(dy, cache):
     xhat, rstd, g = cache[:3]
     dxhat = dy * g.reshape(1, -1, 1, 1)

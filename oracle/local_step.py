@@ -45,6 +45,9 @@ class LocalUpdateOracle:
         self.state = {t["name"]: {} for t in self.table}
         self.names_of_chunk = [[t["name"] for t in self.table if t["chunk"] == k] for k in range(self.K)]
         self.decay = {t["name"]: t["decay"] for t in self.table}
+        self.buffers = {t["name"] for t in self.table if t.get("buffer")}   # state no gradient reaches
+        self.bn_mode = "batch"   # "running": BatchNorm normalises with its running statistics (evaluation)
+        self.training = False    # True inside a training step: BatchNorm then updates its running statistics
         self.ramp = ramp
         self.buf = None          # pipelined: buf[k] = (activation, labels) chunk k+1 reads next
         self.t = 0               # pipelined steps taken since the last reset
@@ -165,26 +168,40 @@ class LocalUpdateOracle:
         cache = {"blocks": []}
         if k == 0:
             u, cc = L.conv2d_fwd(x, p["c0.stem.conv"], 1, 1)
-            u, cb = L.batchnorm_fwd(u, p["c0.stem.bn.g"], p["c0.stem.bn.b"])
+            u, cb = self._bn(u, "c0.stem.bn")
             x, cr = L.relu_fwd(u)
             cache["stem"] = (cc, cb, cr)
         for j in range(self.cfg["blocks_per_stage"]):
             n = f"c{k}.r{j}"
             s = lp_synth.resnet_stage_stride(self.cfg, k) if j == 0 else 1
             u, cc1 = L.conv2d_fwd(x, p[n + ".conv1"], s, 1)
-            u, cb1 = L.batchnorm_fwd(u, p[n + ".bn1.g"], p[n + ".bn1.b"])
+            u, cb1 = self._bn(u, n + ".bn1")
             u, cr1 = L.relu_fwd(u)
             u, cc2 = L.conv2d_fwd(u, p[n + ".conv2"], 1, 1)
-            u, cb2 = L.batchnorm_fwd(u, p[n + ".bn2.g"], p[n + ".bn2.b"])
+            u, cb2 = self._bn(u, n + ".bn2")
             if n + ".sc.conv" in p:
                 sc, ccs = L.conv2d_fwd(x, p[n + ".sc.conv"], s, 0)
-                sc, cbs = L.batchnorm_fwd(sc, p[n + ".sc.bn.g"], p[n + ".sc.bn.b"])
+                sc, cbs = self._bn(sc, n + ".sc.bn")
                 csc = (ccs, cbs)
             else:
                 sc, csc = x, None
             x, cr2 = L.relu_fwd(u + sc)
             cache["blocks"].append((n, cc1, cb1, cr1, cc2, cb2, csc, cr2))
         return x, cache
+
+    def _bn(self, x, name):
+        """BatchNorm `name` on x.  Training and plain forward passes use the batch statistics (App. B.3's
+        networks are trained with them); a training step also moves the running statistics.  In
+        evaluation mode (bn_mode "running") the running statistics normalise instead."""
+        p = self.p
+        if self.bn_mode == "running":
+            return L.batchnorm_eval(x, p[name + ".g"], p[name + ".b"], p[name + ".rm"], p[name + ".rv"]), None
+        y, cache = L.batchnorm_fwd(x, p[name + ".g"], p[name + ".b"])
+        if self.training:
+            n = x.shape[0] * x.shape[2] * x.shape[3]
+            rm, rv = L.batchnorm_running_update(p[name + ".rm"], p[name + ".rv"], cache, n)
+            p[name + ".rm"], p[name + ".rv"] = rm.astype(p[name + ".rm"].dtype), rv.astype(p[name + ".rv"].dtype)
+        return y, cache
 
     def _resnet_bwd(self, k, dx, cache):
         g = {}
@@ -216,7 +233,11 @@ class LocalUpdateOracle:
 
     def local_grads(self, k, inp, y):
         """Steps 2-4 for one chunk: forward, auxiliary loss, backward truncated at `inp`."""
-        h, cache = self.chunk_forward(k, inp)
+        self.training = True
+        try:
+            h, cache = self.chunk_forward(k, inp)
+        finally:
+            self.training = False
         loss, _, dh, g = self.head(k, h, y)
         g.update(self.chunk_backward(k, dh, cache))
         return loss, h, g
@@ -225,6 +246,8 @@ class LocalUpdateOracle:
         """Optimizer update of chunk k's trunk and head from its own gradients only."""
         o = self.cfg["optim"]
         for n in self.names_of_chunk[k]:
+            if n in self.buffers:
+                continue
             if o["kind"] == "sgdm":
                 self.p[n] = O.sgdm_update(self.p[n], grads[n], self.state[n], o["lr"], o["momentum"],
                                           o.get("weight_decay", 0.0), self.decay[n])
@@ -286,15 +309,24 @@ class LocalUpdateOracle:
                     losses[k] = loss
         return z, losses
 
-    def evaluate(self, x, y):
+    def evaluate(self, x, y, bn="batch"):
         """Forward chain with the current weights on a labelled minibatch: per chunk the auxiliary loss,
         the logits [rows, classes], the predicted class of every row (largest logit, lowest index among
         equal ones) and the number of rows predicted correctly (rows labelled -1 are not counted).  Every
-        chunk's head is trained to predict the target on its own (Sec. 3)."""
+        chunk's head is trained to predict the target on its own (Sec. 3).  bn="running": BatchNorm
+        normalises with its running statistics instead of this minibatch's."""
         h = self._cast_input(x)
         out = []
+        self.bn_mode = bn        # "running": BatchNorm uses its running statistics instead of this minibatch's
+        try:
+            hs = []
+            for k in range(self.K):
+                h, _ = self.chunk_forward(k, h)
+                hs.append(h)
+        finally:
+            self.bn_mode = "batch"
         for k in range(self.K):
-            h, _ = self.chunk_forward(k, h)
+            h = hs[k]
             loss, z, _, _ = self.head(k, h, y)
             z2 = z.reshape(-1, z.shape[-1])
             pred = np.argmax(z2, axis=1).astype(np.int32)

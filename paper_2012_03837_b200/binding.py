@@ -73,7 +73,7 @@ def load_library() -> C.CDLL:
     lib.lp_step.argtypes = [vp, vp, vp, ip, vp, vp]
     lib.lp_step_host.argtypes = [vp, vp, vp, ip, vp, vp]
     lib.lp_forward.argtypes = [vp, vp, vp, vp, vp, vp]
-    lib.lp_evaluate.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.lp_evaluate.argtypes = [vp, vp, vp, vp, ip, vp, vp, vp]
     lib.lp_destroy.argtypes = [vp]
     lib.lp_num_tensors.argtypes = [vp]
     lib.lp_tensor_info_get.argtypes = [vp, ip, C.POINTER(lp_tensor_info)]
@@ -187,8 +187,11 @@ def lp_forward(h, x, y, stream, out_logits, out_losses):
     _check(h, _lib.lp_forward(h, _ptr(x), _ptr(y), stream, _ptr(out_logits), _ptr(out_losses)))
 
 
-def lp_evaluate(h, x, y, stream, out_losses=None, out_correct=None, out_pred=None):
-    _check(h, _lib.lp_evaluate(h, _ptr(x), _ptr(y), stream, _ptr(out_losses), _ptr(out_correct), _ptr(out_pred)))
+LP_BN_BATCH, LP_BN_RUNNING = 0, 1
+
+
+def lp_evaluate(h, x, y, stream, out_losses=None, out_correct=None, out_pred=None, bn_mode=LP_BN_BATCH):
+    _check(h, _lib.lp_evaluate(h, _ptr(x), _ptr(y), stream, bn_mode, _ptr(out_losses), _ptr(out_correct), _ptr(out_pred)))
 
 
 def lp_num_tensors(h) -> int:

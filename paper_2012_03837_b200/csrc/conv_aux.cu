@@ -121,6 +121,13 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const BnFinalProb* __r
   int lane = threadIdx.x & 31;
   int c = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (c >= p.C) return;
+  if (!BWD && p.use_running) {                 // evaluation mode: normalise with the running statistics
+    if (lane == 0) {
+      p.mean[c] = p.run_mean[c];
+      p.rstd[c] = (float)(1.0 / sqrt((double)p.run_var[c] + (double)p.eps));
+    }
+    return;
+  }
   double a = 0.0, b = 0.0;
   for (int k = lane; k < p.nblk; k += 32) {
     a += (double)p.part[(size_t)k * 2 * p.C + c];
@@ -141,6 +148,11 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const BnFinalProb* __r
     if (var < 0.0) var = 0.0;
     p.mean[c] = (float)mu;
     p.rstd[c] = (float)(1.0 / sqrt(var + (double)p.eps));
+    if (p.run_mean && !(p.chunk_tab && p.chunk_tab[p.chunk].x == 0.f)) {   // training step: exponential averages
+      const double m = (double)p.momentum, unb = var * ((double)p.rows / (double)(p.rows > 1 ? p.rows - 1 : 1));
+      p.run_mean[c] = (float)((1.0 - m) * (double)p.run_mean[c] + m * mu);
+      p.run_var[c] = (float)((1.0 - m) * (double)p.run_var[c] + m * unb);
+    }
   }
 }
 

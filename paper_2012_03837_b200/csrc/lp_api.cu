@@ -142,7 +142,6 @@ void build_segments(Handle& h) {
   h.d_seg_end = h.upload(ends);
   h.d_seg_chunk = h.upload(chunks);
   h.n_seg = (int)ends.size();
-  h.d_chunk_tab = (float4*)h.dalloc(sizeof(float4) * h.K);
   h.updates.assign(h.K, 0);
 }
 
@@ -158,7 +157,7 @@ bool prepare_chunks(Handle& h, int schedule, cudaStream_t s, std::vector<char>& 
       if (k > h.pipe_steps) { active[k] = 0; any_idle = true; }
   for (int k = 1; k < K; ++k) differ |= h.updates[k] != h.updates[0];
   h.per_chunk_counts = any_idle || differ;
-  if (h.per_chunk_counts) {
+  if (h.per_chunk_counts || h.spec.family == LP_FAMILY_RESNET) {   // BatchNorm reads the active flags every step
     std::vector<float4> tab(K);
     for (int k = 0; k < K; ++k) {
       const double t = (double)(h.updates[k] + 1);
@@ -234,6 +233,7 @@ lp_status lp_create(const lp_model_spec* model, int K, const lp_head_spec* head,
     }
     h.d_losses = (float*)h.dalloc(sizeof(float) * K);
     h.d_status = (int*)h.dalloc(sizeof(int));
+    h.d_chunk_tab = (float4*)h.dalloc(sizeof(float4) * K);
     switch (model->family) {
       case LP_FAMILY_MLP:
         h.layer_widths.assign(model->layer_widths, model->layer_widths + model->n_layers);
@@ -342,12 +342,13 @@ lp_status lp_forward(lp_handle hh, const void* x, const void* y, void* stream, v
   return check_cuda(&h, "lp_forward");
 }
 
-lp_status lp_evaluate(lp_handle hh, const void* x, const void* y, void* stream, float* out_losses, int* out_correct,
-                      int* out_pred) {
+lp_status lp_evaluate(lp_handle hh, const void* x, const void* y, void* stream, int bn_mode, float* out_losses,
+                      int* out_correct, int* out_pred) {
   if (!hh) return LP_ERR_INVALID_ARG;
   Handle& h = hh->h;
   if (!x || !y) return fail(&h, LP_ERR_INVALID_ARG, "null x or y");
   if (!out_losses && !out_correct && !out_pred) return fail(&h, LP_ERR_INVALID_ARG, "no output requested");
+  if (bn_mode != LP_BN_BATCH && bn_mode != LP_BN_RUNNING) return fail(&h, LP_ERR_INVALID_ARG, "bad bn_mode");
   cudaStream_t s = (cudaStream_t)stream;
   lp_status st = copy_inputs(h, x, y, cudaMemcpyDeviceToDevice, s);
   if (st != LP_OK) return st;
@@ -356,7 +357,8 @@ lp_status lp_evaluate(lp_handle hh, const void* x, const void* y, void* stream, 
   ctx.out_pred = out_pred;
   ctx.out_correct = out_correct;
   int half = h.primed ? h.parity ^ 1 : 0;                 // the half no chunk will read next step
-  h.fwd_plan[half].run(ctx);
+  if (bn_mode == LP_BN_RUNNING && h.has_eval_plan) h.eval_plan[half].run(ctx);
+  else h.fwd_plan[half].run(ctx);
   if (out_losses) cudaMemcpyAsync(out_losses, h.d_losses, sizeof(float) * h.K, cudaMemcpyDeviceToDevice, s);
   return check_cuda(&h, "lp_evaluate");
 }

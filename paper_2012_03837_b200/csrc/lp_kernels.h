@@ -176,6 +176,12 @@ void launch_bn_stat_partial(const BnStatProb* d_probs, int n, int max_rows, int 
                             cudaStream_t s, bool vec8 = false);
 struct BnFinalProb {  // fwd: sums -> mean, rstd.  part is [nblk, 2, C]
   const float* part; int nblk; int rows; int C; float* mean; float* rstd; float* dgamma; float* dbeta; float eps;
+  // Running statistics (fwd only, nullable): with use_running == 0 they are moved towards this minibatch's
+  // mean and unbiased variance by `momentum` (training steps); with use_running == 1 nothing is summed and
+  // mean / rstd are taken from them (evaluation mode).
+  float* run_mean; float* run_var; float momentum; int use_running;
+  // the update of the running statistics is skipped while the chunk idles (chunk_tab[chunk].x == 0; see OptimArgs)
+  const float4* chunk_tab; int chunk;
 };
 void launch_bn_finalize(const BnFinalProb* d_probs, int n, int max_c, bool bwd, cudaStream_t s);
 struct BnApplyProb {

@@ -129,6 +129,19 @@ void build_resnet(Handle& h) {
     h.add_tensor(ck + ".head.W", k, {NC, cout}, true);
     h.add_tensor(ck + ".head.b", k, {NC}, false);
   }
+  // running mean / variance of every BatchNorm: state no gradient reaches (their gradient entries stay
+  // zero, so the optimizer sweep leaves them alone); they live in the arena so that tensor access and
+  // checkpoints cover them
+  {
+    std::vector<std::pair<std::string, std::pair<int, int64_t>>> bns;
+    for (auto& t : h.tensors)
+      if (t.name.size() > 2 && t.name.compare(t.name.size() - 2, 2, ".g") == 0 && t.name.find(".bn") != std::string::npos)
+        bns.push_back({t.name.substr(0, t.name.size() - 2), {t.chunk, t.numel}});
+    for (auto& b : bns) {
+      h.add_tensor(b.first + ".rm", b.second.first, {b.second.second}, false);
+      h.add_tensor(b.first + ".rv", b.second.first, {b.second.second}, false);
+    }
+  }
   h.finalize_arena();
   h.rows = B;
 
@@ -216,11 +229,20 @@ void build_resnet(Handle& h) {
     g.a_ms = c.ldk;
     emit_gemm(h, p, {g});
   };
-  auto bn_fwd = [&](Plan& p, const Bn& b, const void* x, void* y, const void* res, bool relu) {
+  // BatchNorm modes of a forward pass: batch statistics only (priming, lp_forward), batch statistics that
+  // also move the running averages (training steps), running statistics (evaluation)
+  enum { BN_BATCH = 0, BN_TRAIN = 1, BN_RUNNING = 2 };
+  auto bn_fwd = [&](Plan& p, const Bn& b, const void* x, void* y, const void* res, bool relu, int mode) {
     int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
-    float* part = fal((size_t)nblk * 2 * b.C);
+    float* part = mode == BN_RUNNING ? nullptr : fal((size_t)nblk * 2 * b.C);
+    float *rm = nullptr, *rv = nullptr;
+    if (mode != BN_BATCH) {
+      const std::string stem = b.g.substr(0, b.g.size() - 2);      // "...bn.g" -> "...bn"
+      rm = h.P32(stem + ".rm"); rv = h.P32(stem + ".rv");
+    }
     BnStatProb sp{x, nullptr, nullptr, nullptr, nullptr, part, (int)b.rows, b.C};
-    BnFinalProb fp{part, nblk, (int)b.rows, b.C, b.mean, b.rstd, nullptr, nullptr, 1e-5f};
+    BnFinalProb fp{part, nblk, (int)b.rows, b.C, b.mean, b.rstd, nullptr, nullptr, 1e-5f, rm, rv, 0.1f, mode == BN_RUNNING ? 1 : 0,
+                   mode == BN_TRAIN ? h.d_chunk_tab : nullptr, h.tensors[h.find(b.g)].chunk};
     BnApplyProb ap{x, y, res, h.P32(b.g), h.P32(b.b), b.mean, b.rstd, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
                    (int)b.rows, b.C, relu ? 1 : 0};
     const BnStatProb* ds = h.upload(std::vector<BnStatProb>{sp});
@@ -229,11 +251,12 @@ void build_resnet(Handle& h) {
     int rows = (int)b.rows, C = b.C;
     bool v8 = bf && C % 8 == 0 && C / 8 <= 256;
     long long elems = b.rows * b.C;
-    p.add(3, [=](const RunCtx& r) {
-      launch_bn_stat_partial(ds, 1, rows, C, false, bf, r.stream, v8);
+    const bool stats = mode != BN_RUNNING;
+    p.add(stats ? 3 : 2, [=](const RunCtx& r) {
+      if (stats) launch_bn_stat_partial(ds, 1, rows, C, false, bf, r.stream, v8);
       launch_bn_finalize(df, 1, C, false, r.stream);
       launch_bn_apply(da, 1, elems, false, bf, r.stream, v8);
-    }, KIND_NORM, (double)elems * es * (3 + (res ? 1 : 0)));
+    }, KIND_NORM, (double)elems * es * ((stats ? 3 : 2) + (res ? 1 : 0)));
   };
 
   auto chunk_in = [&](int k, int rd) -> const void* { return k == 0 ? ch[0].stem_out : h.bnd[rd][k - 1]; };
@@ -241,28 +264,28 @@ void build_resnet(Handle& h) {
     return (!pipelined || k == 0) ? h.y_in : h.lab[rd][k - 1];
   };
 
-  auto forward_chunk = [&](Plan& p, int k, int rd, int wr) {
+  auto forward_chunk = [&](Plan& p, int k, int rd, int wr, int mode) {
     Chunk& c = ch[k];
     if (c.has_stem) {
       LayoutProb lp{h.x_in, c.x_nhwc, B, h.spec.in_channels, h.spec.height, h.spec.width};
       p.add(1, [=](const RunCtx& r) { launch_nchw_to_nhwc(lp, bf, r.stream); }, KIND_CONV_AUX, 2.0 * in_elems * es);
       conv_fwd(p, c.stem, c.x_nhwc);
-      bn_fwd(p, c.stem_bn, c.stem.y, c.stem_out, nullptr, true);
+      bn_fwd(p, c.stem_bn, c.stem.y, c.stem_out, nullptr, true, mode);
     }
     const void* x = chunk_in(k, rd);
     for (size_t j = 0; j < c.blocks.size(); ++j) {
       Block& b = c.blocks[j];
       void* out = b.out ? b.out : h.bnd[wr][k];
       conv_fwd(p, b.c1, x);
-      bn_fwd(p, b.b1, b.c1.y, b.a1, nullptr, true);
+      bn_fwd(p, b.b1, b.c1.y, b.a1, nullptr, true, mode);
       conv_fwd(p, b.c2, b.a1);
       const void* res = x;
       if (b.has_sc) {
         conv_fwd(p, b.cs, x);
-        bn_fwd(p, b.bs, b.cs.y, b.sc, nullptr, false);
+        bn_fwd(p, b.bs, b.cs.y, b.sc, nullptr, false, mode);
         res = b.sc;
       }
-      bn_fwd(p, b.b2, b.c2.y, out, res, true);
+      bn_fwd(p, b.b2, b.c2.y, out, res, true, mode);
       x = out;
     }
   };
@@ -332,7 +355,7 @@ void build_resnet(Handle& h) {
     float* part = fal((size_t)nblk * 2 * b.C);
     Op o; o.kind = OP_BN_BWD;
     o.bn_stat = BnStatProb{x, dy, b.mean, b.rstd, relu_out, part, (int)b.rows, b.C};
-    o.bn_final = BnFinalProb{part, nblk, (int)b.rows, b.C, nullptr, nullptr, h.G(b.g), h.G(b.b), 1e-5f};
+    o.bn_final = BnFinalProb{part, nblk, (int)b.rows, b.C, nullptr, nullptr, h.G(b.g), h.G(b.b), 1e-5f, nullptr, nullptr, 0.f, 0, nullptr, 0};
     o.bn_apply = BnApplyProb{x, nullptr, nullptr, h.P32(b.g), h.P32(b.b), b.mean, b.rstd, dy, relu_out, dx, dres, h.G(b.g), h.G(b.b),
                              (int)b.rows, b.C, 0};
     o.v8 = bf && b.C % 8 == 0 && b.C / 8 <= 256;
@@ -480,7 +503,7 @@ void build_resnet(Handle& h) {
     for (int k = 0; k < K; ++k)
       lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, B, NC, h.n_valid[k]});
     emit_labels(h, p, lps);
-    for (int k = 0; k < K; ++k) forward_chunk(p, k, rd, wr);
+    for (int k = 0; k < K; ++k) forward_chunk(p, k, rd, wr, BN_TRAIN);
     for (int k = 0; k < K; ++k) head_forward(p, k, wr, labels_of(k, pipelined, rd), false);
     std::vector<OpList> lists(K);
     for (int k = 0; k < K; ++k) record_backward(lists[k], k, rd, wr);
@@ -488,8 +511,8 @@ void build_resnet(Handle& h) {
     emit_pending_reduce(h, p);
     emit_optimizer(h, p);
   };
-  auto build_forward = [&](Plan& p, int wr, bool heads) {
-    for (int k = 0; k < K; ++k) forward_chunk(p, k, wr, wr);
+  auto build_forward = [&](Plan& p, int wr, bool heads, int mode) {
+    for (int k = 0; k < K; ++k) forward_chunk(p, k, wr, wr, mode);
     if (!heads) return;
     std::vector<LabelProb> lps;
     for (int k = 0; k < K; ++k) lps.push_back(LabelProb{h.y_in, nullptr, B, NC, h.n_valid[k]});
@@ -497,14 +520,16 @@ void build_resnet(Handle& h) {
     for (int k = 0; k < K; ++k) head_forward(p, k, wr, h.y_in, true);
   };
 
+  h.has_eval_plan = true;
   build_step(h.sync_plan, false, 0, 0);
   for (int par = 0; par < 2; ++par) {
     build_step(h.pipe_plan[par], true, par, 1 - par);
-    build_forward(h.prime_plan[par], par, false);
+    build_forward(h.prime_plan[par], par, false, BN_BATCH);
     std::vector<LabelProb> lps;
     for (int k = 0; k + 1 < K; ++k) lps.push_back(LabelProb{h.y_in, h.lab[par][k], B, NC, h.n_valid[k]});
     if (!lps.empty()) emit_labels(h, h.prime_plan[par], lps);
-    build_forward(h.fwd_plan[par], par, true);
+    build_forward(h.fwd_plan[par], par, true, BN_BATCH);
+    build_forward(h.eval_plan[par], par, true, BN_RUNNING);
   }
 }
 

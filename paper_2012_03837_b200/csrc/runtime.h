@@ -98,6 +98,8 @@ struct Handle {
   std::vector<int*> n_valid;
   // ---- plans
   Plan sync_plan, pipe_plan[2], prime_plan[2], fwd_plan[2];
+  Plan eval_plan[2];                           // RESNET: forward with BatchNorm on its running statistics
+  bool has_eval_plan = false;
   std::vector<ColReduceProb> pending_reduce;   // collected while a plan is being built
   int parity = 0;
   bool primed = false;

@@ -92,13 +92,14 @@ class GpuModel:
         return logits.float().cpu().numpy(), self.losses.cpu().numpy().astype(np.float64)
 
 
-def gpu_evaluate(gm: GpuModel, x, y):
+def gpu_evaluate(gm: GpuModel, x, y, bn: str = "batch"):
     """lp_evaluate on (x, y): (losses [K], correct [K], predictions [K, rows])."""
     xt, yt = gm.device_batch(x, y)
     rows = lp_synth.units_per_step(gm.cfg)
     correct = torch.full((gm.K,), -1, dtype=torch.int32, device=gm.dev)
     pred = torch.full((gm.K, rows), -1, dtype=torch.int32, device=gm.dev)
-    lp.lp_evaluate(gm.h, xt, yt, gm.stream, gm.losses, correct, pred)
+    lp.lp_evaluate(gm.h, xt, yt, gm.stream, gm.losses, correct, pred,
+                   lp.LP_BN_RUNNING if bn == "running" else lp.LP_BN_BATCH)
     torch.cuda.synchronize()
     lp.lp_status_poll(gm.h, gm.stream)
     return gm.losses.cpu().numpy().astype(np.float64), correct.cpu().numpy(), pred.cpu().numpy()

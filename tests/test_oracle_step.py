@@ -130,6 +130,8 @@ def test_single_chunk_equals_backprop(fam):
     tloss, tg = torch_backprop_grads(cfg, params, x, y, 0)
     assert abs(loss - tloss) < 1e-10 * max(1, abs(tloss))
     for n in params:
+        if n in orc.buffers:               # running statistics: no gradient reaches them
+            continue
         assert tg[n] is not None, n
         assert rel(grads[n], tg[n]) < 1e-9, n
 
@@ -147,6 +149,8 @@ def test_last_chunk_gradients_are_backprop_gradients(fam):
     orc.step(x, y, "sync")
     _, tg = torch_backprop_grads(cfg, params, x, y, K - 1)
     for n in orc.names_of_chunk[K - 1]:
+        if n in orc.buffers:
+            continue
         assert rel(orc.last_grads[n], tg[n]) < 1e-9, n
     # ... and an earlier chunk's local gradient is NOT the gradient of the last loss (Sec. 1)
     n0 = orc.names_of_chunk[0][0]
@@ -167,6 +171,8 @@ def test_local_gradients_match_finite_differences(fam):
     for k in range(K):
         loss, h, grads = orc.local_grads(k, inp, y)
         for n in orc.names_of_chunk[k]:
+            if n in orc.buffers:               # running statistics do not enter the training loss
+                continue
             w = orc.p[n]
             flat = w.reshape(-1)
             for idx in rng.choice(flat.size, size=min(4, flat.size), replace=False):
@@ -201,7 +207,8 @@ def test_chunk_update_ignores_other_chunks_heads_and_losses(fam):
         b.step(x, y, "sync")
         for n in a.names_of_chunk[k]:
             assert np.array_equal(a.p[n], b.p[n]), n
-            assert np.array_equal(a.last_grads[n], b.last_grads[n]), n
+            if n not in a.buffers:
+                assert np.array_equal(a.last_grads[n], b.last_grads[n]), n
 
 
 def test_stop_gradient_is_real():
@@ -346,3 +353,62 @@ def test_evaluate_counts_follow_the_logits_and_ties_take_the_lowest_index():
         assert r["correct"] == sum(int(p == t) for p, t in zip(r["pred"], lab) if t >= 0)
     assert np.all(ev[1]["pred"] == 0)
     assert ev[1]["correct"] == int(np.sum(lab == 0))
+
+
+def test_batchnorm_running_statistics_and_evaluation_mode_follow_the_library_routine():
+    """BatchNorm's running mean / variance after training steps, and the evaluation-mode forward that uses
+    them, against torch.nn.functional.batch_norm (momentum 0.1, unbiased variance in the running average);
+    plus the closed form after one step from (0, 1): 0.1 * batch mean and 0.9 + 0.1 * n/(n-1) * batch variance."""
+    cfg = lp_synth.config("c4", dtype="fp32", batch=4, height=6, width=6, stem_channels=4, stage_channels=[4, 8],
+                          blocks_per_stage=1, classes=3)
+    params = spread_params(cfg)
+    for n in params:                       # the running statistics start from (0, 1)
+        if n.endswith(".rm"):
+            params[n] = np.zeros_like(params[n])
+        if n.endswith(".rv"):
+            params[n] = np.ones_like(params[n])
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    P = {n: torch.tensor(a, dtype=torch.float64) for n, a in params.items()}
+    orc.cfg = dict(cfg, optim=dict(kind="sgdm", lr=0.0, momentum=0.0, weight_decay=0.0))   # weights stay put
+    x0, y0 = lp_synth.minibatch(cfg, 0)
+    # closed form for the stem after one step
+    u = F.conv2d(torch.tensor(x0, dtype=torch.float64), P["c0.stem.conv"], padding=1).numpy()
+    n = u.shape[0] * u.shape[2] * u.shape[3]
+    orc.step(x0, y0, "sync")
+    assert np.allclose(orc.p["c0.stem.bn.rm"], 0.1 * u.mean(axis=(0, 2, 3)), rtol=1e-12, atol=1e-14)
+    assert np.allclose(orc.p["c0.stem.bn.rv"], 0.9 + 0.1 * u.var(axis=(0, 2, 3)) * n / (n - 1), rtol=1e-12)
+    # two more steps, then every BatchNorm against the library's running buffers
+    for t in (1, 2):
+        orc.step(*lp_synth.minibatch(cfg, t), "sync")
+    rm = {m[:-3]: torch.zeros(params[m].shape, dtype=torch.float64) for m in params if m.endswith(".rm")}
+    rv = {m: torch.ones_like(v) for m, v in rm.items()}
+
+    def torch_pass(xt, training):
+        bn = lambda v, m: F.batch_norm(v, rm[m], rv[m], P[m + ".g"], P[m + ".b"], training, 0.1, 1e-5)
+        h = F.relu(bn(F.conv2d(xt, P["c0.stem.conv"], padding=1), "c0.stem.bn"))
+        outs = []
+        for k in range(2):
+            nm = f"c{k}.r0"
+            s = lp_synth.resnet_stage_stride(cfg, k)
+            v = F.relu(bn(F.conv2d(h, P[nm + ".conv1"], stride=s, padding=1), nm + ".bn1"))
+            v = bn(F.conv2d(v, P[nm + ".conv2"], padding=1), nm + ".bn2")
+            sc = bn(F.conv2d(h, P[nm + ".sc.conv"], stride=s), nm + ".sc.bn") if nm + ".sc.conv" in P else h
+            h = F.relu(v + sc)
+            outs.append(h)
+        return outs
+    for t in range(3):
+        torch_pass(torch.tensor(lp_synth.minibatch(cfg, t)[0], dtype=torch.float64), True)
+    for m in rm:
+        assert rel(orc.p[m + ".rm"], rm[m].numpy()) < 1e-10, m
+        assert rel(orc.p[m + ".rv"], rv[m].numpy()) < 1e-10, m
+    # evaluation mode: losses from the running statistics, and nothing moves
+    x3, y3 = lp_synth.minibatch(cfg, 3)
+    before = {m: orc.p[m + ".rm"].copy() for m in rm}
+    ev = orc.evaluate(x3, y3, bn="running")
+    outs = torch_pass(torch.tensor(x3, dtype=torch.float64), False)
+    for k in range(2):
+        tl = float(torch_head_loss(cfg, P, k, outs[k], torch.tensor(y3)))
+        assert abs(ev[k]["loss"] - tl) < 1e-10 * max(1.0, abs(tl)), k
+    for m in rm:
+        assert np.array_equal(before[m], orc.p[m + ".rm"])
+    assert abs(orc.evaluate(x3, y3)[0]["loss"] - ev[0]["loss"]) > 1e-6      # batch statistics give another loss
