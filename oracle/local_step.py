@@ -21,6 +21,13 @@ Schedules:
     that step equals a synchronous step; `ramp="idle"` instead leaves chunk k idle (no update,
     loss NaN) until real data reaches it at step k.
 
+Overlapping local parallelism (Sec. 3; cost model in App. A.2): with overlap=True the block trained by
+chunk k's loss also contains the last layer of chunk k-1 (for the transformer: its last block), so that
+loss is back-propagated one layer past the chunk boundary and stops at that layer's input.  The
+shared layer exists once (one forward pass through the network); it receives two gradients, from
+its own chunk's loss and from the next chunk's, and is updated with their average.  Defined for
+the synchronous schedule (both gradients belong to the same minibatch).
+
 Readings the paper leaves open are fixed here: mean loss over valid rows; LM targets are the ids
 shifted left with the last position ignored; LayerNorm/BatchNorm eps 1e-5; exact (erf) GELU; no
 dropout; pre-LayerNorm residual blocks; ResNet shortcut = 1x1 stride-2 convolution + BatchNorm
@@ -36,7 +43,7 @@ from . import optim as O
 
 
 class LocalUpdateOracle:
-    def __init__(self, cfg: dict, params: dict, dtype=np.float32, ramp: str = "prime"):
+    def __init__(self, cfg: dict, params: dict, dtype=np.float32, ramp: str = "prime", overlap: bool = False):
         self.cfg = cfg
         self.dtype = np.dtype(dtype).type
         self.K = lp_synth.num_chunks(cfg)
@@ -49,6 +56,7 @@ class LocalUpdateOracle:
         self.bn_mode = "batch"   # "running": BatchNorm normalises with its running statistics (evaluation)
         self.training = False    # True inside a training step: BatchNorm then updates its running statistics
         self.ramp = ramp
+        self.overlap = overlap   # overlapping local parallelism (Sec. 3, Fig. 2 c): synchronous schedule only
         self.buf = None          # pipelined: buf[k] = (activation, labels) chunk k+1 reads next
         self.t = 0               # pipelined steps taken since the last reset
         self.last_grads = {}
@@ -113,6 +121,7 @@ class LocalUpdateOracle:
             c1, c2 = caches[i]
             du = L.relu_bwd(dx, c2)
             dx, g[f"c{k}.l{i}.W"], g[f"c{k}.l{i}.b"] = L.linear_bwd(du, c1)
+        self._dx_in = dx         # gradient at the chunk input: used only by the overlapping variant
         return g
 
     # LM chunk: (token + position embedding in chunk 0), then pre-LayerNorm transformer blocks
@@ -144,20 +153,27 @@ class LocalUpdateOracle:
             cache["blocks"].append((n, cl1, cq, ca, co, cl2, c1, cg, c2))
         return h, cache
 
+    def _lm_block_bwd(self, dh, block_cache, g):
+        """Backward of one transformer block: fills g with its parameter gradients, returns the gradient
+        at the block input."""
+        (n, cl1, cq, ca, co, cl2, c1, cg, c2) = block_cache
+        b, t, d = dh.shape
+        dgl, g[n + ".W2"], g[n + ".b2"] = L.linear_bwd(dh.reshape(b * t, d), c2)
+        du = L.gelu_bwd(dgl, cg)
+        da2, g[n + ".W1"], g[n + ".b1"] = L.linear_bwd(du, c1)
+        dx, g[n + ".ln2.g"], g[n + ".ln2.b"] = L.layernorm_bwd(da2.reshape(b, t, d), cl2)
+        dh = dh + dx
+        do, g[n + ".Wo"], g[n + ".bo"] = L.linear_bwd(dh.reshape(b * t, d), co)
+        dqkv = L.attention_bwd(do.reshape(b, t, d), ca)
+        da1, g[n + ".Wqkv"], g[n + ".bqkv"] = L.linear_bwd(dqkv.reshape(b * t, 3 * d), cq)
+        dx, g[n + ".ln1.g"], g[n + ".ln1.b"] = L.layernorm_bwd(da1.reshape(b, t, d), cl1)
+        return dh + dx
+
     def _lm_bwd(self, k, dh, cache):
         g = {}
-        b, t, d = dh.shape
-        for (n, cl1, cq, ca, co, cl2, c1, cg, c2) in reversed(cache["blocks"]):
-            dgl, g[n + ".W2"], g[n + ".b2"] = L.linear_bwd(dh.reshape(b * t, d), c2)
-            du = L.gelu_bwd(dgl, cg)
-            da2, g[n + ".W1"], g[n + ".b1"] = L.linear_bwd(du, c1)
-            dx, g[n + ".ln2.g"], g[n + ".ln2.b"] = L.layernorm_bwd(da2.reshape(b, t, d), cl2)
-            dh = dh + dx
-            do, g[n + ".Wo"], g[n + ".bo"] = L.linear_bwd(dh.reshape(b * t, d), co)
-            dqkv = L.attention_bwd(do.reshape(b, t, d), ca)
-            da1, g[n + ".Wqkv"], g[n + ".bqkv"] = L.linear_bwd(dqkv.reshape(b * t, 3 * d), cq)
-            dx, g[n + ".ln1.g"], g[n + ".ln1.b"] = L.layernorm_bwd(da1.reshape(b, t, d), cl1)
-            dh = dh + dx
+        for block_cache in reversed(cache["blocks"]):
+            dh = self._lm_block_bwd(dh, block_cache, g)
+        self._dx_in = dh         # gradient at the chunk input: used only by the overlapping variant
         if k == 0:
             g["c0.tok"], g["c0.pos"] = L.embedding_bwd(dh, cache["emb"])
         return g
@@ -240,7 +256,25 @@ class LocalUpdateOracle:
             self.training = False
         loss, _, dh, g = self.head(k, h, y)
         g.update(self.chunk_backward(k, dh, cache))
+        self._last_cache = cache
         return loss, h, g
+
+    def overlap_grads(self, k_prev, dx, cache_prev):
+        """Overlapping local parallelism (Sec. 3): the gradient of the NEXT chunk's loss with respect to
+        the parameters of the last layer of chunk k_prev (its last Linear+ReLU, or its last transformer
+        block), given that loss's gradient dx at chunk k_prev's output; truncated at that layer's input."""
+        fam = self.cfg["family"]
+        g = {}
+        if fam == "mlp":
+            c1, c2 = cache_prev[-1]
+            i = len(cache_prev) - 1
+            du = L.relu_bwd(dx, c2)
+            _, g[f"c{k_prev}.l{i}.W"], g[f"c{k_prev}.l{i}.b"] = L.linear_bwd(du, c1)
+        elif fam == "lm":
+            self._lm_block_bwd(dx, cache_prev["blocks"][-1], g)
+        else:
+            raise NotImplementedError("overlapping updates: MLP and LM families")
+        return g
 
     def apply_update(self, k, grads):
         """Optimizer update of chunk k's trunk and head from its own gradients only."""
@@ -266,10 +300,18 @@ class LocalUpdateOracle:
         x = self._cast_input(x)
         losses = np.full(K, np.nan, dtype=np.float64)
         all_grads = [None] * K
+        if self.overlap and schedule != "sync":
+            raise ValueError("overlapping updates are defined for the synchronous schedule")
         if schedule == "sync":
-            inp, outs = x, []
+            inp, prev_cache = x, None
             for k in range(K):
                 losses[k], h, all_grads[k] = self.local_grads(k, inp, y)
+                if self.overlap and k > 0:
+                    # chunk k's loss reaches one layer further back; that layer's update is the average of
+                    # its two gradients (App. A.2: "an additional average of gradients")
+                    for n, g2 in self.overlap_grads(k - 1, self._dx_in, prev_cache).items():
+                        all_grads[k - 1][n] = ((all_grads[k - 1][n] + g2) * 0.5).astype(g2.dtype)
+                prev_cache = self._last_cache
                 inp = h                      # handed on as a constant: no gradient flows back
         else:
             if self.buf is None:

@@ -412,3 +412,50 @@ def test_batchnorm_running_statistics_and_evaluation_mode_follow_the_library_rou
     for m in rm:
         assert np.array_equal(before[m], orc.p[m + ".rm"])
     assert abs(orc.evaluate(x3, y3)[0]["loss"] - ev[0]["loss"]) > 1e-6      # batch statistics give another loss
+
+
+# ---------------------------------------------------------------- overlapping local parallelism (Sec. 3, Fig. 2 c)
+
+@pytest.mark.parametrize("fam", ["mlp", "lm"])
+def test_overlapping_updates_average_the_two_backprop_gradients_of_the_shared_layer(fam):
+    """With overlap, the last layer (transformer: last block) of every chunk but the final one also belongs to
+    the next chunk's block.  Its gradient from either loss is that loss's ordinary back-propagation gradient
+    (truncating further down does not change it), so the update must use the mean of two torch autograd
+    gradients; every other parameter keeps its plain local gradient."""
+    cfg = TINY[fam]
+    K = lp_synth.num_chunks(cfg)
+    params = spread_params(cfg, seed=3)
+    x, y = lp_synth.minibatch(cfg, 0)
+    lr = 0.25
+    sgd = dict(kind="sgdm", lr=lr, momentum=0.0, weight_decay=0.0)
+    plain = LocalUpdateOracle(dict(cfg, optim=sgd), params, dtype=np.float64)
+    over = LocalUpdateOracle(dict(cfg, optim=sgd), params, dtype=np.float64, overlap=True)
+    lp_, lo = plain.step(x, y, "sync"), over.step(x, y, "sync")
+    assert np.array_equal(lp_, lo)                      # the forward pass is shared: same losses
+    tg = [torch_backprop_grads(cfg, params, x, y, k)[1] for k in range(K)]
+    shared = set()
+    for k in range(K - 1):
+        if fam == "mlp":
+            last = len(cfg["chunks"][k]) - 1
+            names = [f"c{k}.l{last}.W", f"c{k}.l{last}.b"]
+        else:
+            blk = over._lm_block_names(k)[-1]
+            names = [n for n in over.names_of_chunk[k] if n.startswith(blk + ".")]
+            assert len(names) == 12
+        for n in names:
+            shared.add(n)
+            want = 0.5 * (tg[k][n] + tg[k + 1][n])
+            assert rel(over.last_grads[n], want) < 1e-9, n
+            assert rel(over.last_grads[n], plain.last_grads[n]) > 1e-4, n      # and it is not the greedy gradient
+            assert rel(over.p[n], params[n] - lr * want) < 1e-12, n             # the update applies the average
+    for n in params:
+        if n not in shared:
+            assert np.array_equal(over.last_grads[n], plain.last_grads[n]), n
+            assert np.array_equal(over.p[n], plain.p[n]), n
+
+
+def test_overlapping_updates_need_the_synchronous_schedule():
+    cfg = TINY["mlp"]
+    over = LocalUpdateOracle(cfg, lp_synth.init_params(cfg), dtype=np.float64, overlap=True)
+    with pytest.raises(ValueError):
+        over.step(*lp_synth.minibatch(cfg, 0), "pipelined")
