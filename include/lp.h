@@ -211,6 +211,17 @@ lp_status lp_reset_pipeline(lp_handle h);
 enum { LP_RAMP_PRIME = 0, LP_RAMP_IDLE = 1 };
 lp_status lp_set_ramp(lp_handle h, int ramp);
 
+/*
+ * lp_set_overlap: overlapping local parallelism (Sec. 3, Fig. 2 c; cost in App. A.2).  With on != 0 the
+ * block trained by chunk k's loss also contains the last layer of chunk k-1: that loss is propagated one
+ * layer past the chunk boundary and stops at that layer's input.  The shared layer exists once (one forward
+ * pass); it receives a gradient from its own chunk's loss and one from the next chunk's, and its update
+ * uses their mean.  All other parameters are updated as without overlap.  LP_GRAD of a shared layer then
+ * holds the mean.  Synchronous steps only (a pipelined lp_step returns LP_ERR_UNSUPPORTED while overlap is
+ * on).  Built for the MLP family with K >= 2; otherwise LP_ERR_UNSUPPORTED.
+ */
+lp_status lp_set_overlap(lp_handle h, int on);
+
 /* Read the device status word (synchronises `stream`): LP_OK, or LABEL_RANGE / NONFINITE /
  * TIMEOUT if any kernel since the last poll flagged it.  The word is cleared. */
 lp_status lp_status_poll(lp_handle h, void* stream);

@@ -60,7 +60,7 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
-           "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate"]
+           "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
 
@@ -81,6 +81,7 @@ def load_library() -> C.CDLL:
     lib.lp_set_tensor.argtypes = [vp, ip, ip, vp, C.c_size_t, vp]
     lib.lp_reset_pipeline.argtypes = [vp]
     lib.lp_set_ramp.argtypes = [vp, ip]
+    lib.lp_set_overlap.argtypes = [vp, ip]
     lib.lp_status_poll.argtypes = [vp, vp]
     lib.lp_state_size.argtypes = [vp]
     lib.lp_state_size.restype = C.c_size_t
@@ -222,6 +223,10 @@ LP_RAMP_PRIME, LP_RAMP_IDLE = 0, 1
 
 def lp_set_ramp(h, ramp: int):
     _check(h, _lib.lp_set_ramp(h, ramp))
+
+
+def lp_set_overlap(h, on: bool):
+    _check(h, _lib.lp_set_overlap(h, 1 if on else 0))
 
 
 def lp_status_poll(h, stream=None):

@@ -177,8 +177,9 @@ lp_status run_step(Handle& h, int schedule, cudaStream_t s) {
   const bool any_idle = prepare_chunks(h, schedule, s, active);
   if (schedule == LP_SYNC) {
     if (h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
-    h.sync_plan.run(ctx);
-    launches = h.sync_plan.launches;
+    const Plan& plan = h.overlap ? h.sync_overlap_plan : h.sync_plan;
+    plan.run(ctx);
+    launches = plan.launches;
   } else {
     if (!h.primed && h.ramp == LP_RAMP_PRIME) {
       h.prime_plan[h.parity].run(ctx);
@@ -299,6 +300,7 @@ lp_status lp_step(lp_handle hh, const void* x, const void* y, int schedule, void
   if (!x || !y || !out_losses) return fail(&h, LP_ERR_INVALID_ARG, "null pointer");
   if (schedule != LP_SYNC && schedule != LP_PIPELINED) return fail(&h, LP_ERR_INVALID_ARG, "bad schedule");
   if (schedule == LP_SYNC && h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
+  if (schedule == LP_PIPELINED && h.overlap) return fail(&h, LP_ERR_UNSUPPORTED, "overlapping updates take both gradients of a shared layer from one minibatch: synchronous schedule only");
   cudaStream_t s = (cudaStream_t)stream;
   lp_status st = copy_inputs(h, x, y, cudaMemcpyDeviceToDevice, s);
   if (st != LP_OK) return st;
@@ -315,6 +317,7 @@ lp_status lp_step_host(lp_handle hh, const void* x_host, const void* y_host, int
   if (!x_host || !y_host || !out_losses_host) return fail(&h, LP_ERR_INVALID_ARG, "null pointer");
   if (schedule != LP_SYNC && schedule != LP_PIPELINED) return fail(&h, LP_ERR_INVALID_ARG, "bad schedule");
   if (schedule == LP_SYNC && h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
+  if (schedule == LP_PIPELINED && h.overlap) return fail(&h, LP_ERR_UNSUPPORTED, "overlapping updates take both gradients of a shared layer from one minibatch: synchronous schedule only");
   cudaStream_t s = (cudaStream_t)stream;
   lp_status st = copy_inputs(h, x_host, y_host, cudaMemcpyHostToDevice, s);
   if (st != LP_OK) return st;
@@ -392,6 +395,15 @@ lp_status lp_reset_pipeline(lp_handle hh) {
   hh->h.primed = false;
   hh->h.parity = 0;
   hh->h.pipe_steps = 0;
+  return LP_OK;
+}
+
+lp_status lp_set_overlap(lp_handle hh, int on) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (on && !h.has_overlap_plan)
+    return fail(&h, LP_ERR_UNSUPPORTED, "overlapping updates are built for the MLP family with at least two chunks");
+  h.overlap = on != 0;
   return LP_OK;
 }
 

@@ -211,6 +211,9 @@ void launch_gap_fwd(const GapProb* d_probs, int n, int max_n, int max_c, bool is
 void launch_gap_bwd(const GapProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
 
 struct AddProb { const void* a; const void* b; void* out; long long n; };
+// a[i] = (a[i] + b[i]) / 2 in fp32: the averaged gradient of a layer shared by two overlapping blocks (App. A.2)
+struct AvgProb { float* a; const float* b; long long n; };
+void launch_average_f32(const AvgProb* d_probs, int n, long long max_elems, cudaStream_t s);
 void launch_add(const AddProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
 
 // ---------------------------------------------------------------------------- optimizer

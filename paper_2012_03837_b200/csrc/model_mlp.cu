@@ -96,7 +96,11 @@ void build_mlp(Handle& h) {
     return (!pipelined || k == 0) ? h.y_in : h.lab[rd][k - 1];
   };
 
-  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr) {
+  // Overlapping local parallelism (Sec. 3, Fig. 2 c): the block trained by chunk k's loss also holds the last
+  // layer of chunk k-1.  That layer exists once; the loss of chunk k is propagated one layer past the chunk
+  // boundary into a second gradient for it (g2w / g2b), and its update uses the mean of its two gradients.
+  std::vector<float*> g2w(K, nullptr), g2b(K, nullptr);     // second gradient of chunk k's last layer
+  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr, bool overlap) {
     std::vector<LabelProb> lps;
     for (int k = 0; k < K; ++k)
       lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, B, C,
@@ -134,6 +138,7 @@ void build_mlp(Handle& h) {
     // chunk input (Sec. 3: the gradient stops at the chunk boundary)
     size_t maxl = 0;
     for (int k = 0; k < K; ++k) maxl = std::max(maxl, b.widths[k].size());
+    std::vector<void*> du_over(K, nullptr);        // overlap: gradient at the pre-activation of chunk k-1's last layer
     for (size_t j = 0; j < maxl; ++j) {
       std::vector<GemmProb> g;
       std::vector<ColSumProb> cs;
@@ -149,13 +154,45 @@ void build_mlp(Handle& h) {
         int w = b.widths[k][i];
         g.push_back(gemm_wgrad(du, in, h.G(tn(k, i, "W")), B, w, din));
         if (i > 0) g.push_back(gemm_dgrad(du, h.W(tn(k, i, "W")), dnext, B, w, din, EPI_RELU_MASK, b.y[k][i - 1]));
+        else if (overlap && k > 0) {               // one layer past the boundary: through the ReLU of the shared layer
+          g.push_back(gemm_dgrad(du, h.W(tn(k, 0, "W")), dnext, B, w, din, EPI_RELU_MASK, chunk_in(h, k, rd)));
+          du_over[k] = dnext;
+        }
         cs.push_back(ColSumProb{du, nullptr, B, w, w});
         outs.push_back(h.G(tn(k, i, "b")));
       }
       emit_gemm(h, p, g);
       emit_colsum(h, p, cs, outs);
     }
+    std::vector<AvgProb> avg;
+    long long avg_max = 0;
+    if (overlap) {
+      std::vector<GemmProb> g;
+      std::vector<ColSumProb> cs;
+      std::vector<float*> outs;
+      for (int k = 1; k < K; ++k) {
+        const int q = k - 1, nl = (int)b.widths[q].size(), i = nl - 1;     // the shared layer: chunk q's last
+        const int w = b.widths[q][i], din = i == 0 ? b.d_in[q] : b.widths[q][i - 1];
+        const void* in = i == 0 ? chunk_in(h, q, rd) : b.y[q][i - 1];
+        if (!g2w[q]) { g2w[q] = (float*)h.dalloc((size_t)w * din * sizeof(float)); g2b[q] = (float*)h.dalloc((size_t)w * sizeof(float)); }
+        g.push_back(gemm_wgrad(du_over[k], in, g2w[q], B, w, din));
+        cs.push_back(ColSumProb{du_over[k], nullptr, B, w, w});
+        outs.push_back(g2b[q]);
+        avg.push_back(AvgProb{h.G(tn(q, i, "W")), g2w[q], (long long)w * din});
+        avg.push_back(AvgProb{h.G(tn(q, i, "b")), g2b[q], (long long)w});
+        avg_max = std::max(avg_max, (long long)w * din);
+      }
+      emit_gemm(h, p, g);
+      emit_colsum(h, p, cs, outs);
+    }
     emit_pending_reduce(h, p);
+    if (!avg.empty()) {
+      const AvgProb* d = h.upload(avg);
+      int n = (int)avg.size();
+      double bytes = 0;
+      for (auto& a : avg) bytes += 12.0 * a.n;
+      p.add(1, [=](const RunCtx& r) { launch_average_f32(d, n, avg_max, r.stream); }, KIND_REDUCE, bytes);
+    }
     emit_optimizer(h, p);
   };
 
@@ -183,9 +220,13 @@ void build_mlp(Handle& h) {
     emit_xent_and_loss(h, p, xs, all);
   };
 
-  build_step(h.sync_plan, false, 0, 0);
+  build_step(h.sync_plan, false, 0, 0, false);
+  if (K > 1) {
+    build_step(h.sync_overlap_plan, false, 0, 0, true);
+    h.has_overlap_plan = true;
+  }
   for (int par = 0; par < 2; ++par) {
-    build_step(h.pipe_plan[par], true, par, 1 - par);
+    build_step(h.pipe_plan[par], true, par, 1 - par, false);
     // priming: forward chain into the half the first pipelined step will read, labels alongside
     build_forward(h.prime_plan[par], par, false);
     std::vector<LabelProb> lps;

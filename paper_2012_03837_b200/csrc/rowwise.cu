@@ -279,6 +279,12 @@ __global__ void __launch_bounds__(256) argmax_kernel(const ArgmaxProb* __restric
   }
 }
 
+__global__ void __launch_bounds__(256) average_f32_kernel(const AvgProb* __restrict__ probs) {
+  const AvgProb p = probs[blockIdx.y];
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < p.n; i += (long long)gridDim.x * blockDim.x)
+    p.a[i] = (p.a[i] + p.b[i]) * 0.5f;
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) add_kernel(const AddProb* __restrict__ probs) {
   const AddProb p = probs[blockIdx.y];
@@ -325,6 +331,12 @@ void launch_argmax(const ArgmaxProb* d, int n, int max_rows, bool is_bf16, int* 
   if (n < 1 || max_rows < 1) return;
   dim3 grid(max_rows, n);
   DISPATCH_T(is_bf16, argmax_kernel, grid, 256, s, d, pred, pred_stride, correct);
+}
+void launch_average_f32(const AvgProb* d, int n, long long max_elems, cudaStream_t s) {
+  if (n < 1 || max_elems < 1) return;
+  long long blocks = (max_elems + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  average_f32_kernel<<<dim3((unsigned)blocks, n), 256, 0, s>>>(d);
 }
 void launch_add(const AddProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s) {
   long long blocks = (max_elems + 255) / 256;

@@ -18,7 +18,8 @@ def to_abi_layout(name: str, a: np.ndarray) -> np.ndarray:
 
 
 class GpuModel:
-    def __init__(self, cfg: dict, params: dict | None = None, gemm_backend: int = 0, ramp: str = "prime"):
+    def __init__(self, cfg: dict, params: dict | None = None, gemm_backend: int = 0, ramp: str = "prime",
+                 overlap: bool = False):
         self.cfg = cfg
         m, K, hd, op = lp.specs_from_config(cfg, gemm_backend)
         self._specs = (m, hd, op)
@@ -34,6 +35,8 @@ class GpuModel:
         self.set_params(params if params is not None else lp_synth.init_params(cfg))
         if ramp == "idle":
             lp.lp_set_ramp(self.h, lp.LP_RAMP_IDLE)
+        if overlap:
+            lp.lp_set_overlap(self.h, True)
 
     def close(self):
         if self.h:
@@ -110,11 +113,12 @@ def tensor_rel_err(a: np.ndarray, b: np.ndarray) -> float:
     return float(np.abs(a.astype(np.float64) - b.astype(np.float64)).max() / max(np.abs(b).max(), 1e-30))
 
 
-def run_both(cfg: dict, steps: int, gemm_backend: int = 0, params: dict | None = None, ramp: str = "prime"):
+def run_both(cfg: dict, steps: int, gemm_backend: int = 0, params: dict | None = None, ramp: str = "prime",
+             overlap: bool = False):
     """Run `steps` steps on both sides.  Returns (gpu_losses [steps,K], oracle_losses, gpu model, oracle)."""
     params = params if params is not None else lp_synth.init_params(cfg)
-    gm = GpuModel(cfg, params, gemm_backend, ramp)
-    orc = LocalUpdateOracle(cfg, params, dtype=np.float32, ramp=ramp)
+    gm = GpuModel(cfg, params, gemm_backend, ramp, overlap)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float32, ramp=ramp, overlap=overlap)
     gl, ol = [], []
     for t in range(steps):
         x, y = lp_synth.minibatch(cfg, t)

@@ -322,3 +322,61 @@ def test_idle_ramp_up_resnet_bf16():
     fin = ~np.isnan(ol)
     assert np.all(np.abs(gl[fin] - ol[fin]) <= 2e-2 * np.abs(ol[fin]))
     gm.close()
+
+
+# ------------------------------------------------------------------ overlapping local updates (MLP family)
+
+def check_overlap(cfg, gemm_backend=0):
+    """Synchronous steps with overlapping local updates against the oracle's overlap mode: first-step
+    gradients (the shared layers hold the mean of their two gradients), then losses and weights after ten steps."""
+    from paper_2012_03837_b200 import binding as lp
+    dt = cfg["dtype"]
+    gl, ol, gm, orc = T.run_both(cfg, 1, gemm_backend, overlap=True)
+    gg = gm.get(lp.LP_GRAD)
+    errs = sorted(((T.tensor_rel_err(gg[n], orc.last_grads[n]), n) for n in gg), reverse=True)
+    gm.close()
+    plain = T.run_both(cfg, 1, gemm_backend)[3]
+    shared = [n for n in orc.last_grads if not np.array_equal(orc.last_grads[n], plain.last_grads[n])]
+    print("overlap: first-step gradient error (worst)", [(f"{e:.2e}", n) for e, n in errs[:3]], "shared tensors", sorted(shared))
+    assert len(shared) == 2 * (gl.shape[1] - 1)
+    assert errs[0][0] <= G_TOL[dt], errs[:5]
+    gl, ol, gm, orc = T.run_both(cfg, 10, gemm_backend, overlap=True)
+    lerr = np.abs(gl - ol) / np.abs(ol)
+    werr = T.compare_weights(gm, orc, lp_synth.init_params(cfg))
+    gm.close()
+    worst = {kind: max((e, n) for n, (kd, e) in werr.items() if kd == kind) for kind in ("matrix", "vector", "chunk")}
+    print("overlap: loss rel err max", f"{lerr.max():.2e}", "weights worst", {k: (f"{e:.2e}", n) for k, (e, n) in worst.items()})
+    assert lerr.max() <= LOSS_TOL[dt]
+    assert worst["matrix"][0] <= W_TOL[dt] and worst["chunk"][0] <= W_TOL[dt], worst
+    assert worst["vector"][0] <= V_TOL[dt], worst
+
+
+def test_overlapping_updates_mlp_fp32():
+    check_overlap(lp_synth.config("c1"))
+
+
+def test_overlapping_updates_mlp_fp32_ragged_chunks():
+    check_overlap(lp_synth.config("c1", batch=70, d_in=33, chunks=[[65], [40, 50], [31], [24, 16, 40]], classes=7))
+
+
+@pytest.mark.parametrize("backend", [1, 0])
+def test_overlapping_updates_mlp_bf16(backend):
+    cfg = lp_synth.config("c2", batch=192, d_in=160, chunks=[[256, 192], [320, 256], [128, 256]], classes=200,
+                          schedule="sync")
+    check_overlap(cfg, gemm_backend=backend)
+
+
+def test_overlapping_updates_are_refused_where_they_are_not_defined():
+    from paper_2012_03837_b200 import binding as lp
+    gm = T.GpuModel(lp_synth.config("c1"), overlap=True)
+    x, y = lp_synth.minibatch(gm.cfg, 0)
+    with pytest.raises(lp.LpError) as e:
+        gm.step(x, y, "pipelined")
+    assert lp.LP_ERR[e.value.code] == "UNSUPPORTED"
+    gm.close()
+    lm = T.GpuModel(lp_synth.config("c3", batch=2, seq_len=64, vocab=256, d_model=128, n_heads=2, d_ffn=256,
+                                    blocks_per_chunk=[1, 1]))
+    with pytest.raises(lp.LpError) as e:
+        lp.lp_set_overlap(lm.h, True)
+    assert lp.LP_ERR[e.value.code] == "UNSUPPORTED"
+    lm.close()
