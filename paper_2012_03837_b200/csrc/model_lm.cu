@@ -6,6 +6,7 @@
 //                        a2 = LN2(h1); u = a2 W1^T + b; g = GELU(u); h' = h1 + g W2^T + b.
 // Backward is truncated at the chunk input: for the first block of a chunk k > 0 only LN1's scale
 // and shift gradients are formed, not the gradient of the chunk input (Sec. 3).
+#include <map>
 #include <stdexcept>
 
 #include "gemm_tc.h"
@@ -228,7 +229,103 @@ void build_lm(Handle& h) {
     }
   };
 
-  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr) {
+  // Backward of one transformer block for a list of independent (scratch, block) pairs, as grouped launches.
+  // On entry the gradient at the block output is in the scratch G0; parameter gradients go to the arena, or to
+  // `second` (name -> buffer) when that is given; the gradient at the block input is left in G0 if need_dx.
+  struct BwdItem {
+    ChunkBufs* c; BlockBufs* b; const void* blk_in; bool need_dx; std::map<std::string, float*>* second;
+  };
+  auto GR = [&](const BwdItem& it, const std::string& name) -> float* {
+    return it.second ? it.second->at(name) : h.G(name);
+  };
+  auto block_backward = [&](Plan& p, const std::vector<BwdItem>& items) {
+    if (items.empty()) return;
+    std::vector<GemmProb> g;
+    std::vector<ColSumProb> cs;
+    std::vector<float*> outs;
+    // 1. feed-forward second matrix: dW2, db2, du = (dout W2) * gelu'(u)
+    for (auto& it : items) {
+      ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
+      g.push_back(gemm_wgrad(c.G0, b.g, GR(it, b.name + ".W2"), M, d, F));
+      g.push_back(gemm_dgrad(c.G0, h.W(b.name + ".W2"), c.Gf, M, d, F, EPI_GELU_GRAD, b.u));
+      cs.push_back(ColSumProb{c.G0, nullptr, M, d, d});
+      outs.push_back(GR(it, b.name + ".b2"));
+    }
+    emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
+    g.clear(); cs.clear(); outs.clear();
+    // 2. feed-forward first matrix: dW1, db1, da2
+    for (auto& it : items) {
+      ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
+      g.push_back(gemm_wgrad(c.Gf, b.a2, GR(it, b.name + ".W1"), M, F, d));
+      g.push_back(gemm_dgrad(c.Gf, h.W(b.name + ".W1"), c.G1, M, F, d, EPI_NONE, nullptr));
+      cs.push_back(ColSumProb{c.Gf, nullptr, M, F, F});
+      outs.push_back(GR(it, b.name + ".b1"));
+    }
+    emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
+    g.clear(); cs.clear(); outs.clear();
+    // 3. LN2 backward; the residual path adds dout: dh1 -> G2
+    {
+      std::vector<LnBwdProb> lb;
+      std::vector<float*> dgs, dbs;
+      for (auto& it : items) {
+        ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
+        lb.push_back(LnBwdProb{c.G1, b.h1, h.P32(b.name + ".ln2.g"), b.mean2, b.rstd2, c.G2, c.G0, nullptr, M, d});
+        dgs.push_back(GR(it, b.name + ".ln2.g"));
+        dbs.push_back(GR(it, b.name + ".ln2.b"));
+      }
+      emit_ln_bwd(h, p, lb, dgs, dbs);
+    }
+    // 4. attention output projection: dWo, dbo, do -> G1
+    for (auto& it : items) {
+      ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
+      g.push_back(gemm_wgrad(c.G2, b.o, GR(it, b.name + ".Wo"), M, d, d));
+      g.push_back(gemm_dgrad(c.G2, h.W(b.name + ".Wo"), c.G1, M, d, d, EPI_NONE, nullptr));
+      cs.push_back(ColSumProb{c.G2, nullptr, M, d, d});
+      outs.push_back(GR(it, b.name + ".bo"));
+    }
+    emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
+    g.clear(); cs.clear(); outs.clear();
+    // 5. attention backward: dqkv -> Gq
+    {
+      std::vector<AttnProb> at;
+      for (auto& it : items) {
+        ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
+        at.push_back(AttnProb{b.qkv, b.o, b.lse, c.G1, c.Gq, b.delta, B, T, H});
+      }
+      const AttnProb* dp = h.upload(at);
+      int n = (int)at.size();
+      p.add(2, [=](const RunCtx& c) { launch_attn_bwd(dp, n, B, T, H, bf, c.stream); }, KIND_ATTN,
+            (double)n * 10.0 * B * H * 64.0 * T * (T + 1) / 2);
+    }
+    // 6. qkv projection: dWqkv, dbqkv, da1 -> G1 (needed for LN1's own parameters in every case)
+    for (auto& it : items) {
+      ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
+      g.push_back(gemm_wgrad(c.Gq, b.a1, GR(it, b.name + ".Wqkv"), M, 3 * d, d));
+      g.push_back(gemm_dgrad(c.Gq, h.W(b.name + ".Wqkv"), c.G1, M, 3 * d, d, EPI_NONE, nullptr));
+      cs.push_back(ColSumProb{c.Gq, nullptr, M, 3 * d, 3 * d});
+      outs.push_back(GR(it, b.name + ".bqkv"));
+    }
+    emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
+    g.clear(); cs.clear(); outs.clear();
+    // 7. LN1 backward.  The block-input gradient (dh1 + LN1 path -> G0) is formed only if a
+    //    caller asks for it.
+    {
+      std::vector<LnBwdProb> lb;
+      std::vector<float*> dgs, dbs;
+      for (auto& it : items) {
+        ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
+        const bool need_dx = it.need_dx;
+        lb.push_back(LnBwdProb{c.G1, it.blk_in, h.P32(b.name + ".ln1.g"), b.mean1, b.rstd1,
+                               need_dx ? c.G0 : nullptr, need_dx ? c.G2 : nullptr, nullptr, M, d});
+        dgs.push_back(GR(it, b.name + ".ln1.g"));
+        dbs.push_back(GR(it, b.name + ".ln1.b"));
+      }
+      emit_ln_bwd(h, p, lb, dgs, dbs);
+    }
+  };
+
+  std::vector<std::map<std::string, float*>> second_grads(K);   // overlapping updates: second gradients of chunk k's last block
+  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr, bool overlap) {
     std::vector<LabelProb> lps;
     for (int k = 0; k < K; ++k)
       lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, M, V,
@@ -269,99 +366,55 @@ void build_lm(Handle& h) {
     size_t maxb = 0;
     for (int k = 0; k < K; ++k) maxb = std::max(maxb, cb[k].blocks.size());
     for (size_t jj = 0; jj < maxb; ++jj) {
-      std::vector<int> act;
-      for (int k = 0; k < K; ++k) if (jj < cb[k].blocks.size()) act.push_back(k);
-      auto BJ = [&](int k) -> size_t { return cb[k].blocks.size() - 1 - jj; };
-      std::vector<GemmProb> g;
-      std::vector<ColSumProb> cs;
-      std::vector<float*> outs;
-      // 1. feed-forward second matrix: dW2, db2, du = (dout W2) * gelu'(u)
-      for (int k : act) {
-        ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
-        g.push_back(gemm_wgrad(c.G0, b.g, h.G(b.name + ".W2"), M, d, F));
-        g.push_back(gemm_dgrad(c.G0, h.W(b.name + ".W2"), c.Gf, M, d, F, EPI_GELU_GRAD, b.u));
-        cs.push_back(ColSumProb{c.G0, nullptr, M, d, d});
-        outs.push_back(h.G(b.name + ".b2"));
+      std::vector<BwdItem> items;
+      for (int k = 0; k < K; ++k) {
+        if (jj >= cb[k].blocks.size()) continue;
+        const size_t j = cb[k].blocks.size() - 1 - jj;
+        // The block-input gradient is formed only if something consumes it: an earlier block of the same
+        // chunk, chunk 0's embeddings, or (overlapping updates) the previous chunk's last block.
+        const bool need_dx = (j > 0) || (k == 0) || overlap;
+        items.push_back(BwdItem{&cb[k], &cb[k].blocks[j], block_in(k, j, rd), need_dx, nullptr});
       }
-      emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
-      g.clear(); cs.clear(); outs.clear();
-      // 2. feed-forward first matrix: dW1, db1, da2
-      for (int k : act) {
-        ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
-        g.push_back(gemm_wgrad(c.Gf, b.a2, h.G(b.name + ".W1"), M, F, d));
-        g.push_back(gemm_dgrad(c.Gf, h.W(b.name + ".W1"), c.G1, M, F, d, EPI_NONE, nullptr));
-        cs.push_back(ColSumProb{c.Gf, nullptr, M, F, F});
-        outs.push_back(h.G(b.name + ".b1"));
-      }
-      emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
-      g.clear(); cs.clear(); outs.clear();
-      // 3. LN2 backward; the residual path adds dout: dh1 -> G2
-      {
-        std::vector<LnBwdProb> lb;
-        std::vector<float*> dgs, dbs;
-        for (int k : act) {
-          ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
-          lb.push_back(LnBwdProb{c.G1, b.h1, h.P32(b.name + ".ln2.g"), b.mean2, b.rstd2, c.G2, c.G0, nullptr, M, d});
-          dgs.push_back(h.G(b.name + ".ln2.g"));
-          dbs.push_back(h.G(b.name + ".ln2.b"));
-        }
-        emit_ln_bwd(h, p, lb, dgs, dbs);
-      }
-      // 4. attention output projection: dWo, dbo, do -> G1
-      for (int k : act) {
-        ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
-        g.push_back(gemm_wgrad(c.G2, b.o, h.G(b.name + ".Wo"), M, d, d));
-        g.push_back(gemm_dgrad(c.G2, h.W(b.name + ".Wo"), c.G1, M, d, d, EPI_NONE, nullptr));
-        cs.push_back(ColSumProb{c.G2, nullptr, M, d, d});
-        outs.push_back(h.G(b.name + ".bo"));
-      }
-      emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
-      g.clear(); cs.clear(); outs.clear();
-      // 5. attention backward: dqkv -> Gq
-      {
-        std::vector<AttnProb> at;
-        for (int k : act) {
-          ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
-          at.push_back(AttnProb{b.qkv, b.o, b.lse, c.G1, c.Gq, b.delta, B, T, H});
-        }
-        const AttnProb* dp = h.upload(at);
-        int n = (int)at.size();
-        p.add(2, [=](const RunCtx& c) { launch_attn_bwd(dp, n, B, T, H, bf, c.stream); }, KIND_ATTN,
-              (double)n * 10.0 * B * H * 64.0 * T * (T + 1) / 2);
-      }
-      // 6. qkv projection: dWqkv, dbqkv, da1 -> G1 (needed for LN1's own parameters in every case)
-      for (int k : act) {
-        ChunkBufs& c = cb[k]; BlockBufs& b = c.blocks[BJ(k)];
-        g.push_back(gemm_wgrad(c.Gq, b.a1, h.G(b.name + ".Wqkv"), M, 3 * d, d));
-        g.push_back(gemm_dgrad(c.Gq, h.W(b.name + ".Wqkv"), c.G1, M, 3 * d, d, EPI_NONE, nullptr));
-        cs.push_back(ColSumProb{c.Gq, nullptr, M, 3 * d, 3 * d});
-        outs.push_back(h.G(b.name + ".bqkv"));
-      }
-      emit_gemm(h, p, g); emit_colsum(h, p, cs, outs);
-      g.clear(); cs.clear(); outs.clear();
-      // 7. LN1 backward.  The block-input gradient (dh1 + LN1 path -> G0) is formed only if a
-      //    layer of the same chunk consumes it: an earlier block, or chunk 0's embeddings.
-      {
-        std::vector<LnBwdProb> lb;
-        std::vector<float*> dgs, dbs;
-        for (int k : act) {
-          ChunkBufs& c = cb[k]; size_t j = BJ(k); BlockBufs& b = c.blocks[j];
-          bool need_dx = (j > 0) || (k == 0);
-          lb.push_back(LnBwdProb{c.G1, block_in(k, j, rd), h.P32(b.name + ".ln1.g"), b.mean1, b.rstd1,
-                                 need_dx ? c.G0 : nullptr, need_dx ? c.G2 : nullptr, nullptr, M, d});
-          dgs.push_back(h.G(b.name + ".ln1.g"));
-          dbs.push_back(h.G(b.name + ".ln1.b"));
-        }
-        emit_ln_bwd(h, p, lb, dgs, dbs);
-      }
-      // 8. chunk 0, first block: embedding tables
-      for (int k : act)
-        if (k == 0 && BJ(k) == 0) {
+      block_backward(p, items);
+      // chunk 0, first block: embedding tables
+      for (auto& it : items)
+        if (it.c == &cb[0] && it.b == &cb[0].blocks[0]) {
           EmbedBwdProb e{(const int*)h.x_in, cb[0].G0, h.G("c0.tok"), h.G("c0.pos"), emb_next, emb_first, M, T, d, V, B};
           p.add(6, [e, bf](const RunCtx& c) { launch_embed_bwd(e, bf, c.stream); }, KIND_EMBED, (double)M * d * es + 4.0 * V * d);
         }
     }
+    // ---- overlapping updates (Sec. 3, Fig. 2 c): chunk k's loss, whose gradient at the chunk input now sits in
+    // chunk k's G0, goes on through the last block of chunk k-1 (saved activations of this very minibatch),
+    // into second gradients of that block's parameters; it stops at that block's input.  The block's update
+    // uses the mean of its two gradients.
+    std::vector<AvgProb> avg;
+    long long avg_max = 0;
+    if (overlap) {
+      std::vector<BwdItem> items;
+      for (int k = 1; k < K; ++k) {
+        const size_t j = cb[k - 1].blocks.size() - 1;
+        BlockBufs* sb = &cb[k - 1].blocks[j];
+        auto& second = second_grads[k - 1];
+        if (second.empty())
+          for (const char* suf : {".ln1.g", ".ln1.b", ".Wqkv", ".bqkv", ".Wo", ".bo", ".ln2.g", ".ln2.b", ".W1", ".b1", ".W2", ".b2"})
+            second[sb->name + suf] = fal((size_t)h.tensors[h.find(sb->name + suf)].numel);
+        items.push_back(BwdItem{&cb[k], sb, block_in(k - 1, j, rd), false, &second});
+        for (auto& kv : second) {
+          const long long n = h.tensors[h.find(kv.first)].numel;
+          avg.push_back(AvgProb{h.G(kv.first), kv.second, n});
+          avg_max = std::max(avg_max, n);
+        }
+      }
+      block_backward(p, items);
+    }
     emit_pending_reduce(h, p);
+    if (!avg.empty()) {
+      const AvgProb* dp = h.upload(avg);
+      int n = (int)avg.size();
+      double bytes = 0;
+      for (auto& a : avg) bytes += 12.0 * a.n;
+      p.add(1, [=](const RunCtx& r) { launch_average_f32(dp, n, avg_max, r.stream); }, KIND_REDUCE, bytes);
+    }
     emit_optimizer(h, p);
   };
 
@@ -374,9 +427,13 @@ void build_lm(Handle& h) {
     heads_forward(p, wr, false, wr, true, false);
   };
 
-  build_step(h.sync_plan, false, 0, 0);
+  build_step(h.sync_plan, false, 0, 0, false);
+  if (K > 1) {
+    build_step(h.sync_overlap_plan, false, 0, 0, true);
+    h.has_overlap_plan = true;
+  }
   for (int par = 0; par < 2; ++par) {
-    build_step(h.pipe_plan[par], true, par, 1 - par);
+    build_step(h.pipe_plan[par], true, par, 1 - par, false);
     build_forward(h.prime_plan[par], par, false);
     std::vector<LabelProb> lps;
     for (int k = 0; k + 1 < K; ++k) lps.push_back(LabelProb{h.y_in, h.lab[par][k], M, V, h.n_valid[k]});

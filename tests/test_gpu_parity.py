@@ -326,19 +326,20 @@ def test_idle_ramp_up_resnet_bf16():
 
 # ------------------------------------------------------------------ overlapping local updates (MLP family)
 
-def check_overlap(cfg, gemm_backend=0):
+def check_overlap(cfg, gemm_backend=0, shared_per_boundary=2):
     """Synchronous steps with overlapping local updates against the oracle's overlap mode: first-step
     gradients (the shared layers hold the mean of their two gradients), then losses and weights after ten steps."""
     from paper_2012_03837_b200 import binding as lp
     dt = cfg["dtype"]
     gl, ol, gm, orc = T.run_both(cfg, 1, gemm_backend, overlap=True)
     gg = gm.get(lp.LP_GRAD)
-    errs = sorted(((T.tensor_rel_err(gg[n], orc.last_grads[n]), n) for n in gg), reverse=True)
+    errs = sorted(((T.tensor_rel_err(T.strip_key_bias(n, gg[n]), T.strip_key_bias(n, orc.last_grads[n])), n) for n in gg),
+                  reverse=True)
     gm.close()
     plain = T.run_both(cfg, 1, gemm_backend)[3]
     shared = [n for n in orc.last_grads if not np.array_equal(orc.last_grads[n], plain.last_grads[n])]
     print("overlap: first-step gradient error (worst)", [(f"{e:.2e}", n) for e, n in errs[:3]], "shared tensors", sorted(shared))
-    assert len(shared) == 2 * (gl.shape[1] - 1)
+    assert len(shared) == shared_per_boundary * (gl.shape[1] - 1)
     assert errs[0][0] <= G_TOL[dt], errs[:5]
     gl, ol, gm, orc = T.run_both(cfg, 10, gemm_backend, overlap=True)
     lerr = np.abs(gl - ol) / np.abs(ol)
@@ -374,9 +375,24 @@ def test_overlapping_updates_are_refused_where_they_are_not_defined():
         gm.step(x, y, "pipelined")
     assert lp.LP_ERR[e.value.code] == "UNSUPPORTED"
     gm.close()
-    lm = T.GpuModel(lp_synth.config("c3", batch=2, seq_len=64, vocab=256, d_model=128, n_heads=2, d_ffn=256,
-                                    blocks_per_chunk=[1, 1]))
+    rn = T.GpuModel(lp_synth.config("c4", dtype="fp32", batch=4, height=8, width=8, stem_channels=8,
+                                    stage_channels=[8, 16], blocks_per_stage=1, classes=5))
     with pytest.raises(lp.LpError) as e:
-        lp.lp_set_overlap(lm.h, True)
+        lp.lp_set_overlap(rn.h, True)
     assert lp.LP_ERR[e.value.code] == "UNSUPPORTED"
-    lm.close()
+    rn.close()
+
+
+def test_overlapping_updates_lm_fp32():
+    """The shared layer of the transformer family is a whole block: the next chunk's loss takes a second backward
+    pass through the previous chunk's last block (attention, feed-forward, both LayerNorms)."""
+    cfg = lp_synth.config("c3", dtype="fp32", batch=2, seq_len=80, vocab=300, d_model=128, n_heads=2, d_ffn=192,
+                          blocks_per_chunk=[1, 2, 1])
+    check_overlap(cfg, shared_per_boundary=12)
+
+
+@pytest.mark.parametrize("backend", [1, 0])
+def test_overlapping_updates_lm_bf16(backend):
+    cfg = lp_synth.config("c3", batch=3, seq_len=136, vocab=1000, d_model=128, n_heads=2, d_ffn=320,
+                          blocks_per_chunk=[1, 2, 1])
+    check_overlap(cfg, gemm_backend=backend, shared_per_boundary=12)
