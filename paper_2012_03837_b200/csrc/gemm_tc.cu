@@ -389,11 +389,18 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
       // the pre-activation is stored (C2) and the activation is taken of the value as stored
       pack32(v, pk);
       unpack32(pk, v);
-      put(p.C2, mapC2, pk, nullptr, false, 0);
+      if (p.aux_blocked) {
+        // blocked layout: this warp's 32x32 block is 2 KB of its own; four coalesced 512-byte stores
+        uint4* blk = (uint4*)((bf16*)p.C2 + (((size_t)(m_warp0 >> 5) * (p.ldc >> 5) + (n0 >> 5)) << 10));
+#pragma unroll
+        for (int q = 0; q < 4; ++q) blk[q * 32 + lane] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+      } else {
+        put(p.C2, mapC2, pk, nullptr, false, 0);
+      }
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] = gelu_fast(v[j]);
       pack32(v, pk);
-      put(p.C, mapC, pk, nullptr, false, 1);
+      put(p.C, mapC, pk, nullptr, false, p.aux_blocked ? 0 : 1);
       return;
     case EPI_RELU_MASK:
       load32(p.aux, t);
@@ -713,9 +720,15 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       auto fetch_side = [&](uint4* dst, int c) {
         const int nc = n0 + col0 + c * 32;
         if (side && vec_ok && m < p.M && nc + 32 <= p.N) {
-          const uint4* src = (const uint4*)((const bf16*)side + (size_t)m * p.ldc + nc);
+          if (p.aux_blocked && side == p.aux) {
+            const uint4* blk = (const uint4*)((const bf16*)side + (((size_t)((m0 + quarter * 32) >> 5) * (p.ldc >> 5) + (nc >> 5)) << 10));
 #pragma unroll
-          for (int q = 0; q < 4; ++q) dst[q] = src[q];
+            for (int q = 0; q < 4; ++q) dst[q] = blk[q * 32 + lane];
+          } else {
+            const uint4* src = (const uint4*)((const bf16*)side + (size_t)m * p.ldc + nc);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) dst[q] = src[q];
+          }
         }
       };
       fetch_side(side0, 0);                    // on its way while the accumulator is still being produced
@@ -823,6 +836,12 @@ bool encode_map4(CUtensorMap* out, const void* base, int n, int h, int w, int c,
 
 bool gemm_tc_eligible(const GemmProb& g) {
   if (g.M < 1 || g.N < 1 || g.K < 1) return false;
+  if (g.aux_blocked) {
+    const void* u = g.act == EPI_GELU ? g.C2 : g.aux;
+    if ((g.act != EPI_GELU && g.act != EPI_GELU_GRAD) || g.resid || g.out_f32 || !u || ((uintptr_t)u & 15) ||
+        g.M % 32 || g.N % 32 || g.ldc % 32 || ((uintptr_t)g.C & 15))
+      return false;
+  }
   if (g.conv != CONV_NONE) {
     // implicit 3x3 convolution: whole-row boxes, 64-channel k-slices, filters with 16-byte pitches
     if (g.conv_c < 64 || g.conv_c % 64 || g.conv_n < 1 || !conv_boxes_ok(g.conv_h, g.conv_w)) return false;
@@ -890,10 +909,12 @@ bool gemm_tc_encode(GemmProb& g, void* maps, int cg) {
   g.store_tma = ((g.ldc * esz) % 16 == 0) && (((uintptr_t)g.C & 15) == 0) &&
                 (g.act != EPI_GELU || (((uintptr_t)g.C2 & 15) == 0 && (g.ldc * 2) % 16 == 0));
   if (g.store_tma) {
-    // one bf16 output: pairs of column blocks leave in one store of full 128-byte rows (mode 2)
-    const bool wide = !g.out_f32 && g.act != EPI_GELU;
+    // one bf16 output through the staging buffer: pairs of column blocks leave in one store of full 128-byte
+    // rows (mode 2); the GELU epilogue's second output shares the buffer unless it is stored in blocks
+    const bool two_staged = g.act == EPI_GELU && !g.aux_blocked;
+    const bool wide = !g.out_f32 && !two_staged;
     bool ok = encode_out_map(mapA + 2, g.C, g.N, g.M, g.ldc, g.out_f32 != 0, wide);
-    if (ok && g.act == EPI_GELU) ok = encode_out_map(mapA + 3, g.C2, g.N, g.M, g.ldc, false, false);
+    if (ok && two_staged) ok = encode_out_map(mapA + 3, g.C2, g.N, g.M, g.ldc, false, false);
     g.store_tma = ok ? (wide ? 2 : 1) : 0;
   }
   bool okA, okB;

@@ -53,6 +53,13 @@ struct GemmProb {
   //   CONV_WGRAD : B(n, k) = x[pixel conv_k0 + k shifted by (i-1, j-1)][ci], n = (3i + j) conv_c + ci;
   //                N = 9 conv_c; A(m, k) = dy[pixel k][m] as an ordinary MN-major operand; K = pixels.
   // A is the activation tensor for CONV_FWD / CONV_DGRAD, B for CONV_WGRAD.
+  // Tensor-core kernel only.  The pre-activation that EPI_GELU writes (C2) and EPI_GELU_GRAD reads (aux) has no
+  // other reader, so its layout is free: with aux_blocked it is stored as 32x32 blocks of 2 KB, block
+  // (m / 32, n / 32) at ((m / 32) * (ldc / 32) + n / 32) * 1024 elements, inside a block 16-byte piece q of
+  // row r at q * 256 + r * 8 elements.  A warp's epilogue owns exactly such a block (one row per lane), so
+  // it writes and reads it with four fully coalesced 512-byte accesses instead of 32 scattered row pieces
+  // per access.  Needs M, N and ldc multiples of 32 and a 16-byte aligned buffer.
+  int aux_blocked;
   int conv;
   int conv_n, conv_h, conv_w, conv_c;
   int conv_k0;     // CONV_WGRAD: first pixel of this slice of the reduction (split-K)

@@ -109,6 +109,18 @@ void build_lm(Handle& h) {
   for (int k = 0; k < K; ++k) all.push_back(k);
   const bool bf = h.bf16_mode;
   int* st = h.d_status;
+  // The feed-forward pre-activation u is written by the first feed-forward product's epilogue and read only by
+  // the epilogue of the second one's input gradient.  When both run on the tensor-core kernel, u is kept in
+  // 32x32 blocks (see GemmProb::aux_blocked) so that both touch it with coalesced accesses.
+  bool u_blocked = bf && !h.force_simt && M % 32 == 0 && F % 32 == 0 && !cb.empty() && !cb[0].blocks.empty();
+  if (u_blocked) {
+    BlockBufs& b0 = cb[0].blocks[0];
+    GemmProb f = gemm_fwd(b0.a2, h.W(b0.name + ".W1"), b0.g, M, F, d, h.P32(b0.name + ".b1"), EPI_GELU);
+    f.C2 = b0.u; f.aux_blocked = 1;
+    GemmProb g2 = gemm_dgrad(cb[0].G0, h.W(b0.name + ".W2"), cb[0].Gf, M, d, F, EPI_GELU_GRAD, b0.u);
+    g2.aux_blocked = 1;
+    u_blocked = gemm_tc_eligible(f) && gemm_tc_eligible(g2);
+  }
 
   auto chunk_in = [&](int k, int rd) -> const void* { return k == 0 ? cb[0].emb : h.bnd[rd][k - 1]; };
   auto block_in = [&](int k, size_t j, int rd) -> const void* {
@@ -165,6 +177,7 @@ void build_lm(Handle& h) {
         BlockBufs& b = cb[k].blocks[j];
         GemmProb q = gemm_fwd(b.a2, h.W(b.name + ".W1"), b.g, M, F, d, h.P32(b.name + ".b1"), EPI_GELU);
         q.C2 = b.u;
+        q.aux_blocked = u_blocked ? 1 : 0;
         g.push_back(q);
       }
       emit_gemm(h, p, g);
@@ -248,6 +261,7 @@ void build_lm(Handle& h) {
       ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
       g.push_back(gemm_wgrad(c.G0, b.g, GR(it, b.name + ".W2"), M, d, F));
       g.push_back(gemm_dgrad(c.G0, h.W(b.name + ".W2"), c.Gf, M, d, F, EPI_GELU_GRAD, b.u));
+      g.back().aux_blocked = u_blocked ? 1 : 0;
       cs.push_back(ColSumProb{c.G0, nullptr, M, d, d});
       outs.push_back(GR(it, b.name + ".b2"));
     }
