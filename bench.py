@@ -54,9 +54,10 @@ def describe(cfg):
 # capture summarised under profiles/ and scaled to the launches of a full step.  A figure is only
 # valid for the kernel source it was captured on: it is dropped when that file has changed since.
 TRAFFIC = {
-    # 24 chunks x (head products 2.30 GB measured + block products 1.07 GB algorithmic) over the step's 10 launches
-    "c5": dict(bytes_per_launch=8.1e9, chunks=24, kernel_file="paper_2012_03837_b200/csrc/gemm_tc.cu",
-               kernel_sha256="87de96ac55a1c9fcce4e8533f0cf05f54b63b254f0a8689caf66ae763cd746d1"),
+    # the ten grouped GEMM launches of a one-chunk c5 step move 3.31 GB through DRAM (ncu); every chunk streams its
+    # own operands, so a 24-chunk step moves 24 x 3.31 GB over its ten launches
+    "c5": dict(bytes_per_launch=7.9e9, chunks=24, kernel_file="paper_2012_03837_b200/csrc/gemm_tc.cu",
+               kernel_sha256="baa97055c45470f190829b22031d4777ef3b22a178b03d72424b3005b4d26645"),
 }
 
 
