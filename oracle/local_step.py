@@ -22,7 +22,8 @@ Schedules:
     loss NaN) until real data reaches it at step k.
 
 Overlapping local parallelism (Sec. 3; cost model in App. A.2): with overlap=True the block trained by
-chunk k's loss also contains the last layer of chunk k-1 (for the transformer: its last block), so that
+chunk k's loss also contains the last layer of chunk k-1 (transformer: its last block; ResNet: its last
+BasicBlock), so that
 loss is back-propagated one layer past the chunk boundary and stops at that layer's input.  The
 shared layer exists once (one forward pass through the network); it receives two gradients, from
 its own chunk's loss and from the next chunk's, and is updated with their average.  Defined for
@@ -219,22 +220,28 @@ class LocalUpdateOracle:
             p[name + ".rm"], p[name + ".rv"] = rm.astype(p[name + ".rm"].dtype), rv.astype(p[name + ".rv"].dtype)
         return y, cache
 
+    def _resnet_block_bwd(self, dx, block_cache, g):
+        """Backward of one BasicBlock: fills g with its parameter gradients, returns the gradient at the block
+        input (main branch plus shortcut)."""
+        (n, cc1, cb1, cr1, cc2, cb2, csc, cr2) = block_cache
+        ds = L.relu_bwd(dx, cr2)
+        du, g[n + ".bn2.g"], g[n + ".bn2.b"] = L.batchnorm_bwd(ds, cb2)
+        du, g[n + ".conv2"] = L.conv2d_bwd(du, cc2)
+        du = L.relu_bwd(du, cr1)
+        du, g[n + ".bn1.g"], g[n + ".bn1.b"] = L.batchnorm_bwd(du, cb1)
+        dx, g[n + ".conv1"] = L.conv2d_bwd(du, cc1)
+        if csc is not None:
+            ccs, cbs = csc
+            dsc, g[n + ".sc.bn.g"], g[n + ".sc.bn.b"] = L.batchnorm_bwd(ds, cbs)
+            dsc, g[n + ".sc.conv"] = L.conv2d_bwd(dsc, ccs)
+            return dx + dsc
+        return dx + ds
+
     def _resnet_bwd(self, k, dx, cache):
         g = {}
-        for (n, cc1, cb1, cr1, cc2, cb2, csc, cr2) in reversed(cache["blocks"]):
-            ds = L.relu_bwd(dx, cr2)
-            du, g[n + ".bn2.g"], g[n + ".bn2.b"] = L.batchnorm_bwd(ds, cb2)
-            du, g[n + ".conv2"] = L.conv2d_bwd(du, cc2)
-            du = L.relu_bwd(du, cr1)
-            du, g[n + ".bn1.g"], g[n + ".bn1.b"] = L.batchnorm_bwd(du, cb1)
-            dx, g[n + ".conv1"] = L.conv2d_bwd(du, cc1)
-            if csc is not None:
-                ccs, cbs = csc
-                dsc, g[n + ".sc.bn.g"], g[n + ".sc.bn.b"] = L.batchnorm_bwd(ds, cbs)
-                dsc, g[n + ".sc.conv"] = L.conv2d_bwd(dsc, ccs)
-                dx = dx + dsc
-            else:
-                dx = dx + ds
+        for block_cache in reversed(cache["blocks"]):
+            dx = self._resnet_block_bwd(dx, block_cache, g)
+        self._dx_in = dx         # gradient at the stage input: used only by the overlapping variant
         if "stem" in cache:
             cc, cb, cr = cache["stem"]
             du = L.relu_bwd(dx, cr)
@@ -261,8 +268,8 @@ class LocalUpdateOracle:
 
     def overlap_grads(self, k_prev, dx, cache_prev):
         """Overlapping local parallelism (Sec. 3): the gradient of the NEXT chunk's loss with respect to
-        the parameters of the last layer of chunk k_prev (its last Linear+ReLU, or its last transformer
-        block), given that loss's gradient dx at chunk k_prev's output; truncated at that layer's input."""
+        the parameters of the last layer of chunk k_prev (its last Linear+ReLU, its last transformer block,
+        or its last BasicBlock), given that loss's gradient dx at chunk k_prev's output; truncated at that layer's input."""
         fam = self.cfg["family"]
         g = {}
         if fam == "mlp":
@@ -273,7 +280,7 @@ class LocalUpdateOracle:
         elif fam == "lm":
             self._lm_block_bwd(dx, cache_prev["blocks"][-1], g)
         else:
-            raise NotImplementedError("overlapping updates: MLP and LM families")
+            self._resnet_block_bwd(dx, cache_prev["blocks"][-1], g)
         return g
 
     def apply_update(self, k, grads):
