@@ -218,9 +218,8 @@ lp_status lp_set_ramp(lp_handle h, int ramp);
  * pass); it receives a gradient from its own chunk's loss and one from the next chunk's, and its update
  * uses their mean.  All other parameters are updated as without overlap.  LP_GRAD of a shared layer then
  * holds the mean.  Synchronous steps only (a pipelined lp_step returns LP_ERR_UNSUPPORTED while overlap is
- * on).  For the LM family the shared layer is the previous chunk's last transformer block (App. B.2 trains
- * layer-wise blocks), for the MLP family its last Linear+ReLU.  Built for MLP and LM with K >= 2; otherwise
- * LP_ERR_UNSUPPORTED.
+ * on).  The shared layer is the previous chunk's last Linear+ReLU (MLP), its last transformer block (LM; App.
+ * B.2 trains layer-wise blocks) or its last BasicBlock (RESNET).  Needs K >= 2, otherwise LP_ERR_UNSUPPORTED.
  */
 lp_status lp_set_overlap(lp_handle h, int on);
 

@@ -402,7 +402,7 @@ lp_status lp_set_overlap(lp_handle hh, int on) {
   if (!hh) return LP_ERR_INVALID_ARG;
   Handle& h = hh->h;
   if (on && !h.has_overlap_plan)
-    return fail(&h, LP_ERR_UNSUPPORTED, "overlapping updates are built for the MLP and LM families with at least two chunks");
+    return fail(&h, LP_ERR_UNSUPPORTED, "overlapping updates need at least two chunks");
   h.overlap = on != 0;
   return LP_OK;
 }

@@ -7,6 +7,7 @@
 // Backward is truncated at the chunk input (Sec. 3): the first block of a stage k > 0 forms no input
 // gradient (no dgrad for its first convolution and its shortcut convolution), nor does the stem.
 // The synchronous schedule is the natural one here; the pipelined plans are built too.
+#include <map>
 #include <stdexcept>
 
 #include "runtime.h"
@@ -50,6 +51,10 @@ struct Chunk {
   float* row_loss;
   void* G[4];
   void* dcols;
+  // overlapping updates: scratch for the second backward pass through the previous stage's last block
+  void* GO[3] = {nullptr, nullptr, nullptr};
+  void* dcolsO = nullptr;
+  std::map<std::string, float*> second;        // second gradients of THIS chunk's last block (filled by chunk k+1's loss)
 };
 
 // Backward passes of the chunks are independent of one another (Sec. 3): each chunk records its backward
@@ -310,14 +315,17 @@ void build_resnet(Handle& h) {
   };
 
   // ---- backward, recorded per chunk and emitted in lockstep
-  auto wgrad_prob = [&](const Conv& c, const void* dy, const void* x) {
+  // where a parameter gradient goes: the arena, or a second buffer (overlapping updates)
+  typedef std::map<std::string, float*> GradMap;
+  auto GD = [&](const GradMap* second, const std::string& name) -> float* { return second ? second->at(name) : h.G(name); };
+  auto wgrad_prob = [&](const Conv& c, const void* dy, const void* x, const GradMap* second = nullptr) {
     if (c.imp_fwd) {
-      GemmProb g = gemm_wgrad(dy, x, h.G(c.w), (int)c.M, c.Cout, c.K);
+      GemmProb g = gemm_wgrad(dy, x, GD(second, c.w), (int)c.M, c.Cout, c.K);
       g.b_ks = c.Cin;
       conv_fields(g, c, CONV_WGRAD, c.Cin);
       return g;
     }
-    GemmProb g = gemm_wgrad(dy, c.cols, h.G(c.w), (int)c.M, c.Cout, c.K);
+    GemmProb g = gemm_wgrad(dy, c.cols, GD(second, c.w), (int)c.M, c.Cout, c.K);
     g.b_ks = c.ldk;
     return g;
   };
@@ -350,13 +358,15 @@ void build_resnet(Handle& h) {
   };
   auto rec_nop = [&](OpList& L, int n = 1) { for (int i = 0; i < n; ++i) L.push_back(Op{}); };
   // dx = BN'(dy masked by relu_out > 0); dres (optional) receives the masked dy
-  auto rec_bn_bwd = [&](OpList& L, const Bn& b, const void* x, const void* dy, const void* relu_out, void* dx, void* dres) {
+  auto rec_bn_bwd = [&](OpList& L, const Bn& b, const void* x, const void* dy, const void* relu_out, void* dx, void* dres,
+                        const GradMap* second = nullptr) {
     int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
     float* part = fal((size_t)nblk * 2 * b.C);
+    float *dg = GD(second, b.g), *db = GD(second, b.b);
     Op o; o.kind = OP_BN_BWD;
     o.bn_stat = BnStatProb{x, dy, b.mean, b.rstd, relu_out, part, (int)b.rows, b.C};
-    o.bn_final = BnFinalProb{part, nblk, (int)b.rows, b.C, nullptr, nullptr, h.G(b.g), h.G(b.b), 1e-5f, nullptr, nullptr, 0.f, 0, nullptr, 0};
-    o.bn_apply = BnApplyProb{x, nullptr, nullptr, h.P32(b.g), h.P32(b.b), b.mean, b.rstd, dy, relu_out, dx, dres, h.G(b.g), h.G(b.b),
+    o.bn_final = BnFinalProb{part, nblk, (int)b.rows, b.C, nullptr, nullptr, dg, db, 1e-5f, nullptr, nullptr, 0.f, 0, nullptr, 0};
+    o.bn_apply = BnApplyProb{x, nullptr, nullptr, h.P32(b.g), h.P32(b.b), b.mean, b.rstd, dy, relu_out, dx, dres, dg, db,
                              (int)b.rows, b.C, 0};
     o.v8 = bf && b.C % 8 == 0 && b.C / 8 <= 256;
     o.elems = b.rows * b.C;
@@ -367,8 +377,50 @@ void build_resnet(Handle& h) {
     Op o; o.kind = OP_ADD; o.add = AddProb{acc, other, acc, n}; o.elems = n; L.push_back(std::move(o));
   };
 
-  // Every chunk's list has the same length and the same kind (or a gap) at every position.
-  auto record_backward = [&](OpList& L, int k, int rd, int wr) {
+  // Backward of one BasicBlock, recorded: on entry the gradient at the block output is in gin; parameter
+  // gradients go to the arena or to `second`; if need_dx the gradient at the block input ends up in the
+  // buffer returned (one of gin / gc), otherwise no input gradient is formed (Sec. 3).
+  auto rec_block_bwd = [&](OpList& L, Block& b, const void* x, const void* out, bool need_dx, void* gin, void* ga, void* gb,
+                           void* gc, void* dcols, const GradMap* second) -> void* {
+    long long in_elems_blk = (long long)b.c1.N * b.c1.H * b.c1.W * b.c1.Cin;
+    Op gather;
+    // out = relu(bn2(c2) + shortcut): ga <- d(c2), gb <- gradient of the shortcut branch
+    rec_bn_bwd(L, b.b2, b.c2.y, gin, out, ga, gb, second);
+    {                                                     // dW(c2) and gc <- d(a1) read the same ga: one launch
+      GemmProb dg = dgrad_prob(b.c2, ga, gc, dcols, gather);
+      rec_gemm(L, {wgrad_prob(b.c2, ga, b.a1, second), dg});
+      L.push_back(gather);
+    }
+    rec_bn_bwd(L, b.b1, b.c1.y, gc, b.a1, ga, nullptr, second);   // ga <- d(c1)
+    if (need_dx) {                                        // gc <- d(x) through the main branch
+      GemmProb dg = dgrad_prob(b.c1, ga, gc, dcols, gather);
+      rec_gemm(L, {wgrad_prob(b.c1, ga, x, second), dg});
+      L.push_back(gather);
+    } else {
+      rec_gemm(L, {wgrad_prob(b.c1, ga, x, second)});
+      rec_nop(L);
+    }
+    if (b.has_sc) {
+      rec_bn_bwd(L, b.bs, b.cs.y, gb, nullptr, ga, nullptr, second);   // ga <- d(cs)
+      if (need_dx) {
+        GemmProb dg = dgrad_prob(b.cs, ga, gin, dcols, gather);   // gin <- d(x) through the shortcut
+        rec_gemm(L, {wgrad_prob(b.cs, ga, x, second), dg});
+        L.push_back(gather);
+        rec_add(L, gc, gin, in_elems_blk);
+      } else {
+        rec_gemm(L, {wgrad_prob(b.cs, ga, x, second)});
+        rec_nop(L, 2);
+      }
+    } else {
+      rec_nop(L, 3);
+      if (need_dx) rec_add(L, gc, gb, in_elems_blk); else rec_nop(L);
+    }
+    return gc;                                            // the block-input gradient (if formed)
+  };
+
+  // Every chunk's list has the same kind (or a gap) at every position it shares with another chunk's.
+  std::vector<AvgProb> overlap_avg;                       // filled while an overlapping plan is recorded
+  auto record_backward = [&](OpList& L, int k, int rd, int wr, bool overlap) {
     Chunk& c = ch[k];
     const std::string ck = "c" + std::to_string(k);
     // head: dW_h, db_h, d(pool), then the pool's gradient spread over H*W -> G[0]
@@ -382,41 +434,36 @@ void build_resnet(Handle& h) {
       Block& b = c.blocks[j];
       const void* x = j == 0 ? chunk_in(k, rd) : c.blocks[j - 1].out;
       const void* out = b.out ? b.out : h.bnd[wr][k];
-      bool need_dx = (j > 0) || c.has_stem;
-      long long in_elems_blk = (long long)b.c1.N * b.c1.H * b.c1.W * b.c1.Cin;
-      Op gather;
-      // out = relu(bn2(c2) + shortcut): ga <- d(c2), gb <- gradient of the shortcut branch
-      rec_bn_bwd(L, b.b2, b.c2.y, gin, out, ga, gb);
-      {                                                     // dW(c2) and gc <- d(a1) read the same ga: one launch
-        GemmProb dg = dgrad_prob(b.c2, ga, gc, c.dcols, gather);
-        rec_gemm(L, {wgrad_prob(b.c2, ga, b.a1), dg});
-        L.push_back(gather);
-      }
-      rec_bn_bwd(L, b.b1, b.c1.y, gc, b.a1, ga, nullptr);   // ga <- d(c1)
-      if (need_dx) {                                        // gc <- d(x) through the main branch
-        GemmProb dg = dgrad_prob(b.c1, ga, gc, c.dcols, gather);
-        rec_gemm(L, {wgrad_prob(b.c1, ga, x), dg});
-        L.push_back(gather);
-      } else {
-        rec_gemm(L, {wgrad_prob(b.c1, ga, x)});
-        rec_nop(L);
-      }
-      if (b.has_sc) {
-        rec_bn_bwd(L, b.bs, b.cs.y, gb, nullptr, ga, nullptr);   // ga <- d(cs)
-        if (need_dx) {
-          GemmProb dg = dgrad_prob(b.cs, ga, gin, c.dcols, gather);   // gin <- d(x) through the shortcut
-          rec_gemm(L, {wgrad_prob(b.cs, ga, x), dg});
-          L.push_back(gather);
-          rec_add(L, gc, gin, in_elems_blk);
-        } else {
-          rec_gemm(L, {wgrad_prob(b.cs, ga, x)});
-          rec_nop(L, 2);
+      // the stage-input gradient is needed by the stem (chunk 0) or, with overlapping updates, by the previous
+      // stage's last block
+      bool need_dx = (j > 0) || c.has_stem || (overlap && k > 0);
+      void* dxbuf = rec_block_bwd(L, b, x, out, need_dx, gin, ga, gb, gc, c.dcols, nullptr);
+      gc = gin; gin = dxbuf;                                // the block-input gradient feeds the next (earlier) block
+    }
+    if (overlap && k > 0) {
+      // Overlapping local parallelism (Sec. 3, Fig. 2 c): this stage's loss goes on through the last BasicBlock of
+      // stage k-1 (activations of this very minibatch) into second gradients of its parameters and stops at
+      // that block's input; the block's update uses the mean of its two gradients.
+      Chunk& q = ch[k - 1];
+      Block& sb = q.blocks.back();
+      const size_t nb = q.blocks.size();
+      const void* sx = nb == 1 ? chunk_in(k - 1, rd) : q.blocks[nb - 2].out;
+      if (!c.GO[0]) {
+        size_t act = 0, cols = 0;
+        for (const Conv* cv : {&sb.c1, &sb.c2, &sb.cs}) {
+          if (cv == &sb.cs && !sb.has_sc) continue;
+          act = std::max(act, (size_t)cv->M * cv->Cout);
+          act = std::max(act, (size_t)cv->N * cv->H * cv->W * cv->Cin);
+          if (!cv->imp_dgrad) cols = std::max(cols, (size_t)cv->M * cv->ldk);
         }
-      } else {
-        rec_nop(L, 3);
-        if (need_dx) rec_add(L, gc, gb, in_elems_blk); else rec_nop(L);
+        for (int i = 0; i < 3; ++i) c.GO[i] = h.dalloc(act * es);
+        if (cols) c.dcolsO = h.dalloc(cols * es);
+        std::vector<std::string> names = {sb.c1.w, sb.b1.g, sb.b1.b, sb.c2.w, sb.b2.g, sb.b2.b};
+        if (sb.has_sc) { names.push_back(sb.cs.w); names.push_back(sb.bs.g); names.push_back(sb.bs.b); }
+        for (auto& n : names) q.second[n] = fal((size_t)h.tensors[h.find(n)].numel);
       }
-      std::swap(gin, gc);                                   // the block-input gradient feeds the next (earlier) block
+      rec_block_bwd(L, sb, sx, h.bnd[wr][k - 1], false, gin, c.GO[0], c.GO[1], c.GO[2], c.dcolsO, &q.second);
+      for (auto& kv : q.second) overlap_avg.push_back(AvgProb{h.G(kv.first), kv.second, (long long)h.tensors[h.find(kv.first)].numel});
     }
     if (c.has_stem) {
       rec_bn_bwd(L, c.stem_bn, c.stem.y, gin, c.stem_out, ga, nullptr);
@@ -498,7 +545,7 @@ void build_resnet(Handle& h) {
   std::vector<int> all;
   for (int k = 0; k < K; ++k) all.push_back(k);
 
-  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr) {
+  auto build_step = [&](Plan& p, bool pipelined, int rd, int wr, bool overlap) {
     std::vector<LabelProb> lps;
     for (int k = 0; k < K; ++k)
       lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, B, NC, h.n_valid[k]});
@@ -506,9 +553,19 @@ void build_resnet(Handle& h) {
     for (int k = 0; k < K; ++k) forward_chunk(p, k, rd, wr, BN_TRAIN);
     for (int k = 0; k < K; ++k) head_forward(p, k, wr, labels_of(k, pipelined, rd), false);
     std::vector<OpList> lists(K);
-    for (int k = 0; k < K; ++k) record_backward(lists[k], k, rd, wr);
+    overlap_avg.clear();
+    for (int k = 0; k < K; ++k) record_backward(lists[k], k, rd, wr, overlap);
     flush_ops(p, lists);
     emit_pending_reduce(h, p);
+    if (!overlap_avg.empty()) {
+      const AvgProb* d = h.upload(overlap_avg);
+      int n = (int)overlap_avg.size();
+      long long mx = 0;
+      double bytes = 0;
+      for (auto& a : overlap_avg) { mx = std::max(mx, a.n); bytes += 12.0 * a.n; }
+      p.add(1, [=](const RunCtx& r) { launch_average_f32(d, n, mx, r.stream); }, KIND_REDUCE, bytes);
+      overlap_avg.clear();
+    }
     emit_optimizer(h, p);
   };
   auto build_forward = [&](Plan& p, int wr, bool heads, int mode) {
@@ -521,9 +578,13 @@ void build_resnet(Handle& h) {
   };
 
   h.has_eval_plan = true;
-  build_step(h.sync_plan, false, 0, 0);
+  build_step(h.sync_plan, false, 0, 0, false);
+  if (K > 1) {
+    build_step(h.sync_overlap_plan, false, 0, 0, true);
+    h.has_overlap_plan = true;
+  }
   for (int par = 0; par < 2; ++par) {
-    build_step(h.pipe_plan[par], true, par, 1 - par);
+    build_step(h.pipe_plan[par], true, par, 1 - par, false);
     build_forward(h.prime_plan[par], par, false, BN_BATCH);
     std::vector<LabelProb> lps;
     for (int k = 0; k + 1 < K; ++k) lps.push_back(LabelProb{h.y_in, h.lab[par][k], B, NC, h.n_valid[k]});

@@ -100,7 +100,7 @@ struct Handle {
   Plan sync_plan, pipe_plan[2], prime_plan[2], fwd_plan[2];
   Plan eval_plan[2];                           // RESNET: forward with BatchNorm on its running statistics
   bool has_eval_plan = false;
-  Plan sync_overlap_plan;                      // MLP, LM: synchronous step with overlapping local updates (Sec. 3)
+  Plan sync_overlap_plan;                      // synchronous step with overlapping local updates (Sec. 3)
   bool has_overlap_plan = false;
   bool overlap = false;
   std::vector<ColReduceProb> pending_reduce;   // collected while a plan is being built
