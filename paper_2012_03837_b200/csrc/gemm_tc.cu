@@ -41,11 +41,18 @@ constexpr int A_BYTES = BM * BK * 2;              // 16 KB of A per CTA and stag
 // CG = 2: a pair of CTAs (cluster of 2, tcgen05 cta_group::2) per 256x256 tile; each CTA holds its own
 //         128 rows of A and HALF of the B tile (128x64, 16 KB), so every SM pulls a third fewer bytes per
 //         FLOP through its L2 port and the ring is 6 stages of 32 KB.
-template <int CG> struct Cfg {
-  static constexpr int BNL = BN / CG;                       // rows of B this CTA loads
-  static constexpr int B_BYTES = BNL * BK * 2;
+// W = 1 ("wide", CTA pairs only): a 256x512 tile per pair, computed as two MMAs per k-step that share the A
+//         slice: 16 KB of A and two 16 KB B halves per stage (4 stages of 48 KB).  Per FLOP a CTA then moves
+//         20 % less through shared memory than with the 256x256 tile; both accumulators belong to the one
+//         tile, so the epilogue is not overlapped with the next main loop -- worth it only for long reductions.
+template <int CG, int W = 0> struct Cfg {
+  static constexpr int TN = W ? 2 * BN : BN;                // tile columns
+  static constexpr int NB = W ? 2 : 1;                      // B sub-tiles = MMAs per k-step
+  static constexpr int BNL = BN / CG;                       // rows of one B sub-tile this CTA loads
+  static constexpr int B_SUB_BYTES = BNL * BK * 2;
+  static constexpr int B_BYTES = NB * B_SUB_BYTES;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = CG == 1 ? 4 : 6;
+  static constexpr int STAGES = CG == 1 ? 4 : (W ? 4 : 6);
 };
 constexpr int MAX_STAGES = 6;
 constexpr int EPI_WARPS = 8;                      // two warps per TMEM lane quarter, each takes half of the 256 columns
@@ -484,12 +491,13 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
-template <int CG>
+template <int CG, int W>
 __global__ void __launch_bounds__(NTHREADS, 1)
 gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict__ maps, int nprob, int total_tiles,
                int* status) {
-  using C = Cfg<CG>;
-  constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, BNL = C::BNL;
+  using C = Cfg<CG, W>;
+  constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, BNL = C::BNL, TN = C::TN, NB = C::NB,
+                B_SUB_BYTES = C::B_SUB_BYTES;
   constexpr int TILE_M = BM * CG;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -544,7 +552,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
         const CUtensorMap* mapB = mapA + 1;
         int mt, nt;
         walk.coords(tile, mt, nt);
-        int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN + (int)rank * BNL;
+        int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * TN + (int)rank * BNL;
         if (conv == CONV_NONE) {
           // ---- ordinary operands: 2-D boxes of the A and B matrices
           for (int kb = 0; kb < kb_n; ++kb) {
@@ -561,11 +569,16 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
               } else {
                 tma_load_2d(a_dst, mapA, k0, m0, bar);
               }
-              if (b_mn) {
 #pragma unroll
-                for (int i = 0; i < BNL / 64; ++i) tma_load_2d(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, bar);
-              } else {
-                tma_load_2d(b_dst, mapB, k0, n0, bar);
+              for (int sb = 0; sb < NB; ++sb) {
+                uint8_t* b_sub = b_dst + sb * B_SUB_BYTES;
+                const int ns = n0 + sb * BN;
+                if (b_mn) {
+#pragma unroll
+                  for (int i = 0; i < BNL / 64; ++i) tma_load_2d(b_sub + i * (BK * 128), mapB, ns + i * 64, k0, bar);
+                } else {
+                  tma_load_2d(b_sub, mapB, k0, ns, bar);
+                }
               }
             } else {
               // both CTAs' bytes are counted on the leader's barrier
@@ -577,11 +590,16 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
               } else {
                 tma_load_2d_pair(a_dst, mapA, k0, m0, bar);
               }
-              if (b_mn) {
 #pragma unroll
-                for (int i = 0; i < BNL / 64; ++i) tma_load_2d_pair(b_dst + i * (BK * 128), mapB, n0 + i * 64, k0, bar);
-              } else {
-                tma_load_2d_pair(b_dst, mapB, k0, n0, bar);
+              for (int sb = 0; sb < NB; ++sb) {
+                uint8_t* b_sub = b_dst + sb * B_SUB_BYTES;
+                const int ns = n0 + sb * BN;
+                if (b_mn) {
+#pragma unroll
+                  for (int i = 0; i < BNL / 64; ++i) tma_load_2d_pair(b_sub + i * (BK * 128), mapB, ns + i * 64, k0, bar);
+                } else {
+                  tma_load_2d_pair(b_sub, mapB, k0, ns, bar);
+                }
               }
             }
             if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -666,8 +684,9 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
           idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
         }
-        int ab = it & 1;
-        uint32_t use = (uint32_t)(it >> 1);
+        // wide tiles own both accumulators (barrier set 0); otherwise the two alternate from tile to tile
+        int ab = W ? 0 : (it & 1);
+        uint32_t use = W ? (uint32_t)it : (uint32_t)(it >> 1);
         if (!(ok = mbar_wait(&sh->tmem_empty[ab], (use & 1) ^ 1, sh, status))) break;
         tc_fence_after();
         uint32_t d_tmem = tmem_base + ab * BN;
@@ -682,7 +701,13 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
 #pragma unroll
           for (int k4 = 0; k4 < BK / 16; ++k4) {
             if (CG == 1) tc_mma(d_tmem, adesc + (uint64_t)(k4 * a_step), bdesc + (uint64_t)(k4 * b_step), idesc, (kb | k4) != 0);
-            else tc_mma_pair(d_tmem, adesc + (uint64_t)(k4 * a_step), bdesc + (uint64_t)(k4 * b_step), idesc, (kb | k4) != 0);
+            else {
+              // wide: the two column halves of the tile take the same A slice back to back
+#pragma unroll
+              for (int sb = 0; sb < NB; ++sb)
+                tc_mma_pair(d_tmem + sb * BN, adesc + (uint64_t)(k4 * a_step),
+                            bdesc + (uint64_t)((sb * B_SUB_BYTES) >> 4) + (uint64_t)(k4 * b_step), idesc, (kb | k4) != 0);
+            }
           }
           if (CG == 1) tc_commit(&sh->empty[stage]); else tc_commit_pair(&sh->empty[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -705,14 +730,14 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       const GemmProb p = probs[pi];          // read-only table: fields are fetched where they are used
       int mt, nt;
       walk.coords(tile, mt, nt);
-      int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * BN;
-      int ab = it & 1;
-      uint32_t use = (uint32_t)(it >> 1);
+      int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * TN;
+      int ab = W ? 0 : (it & 1);
+      uint32_t use = W ? (uint32_t)it : (uint32_t)(it >> 1);
       // Each thread owns one accumulator row and walks this warp's half of the columns 32 at a time;
       // the TMEM load of the next 32 columns and the global load of the next block of the side input
       // (residual or activation-derivative operand) are in flight while the current block is stored.
       const int m = m0 + quarter * 32 + lane;
-      const int col0 = ((warp - EPI_FIRST) >> 2) * (BN / 2);
+      const int col0 = ((warp - EPI_FIRST) >> 2) * (TN / 2);
       const bool vec_ok = (p.ldc % 8 == 0) && (((uintptr_t)p.C & 15) == 0) && (!p.C2 || ((uintptr_t)p.C2 & 15) == 0) &&
                           (!p.resid || ((uintptr_t)p.resid & 15) == 0) && (!p.aux || ((uintptr_t)p.aux & 15) == 0);
       const void* side = (p.resid && !p.aux) ? p.resid : (p.aux && !p.resid) ? p.aux : nullptr;
@@ -750,13 +775,13 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       uint32_t acc0[32], acc1[32];
       tc_ld32(trow, acc0);
 #pragma unroll 1
-      for (int c = 0; c < BN / 64; c += 2) {
+      for (int c = 0; c < TN / 64; c += 2) {
         tc_wait_ld();
         tc_ld32(trow + (c + 1) * 32, acc1);
         fetch_side(side1, c + 1);
         emit(acc0, c, side0);
         tc_wait_ld();
-        if (c + 2 < BN / 64) { tc_ld32(trow + (c + 2) * 32, acc0); fetch_side(side0, c + 2); }
+        if (c + 2 < TN / 64) { tc_ld32(trow + (c + 2) * 32, acc0); fetch_side(side0, c + 2); }
         emit(acc1, c + 1, side1);
       }
       if (p.act == EPI_LOGIT_STATS && m < p.M && n0 + col0 < p.N)
@@ -875,9 +900,20 @@ int gemm_tc_choose_cg(const GemmProb* probs, int n) {
   return 2;
 }
 
-int gemm_tc_tiles(GemmProb& g, int tile_start, int cg) {
+bool gemm_tc_wide_ok(const GemmProb& g) {
+  static int off = -1;
+  if (off < 0) {
+    const char* e = getenv("LP_GEMM_WIDE");    // diagnostic override: 0 switches the wide tiles off
+    off = (e && atoi(e) == 0) ? 1 : 0;
+  }
+  // long reductions only (the epilogue of a wide tile is exposed), plain epilogue, columns that fill 512-wide tiles
+  return !off && g.K >= 8192 && g.M > BM && g.N % (2 * BN) == 0 && g.act == EPI_NONE && !g.bias && !g.resid && !g.aux &&
+         g.conv == CONV_NONE && !g.aux_blocked;
+}
+
+int gemm_tc_tiles(GemmProb& g, int tile_start, int cg, int wide) {
   g.tile_start = tile_start;
-  g.tiles_n = (g.N + BN - 1) / BN;
+  g.tiles_n = (g.N + (wide ? 2 : 1) * BN - 1) / ((wide ? 2 : 1) * BN);
   // band height: at least 8 row tiles, more while the band's row panels (tile rows x K) stay within ~32 MB of L2
   const long long panel = (long long)BM * cg * g.K * 2;
   g.raster = (int)std::max(8LL, std::min(4096LL, (32LL << 20) / std::max(panel, 1LL)));
@@ -929,25 +965,29 @@ bool gemm_tc_encode(GemmProb& g, void* maps, int cg) {
 }
 
 cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int nprob, int total_tiles, int* d_status,
-                           int num_sms, cudaStream_t s, int cg) {
-  static bool attr_set[3] = {false, false, false};
-  size_t smem = (cg == 2 ? Cfg<2>::STAGES * Cfg<2>::STAGE_BYTES : Cfg<1>::STAGES * Cfg<1>::STAGE_BYTES) + EPI_WARPS * 4096 + 1024 + sizeof(Shared);
-  if (!attr_set[cg]) {
-    cudaError_t e = cg == 2 ? cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                            : cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                           int num_sms, cudaStream_t s, int cg, int wide) {
+  static bool attr_set[4] = {false, false, false, false};
+  const int which = cg == 1 ? 1 : (wide ? 3 : 2);
+  const size_t ring = cg == 1 ? (size_t)Cfg<1, 0>::STAGES * Cfg<1, 0>::STAGE_BYTES
+                              : (wide ? (size_t)Cfg<2, 1>::STAGES * Cfg<2, 1>::STAGE_BYTES : (size_t)Cfg<2, 0>::STAGES * Cfg<2, 0>::STAGE_BYTES);
+  size_t smem = ring + EPI_WARPS * 4096 + 1024 + sizeof(Shared);
+  if (cg == 1 && wide) return cudaErrorInvalidValue;
+  if (!attr_set[which]) {
+    const void* fn = which == 1 ? (const void*)gemm_tc_kernel<1, 0> : which == 2 ? (const void*)gemm_tc_kernel<2, 0> : (const void*)gemm_tc_kernel<2, 1>;
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // The epilogue warpgroups' register increase must fit into what the launch allocates (threads x
     // compiled register count); otherwise it would wait forever.  Refuse to launch instead.
     cudaFuncAttributes fa;
-    e = cg == 2 ? cudaFuncGetAttributes(&fa, gemm_tc_kernel<2>) : cudaFuncGetAttributes(&fa, gemm_tc_kernel<1>);
+    e = cudaFuncGetAttributes(&fa, fn);
     if (e != cudaSuccess) return e;
     if (32 * EPI_FIRST * CTRL_REGS + 32 * EPI_WARPS * EPI_REGS > NTHREADS * fa.numRegs) return cudaErrorLaunchOutOfResources;
-    attr_set[cg] = true;
+    attr_set[which] = true;
   }
   if (total_tiles == 0) return cudaSuccess;
   if (cg == 1) {
     int grid = total_tiles < num_sms ? total_tiles : num_sms;
-    gemm_tc_kernel<1><<<grid, NTHREADS, smem, s>>>(d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
+    gemm_tc_kernel<1, 0><<<grid, NTHREADS, smem, s>>>(d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
     return cudaGetLastError();
   }
   int pairs = num_sms / 2;
@@ -964,7 +1004,8 @@ cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int npro
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2>, d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
+  if (wide) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 1>, d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 0>, d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
 }
 
 }  // namespace lp

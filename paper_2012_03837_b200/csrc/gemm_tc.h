@@ -10,12 +10,15 @@ bool gemm_tc_eligible(const GemmProb& g);
 // Fill tile_start / tiles_n for 128x256 tiles; returns the number of tiles of this problem.
 // cg = 1: one CTA per 128x256 tile; cg = 2: a pair of CTAs per 256x256 tile (tcgen05 cta_group::2).
 int gemm_tc_choose_cg(const GemmProb* probs, int n);
-int gemm_tc_tiles(GemmProb& g, int tile_start, int cg = 1);
+int gemm_tc_tiles(GemmProb& g, int tile_start, int cg = 1, int wide = 0);
+// True if the problem may run with 256x512 tiles per CTA pair (wide = 1): a long reduction (K >= 8192) with a
+// plain epilogue and N a multiple of 512; such problems go into a launch of their own with cg = 2.
+bool gemm_tc_wide_ok(const GemmProb& g);
 // Encode the four TMA tensor maps [A, B, C, C2] of a problem (128 bytes each, 64-byte aligned host memory);
 // sets g.store_tma when the output's pitch lets the epilogue leave through TMA stores.
 bool gemm_tc_encode(GemmProb& g, void* maps4, int cg = 1);
 // d_maps: device array of 4*nprob tensor maps, [A0, B0, C0, C2_0, A1, ...].
 cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int nprob, int total_tiles, int* d_status,
-                           int num_sms, cudaStream_t s, int cg = 1);
+                           int num_sms, cudaStream_t s, int cg = 1, int wide = 0);
 
 }  // namespace lp

@@ -527,7 +527,7 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream,
   static void* d_tab = nullptr;
   static size_t d_cap = 0;
   struct alignas(64) Map { unsigned char b[128]; };
-  size_t need = 256 + tc.size() * sizeof(GemmProb) + 256 + 4 * tc.size() * sizeof(Map) + simt.size() * sizeof(GemmProb) + 256;
+  size_t need = 1024 + tc.size() * sizeof(GemmProb) + 256 + 4 * tc.size() * sizeof(Map) + simt.size() * sizeof(GemmProb) + 256;
   if (need > d_cap) {
     cudaStreamSynchronize(s);
     if (d_tab) cudaFree(d_tab);
@@ -536,19 +536,23 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream,
   }
   char* cur = (char*)d_tab;
   auto take = [&](size_t bytes) { char* r = cur; cur += (bytes + 255) / 256 * 256; return r; };
-  if (!tc.empty()) {
+  std::vector<GemmProb> lists[2];                       // [1]: long reductions that take the wide tiles
+  for (auto& g : tc) lists[gemm_tc_wide_ok(g) ? 1 : 0].push_back(g);
+  for (int wide = 0; wide < 2; ++wide) {
+    std::vector<GemmProb>& list = lists[wide];
+    if (list.empty()) continue;
     int total = 0;
-    const int cg = gemm_tc_choose_cg(tc.data(), (int)tc.size());
-    for (auto& g : tc) total += gemm_tc_tiles(g, total, cg);
-    std::vector<Map> maps(4 * tc.size());
-    for (size_t i = 0; i < tc.size(); ++i)
-      if (!gemm_tc_encode(tc[i], &maps[4 * i], cg)) return fail(nullptr, LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
-    GemmProb* dp = (GemmProb*)take(tc.size() * sizeof(GemmProb));
+    const int cg = wide ? 2 : gemm_tc_choose_cg(list.data(), (int)list.size());
+    for (auto& g : list) total += gemm_tc_tiles(g, total, cg, wide);
+    std::vector<Map> maps(4 * list.size());
+    for (size_t i = 0; i < list.size(); ++i)
+      if (!gemm_tc_encode(list[i], &maps[4 * i], cg)) return fail(nullptr, LP_ERR_CUDA, "cuTensorMapEncodeTiled failed");
+    GemmProb* dp = (GemmProb*)take(list.size() * sizeof(GemmProb));
     Map* dm = (Map*)take(maps.size() * sizeof(Map));
-    cudaMemcpyAsync(dp, tc.data(), tc.size() * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
+    cudaMemcpyAsync(dp, list.data(), list.size() * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
     cudaMemcpyAsync(dm, maps.data(), maps.size() * sizeof(Map), cudaMemcpyHostToDevice, s);
     cudaStreamSynchronize(s);
-    launch_gemm_tc(dp, dm, (int)tc.size(), total, d_status, num_sms, s, cg);
+    launch_gemm_tc(dp, dm, (int)list.size(), total, d_status, num_sms, s, cg, wide);
   }
   if (!simt.empty()) {
     int t = 0;

@@ -142,26 +142,42 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
     else if (g.conv != CONV_NONE) throw std::runtime_error("internal: implicit convolution problem not accepted by the tensor-core kernel");
     else simt.push_back(g);
   }
-  if (!tc.empty()) {
+  // Long reductions with a plain epilogue run with 256x512 tiles per CTA pair in a launch of their own
+  std::vector<GemmProb> wide_list, normal_list;
+  for (auto& g : tc) (gemm_tc_wide_ok(g) ? wide_list : normal_list).push_back(g);
+  {
+    // ... provided they fill the CTA pairs for a few even waves; a short or ragged wide launch loses more to its
+    // tail than the tile shape gains
+    long long tiles = 0;
+    for (auto& g : wide_list) tiles += (long long)((g.M + 255) / 256) * ((g.N + 511) / 512);
+    const long long pairs = std::max(1, h.num_sms / 2), waves = (tiles + pairs - 1) / pairs;
+    if (!wide_list.empty() && (waves < 3 || (double)tiles / (double)(waves * pairs) < 0.9)) {
+      normal_list.insert(normal_list.end(), wide_list.begin(), wide_list.end());
+      wide_list.clear();
+    }
+  }
+  for (int wide = 0; wide < 2; ++wide) {
+    std::vector<GemmProb>& list = wide ? wide_list : normal_list;
+    if (list.empty()) continue;
     // Longest tiles (largest K) first: the persistent CTAs take tiles in list order, so the long ones do not
     // end up in the tail, and products that walk the same operand in different directions (a weight
     // gradient and an input gradient reading the same dy) are not interleaved in the cache.
-    std::stable_sort(tc.begin(), tc.end(), [](const GemmProb& a, const GemmProb& b) { return a.K > b.K; });
+    std::stable_sort(list.begin(), list.end(), [](const GemmProb& a, const GemmProb& b) { return a.K > b.K; });
     int total = 0;
-    const int cg = gemm_tc_choose_cg(tc.data(), (int)tc.size());
-    for (auto& g : tc) total += gemm_tc_tiles(g, total, cg);
+    const int cg = wide ? 2 : gemm_tc_choose_cg(list.data(), (int)list.size());
+    for (auto& g : list) total += gemm_tc_tiles(g, total, cg, wide);
     struct alignas(64) Map { unsigned char b[128]; };
-    std::vector<Map> maps(4 * tc.size());
-    for (size_t i = 0; i < tc.size(); ++i)
-      if (!gemm_tc_encode(tc[i], &maps[4 * i], cg)) throw std::runtime_error("cuda: cuTensorMapEncodeTiled failed");
-    const GemmProb* d = h.upload(tc);
+    std::vector<Map> maps(4 * list.size());
+    for (size_t i = 0; i < list.size(); ++i)
+      if (!gemm_tc_encode(list[i], &maps[4 * i], cg)) throw std::runtime_error("cuda: cuTensorMapEncodeTiled failed");
+    const GemmProb* d = h.upload(list);
     const void* dm = h.upload(maps);
-    int n = (int)tc.size();
+    int n = (int)list.size();
     int* st = h.d_status;
     int sms = h.num_sms;
     double fl = 0;
-    for (auto& g : tc) fl += 2.0 * g.M * g.N * g.K;
-    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream, cg); }, KIND_GEMM_TC, fl);
+    for (auto& g : list) fl += 2.0 * g.M * g.N * g.K;
+    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream, cg, wide); }, KIND_GEMM_TC, fl);
   }
   if (!simt.empty()) {
     int t = 0;

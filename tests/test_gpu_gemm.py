@@ -45,7 +45,10 @@ def check(t, ref, tag):
 
 
 @pytest.mark.parametrize("backend", [1, 0])
-@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 128), (200, 264, 72), (1000, 520, 328), (136, 1000, 2048)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 128), (200, 264, 72), (1000, 520, 328), (136, 1000, 2048),
+                                   # long reductions with 512-column outputs: the 256x512 tiles (input gradient over
+                                   # 8192 columns; weight gradient over 8200 rows, ragged last k-slice)
+                                   (264, 8192, 512), (8200, 512, 1024)])
 def test_linear_products(M, N, K, backend):
     rng = np.random.default_rng(M + N + K)
     t, descs, ref = problems(M, N, K, rng)
