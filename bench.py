@@ -54,10 +54,11 @@ def describe(cfg):
 # capture summarised under profiles/ and scaled to the launches of a full step.  A figure is only
 # valid for the kernel source it was captured on: it is dropped when that file has changed since.
 TRAFFIC = {
-    # the ten grouped GEMM launches of a one-chunk c5 step move 3.31 GB through DRAM (ncu); every chunk streams its
-    # own operands, so a 24-chunk step moves 24 x 3.31 GB over its ten launches
-    "c5": dict(bytes_per_launch=7.9e9, chunks=24, kernel_file="paper_2012_03837_b200/csrc/gemm_tc.cu",
-               kernel_sha256="baa97055c45470f190829b22031d4777ef3b22a178b03d72424b3005b4d26645"),
+    # per chunk (ncu): head products 1.95 GB (forward 0.56, input gradient 0.61 and weight gradient 0.77 on the
+    # 256x512 tiles), block products 0.77 GB; every chunk streams its own operands, so a 24-chunk step moves
+    # 24 x 2.72 GB = 65 GB over its thirteen GEMM launches
+    "c5": dict(bytes_per_launch=5.0e9, chunks=24, kernel_file="paper_2012_03837_b200/csrc/gemm_tc.cu",
+               kernel_sha256="297e441f4f44da6405351899d1b9ac3f3e38f2c6dc30d61729045443ce7d9930"),
 }
 
 
