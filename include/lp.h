@@ -30,7 +30,7 @@ enum {
   LP_OK = 0,
   LP_ERR_INVALID_ARG = -1, /* null pointer, bad enum, bad index                                  */
   LP_ERR_SHAPE = -2,       /* sizes that the model family cannot take (see lp_model_spec)        */
-  LP_ERR_UNSUPPORTED = -3, /* valid request that this build does not implement                   */
+  LP_ERR_UNSUPPORTED = -3, /* valid request that the library does not implement                 */
   LP_ERR_ALLOC = -4,       /* device allocation failed                                           */
   LP_ERR_CUDA = -5,        /* a CUDA call failed; message holds the CUDA error string            */
   LP_ERR_STATE = -6,       /* call not allowed in the handle's current state                     */
@@ -315,6 +315,53 @@ enum {
 };
 lp_status lp_profile_enable(lp_handle h, int on);
 lp_status lp_profile_read(lp_handle h, double* ms, double* work, int* launches);
+
+/*
+ * FLOP cost model (App. A): what a training run costs in total FLOPs and in sequential FLOPs, the
+ * paper's stand-in for time on ideal hardware.  Host arithmetic only; no device is touched.
+ *
+ * App. A.2 describes a model by its layer count, the forward cost of one layer per example, the cost
+ * of one auxiliary loss per example, the backward multiplier (backward cost / forward cost) and its
+ * parameter count (the optimizer costs ten FLOPs per parameter per step).  The methods:
+ *   BACKPROP     one forward and backward pass, one loss; examples are the only parallelism.
+ *   GREEDY       one auxiliary loss per layer; layers and examples run in parallel.
+ *   OVERLAPPING  as GREEDY, with a second backward pass through all layers but the last and two more
+ *                FLOPs per parameter per step for averaging the two gradients.
+ *   CHUNKED      `chunks` blocks, one auxiliary loss each; blocks and examples run in parallel.
+ *   LAST_LAYERS  back-propagation through the last `chunks` layers only.
+ * Two of the printed per-example formulas are garbled (CHUNKED lacks the layer count, LAST_LAYERS an
+ * addition sign); they are read by analogy with BACKPROP.
+ * total_flops = cost_per_example * steps * batch_size + steps * optimizer cost;
+ * sequential_flops = total_flops / (batch_size * parallelism).
+ * Errors: INVALID_ARG (null pointer, unknown method), SHAPE (negative sizes, chunks outside
+ * [1, layers] for the two methods that use it).
+ *
+ * lp_mlp_layer_flops / lp_mlp_aux_flops are App. A.1's per-example counts for one fully connected
+ * layer with ReLU (input_size -> units) and for a linear classifier with softmax cross-entropy
+ * (units -> classes); they give forward_cost and aux_cost for the MLP family.
+ */
+enum { LP_COST_BACKPROP = 0, LP_COST_GREEDY = 1, LP_COST_OVERLAPPING = 2, LP_COST_CHUNKED = 3,
+       LP_COST_LAST_LAYERS = 4 };
+typedef struct {
+  int method;                 /* LP_COST_*                                        */
+  long long layers;           /* layers (or residual / transformer blocks)        */
+  long long chunks;           /* K for CHUNKED and LAST_LAYERS, ignored otherwise */
+  long long batch_size;       /* examples per step                                */
+  long long steps;            /* optimizer steps of the run                       */
+  double forward_cost;        /* FLOPs of one layer's forward pass, per example   */
+  double aux_cost;            /* FLOPs of one auxiliary loss, per example         */
+  double backward_multiplier; /* backward FLOPs / forward FLOPs                   */
+  double parameters;          /* parameters of the whole model                    */
+} lp_cost_spec;
+typedef struct {
+  double cost_per_example; /* FLOPs of one step for one example, optimizer excluded */
+  double total_flops;
+  double parallelism;      /* units of work that can run at once, per example       */
+  double sequential_flops;
+} lp_cost_result;
+lp_status lp_cost_model(const lp_cost_spec* spec, lp_cost_result* out);
+double lp_mlp_layer_flops(long long input_size, long long units);
+double lp_mlp_aux_flops(long long units, long long classes);
 
 /* Number of kernel launches the last lp_step issued (for reporting). */
 int lp_last_step_launches(lp_handle h);

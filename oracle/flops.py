@@ -37,7 +37,27 @@ def cost_per_example(method: str, forward_cost: float, aux_cost: float, backward
         return ((forward_cost + aux_cost) * layers
                 + (layers - 1) * bm * (2 * forward_cost + aux_cost)
                 + bm * (forward_cost + aux_cost))
+    if method == "last_layers":
+        # full forward pass and one loss, backward pass through the last `chunks` layers only (the printed
+        # formula lacks the "+" between the forward and the auxiliary cost)
+        return (layers * forward_cost + aux_cost) + bm * (chunks * forward_cost + aux_cost)
     raise ValueError(method)
+
+
+def total_cost(method: str, per_example: float, steps: int, batch_size: int, parameters: float) -> float:
+    """Total FLOPs of a run (App. A.2): the optimizer costs ten FLOPs per parameter per step, and the
+    overlapping method two more per parameter for averaging the shared layers' gradients."""
+    optimizer = 10 * parameters + (2 * parameters if method == "overlapping" else 0)
+    return per_example * steps * batch_size + steps * optimizer
+
+
+def parallelism(method: str, layers: int, chunks: int = 1, backward_multiplier: float = 0.0) -> float:
+    """Units that run at once per example (App. A.2); for "last_layers" the trained tail of `chunks`
+    layers is the atomic unit and the remaining forward work is cut into pieces of that size."""
+    if method == "last_layers":
+        bm = backward_multiplier
+        return (layers + chunks * bm) / (chunks * (1 + bm))
+    return {"backprop": 1, "greedy": layers, "overlapping": layers, "chunked": chunks}[method]
 
 
 def sequential_time(method: str, cost: float, batch_size: int, layers: int, chunks: int = 1) -> float:

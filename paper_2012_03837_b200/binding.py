@@ -60,7 +60,8 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
-           "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap"]
+           "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap",
+           "lp_cost_model", "lp_mlp_layer_flops", "lp_mlp_aux_flops"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
 
@@ -323,3 +324,43 @@ def lp_gemm_bf16_static(descs: list, stream=None) -> None:
     code = _lib.lp_gemm_bf16_static(len(descs), arr, stream)
     if code != LP_OK:
         raise LpError(code, (_lib.lp_gemm_static_last_error() or b"").decode())
+
+
+# ---- FLOP cost model (App. A): host arithmetic in the library, no device needed -------------------------
+LP_COST_METHODS = {"backprop": 0, "greedy": 1, "overlapping": 2, "chunked": 3, "last_layers": 4}
+
+
+class lp_cost_spec(C.Structure):
+    _fields_ = [("method", C.c_int), ("layers", C.c_longlong), ("chunks", C.c_longlong),
+                ("batch_size", C.c_longlong), ("steps", C.c_longlong), ("forward_cost", C.c_double),
+                ("aux_cost", C.c_double), ("backward_multiplier", C.c_double), ("parameters", C.c_double)]
+
+
+class lp_cost_result(C.Structure):
+    _fields_ = [("cost_per_example", C.c_double), ("total_flops", C.c_double), ("parallelism", C.c_double),
+                ("sequential_flops", C.c_double)]
+
+
+_lib.lp_cost_model.argtypes = [C.POINTER(lp_cost_spec), C.POINTER(lp_cost_result)]
+_lib.lp_cost_model.restype = C.c_int
+_lib.lp_mlp_layer_flops.argtypes = [C.c_longlong, C.c_longlong]
+_lib.lp_mlp_layer_flops.restype = C.c_double
+_lib.lp_mlp_aux_flops.argtypes = [C.c_longlong, C.c_longlong]
+_lib.lp_mlp_aux_flops.restype = C.c_double
+
+
+def lp_cost_model(method: str, layers: int, batch_size: int, steps: int, forward_cost: float, aux_cost: float,
+                  backward_multiplier: float, parameters: float, chunks: int = 1) -> dict:
+    spec = lp_cost_spec(LP_COST_METHODS[method], layers, chunks, batch_size, steps, forward_cost, aux_cost,
+                        backward_multiplier, parameters)
+    out = lp_cost_result()
+    _check(None, _lib.lp_cost_model(C.byref(spec), C.byref(out)))
+    return {k: getattr(out, k) for k, _ in lp_cost_result._fields_}
+
+
+def lp_mlp_layer_flops(input_size: int, units: int) -> float:
+    return _lib.lp_mlp_layer_flops(input_size, units)
+
+
+def lp_mlp_aux_flops(units: int, classes: int) -> float:
+    return _lib.lp_mlp_aux_flops(units, classes)
