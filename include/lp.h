@@ -42,7 +42,7 @@ enum {
 enum { LP_FAMILY_MLP = 0, LP_FAMILY_LM = 1, LP_FAMILY_RESNET = 2 };
 enum { LP_FP32 = 0, LP_BF16 = 1 }; /* LP_BF16: bf16 matrices and activations, fp32 master weights,
                                       fp32 accumulation, fp32 normalisation statistics and loss  */
-enum { LP_HEAD_LINEAR = 0, LP_HEAD_LN_LINEAR = 1, LP_HEAD_GAP_LINEAR = 2 };
+enum { LP_HEAD_LINEAR = 0, LP_HEAD_LN_LINEAR = 1, LP_HEAD_GAP_LINEAR = 2, LP_HEAD_BN_RELU_GAP_LINEAR = 3 };
 enum { LP_OPT_SGDM = 0, LP_OPT_ADAM = 1 };
 enum { LP_SYNC = 0, LP_PIPELINED = 1 };
 enum { LP_MASTER = 0, LP_WORKING = 1, LP_MOMENT1 = 2, LP_MOMENT2 = 3, LP_GRAD = 4 };
@@ -85,7 +85,9 @@ typedef struct {
 
 /* Auxiliary head of every chunk (Sec. 3: same form as the global objective): softmax
  * cross-entropy over `classes` on top of Linear (MLP), LayerNorm+Linear (LM; classes = vocab) or
- * global-average-pool+Linear (RESNET). */
+ * global-average-pool+Linear (RESNET).  RESNET also takes LP_HEAD_BN_RELU_GAP_LINEAR, the head of
+ * App. B.3: BatchNorm (own scale, shift and running statistics per chunk, tensors
+ * "c<k>.head.bn.{g,b,rm,rv}") and ReLU on the stage output before the spatial mean. */
 typedef struct {
   int kind;
   int classes;

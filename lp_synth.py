@@ -180,6 +180,9 @@ def param_table(cfg: dict) -> list[dict]:
             c_prev = c
             add(f"c{k}.head.W", k, (cfg["classes"], c), "normal", np.sqrt(1.0 / c), True)
             add(f"c{k}.head.b", k, (cfg["classes"],), "zeros")
+            if cfg.get("head") == "bn_relu_gap":
+                add(f"c{k}.head.bn.g", k, (c,), "ones")
+                add(f"c{k}.head.bn.b", k, (c,), "zeros")
         for t in [t for t in out if t["name"].endswith(".g") and ".bn" in t["name"]]:
             stem = t["name"][:-2]
             add(stem + ".rm", t["chunk"], t["shape"], "zeros", buffer=True)

@@ -83,8 +83,10 @@ class LocalUpdateOracle:
             return self._lm_bwd(k, dout, cache)
         return self._resnet_bwd(k, dout, cache)
 
-    def head(self, k, h, y):
-        """Auxiliary head of chunk k on the chunk output h: (loss, logits, dh, head gradients)."""
+    def head(self, k, h, y, training=False):
+        """Auxiliary head of chunk k on the chunk output h: (loss, logits, dh, head gradients).  The ResNet
+        head is spatial mean + Linear, or, with cfg["head"] == "bn_relu_gap", App. B.3's BatchNorm -> ReLU ->
+        spatial mean -> Linear (its BatchNorm follows self.bn_mode; under running statistics dh is None)."""
         fam = self.cfg["family"]
         p = self.p
         g = {}
@@ -100,11 +102,25 @@ class LocalUpdateOracle:
             da, g[f"c{k}.head.W"], g[f"c{k}.head.b"] = L.linear_bwd(dz, c)
             dh, g[f"c{k}.head.ln.g"], g[f"c{k}.head.ln.b"] = L.layernorm_bwd(da.reshape(b, t, d), cln)
         else:
-            a, cg = L.gap_fwd(h)
+            bn_head = self.cfg.get("head") == "bn_relu_gap"
+            r = h
+            if bn_head:
+                self.training = training
+                try:
+                    u, cb = self._bn(h, f"c{k}.head.bn")
+                finally:
+                    self.training = False
+                r, cr = L.relu_fwd(u)
+            a, cg = L.gap_fwd(r)
             z, c = L.linear_fwd(a, p[f"c{k}.head.W"], p[f"c{k}.head.b"])
             loss, dz = L.softmax_xent(z, y)
             da, g[f"c{k}.head.W"], g[f"c{k}.head.b"] = L.linear_bwd(dz, c)
             dh = L.gap_bwd(da, cg)
+            if bn_head:
+                if cb is None:
+                    return loss, z, None, {}
+                du = L.relu_bwd(dh, cr)
+                dh, g[f"c{k}.head.bn.g"], g[f"c{k}.head.bn.b"] = L.batchnorm_bwd(du, cb)
         return loss, z, dh, g
 
     # MLP chunk: a run of Linear + ReLU layers (App. A.1).
@@ -261,7 +277,7 @@ class LocalUpdateOracle:
             h, cache = self.chunk_forward(k, inp)
         finally:
             self.training = False
-        loss, _, dh, g = self.head(k, h, y)
+        loss, _, dh, g = self.head(k, h, y, training=True)
         g.update(self.chunk_backward(k, dh, cache))
         self._last_cache = cache
         return loss, h, g
@@ -368,15 +384,14 @@ class LocalUpdateOracle:
         out = []
         self.bn_mode = bn        # "running": BatchNorm uses its running statistics instead of this minibatch's
         try:
-            hs = []
+            heads = []
             for k in range(self.K):
                 h, _ = self.chunk_forward(k, h)
-                hs.append(h)
+                heads.append(self.head(k, h, y))
         finally:
             self.bn_mode = "batch"
         for k in range(self.K):
-            h = hs[k]
-            loss, z, _, _ = self.head(k, h, y)
+            loss, z, _, _ = heads[k]
             z2 = z.reshape(-1, z.shape[-1])
             pred = np.argmax(z2, axis=1).astype(np.int32)
             lab = np.asarray(y).reshape(-1)

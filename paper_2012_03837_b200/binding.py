@@ -19,7 +19,7 @@ LP_ERR = {-1: "INVALID_ARG", -2: "SHAPE", -3: "UNSUPPORTED", -4: "ALLOC", -5: "C
           -7: "LABEL_RANGE", -8: "NONFINITE", -9: "TIMEOUT"}
 LP_FAMILY_MLP, LP_FAMILY_LM, LP_FAMILY_RESNET = 0, 1, 2
 LP_FP32, LP_BF16 = 0, 1
-LP_HEAD_LINEAR, LP_HEAD_LN_LINEAR, LP_HEAD_GAP_LINEAR = 0, 1, 2
+LP_HEAD_LINEAR, LP_HEAD_LN_LINEAR, LP_HEAD_GAP_LINEAR, LP_HEAD_BN_RELU_GAP_LINEAR = 0, 1, 2, 3
 LP_OPT_SGDM, LP_OPT_ADAM = 0, 1
 LP_SYNC, LP_PIPELINED = 0, 1
 LP_MASTER, LP_WORKING, LP_MOMENT1, LP_MOMENT2, LP_GRAD = 0, 1, 2, 3, 4
@@ -155,7 +155,8 @@ def specs_from_config(cfg: dict, gemm_backend: int = 0):
         keep.append(a)
         m.stage_channels = a
         K = len(cfg["stage_channels"])
-        hd.kind, hd.classes = LP_HEAD_GAP_LINEAR, cfg["classes"]
+        hd.kind = LP_HEAD_BN_RELU_GAP_LINEAR if cfg.get("head") == "bn_relu_gap" else LP_HEAD_GAP_LINEAR
+        hd.classes = cfg["classes"]
     o = cfg["optim"]
     op = lp_optim_spec()
     if o["kind"] == "sgdm":

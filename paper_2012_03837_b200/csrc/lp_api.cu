@@ -66,7 +66,8 @@ void validate(const lp_model_spec* m, int K, const lp_head_spec* hd, const lp_op
       break;
     }
     case LP_FAMILY_RESNET: {
-      if (hd->kind != LP_HEAD_GAP_LINEAR) throw std::invalid_argument("RESNET takes LP_HEAD_GAP_LINEAR");
+      if (hd->kind != LP_HEAD_GAP_LINEAR && hd->kind != LP_HEAD_BN_RELU_GAP_LINEAR)
+        throw std::invalid_argument("RESNET takes LP_HEAD_GAP_LINEAR or LP_HEAD_BN_RELU_GAP_LINEAR");
       if (!m->stage_channels) throw std::invalid_argument("null stage_channels");
       if (m->in_channels < 1 || m->height < 1 || m->width < 1 || m->stem_channels < 1 || m->blocks_per_stage < 1)
         throw ShapeError("RESNET sizes must be positive");

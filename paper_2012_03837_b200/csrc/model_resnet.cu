@@ -48,6 +48,8 @@ struct Chunk {
   std::vector<Block> blocks;
   int C, Hout, Wout;
   void *pool, *z, *dpool;
+  Bn head_bn;                                  // LP_HEAD_BN_RELU_GAP_LINEAR: BatchNorm + ReLU in front of the pool
+  void* hact = nullptr;                        // its output
   float* row_loss;
   void* G[4];
   void* dcols;
@@ -88,6 +90,7 @@ Conv make_conv(const std::string& w, int N, int H, int W, int Cin, int Cout, int
 void build_resnet(Handle& h) {
   const int K = h.K, B = h.spec.batch, NC = h.head.classes;
   const bool bf = h.bf16_mode;
+  const bool head_bn = h.head.kind == LP_HEAD_BN_RELU_GAP_LINEAR;   // App. B.3's head
   const size_t es = h.esize();
   std::vector<Chunk> ch(K);
   int H = h.spec.height, W = h.spec.width, cprev = h.spec.stem_channels;
@@ -133,6 +136,11 @@ void build_resnet(Handle& h) {
     c.C = cout; c.Hout = H; c.Wout = W;
     h.add_tensor(ck + ".head.W", k, {NC, cout}, true);
     h.add_tensor(ck + ".head.b", k, {NC}, false);
+    if (head_bn) {
+      h.add_tensor(ck + ".head.bn.g", k, {cout}, false);
+      h.add_tensor(ck + ".head.bn.b", k, {cout}, false);
+      c.head_bn = Bn{ck + ".head.bn.g", ck + ".head.bn.b", cout, (long long)B * H * W, nullptr, nullptr};
+    }
   }
   // running mean / variance of every BatchNorm: state no gradient reaches (their gradient entries stay
   // zero, so the optimizer sweep leaves them alone); they live in the arena so that tensor access and
@@ -200,6 +208,7 @@ void build_resnet(Handle& h) {
       if (b.has_sc) { alloc_conv(b.cs); alloc_bn(b.bs); track(b.cs); b.sc = h.dalloc((size_t)b.cs.M * b.cs.Cout * es); }
       if (j + 1 < c.blocks.size()) b.out = h.dalloc((size_t)b.c2.M * b.c2.Cout * es);
     }
+    if (head_bn) { alloc_bn(c.head_bn); c.hact = h.dalloc(out_bytes); }
     c.pool = h.dalloc((size_t)B * c.C * es);
     c.dpool = h.dalloc((size_t)B * c.C * es);
     c.z = h.dalloc((size_t)B * NC * es);
@@ -295,10 +304,11 @@ void build_resnet(Handle& h) {
     }
   };
 
-  auto head_forward = [&](Plan& p, int k, int wr, const int* labels, bool copy_logits) {
+  auto head_forward = [&](Plan& p, int k, int wr, const int* labels, bool copy_logits, int mode) {
     Chunk& c = ch[k];
     const std::string ck = "c" + std::to_string(k);
-    GapProb gp{h.bnd[wr][k], c.pool, nullptr, nullptr, B, c.Hout * c.Wout, c.C};
+    if (head_bn) bn_fwd(p, c.head_bn, h.bnd[wr][k], c.hact, nullptr, true, mode);
+    GapProb gp{head_bn ? c.hact : h.bnd[wr][k], c.pool, nullptr, nullptr, B, c.Hout * c.Wout, c.C};
     const GapProb* dg = h.upload(std::vector<GapProb>{gp});
     int C = c.C;
     p.add(1, [=](const RunCtx& r) { launch_gap_fwd(dg, 1, B, C, bf, r.stream); }, KIND_CONV_AUX, (double)B * c.Hout * c.Wout * c.C * es);
@@ -427,8 +437,10 @@ void build_resnet(Handle& h) {
     rec_gemm(L, {gemm_wgrad(c.z, c.pool, h.G(ck + ".head.W"), B, NC, c.C),
                  gemm_dgrad(c.z, h.W(ck + ".head.W"), c.dpool, B, NC, c.C, EPI_NONE, nullptr)});
     { Op o; o.kind = OP_COLSUM; o.colsum = ColSumProb{c.z, nullptr, B, NC, NC}; o.colsum_out = h.G(ck + ".head.b"); L.push_back(std::move(o)); }
-    { Op o; o.kind = OP_GAP_BWD; o.gap = GapProb{nullptr, nullptr, c.dpool, c.G[0], B, c.Hout * c.Wout, c.C};
+    { Op o; o.kind = OP_GAP_BWD; o.gap = GapProb{nullptr, nullptr, c.dpool, head_bn ? c.G[3] : c.G[0], B, c.Hout * c.Wout, c.C};
       o.elems = (long long)B * c.Hout * c.Wout * c.C; L.push_back(std::move(o)); }
+    // head BatchNorm + ReLU: G[3] holds the gradient at their output, G[0] receives the one at the stage output
+    if (head_bn) rec_bn_bwd(L, c.head_bn, h.bnd[wr][k], c.G[3], c.hact, c.G[0], nullptr);
     void *gin = c.G[0], *ga = c.G[1], *gb = c.G[2], *gc = c.G[3];
     for (int j = (int)c.blocks.size() - 1; j >= 0; --j) {
       Block& b = c.blocks[j];
@@ -551,7 +563,7 @@ void build_resnet(Handle& h) {
       lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, B, NC, h.n_valid[k]});
     emit_labels(h, p, lps);
     for (int k = 0; k < K; ++k) forward_chunk(p, k, rd, wr, BN_TRAIN);
-    for (int k = 0; k < K; ++k) head_forward(p, k, wr, labels_of(k, pipelined, rd), false);
+    for (int k = 0; k < K; ++k) head_forward(p, k, wr, labels_of(k, pipelined, rd), false, BN_TRAIN);
     std::vector<OpList> lists(K);
     overlap_avg.clear();
     for (int k = 0; k < K; ++k) record_backward(lists[k], k, rd, wr, overlap);
@@ -574,7 +586,7 @@ void build_resnet(Handle& h) {
     std::vector<LabelProb> lps;
     for (int k = 0; k < K; ++k) lps.push_back(LabelProb{h.y_in, nullptr, B, NC, h.n_valid[k]});
     emit_labels(h, p, lps);
-    for (int k = 0; k < K; ++k) head_forward(p, k, wr, h.y_in, true);
+    for (int k = 0; k < K; ++k) head_forward(p, k, wr, h.y_in, true, mode);
   };
 
   h.has_eval_plan = true;

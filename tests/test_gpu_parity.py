@@ -410,3 +410,56 @@ def test_overlapping_updates_lm_bf16(backend):
     cfg = lp_synth.config("c3", batch=3, seq_len=136, vocab=1000, d_model=128, n_heads=2, d_ffn=320,
                           blocks_per_chunk=[1, 2, 1])
     check_overlap(cfg, gemm_backend=backend, shared_per_boundary=12)
+
+
+# ---------------------------------------------------------------- App. B.3's ResNet head: BatchNorm -> ReLU -> mean -> Linear
+
+@pytest.mark.parametrize("schedule", ["sync", "pipelined"])
+def test_resnet_fp32_batchnorm_head(schedule):
+    cfg = lp_synth.config("c4", dtype="fp32", batch=6, height=12, width=12, stem_channels=8,
+                          stage_channels=[8, 16, 24], blocks_per_stage=2, classes=5, schedule=schedule,
+                          head="bn_relu_gap")
+    check(cfg, w_tol=5e-3, v_tol=5e-2)
+
+
+def test_resnet_bf16_batchnorm_head_implicit_convolutions():
+    cfg = lp_synth.config("c4", batch=32, height=16, width=16, stem_channels=64,
+                          stage_channels=[64, 128], blocks_per_stage=2, classes=10, head="bn_relu_gap")
+    check(cfg, v_tol=0.3)
+
+
+def test_resnet_batchnorm_head_running_statistics_and_evaluation():
+    """The head's own BatchNorm keeps running statistics like every other one ("c<k>.head.bn.rm/.rv"), and
+    lp_evaluate on running statistics normalises the head with them."""
+    cfg = lp_synth.config("c4", batch=32, height=16, width=16, stem_channels=64,
+                          stage_channels=[64, 128], blocks_per_stage=2, classes=10, head="bn_relu_gap")
+    steps = 10
+    gl, ol, gm, orc = T.run_both(cfg, steps)
+    got = gm.get()
+    assert "c1.head.bn.rv" in orc.buffers and "c1.head.bn.rv" in got
+    worst = 0.0
+    for n in sorted(orc.buffers):
+        a, b = got[n].astype(np.float64), orc.p[n].astype(np.float64)
+        worst = max(worst, float(np.linalg.norm(a - b) / np.linalg.norm(b)))
+    assert worst <= 2e-2
+    x, y = lp_synth.minibatch(cfg, steps)
+    run_l, run_c, run_p = T.gpu_evaluate(gm, x, y, "running")
+    bat_l, _, _ = T.gpu_evaluate(gm, x, y, "batch")
+    ref_run = orc.evaluate(x, y, bn="running")
+    ref_bat = orc.evaluate(x, y)
+    print("worst l2 error of the running statistics", f"{worst:.2e}", "losses running", run_l,
+          [r["loss"] for r in ref_run], "batch", bat_l, [r["loss"] for r in ref_bat])
+    for k in range(len(ref_run)):
+        assert abs(run_l[k] - ref_run[k]["loss"]) <= 5e-2 * abs(ref_run[k]["loss"]), k
+        assert abs(bat_l[k] - ref_bat[k]["loss"]) <= 2e-2 * abs(ref_bat[k]["loss"]), k
+        assert run_c[k] == int(np.sum(run_p[k] == y.reshape(-1)))
+    again = gm.get()
+    for n in orc.buffers:
+        assert np.array_equal(got[n], again[n]), n
+    gm.close()
+
+
+def test_overlapping_updates_resnet_fp32_batchnorm_head():
+    cfg = lp_synth.config("c4", dtype="fp32", batch=6, height=12, width=12, stem_channels=8,
+                          stage_channels=[8, 16, 24], blocks_per_stage=2, classes=5, head="bn_relu_gap")
+    check_overlap(cfg, shared_per_boundary=None, w_tol=5e-3, v_tol=5e-2)

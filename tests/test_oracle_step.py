@@ -88,13 +88,18 @@ def torch_forward(cfg, P, x, upto=None):
     return h
 
 
-def torch_head_loss(cfg, P, k, h, y):
+def torch_head_loss(cfg, P, k, h, y, bn_buffers=None, bn_training=True):
+    """bn_buffers: (running means, running variances) by BatchNorm name, for the BatchNorm of App. B.3's head."""
     fam = cfg["family"]
     if fam == "lm":
         a = F.layer_norm(h, (cfg["d_model"],), P[f"c{k}.head.ln.g"], P[f"c{k}.head.ln.b"], 1e-5)
         z = F.linear(a, P[f"c{k}.head.W"], P[f"c{k}.head.b"])
         return F.cross_entropy(z.reshape(-1, z.shape[-1]), y.reshape(-1).long(), ignore_index=-1)
     if fam == "resnet":
+        if cfg.get("head") == "bn_relu_gap":
+            m = f"c{k}.head.bn"
+            rm, rv = (bn_buffers[0][m], bn_buffers[1][m]) if bn_buffers else (None, None)
+            h = F.relu(F.batch_norm(h, rm, rv, P[m + ".g"], P[m + ".b"], bn_training, 0.1, 1e-5))
         h = h.mean(dim=(2, 3))
     return F.cross_entropy(F.linear(h, P[f"c{k}.head.W"], P[f"c{k}.head.b"]), y.long())
 
@@ -412,6 +417,59 @@ def test_batchnorm_running_statistics_and_evaluation_mode_follow_the_library_rou
     for m in rm:
         assert np.array_equal(before[m], orc.p[m + ".rm"])
     assert abs(orc.evaluate(x3, y3)[0]["loss"] - ev[0]["loss"]) > 1e-6      # batch statistics give another loss
+
+
+def test_resnet_head_with_batchnorm_and_relu_follows_reverse_mode_and_the_library_buffers():
+    """App. B.3's auxiliary head (BatchNorm -> ReLU -> spatial mean -> Linear): every chunk's local gradient,
+    the head's own BatchNorm parameters included, against torch autograd of that chunk's loss with the chunk
+    input detached; the head BatchNorm's running statistics and the evaluation-mode loss against torch's
+    batch_norm buffers."""
+    cfg = lp_synth.config("c4", dtype="fp32", batch=4, height=6, width=6, stem_channels=4, stage_channels=[4, 8],
+                          blocks_per_stage=1, classes=3, head="bn_relu_gap")
+    params = spread_params(cfg)
+    assert "c0.head.bn.g" in params and "c1.head.bn.rv" in params
+    for n in params:
+        if n.endswith(".rm"):
+            params[n] = np.zeros_like(params[n])
+        if n.endswith(".rv"):
+            params[n] = np.ones_like(params[n])
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float64)
+    orc.cfg = dict(cfg, optim=dict(kind="sgdm", lr=0.0, momentum=0.0, weight_decay=0.0))
+    x, y = lp_synth.minibatch(cfg, 0)
+    orc.step(x, y, "sync")
+    # chunk 1 (last): full back-propagation of its loss; chunk 0: back-propagation of head 0's loss
+    for k in range(2):
+        _, tg = torch_backprop_grads(cfg, params, x, y, k)
+        for n in orc.names_of_chunk[k]:
+            if n in orc.buffers:
+                continue
+            assert tg[n] is not None, n
+            assert rel(orc.last_grads[n], tg[n]) < 1e-9, n
+    assert np.abs(orc.last_grads["c0.head.bn.g"]).max() > 1e-6
+    # running statistics of the head's BatchNorm after one step, closed form from (0, 1)
+    P = {n: torch.tensor(a, dtype=torch.float64) for n, a in params.items()}
+    h0 = torch_forward(cfg, P, torch.tensor(x, dtype=torch.float64), upto=0).numpy()
+    n = h0.shape[0] * h0.shape[2] * h0.shape[3]
+    assert np.allclose(orc.p["c0.head.bn.rm"], 0.1 * h0.mean(axis=(0, 2, 3)), rtol=1e-12, atol=1e-14)
+    assert np.allclose(orc.p["c0.head.bn.rv"], 0.9 + 0.1 * h0.var(axis=(0, 2, 3)) * n / (n - 1), rtol=1e-12)
+    # a forward pass or an evaluation moves nothing; evaluation on running statistics uses the head's buffers too
+    before = orc.p["c1.head.bn.rm"].copy()
+    orc.forward(x, y)
+    x1, y1 = lp_synth.minibatch(cfg, 1)
+    ev_run = orc.evaluate(x1, y1, bn="running")
+    ev_bat = orc.evaluate(x1, y1)
+    assert np.array_equal(before, orc.p["c1.head.bn.rm"])
+    assert abs(ev_run[0]["loss"] - ev_bat[0]["loss"]) > 1e-6
+    # chunk 0's evaluation loss on running statistics, rebuilt with torch from the oracle's buffers
+    Pn = {n: torch.tensor(a, dtype=torch.float64) for n, a in orc.p.items()}
+    bn = lambda v, m: F.batch_norm(v, Pn[m + ".rm"], Pn[m + ".rv"], Pn[m + ".g"], Pn[m + ".b"], False, 0.1, 1e-5)
+    h = F.relu(bn(F.conv2d(torch.tensor(x1, dtype=torch.float64), Pn["c0.stem.conv"], padding=1), "c0.stem.bn"))
+    v = F.relu(bn(F.conv2d(h, Pn["c0.r0.conv1"], padding=1), "c0.r0.bn1"))
+    v = bn(F.conv2d(v, Pn["c0.r0.conv2"], padding=1), "c0.r0.bn2")
+    h = F.relu(v + h)
+    bufs = ({"c0.head.bn": Pn["c0.head.bn.rm"]}, {"c0.head.bn": Pn["c0.head.bn.rv"]})
+    tl = float(torch_head_loss(cfg, Pn, 0, h, torch.tensor(y1), bufs, False))
+    assert abs(ev_run[0]["loss"] - tl) < 1e-10 * max(1.0, abs(tl))
 
 
 # ---------------------------------------------------------------- overlapping local parallelism (Sec. 3, Fig. 2 c)
