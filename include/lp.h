@@ -81,6 +81,12 @@ typedef struct {
   /* 0: tensor-core GEMMs wherever a problem's sizes allow (default); 1: plain FP32-ALU GEMMs
      everywhere (diagnostic).  The fp32 dtype always uses the FP32-ALU GEMMs. */
   int gemm_backend;
+  /* 0: x is raw data (token ids, NCHW images, MLP rows).  1: the model is an inner piece of a longer chain,
+     placed on its own GPU (Sec. 6: one block per device), and x is the activation the previous piece
+     produced, in the compute dtype: LM -- [batch, seq_len, d_model], no embedding tables; RESNET --
+     NHWC [batch, height, width, in_channels], no stem, and the first stage already starts with stride 2
+     and a 1x1 shortcut; MLP -- no difference.  No gradient is formed for x (Sec. 3). */
+  int input_is_activation;
 } lp_model_spec;
 
 /* Auxiliary head of every chunk (Sec. 3: same form as the global objective): softmax
@@ -197,6 +203,17 @@ lp_status lp_set_tensor(lp_handle h, int i, int which, const void* host_src, siz
 
 /* Forget the activations in flight between chunks; the next pipelined step starts the ramp-up again. */
 lp_status lp_reset_pipeline(lp_handle h);
+
+/*
+ * Output activation of chunk k as the last lp_step left it (the tensor the next chunk reads; Sec. 3: it
+ * carries no gradient), for handing it to the piece of the chain that lives on another GPU (Sec. 6).
+ * lp_chunk_output_bytes gives its size; layout: MLP [batch, width], LM [batch, seq_len, d_model], RESNET
+ * NHWC [batch, H_k, W_k, C_k], compute dtype.  lp_chunk_output copies it device-to-device into dst
+ * (device, caller-owned, at least that many bytes) on `stream`, without host synchronisation.
+ * Errors: INVALID_ARG (null, k outside [0, K), bytes too small), STATE (no step has run yet), CUDA.
+ */
+size_t lp_chunk_output_bytes(lp_handle h, int k);
+lp_status lp_chunk_output(lp_handle h, int k, void* dst, size_t bytes, void* stream);
 
 /*
  * lp_set_ramp: how the pipelined schedule starts after lp_create or lp_reset_pipeline (Sec. 6 speaks only

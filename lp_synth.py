@@ -134,7 +134,7 @@ def param_table(cfg: dict) -> list[dict]:
         s = 0.02
         blk = 0
         for k, nb in enumerate(cfg["blocks_per_chunk"]):
-            if k == 0:
+            if k == 0 and not cfg.get("input_is_activation"):
                 add("c0.tok", 0, (v, d), "normal", s, True)
                 add("c0.pos", 0, (t, d), "normal", s, True)
             for _ in range(nb):
@@ -158,9 +158,10 @@ def param_table(cfg: dict) -> list[dict]:
             add(f"c{k}.head.b", k, (v,), "zeros")
     elif fam == "resnet":
         cin = cfg["in_channels"]
-        c_prev = cfg["stem_channels"]
+        inner = bool(cfg.get("input_is_activation"))     # a later stage on its own: no stem, input = activation
+        c_prev = cin if inner else cfg["stem_channels"]
         for k, c in enumerate(cfg["stage_channels"]):
-            if k == 0:
+            if k == 0 and not inner:
                 add("c0.stem.conv", 0, (c_prev, cin, 3, 3), "normal", np.sqrt(2.0 / (cin * 9)), True)
                 add("c0.stem.bn.g", 0, (c_prev,), "ones")
                 add("c0.stem.bn.b", 0, (c_prev,), "zeros")
@@ -193,8 +194,8 @@ def param_table(cfg: dict) -> list[dict]:
 
 
 def resnet_stage_stride(cfg: dict, k: int) -> int:
-    """Stride of the first convolution of stage k: 1 for the first stage, 2 afterwards."""
-    return 1 if k == 0 else 2
+    """Stride of the first convolution of stage k: 1 for the network's first stage, 2 afterwards."""
+    return 1 if (k == 0 and not cfg.get("input_is_activation")) else 2
 
 
 # ----------------------------------------------------------------------------- random streams

@@ -39,7 +39,7 @@ class lp_model_spec(C.Structure):
                 ("d_ffn", C.c_int), ("blocks_per_chunk", C.POINTER(C.c_int)),
                 ("in_channels", C.c_int), ("height", C.c_int), ("width", C.c_int),
                 ("stem_channels", C.c_int), ("stage_channels", C.POINTER(C.c_int)),
-                ("blocks_per_stage", C.c_int), ("gemm_backend", C.c_int)]
+                ("blocks_per_stage", C.c_int), ("gemm_backend", C.c_int), ("input_is_activation", C.c_int)]
 
 
 class lp_head_spec(C.Structure):
@@ -61,7 +61,7 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
            "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap",
-           "lp_cost_model", "lp_mlp_layer_flops", "lp_mlp_aux_flops"]
+           "lp_cost_model", "lp_mlp_layer_flops", "lp_mlp_aux_flops", "lp_chunk_output_bytes", "lp_chunk_output"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
 
@@ -81,6 +81,9 @@ def load_library() -> C.CDLL:
     lib.lp_get_tensor.argtypes = [vp, ip, ip, vp, C.c_size_t, vp]
     lib.lp_set_tensor.argtypes = [vp, ip, ip, vp, C.c_size_t, vp]
     lib.lp_reset_pipeline.argtypes = [vp]
+    lib.lp_chunk_output_bytes.argtypes = [vp, ip]
+    lib.lp_chunk_output_bytes.restype = C.c_size_t
+    lib.lp_chunk_output.argtypes = [vp, ip, vp, C.c_size_t, vp]
     lib.lp_set_ramp.argtypes = [vp, ip]
     lib.lp_set_overlap.argtypes = [vp, ip]
     lib.lp_status_poll.argtypes = [vp, vp]
@@ -127,6 +130,7 @@ def specs_from_config(cfg: dict, gemm_backend: int = 0):
     m.dtype = LP_BF16 if cfg["dtype"] == "bf16" else LP_FP32
     m.batch = cfg["batch"]
     m.gemm_backend = gemm_backend
+    m.input_is_activation = 1 if cfg.get("input_is_activation") else 0
     hd = lp_head_spec()
     if fam == "mlp":
         m.family = LP_FAMILY_MLP
@@ -225,6 +229,14 @@ LP_RAMP_PRIME, LP_RAMP_IDLE = 0, 1
 
 def lp_set_ramp(h, ramp: int):
     _check(h, _lib.lp_set_ramp(h, ramp))
+
+
+def lp_chunk_output_bytes(h, k: int) -> int:
+    return _lib.lp_chunk_output_bytes(h, k)
+
+
+def lp_chunk_output(h, k: int, dst, nbytes: int, stream=None):
+    _check(h, _lib.lp_chunk_output(h, k, _ptr(dst), nbytes, stream))
 
 
 def lp_set_overlap(h, on: bool):

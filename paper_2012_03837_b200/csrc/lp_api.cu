@@ -181,6 +181,7 @@ lp_status run_step(Handle& h, int schedule, cudaStream_t s) {
     const Plan& plan = h.overlap ? h.sync_overlap_plan : h.sync_plan;
     plan.run(ctx);
     launches = plan.launches;
+    h.last_wr = 0;
   } else {
     if (!h.primed && h.ramp == LP_RAMP_PRIME) {
       h.prime_plan[h.parity].run(ctx);
@@ -193,6 +194,7 @@ lp_status run_step(Handle& h, int schedule, cudaStream_t s) {
     h.pipe_plan[h.parity].run(ctx);
     launches += h.pipe_plan[h.parity].launches;
     if (any_idle) { launch_mask_losses(h.d_losses, h.d_chunk_tab, h.K, s); launches += 1; }
+    h.last_wr = 1 - h.parity;
     h.parity ^= 1;
     h.pipe_steps += 1;
   }
@@ -399,6 +401,21 @@ lp_status lp_reset_pipeline(lp_handle hh) {
   return LP_OK;
 }
 
+size_t lp_chunk_output_bytes(lp_handle hh, int k) {
+  if (!hh || k < 0 || k >= hh->h.K) return 0;
+  return hh->h.bnd_bytes[k];
+}
+
+lp_status lp_chunk_output(lp_handle hh, int k, void* dst, size_t bytes, void* stream) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (!dst || k < 0 || k >= h.K) return fail(&h, LP_ERR_INVALID_ARG, "lp_chunk_output: null destination or chunk index out of range");
+  if (bytes < h.bnd_bytes[k]) return fail(&h, LP_ERR_INVALID_ARG, "lp_chunk_output: destination smaller than lp_chunk_output_bytes");
+  if (h.last_wr < 0) return fail(&h, LP_ERR_STATE, "lp_chunk_output: no training step has run yet");
+  cudaMemcpyAsync(dst, h.bnd[h.last_wr][k], h.bnd_bytes[k], cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  return check_cuda(&h, "lp_chunk_output");
+}
+
 lp_status lp_set_overlap(lp_handle hh, int on) {
   if (!hh) return LP_ERR_INVALID_ARG;
   Handle& h = hh->h;
@@ -463,6 +480,7 @@ static lp_status state_io(lp_handle hh, void* host, size_t bytes, bool save) {
     memcpy(&hd, p, sizeof(hd));
     if (hd.magic != kMagic || hd.n_total != h.n_total || hd.K != h.K) return fail(&h, LP_ERR_STATE, "state blob does not match this handle");
     h.step_count = hd.step_count; h.parity = (int)hd.parity; h.primed = hd.primed != 0;
+    h.last_wr = h.step_count == 0 ? -1 : (h.primed ? h.parity : 0);
     h.ramp = (int)hd.ramp; h.pipe_steps = hd.pipe_steps;
   }
   p += sizeof(hd);

@@ -39,11 +39,13 @@ void build_lm(Handle& h) {
   const int K = h.K, B = h.spec.batch, T = h.spec.seq_len, d = h.spec.d_model, F = h.spec.d_ffn, V = h.spec.vocab,
             H = h.spec.n_heads;
   const int M = B * T;
+  // an inner piece of a chain spread over several GPUs: x is the previous piece's activation, no embeddings
+  const bool inner = h.spec.input_is_activation != 0;
   h.rows = M;
   std::vector<ChunkBufs> cb(K);
   int blk = 0;
   for (int k = 0; k < K; ++k) {
-    if (k == 0) {
+    if (k == 0 && !inner) {
       h.add_tensor("c0.tok", 0, {V, d}, true);
       h.add_tensor("c0.pos", 0, {T, d}, true);
     }
@@ -74,7 +76,7 @@ void build_lm(Handle& h) {
 
   const size_t es = h.esize();
   const size_t md = (size_t)M * d * es;
-  h.x_bytes = (size_t)M * sizeof(int);
+  h.x_bytes = inner ? md : (size_t)M * sizeof(int);
   h.x_in = h.dalloc(h.x_bytes);
   h.y_bytes = (size_t)M * sizeof(int);
   h.y_in = (int*)h.dalloc(h.y_bytes);
@@ -89,7 +91,7 @@ void build_lm(Handle& h) {
     }
     h.n_valid.push_back((int*)h.dalloc(sizeof(int)));
     ChunkBufs& c = cb[k];
-    if (k == 0) c.emb = h.dalloc(md);
+    if (k == 0) c.emb = inner ? h.x_in : h.dalloc(md);
     for (size_t j = 0; j < c.blocks.size(); ++j) {
       BlockBufs& b = c.blocks[j];
       b.a1 = h.dalloc(md); b.qkv = h.dalloc(3 * md); b.o = h.dalloc(md); b.h1 = h.dalloc(md); b.a2 = h.dalloc(md);
@@ -136,7 +138,7 @@ void build_lm(Handle& h) {
   // ---- forward of the trunks of chunks `ks`
   auto forward = [&](Plan& p, const std::vector<int>& ks, int rd, int wr) {
     for (int k : ks)
-      if (k == 0) {
+      if (k == 0 && !inner) {
         EmbedProb e{(const int*)h.x_in, h.W("c0.tok"), h.W("c0.pos"), cb[0].emb, M, T, d, V};
         p.add(1, [e, st, bf](const RunCtx& c) { launch_embed_fwd(e, st, bf, c.stream); }, KIND_EMBED, 3.0 * M * d * es);
       }
@@ -386,13 +388,13 @@ void build_lm(Handle& h) {
         const size_t j = cb[k].blocks.size() - 1 - jj;
         // The block-input gradient is formed only if something consumes it: an earlier block of the same
         // chunk, chunk 0's embeddings, or (overlapping updates) the previous chunk's last block.
-        const bool need_dx = (j > 0) || (k == 0) || overlap;
+        const bool need_dx = (j > 0) || (k == 0 && !inner) || overlap;
         items.push_back(BwdItem{&cb[k], &cb[k].blocks[j], block_in(k, j, rd), need_dx, nullptr});
       }
       block_backward(p, items);
       // chunk 0, first block: embedding tables
       for (auto& it : items)
-        if (it.c == &cb[0] && it.b == &cb[0].blocks[0]) {
+        if (!inner && it.c == &cb[0] && it.b == &cb[0].blocks[0]) {
           EmbedBwdProb e{(const int*)h.x_in, cb[0].G0, h.G("c0.tok"), h.G("c0.pos"), emb_next, emb_first, M, T, d, V, B};
           p.add(6, [e, bf](const RunCtx& c) { launch_embed_bwd(e, bf, c.stream); }, KIND_EMBED, (double)M * d * es + 4.0 * V * d);
         }

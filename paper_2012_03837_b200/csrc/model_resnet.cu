@@ -92,12 +92,15 @@ void build_resnet(Handle& h) {
   const bool bf = h.bf16_mode;
   const bool head_bn = h.head.kind == LP_HEAD_BN_RELU_GAP_LINEAR;   // App. B.3's head
   const size_t es = h.esize();
+  // an inner piece of a chain spread over several GPUs: x is the previous stage's NHWC activation, there is no
+  // stem, and the first stage is a later stage of the network (stride 2, 1x1 shortcut)
+  const bool inner = h.spec.input_is_activation != 0;
   std::vector<Chunk> ch(K);
-  int H = h.spec.height, W = h.spec.width, cprev = h.spec.stem_channels;
+  int H = h.spec.height, W = h.spec.width, cprev = inner ? h.spec.in_channels : h.spec.stem_channels;
   for (int k = 0; k < K; ++k) {
     Chunk& c = ch[k];
     const std::string ck = "c" + std::to_string(k);
-    if (k == 0) {
+    if (k == 0 && !inner) {
       c.has_stem = true;
       c.stem = make_conv("c0.stem.conv", B, H, W, h.spec.in_channels, cprev, 3, 1);
       h.add_tensor("c0.stem.conv", 0, {cprev, 3, 3, h.spec.in_channels}, true);
@@ -109,7 +112,7 @@ void build_resnet(Handle& h) {
     for (int j = 0; j < h.spec.blocks_per_stage; ++j) {
       Block b;
       const std::string p = ck + ".r" + std::to_string(j);
-      int stride = (j == 0 && k > 0) ? 2 : 1;
+      int stride = (j == 0 && (k > 0 || inner)) ? 2 : 1;
       int cin = j == 0 ? cprev : cout;
       b.c1 = make_conv(p + ".conv1", B, H, W, cin, cout, 3, stride);
       h.add_tensor(p + ".conv1", k, {cout, 3, 3, cin}, true);
@@ -273,7 +276,7 @@ void build_resnet(Handle& h) {
     }, KIND_NORM, (double)elems * es * ((stats ? 3 : 2) + (res ? 1 : 0)));
   };
 
-  auto chunk_in = [&](int k, int rd) -> const void* { return k == 0 ? ch[0].stem_out : h.bnd[rd][k - 1]; };
+  auto chunk_in = [&](int k, int rd) -> const void* { return k == 0 ? (inner ? h.x_in : ch[0].stem_out) : h.bnd[rd][k - 1]; };
   auto labels_of = [&](int k, bool pipelined, int rd) -> const int* {
     return (!pipelined || k == 0) ? h.y_in : h.lab[rd][k - 1];
   };

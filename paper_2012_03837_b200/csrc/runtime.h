@@ -105,6 +105,7 @@ struct Handle {
   bool overlap = false;
   std::vector<ColReduceProb> pending_reduce;   // collected while a plan is being built
   int parity = 0;
+  int last_wr = -1;         // boundary-buffer slot the last training step wrote (-1: no step yet)
   bool primed = false;
   long long step_count = 0;
   // ---- ramp-up of the pipelined schedule (Sec. 6): LP_RAMP_PRIME fills the boundary buffers by a forward
