@@ -205,13 +205,15 @@ def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--minibatches", type=int, default=20)
+    ap.add_argument("--override", action="append", default=[], metavar="KEY=JSON",
+                    help="replace a field of the workload, e.g. --override 'blocks_per_chunk=[2,2]'")
     a = ap.parse_args(argv)
     rank, world = int(os.environ.get("RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
     torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", 0)))
     dev = torch.device("cuda", torch.cuda.current_device())
-    dist.init_process_group("nccl", rank=rank, world_size=world)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
     try:
-        cfg = lp_synth.config(a.workload)
+        cfg = lp_synth.config(a.workload, **{k: json.loads(v) for k, v in (o.split("=", 1) for o in a.override)})
         if lp_synth.num_chunks(cfg) != world:
             raise SystemExit(f"workload {a.workload} has {lp_synth.num_chunks(cfg)} chunks: launch that many ranks")
         params = lp_synth.init_params(cfg)
