@@ -77,15 +77,16 @@ __global__ void __launch_bounds__(256) col2im_kernel(const Im2colProb* __restric
   }
 }
 
-// Per-channel partial sums over a block of BN_ROWS rows.
+// Per-channel partial sums over a block of bn_rows_per_block(rows) rows.
 //   forward : part[blk][0][c] = sum x,   part[blk][1][c] = sum x^2
 //   backward: part[blk][0][c] = sum dyr * xhat, part[blk][1][c] = sum dyr, dyr = dy * [relu_out > 0]
 template <typename T, bool BWD>
 __global__ void __launch_bounds__(256) bn_stat_kernel(const BnStatProb* __restrict__ probs) {
   const BnStatProb p = probs[blockIdx.z];
-  int r0 = blockIdx.y * BN_ROWS;
+  const int rpb = bn_rows_per_block(p.rows);
+  int r0 = blockIdx.y * rpb;
   if (r0 >= p.rows) return;
-  int r1 = min(r0 + BN_ROWS, p.rows);
+  int r1 = min(r0 + rpb, p.rows);
   int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= p.C) return;
   const T* x = (const T*)p.x;
@@ -275,15 +276,16 @@ __global__ void __launch_bounds__(256) col2im_vec_kernel(const Im2colProb* __res
   }
 }
 
-// Block of 256 threads = (C/8 channel vectors) x (256 / (C/8) row lanes) over BN_ROWS rows; the row
+// Block of 256 threads = (C/8 channel vectors) x (256 / (C/8) row lanes) over the block's rows; the row
 // lanes are summed through shared memory in lane order.  Requires C % 8 == 0 and C/8 <= 256.
 template <bool BWD>
 __global__ void __launch_bounds__(256) bn_stat_vec_kernel(const BnStatProb* __restrict__ probs) {
   __shared__ float red[256 * 16];
   const BnStatProb p = probs[blockIdx.z];
-  int r0 = blockIdx.y * BN_ROWS;
+  const int rpb = bn_rows_per_block(p.rows);
+  int r0 = blockIdx.y * rpb;
   if (r0 >= p.rows) return;
-  int r1 = min(r0 + BN_ROWS, p.rows);
+  int r1 = min(r0 + rpb, p.rows);
   const int cv = p.C >> 3, ny = 256 / cv;
   const int tx = threadIdx.x % cv, ty = threadIdx.x / cv;
   float a[8], b[8];
@@ -317,27 +319,97 @@ __global__ void __launch_bounds__(256) bn_stat_vec_kernel(const BnStatProb* __re
       }
     }
   }
+  // red[value][thread]: the 16 partial values of a thread go to 16 different rows, so that a warp's stores, and
+  // the loads below (channel vectors of one value and line side by side), touch 32 different banks.
 #pragma unroll
-  for (int t = 0; t < 8; ++t) { red[threadIdx.x * 16 + t] = a[t]; red[threadIdx.x * 16 + 8 + t] = b[t]; }
+  for (int t = 0; t < 8; ++t) { red[t * 256 + threadIdx.x] = a[t]; red[(8 + t) * 256 + threadIdx.x] = b[t]; }
   __syncthreads();
-  // thread (c, which) sums lane 0..ny-1 for channel c
+  // thread (which, t, j) sums lane 0..ny-1 for channel j * 8 + t, in lane order
   for (int idx = threadIdx.x; idx < 2 * p.C; idx += 256) {
-    int which = idx / p.C, c = idx % p.C;
+    const int j = idx % cv, vt = idx / cv;             // vt = which * 8 + t
     float s = 0.f;
-    for (int l = 0; l < ny; ++l) s += red[(l * cv + (c >> 3)) * 16 + which * 8 + (c & 7)];
-    p.part[(size_t)blockIdx.y * 2 * p.C + which * p.C + c] = s;
+    for (int l = 0; l < ny; ++l) s += red[vt * 256 + l * cv + j];
+    p.part[(size_t)blockIdx.y * 2 * p.C + (vt >> 3) * p.C + j * 8 + (vt & 7)] = s;
   }
 }
 
+// y[n, c] = mean over hw of x[n, hw, c], bf16: one block per image.  With C % 8 == 0 and C / 8 <= 256 the block
+// is (C/8 channel vectors) x (256 / (C/8) pixel lanes) reading 16 bytes at a time, the pixel lanes summed through
+// shared memory in lane order; otherwise each thread walks the pixels of its channels.
+__global__ void __launch_bounds__(256) gap_fwd_vec_kernel(const GapProb* __restrict__ probs) {
+  __shared__ float red[256 * 8];
+  const GapProb p = probs[blockIdx.z];
+  const int n = blockIdx.y;
+  if (n >= p.N) return;
+  const bf16* x = (const bf16*)p.x + (size_t)n * p.HW * p.C;
+  bf16* y = (bf16*)p.y + (size_t)n * p.C;
+  const float inv = 1.0f / p.HW;
+  if ((p.C & 7) != 0 || (p.C >> 3) > 256) {
+    for (int c = threadIdx.x; c < p.C; c += 256) {
+      float s = 0.f;
+      for (int i = 0; i < p.HW; ++i) s += __bfloat162float(x[(size_t)i * p.C + c]);
+      y[c] = __float2bfloat16(s * inv);
+    }
+    return;
+  }
+  const int cv = p.C >> 3, ny = 256 / cv;
+  const int tx = threadIdx.x % cv, ty = threadIdx.x / cv;
+  float a[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) a[t] = 0.f;
+  if (ty < ny)
+    for (int i = ty; i < p.HW; i += ny) {
+      float v[8];
+      unpack8(*(const uint4*)(x + (size_t)i * p.C + tx * 8), v);
+#pragma unroll
+      for (int t = 0; t < 8; ++t) a[t] += v[t];
+    }
+#pragma unroll
+  for (int t = 0; t < 8; ++t) red[t * 256 + threadIdx.x] = a[t];
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < p.C; idx += 256) {
+    const int j = idx % cv, t = idx / cv;
+    float s = 0.f;
+    for (int l = 0; l < ny; ++l) s += red[t * 256 + l * cv + j];
+    y[j * 8 + t] = __float2bfloat16(s * inv);
+  }
+}
+
+// The per-channel constants are formed once per block in shared memory (a thread would otherwise issue some
+// thirty scalar loads for every 16 bytes of data).  A thread's channel vector is the same in every pass of the
+// grid-stride loop when the stride is a multiple of C / 8 (always so for power-of-two channel counts): it then
+// keeps its constants in registers.
 template <bool BWD>
 __global__ void __launch_bounds__(256) bn_apply_vec_kernel(const BnApplyProb* __restrict__ probs) {
+  __shared__ __align__(16) float cst[4][2048];          // C <= 2048 (C / 8 <= 256)
   const BnApplyProb p = probs[blockIdx.y];
   const int cv = p.C >> 3;
-  long long total = (long long)p.rows * cv;
+  const long long total = (long long)p.rows * cv;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  if ((long long)blockIdx.x * blockDim.x >= total) return;
+  const bool fixed = stride % cv == 0;
   const bf16* x = (const bf16*)p.x;
   const float inv = 1.0f / (float)p.rows;
-  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
-    int c0 = (int)(e % cv) * 8;
+  // forward: y = (x - mu) * ka + kb;  backward: dx = ka * (dyr - kb - (x - mu) * kc)
+  for (int c = threadIdx.x; c < p.C; c += 256) {
+    const float rs = p.rstd[c];
+    cst[0][c] = p.mean[c];
+    cst[1][c] = rs * p.g[c];
+    cst[2][c] = BWD ? p.dbeta[c] * inv : p.b[c];
+    cst[3][c] = BWD ? rs * p.dgamma[c] * inv : 0.f;
+  }
+  __syncthreads();
+  float mu[8], ka[8], kb[8], kc[8];
+  auto constants = [&](int c0) {
+    *(float4*)&mu[0] = *(const float4*)&cst[0][c0]; *(float4*)&mu[4] = *(const float4*)&cst[0][c0 + 4];
+    *(float4*)&ka[0] = *(const float4*)&cst[1][c0]; *(float4*)&ka[4] = *(const float4*)&cst[1][c0 + 4];
+    *(float4*)&kb[0] = *(const float4*)&cst[2][c0]; *(float4*)&kb[4] = *(const float4*)&cst[2][c0 + 4];
+    if (BWD) { *(float4*)&kc[0] = *(const float4*)&cst[3][c0]; *(float4*)&kc[4] = *(const float4*)&cst[3][c0 + 4]; }
+  };
+  long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (fixed && e < total) constants((int)(e % cv) * 8);
+  for (; e < total; e += stride) {
+    if (!fixed) constants((int)(e % cv) * 8);
     float xv[8], o[8];
     unpack8(*(const uint4*)(x + e * 8), xv);
     if (!BWD) {
@@ -345,7 +417,7 @@ __global__ void __launch_bounds__(256) bn_apply_vec_kernel(const BnApplyProb* __
       if (p.res) unpack8(*(const uint4*)((const bf16*)p.res + e * 8), r);
 #pragma unroll
       for (int t = 0; t < 8; ++t) {
-        float v = (xv[t] - p.mean[c0 + t]) * p.rstd[c0 + t] * p.g[c0 + t] + p.b[c0 + t];
+        float v = (xv[t] - mu[t]) * ka[t] + kb[t];
         if (p.res) v += r[t];
         o[t] = p.relu ? fmaxf(v, 0.f) : v;
       }
@@ -361,10 +433,7 @@ __global__ void __launch_bounds__(256) bn_apply_vec_kernel(const BnApplyProb* __
       }
       if (p.dres_out) *(uint4*)((bf16*)p.dres_out + e * 8) = pack8(g);
 #pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        float xh = (xv[t] - p.mean[c0 + t]) * p.rstd[c0 + t];
-        o[t] = p.rstd[c0 + t] * p.g[c0 + t] * (g[t] - p.dbeta[c0 + t] * inv - xh * p.dgamma[c0 + t] * inv);
-      }
+      for (int t = 0; t < 8; ++t) o[t] = ka[t] * (g[t] - kb[t] - (xv[t] - mu[t]) * kc[t]);
       *(uint4*)((bf16*)p.dx + e * 8) = pack8(o);
     }
   }
@@ -495,9 +564,9 @@ void launch_col2im(const Im2colProb* d, int n, long long max_elems, bool is_bf16
   else if (is_bf16) col2im_kernel<bf16><<<grid, 256, 0, s>>>(d);
   else col2im_kernel<float><<<grid, 256, 0, s>>>(d);
 }
-void launch_bn_stat_partial(const BnStatProb* d, int n, int max_rows, int max_c, bool bwd, bool is_bf16, cudaStream_t s,
+void launch_bn_stat_partial(const BnStatProb* d, int n, int max_blocks, int max_c, bool bwd, bool is_bf16, cudaStream_t s,
                             bool vec8) {
-  dim3 grid((max_c + 255) / 256, (max_rows + BN_ROWS - 1) / BN_ROWS, n);
+  dim3 grid((max_c + 255) / 256, max_blocks, n);
   if (vec8) {
     grid.x = 1;
     if (bwd) bn_stat_vec_kernel<true><<<grid, 256, 0, s>>>(d); else bn_stat_vec_kernel<false><<<grid, 256, 0, s>>>(d);
@@ -518,7 +587,7 @@ void launch_bn_apply(const BnApplyProb* d, int n, long long max_elems, bool bwd,
 }
 void launch_gap_fwd(const GapProb* d, int n, int max_n, int max_c, bool is_bf16, cudaStream_t s) {
   dim3 grid((max_c + 255) / 256, max_n, n);
-  if (is_bf16) gap_fwd_kernel<bf16><<<grid, 256, 0, s>>>(d);
+  if (is_bf16) gap_fwd_vec_kernel<<<dim3(1, max_n, n), 256, 0, s>>>(d);
   else gap_fwd_kernel<float><<<grid, 256, 0, s>>>(d);
 }
 void launch_small_conv_fwd(const SmallConvProb& p, bool w_is_bf16, bool is_bf16, cudaStream_t s) {

@@ -178,8 +178,20 @@ struct BnStatProb {   // per-channel partial sums of x and x^2 (fwd) or of dy an
   const void* x; const void* dy; const float* mean; const float* rstd; const void* relu_out;
   float* part; int rows, C;
 };
-enum { BN_ROWS = 256 };
-void launch_bn_stat_partial(const BnStatProb* d_probs, int n, int max_rows, int max_c, bool bwd, bool is_bf16,
+// Rows summed by one block of the statistics kernels: 256 where that still leaves four blocks per SM of a
+// 148-SM device, fewer (down to 32) for the short tensors of the late stages, whose sums would otherwise
+// run as a few long serial loops on a handful of SMs.
+#if defined(__CUDACC__)
+__host__ __device__
+#endif
+inline int bn_rows_per_block(long long rows) {
+  int rpb = 256;
+  while (rpb > 32 && rows / rpb < 592) rpb >>= 1;
+  return rpb;
+}
+inline int bn_blocks(long long rows) { int rpb = bn_rows_per_block(rows); return (int)((rows + rpb - 1) / rpb); }
+// max_blocks: the largest bn_blocks(rows) among the n problems
+void launch_bn_stat_partial(const BnStatProb* d_probs, int n, int max_blocks, int max_c, bool bwd, bool is_bf16,
                             cudaStream_t s, bool vec8 = false);
 struct BnFinalProb {  // fwd: sums -> mean, rstd.  part is [nblk, 2, C]
   const float* part; int nblk; int rows; int C; float* mean; float* rstd; float* dgamma; float* dbeta; float eps;

@@ -250,7 +250,7 @@ void build_resnet(Handle& h) {
   // also move the running averages (training steps), running statistics (evaluation)
   enum { BN_BATCH = 0, BN_TRAIN = 1, BN_RUNNING = 2 };
   auto bn_fwd = [&](Plan& p, const Bn& b, const void* x, void* y, const void* res, bool relu, int mode) {
-    int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
+    int nblk = bn_blocks(b.rows);
     float* part = mode == BN_RUNNING ? nullptr : fal((size_t)nblk * 2 * b.C);
     float *rm = nullptr, *rv = nullptr;
     if (mode != BN_BATCH) {
@@ -265,12 +265,12 @@ void build_resnet(Handle& h) {
     const BnStatProb* ds = h.upload(std::vector<BnStatProb>{sp});
     const BnFinalProb* df = h.upload(std::vector<BnFinalProb>{fp});
     const BnApplyProb* da = h.upload(std::vector<BnApplyProb>{ap});
-    int rows = (int)b.rows, C = b.C;
+    int C = b.C;
     bool v8 = bf && C % 8 == 0 && C / 8 <= 256;
     long long elems = b.rows * b.C;
     const bool stats = mode != BN_RUNNING;
     p.add(stats ? 3 : 2, [=](const RunCtx& r) {
-      if (stats) launch_bn_stat_partial(ds, 1, rows, C, false, bf, r.stream, v8);
+      if (stats) launch_bn_stat_partial(ds, 1, nblk, C, false, bf, r.stream, v8);
       launch_bn_finalize(df, 1, C, false, r.stream);
       launch_bn_apply(da, 1, elems, false, bf, r.stream, v8);
     }, KIND_NORM, (double)elems * es * ((stats ? 3 : 2) + (res ? 1 : 0)));
@@ -373,7 +373,7 @@ void build_resnet(Handle& h) {
   // dx = BN'(dy masked by relu_out > 0); dres (optional) receives the masked dy
   auto rec_bn_bwd = [&](OpList& L, const Bn& b, const void* x, const void* dy, const void* relu_out, void* dx, void* dres,
                         const GradMap* second = nullptr) {
-    int nblk = (int)((b.rows + BN_ROWS - 1) / BN_ROWS);
+    int nblk = bn_blocks(b.rows);
     float* part = fal((size_t)nblk * 2 * b.C);
     float *dg = GD(second, b.g), *db = GD(second, b.b);
     Op o; o.kind = OP_BN_BWD;
@@ -530,11 +530,11 @@ void build_resnet(Handle& h) {
       }
       for (int v8 = 0; v8 < 2; ++v8) {
         std::vector<BnStatProb> st; std::vector<BnFinalProb> fi; std::vector<BnApplyProb> ap;
-        int rows = 0, C = 0; long long elems = 0; double work = 0;
+        int nb = 0, C = 0; long long elems = 0; double work = 0;
         for (Op* o : at)
           if (o->kind == OP_BN_BWD && (int)o->v8 == v8) {
             st.push_back(o->bn_stat); fi.push_back(o->bn_final); ap.push_back(o->bn_apply);
-            rows = std::max(rows, o->bn_stat.rows); C = std::max(C, o->bn_stat.C); elems = std::max(elems, o->elems); work += o->work;
+            nb = std::max(nb, o->bn_final.nblk); C = std::max(C, o->bn_stat.C); elems = std::max(elems, o->elems); work += o->work;
           }
         if (st.empty()) continue;
         const BnStatProb* ds = h.upload(st);
@@ -543,7 +543,7 @@ void build_resnet(Handle& h) {
         int n = (int)st.size();
         bool vec = v8 != 0;
         p.add(3, [=](const RunCtx& r) {
-          launch_bn_stat_partial(ds, n, rows, C, true, bf, r.stream, vec);
+          launch_bn_stat_partial(ds, n, nb, C, true, bf, r.stream, vec);
           launch_bn_finalize(df, n, C, true, r.stream);
           launch_bn_apply(da, n, elems, true, bf, r.stream, vec);
         }, KIND_NORM, work);

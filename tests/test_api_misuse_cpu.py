@@ -35,6 +35,8 @@ def test_lp_create_rejects_inconsistent_specifications():
         (c3, lambda m, hd, op: setattr(m, "seq_len", 0), None, "SHAPE"),
         (c4, lambda m, hd, op: setattr(m, "height", 4), None, "SHAPE"),           # 4 stages halve a 4-pixel image away
         (c4, lambda m, hd, op: setattr(m, "blocks_per_stage", 0), None, "SHAPE"),
+        (c4, lambda m, hd, op: setattr(hd, "kind", lp.LP_HEAD_LN_LINEAR), None, "INVALID_ARG"),
+        (c1, lambda m, hd, op: setattr(hd, "kind", lp.LP_HEAD_BN_RELU_GAP_LINEAR), None, "INVALID_ARG"),
     ]
     for cfg, mutate, K, want in cases:
         e = create_error(cfg, mutate, K)
@@ -54,6 +56,7 @@ def test_null_handles_and_pointers_are_refused():
                  lambda: L.lp_reset_pipeline(None),
                  lambda: L.lp_set_ramp(None, 0),
                  lambda: L.lp_set_overlap(None, 1),
+                 lambda: L.lp_chunk_output(None, 0, None, 0, None),
                  lambda: L.lp_status_poll(None, None),
                  lambda: L.lp_get_tensor(None, 0, 0, None, 0, None),
                  lambda: L.lp_set_tensor(None, 0, 0, None, 0, None),
