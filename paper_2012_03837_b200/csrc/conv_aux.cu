@@ -130,7 +130,18 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const BnFinalProb* __r
     return;
   }
   double a = 0.0, b = 0.0;
-  for (int k = lane; k < p.nblk; k += 32) {
+  int k = lane;
+  for (; k + 7 * 32 < p.nblk; k += 8 * 32) {     // eight partial blocks per pass: sixteen loads in flight, same order of sums
+    float va[8], vb[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      va[u] = p.part[(size_t)(k + u * 32) * 2 * p.C + c];
+      vb[u] = p.part[(size_t)(k + u * 32) * 2 * p.C + p.C + c];
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) { a += (double)va[u]; b += (double)vb[u]; }
+  }
+  for (; k < p.nblk; k += 32) {
     a += (double)p.part[(size_t)k * 2 * p.C + c];
     b += (double)p.part[(size_t)k * 2 * p.C + p.C + c];
   }
