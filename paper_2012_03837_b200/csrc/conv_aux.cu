@@ -344,6 +344,22 @@ __global__ void __launch_bounds__(256) bn_stat_vec_kernel(const BnStatProb* __re
   }
 }
 
+// dx[n, hw, c] = dy[n, c] / HW, bf16 with C % 8 == 0: eight channels per access
+__global__ void __launch_bounds__(256) gap_bwd_vec_kernel(const GapProb* __restrict__ probs) {
+  const GapProb p = probs[blockIdx.y];
+  const int cv = p.C >> 3;
+  const long long per_image = (long long)p.HW * cv, total = (long long)p.N * per_image;
+  const float inv = 1.0f / p.HW;
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (long long)gridDim.x * blockDim.x) {
+    const int n = (int)(e / per_image), j = (int)(e % cv);
+    float g[8];
+    unpack8(*(const uint4*)((const bf16*)p.dy + (size_t)n * p.C + j * 8), g);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) g[t] *= inv;
+    *(uint4*)((bf16*)p.dx + e * 8) = pack8(g);
+  }
+}
+
 // y[n, c] = mean over hw of x[n, hw, c], bf16: one block per image.  With C % 8 == 0 and C / 8 <= 256 the block
 // is (C/8 channel vectors) x (256 / (C/8) pixel lanes) reading 16 bytes at a time, the pixel lanes summed through
 // shared memory in lane order; otherwise each thread walks the pixels of its channels.
@@ -620,7 +636,11 @@ void launch_small_conv_wgrad(const SmallConvProb& p, bool is_bf16, cudaStream_t 
   if (is_bf16) small_conv_wgrad_kernel<bf16><<<grid, 256, smem, s>>>(p);
   else small_conv_wgrad_kernel<float><<<grid, 256, smem, s>>>(p);
 }
-void launch_gap_bwd(const GapProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s) {
+void launch_gap_bwd(const GapProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8) {
+  if (vec8 && is_bf16) {
+    gap_bwd_vec_kernel<<<dim3(grid_for(max_elems / 8), n), 256, 0, s>>>(d);
+    return;
+  }
   dim3 grid(grid_for(max_elems), n);
   if (is_bf16) gap_bwd_kernel<bf16><<<grid, 256, 0, s>>>(d);
   else gap_bwd_kernel<float><<<grid, 256, 0, s>>>(d);

@@ -227,13 +227,14 @@ void launch_small_conv_wgrad(const SmallConvProb& p, bool is_bf16, cudaStream_t 
 
 struct GapProb { const void* x; void* y; const void* dy; void* dx; int N, HW, C; };
 void launch_gap_fwd(const GapProb* d_probs, int n, int max_n, int max_c, bool is_bf16, cudaStream_t s);
-void launch_gap_bwd(const GapProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
+void launch_gap_bwd(const GapProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8 = false);
 
 struct AddProb { const void* a; const void* b; void* out; long long n; };
 // a[i] = (a[i] + b[i]) / 2 in fp32: the averaged gradient of a layer shared by two overlapping blocks (App. A.2)
 struct AvgProb { float* a; const float* b; long long n; };
 void launch_average_f32(const AvgProb* d_probs, int n, long long max_elems, cudaStream_t s);
-void launch_add(const AddProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s);
+// vec8: bf16, every problem's element count a multiple of 8 and its tensors 16-byte aligned
+void launch_add(const AddProb* d_probs, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8 = false);
 
 // ---------------------------------------------------------------------------- optimizer
 struct OptimArgs {

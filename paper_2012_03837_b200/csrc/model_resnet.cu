@@ -510,14 +510,14 @@ void build_resnet(Handle& h) {
       for (auto& L : lists) if (i < L.size() && L[i].kind != OP_NOP) at.push_back(&L[i]);
       std::vector<GemmProb> gemms;
       std::vector<ColSumProb> cs; std::vector<float*> cs_out;
-      std::vector<GapProb> gaps; long long gap_max = 0; double gap_work = 0;
-      std::vector<AddProb> adds; long long add_max = 0; double add_work = 0;
+      std::vector<GapProb> gaps; long long gap_max = 0; double gap_work = 0; bool gap_vec = bf;
+      std::vector<AddProb> adds; long long add_max = 0; double add_work = 0; bool add_vec = bf;
       for (Op* o : at) {
         switch (o->kind) {
           case OP_GEMM: gemms.insert(gemms.end(), o->gemms.begin(), o->gemms.end()); break;
           case OP_COLSUM: cs.push_back(o->colsum); cs_out.push_back(o->colsum_out); break;
-          case OP_GAP_BWD: gaps.push_back(o->gap); gap_max = std::max(gap_max, o->elems); gap_work += (double)o->elems * es; break;
-          case OP_ADD: adds.push_back(o->add); add_max = std::max(add_max, o->elems); add_work += 3.0 * o->elems * es; break;
+          case OP_GAP_BWD: gaps.push_back(o->gap); gap_vec = gap_vec && o->gap.C % 8 == 0; gap_max = std::max(gap_max, o->elems); gap_work += (double)o->elems * es; break;
+          case OP_ADD: adds.push_back(o->add); add_vec = add_vec && o->elems % 8 == 0; add_max = std::max(add_max, o->elems); add_work += 3.0 * o->elems * es; break;
           default: break;
         }
       }
@@ -526,7 +526,7 @@ void build_resnet(Handle& h) {
       if (!gaps.empty()) {
         const GapProb* dg = h.upload(gaps);
         int n = (int)gaps.size();
-        p.add(1, [=](const RunCtx& r) { launch_gap_bwd(dg, n, gap_max, bf, r.stream); }, KIND_CONV_AUX, gap_work);
+        p.add(1, [=](const RunCtx& r) { launch_gap_bwd(dg, n, gap_max, bf, r.stream, gap_vec); }, KIND_CONV_AUX, gap_work);
       }
       for (int v8 = 0; v8 < 2; ++v8) {
         std::vector<BnStatProb> st; std::vector<BnFinalProb> fi; std::vector<BnApplyProb> ap;
@@ -551,7 +551,7 @@ void build_resnet(Handle& h) {
       if (!adds.empty()) {
         const AddProb* d = h.upload(adds);
         int n = (int)adds.size();
-        p.add(1, [=](const RunCtx& r) { launch_add(d, n, add_max, bf, r.stream); }, KIND_CONV_AUX, add_work);
+        p.add(1, [=](const RunCtx& r) { launch_add(d, n, add_max, bf, r.stream, add_vec); }, KIND_CONV_AUX, add_work);
       }
       for (Op* o : at) if (o->kind == OP_RAW) o->raw(p);
     }

@@ -285,6 +285,25 @@ __global__ void __launch_bounds__(256) average_f32_kernel(const AvgProb* __restr
     p.a[i] = (p.a[i] + p.b[i]) * 0.5f;
 }
 
+// bf16, element count a multiple of 8, 16-byte aligned tensors: eight elements per access
+__global__ void __launch_bounds__(256) add_vec_kernel(const AddProb* __restrict__ probs) {
+  const AddProb p = probs[blockIdx.y];
+  const long long nv = p.n >> 3;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nv; i += (long long)gridDim.x * blockDim.x) {
+    const uint4 ua = ((const uint4*)p.a)[i], ub = ((const uint4*)p.b)[i];
+    const __nv_bfloat162* xa = (const __nv_bfloat162*)&ua;
+    const __nv_bfloat162* xb = (const __nv_bfloat162*)&ub;
+    uint4 uo;
+    __nv_bfloat162* xo = (__nv_bfloat162*)&uo;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const float2 fa = __bfloat1622float2(xa[t]), fb = __bfloat1622float2(xb[t]);
+      xo[t] = __floats2bfloat162_rn(fa.x + fb.x, fa.y + fb.y);
+    }
+    ((uint4*)p.out)[i] = uo;
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) add_kernel(const AddProb* __restrict__ probs) {
   const AddProb p = probs[blockIdx.y];
@@ -338,7 +357,14 @@ void launch_average_f32(const AvgProb* d, int n, long long max_elems, cudaStream
   if (blocks > 148 * 16) blocks = 148 * 16;
   average_f32_kernel<<<dim3((unsigned)blocks, n), 256, 0, s>>>(d);
 }
-void launch_add(const AddProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s) {
+void launch_add(const AddProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8) {
+  if (vec8 && is_bf16) {
+    long long blocks = (max_elems / 8 + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks < 1) blocks = 1;
+    add_vec_kernel<<<dim3((unsigned)blocks, n), 256, 0, s>>>(d);
+    return;
+  }
   long long blocks = (max_elems + 255) / 256;
   if (blocks > 148 * 16) blocks = 148 * 16;
   dim3 grid((unsigned)blocks, n);
