@@ -407,7 +407,7 @@ __global__ void __launch_bounds__(256) gap_fwd_vec_kernel(const GapProb* __restr
 // grid-stride loop when the stride is a multiple of C / 8 (always so for power-of-two channel counts): it then
 // keeps its constants in registers.
 template <bool BWD>
-__global__ void __launch_bounds__(256) bn_apply_vec_kernel(const BnApplyProb* __restrict__ probs) {
+__global__ void __launch_bounds__(256, 4) bn_apply_vec_kernel(const BnApplyProb* __restrict__ probs) {
   __shared__ __align__(16) float cst[4][2048];          // C <= 2048 (C / 8 <= 256)
   const BnApplyProb p = probs[blockIdx.y];
   const int cv = p.C >> 3;
