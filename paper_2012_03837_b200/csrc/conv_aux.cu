@@ -481,8 +481,11 @@ __global__ void __launch_bounds__(256) small_conv_fwd_kernel(SmallConvProb p) {
   const int groups = p.Cout >> 3, ppb = blockDim.x / groups;
   const int g = threadIdx.x % groups, pl = threadIdx.x / groups;
   const long long total = (long long)p.N * p.H * p.W;
-  const long long pix = (long long)blockIdx.x * ppb + pl;
-  if (pl >= ppb || pix >= total) return;
+  if (pl >= ppb) return;
+  // a block keeps the filters for several groups of pixels
+  for (long long grp = blockIdx.x; grp * ppb < total; grp += gridDim.x) {
+  const long long pix = grp * ppb + pl;
+  if (pix >= total) continue;
   const int w0 = (int)(pix % p.W), h0 = (int)((pix / p.W) % p.H);
   const long long img = pix / ((long long)p.W * p.H);
   float acc[8];
@@ -506,8 +509,13 @@ __global__ void __launch_bounds__(256) small_conv_fwd_kernel(SmallConvProb p) {
     }
   }
   T* y = (T*)p.y + pix * p.Cout + g * 8;
+  if (sizeof(T) == 2) {
+    *(uint4*)y = pack8(acc);                            // Cout % 8 == 0: 16-byte aligned
+  } else {
 #pragma unroll
-  for (int t = 0; t < 8; ++t) y[t] = from_f<T>(acc[t]);
+    for (int t = 0; t < 8; ++t) y[t] = from_f<T>(acc[t]);
+  }
+  }
 }
 
 // Filter gradient: thread (co, part) owns the taps/channels k = part, part + parts, ... of output channel co
@@ -620,7 +628,8 @@ void launch_gap_fwd(const GapProb* d, int n, int max_n, int max_c, bool is_bf16,
 void launch_small_conv_fwd(const SmallConvProb& p, bool w_is_bf16, bool is_bf16, cudaStream_t s) {
   const int groups = p.Cout / 8, ppb = 256 / groups;
   const long long total = (long long)p.N * p.H * p.W;
-  const unsigned grid = (unsigned)((total + ppb - 1) / ppb);
+  long long groups_of_pixels = (total + ppb - 1) / ppb;
+  const unsigned grid = (unsigned)(groups_of_pixels < 148 * 8 ? groups_of_pixels : 148 * 8);
   const size_t smem = (size_t)9 * p.Cin * p.Cout * sizeof(float);
   if (is_bf16) {
     if (w_is_bf16) small_conv_fwd_kernel<bf16, bf16><<<grid, 256, smem, s>>>(p);
