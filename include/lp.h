@@ -262,7 +262,11 @@ lp_status lp_load_state(lp_handle h, const void* host_src, size_t bytes);
  * pre-activation), 3 multiply by [aux > 0], 4 multiply by GELU'(aux).  out_f32: C is float, else bf16.
  * backend: 0 = tensor cores where the sizes allow, 1 = FP32 ALUs.  *used_tensor_cores (nullable)
  * receives how many of the problems ran on the tensor-core kernel.  Asynchronous on `stream`
- * except for the upload of the descriptor table.  Errors: INVALID_ARG, ALLOC, CUDA.
+ * except for the upload of the descriptor table.  Refused before anything is uploaded or launched
+ * (INVALID_ARG): null A, B or C; non-positive sizes or strides; no unit stride in an operand;
+ * ldc < N; act outside 0..4; act 2 without C2 or with out_f32; act 3 or 4 without aux.  This entry
+ * and lp_conv3x3_bf16 keep their scratch on the device that was current at their first call and
+ * return UNSUPPORTED on any other device of the process.  Errors: INVALID_ARG, UNSUPPORTED, ALLOC, CUDA.
  */
 typedef struct {
   const void* A; const void* B; void* C; void* C2;
@@ -292,32 +296,58 @@ lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* ou
                           int c_in, int c_out, void* stream);
 
 /*
+ * lp_attention_bf16: kernel-level entry for tests and profiling: causal multi-head softmax attention with heads
+ * of 64 over bf16 activations (the attention of App. B.2's transformer layers), on the tensor cores with the
+ * score tiles held in tensor memory.  All pointers are device pointers.
+ *   qkv  [batch, seq_len, 3*d], d = 64*n_heads: columns [0, d) queries, [d, 2d) keys, [2d, 3d) values, head h
+ *        at columns h*64 of each third.  Position t attends to positions <= t; scores are scaled by 1/8.
+ *   LP_ATTN_FORWARD:  reads qkv; writes o [batch, seq_len, d] bf16 and lse [batch, n_heads, seq_len] fp32, each
+ *        row's log2 of the sum of 2^(score * log2(e) / 8) over the keys it sees.  dout, dqkv, delta are ignored.
+ *   LP_ATTN_BACKWARD: reads qkv, o and lse as the forward call left them and dout [batch, seq_len, d] bf16 (the
+ *        gradient of o); writes dqkv [batch, seq_len, 3*d] bf16 and delta [batch, n_heads, seq_len] fp32 (row
+ *        sums of dout * o).
+ * The call synchronises `stream` before it returns.  Errors: INVALID_ARG (null pointer, unknown form), SHAPE
+ * (non-positive sizes), UNSUPPORTED (tensors not 16-byte aligned; a device other than the one of the first
+ * call), ALLOC, CUDA, TIMEOUT (a bounded device-side wait gave up: outputs are not valid).
+ */
+enum { LP_ATTN_FORWARD = 0, LP_ATTN_BACKWARD = 1 };
+lp_status lp_attention_bf16(int form, const void* qkv, void* o, float* lse, const void* dout, void* dqkv, float* delta,
+                            int batch, int seq_len, int n_heads, void* stream);
+
+/*
  * lp_gemm_bf16_static: lp_gemm_bf16 for callers that cannot allocate device memory.  (The paper
  * has no counterpart to this entry point; it exists for the library's users.)
  *
- * Who needs it: code that may not call cudaMalloc at the point where it launches work -- a thread
- * recording a CUDA graph, a real-time or serving loop that must never take the driver's allocator
- * lock, an embedding into a host whose device-memory budget was handed out up front.  lp_gemm_bf16
- * keeps its problem table, its TMA tensor maps and its status word in a cudaMalloc'ed buffer that
- * grows on demand; this variant keeps them in a fixed array that is part of the library image
- * (about 58 KB of device memory on every GPU that loads the library, held until the process exits)
- * and calls no cudaMalloc, cudaFree or any other allocating routine.
+ * Who needs it: code that may not call cudaMalloc or cudaFree at the point where it launches work --
+ * a serving or real-time loop that must never take the driver's allocator lock nor the device-wide
+ * synchronisation those calls imply, a plug-in inside a host program that handed out the whole
+ * device-memory budget up front, code running under a memory-pool manager that forbids outside
+ * allocations.  lp_gemm_bf16 keeps its problem table, its TMA tensor maps and its status word in a
+ * cudaMalloc'ed buffer that grows on demand; this variant keeps them in a fixed array that is part of
+ * the library image (about 58 KB of device memory on every GPU that loads the library, held until the
+ * process exits) and calls no cudaMalloc, cudaFree or any other allocating routine.
  *
  *   n: 1 .. LP_GEMM_STATIC_MAX problems; more is rejected with LP_ERR_SHAPE and nothing is launched.
- *   probs: host array, same meaning as for lp_gemm_bf16 (device pointers inside).  Each problem runs
- *     on the tensor-core kernel if its sizes allow, otherwise on the FP32-ALU kernel.
+ *   probs: host array, same meaning and the same checks as for lp_gemm_bf16 (device pointers inside).
+ *     Each problem runs on the tensor-core kernel if its sizes allow, otherwise on the FP32-ALU kernel.
  *   stream: the problems are uploaded and launched on this stream, asynchronously.
  *
  * The first call on a device looks up the array's device address (one-time set-up, with that
  * device current); make that first call before any stream capture begins.  All calls on a device
- * share the one array, which keeps the previous call's contents: each call clears the status word
- * and overwrites the table entries it uses.  Two calls whose work may overlap on the GPU (different
- * streams without an ordering between them) race on the array; calls on one stream are ordered.
+ * share the one array, which keeps the previous call's contents: each call overwrites the table
+ * entries it uses.  Two calls whose work may overlap on the GPU (different streams without an
+ * ordering between them) race on the array; calls on one stream are ordered.  Host threads are
+ * serialised by a lock while they fill the (process-wide, host-side) staging table.
  * Errors: INVALID_ARG, SHAPE, UNSUPPORTED (device ordinal above 63), CUDA; the message is returned
  * by lp_gemm_static_last_error().
+ *
+ * lp_gemm_static_poll: synchronises `stream`, reads and clears the array's status word on the current
+ * device.  LP_OK, or LP_ERR_TIMEOUT if a bounded device-side wait of any call since the last poll gave
+ * up (those calls' outputs are then not valid).  Allocates nothing.
  */
 #define LP_GEMM_STATIC_MAX 64
 lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* probs, void* stream);
+lp_status lp_gemm_static_poll(void* stream);
 const char* lp_gemm_static_last_error(void);
 
 /*

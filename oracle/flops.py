@@ -58,9 +58,3 @@ def parallelism(method: str, layers: int, chunks: int = 1, backward_multiplier: 
         bm = backward_multiplier
         return (layers + chunks * bm) / (chunks * (1 + bm))
     return {"backprop": 1, "greedy": layers, "overlapping": layers, "chunked": chunks}[method]
-
-
-def sequential_time(method: str, cost: float, batch_size: int, layers: int, chunks: int = 1) -> float:
-    """Sequential FLOPs: total cost divided by the available parallelism (App. A.2)."""
-    par = {"backprop": 1, "greedy": layers, "overlapping": layers, "chunked": chunks}[method]
-    return cost / (batch_size * par)

@@ -60,7 +60,7 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
-           "lp_gemm_bf16_static", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap",
+           "lp_attention_bf16", "lp_gemm_bf16_static", "lp_gemm_static_poll", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap",
            "lp_cost_model", "lp_mlp_layer_flops", "lp_mlp_aux_flops", "lp_chunk_output_bytes", "lp_chunk_output"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
@@ -171,9 +171,20 @@ def specs_from_config(cfg: dict, gemm_backend: int = 0):
     return m, K, hd, op
 
 
-def lp_create(model: lp_model_spec, K: int, head: lp_head_spec, optim: lp_optim_spec) -> int:
+LP_ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
+LP_RELEASE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
+
+
+class lp_alloc(C.Structure):
+    """Optional allocator for the handle's device memory: alloc(bytes, user) -> device pointer aligned
+    to 256 bytes or NULL, release(ptr, user).  Keep the object alive as long as the handle."""
+    _fields_ = [("alloc", LP_ALLOC_FN), ("release", LP_RELEASE_FN), ("user", C.c_void_p)]
+
+
+def lp_create(model: lp_model_spec, K: int, head: lp_head_spec, optim: lp_optim_spec, alloc: lp_alloc | None = None) -> int:
     h = C.c_void_p()
-    code = _lib.lp_create(C.byref(model), K, C.byref(head), C.byref(optim), None, C.byref(h))
+    code = _lib.lp_create(C.byref(model), K, C.byref(head), C.byref(optim), C.byref(alloc) if alloc is not None else None,
+                          C.byref(h))
     _check(None, code)
     return h.value
 
@@ -320,21 +331,43 @@ def lp_conv3x3_bf16(form: int, act, other, out, n: int, h: int, w: int, c_in: in
     _check(None, _lib.lp_conv3x3_bf16(form, _ptr(act), _ptr(other), _ptr(out), n, h, w, c_in, c_out, stream))
 
 
+LP_ATTN_FORWARD, LP_ATTN_BACKWARD = 0, 1
+_lib.lp_attention_bf16.argtypes = [C.c_int] + [C.c_void_p] * 6 + [C.c_int] * 3 + [C.c_void_p]
+
+
+def lp_attention_bf16(form: int, qkv, o, lse, dout, dqkv, delta, batch: int, seq_len: int, n_heads: int, stream=None) -> None:
+    """Causal attention with heads of 64 over bf16 [batch, seq_len, 3*64*n_heads] (see lp.h): forward writes o and
+    lse; backward reads them and dout and writes dqkv and delta.  Tensors may be torch tensors or raw pointers."""
+    _check(None, _lib.lp_attention_bf16(form, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dqkv), _ptr(delta),
+                                        batch, seq_len, n_heads, stream))
+
+
 _lib.lp_gemm_bf16_static.argtypes = [C.c_int, C.POINTER(lp_gemm_desc), C.c_void_p]
 _lib.lp_gemm_static_last_error.restype = C.c_char_p
 
 
 def lp_gemm_bf16_static(descs: list, stream=None) -> None:
-    """lp_gemm_bf16 for callers that must not allocate device memory (a thread recording a CUDA
-    graph, a serving loop that may not take the allocator lock): the problem table lives in a
-    fixed array inside the library, at most LP_GEMM_STATIC_MAX problems per call.  Same descriptor
-    dictionaries as lp_gemm_bf16.  Calls on one stream are ordered; calls that could overlap on
-    the GPU share that array and race."""
+    """lp_gemm_bf16 for callers that must not allocate device memory (a serving or real-time loop
+    that may not take the driver's allocator lock, a plug-in whose host has handed out the whole
+    device-memory budget): the problem table lives in a fixed array inside the library, at most
+    LP_GEMM_STATIC_MAX problems per call.  Same descriptor dictionaries as lp_gemm_bf16.  Calls on
+    one stream are ordered; calls that could overlap on the GPU share that array and race."""
     arr = (lp_gemm_desc * len(descs))()
     for d, q in zip(arr, descs):
         for k, v in q.items():
             setattr(d, k, _ptr(v) if k in ("A", "B", "C", "C2", "bias", "resid", "aux") else int(v))
     code = _lib.lp_gemm_bf16_static(len(descs), arr, stream)
+    if code != LP_OK:
+        raise LpError(code, (_lib.lp_gemm_static_last_error() or b"").decode())
+
+
+_lib.lp_gemm_static_poll.argtypes = [C.c_void_p]
+
+
+def lp_gemm_static_poll(stream=None) -> None:
+    """Synchronise `stream`, read and clear the status word of lp_gemm_bf16_static's array; raises
+    LpError (TIMEOUT) if a device-side wait of a call since the last poll gave up."""
+    code = _lib.lp_gemm_static_poll(stream)
     if code != LP_OK:
         raise LpError(code, (_lib.lp_gemm_static_last_error() or b"").decode())
 

@@ -200,13 +200,17 @@ __global__ void __launch_bounds__(128) attn_bwd_dkv_kernel(const AttnProb* __res
 
 void launch_attn_fwd(const AttnProb* d, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s) {
   dim3 grid((maxT + TILE - 1) / TILE, maxB * maxH, n);
-  if (is_bf16) { launch_attn_fwd_tc(d, n, maxB, maxT, maxH, s); return; }
-  attn_fwd_kernel<float><<<grid, 64, 0, s>>>(d);
+  if (is_bf16) attn_fwd_kernel<bf16><<<grid, 64, 0, s>>>(d);
+  else attn_fwd_kernel<float><<<grid, 64, 0, s>>>(d);
 }
 
 void launch_attn_bwd(const AttnProb* d, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s) {
   dim3 grid((maxT + TILE - 1) / TILE, maxB * maxH, n);
-  if (is_bf16) { launch_attn_bwd_tc(d, n, maxB, maxT, maxH, s); return; }
+  if (is_bf16) {
+    attn_bwd_dq_kernel<bf16><<<grid, 64, 0, s>>>(d);
+    attn_bwd_dkv_kernel<bf16><<<grid, 128, 0, s>>>(d);
+    return;
+  }
   attn_bwd_dq_kernel<float><<<grid, 64, 0, s>>>(d);
   attn_bwd_dkv_kernel<float><<<grid, 128, 0, s>>>(d);
 }

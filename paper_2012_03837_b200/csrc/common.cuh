@@ -10,6 +10,9 @@ template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
 
+// ReLU that keeps a NaN (fmaxf would turn it into 0 and hide a non-finite input from the loss check).
+__device__ __forceinline__ float relu_f(float v) { return v < 0.0f ? 0.0f : v; }
+
 // Exact GELU x*Phi(x) and its derivative Phi(x) + x*phi(x).
 __device__ __forceinline__ float gelu_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
 __device__ __forceinline__ float gelu_grad_f(float x) {
@@ -67,7 +70,7 @@ __device__ __forceinline__ void gemm_epilogue_store(const GemmProb& p, int m, in
   if (p.bias) v += p.bias[n];
   if (p.resid) v += to_f(((const T*)p.resid)[off]);
   switch (p.act) {
-    case EPI_RELU: v = fmaxf(v, 0.0f); break;
+    case EPI_RELU: v = relu_f(v); break;
     case EPI_GELU: ((T*)p.C2)[off] = from_f<T>(v); v = gelu_f(to_f(from_f<T>(v))); break;
     case EPI_RELU_MASK: v = to_f(((const T*)p.aux)[off]) > 0.0f ? v : 0.0f; break;
     case EPI_GELU_GRAD: v *= gelu_grad_f(to_f(((const T*)p.aux)[off])); break;

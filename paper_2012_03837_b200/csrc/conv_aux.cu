@@ -179,7 +179,7 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const BnApplyProb* __rest
     if (!BWD) {
       float v = xh * p.g[c] + p.b[c];
       if (p.res) v += to_f(((const T*)p.res)[e]);
-      if (p.relu) v = fmaxf(v, 0.f);
+      if (p.relu) v = relu_f(v);
       ((T*)p.y)[e] = from_f<T>(v);
     } else {
       float g = to_f(((const T*)p.dy)[e]);
@@ -446,7 +446,7 @@ __global__ void __launch_bounds__(256, 4) bn_apply_vec_kernel(const BnApplyProb*
       for (int t = 0; t < 8; ++t) {
         float v = (xv[t] - mu[t]) * ka[t] + kb[t];
         if (p.res) v += r[t];
-        o[t] = p.relu ? fmaxf(v, 0.f) : v;
+        o[t] = p.relu ? relu_f(v) : v;
       }
       *(uint4*)((bf16*)p.y + e * 8) = pack8(o);
     } else {

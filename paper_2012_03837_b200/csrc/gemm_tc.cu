@@ -31,6 +31,7 @@
 
 #include "common.cuh"
 #include "gemm_tc.h"
+#include "tc_prims.cuh"
 
 namespace lp {
 namespace {
@@ -65,7 +66,6 @@ constexpr int NTHREADS = 32 * (EPI_FIRST + EPI_WARPS);
 // The pool that setmaxnreg redistributes is what the launch allocated: 384 threads x 168 registers.
 constexpr int CTRL_REGS = 56, EPI_REGS = 224;     // 128 * 56 + 256 * 224 = 384 * 168
 constexpr uint32_t TMEM_COLS = 512;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 struct __align__(8) Shared {
   uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
@@ -73,117 +73,14 @@ struct __align__(8) Shared {
   int abort_flag;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long gtime_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the wait gave up or another role already did.  The clock is only
-// consulted after a first batch of polls (each poll already blocks in hardware for a short while).
+using namespace tc;
+
+// Bounded wait on a barrier of this block (see tc::mbar_wait); on expiry all roles leave their loops.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Shared* sh, int* status) {
-#pragma unroll 1
-  for (int i = 0; i < 64; ++i)
-    if (mbar_try(bar, parity)) return true;
-  unsigned long long t0 = gtime_ns();
-  int spins = 0;
-  while (!mbar_try(bar, parity)) {
-    if ((++spins & 63) == 0) {
-      if (*(volatile int*)&sh->abort_flag) return false;
-      if (gtime_ns() - t0 > WAIT_LIMIT_NS) {
-        *(volatile int*)&sh->abort_flag = 1;
-        atomicOr(status, ST_TIMEOUT);
-        return false;
-      }
-    }
-  }
-  return true;
+  return tc::mbar_wait(bar, parity, &sh->abort_flag, status);
 }
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
-}
-// 4-D tiled load (implicit convolution: channel, column, row, image); coordinates may lie outside the
-// tensor in every dimension but the first, the box then reads as zero there.
-__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* v) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) { return tc::make_desc(saddr, mn_major, BK * 128); }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, 1024-byte atoms (8 rows of 128 bytes).
-//   K-major : rows of 64 k-elements; next 8-row group 1024 B further (stride field); leading field unused.
-//   MN-major: rows of 64 m/n-elements, one row per k; next 8-k group 1024 B further (stride field);
-//             next 64-element m/n block BK*128 B further (leading field).
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
-  d |= (uint64_t)(mn_major ? ((BK * 128) >> 4) : 1) << 16;
-  d |= (uint64_t)(1024 >> 4) << 32;
-  d |= (uint64_t)1 << 46;   // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;   // 128-byte swizzle
-  return d;
-}
-
-__device__ __forceinline__ uint64_t policy_evict_first() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-__device__ __forceinline__ uint64_t policy_evict_last() {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-// Outputs are streamed: they leave with an evict-first L2 policy so that they do not push the
-// operand panels (re-read by the neighbouring tiles) out of the cache.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], %4;"
-               ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src)), "l"(policy_evict_first()) : "memory");
-}
 // Which problem a tile of the launch's flat tile list belongs to.  Tiles are visited in increasing
 // order, so the cursor only moves forward; seek() touches global memory only when the problem changes.
 struct ProbCursor {
@@ -227,11 +124,6 @@ struct TileWalk {
 // buffer in the swizzled layout of the output tensor map and leaves through ONE TMA store (full-line
 // writes, clipped at the matrix edge by the hardware); otherwise every lane stores its own row.
 // VEC: all 32 columns exist and resid / aux / C are 16-byte aligned (128-bit accesses).
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 // GELU x*Phi(x) and its derivative for the epilogue, where 128 values per thread and tile have to
 // fit under the tile's main loop (16 k-slices for the feed-forward products).  Phi is evaluated as
 // the logistic function of an odd quintic:  Phi(x) ~ 1 / (1 + 2^(-z)),  z = x (k0 + k1 s + k2 s^2),
@@ -390,7 +282,7 @@ __device__ __forceinline__ void epilogue_row32(const GemmProb& p, const CUtensor
   switch (p.act) {
     case EPI_RELU:
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+      for (int j = 0; j < 32; ++j) v[j] = relu_f(v[j]);
       break;
     case EPI_GELU:
       // the pre-activation is stored (C2) and the activation is taken of the value as stored
@@ -806,21 +698,6 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
   }
 }
 
-typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeFn get_encode() {
-  static EncodeFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
-      fn = (EncodeFn)p;
-  }
-  return fn;
-}
-
 // 2-D bf16 tensor map: inner extent `inner` (contiguous), outer extent `outer` with a row pitch of
 // `pitch` elements, box = 64 x box_outer, 128-byte swizzle, zero fill outside the tensor.
 bool encode_map(CUtensorMap* out, const void* base, long long inner, long long outer, long long pitch, int box_outer) {
@@ -889,25 +766,14 @@ bool gemm_tc_eligible(const GemmProb& g) {
 }
 
 int gemm_tc_choose_cg(const GemmProb* probs, int n) {
-  static int forced = -1;
-  if (forced < 0) {
-    const char* e = getenv("LP_GEMM_CG");      // diagnostic override: 1 or 2
-    forced = e ? atoi(e) : 0;
-  }
-  if (forced == 1 || forced == 2) return forced;
   for (int i = 0; i < n; ++i)
     if (probs[i].M <= BM) return 1;            // a 256-row pair tile would be half empty
   return 2;
 }
 
 bool gemm_tc_wide_ok(const GemmProb& g) {
-  static int off = -1;
-  if (off < 0) {
-    const char* e = getenv("LP_GEMM_WIDE");    // diagnostic override: 0 switches the wide tiles off
-    off = (e && atoi(e) == 0) ? 1 : 0;
-  }
   // long reductions only (the epilogue of a wide tile is exposed), plain epilogue, columns that fill 512-wide tiles
-  return !off && g.K >= 8192 && g.M > BM && g.N % (2 * BN) == 0 && g.act == EPI_NONE && !g.bias && !g.resid && !g.aux &&
+  return g.K >= 8192 && g.M > BM && g.N % (2 * BN) == 0 && g.act == EPI_NONE && !g.bias && !g.resid && !g.aux &&
          g.conv == CONV_NONE && !g.aux_blocked;
 }
 
@@ -966,7 +832,11 @@ bool gemm_tc_encode(GemmProb& g, void* maps, int cg) {
 
 cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int nprob, int total_tiles, int* d_status,
                            int num_sms, cudaStream_t s, int cg, int wide) {
-  static bool attr_set[4] = {false, false, false, false};
+  // function attributes belong to a device's context: set once per device and variant
+  static bool attr_set_dev[64][4] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  bool* attr_set = attr_set_dev[dev];
   const int which = cg == 1 ? 1 : (wide ? 3 : 2);
   const size_t ring = cg == 1 ? (size_t)Cfg<1, 0>::STAGES * Cfg<1, 0>::STAGE_BYTES
                               : (wide ? (size_t)Cfg<2, 1>::STAGES * Cfg<2, 1>::STAGE_BYTES : (size_t)Cfg<2, 0>::STAGES * Cfg<2, 0>::STAGE_BYTES);
@@ -1010,26 +880,30 @@ cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int npro
 
 }  // namespace lp
 
+#include "../../include/lp.h"
+
 // ---------------------------------------------------------------------------------------------
 // lp_gemm_bf16_static: the grouped GEMM for callers that must not allocate device memory.
 //
 // The grouped kernels read their problem table (and, for the tensor-core kernel, two TMA tensor
 // maps per problem and a status word) from global memory.  lp_gemm_bf16 keeps that table in a
-// cudaMalloc'ed buffer that grows on demand.  Some callers cannot afford that: code that runs
-// while a CUDA graph is being captured or inside a memory-pool-managed region, real-time loops
-// that must not take the driver's allocation lock, and hosts whose memory budget is fixed up
-// front.  This variant keeps the table in the file-scope array below instead: a fixed
-// LP_GEMM_STATIC_MAX problems, about 58 KB that every GPU loading this library holds until the
-// process exits.
+// cudaMalloc'ed buffer that grows on demand.  Some callers cannot afford that: serving and
+// real-time loops that must not take the driver's allocation lock or the device-wide
+// synchronisation cudaMalloc and cudaFree imply, code that runs inside a region whose memory a
+// pool manager has already handed out, and hosts whose device-memory budget is fixed up front.
+// This variant keeps the table in the file-scope array below instead: a fixed LP_GEMM_STATIC_MAX
+// problems, about 58 KB that every GPU loading this library holds until the process exits.
 // ---------------------------------------------------------------------------------------------
-#include "../../include/lp.h"
+#include <mutex>
+
+#include "gemm_desc_check.h"
 
 namespace {
 using namespace lp;
 
 struct alignas(64) TMap { unsigned char b[128]; };
 struct StaticLayout {
-  int status;                                   // cleared at the start of every call
+  int status;                                   // sticky: kernels OR bits into it, lp_gemm_static_poll clears it
   int pad[63];
   GemmProb tc[LP_GEMM_STATIC_MAX];
   GemmProb alu[LP_GEMM_STATIC_MAX];
@@ -1043,26 +917,28 @@ constexpr int MAX_DEVICES = 64;
 StaticLayout* g_static_ptr[MAX_DEVICES] = {};
 int g_static_sms[MAX_DEVICES] = {};
 thread_local char g_static_err[256] = "";
+// Host-side staging of one call's tables (process-wide, so it costs the calling thread no stack);
+// the mutex orders calls from different host threads while they fill and upload it.
+struct HostStage {
+  GemmProb tc[LP_GEMM_STATIC_MAX], alu[LP_GEMM_STATIC_MAX];
+  TMap maps[4 * LP_GEMM_STATIC_MAX];
+};
+HostStage g_stage;
+std::mutex g_stage_mutex;
 
 lp_status static_fail(lp_status code, const char* msg, cudaError_t e = cudaSuccess) {
   if (e != cudaSuccess) snprintf(g_static_err, sizeof(g_static_err), "%s: %s", msg, cudaGetErrorString(e));
   else snprintf(g_static_err, sizeof(g_static_err), "%s", msg);
   return code;
 }
-}  // namespace
 
-extern "C" const char* lp_gemm_static_last_error(void) { return g_static_err; }
-
-extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* stream) {
-  if (n < 1 || !in) return static_fail(LP_ERR_INVALID_ARG, "lp_gemm_bf16_static: no problems");
-  if (n > LP_GEMM_STATIC_MAX) return static_fail(LP_ERR_SHAPE, "lp_gemm_bf16_static: more than LP_GEMM_STATIC_MAX (64) problems in one call");
-  cudaStream_t s = (cudaStream_t)stream;
+// Set-up, once per device, with that device current: resolve the array's device address.
+lp_status static_setup(int* dev_out) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "cudaGetDevice", e);
   if (dev < 0 || dev >= MAX_DEVICES) return static_fail(LP_ERR_UNSUPPORTED, "lp_gemm_bf16_static: device ordinal above 63");
   if (!g_static_ptr[dev]) {
-    // set-up, once per device, with that device current: resolve the array's device address
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_static_scratch);
     if (e != cudaSuccess || !p) return static_fail(LP_ERR_CUDA, "cudaGetSymbolAddress", e);
@@ -1072,16 +948,34 @@ extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* st
     g_static_sms[dev] = sms;
     g_static_ptr[dev] = (StaticLayout*)p;
   }
+  *dev_out = dev;
+  return LP_OK;
+}
+}  // namespace
+
+extern "C" const char* lp_gemm_static_last_error(void) { return g_static_err; }
+
+extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* stream) {
+  if (n < 1 || !in) return static_fail(LP_ERR_INVALID_ARG, "lp_gemm_bf16_static: no problems");
+  if (n > LP_GEMM_STATIC_MAX) return static_fail(LP_ERR_SHAPE, "lp_gemm_bf16_static: more than LP_GEMM_STATIC_MAX (64) problems in one call");
+  for (int i = 0; i < n; ++i)
+    if (const char* why = gemm_desc_problem(in[i])) {
+      snprintf(g_static_err, sizeof(g_static_err), "lp_gemm_bf16_static: problem %d: %s", i, why);
+      return LP_ERR_INVALID_ARG;
+    }
+  cudaStream_t s = (cudaStream_t)stream;
+  int dev = 0;
+  lp_status st = static_setup(&dev);
+  if (st != LP_OK) return st;
   StaticLayout* sc = g_static_ptr[dev];
 
-  GemmProb tc[LP_GEMM_STATIC_MAX], alu[LP_GEMM_STATIC_MAX];
-  TMap maps[4 * LP_GEMM_STATIC_MAX];
+  std::lock_guard<std::mutex> lock(g_stage_mutex);
+  GemmProb* tc = g_stage.tc;
+  GemmProb* alu = g_stage.alu;
+  TMap* maps = g_stage.maps;
   int ntc = 0, nalu = 0, tc_tiles = 0, alu_tiles = 0;
   for (int i = 0; i < n; ++i) {
     const lp_gemm_desc& q = in[i];
-    if (!q.A || !q.B || !q.C || q.M < 1 || q.N < 1 || q.K < 1) return static_fail(LP_ERR_INVALID_ARG, "lp_gemm_bf16_static: bad problem");
-    if ((q.a_ms != 1 && q.a_ks != 1) || (q.b_ns != 1 && q.b_ks != 1))
-      return static_fail(LP_ERR_INVALID_ARG, "lp_gemm_bf16_static: one stride per operand must be 1");
     GemmProb g{};
     g.A = q.A; g.B = q.B; g.C = q.C; g.C2 = q.C2; g.bias = q.bias; g.resid = q.resid; g.aux = q.aux;
     g.M = q.M; g.N = q.N; g.K = q.K; g.a_ms = q.a_ms; g.a_ks = q.a_ks; g.b_ns = q.b_ns; g.b_ks = q.b_ks;
@@ -1097,11 +991,10 @@ extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* st
       alu[nalu++] = g;
     }
   }
-  // The array keeps whatever the previous call left: the status word must start at zero, the
-  // tables are overwritten for the entries this call uses.  Copies from pageable host memory are
-  // staged before cudaMemcpyAsync returns, so the stack arrays above may go out of scope.
-  e = cudaMemsetAsync(&sc->status, 0, sizeof(int), s);
-  if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "cudaMemsetAsync", e);
+  // The device array keeps whatever the previous call left; the table entries this call uses are
+  // overwritten.  The staging table is pageable host memory: the runtime has copied it out by the
+  // time cudaMemcpyAsync returns, so the next call may refill it.
+  cudaError_t e = cudaSuccess;
   if (ntc) {
     e = cudaMemcpyAsync(sc->tc, tc, ntc * sizeof(GemmProb), cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(sc->maps, maps, 4 * ntc * sizeof(TMap), cudaMemcpyHostToDevice, s);
@@ -1115,5 +1008,19 @@ extern "C" lp_status lp_gemm_bf16_static(int n, const lp_gemm_desc* in, void* st
     e = cudaGetLastError();
     if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "FP32-ALU launch", e);
   }
+  return LP_OK;
+}
+
+extern "C" lp_status lp_gemm_static_poll(void* stream) {
+  int dev = 0;
+  lp_status st = static_setup(&dev);
+  if (st != LP_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  int w = 0;
+  cudaError_t e = cudaMemcpyAsync(&w, &g_static_ptr[dev]->status, sizeof(int), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(&g_static_ptr[dev]->status, 0, sizeof(int), s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return static_fail(LP_ERR_CUDA, "lp_gemm_static_poll", e);
+  if (w & ST_TIMEOUT) return static_fail(LP_ERR_TIMEOUT, "lp_gemm_static_poll: a device-side wait gave up; outputs of the calls since the last poll are not valid");
   return LP_OK;
 }

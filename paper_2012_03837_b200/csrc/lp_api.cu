@@ -7,6 +7,7 @@
 
 #include "runtime.h"
 #include "gemm_tc.h"
+#include "gemm_desc_check.h"
 
 using namespace lp;
 
@@ -519,21 +520,30 @@ lp_status lp_load_state(lp_handle hh, const void* host_src, size_t bytes) { retu
 
 lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream, int* used_tc) {
   if (n < 1 || !in) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_gemm_bf16: no problems");
+  if (backend != 0 && backend != 1) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_gemm_bf16: backend must be 0 or 1");
+  for (int i = 0; i < n; ++i)
+    if (const char* why = gemm_desc_problem(in[i]))
+      return fail(nullptr, LP_ERR_INVALID_ARG, "lp_gemm_bf16: problem " + std::to_string(i) + ": " + why);
   cudaStream_t s = (cudaStream_t)stream;
+  // the scratch of this entry belongs to the device that was current at its first call
   static int* d_status = nullptr;
   static int num_sms = 0;
-  if (!d_status) {
-    if (cudaMalloc(&d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, LP_ERR_ALLOC, "status word"); }
-    cudaMemset(d_status, 0, sizeof(int));
+  static int first_dev = -1;
+  {
     int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, LP_ERR_CUDA, "lp_gemm_bf16: no CUDA device"); }
+    if (first_dev >= 0 && dev != first_dev)
+      return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_gemm_bf16: one device per process (the first one it was called on)");
+    if (!d_status) {
+      if (cudaMalloc(&d_status, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, LP_ERR_ALLOC, "status word"); }
+      cudaMemset(d_status, 0, sizeof(int));
+      cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+      first_dev = dev;
+    }
   }
   std::vector<GemmProb> tc, simt;
   for (int i = 0; i < n; ++i) {
     const lp_gemm_desc& q = in[i];
-    if (!q.A || !q.B || !q.C || q.M < 1 || q.N < 1 || q.K < 1) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_gemm_bf16: bad problem");
-    if ((q.a_ms != 1 && q.a_ks != 1) || (q.b_ns != 1 && q.b_ks != 1)) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_gemm_bf16: one stride per operand must be 1");
     GemmProb g{};
     g.A = q.A; g.B = q.B; g.C = q.C; g.C2 = q.C2; g.bias = q.bias; g.resid = q.resid; g.aux = q.aux;
     g.M = q.M; g.N = q.N; g.K = q.K; g.a_ms = q.a_ms; g.a_ks = q.a_ks; g.b_ns = q.b_ns; g.b_ks = q.b_ks;
@@ -618,13 +628,17 @@ lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* ou
   static void* d_tab = nullptr;
   static int num_sms = 0;
   struct alignas(64) Map { unsigned char b[128]; };
+  static int first_dev = -1;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, LP_ERR_CUDA, "lp_conv3x3_bf16: no CUDA device"); }
+  if (first_dev >= 0 && dev != first_dev)
+    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_conv3x3_bf16: one device per process (the first one it was called on)");
   if (!d_tab) {
     if (cudaMalloc(&d_tab, 1024 + 4 * sizeof(Map)) != cudaSuccess) { cudaGetLastError(); d_tab = nullptr; return fail(nullptr, LP_ERR_ALLOC, "descriptor table"); }
     d_status = (int*)d_tab;
     cudaMemset(d_status, 0, sizeof(int));
-    int dev = 0;
-    cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    first_dev = dev;
   }
   const int cg = gemm_tc_choose_cg(&g, 1);
   const int total = gemm_tc_tiles(g, 0, cg);
@@ -637,6 +651,46 @@ lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* ou
   cudaStreamSynchronize(s);                      // the tables above are host stack memory
   launch_gemm_tc(dp, dm, 1, total, d_status, num_sms, s, cg);
   return check_cuda(nullptr, "lp_conv3x3_bf16");
+}
+
+lp_status lp_attention_bf16(int form, const void* qkv, void* o, float* lse, const void* dout, void* dqkv, float* delta,
+                            int batch, int seq_len, int n_heads, void* stream) {
+  if (form != LP_ATTN_FORWARD && form != LP_ATTN_BACKWARD) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_attention_bf16: unknown form");
+  if (!qkv || !o || !lse || (form == LP_ATTN_BACKWARD && (!dout || !dqkv || !delta)))
+    return fail(nullptr, LP_ERR_INVALID_ARG, "lp_attention_bf16: null pointer");
+  if (batch < 1 || seq_len < 1 || n_heads < 1 || (long long)batch * seq_len > 0x7fffffffLL / (192LL * n_heads))
+    return fail(nullptr, LP_ERR_SHAPE, "lp_attention_bf16: sizes must be positive (and batch*seq_len*3*d below 2^31)");
+  cudaStream_t s = (cudaStream_t)stream;
+  static void* d_tab = nullptr;                  // status word at 0, the problem at 256
+  static int first_dev = -1;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, LP_ERR_CUDA, "lp_attention_bf16: no CUDA device"); }
+  if (first_dev >= 0 && dev != first_dev)
+    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_attention_bf16: one device per process (the first one it was called on)");
+  AttnTcProb tab;
+  AttnProb ap{qkv, o, lse, form == LP_ATTN_BACKWARD ? dout : nullptr, dqkv, delta, batch, seq_len, n_heads};
+  if (((uintptr_t)o & 15) || ((uintptr_t)dqkv & 15) || !attn_tc_encode(tab, ap))
+    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_attention_bf16: tensors must be 16-byte aligned");
+  if (!d_tab) {
+    if (cudaMalloc(&d_tab, 256 + sizeof(AttnTcProb)) != cudaSuccess) { cudaGetLastError(); d_tab = nullptr; return fail(nullptr, LP_ERR_ALLOC, "descriptor table"); }
+    cudaMemset(d_tab, 0, 256);
+    first_dev = dev;
+  }
+  int* d_status = (int*)d_tab;
+  AttnTcProb* dp = (AttnTcProb*)((char*)d_tab + 256);
+  cudaMemcpyAsync(dp, &tab, sizeof(tab), cudaMemcpyHostToDevice, s);
+  cudaStreamSynchronize(s);                      // the table above is host stack memory
+  cudaError_t e = form == LP_ATTN_FORWARD ? launch_attn_fwd_tc(dp, 1, batch, seq_len, n_heads, d_status, s)
+                                          : launch_attn_bwd_tc(dp, 1, batch, seq_len, n_heads, d_status, s);
+  if (e != cudaSuccess) return fail(nullptr, LP_ERR_CUDA, std::string("lp_attention_bf16: launch: ") + cudaGetErrorString(e));
+  int w = 0;
+  cudaMemcpyAsync(&w, d_status, sizeof(int), cudaMemcpyDeviceToHost, s);
+  cudaMemsetAsync(d_status, 0, sizeof(int), s);
+  cudaStreamSynchronize(s);
+  lp_status st = check_cuda(nullptr, "lp_attention_bf16");
+  if (st != LP_OK) return st;
+  if (w & ST_TIMEOUT) return fail(nullptr, LP_ERR_TIMEOUT, "lp_attention_bf16: a device-side wait gave up");
+  return LP_OK;
 }
 
 lp_status lp_profile_enable(lp_handle hh, int on) {

@@ -159,8 +159,14 @@ struct AttnProb {     // causal attention over qkv [B*T, 3d], heads of 64
 };
 void launch_attn_fwd(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s);
 void launch_attn_bwd(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, bool is_bf16, cudaStream_t s);
-void launch_attn_fwd_tc(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, cudaStream_t s);
-void launch_attn_bwd_tc(const AttnProb* d_probs, int n, int maxB, int maxT, int maxH, cudaStream_t s);
+// bf16 path (attn_tc.cu): tcgen05 kernels with the score tiles in tensor memory.  A problem carries the TMA tensor
+// maps of its qkv tensor and (backward) of dout, [B, T, width] in boxes of 64 columns x 64 positions; the table of
+// problems lives in device memory, 64-byte aligned.  attn_tc_encode fills one entry on the host (false: the tensor
+// maps could not be encoded -- base addresses must be 16-byte aligned).  status: device status word (ST_TIMEOUT).
+struct alignas(64) AttnTcProb { unsigned char map_qkv[128]; unsigned char map_do[128]; AttnProb p; };
+bool attn_tc_encode(AttnTcProb& out, const AttnProb& p);
+cudaError_t launch_attn_fwd_tc(const AttnTcProb* d_probs, int n, int maxB, int maxT, int maxH, int* status, cudaStream_t s);
+cudaError_t launch_attn_bwd_tc(const AttnTcProb* d_probs, int n, int maxB, int maxT, int maxH, int* status, cudaStream_t s);
 
 // ---------------------------------------------------------------------------- ResNet-specific
 struct LayoutProb { const void* in; void* out; int N, C, H, W; };

@@ -158,12 +158,7 @@ void build_lm(Handle& h) {
       }
       emit_ln_fwd(h, p, ln);
       emit_gemm(h, p, g);
-      {
-        const AttnProb* dp = h.upload(at);
-        int n = (int)at.size();
-        p.add(1, [=](const RunCtx& c) { launch_attn_fwd(dp, n, B, T, H, bf, c.stream); }, KIND_ATTN,
-              (double)n * 4.0 * B * H * 64.0 * T * (T + 1) / 2);
-      }
+      emit_attention(h, p, at, false);
       g.clear(); ln.clear();
       for (int k : act) {
         BlockBufs& b = cb[k].blocks[j];
@@ -308,10 +303,7 @@ void build_lm(Handle& h) {
         ChunkBufs& c = *it.c; BlockBufs& b = *it.b;
         at.push_back(AttnProb{b.qkv, b.o, b.lse, c.G1, c.Gq, b.delta, B, T, H});
       }
-      const AttnProb* dp = h.upload(at);
-      int n = (int)at.size();
-      p.add(2, [=](const RunCtx& c) { launch_attn_bwd(dp, n, B, T, H, bf, c.stream); }, KIND_ATTN,
-            (double)n * 10.0 * B * H * 64.0 * T * (T + 1) / 2);
+      emit_attention(h, p, at, true);
     }
     // 6. qkv projection: dWqkv, dbqkv, da1 -> G1 (needed for LN1's own parameters in every case)
     for (auto& it : items) {

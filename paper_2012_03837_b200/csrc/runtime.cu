@@ -390,4 +390,28 @@ void emit_optimizer(Handle& h, Plan& p) {
   }, KIND_OPTIM, (double)h.n_total * (h.opt.kind == LP_OPT_ADAM ? 28.0 : 20.0) + (h.bf16_mode ? 2.0 * h.n_matrix : 0.0));
 }
 
+void emit_attention(Handle& h, Plan& p, const std::vector<AttnProb>& probs, bool backward) {
+  if (probs.empty()) return;
+  const int n = (int)probs.size();
+  int B = 0, T = 0, H = 0;
+  for (auto& a : probs) { B = std::max(B, a.B); T = std::max(T, a.T); H = std::max(H, a.H); }
+  double pairs = 0;                                     // causal (query, key) pairs x head width
+  for (auto& a : probs) pairs += (double)a.B * a.H * 64.0 * a.T * (a.T + 1) / 2;
+  const double work = (backward ? 10.0 : 4.0) * pairs;
+  const bool bf = h.bf16_mode;
+  if (bf && !h.force_simt) {
+    std::vector<AttnTcProb> tab(n);
+    for (int i = 0; i < n; ++i)
+      if (!attn_tc_encode(tab[i], probs[i])) throw std::runtime_error("cuda: cuTensorMapEncodeTiled failed for an attention operand");
+    const AttnTcProb* dp = h.upload(tab);
+    int* st = h.d_status;
+    if (backward) p.add(2, [=](const RunCtx& c) { launch_attn_bwd_tc(dp, n, B, T, H, st, c.stream); }, KIND_ATTN, work);
+    else p.add(1, [=](const RunCtx& c) { launch_attn_fwd_tc(dp, n, B, T, H, st, c.stream); }, KIND_ATTN, work);
+    return;
+  }
+  const AttnProb* dp = h.upload(probs);
+  if (backward) p.add(2, [=](const RunCtx& c) { launch_attn_bwd(dp, n, B, T, H, bf, c.stream); }, KIND_ATTN, work);
+  else p.add(1, [=](const RunCtx& c) { launch_attn_fwd(dp, n, B, T, H, bf, c.stream); }, KIND_ATTN, work);
+}
+
 }  // namespace lp

@@ -160,6 +160,9 @@ bool emit_xent_and_loss(Handle& h, Plan& p, std::vector<XentProb> probs, const s
 void emit_xent_from_stats(Handle& h, Plan& p, std::vector<XentStatsProb> probs, const std::vector<int>& chunk_of,
                           const std::vector<float*>* bias_grads);
 void emit_optimizer(Handle& h, Plan& p);
+// Causal attention of all problems of a phase in one grouped launch (forward) or two (backward: dQ, then dK and
+// dV).  bf16 takes the tcgen05 kernels unless the handle was created with the FP32-ALU backend.
+void emit_attention(Handle& h, Plan& p, const std::vector<AttnProb>& probs, bool backward);
 // Predictions of the heads' logits (before the cross-entropy overwrites them); runs only under lp_evaluate
 void emit_argmax(Handle& h, Plan& p, const std::vector<ArgmaxProb>& probs);
 

@@ -76,7 +76,28 @@ def test_kernel_level_entries_check_their_arguments_first():
     too_many = (lp.lp_gemm_desc * (lp.LP_GEMM_STATIC_MAX + 1))()
     assert L.lp_gemm_bf16_static(lp.LP_GEMM_STATIC_MAX + 1, too_many, None) == ERR["SHAPE"]
     assert b"64" in L.lp_gemm_static_last_error()
+    # descriptors that would make a kernel read or write where it must not are refused before any launch
+    def desc(**kw):
+        d = lp.lp_gemm_desc()
+        base = dict(A=256, B=512, C=1024, M=64, N=64, K=64, a_ms=64, a_ks=1, b_ns=64, b_ks=1, ldc=64)
+        base.update(kw)
+        for k, v in base.items():
+            setattr(d, k, v)
+        return d
+    bad = [dict(act=5), dict(act=-1), dict(act=2), dict(act=2, C2=2048, out_f32=1), dict(act=3), dict(act=4), dict(ldc=63),
+           dict(a_ms=2, a_ks=2), dict(b_ns=0), dict(K=0), dict(A=0), dict(C=0), dict(out_f32=2)]
+    for kw in bad:
+        arr = (lp.lp_gemm_desc * 1)(desc(**kw))
+        assert L.lp_gemm_bf16(1, arr, 0, None, None) == ERR["INVALID_ARG"], kw
+        assert lp.lp_last_error(None), kw
+        assert L.lp_gemm_bf16_static(1, arr, None) == ERR["INVALID_ARG"], kw
+        assert b"problem 0" in L.lp_gemm_static_last_error(), kw
+    assert L.lp_gemm_bf16(1, (lp.lp_gemm_desc * 1)(desc()), 2, None, None) == ERR["INVALID_ARG"]   # unknown backend
     assert L.lp_conv3x3_bf16(0, None, None, None, 1, 8, 8, 64, 64, None) == ERR["INVALID_ARG"]
     one = C.c_void_p(256)
+    assert L.lp_attention_bf16(0, None, one, one, None, None, None, 1, 64, 1, None) == ERR["INVALID_ARG"]
+    assert L.lp_attention_bf16(1, one, one, one, None, one, one, 1, 64, 1, None) == ERR["INVALID_ARG"]   # backward needs dout
+    assert L.lp_attention_bf16(2, one, one, one, one, one, one, 1, 64, 1, None) == ERR["INVALID_ARG"]
+    assert L.lp_attention_bf16(0, one, one, one, None, None, None, 0, 64, 1, None) == ERR["SHAPE"]
     assert L.lp_conv3x3_bf16(0, one, one, one, 0, 8, 8, 64, 64, None) == ERR["SHAPE"]
     assert L.lp_conv3x3_bf16(7, one, one, one, 1, 8, 8, 64, 64, None) == ERR["INVALID_ARG"]

@@ -1,12 +1,18 @@
 """Parity at the full sizes of the five workloads, in the launch configuration bench.py times.
 
-c1 runs in test_gpu_parity.py.  c2 runs all ten steps against the oracle.  c3 and c4 run three steps
-(an oracle step costs 10-20 s of CPU there).  c5 (55 TFLOP per step) is checked on what the oracle can
-compute one by one: chunks 0 and 1 of the 24 (their weights do not depend on the chunks above them, so a
-two-chunk oracle with the same seeded weights reproduces them exactly), plus properties that hold at
-any size (initial losses near ln V for every chunk, first Adam step bounded by the learning rate).
+c1 runs in test_gpu_parity.py.  c2, c3 and c4 run ten steps against the oracle.  c2's bounds follow, step by
+step, what two correct evaluations of that workload differ by (tests/golden/c2_conditioning.json, made by the
+CPU oracle alone): 2e-2 while that stays below 1e-2, twice the oracle-against-oracle gap afterwards.  c5
+(55 TFLOP per step) is checked on what the oracle can compute one by one.  A chunk's update depends on the
+chunks below it only through the activation it receives (Sec. 3), so (a) for chunks 0, 1, 12 and 23 the oracle
+forms the input by a forward pass through the blocks below and one local update of that chunk alone, and (b) a
+three-chunk oracle with the same seeded weights reproduces chunks 0-2 of the 24 over three pipelined steps
+(both halves of the boundary buffers, labels carried with the activations); plus properties that hold at any
+size (initial losses near ln V for every chunk, first Adam step bounded by the learning rate).
 """
+import json
 import math
+import os
 
 import numpy as np
 import pytest
@@ -19,72 +25,146 @@ from tests.test_gpu_parity import check
 
 pytestmark = pytest.mark.gpu
 
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "c2_conditioning.json")
+
+
+def matrix_gaps(gm, orc):
+    """Per chunk: the largest ||a-b||_2 / ||b||_2 over its weight matrices."""
+    got = gm.get(lp.LP_MASTER)
+    out = [0.0] * gm.K
+    for n, a in got.items():
+        if a.ndim >= 2:
+            k = gm.index[n][1]["chunk"]
+            b = orc.p[n].astype(np.float64)
+            out[k] = max(out[k], float(np.linalg.norm(a.astype(np.float64) - b) / np.linalg.norm(b)))
+    return out
+
+
+def run_c2(cfg, witness, base_w, base_loss):
+    """Ten steps of c2, compared after every step.  Bound at step t, chunk k: max(base, 2 x the gap between two
+    correct evaluations at that step and chunk) for the weights; for the losses max(base, 2 x the largest such
+    gap of the ten steps) -- the transient of a loss gap moves down the pipeline with the minibatch that caused
+    it, so it is not tied to one step."""
+    gold = json.load(open(GOLDEN))["steps"]
+    loss_tol = max(base_loss, 2 * max(max(s[witness]["loss"]) for s in gold))
+    params = lp_synth.init_params(cfg)
+    gm = T.GpuModel(cfg, params)
+    orc = LocalUpdateOracle(cfg, params, dtype=np.float32)
+    report = []
+    for t in range(10):
+        x, y = lp_synth.minibatch(cfg, t)
+        gl, ol = gm.step(x, y), orc.step(x, y)
+        lerr = np.abs(gl - ol) / np.abs(ol)
+        w = matrix_gaps(gm, orc)
+        tol = [max(base_w, 2 * g) for g in gold[t][witness]["weights"]]
+        report.append((t + 1, float(lerr.max()), max(w), max(tol)))
+        print(f"c2 {cfg['dtype']} step {t + 1}: loss err {lerr.max():.2e} (tol {loss_tol:.2e}); weights per chunk",
+              [f"{a:.1e}/{b:.1e}" for a, b in zip(w, tol)])
+        assert lerr.max() <= loss_tol, (t, lerr)
+        assert all(a <= b for a, b in zip(w, tol)), (t, w, tol)
+    gm.close()
+    return report
+
 
 def test_c2_wide_mlp_full_size_fp32_storage():
-    """The c2 network and schedule with fp32 storage (FP32-ALU kernels).  This shows how ill-conditioned the
-    workload is: Adam's first step moves every weight by +-1e-3 (a thirtieth of the He-normal scale 0.031)
-    whatever its gradient's size, the losses fall to ln 1000 within ten steps, and fp32 summation-order
-    differences alone grow to 2.5e-2 of the weight norm and 5e-3 of a loss (a transient that follows
-    minibatch 1 down the pipeline).  No implementation whose rounding order differs from the oracle's can do
-    better, so these bounds, not 1e-3, are what this network admits."""
-    check(lp_synth.config("c2", dtype="fp32"), steps=10, grads_first=False, w_tol=5e-2, v_tol=0.5, loss_tol=1e-2)
+    """The c2 network and schedule with fp32 storage (FP32-ALU kernels) against the fp32 oracle: two fp32
+    evaluations that differ in summation order only.  The witness is the oracle in fp32 against itself in fp64,
+    which reaches 2.2e-2 of a weight matrix's norm after ten steps on the CPU alone."""
+    run_c2(lp_synth.config("c2", dtype="fp32"), "fp32_vs_fp64", 1e-3, 1e-4)
 
 
 def test_c2_wide_mlp_bf16_full_size():
-    # On top of the above, bf16 activation rounding flips ReLU decisions behind up to 14 layers: measured
-    # 5.6e-2 of the weight norm at chunk 7 (1.5e-2 at chunk 0) and 3e-2 on one loss of the same transient.
-    check(lp_synth.config("c2"), steps=10, grads_first=False, w_tol=1e-1, v_tol=0.6, loss_tol=5e-2)
+    """bf16 storage.  The witness is the fp32 oracle with nothing but its chunk outputs rounded to bf16, against
+    the plain fp32 oracle: 2e-2 is crossed at step 4 and 5.4e-2 is reached at step 10 on the CPU alone."""
+    run_c2(lp_synth.config("c2"), "bf16io_vs_fp32", 2e-2, 2e-2)
 
 
 def test_c3_transformer_bf16_full_size():
-    check(lp_synth.config("c3"), steps=3, grads_first=False)
+    check(lp_synth.config("c3"), steps=10, grads_first=False)
 
 
 def test_c4_resnet_bf16_full_size():
-    check(lp_synth.config("c4"), steps=3, grads_first=False, v_tol=0.3)
+    check(lp_synth.config("c4"), steps=10, grads_first=False, v_tol=0.3)
 
 
-def test_c5_large_transformer_sampled_chunks():
+def l2_rel(a, b):
+    a, b = a.astype(np.float64), b.astype(np.float64)
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
+
+
+def test_c5_large_transformer_sampled_chunks_and_pipelined_steps():
     cfg = lp_synth.config("c5")
-    small = lp_synth.config("c5", blocks_per_chunk=[1, 1])
-    p_small = lp_synth.init_params(small)
+    K = lp_synth.num_chunks(cfg)
     params = lp_synth.init_params(cfg)
-    for n, a in p_small.items():                     # same seeded stream per tensor index
-        assert np.array_equal(a, params[n]), n
     gm = T.GpuModel(cfg, params)
-    del params
-    x, y = lp_synth.minibatch(cfg, 0)
-    losses = gm.step(x, y)                           # pipelined step 0: priming forward + one update of all 24 chunks
+    lr = cfg["optim"]["lr"]
     # logits of a fresh head are N(0, s^2) with s^2 = 0.02^2 * d_model (LayerNorm output has unit variance), so
     # the expected loss is ln V + s^2 / 2 (log-normal mean of the partition function)
     expect0 = math.log(cfg["vocab"]) + 0.5 * 0.02 ** 2 * cfg["d_model"]
-    assert np.all(np.abs(losses - expect0) < 0.05), losses
 
-    orc = LocalUpdateOracle(small, p_small, dtype=np.float32)
-    ol = orc.step(x, y, "pipelined")
-    print("c5 step-0 losses chunk 0/1: gpu", losses[:2], "oracle", ol)
-    assert np.all(np.abs(losses[:2] - ol) / np.abs(ol) <= 2e-2)
-
+    # ---- (a) step 0 (pipelined, primed: every chunk trains on minibatch 0), chunks 0, 1, 12, 23
+    x0, y0 = lp_synth.minibatch(cfg, 0)
+    losses0 = gm.step(x0, y0)
+    assert np.all(np.abs(losses0 - expect0) < 0.05), losses0
+    full = LocalUpdateOracle(cfg, params, dtype=np.float32)
+    sampled = (0, 1, 12, 23)
+    inputs, h = {}, full._cast_input(x0)
+    for k in range(K):
+        if k in sampled:
+            inputs[k] = h
+        if k < K - 1:
+            h, _ = full.chunk_forward(k, h)          # initial weights: the priming pass of the first pipelined step
     worst_g, worst_w = 0.0, 0.0
+    for k in sampled:
+        loss, _, grads = full.local_grads(k, inputs[k], y0)
+        full.apply_update(k, grads)
+        assert abs(losses0[k] - loss) / abs(loss) <= 2e-2, (k, losses0[k], loss)
+        for n, g_ref in grads.items():
+            i, info = gm.index[n]
+            g = np.empty(info["shape"], np.float32)
+            w = np.empty(info["shape"], np.float32)
+            lp.lp_get_tensor(gm.h, i, lp.LP_GRAD, g, gm.stream)
+            lp.lp_get_tensor(gm.h, i, lp.LP_MASTER, w, gm.stream)
+            if g.ndim == 2:
+                ge = l2_rel(g, g_ref)
+                worst_g = max(worst_g, ge)
+                assert ge <= 0.1, (n, ge)            # bf16 rounding of the activations: a few percent in l2
+                we = l2_rel(w, full.p[n])
+                worst_w = max(worst_w, we)
+                assert we <= 2e-2, (n, we)
+            # first Adam step: |dw| = lr |g| / (|g| + eps) <= lr
+            dw = np.abs(w.astype(np.float64) - params[n].astype(np.float64)).max()
+            assert dw <= lr * (1 + 1e-3), (n, dw)
+        print(f"c5 step 0 chunk {k}: loss gpu {losses0[k]:.5f} oracle {loss:.5f}")
+    print("c5 sampled chunks: worst first-step matrix gradient error (l2)", worst_g, "worst matrix error after the update", worst_w)
+    del full, inputs
+
+    # ---- (b) three pipelined steps, chunks 0-2 against a three-chunk oracle (same seeded tensors)
+    small = lp_synth.config("c5", blocks_per_chunk=[1, 1, 1])
+    p_small = lp_synth.init_params(small)
+    for n, a in p_small.items():                     # same seeded stream per tensor
+        assert np.array_equal(a, params[n]), n
+    del params
+    orc = LocalUpdateOracle(small, p_small, dtype=np.float32)
+    ol = orc.step(x0, y0, "pipelined")
+    assert np.all(np.abs(losses0[:3] - ol) / np.abs(ol) <= 2e-2), (losses0[:3], ol)
+    for t in (1, 2):
+        x, y = lp_synth.minibatch(cfg, t)
+        gl = gm.step(x, y)
+        ol = orc.step(x, y, "pipelined")
+        print(f"c5 pipelined step {t}: losses chunk 0-2 gpu", gl[:3], "oracle", ol)
+        assert np.all(np.abs(gl[:3] - ol) / np.abs(ol) <= 2e-2), (t, gl[:3], ol)
+        # chunks k > 0 see an older minibatch again with the labels they have just trained on: every loss stays
+        # finite and in the neighbourhood of its initial value
+        assert np.all(np.isfinite(gl)) and np.all(np.abs(gl - expect0) < 1.5), gl
+    worst = 0.0
     for n in p_small:
         i, info = gm.index[n]
-        g = np.empty(info["shape"], np.float32)
-        w = np.empty(info["shape"], np.float32)
-        lp.lp_get_tensor(gm.h, i, lp.LP_GRAD, g, gm.stream)
-        lp.lp_get_tensor(gm.h, i, lp.LP_MASTER, w, gm.stream)
-        ge = T.tensor_rel_err(T.strip_key_bias(n, g), T.strip_key_bias(n, orc.last_grads[n]))
-        worst_g = max(worst_g, ge)
-        # first Adam step: |dw| = lr |g| / (|g| + eps) <= lr
-        dw = np.abs(w.astype(np.float64) - p_small[n].astype(np.float64)).max()
-        assert dw <= cfg["optim"]["lr"] * (1 + 1e-3), (n, dw)
-        if w.ndim == 2:
-            we = np.linalg.norm(w.astype(np.float64) - orc.p[n]) / np.linalg.norm(orc.p[n])
-            worst_w = max(worst_w, we)
-    print("c5 chunk 0/1: worst first-step gradient error", worst_g, "worst matrix error after the update", worst_w)
-    assert worst_g <= 0.35
-    assert worst_w <= 2e-2
-    # one more step keeps every loss finite and in the neighbourhood of the initial value (chunks k > 0 now see
-    # minibatch 0 again, one chunk further down, with the labels they have just trained on: their loss drops ~0.4)
-    losses2 = gm.step(*lp_synth.minibatch(cfg, 1))
-    assert np.all(np.isfinite(losses2)) and np.all(np.abs(losses2 - expect0) < 1.0), losses2
+        if len(info["shape"]) == 2:
+            w = np.empty(info["shape"], np.float32)
+            lp.lp_get_tensor(gm.h, i, lp.LP_MASTER, w, gm.stream)
+            e = l2_rel(w, orc.p[n])
+            worst = max(worst, e)
+            assert e <= 2e-2, (n, e)
+    print("c5 chunks 0-2 after three pipelined steps: worst matrix error", worst)
     gm.close()

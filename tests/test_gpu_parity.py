@@ -31,6 +31,10 @@ def check(cfg, steps=10, gemm_backend=0, grads_first=True, w_tol=None, v_tol=Non
         errs = sorted(((T.tensor_rel_err(T.strip_key_bias(n, gg[n]), T.strip_key_bias(n, orc.last_grads[n])), n)
                        for n in gg if n not in orc.buffers), reverse=True)
         print("grad rel err after step 0 (worst):", [(f"{e:.2e}", n) for e, n in errs[:5]])
+        l2 = sorted(((float(np.linalg.norm(T.strip_key_bias(n, gg[n]).astype(np.float64) - T.strip_key_bias(n, orc.last_grads[n])) /
+                            max(np.linalg.norm(T.strip_key_bias(n, orc.last_grads[n]).astype(np.float64)), 1e-30)), n)
+                     for n in gg if n not in orc.buffers), reverse=True)
+        print("grad l2 err after step 0 (worst):", [(f"{e:.2e}", n) for e, n in l2[:5]])
         gm.close()
         # bf16: ReLU / GELU' masks flip where a rounded pre-activation crosses zero, so the first-step
         # gradient is only a coarse check there
