@@ -40,6 +40,7 @@ enum {
 };
 
 enum { LP_FAMILY_MLP = 0, LP_FAMILY_LM = 1, LP_FAMILY_RESNET = 2 };
+enum { LP_BLOCK_BASIC = 0, LP_BLOCK_BOTTLENECK = 1 };
 enum { LP_FP32 = 0, LP_BF16 = 1 }; /* LP_BF16: bf16 matrices and activations, fp32 master weights,
                                       fp32 accumulation, fp32 normalisation statistics and loss  */
 enum { LP_HEAD_LINEAR = 0, LP_HEAD_LN_LINEAR = 1, LP_HEAD_GAP_LINEAR = 2, LP_HEAD_BN_RELU_GAP_LINEAR = 3 };
@@ -58,8 +59,9 @@ enum { LP_MASTER = 0, LP_WORKING = 1, LP_MOMENT1 = 2, LP_MOMENT2 = 3, LP_GRAD = 
  *    (n_heads heads of d_model/n_heads = 64) and a GELU feed-forward of width d_ffn; chunk k holds
  *    blocks_per_chunk[k] blocks.
  *  RESNET (App. B.3): 3x3 stem convolution + BatchNorm + ReLU (in chunk 0), then K stages of
- *    blocks_per_stage BasicBlocks with stage_channels[k] channels; stages after the first start
- *    with stride 2 and a 1x1-convolution + BatchNorm shortcut.  BatchNorm uses batch statistics
+ *    blocks_per_stage (or stage_blocks[k]) BasicBlocks with stage_channels[k] channels, or bottleneck
+ *    blocks (block_kind); stages after the first start with stride 2 and a 1x1-convolution + BatchNorm
+ *    shortcut.  BatchNorm uses batch statistics
  *    (and keeps running statistics, which lp_evaluate can use).
  */
 typedef struct {
@@ -87,6 +89,14 @@ typedef struct {
      NHWC [batch, height, width, in_channels], no stem, and the first stage already starts with stride 2
      and a 1x1 shortcut; MLP -- no difference.  No gradient is formed for x (Sec. 3). */
   int input_is_activation;
+  /* RESNET: LP_BLOCK_BASIC (0, default): BasicBlocks, two 3x3 convolutions.  LP_BLOCK_BOTTLENECK: the blocks of the
+     deeper networks (Sec. 4.3 trains a ResNet-50): 1x1 convolution to stage_channels[k], 3x3 convolution (it
+     carries the stage's stride), 1x1 convolution to 4 * stage_channels[k], each followed by BatchNorm and the first
+     two by ReLU; identity shortcut, or 1x1 convolution + BatchNorm where the shape changes; ReLU after the sum.
+     A stage's output then has 4 * stage_channels[k] channels. */
+  int block_kind;
+  /* RESNET, nullable: [K] blocks per stage (a ResNet-50 has 3, 4, 6, 3); NULL: blocks_per_stage in every stage. */
+  const int* stage_blocks;
 } lp_model_spec;
 
 /* Auxiliary head of every chunk (Sec. 3: same form as the global objective): softmax
@@ -294,6 +304,20 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* probs, int backend, void* stre
 enum { LP_CONV_FORWARD = 0, LP_CONV_INPUT_GRAD = 1, LP_CONV_FILTER_GRAD = 2 };
 lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* out, int n, int h, int w,
                           int c_in, int c_out, void* stream);
+
+/*
+ * lp_conv2d_bf16: the same entry for all convolutions of App. B.3's residual networks that run as implicit GEMMs:
+ * ksize 3 (zero padding 1) or 1 (no padding), stride 1 or 2.  h x w is the INPUT image; the output image is
+ * ho x wo with ho = (h - 1) / stride + 1, wo = (w - 1) / stride + 1.  The operand tiles are TMA boxes that step
+ * through the input activation with the stride, one shifted box per filter tap.
+ *   LP_CONV_FORWARD:     act = x [n,h,w,c_in], other = filters [c_out,ksize,ksize,c_in] bf16, out = y [n,ho,wo,c_out] bf16
+ *                        y[n,p,q,o] = sum_{i,j,c} x[n, stride p + i - pad, stride q + j - pad, c] * filters[o,i,j,c]
+ *   LP_CONV_FILTER_GRAD: act = x, other = dy [n,ho,wo,c_out] bf16, out = dW [c_out,ksize,ksize,c_in] fp32
+ *   LP_CONV_INPUT_GRAD:  ksize 3, stride 1 only (otherwise LP_ERR_UNSUPPORTED): as lp_conv3x3_bf16.
+ * Accepted sizes: as for lp_conv3x3_bf16, with wo and ho*wo in place of w and h*w.  Errors: as lp_conv3x3_bf16.
+ */
+lp_status lp_conv2d_bf16(int form, const void* act, const void* other, void* out, int n, int h, int w,
+                         int c_in, int c_out, int ksize, int stride, void* stream);
 
 /*
  * lp_attention_bf16: kernel-level entry for tests and profiling: causal multi-head softmax attention with heads

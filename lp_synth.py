@@ -165,19 +165,33 @@ def param_table(cfg: dict) -> list[dict]:
                 add("c0.stem.conv", 0, (c_prev, cin, 3, 3), "normal", np.sqrt(2.0 / (cin * 9)), True)
                 add("c0.stem.bn.g", 0, (c_prev,), "ones")
                 add("c0.stem.bn.b", 0, (c_prev,), "zeros")
-            for j in range(cfg["blocks_per_stage"]):
+            bottleneck = cfg.get("block") == "bottleneck"
+            c_out = 4 * c if bottleneck else c           # a bottleneck block leaves four times its inner width
+            for j in range(resnet_stage_blocks(cfg, k)):
                 p = f"c{k}.r{j}"
-                c_in_blk = c_prev if j == 0 else c
-                add(p + ".conv1", k, (c, c_in_blk, 3, 3), "normal", np.sqrt(2.0 / (c_in_blk * 9)), True)
-                add(p + ".bn1.g", k, (c,), "ones")
-                add(p + ".bn1.b", k, (c,), "zeros")
-                add(p + ".conv2", k, (c, c, 3, 3), "normal", np.sqrt(2.0 / (c * 9)), True)
-                add(p + ".bn2.g", k, (c,), "ones")
-                add(p + ".bn2.b", k, (c,), "zeros")
-                if j == 0 and (resnet_stage_stride(cfg, k) != 1 or c_in_blk != c):
-                    add(p + ".sc.conv", k, (c, c_in_blk, 1, 1), "normal", np.sqrt(2.0 / c_in_blk), True)
-                    add(p + ".sc.bn.g", k, (c,), "ones")
-                    add(p + ".sc.bn.b", k, (c,), "zeros")
+                c_in_blk = c_prev if j == 0 else c_out
+                if bottleneck:
+                    add(p + ".conv1", k, (c, c_in_blk, 1, 1), "normal", np.sqrt(2.0 / c_in_blk), True)
+                    add(p + ".bn1.g", k, (c,), "ones")
+                    add(p + ".bn1.b", k, (c,), "zeros")
+                    add(p + ".conv2", k, (c, c, 3, 3), "normal", np.sqrt(2.0 / (c * 9)), True)
+                    add(p + ".bn2.g", k, (c,), "ones")
+                    add(p + ".bn2.b", k, (c,), "zeros")
+                    add(p + ".conv3", k, (c_out, c, 1, 1), "normal", np.sqrt(2.0 / c), True)
+                    add(p + ".bn3.g", k, (c_out,), "ones")
+                    add(p + ".bn3.b", k, (c_out,), "zeros")
+                else:
+                    add(p + ".conv1", k, (c, c_in_blk, 3, 3), "normal", np.sqrt(2.0 / (c_in_blk * 9)), True)
+                    add(p + ".bn1.g", k, (c,), "ones")
+                    add(p + ".bn1.b", k, (c,), "zeros")
+                    add(p + ".conv2", k, (c, c, 3, 3), "normal", np.sqrt(2.0 / (c * 9)), True)
+                    add(p + ".bn2.g", k, (c,), "ones")
+                    add(p + ".bn2.b", k, (c,), "zeros")
+                if j == 0 and (resnet_stage_stride(cfg, k) != 1 or c_in_blk != c_out):
+                    add(p + ".sc.conv", k, (c_out, c_in_blk, 1, 1), "normal", np.sqrt(2.0 / c_in_blk), True)
+                    add(p + ".sc.bn.g", k, (c_out,), "ones")
+                    add(p + ".sc.bn.b", k, (c_out,), "zeros")
+            c = c_out
             c_prev = c
             add(f"c{k}.head.W", k, (cfg["classes"], c), "normal", np.sqrt(1.0 / c), True)
             add(f"c{k}.head.b", k, (cfg["classes"],), "zeros")
@@ -191,6 +205,13 @@ def param_table(cfg: dict) -> list[dict]:
     else:
         raise ValueError(fam)
     return out
+
+
+def resnet_stage_blocks(cfg: dict, k: int) -> int:
+    """Residual blocks in stage k: cfg["blocks_per_stage"] is one count for all stages or a list per stage
+    (a ResNet-50 has 3, 4, 6, 3)."""
+    n = cfg["blocks_per_stage"]
+    return int(n[k]) if isinstance(n, (list, tuple)) else int(n)
 
 
 def resnet_stage_stride(cfg: dict, k: int) -> int:

@@ -195,7 +195,7 @@ class LocalUpdateOracle:
             g["c0.tok"], g["c0.pos"] = L.embedding_bwd(dh, cache["emb"])
         return g
 
-    # ResNet chunk: one stage of BasicBlocks (stem convolution in chunk 0), App. B.3.
+    # ResNet chunk: one stage of BasicBlocks or bottleneck blocks (stem convolution in chunk 0), App. B.3.
     def _resnet_fwd(self, k, x):
         p = self.p
         cache = {"blocks": []}
@@ -204,9 +204,13 @@ class LocalUpdateOracle:
             u, cb = self._bn(u, "c0.stem.bn")
             x, cr = L.relu_fwd(u)
             cache["stem"] = (cc, cb, cr)
-        for j in range(self.cfg["blocks_per_stage"]):
+        for j in range(lp_synth.resnet_stage_blocks(self.cfg, k)):
             n = f"c{k}.r{j}"
             s = lp_synth.resnet_stage_stride(self.cfg, k) if j == 0 else 1
+            if self.cfg.get("block") == "bottleneck":
+                x, bc = self._bottleneck_fwd(x, n, s)
+                cache["blocks"].append(bc)
+                continue
             u, cc1 = L.conv2d_fwd(x, p[n + ".conv1"], s, 1)
             u, cb1 = self._bn(u, n + ".bn1")
             u, cr1 = L.relu_fwd(u)
@@ -221,6 +225,48 @@ class LocalUpdateOracle:
             x, cr2 = L.relu_fwd(u + sc)
             cache["blocks"].append((n, cc1, cb1, cr1, cc2, cb2, csc, cr2))
         return x, cache
+
+    def _bottleneck_fwd(self, x, n, s):
+        """Bottleneck block of the deeper residual networks (Sec. 4.3 trains a ResNet-50; App. B.3): 1x1
+        convolution to the stage's inner width, 3x3 convolution (carrying the block's stride), 1x1 convolution
+        to four times that width, each followed by BatchNorm and the first two by ReLU; the shortcut is the
+        identity or, where the shape changes, a 1x1 convolution with the block's stride and BatchNorm; ReLU
+        after the sum."""
+        p = self.p
+        u, cc1 = L.conv2d_fwd(x, p[n + ".conv1"], 1, 0)
+        u, cb1 = self._bn(u, n + ".bn1")
+        u, cr1 = L.relu_fwd(u)
+        u, cc2 = L.conv2d_fwd(u, p[n + ".conv2"], s, 1)
+        u, cb2 = self._bn(u, n + ".bn2")
+        u, cr2 = L.relu_fwd(u)
+        u, cc3 = L.conv2d_fwd(u, p[n + ".conv3"], 1, 0)
+        u, cb3 = self._bn(u, n + ".bn3")
+        if n + ".sc.conv" in p:
+            sc, ccs = L.conv2d_fwd(x, p[n + ".sc.conv"], s, 0)
+            sc, cbs = self._bn(sc, n + ".sc.bn")
+            csc = (ccs, cbs)
+        else:
+            sc, csc = x, None
+        y, cr3 = L.relu_fwd(u + sc)
+        return y, ("bottleneck", n, cc1, cb1, cr1, cc2, cb2, cr2, cc3, cb3, csc, cr3)
+
+    def _bottleneck_bwd(self, dx, block_cache, g):
+        (_, n, cc1, cb1, cr1, cc2, cb2, cr2, cc3, cb3, csc, cr3) = block_cache
+        ds = L.relu_bwd(dx, cr3)
+        du, g[n + ".bn3.g"], g[n + ".bn3.b"] = L.batchnorm_bwd(ds, cb3)
+        du, g[n + ".conv3"] = L.conv2d_bwd(du, cc3)
+        du = L.relu_bwd(du, cr2)
+        du, g[n + ".bn2.g"], g[n + ".bn2.b"] = L.batchnorm_bwd(du, cb2)
+        du, g[n + ".conv2"] = L.conv2d_bwd(du, cc2)
+        du = L.relu_bwd(du, cr1)
+        du, g[n + ".bn1.g"], g[n + ".bn1.b"] = L.batchnorm_bwd(du, cb1)
+        dx, g[n + ".conv1"] = L.conv2d_bwd(du, cc1)
+        if csc is not None:
+            ccs, cbs = csc
+            dsc, g[n + ".sc.bn.g"], g[n + ".sc.bn.b"] = L.batchnorm_bwd(ds, cbs)
+            dsc, g[n + ".sc.conv"] = L.conv2d_bwd(dsc, ccs)
+            return dx + dsc
+        return dx + ds
 
     def _bn(self, x, name):
         """BatchNorm `name` on x.  Training and plain forward passes use the batch statistics (App. B.3's
@@ -237,8 +283,10 @@ class LocalUpdateOracle:
         return y, cache
 
     def _resnet_block_bwd(self, dx, block_cache, g):
-        """Backward of one BasicBlock: fills g with its parameter gradients, returns the gradient at the block
-        input (main branch plus shortcut)."""
+        """Backward of one BasicBlock (or bottleneck block): fills g with its parameter gradients, returns the
+        gradient at the block input (main branch plus shortcut)."""
+        if block_cache[0] == "bottleneck":
+            return self._bottleneck_bwd(dx, block_cache, g)
         (n, cc1, cb1, cr1, cc2, cb2, csc, cr2) = block_cache
         ds = L.relu_bwd(dx, cr2)
         du, g[n + ".bn2.g"], g[n + ".bn2.b"] = L.batchnorm_bwd(ds, cb2)

@@ -19,6 +19,7 @@ LP_ERR = {-1: "INVALID_ARG", -2: "SHAPE", -3: "UNSUPPORTED", -4: "ALLOC", -5: "C
           -7: "LABEL_RANGE", -8: "NONFINITE", -9: "TIMEOUT"}
 LP_FAMILY_MLP, LP_FAMILY_LM, LP_FAMILY_RESNET = 0, 1, 2
 LP_FP32, LP_BF16 = 0, 1
+LP_BLOCK_BASIC, LP_BLOCK_BOTTLENECK = 0, 1
 LP_HEAD_LINEAR, LP_HEAD_LN_LINEAR, LP_HEAD_GAP_LINEAR, LP_HEAD_BN_RELU_GAP_LINEAR = 0, 1, 2, 3
 LP_OPT_SGDM, LP_OPT_ADAM = 0, 1
 LP_SYNC, LP_PIPELINED = 0, 1
@@ -39,7 +40,8 @@ class lp_model_spec(C.Structure):
                 ("d_ffn", C.c_int), ("blocks_per_chunk", C.POINTER(C.c_int)),
                 ("in_channels", C.c_int), ("height", C.c_int), ("width", C.c_int),
                 ("stem_channels", C.c_int), ("stage_channels", C.POINTER(C.c_int)),
-                ("blocks_per_stage", C.c_int), ("gemm_backend", C.c_int), ("input_is_activation", C.c_int)]
+                ("blocks_per_stage", C.c_int), ("gemm_backend", C.c_int), ("input_is_activation", C.c_int),
+                ("block_kind", C.c_int), ("stage_blocks", C.POINTER(C.c_int))]
 
 
 class lp_head_spec(C.Structure):
@@ -60,7 +62,7 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
-           "lp_attention_bf16", "lp_gemm_bf16_static", "lp_gemm_static_poll", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap",
+           "lp_attention_bf16", "lp_gemm_bf16_static", "lp_gemm_static_poll", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_conv2d_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap",
            "lp_cost_model", "lp_mlp_layer_flops", "lp_mlp_aux_flops", "lp_chunk_output_bytes", "lp_chunk_output"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
@@ -154,10 +156,17 @@ def specs_from_config(cfg: dict, gemm_backend: int = 0):
     else:
         m.family = LP_FAMILY_RESNET
         m.in_channels, m.height, m.width = cfg["in_channels"], cfg["height"], cfg["width"]
-        m.stem_channels, m.blocks_per_stage = cfg["stem_channels"], cfg["blocks_per_stage"]
+        m.stem_channels = cfg["stem_channels"]
         a = _ints(cfg["stage_channels"])
         keep.append(a)
         m.stage_channels = a
+        m.block_kind = LP_BLOCK_BOTTLENECK if cfg.get("block") == "bottleneck" else LP_BLOCK_BASIC
+        if isinstance(cfg["blocks_per_stage"], (list, tuple)):
+            sb = _ints(cfg["blocks_per_stage"])
+            keep.append(sb)
+            m.stage_blocks, m.blocks_per_stage = sb, max(cfg["blocks_per_stage"])
+        else:
+            m.blocks_per_stage = cfg["blocks_per_stage"]
         K = len(cfg["stage_channels"])
         hd.kind = LP_HEAD_BN_RELU_GAP_LINEAR if cfg.get("head") == "bn_relu_gap" else LP_HEAD_GAP_LINEAR
         hd.classes = cfg["classes"]
@@ -340,6 +349,16 @@ def lp_attention_bf16(form: int, qkv, o, lse, dout, dqkv, delta, batch: int, seq
     lse; backward reads them and dout and writes dqkv and delta.  Tensors may be torch tensors or raw pointers."""
     _check(None, _lib.lp_attention_bf16(form, _ptr(qkv), _ptr(o), _ptr(lse), _ptr(dout), _ptr(dqkv), _ptr(delta),
                                         batch, seq_len, n_heads, stream))
+
+
+_lib.lp_conv2d_bf16.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p] + [C.c_int] * 7 + [C.c_void_p]
+
+
+def lp_conv2d_bf16(form: int, act, other, out, n: int, h: int, w: int, c_in: int, c_out: int, ksize: int, stride: int,
+                   stream=None) -> None:
+    """One implicit-GEMM convolution over bf16 NHWC tensors: 3x3 (padding 1) or 1x1, stride 1 or 2; forward, filter
+    gradient, or (3x3 stride 1) input gradient (see lp.h)."""
+    _check(None, _lib.lp_conv2d_bf16(form, _ptr(act), _ptr(other), _ptr(out), n, h, w, c_in, c_out, ksize, stride, stream))
 
 
 _lib.lp_gemm_bf16_static.argtypes = [C.c_int, C.POINTER(lp_gemm_desc), C.c_void_p]

@@ -501,6 +501,10 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
         // ---- implicit convolution: one operand is fetched as shifted boxes of the activation tensor
         const GemmProb& p = probs[cur.pi];
         const int cv_c = p.conv_c, cv_w = p.conv_w, cv_hw = p.conv_h * p.conv_w, cv_n = p.conv_n, cv_k0 = p.conv_k0, p_n = p.N;
+        const int cv_s = p.conv_stride > 1 ? p.conv_stride : 1, cv_taps = p.conv_taps ? p.conv_taps : 9;
+        // tap t of the filter -> offset of the input pixel (3x3 with padding 1, or the single tap of a 1x1 filter)
+        auto tap_di = [&](int t) { return cv_taps == 1 ? 0 : t / 3 - 1; };
+        auto tap_dj = [&](int t) { return cv_taps == 1 ? 0 : t - (t / 3) * 3 - 1; };
         // this CTA's 128 output pixels start at row a_h0 of image a_img (whole rows)
         int a_img = 0, a_h0 = 0;
         if (conv != CONV_WGRAD) { a_img = m0 / cv_hw; a_h0 = (m0 - a_img * cv_hw) / cv_w; }
@@ -530,15 +534,15 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
             for (int i = 0; i < BNL / 64; ++i) {
               const int col = n0 + i * 64;
               const int t = col / cv_c, c0 = col - t * cv_c;
-              if (t < 9) ld4(b_dst + i * (BK * 128), mapB, c0, t - (t / 3) * 3 - 1, h0 + t / 3 - 1, img);
+              if (t < cv_taps) ld4(b_dst + i * (BK * 128), mapB, c0, tap_dj(t), h0 * cv_s + tap_di(t), img);
               else ld4(b_dst + i * (BK * 128), mapB, 0, 0, 0, cv_n);        // beyond the last tap: an all-zero box
             }
           } else {
             // k-slice -> (filter tap, channel block); A: 128 pixels shifted by the tap (mirrored for the input gradient)
             const int cb = cv_c >> 6, tap = kb / cb, ch0 = (kb - tap * cb) << 6;
-            int di = tap / 3 - 1, dj = tap - (tap / 3) * 3 - 1;
+            int di = tap_di(tap), dj = tap_dj(tap);
             if (conv == CONV_DGRAD) { di = -di; dj = -dj; }
-            ld4(a_dst, mapA, ch0, dj, a_h0 + di, a_img);
+            ld4(a_dst, mapA, ch0, dj, a_h0 * cv_s + di, a_img);
             if (conv == CONV_FWD) {
               ld2(b_dst, mapB, k0, n0);                  // filters [N, 9 conv_c], reduction index contiguous
             } else {
@@ -717,17 +721,20 @@ bool encode_map(CUtensorMap* out, const void* base, long long inner, long long o
 // 64 channels x whole image rows that hold `pixels` pixels (128: a K-major A tile; 64: one k-slice of an
 // MN-major B tile), i.e. (w, pixels / w, 1) inside an image or (w, h, pixels / (h w)) across small images.
 // 128-byte swizzle; everything outside the tensor (the padding ring of the convolution) reads as zero.
-bool encode_map4(CUtensorMap* out, const void* base, int n, int h, int w, int c, int pixels) {
+// The boxes are counted in pixels of the OUTPUT image h x w; with a stride s the tensor is the input image
+// hin x win and a box steps through it s pixels at a time (traversed extent s times the pixels it delivers).
+bool encode_map4(CUtensorMap* out, const void* base, int n, int h, int w, int c, int pixels, int hin, int win, int s) {
   EncodeFn fn = get_encode();
   if (!fn) return false;
   const long long hw = (long long)h * w;
   cuuint32_t bw = (cuuint32_t)w, bh, bn;
   if (hw >= pixels) { bh = (cuuint32_t)(pixels / w); bn = 1; }
   else { bh = (cuuint32_t)h; bn = (cuuint32_t)(pixels / hw); }
-  cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
-  cuuint64_t strides[3] = {(cuuint64_t)c * 2, (cuuint64_t)w * c * 2, (cuuint64_t)hw * c * 2};
-  cuuint32_t box[4] = {64u, bw, bh, bn};
-  cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+  if (bw * s > 256 || bh * s > 256) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)c, (cuuint64_t)win, (cuuint64_t)hin, (cuuint64_t)n};
+  cuuint64_t strides[3] = {(cuuint64_t)c * 2, (cuuint64_t)win * c * 2, (cuuint64_t)hin * win * c * 2};
+  cuuint32_t box[4] = {64u, bw * (cuuint32_t)s, bh * (cuuint32_t)s, bn};
+  cuuint32_t estr[4] = {1u, (cuuint32_t)s, (cuuint32_t)s, 1u};
   CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -745,14 +752,20 @@ bool gemm_tc_eligible(const GemmProb& g) {
       return false;
   }
   if (g.conv != CONV_NONE) {
-    // implicit 3x3 convolution: whole-row boxes, 64-channel k-slices, filters with 16-byte pitches
+    // implicit convolution: whole-row boxes, 64-channel k-slices, filters with 16-byte pitches
     if (g.conv_c < 64 || g.conv_c % 64 || g.conv_n < 1 || !conv_boxes_ok(g.conv_h, g.conv_w)) return false;
     if (((uintptr_t)g.A & 15) || ((uintptr_t)g.B & 15)) return false;
+    const int s = g.conv_stride > 1 ? g.conv_stride : 1, taps = g.conv_taps ? g.conv_taps : 9;
+    const int hin = g.conv_hin ? g.conv_hin : g.conv_h, win = g.conv_win ? g.conv_win : g.conv_w;
+    if (s > 2 || (taps != 9 && taps != 1) || g.conv_w * s > 256) return false;
+    // the output image is what a convolution with this stride makes of the input image
+    // (3x3 with padding 1 and 1x1 without padding give the same size)
+    if (g.conv_h != (hin - 1) / s + 1 || g.conv_w != (win - 1) / s + 1) return false;
     const long long pixels = (long long)g.conv_n * g.conv_h * g.conv_w;
-    if (g.conv == CONV_FWD) return g.K == 9 * g.conv_c && g.M == pixels && g.b_ks == 1 && g.b_ns % 8 == 0 && get_encode() != nullptr;
-    if (g.conv == CONV_DGRAD) return g.K == 9 * g.conv_c && g.M == pixels && g.N % 8 == 0 && get_encode() != nullptr;
+    if (g.conv == CONV_FWD) return g.K == taps * g.conv_c && g.M == pixels && g.b_ks == 1 && g.b_ns % 8 == 0 && get_encode() != nullptr;
+    if (g.conv == CONV_DGRAD) return s == 1 && taps == 9 && g.K == 9 * g.conv_c && g.M == pixels && g.N % 8 == 0 && get_encode() != nullptr;
     if (g.conv == CONV_WGRAD)
-      return g.N == 9 * g.conv_c && g.a_ms == 1 && g.a_ks % 8 == 0 && g.conv_k0 % 64 == 0 && g.conv_k0 + g.K <= pixels &&
+      return g.N == taps * g.conv_c && g.a_ms == 1 && g.a_ks % 8 == 0 && g.conv_k0 % 64 == 0 && g.conv_k0 + g.K <= pixels &&
              get_encode() != nullptr;
     return false;
   }
@@ -820,10 +833,12 @@ bool gemm_tc_encode(GemmProb& g, void* maps, int cg) {
     g.store_tma = ok ? (wide ? 2 : 1) : 0;
   }
   bool okA, okB;
-  if (g.conv == CONV_FWD || g.conv == CONV_DGRAD) okA = encode_map4(mapA, g.A, g.conv_n, g.conv_h, g.conv_w, g.conv_c, BM);
+  const int cs = g.conv_stride > 1 ? g.conv_stride : 1;
+  const int chin = g.conv_hin ? g.conv_hin : g.conv_h, cwin = g.conv_win ? g.conv_win : g.conv_w;
+  if (g.conv == CONV_FWD || g.conv == CONV_DGRAD) okA = encode_map4(mapA, g.A, g.conv_n, g.conv_h, g.conv_w, g.conv_c, BM, chin, cwin, cs);
   else if (g.a_ms == 1) okA = encode_map(mapA, g.A, g.M, g.K, g.a_ks, BK);       // MN-major: rows are k
   else okA = encode_map(mapA, g.A, g.K, g.M, g.a_ms, BM);
-  if (g.conv == CONV_WGRAD) okB = encode_map4(mapB, g.B, g.conv_n, g.conv_h, g.conv_w, g.conv_c, BK);
+  if (g.conv == CONV_WGRAD) okB = encode_map4(mapB, g.B, g.conv_n, g.conv_h, g.conv_w, g.conv_c, BK, chin, cwin, cs);
   else if (g.conv == CONV_DGRAD) okB = encode_map(mapB, g.B, 9LL * g.N, g.conv_c, 9LL * g.N, BK);   // rows: output channel
   else if (g.b_ns == 1) okB = encode_map(mapB, g.B, g.N, g.K, g.b_ks, BK);
   else okB = encode_map(mapB, g.B, g.K, g.N, g.b_ns, BN / cg);

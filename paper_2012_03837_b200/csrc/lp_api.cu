@@ -73,6 +73,11 @@ void validate(const lp_model_spec* m, int K, const lp_head_spec* hd, const lp_op
       if (m->in_channels < 1 || m->height < 1 || m->width < 1 || m->stem_channels < 1 || m->blocks_per_stage < 1)
         throw ShapeError("RESNET sizes must be positive");
       if ((m->height >> (K - 1)) < 1 || (m->width >> (K - 1)) < 1) throw ShapeError("image too small for K stages");
+      if (m->block_kind != LP_BLOCK_BASIC && m->block_kind != LP_BLOCK_BOTTLENECK) throw std::invalid_argument("block_kind");
+      for (int k = 0; k < K; ++k) {
+        if (m->stage_channels[k] < 1) throw ShapeError("stage_channels must be positive");
+        if (m->stage_blocks && m->stage_blocks[k] < 1) throw ShapeError("every stage needs at least one block");
+      }
       break;
     }
     default: throw std::invalid_argument("family");
@@ -254,6 +259,8 @@ lp_status lp_create(const lp_model_spec* model, int K, const lp_head_spec* head,
       default:
         h.stage_channels.assign(model->stage_channels, model->stage_channels + K);
         h.spec.stage_channels = nullptr;
+        for (int k = 0; k < K; ++k) h.stage_blocks.push_back(model->stage_blocks ? model->stage_blocks[k] : model->blocks_per_stage);
+        h.spec.stage_blocks = nullptr;
         build_resnet(h);
         break;
     }
@@ -596,33 +603,43 @@ lp_status lp_gemm_bf16(int n, const lp_gemm_desc* in, int backend, void* stream,
 
 lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* out, int n, int hgt, int wid, int c_in,
                           int c_out, void* stream) {
-  if (!act || !other || !out) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_conv3x3_bf16: null pointer");
-  if (n < 1 || hgt < 1 || wid < 1 || c_in < 1 || c_out < 1) return fail(nullptr, LP_ERR_SHAPE, "lp_conv3x3_bf16: sizes must be positive");
-  const long long pixels = (long long)n * hgt * wid;
-  if (pixels > 0x7fffffffLL) return fail(nullptr, LP_ERR_SHAPE, "lp_conv3x3_bf16: too many pixels");
+  return lp_conv2d_bf16(form, act, other, out, n, hgt, wid, c_in, c_out, 3, 1, stream);
+}
+
+lp_status lp_conv2d_bf16(int form, const void* act, const void* other, void* out, int n, int hgt, int wid, int c_in,
+                         int c_out, int ksize, int stride, void* stream) {
+  if (!act || !other || !out) return fail(nullptr, LP_ERR_INVALID_ARG, "lp_conv2d_bf16: null pointer");
+  if (n < 1 || hgt < 1 || wid < 1 || c_in < 1 || c_out < 1) return fail(nullptr, LP_ERR_SHAPE, "lp_conv2d_bf16: sizes must be positive");
+  if ((ksize != 3 && ksize != 1) || (stride != 1 && stride != 2))
+    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_conv2d_bf16: 3x3 (padding 1) or 1x1 filters, stride 1 or 2");
+  const int ho = (hgt - 1) / stride + 1, wo = (wid - 1) / stride + 1, taps = ksize * ksize;
+  const long long pixels = (long long)n * ho * wo;
+  if ((long long)n * hgt * wid > 0x7fffffffLL) return fail(nullptr, LP_ERR_SHAPE, "lp_conv2d_bf16: too many pixels");
   GemmProb g{};
-  g.conv_n = n; g.conv_h = hgt; g.conv_w = wid;
+  g.conv_n = n; g.conv_h = ho; g.conv_w = wo; g.conv_hin = hgt; g.conv_win = wid; g.conv_stride = stride; g.conv_taps = taps;
   switch (form) {
-    case LP_CONV_FORWARD:        // act = x [n,h,w,c_in], other = filters [c_out,3,3,c_in], out = y [n,h,w,c_out]
-      g.A = act; g.B = other; g.C = out; g.M = (int)pixels; g.N = c_out; g.K = 9 * c_in;
-      g.a_ms = c_in; g.a_ks = 1; g.b_ns = 9LL * c_in; g.b_ks = 1; g.ldc = c_out;
+    case LP_CONV_FORWARD:        // act = x [n,h,w,c_in], other = filters [c_out,k,k,c_in], out = y [n,ho,wo,c_out]
+      g.A = act; g.B = other; g.C = out; g.M = (int)pixels; g.N = c_out; g.K = taps * c_in;
+      g.a_ms = c_in; g.a_ks = 1; g.b_ns = (long long)taps * c_in; g.b_ks = 1; g.ldc = c_out;
       g.conv = CONV_FWD; g.conv_c = c_in;
       break;
     case LP_CONV_INPUT_GRAD:     // act = dy [n,h,w,c_out], other = filters, out = dx [n,h,w,c_in]
+      if (ksize != 3 || stride != 1) return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_conv2d_bf16: the input gradient exists for 3x3, stride 1");
       g.A = act; g.B = other; g.C = out; g.M = (int)pixels; g.N = c_in; g.K = 9 * c_out;
       g.a_ms = c_out; g.a_ks = 1; g.b_ns = 1; g.b_ks = 9LL * c_in; g.ldc = c_in;
       g.conv = CONV_DGRAD; g.conv_c = c_out;
       break;
-    case LP_CONV_FILTER_GRAD:    // act = x [n,h,w,c_in], other = dy [n,h,w,c_out], out = dW [c_out,3,3,c_in] fp32
-      g.A = other; g.B = act; g.C = out; g.M = c_out; g.N = 9 * c_in; g.K = (int)pixels;
-      g.a_ms = 1; g.a_ks = c_out; g.b_ns = 1; g.b_ks = c_in; g.ldc = 9 * c_in; g.out_f32 = 1;
+    case LP_CONV_FILTER_GRAD:    // act = x [n,h,w,c_in], other = dy [n,ho,wo,c_out], out = dW [c_out,k,k,c_in] fp32
+      g.A = other; g.B = act; g.C = out; g.M = c_out; g.N = taps * c_in; g.K = (int)pixels;
+      g.a_ms = 1; g.a_ks = c_out; g.b_ns = 1; g.b_ks = c_in; g.ldc = taps * c_in; g.out_f32 = 1;
       g.conv = CONV_WGRAD; g.conv_c = c_in;
       break;
-    default: return fail(nullptr, LP_ERR_INVALID_ARG, "lp_conv3x3_bf16: unknown form");
+    default: return fail(nullptr, LP_ERR_INVALID_ARG, "lp_conv2d_bf16: unknown form");
   }
   if (!gemm_tc_eligible(g))
-    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_conv3x3_bf16: needs 16-byte aligned tensors, the shifted operand's channels a multiple of 64, "
-                                             "the other channel count a multiple of 8, a width dividing 64 and h*w dividing or divisible by 128");
+    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_conv2d_bf16: needs 16-byte aligned tensors, the shifted operand's channels a multiple of 64, "
+                                             "the other channel count a multiple of 8, an output width dividing 64 and output h*w dividing or "
+                                             "divisible by 128");
   cudaStream_t s = (cudaStream_t)stream;
   static int* d_status = nullptr;
   static void* d_tab = nullptr;
@@ -630,9 +647,9 @@ lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* ou
   struct alignas(64) Map { unsigned char b[128]; };
   static int first_dev = -1;
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, LP_ERR_CUDA, "lp_conv3x3_bf16: no CUDA device"); }
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, LP_ERR_CUDA, "lp_conv2d_bf16: no CUDA device"); }
   if (first_dev >= 0 && dev != first_dev)
-    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_conv3x3_bf16: one device per process (the first one it was called on)");
+    return fail(nullptr, LP_ERR_UNSUPPORTED, "lp_conv2d_bf16: one device per process (the first one it was called on)");
   if (!d_tab) {
     if (cudaMalloc(&d_tab, 1024 + 4 * sizeof(Map)) != cudaSuccess) { cudaGetLastError(); d_tab = nullptr; return fail(nullptr, LP_ERR_ALLOC, "descriptor table"); }
     d_status = (int*)d_tab;
@@ -650,7 +667,7 @@ lp_status lp_conv3x3_bf16(int form, const void* act, const void* other, void* ou
   cudaMemcpyAsync(dm, maps, sizeof(maps), cudaMemcpyHostToDevice, s);
   cudaStreamSynchronize(s);                      // the tables above are host stack memory
   launch_gemm_tc(dp, dm, 1, total, d_status, num_sms, s, cg);
-  return check_cuda(nullptr, "lp_conv3x3_bf16");
+  return check_cuda(nullptr, "lp_conv2d_bf16");
 }
 
 lp_status lp_attention_bf16(int form, const void* qkv, void* o, float* lse, const void* dout, void* dqkv, float* delta,

@@ -42,10 +42,14 @@ struct GemmProb {
   int tiles_n;
   int store_tma;   // tensor-core kernel: outputs leave through TMA stores (set by the launcher when C's pitch allows)
   int raster;      // tensor-core kernel: row tiles per band of the tile walk (set by the launcher)
-  // Implicit 3x3 convolution, stride 1, padding 1, over NHWC activations (tensor-core kernel only; App. B.3's
-  // residual blocks).  One operand is never materialised as a matrix: its tiles are fetched as shifted boxes
-  // of the activation tensor [conv_n, conv_h, conv_w, conv_c], one shift per filter tap (i, j), rows and
-  // columns outside the image reading as zero.
+  // Implicit convolution over NHWC activations (tensor-core kernel only; App. B.3's residual blocks): 3x3 with
+  // padding 1 (conv_taps = 9) or 1x1 without padding (conv_taps = 1), stride conv_stride = 1 or 2.  One operand
+  // is never materialised as a matrix: its tiles are fetched as boxes of the activation tensor
+  // [conv_n, conv_hin, conv_win, conv_c] that step through it with the stride, one shifted box per filter tap
+  // (i, j), rows and columns outside the image reading as zero.  conv_h x conv_w is the OUTPUT image (the rows of
+  // the GEMM are its pixels); for stride 1 it equals the input image.  The formulas below are written for the
+  // 3x3, stride-1 case; with a stride s the input pixel of output pixel (p, q) and tap (i, j) is
+  // (s p + i - 1, s q + j - 1), for 1x1 it is (s p, s q).  CONV_DGRAD exists for stride 1 only.
   //   CONV_FWD   : A(m, k) = x[pixel m shifted by (i-1, j-1)][c],  k = (3i + j) conv_c + c;  K = 9 conv_c;
   //                B = filters [N, 9 conv_c] (reduction index contiguous).
   //   CONV_DGRAD : A(m, k) = dy[pixel m shifted by (1-i, 1-j)][co], k = (3i + j) conv_c + co; K = 9 conv_c;
@@ -63,6 +67,7 @@ struct GemmProb {
   int conv;
   int conv_n, conv_h, conv_w, conv_c;
   int conv_k0;     // CONV_WGRAD: first pixel of this slice of the reduction (split-K)
+  int conv_hin, conv_win, conv_stride, conv_taps;   // 0 = defaults: input image = output image, stride 1, 9 taps
 };
 enum { CONV_NONE = 0, CONV_FWD = 1, CONV_DGRAD = 2, CONV_WGRAD = 3 };
 // True if an image of h x w pixels can be walked in whole-row boxes of 128 and of 64 pixels.

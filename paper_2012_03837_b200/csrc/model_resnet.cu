@@ -27,6 +27,8 @@ struct Conv {
   bool imp_fwd = false, imp_dgrad = false;
   // few-channel direct convolution on the FP32 ALUs (the stem): forward and filter gradient, no im2col
   bool small = false;
+  // 1x1, stride 1: the NHWC activation [pixels, Cin] is the GEMM operand as it stands, in every backend
+  bool pointwise = false;
 };
 struct Bn {
   std::string g, b;
@@ -35,10 +37,12 @@ struct Bn {
   float *mean, *rstd;
 };
 struct Block {
-  Conv c1, c2, cs;
-  Bn b1, b2, bs;
-  bool has_sc = false;
-  void *a1 = nullptr, *sc = nullptr, *out = nullptr;   // out is null for the chunk's last block (boundary buffer)
+  Conv c1, c2, c3, cs;                                   // c3: third convolution of a bottleneck block
+  Bn b1, b2, b3, bs;
+  bool has_sc = false, bottleneck = false;
+  void *a1 = nullptr, *a2 = nullptr, *sc = nullptr, *out = nullptr;   // out is null for the chunk's last block (boundary buffer)
+  const Conv& last() const { return bottleneck ? c3 : c2; }
+  const Bn& last_bn() const { return bottleneck ? b3 : b2; }
 };
 struct Chunk {
   bool has_stem = false;
@@ -82,6 +86,7 @@ Conv make_conv(const std::string& w, int N, int H, int W, int Cin, int Cout, int
   c.M = (long long)N * c.Ho * c.Wo;
   c.K = k * k * Cin;
   c.ldk = (c.K + 7) / 8 * 8;
+  c.pointwise = k == 1 && stride == 1;
   return c;
 }
 
@@ -108,22 +113,38 @@ void build_resnet(Handle& h) {
       h.add_tensor("c0.stem.bn.b", 0, {cprev}, false);
       c.stem_bn = Bn{"c0.stem.bn.g", "c0.stem.bn.b", cprev, c.stem.M, nullptr, nullptr};
     }
-    int cout = h.stage_channels[k];
-    for (int j = 0; j < h.spec.blocks_per_stage; ++j) {
+    const bool bottleneck = h.spec.block_kind == LP_BLOCK_BOTTLENECK;
+    const int cmid = h.stage_channels[k];
+    int cout = bottleneck ? 4 * cmid : cmid;                 // a bottleneck block leaves four times its inner width
+    for (int j = 0; j < h.stage_blocks[k]; ++j) {
       Block b;
+      b.bottleneck = bottleneck;
       const std::string p = ck + ".r" + std::to_string(j);
       int stride = (j == 0 && (k > 0 || inner)) ? 2 : 1;
       int cin = j == 0 ? cprev : cout;
-      b.c1 = make_conv(p + ".conv1", B, H, W, cin, cout, 3, stride);
-      h.add_tensor(p + ".conv1", k, {cout, 3, 3, cin}, true);
-      h.add_tensor(p + ".bn1.g", k, {cout}, false);
-      h.add_tensor(p + ".bn1.b", k, {cout}, false);
-      b.b1 = Bn{p + ".bn1.g", p + ".bn1.b", cout, b.c1.M, nullptr, nullptr};
-      b.c2 = make_conv(p + ".conv2", B, b.c1.Ho, b.c1.Wo, cout, cout, 3, 1);
-      h.add_tensor(p + ".conv2", k, {cout, 3, 3, cout}, true);
-      h.add_tensor(p + ".bn2.g", k, {cout}, false);
-      h.add_tensor(p + ".bn2.b", k, {cout}, false);
-      b.b2 = Bn{p + ".bn2.g", p + ".bn2.b", cout, b.c2.M, nullptr, nullptr};
+      auto add_bn = [&](const std::string& n, int C, long long rows) {
+        h.add_tensor(n + ".g", k, {C}, false);
+        h.add_tensor(n + ".b", k, {C}, false);
+        return Bn{n + ".g", n + ".b", C, rows, nullptr, nullptr};
+      };
+      if (bottleneck) {
+        b.c1 = make_conv(p + ".conv1", B, H, W, cin, cmid, 1, 1);
+        h.add_tensor(p + ".conv1", k, {cmid, 1, 1, cin}, true);
+        b.b1 = add_bn(p + ".bn1", cmid, b.c1.M);
+        b.c2 = make_conv(p + ".conv2", B, H, W, cmid, cmid, 3, stride);
+        h.add_tensor(p + ".conv2", k, {cmid, 3, 3, cmid}, true);
+        b.b2 = add_bn(p + ".bn2", cmid, b.c2.M);
+        b.c3 = make_conv(p + ".conv3", B, b.c2.Ho, b.c2.Wo, cmid, cout, 1, 1);
+        h.add_tensor(p + ".conv3", k, {cout, 1, 1, cmid}, true);
+        b.b3 = add_bn(p + ".bn3", cout, b.c3.M);
+      } else {
+        b.c1 = make_conv(p + ".conv1", B, H, W, cin, cout, 3, stride);
+        h.add_tensor(p + ".conv1", k, {cout, 3, 3, cin}, true);
+        b.b1 = add_bn(p + ".bn1", cout, b.c1.M);
+        b.c2 = make_conv(p + ".conv2", B, b.c1.Ho, b.c1.Wo, cout, cout, 3, 1);
+        h.add_tensor(p + ".conv2", k, {cout, 3, 3, cout}, true);
+        b.b2 = add_bn(p + ".bn2", cout, b.c2.M);
+      }
       b.has_sc = j == 0 && (stride != 1 || cin != cout);
       if (b.has_sc) {
         b.cs = make_conv(p + ".sc.conv", B, H, W, cin, cout, 1, stride);
@@ -132,7 +153,7 @@ void build_resnet(Handle& h) {
         h.add_tensor(p + ".sc.bn.b", k, {cout}, false);
         b.bs = Bn{p + ".sc.bn.g", p + ".sc.bn.b", cout, b.cs.M, nullptr, nullptr};
       }
-      H = b.c1.Ho; W = b.c1.Wo;
+      H = b.last().Ho; W = b.last().Wo;
       c.blocks.push_back(b);
     }
     cprev = cout;
@@ -168,16 +189,21 @@ void build_resnet(Handle& h) {
   h.y_bytes = (size_t)B * sizeof(int);
   h.y_in = (int*)h.dalloc(h.y_bytes);
   auto fal = [&](size_t n) { return (float*)h.dalloc(n * sizeof(float)); };
-  // 3x3 stride-1 convolutions whose channel counts are multiples of 64 run as implicit GEMMs: the activation
-  // tensor itself is the operand (shifted TMA boxes per filter tap), nothing 9 times its size is written.
+  // 3x3 (padding 1) and 1x1 convolutions with stride 1 or 2 whose input channel count is a multiple of 64 run
+  // as implicit GEMMs: the activation tensor itself is the operand (TMA boxes that step through it with the
+  // stride, one shifted box per filter tap), nothing 9 times its size is written.  Forward and filter gradient
+  // for both strides; the input gradient in this form for the 3x3 stride-1 convolutions (the stride-2
+  // convolutions open a stage, so their input gradient is only needed by the overlapping variant).
   auto set_implicit = [&](Conv& c) {
-    const bool base = bf && !h.force_simt && c.k == 3 && c.stride == 1 && conv_boxes_ok(c.H, c.W);
+    const bool shape = (c.k == 3 && c.pad == 1) || (c.k == 1 && c.pad == 0);
+    const bool base = bf && !h.force_simt && shape && (c.stride == 1 || c.stride == 2) && conv_boxes_ok(c.Ho, c.Wo) &&
+                      c.Wo * c.stride <= 256;
     c.imp_fwd = base && c.Cin % 64 == 0 && c.Cout % 8 == 0;
-    c.imp_dgrad = base && c.Cout % 64 == 0 && c.Cin % 8 == 0;
+    c.imp_dgrad = base && c.k == 3 && c.stride == 1 && c.Cout % 64 == 0 && c.Cin % 8 == 0;
   };
   auto alloc_conv = [&](Conv& c) {
     set_implicit(c);
-    if (!c.imp_fwd && !c.small) c.cols = h.dalloc((size_t)c.M * c.ldk * es);
+    if (!c.imp_fwd && !c.small && !c.pointwise) c.cols = h.dalloc((size_t)c.M * c.ldk * es);
     c.y = h.dalloc((size_t)c.M * c.Cout * es);
   };
   auto alloc_bn = [&](Bn& b) { b.mean = fal(b.C); b.rstd = fal(b.C); };
@@ -194,7 +220,7 @@ void build_resnet(Handle& h) {
     auto track = [&](const Conv& cv) {
       max_act = std::max(max_act, (size_t)cv.M * cv.Cout);
       max_act = std::max(max_act, (size_t)cv.N * cv.H * cv.W * cv.Cin);
-      if (!cv.imp_dgrad) max_cols = std::max(max_cols, (size_t)cv.M * cv.ldk);
+      if (!cv.imp_dgrad && !cv.pointwise) max_cols = std::max(max_cols, (size_t)cv.M * cv.ldk);
     };
     if (c.has_stem) {
       c.x_nhwc = h.dalloc(in_elems * es);
@@ -208,8 +234,12 @@ void build_resnet(Handle& h) {
       alloc_conv(b.c1); alloc_bn(b.b1); track(b.c1);
       alloc_conv(b.c2); alloc_bn(b.b2); track(b.c2);
       b.a1 = h.dalloc((size_t)b.c1.M * b.c1.Cout * es);
+      if (b.bottleneck) {
+        alloc_conv(b.c3); alloc_bn(b.b3); track(b.c3);
+        b.a2 = h.dalloc((size_t)b.c2.M * b.c2.Cout * es);
+      }
       if (b.has_sc) { alloc_conv(b.cs); alloc_bn(b.bs); track(b.cs); b.sc = h.dalloc((size_t)b.cs.M * b.cs.Cout * es); }
-      if (j + 1 < c.blocks.size()) b.out = h.dalloc((size_t)b.c2.M * b.c2.Cout * es);
+      if (j + 1 < c.blocks.size()) b.out = h.dalloc((size_t)b.last().M * b.last().Cout * es);
     }
     if (head_bn) { alloc_bn(c.head_bn); c.hact = h.dalloc(out_bytes); }
     c.pool = h.dalloc((size_t)B * c.C * es);
@@ -222,12 +252,17 @@ void build_resnet(Handle& h) {
 
   // ---- op emitters (one problem per launch: the stages differ in every size)
   auto conv_fields = [&](GemmProb& g, const Conv& c, int mode, int channels) {
-    g.conv = mode; g.conv_n = c.N; g.conv_h = c.H; g.conv_w = c.W; g.conv_c = channels; g.conv_k0 = 0;
+    g.conv = mode; g.conv_n = c.N; g.conv_h = c.Ho; g.conv_w = c.Wo; g.conv_c = channels; g.conv_k0 = 0;
+    g.conv_hin = c.H; g.conv_win = c.W; g.conv_stride = c.stride; g.conv_taps = c.k * c.k;
   };
   auto conv_fwd = [&](Plan& p, const Conv& c, const void* x) {
     if (c.small) {
       SmallConvProb sp{x, h.W(c.w), c.y, nullptr, nullptr, c.N, c.H, c.W, c.Cin, c.Cout};
       p.add(1, [=](const RunCtx& r) { launch_small_conv_fwd(sp, bf, bf, r.stream); }, KIND_GEMM_ALU, 2.0 * c.M * c.Cout * c.K);
+      return;
+    }
+    if (c.pointwise) {                                       // y [pixels, Cout] = x [pixels, Cin] W^T
+      emit_gemm(h, p, {gemm_fwd(x, h.W(c.w), c.y, (int)c.M, c.Cout, c.Cin, nullptr, EPI_NONE)});
       return;
     }
     if (c.imp_fwd) {
@@ -296,13 +331,17 @@ void build_resnet(Handle& h) {
       conv_fwd(p, b.c1, x);
       bn_fwd(p, b.b1, b.c1.y, b.a1, nullptr, true, mode);
       conv_fwd(p, b.c2, b.a1);
+      if (b.bottleneck) {
+        bn_fwd(p, b.b2, b.c2.y, b.a2, nullptr, true, mode);
+        conv_fwd(p, b.c3, b.a2);
+      }
       const void* res = x;
       if (b.has_sc) {
         conv_fwd(p, b.cs, x);
         bn_fwd(p, b.bs, b.cs.y, b.sc, nullptr, false, mode);
         res = b.sc;
       }
-      bn_fwd(p, b.b2, b.c2.y, out, res, true, mode);
+      bn_fwd(p, b.last_bn(), b.last().y, out, res, true, mode);
       x = out;
     }
   };
@@ -332,6 +371,7 @@ void build_resnet(Handle& h) {
   typedef std::map<std::string, float*> GradMap;
   auto GD = [&](const GradMap* second, const std::string& name) -> float* { return second ? second->at(name) : h.G(name); };
   auto wgrad_prob = [&](const Conv& c, const void* dy, const void* x, const GradMap* second = nullptr) {
+    if (c.pointwise) return gemm_wgrad(dy, x, GD(second, c.w), (int)c.M, c.Cout, c.Cin);
     if (c.imp_fwd) {
       GemmProb g = gemm_wgrad(dy, x, GD(second, c.w), (int)c.M, c.Cout, c.K);
       g.b_ks = c.Cin;
@@ -345,6 +385,7 @@ void build_resnet(Handle& h) {
   // the input gradient of a convolution: its GEMM problem and, for the explicit form, the col2im gather after it
   auto dgrad_prob = [&](const Conv& c, const void* dy, void* dx, void* dcols, Op& gather) {
     gather = Op{};
+    if (c.pointwise) return gemm_dgrad(dy, h.W(c.w), dx, (int)c.M, c.Cout, c.Cin, EPI_NONE, nullptr);
     if (c.imp_dgrad) {
       GemmProb g{};
       g.A = dy; g.B = h.W(c.w); g.C = dx;
@@ -397,8 +438,19 @@ void build_resnet(Handle& h) {
                            void* gc, void* dcols, const GradMap* second) -> void* {
     long long in_elems_blk = (long long)b.c1.N * b.c1.H * b.c1.W * b.c1.Cin;
     Op gather;
-    // out = relu(bn2(c2) + shortcut): ga <- d(c2), gb <- gradient of the shortcut branch
-    rec_bn_bwd(L, b.b2, b.c2.y, gin, out, ga, gb, second);
+    if (b.bottleneck) {
+      // out = relu(bn3(c3) + shortcut): ga <- d(c3), gb <- gradient of the shortcut branch
+      rec_bn_bwd(L, b.b3, b.c3.y, gin, out, ga, gb, second);
+      {                                                   // dW(c3) and gc <- d(a2)
+        GemmProb dg = dgrad_prob(b.c3, ga, gc, dcols, gather);
+        rec_gemm(L, {wgrad_prob(b.c3, ga, b.a2, second), dg});
+        L.push_back(gather);
+      }
+      rec_bn_bwd(L, b.b2, b.c2.y, gc, b.a2, ga, nullptr, second);   // ga <- d(c2)
+    } else {
+      // out = relu(bn2(c2) + shortcut): ga <- d(c2), gb <- gradient of the shortcut branch
+      rec_bn_bwd(L, b.b2, b.c2.y, gin, out, ga, gb, second);
+    }
     {                                                     // dW(c2) and gc <- d(a1) read the same ga: one launch
       GemmProb dg = dgrad_prob(b.c2, ga, gc, dcols, gather);
       rec_gemm(L, {wgrad_prob(b.c2, ga, b.a1, second), dg});
@@ -465,15 +517,16 @@ void build_resnet(Handle& h) {
       const void* sx = nb == 1 ? chunk_in(k - 1, rd) : q.blocks[nb - 2].out;
       if (!c.GO[0]) {
         size_t act = 0, cols = 0;
-        for (const Conv* cv : {&sb.c1, &sb.c2, &sb.cs}) {
-          if (cv == &sb.cs && !sb.has_sc) continue;
+        for (const Conv* cv : {&sb.c1, &sb.c2, &sb.c3, &sb.cs}) {
+          if ((cv == &sb.cs && !sb.has_sc) || (cv == &sb.c3 && !sb.bottleneck)) continue;
           act = std::max(act, (size_t)cv->M * cv->Cout);
           act = std::max(act, (size_t)cv->N * cv->H * cv->W * cv->Cin);
-          if (!cv->imp_dgrad) cols = std::max(cols, (size_t)cv->M * cv->ldk);
+          if (!cv->imp_dgrad && !cv->pointwise) cols = std::max(cols, (size_t)cv->M * cv->ldk);
         }
         for (int i = 0; i < 3; ++i) c.GO[i] = h.dalloc(act * es);
         if (cols) c.dcolsO = h.dalloc(cols * es);
         std::vector<std::string> names = {sb.c1.w, sb.b1.g, sb.b1.b, sb.c2.w, sb.b2.g, sb.b2.b};
+        if (sb.bottleneck) { names.push_back(sb.c3.w); names.push_back(sb.b3.g); names.push_back(sb.b3.b); }
         if (sb.has_sc) { names.push_back(sb.cs.w); names.push_back(sb.bs.g); names.push_back(sb.bs.b); }
         for (auto& n : names) q.second[n] = fal((size_t)h.tensors[h.find(n)].numel);
       }

@@ -67,7 +67,7 @@ struct Plan {
 struct Handle {
   // ---- specification
   lp_model_spec spec{};
-  std::vector<int> layer_widths, per_chunk, stage_channels;
+  std::vector<int> layer_widths, per_chunk, stage_channels, stage_blocks;
   lp_head_spec head{};
   lp_optim_spec opt{};
   int K = 0;

@@ -4,8 +4,10 @@ products of the transformer workloads in forward, input-gradient and weight-grad
     python -m paper_2012_03837_b200.kernel_bench [--shape qkv|out|ffn1|ffn2|head|all] [--form fwd|dgrad|wgrad|all]
                                                  [--d 1024] [--rows 8192] [--vocab 32768] [--groups 4] [--reps 10]
                                                  [--epilogue none|model]
+    python -m paper_2012_03837_b200.kernel_bench --shape attn [--batch 64] [--seq 512] [--heads 16] [--reps 10]
 
-Prints one JSON line per (shape, form): milliseconds per launch and TFLOP/s (2*M*N*K per problem).
+Prints one JSON line per (shape, form): milliseconds per launch and TFLOP/s (2*M*N*K per problem; attention:
+4 (forward) or 10 (backward) x batch x heads x 64 x T(T+1)/2).
 Inputs are larger than the L2 cache in total, so every launch streams its operands from HBM.
 """
 from __future__ import annotations
@@ -63,6 +65,29 @@ def descs(form, rows, n_out, n_in, groups, epilogue=(False, False, EPI_NONE)):
     return out, keep
 
 
+def attention(a):
+    """Causal attention (lp_attention_bf16) forward and backward on [batch, seq, 3 * 64 * heads]."""
+    B, T, H = a.batch, a.seq, a.heads
+    d = 64 * H
+    bf = dict(dtype=torch.bfloat16, device="cuda")
+    qkv, dout = torch.randn(B, T, 3 * d, **bf), torch.randn(B, T, d, **bf)
+    o, dqkv = torch.empty(B, T, d, **bf), torch.empty(B, T, 3 * d, **bf)
+    lse = torch.empty(B, H, T, dtype=torch.float32, device="cuda")
+    delta = torch.empty_like(lse)
+    pairs = B * H * 64.0 * T * (T + 1) / 2
+    for form, name, mult in ((lp.LP_ATTN_FORWARD, "fwd", 4.0), (lp.LP_ATTN_BACKWARD, "bwd", 10.0)):
+        for _ in range(2):
+            lp.lp_attention_bf16(form, qkv, o, lse, dout, dqkv, delta, B, T, H)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(a.reps):
+            lp.lp_attention_bf16(form, qkv, o, lse, dout, dqkv, delta, B, T, H)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / a.reps          # each call synchronises: includes ~20 us of host latency
+        print(json.dumps(dict(shape="attn", form=name, batch=B, seq=T, heads=H, ms_per_call=ms, tflops=mult * pairs / ms / 1e9)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--shape", default="all")
@@ -75,7 +100,13 @@ def main():
     ap.add_argument("--backend", type=int, default=0)
     ap.add_argument("--epilogue", default="none", choices=["none", "model"],
                     help="model: the bias / residual / GELU / GELU' epilogue that product has in the transformer block")
+    ap.add_argument("--batch", type=int, default=64)
+    ap.add_argument("--seq", type=int, default=512)
+    ap.add_argument("--heads", type=int, default=16)
     a = ap.parse_args()
+    if a.shape == "attn":
+        attention(a)
+        return
     sh = shapes(a.d, 4 * a.d, a.vocab)
     names = list(sh) if a.shape == "all" else [a.shape]
     forms = ["fwd", "dgrad", "wgrad"] if a.form == "all" else [a.form]

@@ -134,6 +134,44 @@ def test_implicit_convolution_against_the_oracle(n, h, w, c_in, c_out):
         assert err < tol, (name, err)
 
 
+@pytest.mark.parametrize("n,h,w,c_in,c_out,ksize,stride", [
+    (3, 32, 32, 64, 128, 3, 2),    # first convolution of a stage: 32x32 -> 16x16, boxes step through the input by 2
+    (6, 16, 16, 128, 256, 3, 2),   # 16x16 -> 8x8: 128-pixel boxes span two output images
+    (20, 8, 8, 256, 128, 3, 2),    # 8x8 -> 4x4: boxes of eight (four) whole output images, ragged last tile
+    (3, 32, 32, 64, 128, 1, 2),    # the 1x1 stride-2 shortcut
+    (10, 8, 8, 128, 72, 1, 2),     # ... across images, output channels not a multiple of 64
+    (2, 16, 16, 128, 64, 1, 1),    # a 1x1 stride-1 convolution (bottleneck blocks)
+])
+def test_strided_and_pointwise_implicit_convolutions_against_the_oracle(n, h, w, c_in, c_out, ksize, stride):
+    """Forward and filter gradient of the stage-opening convolutions of App. B.3's networks (3x3 stride 2, 1x1
+    stride 2) and of 1x1 convolutions, through lp_conv2d_bf16 against the oracle's convolution."""
+    rng = np.random.default_rng(n * 1000 + h * 10 + c_in + ksize)
+    pad = 1 if ksize == 3 else 0
+    ho, wo = (h - 1) // stride + 1, (w - 1) // stride + 1
+    x = lp_synth.bf16_round(rng.standard_normal((n, c_in, h, w)).astype(np.float32))
+    W = lp_synth.bf16_round((rng.standard_normal((c_out, c_in, ksize, ksize)) / np.sqrt(ksize * ksize * c_in)).astype(np.float32))
+    dy = lp_synth.bf16_round(rng.standard_normal((n, c_out, ho, wo)).astype(np.float32))
+    y_ref, cache = L.conv2d_fwd(x.astype(np.float64), W.astype(np.float64), stride, pad)
+    assert y_ref.shape == (n, c_out, ho, wo)
+    _, dW_ref = L.conv2d_bwd(dy.astype(np.float64), cache)
+    nhwc = lambda a: np.ascontiguousarray(a.transpose(0, 2, 3, 1))
+    xd, dyd = bf(nhwc(x)), bf(nhwc(dy))
+    Wd = bf(np.ascontiguousarray(W.transpose(0, 2, 3, 1)))
+    y = torch.zeros(n, ho, wo, c_out, dtype=torch.bfloat16, device="cuda")
+    dW = torch.zeros(c_out, ksize, ksize, c_in, dtype=torch.float32, device="cuda")
+    lp.lp_conv2d_bf16(lp.LP_CONV_FORWARD, xd, Wd, y, n, h, w, c_in, c_out, ksize, stride)
+    lp.lp_conv2d_bf16(lp.LP_CONV_FILTER_GRAD, xd, dyd, dW, n, h, w, c_in, c_out, ksize, stride)
+    torch.cuda.synchronize()
+    got = dict(y=y.float().cpu().numpy().transpose(0, 3, 1, 2), dW=dW.cpu().numpy().transpose(0, 3, 1, 2))
+    ref = dict(y=y_ref, dW=dW_ref)
+    for name in got:
+        err = np.abs(got[name].astype(np.float64) - ref[name]).max() / np.abs(ref[name]).max()
+        assert err < (1e-2 if name != "dW" else 1e-4), (name, err)
+    with pytest.raises(lp.LpError) as e:                     # no input gradient in this form for a stride
+        lp.lp_conv2d_bf16(lp.LP_CONV_INPUT_GRAD, dyd, Wd, y, n, h, w, c_in, c_out, ksize, 2)
+    assert lp.LP_ERR[e.value.code] == "UNSUPPORTED"
+
+
 def test_implicit_convolution_rejects_what_it_cannot_tile():
     t = torch.zeros(1 << 16, dtype=torch.bfloat16, device="cuda")
     for form, args in [(lp.LP_CONV_FORWARD, (2, 12, 12, 64, 64)),       # width does not divide 64

@@ -19,7 +19,25 @@ pytestmark = pytest.mark.gpu
 LOSS_TOL = {"fp32": 1e-4, "bf16": 2e-2}
 W_TOL = {"fp32": 1e-3, "bf16": 2e-2}          # matrices and whole chunks: ||a-b|| / ||b||
 V_TOL = {"fp32": 1e-3, "bf16": 2e-1}          # vectors: ||a-b|| / ||b - init|| (error of the update itself)
-G_TOL = {"fp32": 1e-3, "bf16": 0.35}          # first-step gradients, max|a-b| / max|b| (coarse sanity in bf16)
+# First-step gradients, per tensor ||a-b||_2 / ||b||_2.  bf16: the rounding of stored activations flips ReLU / GELU'
+# decisions of units whose pre-activation lies within rounding of zero; measured on these workloads: MLP <= 6.2e-2,
+# transformer <= 8.5e-3, ResNet (BatchNorm centres every ReLU input at zero) <= 2.2e-1.
+G_TOL = {("fp32", "mlp"): 1e-3, ("fp32", "lm"): 1e-3, ("fp32", "resnet"): 1e-3,
+         ("bf16", "mlp"): 1e-1, ("bf16", "lm"): 3e-2, ("bf16", "resnet"): 3e-1}
+
+
+def grad_l2_errors(gm, orc):
+    """Per tensor ||a-b||_2 / ||b||_2 of the last step's gradients, worst first."""
+    from paper_2012_03837_b200 import binding as lp
+    gg = gm.get(lp.LP_GRAD)
+    out = []
+    for n in gg:
+        if n in orc.buffers:
+            continue
+        a = T.strip_key_bias(n, gg[n]).astype(np.float64)
+        b = T.strip_key_bias(n, orc.last_grads[n]).astype(np.float64)
+        out.append((float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)), n))
+    return sorted(out, reverse=True)
 
 
 def check(cfg, steps=10, gemm_backend=0, grads_first=True, w_tol=None, v_tol=None, loss_tol=None):
@@ -27,18 +45,10 @@ def check(cfg, steps=10, gemm_backend=0, grads_first=True, w_tol=None, v_tol=Non
     dt = cfg["dtype"]
     if grads_first:
         gl, ol, gm, orc = T.run_both(cfg, 1, gemm_backend)
-        gg = gm.get(lp.LP_GRAD)
-        errs = sorted(((T.tensor_rel_err(T.strip_key_bias(n, gg[n]), T.strip_key_bias(n, orc.last_grads[n])), n)
-                       for n in gg if n not in orc.buffers), reverse=True)
-        print("grad rel err after step 0 (worst):", [(f"{e:.2e}", n) for e, n in errs[:5]])
-        l2 = sorted(((float(np.linalg.norm(T.strip_key_bias(n, gg[n]).astype(np.float64) - T.strip_key_bias(n, orc.last_grads[n])) /
-                            max(np.linalg.norm(T.strip_key_bias(n, orc.last_grads[n]).astype(np.float64)), 1e-30)), n)
-                     for n in gg if n not in orc.buffers), reverse=True)
+        l2 = grad_l2_errors(gm, orc)
         print("grad l2 err after step 0 (worst):", [(f"{e:.2e}", n) for e, n in l2[:5]])
         gm.close()
-        # bf16: ReLU / GELU' masks flip where a rounded pre-activation crosses zero, so the first-step
-        # gradient is only a coarse check there
-        assert errs[0][0] <= G_TOL[dt], errs[:5]
+        assert l2[0][0] <= G_TOL[(dt, cfg["family"])], l2[:5]
     gl, ol, gm, orc = T.run_both(cfg, steps, gemm_backend)
     lerr = np.abs(gl - ol) / np.abs(ol)
     werr = T.compare_weights(gm, orc, lp_synth.init_params(cfg))
@@ -116,6 +126,77 @@ def test_resnet_bf16_implicit_convolutions(size, schedule):
     cfg = lp_synth.config("c4", batch=32, height=size, width=size, stem_channels=64,
                           stage_channels=[64, 128], blocks_per_stage=2, classes=10, schedule=schedule)
     check(cfg, v_tol=0.3)
+
+
+@pytest.mark.parametrize("schedule", ["sync", "pipelined"])
+def test_resnet_bottleneck_fp32_small(schedule):
+    """Bottleneck blocks (1x1 - 3x3 - 1x1, Sec. 4.3's ResNet-50 is built of them), unequal block counts per stage,
+    fp32: the 1x1 stride-1 convolutions are plain products over the NHWC activation, the others im2col + product."""
+    cfg = lp_synth.config("c4", dtype="fp32", batch=6, height=12, width=12, stem_channels=8, block="bottleneck",
+                          stage_channels=[4, 6, 8], blocks_per_stage=[2, 1, 2], classes=5, schedule=schedule)
+    check(cfg, w_tol=5e-3, v_tol=5e-2)
+
+
+@pytest.mark.parametrize("backend", [1, 0])
+def test_resnet_bottleneck_bf16(backend):
+    """Bottleneck stages of 64 and 128 inner channels (256 and 512 out) on 16x16 images in bf16: with the tensor-core
+    backend the 3x3 convolutions (stride 1, and stride 2 at the start of the second stage) and the 1x1 stride-2
+    shortcut run as implicit GEMMs, the 1x1 stride-1 convolutions as plain GEMMs."""
+    cfg = lp_synth.config("c4", batch=32, height=16, width=16, stem_channels=64, block="bottleneck",
+                          stage_channels=[64, 128], blocks_per_stage=[2, 2], classes=10)
+    # twelve BatchNorm-ReLU layers per chunk at batch 32: both backends (they share no GEMM or convolution kernel)
+    # end at 2.5e-2 of a filter's norm after ten steps of lr 0.1 / momentum 0.9
+    check(cfg, gemm_backend=backend, w_tol=3e-2, v_tol=0.3)
+
+
+def per_chunk_worst(errs):
+    out = {}
+    for e, n in errs:
+        k = n.split(".")[0]
+        out[k] = max(out.get(k, 0.0), e)
+    return out
+
+
+def test_resnet50_shaped_stages_one_step_against_the_oracle():
+    """The stage layout of a ResNet-50 (3, 4, 6, 3 bottleneck blocks of inner width 64, 128, 256, 512; K = 4 chunks),
+    on 32x32 inputs with the 3x3 stem: one synchronous local update step.
+    fp32: losses and first-step gradients against the oracle.
+    bf16: fifty BatchNorm-ReLU layers at random initial weights turn the bf16 rounding of the stored activations
+    into first-step gradient differences that grow with depth (about 0.2, 0.4, 0.9 and 1.1 of a gradient's norm in the
+    four chunks).  That is a property of the storage format, not of the kernels: the fp32 oracle with nothing but
+    bf16 storage of its activations and weight matrices (the witness of tests/golden/make_conditioning.py) differs
+    from the plain fp32 oracle by the same amounts, and so do both GEMM backends.  The bf16 run is therefore held
+    to 1.5 x the witness's per-chunk difference."""
+    import importlib.util
+    import os
+    cfg = lp_synth.config("c4", batch=32, block="bottleneck", blocks_per_stage=[3, 4, 6, 3])
+    gl, ol, gm, orc = T.run_both(dict(cfg, dtype="fp32"), 1)
+    l2 = grad_l2_errors(gm, orc)
+    gm.close()
+    print("resnet-50 stages fp32: losses gpu", gl[0], "oracle", ol[0], "worst gradient l2 errors", [(f"{e:.2e}", n) for e, n in l2[:3]])
+    assert np.all(np.abs(gl - ol) / np.abs(ol) <= 1e-4)
+    assert l2[0][0] <= 5e-3, l2[:5]
+
+    spec = importlib.util.spec_from_file_location(
+        "make_conditioning", os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "make_conditioning.py"))
+    mc = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mc)
+    params = lp_synth.init_params(cfg)
+    gl, ol, gm, orc = T.run_both(cfg, 1, params=params)
+    got = per_chunk_worst(grad_l2_errors(gm, orc))
+    gm.close()
+    wit = mc.Bf16StorageOracle(cfg, params, dtype=np.float32)
+    wl = wit.step(*lp_synth.minibatch(cfg, 0))
+
+    class _W:                                              # the witness's gradients in the shape grad_l2_errors takes
+        def get(self, which):
+            return wit.last_grads
+    want = per_chunk_worst(grad_l2_errors(_W(), orc))
+    print("resnet-50 stages bf16: per-chunk worst gradient l2 difference: gpu", got, "witness", want)
+    for k in want:
+        assert got[k] <= 1.5 * want[k] + 1e-2, (k, got[k], want[k])
+    loss_tol = np.maximum(2e-2, 2 * np.abs(wl - ol) / np.abs(ol))
+    assert np.all(np.abs(gl - ol) / np.abs(ol) <= loss_tol), (gl, ol, wl)
 
 
 def test_sync_and_pipelined_agree_on_step0():
@@ -336,15 +417,13 @@ def check_overlap(cfg, gemm_backend=0, shared_per_boundary=2, w_tol=None, v_tol=
     from paper_2012_03837_b200 import binding as lp
     dt = cfg["dtype"]
     gl, ol, gm, orc = T.run_both(cfg, 1, gemm_backend, overlap=True)
-    gg = gm.get(lp.LP_GRAD)
-    errs = sorted(((T.tensor_rel_err(T.strip_key_bias(n, gg[n]), T.strip_key_bias(n, orc.last_grads[n])), n) for n in gg
-                   if n not in orc.buffers), reverse=True)
+    errs = grad_l2_errors(gm, orc)
     gm.close()
     plain = T.run_both(cfg, 1, gemm_backend)[3]
     shared = [n for n in orc.last_grads if not np.array_equal(orc.last_grads[n], plain.last_grads[n])]
     print("overlap: first-step gradient error (worst)", [(f"{e:.2e}", n) for e, n in errs[:3]], "shared tensors", sorted(shared))
     assert shared and (shared_per_boundary is None or len(shared) == shared_per_boundary * (gl.shape[1] - 1))
-    assert errs[0][0] <= G_TOL[dt], errs[:5]
+    assert errs[0][0] <= G_TOL[(dt, cfg["family"])], errs[:5]
     gl, ol, gm, orc = T.run_both(cfg, 10, gemm_backend, overlap=True)
     lerr = np.abs(gl - ol) / np.abs(ol)
     werr = T.compare_weights(gm, orc, lp_synth.init_params(cfg))

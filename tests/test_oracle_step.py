@@ -17,7 +17,11 @@ TINY = {
                           blocks_per_chunk=[1, 2, 1]),
     "resnet": lp_synth.config("c4", batch=3, height=4, width=4, stem_channels=4,
                               stage_channels=[4, 6], blocks_per_stage=2, classes=3),
+    # bottleneck blocks (1x1 - 3x3 - 1x1, four times the inner width out), two then one block per stage
+    "bottleneck": lp_synth.config("c4", batch=3, height=4, width=4, stem_channels=4, block="bottleneck",
+                                  stage_channels=[2, 3], blocks_per_stage=[2, 1], classes=3),
 }
+FAMS = ["mlp", "lm", "resnet", "bottleneck"]
 
 
 def one_chunk(cfg):
@@ -72,9 +76,17 @@ def torch_forward(cfg, P, x, upto=None):
         if k == 0:
             h = F.relu(F.batch_norm(F.conv2d(h, P["c0.stem.conv"], padding=1), None, None,
                                     P["c0.stem.bn.g"], P["c0.stem.bn.b"], True, 0.1, 1e-5))
-        for j in range(cfg["blocks_per_stage"]):
+        for j in range(lp_synth.resnet_stage_blocks(cfg, k)):
             n = f"c{k}.r{j}"
             s = lp_synth.resnet_stage_stride(cfg, k) if j == 0 else 1
+            bn = lambda t, m: F.batch_norm(t, None, None, P[m + ".g"], P[m + ".b"], True, 0.1, 1e-5)
+            if cfg.get("block") == "bottleneck":
+                u = F.relu(bn(F.conv2d(h, P[n + ".conv1"]), n + ".bn1"))
+                u = F.relu(bn(F.conv2d(u, P[n + ".conv2"], stride=s, padding=1), n + ".bn2"))
+                u = bn(F.conv2d(u, P[n + ".conv3"]), n + ".bn3")
+                sc = bn(F.conv2d(h, P[n + ".sc.conv"], stride=s), n + ".sc.bn") if n + ".sc.conv" in P else h
+                h = F.relu(u + sc)
+                continue
             u = F.conv2d(h, P[n + ".conv1"], stride=s, padding=1)
             u = F.relu(F.batch_norm(u, None, None, P[n + ".bn1.g"], P[n + ".bn1.b"], True, 0.1, 1e-5))
             u = F.conv2d(u, P[n + ".conv2"], padding=1)
@@ -120,12 +132,12 @@ def rel(a, b):
 
 # ---------------------------------------------------------------- P1: K = 1 is back-propagation
 
-@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+@pytest.mark.parametrize("fam", FAMS)
 def test_single_chunk_equals_backprop(fam):
     cfg = TINY[fam]
-    if fam == "resnet":
+    if fam in ("resnet", "bottleneck"):
         cfg = lp_synth.config("c4", **{k: v for k, v in cfg.items() if k != "name"})
-        cfg["stage_channels"] = [4]
+        cfg["stage_channels"] = cfg["stage_channels"][:1]      # a ResNet chunk is a stage: one stage = one chunk
     else:
         cfg = one_chunk(cfg)
     params = spread_params(cfg)
@@ -143,7 +155,7 @@ def test_single_chunk_equals_backprop(fam):
 
 # ---------------------------------------------------------------- P2: last chunk = backprop's gradient
 
-@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+@pytest.mark.parametrize("fam", FAMS)
 def test_last_chunk_gradients_are_backprop_gradients(fam):
     cfg = TINY[fam]
     K = lp_synth.num_chunks(cfg)
@@ -164,7 +176,7 @@ def test_last_chunk_gradients_are_backprop_gradients(fam):
 
 # ---------------------------------------------------------------- P3: finite differences, input frozen
 
-@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+@pytest.mark.parametrize("fam", FAMS)
 def test_local_gradients_match_finite_differences(fam):
     cfg = TINY[fam]
     K = lp_synth.num_chunks(cfg)
@@ -196,7 +208,7 @@ def test_local_gradients_match_finite_differences(fam):
 
 # ---------------------------------------------------------------- P4: chunks are independent
 
-@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+@pytest.mark.parametrize("fam", FAMS)
 def test_chunk_update_ignores_other_chunks_heads_and_losses(fam):
     cfg = TINY[fam]
     K = lp_synth.num_chunks(cfg)
@@ -246,7 +258,7 @@ def test_stop_gradient_is_real():
 
 # ---------------------------------------------------------------- P5: schedules
 
-@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+@pytest.mark.parametrize("fam", FAMS)
 def test_sync_and_pipelined_agree_on_step0(fam):
     cfg = TINY[fam]
     params = spread_params(cfg)
@@ -474,7 +486,7 @@ def test_resnet_head_with_batchnorm_and_relu_follows_reverse_mode_and_the_librar
 
 # ---------------------------------------------------------------- overlapping local parallelism (Sec. 3, Fig. 2 c)
 
-@pytest.mark.parametrize("fam", ["mlp", "lm", "resnet"])
+@pytest.mark.parametrize("fam", FAMS)
 def test_overlapping_updates_average_the_two_backprop_gradients_of_the_shared_layer(fam):
     """With overlap, the last layer (transformer: last block) of every chunk but the final one also belongs to
     the next chunk's block.  Its gradient from either loss is that loss's ordinary back-propagation gradient
@@ -501,9 +513,9 @@ def test_overlapping_updates_average_the_two_backprop_gradients_of_the_shared_la
             names = [n for n in over.names_of_chunk[k] if n.startswith(blk + ".")]
             assert len(names) == 12
         else:
-            blk = f"c{k}.r{cfg['blocks_per_stage'] - 1}"
+            blk = f"c{k}.r{lp_synth.resnet_stage_blocks(cfg, k) - 1}"
             names = [n for n in over.names_of_chunk[k] if n.startswith(blk + ".") and n not in over.buffers]
-            assert len(names) == 6
+            assert len(names) == (9 if fam == "bottleneck" else 6)
         for n in names:
             shared.add(n)
             want = 0.5 * (tg[k][n] + tg[k + 1][n])
