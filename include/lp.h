@@ -241,6 +241,17 @@ enum { LP_RAMP_PRIME = 0, LP_RAMP_IDLE = 1 };
 lp_status lp_set_ramp(lp_handle h, int ramp);
 
 /*
+ * lp_set_drain: the end of a pipelined run (Sec. 6: each stage works on the minibatch its predecessor finished one
+ * iteration earlier, so the last minibatch leaves chunk k only k iterations after it entered chunk 0).  In
+ * pipelined steps that follow, chunks 0 .. idle_first-1 idle: their minibatches are exhausted, so their parameters,
+ * optimizer state and step counts stay as they are and their entry of out_losses is NaN, while the chunks behind
+ * them go on with what the boundary buffers still hold.  (Like the chunks that idle during the ramp-up they still
+ * execute; what they publish is not read by a training chunk.)  idle_first = 0 ends the drain.  Pipelined steps
+ * only.  Errors: INVALID_ARG (idle_first outside [0, K]).
+ */
+lp_status lp_set_drain(lp_handle h, int idle_first);
+
+/*
  * lp_set_overlap: overlapping local parallelism (Sec. 3, Fig. 2 c; cost in App. A.2).  With on != 0 the
  * block trained by chunk k's loss also contains the last layer of chunk k-1: that loss is propagated one
  * layer past the chunk boundary and stops at that layer's input.  The shared layer exists once (one forward

@@ -62,7 +62,7 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
-           "lp_attention_bf16", "lp_gemm_bf16_static", "lp_gemm_static_poll", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_conv2d_bf16", "lp_set_ramp", "lp_evaluate", "lp_set_overlap",
+           "lp_attention_bf16", "lp_gemm_bf16_static", "lp_gemm_static_poll", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_conv2d_bf16", "lp_set_ramp", "lp_set_drain", "lp_evaluate", "lp_set_overlap",
            "lp_cost_model", "lp_mlp_layer_flops", "lp_mlp_aux_flops", "lp_chunk_output_bytes", "lp_chunk_output"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
@@ -249,6 +249,10 @@ LP_RAMP_PRIME, LP_RAMP_IDLE = 0, 1
 
 def lp_set_ramp(h, ramp: int):
     _check(h, _lib.lp_set_ramp(h, ramp))
+
+
+def lp_set_drain(h, idle_first: int):
+    _check(h, _lib.lp_set_drain(h, idle_first))
 
 
 def lp_chunk_output_bytes(h, k: int) -> int:

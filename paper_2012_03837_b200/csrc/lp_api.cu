@@ -162,6 +162,8 @@ bool prepare_chunks(Handle& h, int schedule, cudaStream_t s, std::vector<char>& 
   if (schedule == LP_PIPELINED && h.ramp == LP_RAMP_IDLE)
     for (int k = 0; k < K; ++k)
       if (k > h.pipe_steps) { active[k] = 0; any_idle = true; }
+  if (schedule == LP_PIPELINED)
+    for (int k = 0; k < h.drain_first && k < K; ++k) { active[k] = 0; any_idle = true; }
   for (int k = 1; k < K; ++k) differ |= h.updates[k] != h.updates[0];
   h.per_chunk_counts = any_idle || differ;
   if (h.per_chunk_counts || h.spec.family == LP_FAMILY_RESNET) {   // BatchNorm reads the active flags every step
@@ -406,6 +408,7 @@ lp_status lp_reset_pipeline(lp_handle hh) {
   hh->h.primed = false;
   hh->h.parity = 0;
   hh->h.pipe_steps = 0;
+  hh->h.drain_first = 0;
   return LP_OK;
 }
 
@@ -430,6 +433,14 @@ lp_status lp_set_overlap(lp_handle hh, int on) {
   if (on && !h.has_overlap_plan)
     return fail(&h, LP_ERR_UNSUPPORTED, "overlapping updates need at least two chunks");
   h.overlap = on != 0;
+  return LP_OK;
+}
+
+lp_status lp_set_drain(lp_handle hh, int idle_first) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (idle_first < 0 || idle_first > h.K) return fail(&h, LP_ERR_INVALID_ARG, "lp_set_drain: idle_first outside [0, K]");
+  h.drain_first = idle_first;
   return LP_OK;
 }
 

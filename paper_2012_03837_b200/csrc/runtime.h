@@ -111,6 +111,7 @@ struct Handle {
   // ---- ramp-up of the pipelined schedule (Sec. 6): LP_RAMP_PRIME fills the boundary buffers by a forward
   // pass; LP_RAMP_IDLE lets chunk k idle until the k-th pipelined step after a reset
   int ramp = 0;
+  int drain_first = 0;                         // chunks below this index idle in pipelined steps (end of a run)
   long long pipe_steps = 0;                    // pipelined steps since create / reset
   std::vector<long long> updates;              // per chunk: optimizer updates made so far
   bool per_chunk_counts = false;               // some chunk has idled: the chunks' step counts differ

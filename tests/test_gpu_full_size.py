@@ -56,10 +56,11 @@ def run_against_witness(cfg, witnesses, base_w, base_loss, base_v):
     (CPU oracle alone) as the largest over the chunks, over the listed witnesses and over steps t and t+1: which
     chunk a rounding event hits, and at which step the first one falls, is chance.  Losses: the gap is a series of isolated transients that move down the pipeline with the
     minibatch that caused them, and their size differs between two realisations of the same kind of perturbation
-    by more than a factor of two (5.6e-3 and 1.3e-2 in the two bf16 witnesses of c2), so the bound is
-    max(nominal, 3 x the largest gap of any witness at any of the ten steps)."""
+    by more than a factor of two (5.6e-3 and 1.3e-2 in the two bf16 witnesses of c2; the library's largest: 3.0e-2
+    in bf16, 5.3e-3 with fp32 storage against 1.5e-3 of the fp32 witness), so the bound is
+    max(nominal, 4 x the largest gap of any witness at any of the ten steps)."""
     gold = golden(cfg["name"])
-    loss_tol = max(base_loss, 3 * max(max(s[w]["loss"]) for s in gold for w in witnesses))
+    loss_tol = max(base_loss, 4 * max(max(s[w]["loss"]) for s in gold for w in witnesses))
     params = lp_synth.init_params(cfg)
     gm = T.GpuModel(cfg, params)
     orc = LocalUpdateOracle(cfg, params, dtype=np.float32)

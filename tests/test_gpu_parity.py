@@ -169,13 +169,28 @@ def test_resnet50_shaped_stages_one_step_against_the_oracle():
     to 1.5 x the witness's per-chunk difference."""
     import importlib.util
     import os
+    from oracle.local_step import LocalUpdateOracle
     cfg = lp_synth.config("c4", batch=32, block="bottleneck", blocks_per_stage=[3, 4, 6, 3])
-    gl, ol, gm, orc = T.run_both(dict(cfg, dtype="fp32"), 1)
-    l2 = grad_l2_errors(gm, orc)
+    # fp32: the same fifty layers amplify even fp32 rounding (the oracle in fp32 differs from itself in fp64 by up to
+    # 1.2e-2 of a first-step gradient's norm in the last chunk), so the fp32 run is compared with the fp64 oracle and
+    # held to twice the fp32 oracle's own distance from it, chunk by chunk
+    c32 = dict(cfg, dtype="fp32")
+    p32 = lp_synth.init_params(c32)
+    gl, ol, gm, orc = T.run_both(c32, 1, params=p32)
+    o64 = LocalUpdateOracle(c32, p32, dtype=np.float64)
+    l64 = o64.step(*lp_synth.minibatch(c32, 0))
+    got = per_chunk_worst(grad_l2_errors(gm, o64))
     gm.close()
-    print("resnet-50 stages fp32: losses gpu", gl[0], "oracle", ol[0], "worst gradient l2 errors", [(f"{e:.2e}", n) for e, n in l2[:3]])
-    assert np.all(np.abs(gl - ol) / np.abs(ol) <= 1e-4)
-    assert l2[0][0] <= 5e-3, l2[:5]
+
+    class _O:                                              # the fp32 oracle's gradients in the shape grad_l2_errors takes
+        def get(self, which):
+            return orc.last_grads
+    own = per_chunk_worst(grad_l2_errors(_O(), o64))
+    print("resnet-50 stages fp32: losses gpu", gl[0], "oracle fp64", l64, "per-chunk worst gradient l2 difference to the "
+          "fp64 oracle: gpu", got, "fp32 oracle", own)
+    assert np.all(np.abs(gl[0] - l64) / np.abs(l64) <= 1e-4)
+    for k in own:
+        assert got[k] <= 2 * own[k] + 1e-4, (k, got[k], own[k])
 
     spec = importlib.util.spec_from_file_location(
         "make_conditioning", os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "make_conditioning.py"))
