@@ -263,6 +263,33 @@ struct OptimArgs {
   const float4* chunk_tab;
 };
 void launch_optim(const OptimArgs& a, cudaStream_t s);
+
+// ---------------------------------------------------------------------------- single-launch MLP step (fp32)
+// A step as a list of phases; the blocks of one cooperative launch share a phase's work units round-robin and
+// meet at a grid-wide barrier between phases.  A task is a run of units of one kind: 16x16 or 32x32 output
+// tiles of a GEMM (GemmProb, fp32 operands; tiles_n = tiles along N), groups of 8 softmax cross-entropy rows,
+// groups of 256 columns of a column sum, one loss reduction, one label check, groups of 1024 arena elements
+// of the optimizer sweep.
+enum FusedTaskType { FT_GEMM16 = 0, FT_GEMM32, FT_XENT, FT_COLSUM, FT_LOSS, FT_LABELS, FT_OPTIM };
+struct FusedTask { int type, index, unit_start, units; };      // index into the array of its kind
+struct FusedPhase { int task_begin, task_end, units; };
+struct FusedXent { float* z; const int* y; const int* n_valid; float* row_loss; int rows, classes, ld; };
+struct FusedColSum { const float* x; float* out; int rows, cols, ld; };
+struct FusedArgs {
+  const FusedPhase* phases; int n_phases;
+  const FusedTask* tasks;
+  const GemmProb* gemms; const FusedXent* xents; const FusedColSum* colsums; const LossProb* losses;
+  const LabelProb* labels;
+  OptimArgs opt;                      // chunk_tab non-null: per-chunk mode (idle chunks make no update, read NaN)
+  float* d_losses; int* status;
+  unsigned long long* counter;        // [2], zero between launches: barrier arrivals, blocks that have left
+  // the step's inputs are read where the caller holds them: an operand or label pointer equal to x_slot /
+  // y_slot (the handle's own input buffers, which the task tables name) is replaced by x / y
+  const void* x_slot; const int* y_slot; const void* x; const int* y;
+};
+// Blocks of one cooperative launch (one per SM), or 0 if the kernel cannot be resident.
+int fused_mlp_max_blocks(int num_sms);
+cudaError_t launch_fused_mlp_step(const FusedArgs& args, int blocks, cudaStream_t s);
 // losses[k] = NaN for the chunks whose chunk_tab entry is inactive
 void launch_mask_losses(float* losses, const float4* chunk_tab, int K, cudaStream_t s);
 
