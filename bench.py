@@ -385,7 +385,11 @@ def measure(lp, torch, cfg, steps, warmup, dist, dev, rank, world, local, cpu_st
         ams, aflop, al = prof["gemm_alu"]
         achieved = aflop / max(ams * 1e-3, 1e-12) / 1e12
         peak = 148 * 128 * 2 * 1.965e9 / 1e12        # FP32 FMA lanes x 2 FLOP x max SM clock
-        roof = dict(bound="alu", kernel="gemm_simt_kernel (grouped FP32-ALU GEMM)", achieved=achieved, peak=peak,
+        one_launch = launches == steps
+        roof = dict(bound="alu",
+                    kernel=("fused_mlp_step_kernel (the whole step as one cooperative launch: a chain of dependent "
+                            "phases, bound by their latency, not by the FP32 lanes)") if one_launch
+                    else "gemm_simt_kernel (grouped FP32-ALU GEMM)", achieved=achieved, peak=peak,
                     unit="TFLOP/s", frac=achieved / peak, peak_source="148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
                     traffic=None, launches=al, ms_per_launch=ams / max(al, 1), share_of_step=ams / ms_profiled)
     breakdown = {}

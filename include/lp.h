@@ -252,6 +252,20 @@ lp_status lp_set_ramp(lp_handle h, int ramp);
 lp_status lp_set_drain(lp_handle h, int idle_first);
 
 /*
+ * lp_set_fused_step: the single-launch form of the step.  A small MLP with fp32 storage (a step of at most a few
+ * GFLOP, K <= 64) is bound by the latency of its dependent launches, not by arithmetic; for such a handle the
+ * whole step of Sec. 3 -- label check, forward of every chunk, heads, losses, backward inside each chunk,
+ * per-chunk optimizer update -- runs as ONE cooperative launch whose thread blocks walk the phases of the step
+ * together, with a grid-wide barrier (bounded wait: LP_ERR_TIMEOUT at the next lp_status_poll) between phases.
+ * Same arithmetic as the grouped launches up to the order of fp32 sums; every sum has a fixed order, so a step
+ * is bit-reproducible.  lp_step then reads x and y where the caller holds them (no copy into the handle).  It is
+ * on by default where it is available and never used with overlapping updates (lp_set_overlap).  on = 0 selects
+ * the grouped launches.  Errors: UNSUPPORTED (on != 0 for a handle that has no single-launch form: another
+ * family, bf16 storage, a larger network).
+ */
+lp_status lp_set_fused_step(lp_handle h, int on);
+
+/*
  * lp_set_overlap: overlapping local parallelism (Sec. 3, Fig. 2 c; cost in App. A.2).  With on != 0 the
  * block trained by chunk k's loss also contains the last layer of chunk k-1: that loss is propagated one
  * layer past the chunk boundary and stops at that layer's input.  The shared layer exists once (one forward

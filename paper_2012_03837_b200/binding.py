@@ -62,7 +62,7 @@ EXPORTS = ["lp_create", "lp_step", "lp_step_host", "lp_forward", "lp_destroy", "
            "lp_tensor_info_get", "lp_get_tensor", "lp_set_tensor", "lp_reset_pipeline", "lp_status_poll",
            "lp_state_size", "lp_save_state", "lp_load_state", "lp_last_step_launches", "lp_device_bytes",
            "lp_last_error", "lp_gemm_bf16", "lp_profile_enable", "lp_profile_read",
-           "lp_attention_bf16", "lp_gemm_bf16_static", "lp_gemm_static_poll", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_conv2d_bf16", "lp_set_ramp", "lp_set_drain", "lp_evaluate", "lp_set_overlap",
+           "lp_attention_bf16", "lp_gemm_bf16_static", "lp_gemm_static_poll", "lp_gemm_static_last_error", "lp_conv3x3_bf16", "lp_conv2d_bf16", "lp_set_ramp", "lp_set_drain", "lp_set_fused_step", "lp_evaluate", "lp_set_overlap",
            "lp_cost_model", "lp_mlp_layer_flops", "lp_mlp_aux_flops", "lp_chunk_output_bytes", "lp_chunk_output"]
 LP_KIND_NAMES = ["other", "gemm_tc", "gemm_alu", "norm", "xent", "attn", "optim", "reduce", "embed", "conv_aux"]
 
@@ -87,6 +87,8 @@ def load_library() -> C.CDLL:
     lib.lp_chunk_output_bytes.restype = C.c_size_t
     lib.lp_chunk_output.argtypes = [vp, ip, vp, C.c_size_t, vp]
     lib.lp_set_ramp.argtypes = [vp, ip]
+    lib.lp_set_drain.argtypes = [vp, ip]
+    lib.lp_set_fused_step.argtypes = [vp, ip]
     lib.lp_set_overlap.argtypes = [vp, ip]
     lib.lp_status_poll.argtypes = [vp, vp]
     lib.lp_state_size.argtypes = [vp]
@@ -253,6 +255,10 @@ def lp_set_ramp(h, ramp: int):
 
 def lp_set_drain(h, idle_first: int):
     _check(h, _lib.lp_set_drain(h, idle_first))
+
+
+def lp_set_fused_step(h, on: bool):
+    _check(h, _lib.lp_set_fused_step(h, 1 if on else 0))
 
 
 def lp_chunk_output_bytes(h, k: int) -> int:

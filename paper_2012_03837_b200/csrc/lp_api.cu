@@ -179,16 +179,48 @@ bool prepare_chunks(Handle& h, int schedule, cudaStream_t s, std::vector<char>& 
   return any_idle;
 }
 
-lp_status run_step(Handle& h, int schedule, cudaStream_t s) {
+// Whether this step runs as the single cooperative launch (small fp32 MLP), and whether that launch may read
+// the caller's device buffers in place (not when a priming pass, which reads the handle's own, comes first).
+bool step_is_fused(const Handle& h) { return h.use_fused && h.fused_blocks > 0 && !h.overlap; }
+bool step_reads_in_place(const Handle& h, int schedule) {
+  return step_is_fused(h) && !(schedule == LP_PIPELINED && !h.primed && h.ramp == LP_RAMP_PRIME);
+}
+
+int run_fused(Handle& h, const Handle::FusedProgram& fp, const RunCtx& c) {
+  FusedArgs a = fp.args;
+  a.opt = optimizer_args(h);
+  a.x = c.x ? c.x : h.x_in;
+  a.y = c.y ? c.y : h.y_in;
+  ProfRecord r{KIND_GEMM_ALU, 1, fp.flops, nullptr, nullptr};
+  if (c.prof) {
+    cudaEventCreate(&r.e0);
+    cudaEventCreate(&r.e1);
+    cudaEventRecord(r.e0, c.stream);
+  }
+  launch_fused_mlp_step(a, h.fused_blocks, c.stream);
+  if (c.prof) {
+    cudaEventRecord(r.e1, c.stream);
+    c.prof->push_back(r);
+  }
+  return 1;
+}
+
+lp_status run_step(Handle& h, int schedule, cudaStream_t s, const void* x = nullptr, const int* y = nullptr) {
   RunCtx ctx{s, nullptr, h.profiling ? &h.prof : nullptr};
+  const bool fused = step_is_fused(h);
+  if (x && step_reads_in_place(h, schedule)) { ctx.x = x; ctx.y = y; }
   int launches = 0;
   std::vector<char> active;
   const bool any_idle = prepare_chunks(h, schedule, s, active);
   if (schedule == LP_SYNC) {
     if (h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
-    const Plan& plan = h.overlap ? h.sync_overlap_plan : h.sync_plan;
-    plan.run(ctx);
-    launches = plan.launches;
+    if (fused) {
+      launches = run_fused(h, h.fused_sync, ctx);
+    } else {
+      const Plan& plan = h.overlap ? h.sync_overlap_plan : h.sync_plan;
+      plan.run(ctx);
+      launches = plan.launches;
+    }
     h.last_wr = 0;
   } else {
     if (!h.primed && h.ramp == LP_RAMP_PRIME) {
@@ -199,9 +231,13 @@ lp_status run_step(Handle& h, int schedule, cudaStream_t s) {
     // Idle chunks run through the plan as well, on whatever their boundary buffer holds (finite values:
     // zeros after lp_create); the optimizer leaves their parameters alone, their losses read NaN, and
     // what they publish is overwritten before an active chunk reads it.
-    h.pipe_plan[h.parity].run(ctx);
-    launches += h.pipe_plan[h.parity].launches;
-    if (any_idle) { launch_mask_losses(h.d_losses, h.d_chunk_tab, h.K, s); launches += 1; }
+    if (fused) {
+      launches += run_fused(h, h.fused_pipe[h.parity], ctx);          // masks the idle chunks' losses itself
+    } else {
+      h.pipe_plan[h.parity].run(ctx);
+      launches += h.pipe_plan[h.parity].launches;
+      if (any_idle) { launch_mask_losses(h.d_losses, h.d_chunk_tab, h.K, s); launches += 1; }
+    }
     h.last_wr = 1 - h.parity;
     h.parity ^= 1;
     h.pipe_steps += 1;
@@ -315,9 +351,14 @@ lp_status lp_step(lp_handle hh, const void* x, const void* y, int schedule, void
   if (schedule == LP_SYNC && h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
   if (schedule == LP_PIPELINED && h.overlap) return fail(&h, LP_ERR_UNSUPPORTED, "overlapping updates take both gradients of a shared layer from one minibatch: synchronous schedule only");
   cudaStream_t s = (cudaStream_t)stream;
-  lp_status st = copy_inputs(h, x, y, cudaMemcpyDeviceToDevice, s);
-  if (st != LP_OK) return st;
-  st = run_step(h, schedule, s);
+  lp_status st = LP_OK;
+  if (step_reads_in_place(h, schedule)) {
+    st = run_step(h, schedule, s, x, (const int*)y);
+  } else {
+    st = copy_inputs(h, x, y, cudaMemcpyDeviceToDevice, s);
+    if (st != LP_OK) return st;
+    st = run_step(h, schedule, s);
+  }
   if (st != LP_OK) return st;
   cudaMemcpyAsync(out_losses, h.d_losses, sizeof(float) * h.K, cudaMemcpyDeviceToDevice, s);
   return check_cuda(&h, "lp_step");
@@ -441,6 +482,14 @@ lp_status lp_set_drain(lp_handle hh, int idle_first) {
   Handle& h = hh->h;
   if (idle_first < 0 || idle_first > h.K) return fail(&h, LP_ERR_INVALID_ARG, "lp_set_drain: idle_first outside [0, K]");
   h.drain_first = idle_first;
+  return LP_OK;
+}
+
+lp_status lp_set_fused_step(lp_handle hh, int on) {
+  if (!hh) return LP_ERR_INVALID_ARG;
+  Handle& h = hh->h;
+  if (on && h.fused_blocks <= 0) return fail(&h, LP_ERR_UNSUPPORTED, "lp_set_fused_step: this handle has no single-launch form of the step");
+  h.use_fused = on != 0;
   return LP_OK;
 }
 

@@ -266,20 +266,31 @@ void launch_optim(const OptimArgs& a, cudaStream_t s);
 
 // ---------------------------------------------------------------------------- single-launch MLP step (fp32)
 // A step as a list of phases; the blocks of one cooperative launch share a phase's work units round-robin and
-// meet at a grid-wide barrier between phases.  A task is a run of units of one kind: 16x16 or 32x32 output
-// tiles of a GEMM (GemmProb, fp32 operands; tiles_n = tiles along N), groups of 8 softmax cross-entropy rows,
-// groups of 256 columns of a column sum, one loss reduction, one label check, groups of 1024 arena elements
-// of the optimizer sweep.
-enum FusedTaskType { FT_GEMM16 = 0, FT_GEMM32, FT_XENT, FT_COLSUM, FT_LOSS, FT_LABELS, FT_OPTIM };
+// meet at a grid-wide barrier between phases.  A task is a run of units of one kind, a unit being what one block
+// of FUSED_THREADS threads does at a time: a 16x16 or 32x32 output tile of a GEMM, one softmax cross-entropy row
+// per warp, one column of a column sum per thread, one loss reduction, one label check, four arena elements of
+// the optimizer sweep per thread, one 128-byte line per thread of a range to be brought into L2 ahead of its use.
+enum { FUSED_THREADS = 512 };
+enum FusedTaskType { FT_GEMM16 = 0, FT_GEMM32, FT_XENT, FT_COLSUM, FT_LOSS, FT_LABELS, FT_OPTIM, FT_PREFETCH };
 struct FusedTask { int type, index, unit_start, units; };      // index into the array of its kind
 struct FusedPhase { int task_begin, task_end, units; };
+// C[m,n] = epilogue(sum_k A(m,k) B(n,k)) with the operand conventions of GemmProb, fp32 throughout; act is
+// EPI_NONE, EPI_RELU (after the bias) or EPI_RELU_MASK (aux = the layer's output, [M, ldc])
+struct FusedGemm {
+  const float* A; const float* B; float* C; const float* bias; const float* aux;
+  int M, N, K, ldc, act, tiles_n;
+  int a_ms, a_ks, b_ns, b_ks;
+};
 struct FusedXent { float* z; const int* y; const int* n_valid; float* row_loss; int rows, classes, ld; };
 struct FusedColSum { const float* x; float* out; int rows, cols, ld; };
+struct FusedPrefetch { const void* p; long long bytes; };
+enum { FUSED_MAX_PHASES = 64, FUSED_MAX_TASKS = 256, FUSED_MAX_GEMMS = 64 };   // tables that are held in shared memory
 struct FusedArgs {
   const FusedPhase* phases; int n_phases;
-  const FusedTask* tasks;
-  const GemmProb* gemms; const FusedXent* xents; const FusedColSum* colsums; const LossProb* losses;
-  const LabelProb* labels;
+  const FusedTask* tasks; int n_tasks;
+  const FusedGemm* gemms; int n_gemms;
+  const FusedXent* xents; const FusedColSum* colsums; const LossProb* losses; const LabelProb* labels;
+  const FusedPrefetch* prefetches;
   OptimArgs opt;                      // chunk_tab non-null: per-chunk mode (idle chunks make no update, read NaN)
   float* d_losses; int* status;
   unsigned long long* counter;        // [2], zero between launches: barrier arrivals, blocks that have left

@@ -43,6 +43,59 @@ void forward_level(Handle& h, MlpBufs& b, Plan& p, const std::vector<int>& ks, i
   }
 }
 
+// Collects the phases of a single-launch step (FusedArgs).  The GEMMs of a phase are held back until the phase
+// ends: whether they are cut into 16x16 or 32x32 tiles depends on how many tiles the whole phase has.
+struct FusedBuilder {
+  std::vector<FusedPhase> phases;
+  std::vector<FusedTask> tasks;
+  std::vector<FusedGemm> gemms;
+  std::vector<GemmProb> held;
+  std::vector<FusedPrefetch> prefetches;
+  std::vector<FusedXent> xents;
+  std::vector<FusedColSum> colsums;
+  std::vector<LossProb> losses;
+  std::vector<LabelProb> labels;
+  int grid = 148;
+  double flops = 0;
+
+  void begin() { phases.push_back(FusedPhase{(int)tasks.size(), (int)tasks.size(), 0}); held.clear(); }
+  void add(int type, int index, int n) {
+    if (n <= 0) return;
+    tasks.push_back(FusedTask{type, index, phases.back().units, n});
+    phases.back().units += n;
+    phases.back().task_end = (int)tasks.size();
+  }
+  void gemm(const GemmProb& g) { held.push_back(g); }
+  void xent(const FusedXent& x) { xents.push_back(x); add(FT_XENT, (int)xents.size() - 1, (x.rows + FUSED_THREADS / 32 - 1) / (FUSED_THREADS / 32)); }
+  void colsum(const FusedColSum& c) { colsums.push_back(c); add(FT_COLSUM, (int)colsums.size() - 1, (c.cols + FUSED_THREADS - 1) / FUSED_THREADS); }
+  void loss(const LossProb& l) { losses.push_back(l); add(FT_LOSS, (int)losses.size() - 1, 1); }
+  void label(const LabelProb& l) { labels.push_back(l); add(FT_LABELS, (int)labels.size() - 1, 1); }
+  void optim(long long n_total) { add(FT_OPTIM, 0, (int)((n_total / 4 + FUSED_THREADS - 1) / FUSED_THREADS)); }
+  void prefetch(const void* p, long long bytes) {
+    prefetches.push_back(FusedPrefetch{p, bytes});
+    add(FT_PREFETCH, (int)prefetches.size() - 1, (int)((bytes + 128 * FUSED_THREADS - 1) / (128 * FUSED_THREADS)));
+  }
+  void end() {
+    flush();
+    if (phases.back().units == 0) phases.pop_back();
+  }
+  void flush() {                                         // cut the held GEMMs into tiles
+    long long t16 = 0;
+    for (auto& g : held) t16 += (long long)((g.M + 15) / 16) * ((g.N + 15) / 16);
+    const bool crowded = t16 > 2ll * grid;             // more than two waves of small tiles: cut larger ones
+    for (auto& g : held) {
+      const bool big = crowded && g.M >= 32 && g.N >= 32;
+      const int T = big ? 32 : 16;
+      FusedGemm f{(const float*)g.A, (const float*)g.B, (float*)g.C, g.bias, (const float*)g.aux,
+                  g.M, g.N, g.K, g.ldc, g.act, (g.N + T - 1) / T, (int)g.a_ms, (int)g.a_ks, (int)g.b_ns, (int)g.b_ks};
+      gemms.push_back(f);
+      add(big ? FT_GEMM32 : FT_GEMM16, (int)gemms.size() - 1, ((g.M + T - 1) / T) * f.tiles_n);
+      flops += 2.0 * g.M * g.N * g.K;
+    }
+    held.clear();
+  }
+};
+
 }  // namespace
 
 void build_mlp(Handle& h) {
@@ -219,6 +272,128 @@ void build_mlp(Handle& h) {
     emit_argmax(h, p, am);
     emit_xent_and_loss(h, p, xs, all);
   };
+
+  unsigned long long* fused_counter = nullptr;
+  // The same step as one cooperative launch (fp32 storage, small networks: a step of at most a few GFLOP on
+  // at most 64 chunks; larger ones are bound by arithmetic and keep the grouped launches above).
+  auto build_fused = [&](Handle::FusedProgram& fp, bool pipelined, int rd, int wr) {
+    FusedBuilder fb;
+    fb.grid = h.fused_blocks;
+    fb.begin();
+    for (int k = 0; k < K; ++k)
+      fb.label(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, B, C, h.n_valid[k]});
+    auto layer = [&](int k, int i) {
+      const bool last = i + 1 == (int)b.widths[k].size();
+      const void* in = i == 0 ? chunk_in(h, k, rd) : b.y[k][i - 1];
+      const int din = i == 0 ? b.d_in[k] : b.widths[k][i - 1];
+      fb.gemm(gemm_fwd(in, h.W(tn(k, i, "W")), last ? h.bnd[wr][k] : b.y[k][i], B, b.widths[k][i], din,
+                       h.P32(tn(k, i, "b")), EPI_RELU));
+    };
+    size_t maxl = 0;
+    for (int k = 0; k < K; ++k) maxl = std::max(maxl, b.widths[k].size());
+    // The label checks share the first forward phase, and so does a sweep that asks for the parameters and
+    // the optimizer state to be brought into L2 (the blocks that have no tile in that phase issue it): the
+    // later phases then find their operands there instead of waiting for DRAM one phase after the other.
+    bool first = true;
+    auto end_phase = [&]() {
+      if (first) {
+        fb.flush();
+        const long long bytes = h.n_total * (long long)sizeof(float);
+        if (bytes <= (4ll << 20)) {
+          fb.prefetch(h.master, bytes);
+          fb.prefetch(h.m1, bytes);
+          if (h.m2) fb.prefetch(h.m2, bytes);
+        }
+      }
+      first = false;
+      fb.end();
+    };
+    if (pipelined) {
+      for (size_t i = 0; i < maxl; ++i) {
+        if (!first) fb.begin();
+        for (int k = 0; k < K; ++k) if (i < b.widths[k].size()) layer(k, (int)i);
+        end_phase();
+      }
+    } else {
+      for (int k = 0; k < K; ++k)
+        for (int i = 0; i < (int)b.widths[k].size(); ++i) {
+          if (!first) fb.begin();
+          layer(k, i);
+          end_phase();
+        }
+    }
+    fb.begin();                                          // heads: logits
+    for (int k = 0; k < K; ++k)
+      fb.gemm(gemm_fwd(h.bnd[wr][k], h.W(hn(k, "W")), b.z[k], B, C, b.widths[k].back(), h.P32(hn(k, "b")), EPI_NONE));
+    fb.end();
+    fb.begin();                                          // losses of the rows, dlogits in place
+    for (int k = 0; k < K; ++k)
+      fb.xent(FusedXent{(float*)b.z[k], labels_of(k, pipelined, rd), h.n_valid[k], b.row_loss[k], B, C, C});
+    fb.end();
+    fb.begin();                                          // head backward, chunk losses
+    for (int k = 0; k < K; ++k) {
+      const int D = b.widths[k].back();
+      fb.gemm(gemm_wgrad(b.z[k], h.bnd[wr][k], h.G(hn(k, "W")), B, C, D));
+      fb.gemm(gemm_dgrad(b.z[k], h.W(hn(k, "W")), b.g0[k], B, C, D, EPI_RELU_MASK, h.bnd[wr][k]));
+      fb.colsum(FusedColSum{(const float*)b.z[k], h.G(hn(k, "b")), B, C, C});
+      fb.loss(LossProb{b.row_loss[k], h.n_valid[k], B, k});
+    }
+    fb.end();
+    for (size_t j = 0; j < maxl; ++j) {                  // trunk backward, aligned from the last layer of each chunk
+      fb.begin();
+      for (int k = 0; k < K; ++k) {
+        const int nl = (int)b.widths[k].size();
+        if ((int)j >= nl) continue;
+        const int i = nl - 1 - (int)j;
+        void* du = (j % 2 == 0) ? b.g0[k] : b.g1[k];
+        void* dnext = (j % 2 == 0) ? b.g1[k] : b.g0[k];
+        const void* in = i == 0 ? chunk_in(h, k, rd) : b.y[k][i - 1];
+        const int din = i == 0 ? b.d_in[k] : b.widths[k][i - 1];
+        const int w = b.widths[k][i];
+        fb.gemm(gemm_wgrad(du, in, h.G(tn(k, i, "W")), B, w, din));
+        if (i > 0) fb.gemm(gemm_dgrad(du, h.W(tn(k, i, "W")), dnext, B, w, din, EPI_RELU_MASK, b.y[k][i - 1]));
+        fb.colsum(FusedColSum{(const float*)du, h.G(tn(k, i, "b")), B, w, w});
+      }
+      fb.end();
+    }
+    fb.begin();
+    fb.optim(h.n_total);
+    fb.end();
+    FusedArgs& a = fp.args;
+    a.phases = h.upload(fb.phases);
+    a.n_phases = (int)fb.phases.size();
+    a.tasks = h.upload(fb.tasks);
+    a.n_tasks = (int)fb.tasks.size();
+    a.gemms = h.upload(fb.gemms);
+    a.n_gemms = (int)fb.gemms.size();
+    a.prefetches = h.upload(fb.prefetches);
+    a.xents = h.upload(fb.xents);
+    a.colsums = h.upload(fb.colsums);
+    a.losses = h.upload(fb.losses);
+    a.labels = h.upload(fb.labels);
+    a.d_losses = h.d_losses;
+    a.status = h.d_status;
+    a.counter = fused_counter;
+    a.x_slot = h.x_in;
+    a.y_slot = h.y_in;
+    fp.flops = fb.flops;
+    fp.ok = true;
+  };
+  double step_flops = 0;
+  {
+    int prev_w = h.spec.d_in;
+    for (int k = 0; k < K; ++k) {
+      for (int w : b.widths[k]) { step_flops += 6.0 * B * w * prev_w; prev_w = w; }
+      step_flops += 6.0 * B * C * prev_w;
+    }
+  }
+  if (!h.bf16_mode && K <= 64 && step_flops <= 4e9) h.fused_blocks = fused_mlp_max_blocks(h.num_sms);
+  if (h.fused_blocks > 0) {
+    fused_counter = (unsigned long long*)h.dalloc(2 * sizeof(unsigned long long));
+    build_fused(h.fused_sync, false, 0, 0);
+    for (int par = 0; par < 2; ++par) build_fused(h.fused_pipe[par], true, par, 1 - par);
+    h.use_fused = true;
+  }
 
   build_step(h.sync_plan, false, 0, 0, false);
   if (K > 1) {

@@ -369,25 +369,28 @@ void emit_argmax(Handle& h, Plan& p, const std::vector<ArgmaxProb>& probs) {
   });
 }
 
+OptimArgs optimizer_args(const Handle& h) {
+  OptimArgs a{};
+  a.master = h.master; a.m1 = h.m1; a.m2 = h.m2; a.grad = h.grad; a.working = h.working;
+  a.n_total = h.n_total; a.n_matrix = h.n_matrix;
+  a.kind = h.opt.kind; a.lr = h.opt.lr; a.momentum = h.opt.momentum; a.weight_decay = h.opt.weight_decay;
+  a.beta1 = h.opt.beta1; a.beta2 = h.opt.beta2; a.eps = h.opt.eps;
+  // all chunks share one step count here (otherwise the per-chunk table below carries theirs)
+  double t = (double)((h.updates.empty() ? h.step_count : h.updates[0]) + 1);
+  a.omb1 = (float)(1.0 - (double)h.opt.beta1);
+  a.omb2 = (float)(1.0 - (double)h.opt.beta2);
+  a.bc1 = (float)(1.0 - pow((double)h.opt.beta1, t));
+  a.bc2 = (float)(1.0 - pow((double)h.opt.beta2, t));
+  if (h.per_chunk_counts) {   // the step driver has filled d_chunk_tab for this step
+    a.seg_end = h.d_seg_end; a.seg_chunk = h.d_seg_chunk; a.n_seg = h.n_seg; a.chunk_tab = h.d_chunk_tab;
+  }
+  return a;
+}
+
 void emit_optimizer(Handle& h, Plan& p) {
   Handle* hp = &h;
-  p.add(1, [hp](const RunCtx& c) {
-    OptimArgs a{};
-    a.master = hp->master; a.m1 = hp->m1; a.m2 = hp->m2; a.grad = hp->grad; a.working = hp->working;
-    a.n_total = hp->n_total; a.n_matrix = hp->n_matrix;
-    a.kind = hp->opt.kind; a.lr = hp->opt.lr; a.momentum = hp->opt.momentum; a.weight_decay = hp->opt.weight_decay;
-    a.beta1 = hp->opt.beta1; a.beta2 = hp->opt.beta2; a.eps = hp->opt.eps;
-    // all chunks share one step count here (otherwise the per-chunk table below carries theirs)
-    double t = (double)((hp->updates.empty() ? hp->step_count : hp->updates[0]) + 1);
-    a.omb1 = (float)(1.0 - (double)hp->opt.beta1);
-    a.omb2 = (float)(1.0 - (double)hp->opt.beta2);
-    a.bc1 = (float)(1.0 - pow((double)hp->opt.beta1, t));
-    a.bc2 = (float)(1.0 - pow((double)hp->opt.beta2, t));
-    if (hp->per_chunk_counts) {   // the step driver has filled d_chunk_tab for this step
-      a.seg_end = hp->d_seg_end; a.seg_chunk = hp->d_seg_chunk; a.n_seg = hp->n_seg; a.chunk_tab = hp->d_chunk_tab;
-    }
-    launch_optim(a, c.stream);
-  }, KIND_OPTIM, (double)h.n_total * (h.opt.kind == LP_OPT_ADAM ? 28.0 : 20.0) + (h.bf16_mode ? 2.0 * h.n_matrix : 0.0));
+  p.add(1, [hp](const RunCtx& c) { launch_optim(optimizer_args(*hp), c.stream); }, KIND_OPTIM,
+        (double)h.n_total * (h.opt.kind == LP_OPT_ADAM ? 28.0 : 20.0) + (h.bf16_mode ? 2.0 * h.n_matrix : 0.0));
 }
 
 void emit_attention(Handle& h, Plan& p, const std::vector<AttnProb>& probs, bool backward) {

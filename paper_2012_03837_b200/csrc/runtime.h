@@ -32,6 +32,8 @@ struct RunCtx {
   std::vector<ProfRecord>* prof;         // non-null: bracket every op with events
   int* out_pred = nullptr;               // lp_evaluate only: per-row predictions [K, rows]
   int* out_correct = nullptr;            // lp_evaluate only: per-chunk count of correct predictions
+  const void* x = nullptr;               // training step: where the caller holds the step's inputs (device), when the
+  const int* y = nullptr;                // step may read them in place; null: the handle's own input buffers
 };
 
 struct PlanOp {
@@ -119,6 +121,11 @@ struct Handle {
   const int* d_seg_chunk = nullptr;
   int n_seg = 0;
   float4* d_chunk_tab = nullptr;
+  // ---- single-launch step of a small fp32 MLP (fused_mlp.cu): the same work as sync_plan / pipe_plan[par]
+  struct FusedProgram { FusedArgs args{}; double flops = 0; bool ok = false; };
+  FusedProgram fused_sync, fused_pipe[2];
+  int fused_blocks = 0;                        // blocks of the cooperative launch; 0: not available for this handle
+  bool use_fused = false;                      // lp_set_fused_step; on by default where available
   int last_launches = 0;
   bool profiling = false;
   std::vector<ProfRecord> prof;
@@ -161,6 +168,7 @@ bool emit_xent_and_loss(Handle& h, Plan& p, std::vector<XentProb> probs, const s
 void emit_xent_from_stats(Handle& h, Plan& p, std::vector<XentStatsProb> probs, const std::vector<int>& chunk_of,
                           const std::vector<float*>* bias_grads);
 void emit_optimizer(Handle& h, Plan& p);
+OptimArgs optimizer_args(const Handle& h);     // the optimizer sweep of the step about to run
 // Causal attention of all problems of a phase in one grouped launch (forward) or two (backward: dQ, then dK and
 // dV).  bf16 takes the tcgen05 kernels unless the handle was created with the FP32-ALU backend.
 void emit_attention(Handle& h, Plan& p, const std::vector<AttnProb>& probs, bool backward);

@@ -19,7 +19,7 @@ def to_abi_layout(name: str, a: np.ndarray) -> np.ndarray:
 
 class GpuModel:
     def __init__(self, cfg: dict, params: dict | None = None, gemm_backend: int = 0, ramp: str = "prime",
-                 overlap: bool = False):
+                 overlap: bool = False, fused: bool | None = None):
         self.cfg = cfg
         m, K, hd, op = lp.specs_from_config(cfg, gemm_backend)
         self._specs = (m, hd, op)
@@ -37,6 +37,8 @@ class GpuModel:
             lp.lp_set_ramp(self.h, lp.LP_RAMP_IDLE)
         if overlap:
             lp.lp_set_overlap(self.h, True)
+        if fused is not None:                       # None: the library's default (single launch where available)
+            lp.lp_set_fused_step(self.h, fused)
 
     def close(self):
         if self.h:
@@ -114,10 +116,10 @@ def tensor_rel_err(a: np.ndarray, b: np.ndarray) -> float:
 
 
 def run_both(cfg: dict, steps: int, gemm_backend: int = 0, params: dict | None = None, ramp: str = "prime",
-             overlap: bool = False):
+             overlap: bool = False, fused: bool | None = None):
     """Run `steps` steps on both sides.  Returns (gpu_losses [steps,K], oracle_losses, gpu model, oracle)."""
     params = params if params is not None else lp_synth.init_params(cfg)
-    gm = GpuModel(cfg, params, gemm_backend, ramp, overlap)
+    gm = GpuModel(cfg, params, gemm_backend, ramp, overlap, fused)
     orc = LocalUpdateOracle(cfg, params, dtype=np.float32, ramp=ramp, overlap=overlap)
     gl, ol = [], []
     for t in range(steps):

@@ -40,16 +40,18 @@ def grad_l2_errors(gm, orc):
     return sorted(out, reverse=True)
 
 
-def check(cfg, steps=10, gemm_backend=0, grads_first=True, w_tol=None, v_tol=None, loss_tol=None):
+def check(cfg, steps=10, gemm_backend=0, grads_first=True, w_tol=None, v_tol=None, loss_tol=None, fused=None):
     from paper_2012_03837_b200 import binding as lp
     dt = cfg["dtype"]
     if grads_first:
-        gl, ol, gm, orc = T.run_both(cfg, 1, gemm_backend)
+        gl, ol, gm, orc = T.run_both(cfg, 1, gemm_backend, fused=fused)
         l2 = grad_l2_errors(gm, orc)
         print("grad l2 err after step 0 (worst):", [(f"{e:.2e}", n) for e, n in l2[:5]])
         gm.close()
         assert l2[0][0] <= G_TOL[(dt, cfg["family"])], l2[:5]
-    gl, ol, gm, orc = T.run_both(cfg, steps, gemm_backend)
+    gl, ol, gm, orc = T.run_both(cfg, steps, gemm_backend, fused=fused)
+    if fused is not None:                                    # one cooperative launch, or the grouped launches
+        assert (lp.lp_last_step_launches(gm.h) == 1) == fused, lp.lp_last_step_launches(gm.h)
     lerr = np.abs(gl - ol) / np.abs(ol)
     werr = T.compare_weights(gm, orc, lp_synth.init_params(cfg))
     gm.close()
@@ -63,12 +65,47 @@ def check(cfg, steps=10, gemm_backend=0, grads_first=True, w_tol=None, v_tol=Non
     assert worst["vector"][0] <= (v_tol or V_TOL[dt]), worst
 
 
-def test_c1_mlp_fp32_full_size():
-    check(lp_synth.config("c1"))
+# The fp32 MLP step exists twice: as one cooperative launch (the default for a network this small) and as grouped
+# launches (what larger networks and the other families use); both are held to the same bounds.
+@pytest.mark.parametrize("fused", [True, False])
+def test_c1_mlp_fp32_full_size(fused):
+    check(lp_synth.config("c1"), fused=fused)
 
 
-def test_mlp_fp32_ragged_pipelined():
-    check(lp_synth.config("c1", batch=70, d_in=33, chunks=[[65], [40, 50], [31]], classes=7, schedule="pipelined"))
+@pytest.mark.parametrize("fused", [True, False])
+def test_mlp_fp32_ragged_pipelined(fused):
+    check(lp_synth.config("c1", batch=70, d_in=33, chunks=[[65], [40, 50], [31]], classes=7, schedule="pipelined"),
+          fused=fused)
+
+
+@pytest.mark.parametrize("schedule", ["sync", "pipelined"])
+def test_mlp_fp32_single_launch_many_tiles_and_classes(schedule):
+    """Sizes that make the single-launch step cut 32x32 tiles, loop over slices of the reduction index (widths
+    above 256) and run softmax rows wider than a warp; Adam with weight-free biases."""
+    cfg = lp_synth.config("c1", batch=200, d_in=300, chunks=[[520, 130], [257], [96, 300]], classes=70, schedule=schedule)
+    cfg["optim"] = dict(kind="adam", lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
+    check(cfg, fused=True)
+
+
+def test_single_launch_step_is_bit_reproducible_and_refused_where_it_does_not_exist():
+    from paper_2012_03837_b200 import binding as lp
+    cfg = lp_synth.config("c1", batch=70, d_in=33, chunks=[[65], [40, 50], [31]], classes=7, schedule="pipelined")
+    outs = []
+    for _ in range(2):
+        gm = T.GpuModel(cfg, fused=True)
+        ls = [gm.step(*lp_synth.minibatch(cfg, t)) for t in range(4)]
+        assert lp.lp_last_step_launches(gm.h) == 1
+        outs.append((np.array(ls), gm.get()))
+        gm.close()
+    assert np.array_equal(outs[0][0], outs[1][0])
+    for n in outs[0][1]:
+        assert np.array_equal(outs[0][1][n], outs[1][1][n]), n
+    gm = T.GpuModel(lp_synth.config("c2", batch=64, d_in=64, chunks=[[64], [64]], classes=16))     # bf16 storage
+    with pytest.raises(lp.LpError) as e:
+        lp.lp_set_fused_step(gm.h, True)
+    assert lp.LP_ERR[e.value.code] == "UNSUPPORTED"
+    lp.lp_set_fused_step(gm.h, False)
+    gm.close()
 
 
 @pytest.mark.parametrize("backend", [1, 0])
@@ -244,11 +281,11 @@ def test_run_to_run_bit_reproducible():
 
 # ------------------------------------------------------------------ idle ramp-up of the pipelined schedule
 
-def check_idle(cfg, steps=10):
+def check_idle(cfg, steps=10, fused=None):
     """Pipelined steps with the idle ramp-up (chunk k waits until the k-th step brings it real data) against the
     oracle run with ramp="idle": the same chunks idle (NaN loss, bit-exact pattern), the others agree."""
     dt = cfg["dtype"]
-    gl, ol, gm, orc = T.run_both(cfg, steps, ramp="idle")
+    gl, ol, gm, orc = T.run_both(cfg, steps, ramp="idle", fused=fused)
     K = gl.shape[1]
     assert np.array_equal(np.isnan(gl), np.isnan(ol)), (gl, ol)
     for t in range(steps):
@@ -264,15 +301,17 @@ def check_idle(cfg, steps=10):
     assert worst["vector"][0] <= V_TOL[dt], worst
 
 
-def test_idle_ramp_up_mlp_fp32():
-    check_idle(lp_synth.config("c1", schedule="pipelined"))
+@pytest.mark.parametrize("fused", [True, False])
+def test_idle_ramp_up_mlp_fp32(fused):
+    check_idle(lp_synth.config("c1", schedule="pipelined"), fused=fused)
 
 
-def test_idle_ramp_up_mlp_fp32_adam():
+@pytest.mark.parametrize("fused", [True, False])
+def test_idle_ramp_up_mlp_fp32_adam(fused):
     """Adam's bias correction follows each chunk's own step count (chunk k has made k fewer updates)."""
     cfg = lp_synth.config("c1", schedule="pipelined", batch=48, d_in=40, chunks=[[64], [48, 56], [32], [72]], classes=6)
     cfg["optim"] = dict(kind="adam", lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8)
-    check_idle(cfg)
+    check_idle(cfg, fused=fused)
 
 
 def test_idle_ramp_up_lm_bf16():
