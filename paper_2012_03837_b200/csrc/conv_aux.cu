@@ -4,6 +4,7 @@
 // convolution is the GEMM  y[M, C_out] = cols[M, kh*kw*C_in] * W[C_out, kh*kw*C_in]^T.
 // blockIdx.y selects the problem.  All reductions have a fixed order.
 #include "common.cuh"
+#include "grid_barrier.cuh"
 
 namespace lp {
 namespace {
@@ -117,11 +118,7 @@ __global__ void __launch_bounds__(256) bn_stat_kernel(const BnStatProb* __restri
 // forward: mean and 1/sqrt(biased variance + eps); backward: dgamma, dbeta.  One warp per channel:
 // lane l sums partial blocks l, l+32, ... in double, then a fixed shuffle tree combines the lanes.
 template <bool BWD>
-__global__ void __launch_bounds__(256) bn_finalize_kernel(const BnFinalProb* __restrict__ probs) {
-  const BnFinalProb p = probs[blockIdx.y];
-  int lane = threadIdx.x & 31;
-  int c = blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (c >= p.C) return;
+__device__ __forceinline__ void bn_finalize_channel(const BnFinalProb& p, int c, int lane) {
   if (!BWD && p.use_running) {                 // evaluation mode: normalise with the running statistics
     if (lane == 0) {
       p.mean[c] = p.run_mean[c];
@@ -135,15 +132,15 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const BnFinalProb* __r
     float va[8], vb[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      va[u] = p.part[(size_t)(k + u * 32) * 2 * p.C + c];
-      vb[u] = p.part[(size_t)(k + u * 32) * 2 * p.C + p.C + c];
+      va[u] = __ldcg(p.part + (size_t)(k + u * 32) * 2 * p.C + c);
+      vb[u] = __ldcg(p.part + (size_t)(k + u * 32) * 2 * p.C + p.C + c);
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) { a += (double)va[u]; b += (double)vb[u]; }
   }
   for (; k < p.nblk; k += 32) {
-    a += (double)p.part[(size_t)k * 2 * p.C + c];
-    b += (double)p.part[(size_t)k * 2 * p.C + p.C + c];
+    a += (double)__ldcg(p.part + (size_t)k * 2 * p.C + c);
+    b += (double)__ldcg(p.part + (size_t)k * 2 * p.C + p.C + c);
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -166,6 +163,12 @@ __global__ void __launch_bounds__(256) bn_finalize_kernel(const BnFinalProb* __r
       p.run_var[c] = (float)((1.0 - m) * (double)p.run_var[c] + m * unb);
     }
   }
+}
+template <bool BWD>
+__global__ void __launch_bounds__(256) bn_finalize_kernel(const BnFinalProb* __restrict__ probs) {
+  const BnFinalProb p = probs[blockIdx.y];
+  const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (c < p.C) bn_finalize_channel<BWD>(p, c, threadIdx.x & 31);
 }
 
 template <typename T, bool BWD>
@@ -289,36 +292,47 @@ __global__ void __launch_bounds__(256) col2im_vec_kernel(const Im2colProb* __res
 
 // Block of 256 threads = (C/8 channel vectors) x (256 / (C/8) row lanes) over the block's rows; the row
 // lanes are summed through shared memory in lane order.  Requires C % 8 == 0 and C/8 <= 256.
-template <bool BWD>
-__global__ void __launch_bounds__(256) bn_stat_vec_kernel(const BnStatProb* __restrict__ probs) {
-  __shared__ float red[256 * 16];
-  const BnStatProb p = probs[blockIdx.z];
+// Thread (tx, ty) of the block adds rows r0 + ty, r0 + ty + ny, ... of its channel vector tx to a / b.
+template <bool BWD, int U>
+__device__ __forceinline__ void bn_stat_vec_accum(const BnStatProb& p, int row_block, float (&a)[8], float (&b)[8]) {
   const int rpb = bn_rows_per_block(p.rows);
-  int r0 = blockIdx.y * rpb;
-  if (r0 >= p.rows) return;
-  int r1 = min(r0 + rpb, p.rows);
+  const int r0 = row_block * rpb;
+  const int r1 = min(r0 + rpb, p.rows);
   const int cv = p.C >> 3, ny = 256 / cv;
   const int tx = threadIdx.x % cv, ty = threadIdx.x / cv;
-  float a[8], b[8];
+  if (ty >= ny) return;
+  const bf16* x = (const bf16*)p.x;
+  float mu[8], rs[8];
+  if (BWD) {
 #pragma unroll
-  for (int t = 0; t < 8; ++t) { a[t] = 0.f; b[t] = 0.f; }
-  if (ty < ny) {
-    const bf16* x = (const bf16*)p.x;
-    float mu[8], rs[8];
-    if (BWD) {
+    for (int t = 0; t < 8; ++t) { mu[t] = p.mean[tx * 8 + t]; rs[t] = p.rstd[tx * 8 + t]; }
+  }
+  // several rows per pass, every load of a pass issued before the first sum (the rows are added in their order)
+  for (int r = r0 + ty; r < r1; r += U * ny) {
+    uint4 xr[U], gr[U], rr[U];
 #pragma unroll
-      for (int t = 0; t < 8; ++t) { mu[t] = p.mean[tx * 8 + t]; rs[t] = p.rstd[tx * 8 + t]; }
+    for (int u = 0; u < U; ++u) {
+      const int ru = r + u * ny;
+      if (ru < r1) {
+        const size_t off = (size_t)ru * p.C + tx * 8;
+        xr[u] = *(const uint4*)(x + off);
+        if (BWD) {
+          gr[u] = *(const uint4*)((const bf16*)p.dy + off);
+          if (p.relu_out) rr[u] = *(const uint4*)((const bf16*)p.relu_out + off);
+        }
+      }
     }
-    for (int r = r0 + ty; r < r1; r += ny) {
-      size_t off = (size_t)r * p.C + tx * 8;
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (r + u * ny >= r1) break;
       float xv[8];
-      unpack8(*(const uint4*)(x + off), xv);
+      unpack8(xr[u], xv);
       if (BWD) {
         float g[8];
-        unpack8(*(const uint4*)((const bf16*)p.dy + off), g);
+        unpack8(gr[u], g);
         if (p.relu_out) {
           float ro[8];
-          unpack8(*(const uint4*)((const bf16*)p.relu_out + off), ro);
+          unpack8(rr[u], ro);
 #pragma unroll
           for (int t = 0; t < 8; ++t) if (!(ro[t] > 0.f)) g[t] = 0.f;
         }
@@ -330,6 +344,11 @@ __global__ void __launch_bounds__(256) bn_stat_vec_kernel(const BnStatProb* __re
       }
     }
   }
+}
+// The block's row lanes summed through shared memory in lane order; row `out_row` of the partial sums [.][2][C].
+__device__ __forceinline__ void bn_stat_vec_reduce(const BnStatProb& p, int out_row, const float (&a)[8], const float (&b)[8],
+                                                   float* red) {   // red: 256 * 16 floats
+  const int cv = p.C >> 3, ny = 256 / cv;
   // red[value][thread]: the 16 partial values of a thread go to 16 different rows, so that a warp's stores, and
   // the loads below (channel vectors of one value and line side by side), touch 32 different banks.
 #pragma unroll
@@ -340,8 +359,19 @@ __global__ void __launch_bounds__(256) bn_stat_vec_kernel(const BnStatProb* __re
     const int j = idx % cv, vt = idx / cv;             // vt = which * 8 + t
     float s = 0.f;
     for (int l = 0; l < ny; ++l) s += red[vt * 256 + l * cv + j];
-    p.part[(size_t)blockIdx.y * 2 * p.C + (vt >> 3) * p.C + j * 8 + (vt & 7)] = s;
+    p.part[(size_t)out_row * 2 * p.C + (vt >> 3) * p.C + j * 8 + (vt & 7)] = s;
   }
+}
+template <bool BWD>
+__global__ void __launch_bounds__(256) bn_stat_vec_kernel(const BnStatProb* __restrict__ probs) {
+  __shared__ float red[256 * 16];
+  const BnStatProb p = probs[blockIdx.z];
+  if ((long long)blockIdx.y * bn_rows_per_block(p.rows) >= p.rows) return;
+  float a[8], b[8];
+#pragma unroll
+  for (int t = 0; t < 8; ++t) { a[t] = 0.f; b[t] = 0.f; }
+  bn_stat_vec_accum<BWD, BWD ? 2 : 4>(p, blockIdx.y, a, b);
+  bn_stat_vec_reduce(p, blockIdx.y, a, b, red);
 }
 
 // dx[n, hw, c] = dy[n, c] / HW, bf16 with C % 8 == 0: eight channels per access
@@ -406,24 +436,22 @@ __global__ void __launch_bounds__(256) gap_fwd_vec_kernel(const GapProb* __restr
 // thirty scalar loads for every 16 bytes of data).  A thread's channel vector is the same in every pass of the
 // grid-stride loop when the stride is a multiple of C / 8 (always so for power-of-two channel counts): it then
 // keeps its constants in registers.
-template <bool BWD>
-__global__ void __launch_bounds__(256, 4) bn_apply_vec_kernel(const BnApplyProb* __restrict__ probs) {
-  __shared__ __align__(16) float cst[4][2048];          // C <= 2048 (C / 8 <= 256)
-  const BnApplyProb p = probs[blockIdx.y];
+// Elements first, first + stride, ... (in 16-byte vectors) of one problem; every thread of the block calls it
+// (the constants are formed by the whole block).
+template <bool BWD, int U>
+__device__ __forceinline__ void bn_apply_vec_range(const BnApplyProb& p, long long first, long long stride, float (*cst)[2048]) {
   const int cv = p.C >> 3;
   const long long total = (long long)p.rows * cv;
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  if ((long long)blockIdx.x * blockDim.x >= total) return;
   const bool fixed = stride % cv == 0;
   const bf16* x = (const bf16*)p.x;
   const float inv = 1.0f / (float)p.rows;
   // forward: y = (x - mu) * ka + kb;  backward: dx = ka * (dyr - kb - (x - mu) * kc)
   for (int c = threadIdx.x; c < p.C; c += 256) {
-    const float rs = p.rstd[c];
-    cst[0][c] = p.mean[c];
+    const float rs = __ldcg(p.rstd + c);
+    cst[0][c] = __ldcg(p.mean + c);
     cst[1][c] = rs * p.g[c];
-    cst[2][c] = BWD ? p.dbeta[c] * inv : p.b[c];
-    cst[3][c] = BWD ? rs * p.dgamma[c] * inv : 0.f;
+    cst[2][c] = BWD ? __ldcg(p.dbeta + c) * inv : p.b[c];
+    cst[3][c] = BWD ? rs * __ldcg(p.dgamma + c) * inv : 0.f;
   }
   __syncthreads();
   float mu[8], ka[8], kb[8], kc[8];
@@ -433,37 +461,175 @@ __global__ void __launch_bounds__(256, 4) bn_apply_vec_kernel(const BnApplyProb*
     *(float4*)&kb[0] = *(const float4*)&cst[2][c0]; *(float4*)&kb[4] = *(const float4*)&cst[2][c0 + 4];
     if (BWD) { *(float4*)&kc[0] = *(const float4*)&cst[3][c0]; *(float4*)&kc[4] = *(const float4*)&cst[3][c0 + 4]; }
   };
-  long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  long long e = first;
   if (fixed && e < total) constants((int)(e % cv) * 8);
-  for (; e < total; e += stride) {
-    if (!fixed) constants((int)(e % cv) * 8);
-    float xv[8], o[8];
-    unpack8(*(const uint4*)(x + e * 8), xv);
-    if (!BWD) {
-      float r[8];
-      if (p.res) unpack8(*(const uint4*)((const bf16*)p.res + e * 8), r);
+  // U vectors per pass, every load of a pass issued before the first store: enough bytes in flight per SM to
+  // cover the memory latency with two or three blocks of 256 threads
+  for (; e < total; e += stride * U) {
+    uint4 xr[U], ar[U], rr[U];
 #pragma unroll
-      for (int t = 0; t < 8; ++t) {
-        float v = (xv[t] - mu[t]) * ka[t] + kb[t];
-        if (p.res) v += r[t];
-        o[t] = p.relu ? relu_f(v) : v;
+    for (int u = 0; u < U; ++u) {
+      const long long eu = e + u * stride;
+      if (eu < total) {
+        xr[u] = *(const uint4*)(x + eu * 8);
+        if (!BWD) {
+          if (p.res) ar[u] = *(const uint4*)((const bf16*)p.res + eu * 8);
+        } else {
+          ar[u] = *(const uint4*)((const bf16*)p.dy + eu * 8);
+          if (p.relu_out) rr[u] = *(const uint4*)((const bf16*)p.relu_out + eu * 8);
+        }
       }
-      *(uint4*)((bf16*)p.y + e * 8) = pack8(o);
-    } else {
-      float g[8];
-      unpack8(*(const uint4*)((const bf16*)p.dy + e * 8), g);
-      if (p.relu_out) {
-        float ro[8];
-        unpack8(*(const uint4*)((const bf16*)p.relu_out + e * 8), ro);
+    }
 #pragma unroll
-        for (int t = 0; t < 8; ++t) if (!(ro[t] > 0.f)) g[t] = 0.f;
+    for (int u = 0; u < U; ++u) {
+      const long long eu = e + u * stride;
+      if (eu >= total) break;
+      if (!fixed) constants((int)(eu % cv) * 8);
+      float xv[8], o[8];
+      unpack8(xr[u], xv);
+      if (!BWD) {
+        float r[8];
+        if (p.res) unpack8(ar[u], r);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          float v = (xv[t] - mu[t]) * ka[t] + kb[t];
+          if (p.res) v += r[t];
+          o[t] = p.relu ? relu_f(v) : v;
+        }
+        *(uint4*)((bf16*)p.y + eu * 8) = pack8(o);
+      } else {
+        float g[8];
+        unpack8(ar[u], g);
+        if (p.relu_out) {
+          float ro[8];
+          unpack8(rr[u], ro);
+#pragma unroll
+          for (int t = 0; t < 8; ++t) if (!(ro[t] > 0.f)) g[t] = 0.f;
+        }
+        if (p.dres_out) *(uint4*)((bf16*)p.dres_out + eu * 8) = pack8(g);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) o[t] = ka[t] * (g[t] - kb[t] - (xv[t] - mu[t]) * kc[t]);
+        *(uint4*)((bf16*)p.dx + eu * 8) = pack8(o);
       }
-      if (p.dres_out) *(uint4*)((bf16*)p.dres_out + e * 8) = pack8(g);
-#pragma unroll
-      for (int t = 0; t < 8; ++t) o[t] = ka[t] * (g[t] - kb[t] - (xv[t] - mu[t]) * kc[t]);
-      *(uint4*)((bf16*)p.dx + e * 8) = pack8(o);
     }
   }
+}
+template <bool BWD>
+__global__ void __launch_bounds__(256, 3) bn_apply_vec_kernel(const BnApplyProb* __restrict__ probs) {
+  __shared__ __align__(16) float cst[4][2048];          // C <= 2048 (C / 8 <= 256)
+  const BnApplyProb p = probs[blockIdx.y];
+  if ((long long)blockIdx.x * blockDim.x >= (long long)p.rows * (p.C >> 3)) return;
+  bn_apply_vec_range<BWD, BWD ? 2 : 4>(p, (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x, cst);
+}
+
+// Per-channel totals of the fused kernel: one block per tile of 8 channels (a 32-byte sector of a row of the
+// partial sums [nrow][2][C]).  Lane (channel cs, row lane rl) of warp w takes rows 4 w + rl, + 32, + 64, ...; both
+// sums of up to 16 rows are in flight at once.  A lane adds its rows in double in row order, then the four row
+// lanes and the eight warps are added in a fixed order.
+template <bool BWD>
+__device__ __forceinline__ void bn_finalize_tile(const BnFinalProb& p, int tile, double (*wsum)[2][8]) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int cs = lane & 7, rl = lane >> 3;
+  const int c = tile * 8 + cs;                 // < C: C is a multiple of 8
+  if (!BWD && p.use_running) {                 // evaluation mode: normalise with the running statistics
+    if (warp == 0 && rl == 0) {
+      p.mean[c] = p.run_mean[c];
+      p.rstd[c] = (float)(1.0 / sqrt((double)p.run_var[c] + (double)p.eps));
+    }
+    return;
+  }
+  constexpr int PER = 16;                      // rows of each sum a lane has in flight at once
+  double sa = 0.0, sb = 0.0;
+  for (int k0 = warp * 4 + rl; k0 < p.nblk; k0 += 32 * PER) {
+    float va[PER], vb[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int k = k0 + 32 * i;
+      va[i] = k < p.nblk ? __ldcg(p.part + (size_t)k * 2 * p.C + c) : 0.0f;
+      vb[i] = k < p.nblk ? __ldcg(p.part + (size_t)k * 2 * p.C + p.C + c) : 0.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < PER; ++i) { sa += (double)va[i]; sb += (double)vb[i]; }
+  }
+  sa += __shfl_xor_sync(0xffffffffu, sa, 8);  sb += __shfl_xor_sync(0xffffffffu, sb, 8);
+  sa += __shfl_xor_sync(0xffffffffu, sa, 16); sb += __shfl_xor_sync(0xffffffffu, sb, 16);
+  if (rl == 0) { wsum[warp][0][cs] = sa; wsum[warp][1][cs] = sb; }
+  __syncthreads();
+  if (warp == 0 && rl == 0) {
+    double a = 0.0, b = 0.0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { a += wsum[w][0][cs]; b += wsum[w][1][cs]; }
+    if (BWD) {
+      p.dgamma[c] = (float)a;
+      p.dbeta[c] = (float)b;
+    } else {
+      double mu = a / p.rows;
+      double var = b / p.rows - mu * mu;
+      if (var < 0.0) var = 0.0;
+      p.mean[c] = (float)mu;
+      p.rstd[c] = (float)(1.0 / sqrt(var + (double)p.eps));
+      if (p.run_mean && !(p.chunk_tab && p.chunk_tab[p.chunk].x == 0.f)) {   // training step: exponential averages
+        const double m = (double)p.momentum, unb = var * ((double)p.rows / (double)(p.rows > 1 ? p.rows - 1 : 1));
+        p.run_mean[c] = (float)((1.0 - m) * (double)p.run_mean[c] + m * mu);
+        p.run_var[c] = (float)((1.0 - m) * (double)p.run_var[c] + m * unb);
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// BatchNorm of a whole launch group in ONE cooperative launch (bf16, C % 8 == 0): the three passes above --
+// partial sums, per-channel totals, normalisation -- separated by grid-wide barriers instead of kernel
+// boundaries.  The tensor the first pass has just pulled through L2 is still there for the third (a 33 MB
+// activation of the first stage is read from HBM once, not twice), two launch latencies go away, and since the
+// blocks are known to be co-resident each of them sums ALL its blocks of rows into one partial row, so the
+// second pass adds a few hundred rows per channel instead of a thousand.  fin.nblk of a problem is the number
+// of partial rows the launch produces for it: min(blocks of rows, blocks of the launch).
+template <bool BWD>
+__global__ void __launch_bounds__(256, BWD ? 2 : 3) bn_fused_kernel(const BnFusedProb* __restrict__ probs, int n, int stats,
+                                                                    unsigned long long* counter, int* status) {
+  __shared__ __align__(16) float buf[4][2048];
+  __shared__ double wsum[8][2][8];
+  constexpr int U = 4;
+  bool alive = true;
+  if (stats) {
+    int item = blockIdx.x;
+    for (int i = 0; i < n; ++i) {                        // (problem, block of rows) pairs, round-robin over the blocks
+      const BnStatProb p = probs[i].st;
+      const int nblk = bn_blocks(p.rows);
+      if (item < nblk) {
+        const int out_row = item;                        // < gridDim.x
+        float a[8], b[8];
+#pragma unroll
+        for (int t = 0; t < 8; ++t) { a[t] = 0.f; b[t] = 0.f; }
+        for (; item < nblk; item += gridDim.x) bn_stat_vec_accum<BWD, U>(p, item, a, b);
+        bn_stat_vec_reduce(p, out_row, a, b, &buf[0][0]);
+        __syncthreads();
+      }
+      item -= nblk;
+    }
+    alive = grid_barrier(counter, (unsigned long long)gridDim.x, status);
+  }
+  if (alive) {
+    int tile = blockIdx.x;
+    for (int i = 0; i < n; ++i) {                        // one block per (problem, tile of 8 channels)
+      const int tiles = probs[i].fin.C >> 3;
+      if (tile < tiles) {
+        const BnFinalProb p = probs[i].fin;
+        for (; tile < tiles; tile += gridDim.x) bn_finalize_tile<BWD>(p, tile, wsum);
+      }
+      tile -= tiles;
+    }
+    alive = grid_barrier(counter, (unsigned long long)(stats ? 2 : 1) * gridDim.x, status);
+  }
+  if (alive) {
+    for (int i = 0; i < n; ++i) {
+      const BnApplyProb p = probs[i].ap;
+      bn_apply_vec_range<BWD, U>(p, (long long)blockIdx.x * blockDim.x + threadIdx.x, (long long)gridDim.x * blockDim.x, buf);
+      __syncthreads();
+    }
+  }
+  grid_barrier_leave(counter);
 }
 
 // ------------------------------------------------------------------ few-channel 3x3 convolution (the stem)
@@ -619,6 +785,23 @@ void launch_bn_apply(const BnApplyProb* d, int n, long long max_elems, bool bwd,
     if (bwd) bn_apply_vec_kernel<true><<<grid, 256, 0, s>>>(d); else bn_apply_vec_kernel<false><<<grid, 256, 0, s>>>(d);
   } else if (is_bf16) { if (bwd) bn_apply_kernel<bf16, true><<<grid, 256, 0, s>>>(d); else bn_apply_kernel<bf16, false><<<grid, 256, 0, s>>>(d); }
   else { if (bwd) bn_apply_kernel<float, true><<<grid, 256, 0, s>>>(d); else bn_apply_kernel<float, false><<<grid, 256, 0, s>>>(d); }
+}
+int bn_fused_max_blocks(int num_sms, bool bwd) {
+  int per_sm = 0;
+  const cudaError_t e = bwd ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bn_fused_kernel<true>, 256, 0)
+                            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, bn_fused_kernel<false>, 256, 0);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return 0;
+  }
+  return num_sms * per_sm;
+}
+cudaError_t launch_bn_fused(const BnFusedProb* d, int n, bool bwd, bool stats, int blocks, unsigned long long* counter,
+                            int* d_status, cudaStream_t s) {
+  int st = stats ? 1 : 0;
+  void* params[] = {(void*)&d, (void*)&n, (void*)&st, (void*)&counter, (void*)&d_status};
+  const void* fn = bwd ? (const void*)bn_fused_kernel<true> : (const void*)bn_fused_kernel<false>;
+  return cudaLaunchCooperativeKernel(fn, dim3(blocks), dim3(256), params, 0, s);
 }
 void launch_gap_fwd(const GapProb* d, int n, int max_n, int max_c, bool is_bf16, cudaStream_t s) {
   dim3 grid((max_c + 255) / 256, max_n, n);

@@ -12,6 +12,7 @@
 #include <algorithm>
 
 #include "common.cuh"
+#include "grid_barrier.cuh"
 #include "optim_update.cuh"
 
 namespace lp {
@@ -19,38 +20,6 @@ namespace {
 
 constexpr int NT = FUSED_THREADS, NW = NT / 32;
 constexpr int SMEM_FLOATS = 10240;         // dynamic shared memory: the staged operands of a tile, later its partial tiles
-constexpr long long BARRIER_LIMIT_NS = 2000000000ll;
-
-__device__ __forceinline__ long long now_ns() {
-  long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// All blocks of the (cooperative, hence co-resident) launch arrive; returns false if the wait was given up, in
-// which case ST_TIMEOUT is raised and every block that sees it leaves the kernel.
-__device__ bool grid_barrier(unsigned long long* counter, unsigned long long target, int* status) {
-  __shared__ int ok;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(counter, 1ull);
-    const long long t0 = now_ns();
-    int good = 1;
-    while (*(volatile unsigned long long*)counter < target) {
-      if ((*(volatile int*)status & ST_TIMEOUT) || now_ns() - t0 > BARRIER_LIMIT_NS) {
-        atomicOr(status, ST_TIMEOUT);
-        good = 0;
-        break;
-      }
-    }
-    __threadfence();
-    ok = good;
-  }
-  __syncthreads();
-  return ok != 0;
-}
-
 // One TM x TN tile of C = epilogue(A B^T).  The sixteen warps form KS groups; group g takes the g-th of KS
 // contiguous pieces of each staged slice of the reduction index, and the NW / KS warps of a group share the rows
 // of the tile among them, each lane owning an RM x RN patch.  The KS partial tiles are added in group order.
@@ -318,16 +287,7 @@ __global__ void __launch_bounds__(NT, 1) fused_mlp_step_kernel(FusedArgs a) {
     }
     if (ph + 1 < a.n_phases) alive = grid_barrier(a.counter, (unsigned long long)(ph + 1) * gridDim.x, a.status);
   }
-  // the last block to leave puts the barrier back to zero for the next launch
-  __syncthreads();
-  if (tid == 0) {
-    __threadfence();
-    if (atomicAdd(a.counter + 1, 1ull) == (unsigned long long)gridDim.x - 1) {
-      a.counter[0] = 0ull;
-      a.counter[1] = 0ull;
-      __threadfence();
-    }
-  }
+  grid_barrier_leave(a.counter);
 }
 
 }  // namespace

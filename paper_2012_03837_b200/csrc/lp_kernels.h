@@ -200,6 +200,9 @@ inline int bn_rows_per_block(long long rows) {
   while (rpb > 32 && rows / rpb < 592) rpb >>= 1;
   return rpb;
 }
+#if defined(__CUDACC__)
+__host__ __device__
+#endif
 inline int bn_blocks(long long rows) { int rpb = bn_rows_per_block(rows); return (int)((rows + rpb - 1) / rpb); }
 // max_blocks: the largest bn_blocks(rows) among the n problems
 void launch_bn_stat_partial(const BnStatProb* d_probs, int n, int max_blocks, int max_c, bool bwd, bool is_bf16,
@@ -223,6 +226,17 @@ struct BnApplyProb {
   int rows, C, relu;
 };
 void launch_bn_apply(const BnApplyProb* d_probs, int n, long long max_elems, bool bwd, bool is_bf16, cudaStream_t s, bool vec8 = false);
+// The three passes of a group of BatchNorms (bf16, C % 8 == 0, C / 8 <= 256 in every problem) as one cooperative
+// launch with bounded grid-wide barriers in between.  Every block of the launch sums all its blocks of rows into
+// ONE row of the partial sums, so fin.nblk must be min(bn_blocks(rows), blocks) -- deterministic, but not the
+// summation order of the separate launches.  stats = false: the statistics pass is left out (evaluation mode: the
+// finalize pass takes the running ones).  blocks = bn_fused_max_blocks(SM count, bwd) (0: the kernel cannot be
+// co-resident; use the separate launches); counter: two zeroed 64-bit words owned by the caller, shared by all
+// launches of one stream.
+struct BnFusedProb { BnStatProb st; BnFinalProb fin; BnApplyProb ap; };
+int bn_fused_max_blocks(int num_sms, bool bwd);
+cudaError_t launch_bn_fused(const BnFusedProb* d_probs, int n, bool bwd, bool stats, int blocks, unsigned long long* counter,
+                            int* d_status, cudaStream_t s);
 
 // 3x3 stride-1 convolution of an image with very few channels (9 * Cin <= 32: the stem of App. B.3's
 // networks, which a 64-deep tensor-core k-slice would leave mostly empty), on the FP32 ALUs with fp32

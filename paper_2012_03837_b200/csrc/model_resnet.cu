@@ -189,6 +189,14 @@ void build_resnet(Handle& h) {
   h.y_bytes = (size_t)B * sizeof(int);
   h.y_in = (int*)h.dalloc(h.y_bytes);
   auto fal = [&](size_t n) { return (float*)h.dalloc(n * sizeof(float)); };
+  if (bf) {
+    h.bn_fused_blocks[0] = bn_fused_max_blocks(h.num_sms, false);
+    h.bn_fused_blocks[1] = bn_fused_max_blocks(h.num_sms, true);
+    h.d_grid_counter = (unsigned long long*)h.dalloc(2 * sizeof(unsigned long long));
+  }
+  const int bn_blocks_fused = h.bn_fused_blocks[0], bn_blocks_fused_bwd = h.bn_fused_blocks[1];
+  unsigned long long* const grid_counter = h.d_grid_counter;
+  int* const d_status = h.d_status;
   // 3x3 (padding 1) and 1x1 convolutions with stride 1 or 2 whose input channel count is a multiple of 64 run
   // as implicit GEMMs: the activation tensor itself is the operand (TMA boxes that step through it with the
   // stride, one shifted box per filter tap), nothing 9 times its size is written.  Forward and filter gradient
@@ -304,6 +312,14 @@ void build_resnet(Handle& h) {
     bool v8 = bf && C % 8 == 0 && C / 8 <= 256;
     long long elems = b.rows * b.C;
     const bool stats = mode != BN_RUNNING;
+    if (v8 && bn_blocks_fused > 0) {                     // the three passes as one cooperative launch
+      BnFinalProb ff = fp;
+      ff.nblk = std::min(nblk, bn_blocks_fused);         // one partial row per block of the launch
+      const BnFusedProb* dfp = h.upload(std::vector<BnFusedProb>{BnFusedProb{sp, ff, ap}});
+      p.add(1, [=](const RunCtx& r) { launch_bn_fused(dfp, 1, false, stats, bn_blocks_fused, grid_counter, d_status, r.stream); },
+            KIND_NORM, (double)elems * es * ((stats ? 3 : 2) + (res ? 1 : 0)));
+      return;
+    }
     p.add(stats ? 3 : 2, [=](const RunCtx& r) {
       if (stats) launch_bn_stat_partial(ds, 1, nblk, C, false, bf, r.stream, v8);
       launch_bn_finalize(df, 1, C, false, r.stream);
@@ -595,6 +611,17 @@ void build_resnet(Handle& h) {
         const BnApplyProb* da = h.upload(ap);
         int n = (int)st.size();
         bool vec = v8 != 0;
+        if (vec && bn_blocks_fused_bwd > 0) {
+          std::vector<BnFusedProb> fu;
+          for (int i = 0; i < n; ++i) {
+            fu.push_back(BnFusedProb{st[i], fi[i], ap[i]});
+            fu.back().fin.nblk = std::min(fi[i].nblk, bn_blocks_fused_bwd);   // one partial row per block of the launch
+          }
+          const BnFusedProb* dfp = h.upload(fu);
+          p.add(1, [=](const RunCtx& r) { launch_bn_fused(dfp, n, true, true, bn_blocks_fused_bwd, grid_counter, d_status, r.stream); },
+                KIND_NORM, work);
+          continue;
+        }
         p.add(3, [=](const RunCtx& r) {
           launch_bn_stat_partial(ds, n, nb, C, true, bf, r.stream, vec);
           launch_bn_finalize(df, n, C, true, r.stream);

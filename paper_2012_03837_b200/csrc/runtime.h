@@ -126,6 +126,10 @@ struct Handle {
   FusedProgram fused_sync, fused_pipe[2];
   int fused_blocks = 0;                        // blocks of the cooperative launch; 0: not available for this handle
   bool use_fused = false;                      // lp_set_fused_step; on by default where available
+  // ---- cooperative launches with grid-wide barriers (grid_barrier.cuh): two zeroed words shared by the launches
+  // of this handle (they run on one stream, one after the other), and the BatchNorm kernel's grid (0: unavailable)
+  unsigned long long* d_grid_counter = nullptr;
+  int bn_fused_blocks[2] = {0, 0};             // forward, backward
   int last_launches = 0;
   bool profiling = false;
   std::vector<ProfRecord> prof;
