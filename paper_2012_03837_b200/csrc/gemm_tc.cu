@@ -26,6 +26,8 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <queue>
+#include <vector>
 #include <cstdio>
 #include <cstdlib>
 
@@ -386,7 +388,7 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
 template <int CG, int W>
 __global__ void __launch_bounds__(NTHREADS, 1)
 gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict__ maps, int nprob, int total_tiles,
-               int* status) {
+               int* status, const int* __restrict__ sched, const int* __restrict__ sched_off) {
   using C = Cfg<CG, W>;
   constexpr int STAGES = C::STAGES, STAGE_BYTES = C::STAGE_BYTES, BNL = C::BNL, TN = C::TN, NB = C::NB,
                 B_SUB_BYTES = C::B_SUB_BYTES;
@@ -398,6 +400,13 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = CG == 2 ? cluster_rank() : 0;          // 0 = the CTA that issues the pair's MMAs
   const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
+  // The tiles of this CTA (pair), in increasing order: every tile_step-th tile of the launch, or -- when the
+  // launch mixes tiles of very different lengths -- the list a host-side balancer made for it (gemm_tc_schedule).
+  // All roles, and both CTAs of a pair, walk the same list.
+  const int my_begin = sched ? sched_off[first_tile] : 0;
+  const int my_count = sched ? sched_off[first_tile + 1] - my_begin
+                             : (first_tile < total_tiles ? (total_tiles - first_tile + tile_step - 1) / tile_step : 0);
+  auto tile_at = [&](int i) { return sched ? sched[my_begin + i] : first_tile + i * tile_step; };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh->full[s], CG); mbar_init(&sh->empty[s], 1); }
@@ -432,19 +441,26 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       bool a_mn = false, b_mn = false;
       int kb_n = 0;
       int conv = 0;
-      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step) {
+      int bnl = BNL;                                 // B rows (columns of the tile) this CTA loads per sub-tile
+      uint32_t stage_tx = STAGE_BYTES;               // bytes a stage receives: less for a narrow tile
+      int tile_next = my_count > 0 ? tile_at(0) : 0;
+      for (int ti = 0; ti < my_count && ok; ++ti) {
+        const int tile = tile_next;
+        if (ti + 1 < my_count) tile_next = tile_at(ti + 1);   // on its way while this tile's loads are issued
         if (cur.seek(tile)) {                        // problem changed: re-read its fields (once per problem, not per tile)
           const GemmProb& p = probs[cur.pi];
           walk.set(p, TILE_M);
           a_mn = p.a_ms == 1; b_mn = p.b_ns == 1;
           kb_n = (p.K + BK - 1) / BK;
           conv = p.conv;
+          bnl = p.tile_n / CG;
+          stage_tx = (uint32_t)(A_BYTES + NB * bnl * BK * 2);
         }
         const CUtensorMap* mapA = maps + 4 * cur.pi;
         const CUtensorMap* mapB = mapA + 1;
         int mt, nt;
         walk.coords(tile, mt, nt);
-        int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * TN + (int)rank * BNL;
+        int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * (TN / BN) * (bnl * CG) + (int)rank * bnl;
         if (conv == CONV_NONE) {
           // ---- ordinary operands: 2-D boxes of the A and B matrices
           for (int kb = 0; kb < kb_n; ++kb) {
@@ -454,7 +470,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
             int k0 = kb * BK;
             if (CG == 1) {
               uint64_t* bar = &sh->full[stage];
-              mbar_expect_tx(bar, STAGE_BYTES);
+              mbar_expect_tx(bar, stage_tx);
               if (a_mn) {
 #pragma unroll
                 for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, bar);
@@ -466,8 +482,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
                 uint8_t* b_sub = b_dst + sb * B_SUB_BYTES;
                 const int ns = n0 + sb * BN;
                 if (b_mn) {
-#pragma unroll
-                  for (int i = 0; i < BNL / 64; ++i) tma_load_2d(b_sub + i * (BK * 128), mapB, ns + i * 64, k0, bar);
+                  for (int i = 0; i < bnl / 64; ++i) tma_load_2d(b_sub + i * (BK * 128), mapB, ns + i * 64, k0, bar);
                 } else {
                   tma_load_2d(b_sub, mapB, k0, ns, bar);
                 }
@@ -475,7 +490,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
             } else {
               // both CTAs' bytes are counted on the leader's barrier
               uint32_t bar = map_to_rank(smem_u32(&sh->full[stage]), 0);
-              mbar_expect_tx_cluster(bar, STAGE_BYTES);
+              mbar_expect_tx_cluster(bar, stage_tx);
               if (a_mn) {
 #pragma unroll
                 for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0, bar);
@@ -487,8 +502,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
                 uint8_t* b_sub = b_dst + sb * B_SUB_BYTES;
                 const int ns = n0 + sb * BN;
                 if (b_mn) {
-#pragma unroll
-                  for (int i = 0; i < BNL / 64; ++i) tma_load_2d_pair(b_sub + i * (BK * 128), mapB, ns + i * 64, k0, bar);
+                  for (int i = 0; i < bnl / 64; ++i) tma_load_2d_pair(b_sub + i * (BK * 128), mapB, ns + i * 64, k0, bar);
                 } else {
                   tma_load_2d_pair(b_sub, mapB, k0, ns, bar);
                 }
@@ -515,8 +529,8 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
           int k0 = kb * BK;
           uint64_t* bar1 = &sh->full[stage];
           uint32_t bar2 = 0;
-          if (CG == 1) mbar_expect_tx(bar1, STAGE_BYTES);
-          else { bar2 = map_to_rank(smem_u32(bar1), 0); mbar_expect_tx_cluster(bar2, STAGE_BYTES); }
+          if (CG == 1) mbar_expect_tx(bar1, stage_tx);
+          else { bar2 = map_to_rank(smem_u32(bar1), 0); mbar_expect_tx_cluster(bar2, stage_tx); }
           auto ld2 = [&](void* dst, const CUtensorMap* map, int x, int y) {
             if (CG == 1) tma_load_2d(dst, map, x, y, bar1); else tma_load_2d_pair(dst, map, x, y, bar2);
           };
@@ -530,8 +544,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
             for (int i = 0; i < BM / 64; ++i) ld2(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0);
             const int kp = cv_k0 + k0;
             const int img = kp / cv_hw, h0 = (kp - img * cv_hw) / cv_w;
-#pragma unroll
-            for (int i = 0; i < BNL / 64; ++i) {
+            for (int i = 0; i < bnl / 64; ++i) {
               const int col = n0 + i * 64;
               const int t = col / cv_c, c0 = col - t * cv_c;
               if (t < cv_taps) ld4(b_dst + i * (BK * 128), mapB, c0, tap_dj(t), h0 * cv_s + tap_di(t), img);
@@ -547,8 +560,7 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
               ld2(b_dst, mapB, k0, n0);                  // filters [N, 9 conv_c], reduction index contiguous
             } else {
               // filters [conv_c, 3, 3, N] read in place: rows = output channel (the reduction), columns (tap, n)
-#pragma unroll
-              for (int i = 0; i < BNL / 64; ++i) ld2(b_dst + i * (BK * 128), mapB, tap * p_n + n0 + i * 64, ch0);
+              for (int i = 0; i < bnl / 64; ++i) ld2(b_dst + i * (BK * 128), mapB, tap * p_n + n0 + i * 64, ch0);
             }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
@@ -572,13 +584,16 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       bool a_mn = false, b_mn = false;
       int kb_n = 0;
       uint32_t idesc = 0;
-      for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
+      int tile_next = my_count > 0 ? tile_at(0) : 0;
+      for (; it < my_count && ok; ++it) {
+        const int tile = tile_next;
+        if (it + 1 < my_count) tile_next = tile_at(it + 1);
         if (cur.seek(tile)) {
           const GemmProb& p = probs[cur.pi];
           a_mn = p.a_ms == 1; b_mn = p.b_ns == 1;
           kb_n = (p.K + BK - 1) / BK;
           idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-                  ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+                  ((uint32_t)(p.tile_n >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
         }
         // wide tiles own both accumulators (barrier set 0); otherwise the two alternate from tile to tile
         int ab = W ? 0 : (it & 1);
@@ -620,13 +635,16 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
     bool ok = true;
     ProbCursor cur(probs, nprob);
     TileWalk walk;
-    for (int tile = first_tile; tile < total_tiles && ok; tile += tile_step, ++it) {
+    int tile_next = my_count > 0 ? tile_at(0) : 0;
+    for (; it < my_count && ok; ++it) {
+      const int tile = tile_next;
+      if (it + 1 < my_count) tile_next = tile_at(it + 1);
       if (cur.seek(tile)) walk.set(probs[cur.pi], TILE_M);
       const int pi = cur.pi;
       const GemmProb p = probs[pi];          // read-only table: fields are fetched where they are used
       int mt, nt;
       walk.coords(tile, mt, nt);
-      int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * TN;
+      int m0 = mt * TILE_M + (int)rank * BM, n0 = nt * (TN / BN) * p.tile_n;
       int ab = W ? 0 : (it & 1);
       uint32_t use = W ? (uint32_t)it : (uint32_t)(it >> 1);
       // Each thread owns one accumulator row and walks this warp's half of the columns 32 at a time;
@@ -634,6 +652,9 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
       // (residual or activation-derivative operand) are in flight while the current block is stored.
       const int m = m0 + quarter * 32 + lane;
       const int col0 = ((warp - EPI_FIRST) >> 2) * (TN / 2);
+      // 32-column blocks of this warp's half that the tile has: all of them, or for a narrow tile (one MMA of
+      // 64 or 128 columns) those of the first half only; always an even number
+      const int nblk32 = W ? TN / 64 : max(0, min(TN / 2, p.tile_n - col0)) >> 5;
       const bool vec_ok = (p.ldc % 8 == 0) && (((uintptr_t)p.C & 15) == 0) && (!p.C2 || ((uintptr_t)p.C2 & 15) == 0) &&
                           (!p.resid || ((uintptr_t)p.resid & 15) == 0) && (!p.aux || ((uintptr_t)p.aux & 15) == 0);
       const void* side = (p.resid && !p.aux) ? p.resid : (p.aux && !p.resid) ? p.aux : nullptr;
@@ -669,15 +690,15 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
         else epilogue_row32<false>(p, mapC, mapC + 1, stg, m, m_warp0, nc, a, lane, c, run, nullptr, nullptr);
       };
       uint32_t acc0[32], acc1[32];
-      tc_ld32(trow, acc0);
+      if (nblk32 > 0) tc_ld32(trow, acc0);
 #pragma unroll 1
-      for (int c = 0; c < TN / 64; c += 2) {
+      for (int c = 0; c < nblk32; c += 2) {
         tc_wait_ld();
         tc_ld32(trow + (c + 1) * 32, acc1);
         fetch_side(side1, c + 1);
         emit(acc0, c, side0);
         tc_wait_ld();
-        if (c + 2 < TN / 64) { tc_ld32(trow + (c + 2) * 32, acc0); fetch_side(side0, c + 2); }
+        if (c + 2 < nblk32) { tc_ld32(trow + (c + 2) * 32, acc0); fetch_side(side0, c + 2); }
         emit(acc1, c + 1, side1);
       }
       if (p.act == EPI_LOGIT_STATS && m < p.M && n0 + col0 < p.N)
@@ -792,7 +813,18 @@ bool gemm_tc_wide_ok(const GemmProb& g) {
 
 int gemm_tc_tiles(GemmProb& g, int tile_start, int cg, int wide) {
   g.tile_start = tile_start;
-  g.tiles_n = (g.N + (wide ? 2 : 1) * BN - 1) / ((wide ? 2 : 1) * BN);
+  // A problem with at most 128 columns (the 64- and 128-channel convolutions of the early ResNet stages) gets
+  // one column tile of 64 or 128 instead of 256: the MMA, the B boxes and the accumulator read-back shrink with
+  // it.  Every CTA must still receive whole boxes: 64 columns where B arrives in 64-column blocks (MN-major B,
+  // the implicit input and filter gradients), 32 rows otherwise.
+  g.tile_n = BN;
+  if (!wide && g.act != EPI_LOGIT_STATS && g.conv != CONV_WGRAD) {
+    const bool blocks64 = g.conv == CONV_NONE ? g.b_ns == 1 : g.conv != CONV_FWD;
+    const int unit = (blocks64 ? 64 : 32) * cg;
+    if (g.N <= 64 && unit <= 64) g.tile_n = 64;
+    else if (g.N <= 128 && unit <= 128) g.tile_n = 128;
+  }
+  g.tiles_n = (g.N + (wide ? 2 : 1) * g.tile_n - 1) / ((wide ? 2 : 1) * g.tile_n);
   // band height: at least 8 row tiles, more while the band's row panels (tile rows x K) stay within ~32 MB of L2
   const long long panel = (long long)BM * cg * g.K * 2;
   g.raster = (int)std::max(8LL, std::min(4096LL, (32LL << 20) / std::max(panel, 1LL)));
@@ -841,12 +873,49 @@ bool gemm_tc_encode(GemmProb& g, void* maps, int cg) {
   if (g.conv == CONV_WGRAD) okB = encode_map4(mapB, g.B, g.conv_n, g.conv_h, g.conv_w, g.conv_c, BK, chin, cwin, cs);
   else if (g.conv == CONV_DGRAD) okB = encode_map(mapB, g.B, 9LL * g.N, g.conv_c, 9LL * g.N, BK);   // rows: output channel
   else if (g.b_ns == 1) okB = encode_map(mapB, g.B, g.N, g.K, g.b_ks, BK);
-  else okB = encode_map(mapB, g.B, g.K, g.N, g.b_ns, BN / cg);
+  else okB = encode_map(mapB, g.B, g.K, g.N, g.b_ns, (g.tile_n ? g.tile_n : BN) / cg);
   return okA && okB;
 }
 
+int gemm_tc_grid_units(int total_tiles, int num_sms, int cg) {
+  const int units = cg == 1 ? num_sms : num_sms / 2;
+  return total_tiles < units ? total_tiles : units;
+}
+
+// Longest-processing-time assignment of the launch's tiles to its CTAs (pairs).  A tile costs its k-slices plus a
+// few for the epilogue.  Tiles are taken in index order (the caller lists long problems first) and each goes to
+// the least loaded unit, the lowest index among equals: for tiles of one length this is exactly the round-robin
+// walk of the kernel, so a uniform launch needs no schedule and gets none.
+bool gemm_tc_schedule(const GemmProb* probs, int nprob, int total_tiles, int num_sms, int cg, std::vector<int>& sched,
+                      std::vector<int>& off) {
+  sched.clear(); off.clear();
+  const int units = gemm_tc_grid_units(total_tiles, num_sms, cg);
+  if (nprob < 2 || units < 1 || total_tiles <= units) return false;
+  std::vector<int> cost(total_tiles);
+  int lo = 1 << 30, hi = 0;
+  for (int i = 0; i < nprob; ++i) {
+    const int end = i + 1 < nprob ? probs[i + 1].tile_start : total_tiles;
+    const int c = (probs[i].K + BK - 1) / BK + 4;
+    for (int t = probs[i].tile_start; t < end; ++t) cost[t] = c;
+    if (end > probs[i].tile_start) { lo = std::min(lo, c); hi = std::max(hi, c); }
+  }
+  if (hi <= lo + lo / 4) return false;                 // lengths within 25 %: the round-robin walk is as good
+  std::vector<std::vector<int>> lists(units);
+  typedef std::pair<long long, int> Load;                // (load, unit): smallest load first, lowest unit among equals
+  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> q;
+  for (int u = 0; u < units; ++u) q.push(Load(0, u));
+  for (int t = 0; t < total_tiles; ++t) {
+    Load l = q.top(); q.pop();
+    lists[l.second].push_back(t);
+    q.push(Load(l.first + cost[t], l.second));
+  }
+  off.push_back(0);
+  for (auto& l : lists) { sched.insert(sched.end(), l.begin(), l.end()); off.push_back((int)sched.size()); }
+  return true;
+}
+
 cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int nprob, int total_tiles, int* d_status,
-                           int num_sms, cudaStream_t s, int cg, int wide) {
+                           int num_sms, cudaStream_t s, int cg, int wide, const int* d_sched, const int* d_sched_off) {
   // function attributes belong to a device's context: set once per device and variant
   static bool attr_set_dev[64][4] = {};
   int dev = 0;
@@ -871,12 +940,12 @@ cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int npro
   }
   if (total_tiles == 0) return cudaSuccess;
   if (cg == 1) {
-    int grid = total_tiles < num_sms ? total_tiles : num_sms;
-    gemm_tc_kernel<1, 0><<<grid, NTHREADS, smem, s>>>(d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
+    int grid = gemm_tc_grid_units(total_tiles, num_sms, 1);
+    gemm_tc_kernel<1, 0><<<grid, NTHREADS, smem, s>>>(d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status,
+                                                      d_sched, d_sched_off);
     return cudaGetLastError();
   }
-  int pairs = num_sms / 2;
-  if (total_tiles < pairs) pairs = total_tiles;
+  int pairs = gemm_tc_grid_units(total_tiles, num_sms, 2);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
   cfg.blockDim = dim3(NTHREADS);
@@ -889,8 +958,10 @@ cudaError_t launch_gemm_tc(const GemmProb* d_probs, const void* d_maps, int npro
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (wide) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 1>, d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 0>, d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status);
+  if (wide) return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 1>, d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status,
+                                      d_sched, d_sched_off);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<2, 0>, d_probs, (const CUtensorMap*)d_maps, nprob, total_tiles, d_status,
+                            d_sched, d_sched_off);
 }
 
 }  // namespace lp

@@ -40,6 +40,7 @@ struct GemmProb {
   int out_f32;
   int tile_start;  // first tile index of this problem in the launch (filled by the launcher)
   int tiles_n;
+  int tile_n;      // tensor-core kernel: columns of a tile and of its MMA, 64 / 128 / 256 (set by the launcher)
   int store_tma;   // tensor-core kernel: outputs leave through TMA stores (set by the launcher when C's pitch allows)
   int raster;      // tensor-core kernel: row tiles per band of the tile walk (set by the launcher)
   // Implicit convolution over NHWC activations (tensor-core kernel only; App. B.3's residual blocks): 3x3 with

@@ -177,7 +177,11 @@ void emit_gemm(Handle& h, Plan& p, std::vector<GemmProb> probs) {
     int sms = h.num_sms;
     double fl = 0;
     for (auto& g : list) fl += 2.0 * g.M * g.N * g.K;
-    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream, cg, wide); }, KIND_GEMM_TC, fl);
+    // tiles of very different lengths in one launch: a balanced assignment to the CTAs, made once here
+    std::vector<int> sched, off;
+    const int *dsched = nullptr, *doff = nullptr;
+    if (gemm_tc_schedule(list.data(), n, total, sms, cg, sched, off)) { dsched = h.upload(sched); doff = h.upload(off); }
+    p.add(1, [=](const RunCtx& c) { launch_gemm_tc(d, dm, n, total, st, sms, c.stream, cg, wide, dsched, doff); }, KIND_GEMM_TC, fl);
   }
   if (!simt.empty()) {
     int t = 0;

@@ -48,7 +48,10 @@ def check(t, ref, tag):
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 128), (200, 264, 72), (1000, 520, 328), (136, 1000, 2048),
                                    # long reductions with 512-column outputs: the 256x512 tiles (input gradient over
                                    # 8192 columns; weight gradient over 8200 rows, ragged last k-slice)
-                                   (264, 8192, 512), (8200, 512, 1024)])
+                                   (264, 8192, 512), (8200, 512, 1024),
+                                   # at most 128 output columns: column tiles of 64 and 128 (K-major B in 32-row boxes
+                                   # per CTA of a pair; MN-major B in 64-column blocks), ragged in both directions
+                                   (520, 64, 192), (300, 128, 64), (136, 96, 256), (1000, 40, 136)])
 def test_linear_products(M, N, K, backend):
     rng = np.random.default_rng(M + N + K)
     t, descs, ref = problems(M, N, K, rng)
