@@ -633,110 +633,166 @@ __global__ void __launch_bounds__(256, BWD ? 2 : 3) bn_fused_kernel(const BnFuse
 }
 
 // ------------------------------------------------------------------ few-channel 3x3 convolution (the stem)
-// Forward: Cout / 8 threads per pixel, 8 output channels each; filters transposed to [k][Cout] in shared
-// memory (a pixel's threads read consecutive 32-byte pieces, threads of different pixels the same ones).
+// Both kernels stage, for a group of consecutive pixels, the 9 * Cin input values around each pixel (zero outside
+// the image) in shared memory as fp32, padded to 32 per pixel, and work on register tiles from there: a thread
+// re-reads from shared memory one value per four to eight multiply-adds instead of one per multiply-add.
+constexpr int SC_KP = 32;                             // staged reduction length per pixel: 9 * Cin <= 32, zero padded
+
+// patch[pl][k] for pixels base .. base + NPIX - 1 (k = tap * Cin + c), row pitch SC_KP + 4 floats.  blockDim.x / NPIX
+// threads share a pixel; each stages the same SC_KP / (threads per pixel) values of k for every pixel it meets, so
+// the tap offsets of those k are worked out once (StageTaps) and a pixel's coordinates once per thread and group:
+// no division per staged value.
+template <int NPIX>
+struct StageTaps {
+  static constexpr int TPP = 256 / NPIX, KPER = SC_KP / TPP;
+  int pl, k0;
+  signed char dh[KPER], dw[KPER], c[KPER];            // c < 0: k beyond 9 * Cin (stays zero)
+  __device__ __forceinline__ void init(int Cin) {
+    pl = threadIdx.x / TPP; k0 = (threadIdx.x % TPP) * KPER;
+#pragma unroll
+    for (int j = 0; j < KPER; ++j) {
+      const int k = k0 + j, tap = k / Cin;
+      dh[j] = (signed char)(tap / 3 - 1); dw[j] = (signed char)(tap % 3 - 1);
+      c[j] = (signed char)(k < 9 * Cin ? k - tap * Cin : -1);
+    }
+  }
+};
+template <typename T, int NPIX>
+__device__ __forceinline__ void stage_patch(const SmallConvProb& p, const StageTaps<NPIX>& st, long long base, long long total,
+                                            float* patch) {
+  const T* x = (const T*)p.x;
+  const int pix = (int)base + st.pl;                   // the pixel count of a problem is below 2^31 (checked by the launchers)
+  const bool in = pix < total;
+  const int row = in ? pix / p.W : 0;
+  const int w0 = in ? pix - row * p.W : 0;
+  const int h0 = row % p.H;
+  const T* img = x + (size_t)(row - h0) * p.W * p.Cin;   // first pixel of the image
+  float* dst = patch + st.pl * (SC_KP + 4) + st.k0;
+#pragma unroll
+  for (int j = 0; j < StageTaps<NPIX>::KPER; ++j) {
+    const int hh = h0 + st.dh[j], ww = w0 + st.dw[j];
+    float v = 0.f;
+    if (in && st.c[j] >= 0 && hh >= 0 && hh < p.H && ww >= 0 && ww < p.W) v = to_f(img[((size_t)hh * p.W + ww) * p.Cin + st.c[j]]);
+    dst[j] = v;
+  }
+}
+
+// Forward: a block of 256 threads takes groups of 64 pixels; thread (pixel pair, group of 8 output channels)
+// holds 2 x 8 sums.  Filters transposed to [k][Cout] in shared memory once per block.
+constexpr int SCF_PIX = 64;
 template <typename T, typename WT>
 __global__ void __launch_bounds__(256) small_conv_fwd_kernel(SmallConvProb p) {
-  extern __shared__ float ws[];                       // [9 * Cin][Cout]
+  extern __shared__ __align__(16) float sc_smem[];    // [9 * Cin][Cout] filters, then [SCF_PIX][SC_KP + 4] patch
   const int K = 9 * p.Cin;
+  float* ws = sc_smem;
+  float* patch = sc_smem + K * p.Cout;
   for (int i = threadIdx.x; i < K * p.Cout; i += blockDim.x) {
     int co = i / K, k = i - co * K;
     ws[k * p.Cout + co] = to_f(((const WT*)p.w)[i]);
   }
-  __syncthreads();
-  const int groups = p.Cout >> 3, ppb = blockDim.x / groups;
-  const int g = threadIdx.x % groups, pl = threadIdx.x / groups;
+  const int groups = p.Cout >> 3;                     // threads per pixel pair
+  const int pairs = blockDim.x / groups;              // pixel pairs a pass of the block covers
+  const int g = threadIdx.x % groups, pp = threadIdx.x / groups;
   const long long total = (long long)p.N * p.H * p.W;
-  if (pl >= ppb) return;
-  // a block keeps the filters for several groups of pixels
-  for (long long grp = blockIdx.x; grp * ppb < total; grp += gridDim.x) {
-  const long long pix = grp * ppb + pl;
-  if (pix >= total) continue;
-  const int w0 = (int)(pix % p.W), h0 = (int)((pix / p.W) % p.H);
-  const long long img = pix / ((long long)p.W * p.H);
-  float acc[8];
+  StageTaps<SCF_PIX> taps;
+  taps.init(p.Cin);
+  for (long long base = (long long)blockIdx.x * SCF_PIX; base < total; base += (long long)gridDim.x * SCF_PIX) {
+    __syncthreads();                                  // filters staged / the previous group's patch has been read
+    stage_patch<T, SCF_PIX>(p, taps, base, total, patch);
+    __syncthreads();
+    for (int q = pp; q < SCF_PIX / 2; q += pairs) {
+      const float* x0 = patch + (2 * q) * (SC_KP + 4);
+      const float* x1 = x0 + (SC_KP + 4);
+      float a0[8], a1[8];
 #pragma unroll
-  for (int t = 0; t < 8; ++t) acc[t] = 0.f;
-  const T* x = (const T*)p.x;
-  for (int i = 0; i < 3; ++i) {
-    const int hh = h0 + i - 1;
-    if (hh < 0 || hh >= p.H) continue;
-    for (int j = 0; j < 3; ++j) {
-      const int ww = w0 + j - 1;
-      if (ww < 0 || ww >= p.W) continue;
-      const T* xp = x + ((img * p.H + hh) * p.W + ww) * p.Cin;
-      for (int c = 0; c < p.Cin; ++c) {
-        const float xv = to_f(xp[c]);
-        const float4* wr = (const float4*)(ws + ((i * 3 + j) * p.Cin + c) * p.Cout + g * 8);
-        const float4 w0v = wr[0], w1v = wr[1];
-        acc[0] = fmaf(xv, w0v.x, acc[0]); acc[1] = fmaf(xv, w0v.y, acc[1]); acc[2] = fmaf(xv, w0v.z, acc[2]); acc[3] = fmaf(xv, w0v.w, acc[3]);
-        acc[4] = fmaf(xv, w1v.x, acc[4]); acc[5] = fmaf(xv, w1v.y, acc[5]); acc[6] = fmaf(xv, w1v.z, acc[6]); acc[7] = fmaf(xv, w1v.w, acc[7]);
+      for (int t = 0; t < 8; ++t) { a0[t] = 0.f; a1[t] = 0.f; }
+      for (int k = 0; k < K; ++k) {
+        const float4* wr = (const float4*)(ws + k * p.Cout + g * 8);
+        const float4 w0 = wr[0], w1 = wr[1];
+        const float u = x0[k], v = x1[k];
+        a0[0] = fmaf(u, w0.x, a0[0]); a0[1] = fmaf(u, w0.y, a0[1]); a0[2] = fmaf(u, w0.z, a0[2]); a0[3] = fmaf(u, w0.w, a0[3]);
+        a0[4] = fmaf(u, w1.x, a0[4]); a0[5] = fmaf(u, w1.y, a0[5]); a0[6] = fmaf(u, w1.z, a0[6]); a0[7] = fmaf(u, w1.w, a0[7]);
+        a1[0] = fmaf(v, w0.x, a1[0]); a1[1] = fmaf(v, w0.y, a1[1]); a1[2] = fmaf(v, w0.z, a1[2]); a1[3] = fmaf(v, w0.w, a1[3]);
+        a1[4] = fmaf(v, w1.x, a1[4]); a1[5] = fmaf(v, w1.y, a1[5]); a1[6] = fmaf(v, w1.z, a1[6]); a1[7] = fmaf(v, w1.w, a1[7]);
+      }
+#pragma unroll
+      for (int h2 = 0; h2 < 2; ++h2) {
+        const long long pix = base + 2 * q + h2;
+        if (pix >= total) continue;
+        const float* a = h2 ? a1 : a0;
+        T* y = (T*)p.y + pix * p.Cout + g * 8;
+        if (sizeof(T) == 2) {
+          *(uint4*)y = pack8(a);                      // Cout % 8 == 0: 16-byte aligned
+        } else {
+#pragma unroll
+          for (int t = 0; t < 8; ++t) y[t] = from_f<T>(a[t]);
+        }
       }
     }
-  }
-  T* y = (T*)p.y + pix * p.Cout + g * 8;
-  if (sizeof(T) == 2) {
-    *(uint4*)y = pack8(acc);                            // Cout % 8 == 0: 16-byte aligned
-  } else {
-#pragma unroll
-    for (int t = 0; t < 8; ++t) y[t] = from_f<T>(acc[t]);
-  }
   }
 }
 
-// Filter gradient: thread (co, part) owns the taps/channels k = part, part + parts, ... of output channel co
-// (parts = 256 / Cout); a block walks its pixels in groups of 32 staged in shared memory: the 9*Cin input
-// values around each pixel and its Cout output gradients.
+// Filter gradient: part[blk][co * 9 Cin + k] = sum over block blk's SMALLCONV_PIXELS pixels of dy[pixel, co] *
+// patch[pixel, k].  Thread (pixel lane, group of 8 k, group of 4 output channels) holds 4 x 8 sums over the pixels
+// of its lane (pixel index mod lanes) of each staged group of 32; the lanes are added in lane order at the end.
 template <typename T>
 __global__ void __launch_bounds__(256) small_conv_wgrad_kernel(SmallConvProb p) {
-  __shared__ float patch[32][33];
-  extern __shared__ float dys[];                      // [32][Cout]
-  const int K = 9 * p.Cin, parts = blockDim.x / p.Cout;
-  const int co = threadIdx.x % p.Cout, part = threadIdx.x / p.Cout;
+  extern __shared__ __align__(16) float sc_smem[];    // [32][SC_KP + 4] patch, [32][Cout] dy; later [lanes][Cout * 32] sums
+  const int K = 9 * p.Cin;
+  float* patch = sc_smem;
+  float* dys = sc_smem + 32 * (SC_KP + 4);
+  const int cgroups = p.Cout >> 2;                    // threads along the output channels
+  const int per_lane = cgroups * (SC_KP / 8);         // threads of one pixel lane
+  const int lanes = blockDim.x / per_lane;            // 256 / (Cout): 4 for Cout = 64
+  const int lane_q = threadIdx.x / per_lane, r = threadIdx.x % per_lane;
+  const int kq = r / cgroups, c4 = r % cgroups;
   const long long total = (long long)p.N * p.H * p.W;
   const long long p0 = (long long)blockIdx.x * SMALLCONV_PIXELS;
-  float acc[8];                                       // ceil(32 / parts) <= 8 for parts >= 4
+  float acc[4][8];
 #pragma unroll
-  for (int t = 0; t < 8; ++t) acc[t] = 0.f;
-  const T* x = (const T*)p.x;
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
   const T* dy = (const T*)p.dy;
+  StageTaps<32> taps;
+  taps.init(p.Cin);
   for (long long base = p0; base < p0 + SMALLCONV_PIXELS && base < total; base += 32) {
     __syncthreads();
-    for (int i = threadIdx.x; i < 32 * K; i += blockDim.x) {
-      const int pl = i / K, k = i - pl * K;
-      const long long pix = base + pl;
-      float v = 0.f;
-      if (pix < total) {
-        const int tap = k / p.Cin, c = k - tap * p.Cin;
-        const int ww = (int)(pix % p.W) + tap % 3 - 1, hh = (int)((pix / p.W) % p.H) + tap / 3 - 1;
-        if (hh >= 0 && hh < p.H && ww >= 0 && ww < p.W)
-          v = to_f(x[((pix / ((long long)p.W * p.H) * p.H + hh) * p.W + ww) * p.Cin + c]);
-      }
-      patch[pl][k] = v;
-    }
+    stage_patch<T, 32>(p, taps, base, total, patch);
     for (int i = threadIdx.x; i < 32 * p.Cout; i += blockDim.x) {
       const long long pix = base + i / p.Cout;
       dys[i] = pix < total ? to_f(dy[pix * p.Cout + i % p.Cout]) : 0.f;
     }
     __syncthreads();
-    if (part < parts) {
-      for (int pl = 0; pl < 32; ++pl) {
-        const float d = dys[pl * p.Cout + co];
+    if (lane_q < lanes) {
+      for (int pl = lane_q; pl < 32; pl += lanes) {
+        const float4 d = *(const float4*)(dys + pl * p.Cout + c4 * 4);
+        const float4 u0 = *(const float4*)(patch + pl * (SC_KP + 4) + kq * 8);
+        const float4 u1 = *(const float4*)(patch + pl * (SC_KP + 4) + kq * 8 + 4);
+        const float dv[4] = {d.x, d.y, d.z, d.w};
+        const float uv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-          const int k = part + t * parts;
-          if (k < K) acc[t] = fmaf(d, patch[pl][k], acc[t]);
-        }
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(dv[i], uv[j], acc[i][j]);
       }
     }
   }
-  if (part < parts) {
-    float* out = p.part + (size_t)blockIdx.x * p.Cout * K + (size_t)co * K;
+  __syncthreads();
+  float* red = sc_smem;                               // [lanes][Cout][32]
+  if (lane_q < lanes) {
 #pragma unroll
-    for (int t = 0; t < 8; ++t) {
-      const int k = part + t * parts;
-      if (k < K) out[k] = acc[t];
-    }
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) red[(lane_q * p.Cout + c4 * 4 + i) * SC_KP + kq * 8 + j] = acc[i][j];
+  }
+  __syncthreads();
+  float* out = p.part + (size_t)blockIdx.x * p.Cout * K;
+  for (int o = threadIdx.x; o < p.Cout * K; o += blockDim.x) {
+    const int co = o / K, k = o - co * K;
+    float sum = 0.f;
+    for (int l = 0; l < lanes; ++l) sum += red[(l * p.Cout + co) * SC_KP + k];
+    out[o] = sum;
   }
 }
 
@@ -809,11 +865,11 @@ void launch_gap_fwd(const GapProb* d, int n, int max_n, int max_c, bool is_bf16,
   else gap_fwd_kernel<float><<<grid, 256, 0, s>>>(d);
 }
 void launch_small_conv_fwd(const SmallConvProb& p, bool w_is_bf16, bool is_bf16, cudaStream_t s) {
-  const int groups = p.Cout / 8, ppb = 256 / groups;
   const long long total = (long long)p.N * p.H * p.W;
-  long long groups_of_pixels = (total + ppb - 1) / ppb;
-  const unsigned grid = (unsigned)(groups_of_pixels < 148 * 8 ? groups_of_pixels : 148 * 8);
-  const size_t smem = (size_t)9 * p.Cin * p.Cout * sizeof(float);
+  if (total >= (1LL << 31) - 64) return;               // the builder does not choose these kernels for such an input
+  long long groups = (total + SCF_PIX - 1) / SCF_PIX;
+  const unsigned grid = (unsigned)std::min<long long>(groups, 148LL * 8);
+  const size_t smem = ((size_t)9 * p.Cin * p.Cout + (size_t)SCF_PIX * (SC_KP + 4)) * sizeof(float);
   if (is_bf16) {
     if (w_is_bf16) small_conv_fwd_kernel<bf16, bf16><<<grid, 256, smem, s>>>(p);
     else small_conv_fwd_kernel<bf16, float><<<grid, 256, smem, s>>>(p);
@@ -823,8 +879,11 @@ void launch_small_conv_fwd(const SmallConvProb& p, bool w_is_bf16, bool is_bf16,
 }
 void launch_small_conv_wgrad(const SmallConvProb& p, bool is_bf16, cudaStream_t s) {
   const long long total = (long long)p.N * p.H * p.W;
+  if (total >= (1LL << 31) - 64) return;
   const unsigned grid = (unsigned)((total + SMALLCONV_PIXELS - 1) / SMALLCONV_PIXELS);
-  const size_t smem = (size_t)32 * p.Cout * sizeof(float);
+  const int lanes = 256 / ((p.Cout / 4) * (SC_KP / 8));
+  const size_t stage = (size_t)32 * (SC_KP + 4) + (size_t)32 * p.Cout, red = (size_t)lanes * p.Cout * SC_KP;
+  const size_t smem = std::max(stage, red) * sizeof(float);
   if (is_bf16) small_conv_wgrad_kernel<bf16><<<grid, 256, smem, s>>>(p);
   else small_conv_wgrad_kernel<float><<<grid, 256, smem, s>>>(p);
 }

@@ -885,7 +885,8 @@ int gemm_tc_grid_units(int total_tiles, int num_sms, int cg) {
 // Longest-processing-time assignment of the launch's tiles to its CTAs (pairs).  A tile costs its k-slices plus a
 // few for the epilogue.  Tiles are taken in index order (the caller lists long problems first) and each goes to
 // the least loaded unit, the lowest index among equals: for tiles of one length this is exactly the round-robin
-// walk of the kernel, so a uniform launch needs no schedule and gets none.
+// walk of the kernel, so a uniform launch needs no schedule and gets none; nor does a launch whose busiest unit
+// would gain less than a tenth.
 bool gemm_tc_schedule(const GemmProb* probs, int nprob, int total_tiles, int num_sms, int cg, std::vector<int>& sched,
                       std::vector<int>& off) {
   sched.clear(); off.clear();
@@ -900,6 +901,10 @@ bool gemm_tc_schedule(const GemmProb* probs, int nprob, int total_tiles, int num
     if (end > probs[i].tile_start) { lo = std::min(lo, c); hi = std::max(hi, c); }
   }
   if (hi <= lo + lo / 4) return false;                 // lengths within 25 %: the round-robin walk is as good
+  // what the kernel's own walk (unit u takes tiles u, u + units, ...) would make the busiest unit do
+  std::vector<long long> rr(units, 0);
+  for (int t = 0; t < total_tiles; ++t) rr[t % units] += cost[t];
+  const long long rr_max = *std::max_element(rr.begin(), rr.end());
   std::vector<std::vector<int>> lists(units);
   typedef std::pair<long long, int> Load;                // (load, unit): smallest load first, lowest unit among equals
   std::priority_queue<Load, std::vector<Load>, std::greater<Load>> q;
@@ -909,6 +914,9 @@ bool gemm_tc_schedule(const GemmProb* probs, int nprob, int total_tiles, int num
     lists[l.second].push_back(t);
     q.push(Load(l.first + cost[t], l.second));
   }
+  long long lpt_max = 0;
+  while (!q.empty()) { lpt_max = std::max(lpt_max, q.top().first); q.pop(); }
+  if (lpt_max * 10 > rr_max * 9) return false;          // less than a tenth to gain: keep the walk (and its L2 locality)
   off.push_back(0);
   for (auto& l : lists) { sched.insert(sched.end(), l.begin(), l.end()); off.push_back((int)sched.size()); }
   return true;

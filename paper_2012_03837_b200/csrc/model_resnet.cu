@@ -233,7 +233,7 @@ void build_resnet(Handle& h) {
     if (c.has_stem) {
       c.x_nhwc = h.dalloc(in_elems * es);
       c.stem.small = c.stem.k == 3 && c.stem.stride == 1 && 9 * c.stem.Cin <= 32 && c.stem.Cout % 8 == 0 &&
-                     c.stem.Cout <= 64 && 256 % c.stem.Cout == 0;
+                     c.stem.Cout <= 64 && 256 % c.stem.Cout == 0 && c.stem.M < (1LL << 30);
       alloc_conv(c.stem); alloc_bn(c.stem_bn); track(c.stem);
       c.stem_out = h.dalloc((size_t)c.stem.M * c.stem.Cout * es);
     }
@@ -362,24 +362,40 @@ void build_resnet(Handle& h) {
     }
   };
 
-  auto head_forward = [&](Plan& p, int k, int wr, const int* labels, bool copy_logits, int mode) {
-    Chunk& c = ch[k];
-    const std::string ck = "c" + std::to_string(k);
-    if (head_bn) bn_fwd(p, c.head_bn, h.bnd[wr][k], c.hact, nullptr, true, mode);
-    GapProb gp{head_bn ? c.hact : h.bnd[wr][k], c.pool, nullptr, nullptr, B, c.Hout * c.Wout, c.C};
-    const GapProb* dg = h.upload(std::vector<GapProb>{gp});
-    int C = c.C;
-    p.add(1, [=](const RunCtx& r) { launch_gap_fwd(dg, 1, B, C, bf, r.stream); }, KIND_CONV_AUX, (double)B * c.Hout * c.Wout * c.C * es);
-    emit_gemm(h, p, {gemm_fwd(c.pool, h.W(ck + ".head.W"), c.z, B, NC, c.C, h.P32(ck + ".head.b"), EPI_NONE)});
-    if (copy_logits && k == K - 1) {
-      void* zlast = c.z;
+  // The heads of all chunks (Sec. 3: each reads only its own chunk's output): one grouped launch per step of the
+  // head -- spatial means, logits, predictions (evaluation), cross-entropy and losses.
+  auto heads_forward = [&](Plan& p, int wr, const std::function<const int*(int)>& labels, bool copy_logits, int mode) {
+    std::vector<GapProb> gaps;
+    std::vector<GemmProb> logits;
+    std::vector<ArgmaxProb> am;
+    std::vector<XentProb> xs;
+    std::vector<int> all_chunks;
+    double gap_bytes = 0;
+    int gap_c = 0;
+    for (int k = 0; k < K; ++k) {
+      Chunk& c = ch[k];
+      const std::string ck = "c" + std::to_string(k);
+      if (head_bn) bn_fwd(p, c.head_bn, h.bnd[wr][k], c.hact, nullptr, true, mode);
+      gaps.push_back(GapProb{head_bn ? c.hact : h.bnd[wr][k], c.pool, nullptr, nullptr, B, c.Hout * c.Wout, c.C});
+      gap_bytes += (double)B * c.Hout * c.Wout * c.C * es;
+      gap_c = std::max(gap_c, c.C);
+      logits.push_back(gemm_fwd(c.pool, h.W(ck + ".head.W"), c.z, B, NC, c.C, h.P32(ck + ".head.b"), EPI_NONE));
+      am.push_back(ArgmaxProb{c.z, labels(k), B, NC, NC, k});
+      xs.push_back(XentProb{c.z, labels(k), h.n_valid[k], c.row_loss, B, NC, NC, nullptr});
+      all_chunks.push_back(k);
+    }
+    const GapProb* dg = h.upload(gaps);
+    p.add(1, [=](const RunCtx& r) { launch_gap_fwd(dg, K, B, gap_c, bf, r.stream); }, KIND_CONV_AUX, gap_bytes);
+    emit_gemm(h, p, logits);
+    if (copy_logits) {
+      void* zlast = ch[K - 1].z;
       size_t zbytes = (size_t)B * NC * es;
       p.add(0, [zlast, zbytes](const RunCtx& r) {
         if (r.out_logits) cudaMemcpyAsync(r.out_logits, zlast, zbytes, cudaMemcpyDeviceToDevice, r.stream);
       });
+      emit_argmax(h, p, am);
     }
-    if (copy_logits) emit_argmax(h, p, {ArgmaxProb{c.z, labels, B, NC, NC, k}});
-    emit_xent_and_loss(h, p, {XentProb{c.z, labels, h.n_valid[k], c.row_loss, B, NC, NC, nullptr}}, {k});
+    emit_xent_and_loss(h, p, xs, all_chunks);
   };
 
   // ---- backward, recorded per chunk and emitted in lockstep
@@ -646,7 +662,7 @@ void build_resnet(Handle& h) {
       lps.push_back(LabelProb{labels_of(k, pipelined, rd), (pipelined && k < K - 1) ? h.lab[wr][k] : nullptr, B, NC, h.n_valid[k]});
     emit_labels(h, p, lps);
     for (int k = 0; k < K; ++k) forward_chunk(p, k, rd, wr, BN_TRAIN);
-    for (int k = 0; k < K; ++k) head_forward(p, k, wr, labels_of(k, pipelined, rd), false, BN_TRAIN);
+    heads_forward(p, wr, [&](int k) { return labels_of(k, pipelined, rd); }, false, BN_TRAIN);
     std::vector<OpList> lists(K);
     overlap_avg.clear();
     for (int k = 0; k < K; ++k) record_backward(lists[k], k, rd, wr, overlap);
@@ -669,7 +685,7 @@ void build_resnet(Handle& h) {
     std::vector<LabelProb> lps;
     for (int k = 0; k < K; ++k) lps.push_back(LabelProb{h.y_in, nullptr, B, NC, h.n_valid[k]});
     emit_labels(h, p, lps);
-    for (int k = 0; k < K; ++k) head_forward(p, k, wr, h.y_in, true, mode);
+    heads_forward(p, wr, [&](int) { return (const int*)h.y_in; }, true, mode);
   };
 
   h.has_eval_plan = true;
