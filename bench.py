@@ -67,11 +67,11 @@ def describe(cfg, world=1):
 # capture summarised under profiles/ and scaled to the launches of a full step.  A figure is only
 # valid for the kernel source it was captured on: it is dropped when that file has changed since.
 TRAFFIC = {
-    # per chunk (ncu): head products 1.95 GB (forward 0.56, input gradient 0.61 and weight gradient 0.77 on the
-    # 256x512 tiles), block products 0.77 GB; every chunk streams its own operands, so a 24-chunk step moves
-    # 24 x 2.72 GB = 65 GB over its thirteen GEMM launches
+    # per chunk (ncu): head products 1.95 GB (forward 0.57, input gradient 0.61 and weight gradient 0.77 on the
+    # 256x512 tiles), block products 0.76 GB; every chunk streams its own operands, so a 24-chunk step moves
+    # 24 x 2.71 GB = 65 GB over its thirteen GEMM launches
     "c5": dict(bytes_per_launch=5.0e9, chunks=24, kernel_file="paper_2012_03837_b200/csrc/gemm_tc.cu",
-               kernel_sha256="297e441f4f44da6405351899d1b9ac3f3e38f2c6dc30d61729045443ce7d9930"),
+               kernel_sha256="81aead8e0c8b6843a85a1c65735b723708c596eae43919f2823f6cb3ac48cf67"),
 }
 
 

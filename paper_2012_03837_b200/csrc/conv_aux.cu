@@ -735,17 +735,18 @@ __global__ void __launch_bounds__(256) small_conv_fwd_kernel(SmallConvProb p) {
 // Filter gradient: part[blk][co * 9 Cin + k] = sum over block blk's SMALLCONV_PIXELS pixels of dy[pixel, co] *
 // patch[pixel, k].  Thread (pixel lane, group of 8 k, group of 4 output channels) holds 4 x 8 sums over the pixels
 // of its lane (pixel index mod lanes) of each staged group of 32; the lanes are added in lane order at the end.
-template <typename T>
+// COUT is a template parameter (8, 16, 32 or 64): every index computation is a shift and the loops unroll.
+template <typename T, int COUT>
 __global__ void __launch_bounds__(256) small_conv_wgrad_kernel(SmallConvProb p) {
-  extern __shared__ __align__(16) float sc_smem[];    // [32][SC_KP + 4] patch, [32][Cout] dy; later [lanes][Cout * 32] sums
+  extern __shared__ __align__(16) float sc_smem[];    // [32][SC_KP + 4] patch, [32][COUT] dy; later [lanes][COUT * 32] sums
   const int K = 9 * p.Cin;
   float* patch = sc_smem;
   float* dys = sc_smem + 32 * (SC_KP + 4);
-  const int cgroups = p.Cout >> 2;                    // threads along the output channels
-  const int per_lane = cgroups * (SC_KP / 8);         // threads of one pixel lane
-  const int lanes = blockDim.x / per_lane;            // 256 / (Cout): 4 for Cout = 64
-  const int lane_q = threadIdx.x / per_lane, r = threadIdx.x % per_lane;
-  const int kq = r / cgroups, c4 = r % cgroups;
+  constexpr int CG4 = COUT / 4;                       // threads along the output channels
+  constexpr int PER_LANE = CG4 * (SC_KP / 8);         // threads of one pixel lane
+  constexpr int LANES = 256 / PER_LANE;               // 4 for COUT = 64
+  const int lane_q = threadIdx.x / PER_LANE, r = threadIdx.x % PER_LANE;
+  const int kq = r / CG4, c4 = r % CG4;
   const long long total = (long long)p.N * p.H * p.W;
   const long long p0 = (long long)blockIdx.x * SMALLCONV_PIXELS;
   float acc[4][8];
@@ -759,39 +760,53 @@ __global__ void __launch_bounds__(256) small_conv_wgrad_kernel(SmallConvProb p) 
   for (long long base = p0; base < p0 + SMALLCONV_PIXELS && base < total; base += 32) {
     __syncthreads();
     stage_patch<T, 32>(p, taps, base, total, patch);
-    for (int i = threadIdx.x; i < 32 * p.Cout; i += blockDim.x) {
-      const long long pix = base + i / p.Cout;
-      dys[i] = pix < total ? to_f(dy[pix * p.Cout + i % p.Cout]) : 0.f;
+    // the 32 x COUT output gradients of the group are contiguous in memory: eight values per thread
+    for (int i8 = threadIdx.x; i8 < 32 * COUT / 8; i8 += 256) {
+      const long long pix = base + (i8 * 8) / COUT;
+      float v[8];
+      if (pix < total) {
+        if (sizeof(T) == 2) {
+          unpack8(*(const uint4*)((const bf16*)p.dy + (size_t)base * COUT + i8 * 8), v);
+        } else {
+#pragma unroll
+          for (int t = 0; t < 8; ++t) v[t] = to_f(dy[(size_t)base * COUT + i8 * 8 + t]);
+        }
+      } else {
+#pragma unroll
+        for (int t = 0; t < 8; ++t) v[t] = 0.f;
+      }
+      *(float4*)(dys + i8 * 8) = make_float4(v[0], v[1], v[2], v[3]);
+      *(float4*)(dys + i8 * 8 + 4) = make_float4(v[4], v[5], v[6], v[7]);
     }
     __syncthreads();
-    if (lane_q < lanes) {
-      for (int pl = lane_q; pl < 32; pl += lanes) {
-        const float4 d = *(const float4*)(dys + pl * p.Cout + c4 * 4);
-        const float4 u0 = *(const float4*)(patch + pl * (SC_KP + 4) + kq * 8);
-        const float4 u1 = *(const float4*)(patch + pl * (SC_KP + 4) + kq * 8 + 4);
-        const float dv[4] = {d.x, d.y, d.z, d.w};
-        const float uv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+    for (int pl = lane_q; pl < 32; pl += LANES) {
+      const float4 d = *(const float4*)(dys + pl * COUT + c4 * 4);
+      const float4 u0 = *(const float4*)(patch + pl * (SC_KP + 4) + kq * 8);
+      const float4 u1 = *(const float4*)(patch + pl * (SC_KP + 4) + kq * 8 + 4);
+      const float dv[4] = {d.x, d.y, d.z, d.w};
+      const float uv[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
 #pragma unroll
-          for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(dv[i], uv[j], acc[i][j]);
-      }
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(dv[i], uv[j], acc[i][j]);
     }
   }
   __syncthreads();
-  float* red = sc_smem;                               // [lanes][Cout][32]
-  if (lane_q < lanes) {
+  float* red = sc_smem;                               // [LANES][COUT][32]
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int j = 0; j < 8; ++j) red[(lane_q * p.Cout + c4 * 4 + i) * SC_KP + kq * 8 + j] = acc[i][j];
+  for (int i = 0; i < 4; ++i) {
+    float* dst = red + (lane_q * COUT + c4 * 4 + i) * SC_KP + kq * 8;
+    *(float4*)dst = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    *(float4*)(dst + 4) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
   }
   __syncthreads();
-  float* out = p.part + (size_t)blockIdx.x * p.Cout * K;
-  for (int o = threadIdx.x; o < p.Cout * K; o += blockDim.x) {
+  float* out = p.part + (size_t)blockIdx.x * COUT * K;
+  for (int o = threadIdx.x; o < COUT * K; o += blockDim.x) {
     const int co = o / K, k = o - co * K;
     float sum = 0.f;
-    for (int l = 0; l < lanes; ++l) sum += red[(l * p.Cout + co) * SC_KP + k];
+#pragma unroll
+    for (int l = 0; l < LANES; ++l) sum += red[(l * COUT + co) * SC_KP + k];
     out[o] = sum;
   }
 }
@@ -884,8 +899,19 @@ void launch_small_conv_wgrad(const SmallConvProb& p, bool is_bf16, cudaStream_t 
   const int lanes = 256 / ((p.Cout / 4) * (SC_KP / 8));
   const size_t stage = (size_t)32 * (SC_KP + 4) + (size_t)32 * p.Cout, red = (size_t)lanes * p.Cout * SC_KP;
   const size_t smem = std::max(stage, red) * sizeof(float);
-  if (is_bf16) small_conv_wgrad_kernel<bf16><<<grid, 256, smem, s>>>(p);
-  else small_conv_wgrad_kernel<float><<<grid, 256, smem, s>>>(p);
+#define LP_WGRAD(CO)                                                                      \
+  do {                                                                                    \
+    if (is_bf16) small_conv_wgrad_kernel<bf16, CO><<<grid, 256, smem, s>>>(p);            \
+    else small_conv_wgrad_kernel<float, CO><<<grid, 256, smem, s>>>(p);                   \
+  } while (0)
+  switch (p.Cout) {
+    case 8: LP_WGRAD(8); break;
+    case 16: LP_WGRAD(16); break;
+    case 32: LP_WGRAD(32); break;
+    case 64: LP_WGRAD(64); break;
+    default: break;                                      // the builder chooses these kernels for these widths only
+  }
+#undef LP_WGRAD
 }
 void launch_gap_bwd(const GapProb* d, int n, long long max_elems, bool is_bf16, cudaStream_t s, bool vec8) {
   if (vec8 && is_bf16) {
