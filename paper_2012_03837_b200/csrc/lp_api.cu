@@ -197,12 +197,13 @@ int run_fused(Handle& h, const Handle::FusedProgram& fp, const RunCtx& c) {
     cudaEventCreate(&r.e1);
     cudaEventRecord(r.e0, c.stream);
   }
-  launch_fused_mlp_step(a, h.fused_blocks, c.stream);
+  const bool launched = launch_fused_mlp_step(a, h.fused_blocks, c.stream) == cudaSuccess;
+  if (!launched) cudaGetLastError();          // the device cannot hold the cooperative grid right now
   if (c.prof) {
     cudaEventRecord(r.e1, c.stream);
     c.prof->push_back(r);
   }
-  return 1;
+  return launched ? 1 : 0;
 }
 
 lp_status run_step(Handle& h, int schedule, cudaStream_t s, const void* x = nullptr, const int* y = nullptr) {
@@ -214,9 +215,12 @@ lp_status run_step(Handle& h, int schedule, cudaStream_t s, const void* x = null
   const bool any_idle = prepare_chunks(h, schedule, s, active);
   if (schedule == LP_SYNC) {
     if (h.primed) return fail(&h, LP_ERR_STATE, "a pipeline is in flight: call lp_reset_pipeline before a synchronous step");
-    if (fused) {
-      launches = run_fused(h, h.fused_sync, ctx);
-    } else {
+    if (fused) launches = run_fused(h, h.fused_sync, ctx);
+    if (fused && launches == 0) {               // refused: the grouped launches do the same step
+      if (ctx.x) { copy_inputs(h, ctx.x, ctx.y, cudaMemcpyDeviceToDevice, s); ctx.x = nullptr; ctx.y = nullptr; }
+      h.sync_plan.run(ctx);
+      launches = h.sync_plan.launches;
+    } else if (!fused) {
       const Plan& plan = h.overlap ? h.sync_overlap_plan : h.sync_plan;
       plan.run(ctx);
       launches = plan.launches;
@@ -231,9 +235,11 @@ lp_status run_step(Handle& h, int schedule, cudaStream_t s, const void* x = null
     // Idle chunks run through the plan as well, on whatever their boundary buffer holds (finite values:
     // zeros after lp_create); the optimizer leaves their parameters alone, their losses read NaN, and
     // what they publish is overwritten before an active chunk reads it.
-    if (fused) {
-      launches += run_fused(h, h.fused_pipe[h.parity], ctx);          // masks the idle chunks' losses itself
-    } else {
+    int fused_done = 0;
+    if (fused) fused_done = run_fused(h, h.fused_pipe[h.parity], ctx);   // masks the idle chunks' losses itself
+    launches += fused_done;
+    if (fused && fused_done == 0 && ctx.x) { copy_inputs(h, ctx.x, ctx.y, cudaMemcpyDeviceToDevice, s); ctx.x = nullptr; ctx.y = nullptr; }
+    if (!fused || fused_done == 0) {
       h.pipe_plan[h.parity].run(ctx);
       launches += h.pipe_plan[h.parity].launches;
       if (any_idle) { launch_mask_losses(h.d_losses, h.d_chunk_tab, h.K, s); launches += 1; }

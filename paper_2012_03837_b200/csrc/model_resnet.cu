@@ -316,8 +316,15 @@ void build_resnet(Handle& h) {
       BnFinalProb ff = fp;
       ff.nblk = std::min(nblk, bn_blocks_fused);         // one partial row per block of the launch
       const BnFusedProb* dfp = h.upload(std::vector<BnFusedProb>{BnFusedProb{sp, ff, ap}});
-      p.add(1, [=](const RunCtx& r) { launch_bn_fused(dfp, 1, false, stats, bn_blocks_fused, grid_counter, d_status, r.stream); },
-            KIND_NORM, (double)elems * es * ((stats ? 3 : 2) + (res ? 1 : 0)));
+      // (should the cooperative launch be refused -- the device cannot hold the grid right now -- the three
+      // separate launches do the same work; their partial sums use one row per block of rows)
+      p.add(1, [=](const RunCtx& r) {
+        if (launch_bn_fused(dfp, 1, false, stats, bn_blocks_fused, grid_counter, d_status, r.stream) == cudaSuccess) return;
+        cudaGetLastError();
+        if (stats) launch_bn_stat_partial(ds, 1, nblk, C, false, bf, r.stream, v8);
+        launch_bn_finalize(df, 1, C, false, r.stream);
+        launch_bn_apply(da, 1, elems, false, bf, r.stream, v8);
+      }, KIND_NORM, (double)elems * es * ((stats ? 3 : 2) + (res ? 1 : 0)));
       return;
     }
     p.add(stats ? 3 : 2, [=](const RunCtx& r) {
@@ -634,8 +641,13 @@ void build_resnet(Handle& h) {
             fu.back().fin.nblk = std::min(fi[i].nblk, bn_blocks_fused_bwd);   // one partial row per block of the launch
           }
           const BnFusedProb* dfp = h.upload(fu);
-          p.add(1, [=](const RunCtx& r) { launch_bn_fused(dfp, n, true, true, bn_blocks_fused_bwd, grid_counter, d_status, r.stream); },
-                KIND_NORM, work);
+          p.add(1, [=](const RunCtx& r) {
+            if (launch_bn_fused(dfp, n, true, true, bn_blocks_fused_bwd, grid_counter, d_status, r.stream) == cudaSuccess) return;
+            cudaGetLastError();
+            launch_bn_stat_partial(ds, n, nb, C, true, bf, r.stream, vec);
+            launch_bn_finalize(df, n, C, true, r.stream);
+            launch_bn_apply(da, n, elems, true, bf, r.stream, vec);
+          }, KIND_NORM, work);
           continue;
         }
         p.add(3, [=](const RunCtx& r) {
