@@ -678,21 +678,22 @@ __device__ __forceinline__ void stage_patch(const SmallConvProb& p, const StageT
 }
 
 // Forward: a block of 256 threads takes groups of 64 pixels; thread (pixel pair, group of 8 output channels)
-// holds 2 x 8 sums.  Filters transposed to [k][Cout] in shared memory once per block.
+// holds 2 x 8 sums.  Filters transposed to [k][COUT] in shared memory once per block.  COUT is a template
+// parameter (8, 16, 32 or 64): the index computations are shifts and the pair loop has a fixed trip count.
 constexpr int SCF_PIX = 64;
-template <typename T, typename WT>
+template <typename T, typename WT, int COUT>
 __global__ void __launch_bounds__(256) small_conv_fwd_kernel(SmallConvProb p) {
-  extern __shared__ __align__(16) float sc_smem[];    // [9 * Cin][Cout] filters, then [SCF_PIX][SC_KP + 4] patch
+  extern __shared__ __align__(16) float sc_smem[];    // [9 * Cin][COUT] filters, then [SCF_PIX][SC_KP + 4] patch
   const int K = 9 * p.Cin;
   float* ws = sc_smem;
-  float* patch = sc_smem + K * p.Cout;
-  for (int i = threadIdx.x; i < K * p.Cout; i += blockDim.x) {
+  float* patch = sc_smem + K * COUT;
+  for (int i = threadIdx.x; i < K * COUT; i += blockDim.x) {
     int co = i / K, k = i - co * K;
-    ws[k * p.Cout + co] = to_f(((const WT*)p.w)[i]);
+    ws[k * COUT + co] = to_f(((const WT*)p.w)[i]);
   }
-  const int groups = p.Cout >> 3;                     // threads per pixel pair
-  const int pairs = blockDim.x / groups;              // pixel pairs a pass of the block covers
-  const int g = threadIdx.x % groups, pp = threadIdx.x / groups;
+  constexpr int GROUPS = COUT / 8;                    // threads per pixel pair
+  constexpr int PAIRS = 256 / GROUPS;                 // pixel pairs a pass of the block covers
+  const int g = threadIdx.x % GROUPS, pp = threadIdx.x / GROUPS;
   const long long total = (long long)p.N * p.H * p.W;
   StageTaps<SCF_PIX> taps;
   taps.init(p.Cin);
@@ -700,29 +701,38 @@ __global__ void __launch_bounds__(256) small_conv_fwd_kernel(SmallConvProb p) {
     __syncthreads();                                  // filters staged / the previous group's patch has been read
     stage_patch<T, SCF_PIX>(p, taps, base, total, patch);
     __syncthreads();
-    for (int q = pp; q < SCF_PIX / 2; q += pairs) {
+#pragma unroll
+    for (int q0 = 0; q0 < SCF_PIX / 2; q0 += PAIRS) {
+      const int q = q0 + pp;
+      if (q >= SCF_PIX / 2) break;
       const float* x0 = patch + (2 * q) * (SC_KP + 4);
       const float* x1 = x0 + (SC_KP + 4);
       float a0[8], a1[8];
 #pragma unroll
       for (int t = 0; t < 8; ++t) { a0[t] = 0.f; a1[t] = 0.f; }
-      for (int k = 0; k < K; ++k) {
-        const float4* wr = (const float4*)(ws + k * p.Cout + g * 8);
-        const float4 w0 = wr[0], w1 = wr[1];
-        const float u = x0[k], v = x1[k];
-        a0[0] = fmaf(u, w0.x, a0[0]); a0[1] = fmaf(u, w0.y, a0[1]); a0[2] = fmaf(u, w0.z, a0[2]); a0[3] = fmaf(u, w0.w, a0[3]);
-        a0[4] = fmaf(u, w1.x, a0[4]); a0[5] = fmaf(u, w1.y, a0[5]); a0[6] = fmaf(u, w1.z, a0[6]); a0[7] = fmaf(u, w1.w, a0[7]);
-        a1[0] = fmaf(v, w0.x, a1[0]); a1[1] = fmaf(v, w0.y, a1[1]); a1[2] = fmaf(v, w0.z, a1[2]); a1[3] = fmaf(v, w0.w, a1[3]);
-        a1[4] = fmaf(v, w1.x, a1[4]); a1[5] = fmaf(v, w1.y, a1[5]); a1[6] = fmaf(v, w1.z, a1[6]); a1[7] = fmaf(v, w1.w, a1[7]);
+      for (int k4 = 0; k4 < K; k4 += 4) {             // the patch is zero beyond K, the filter rows are not read there
+        const float4 u4 = *(const float4*)(x0 + k4), v4 = *(const float4*)(x1 + k4);
+        const float uu[4] = {u4.x, u4.y, u4.z, u4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (k4 + j >= K) break;
+          const float4* wr = (const float4*)(ws + (k4 + j) * COUT + g * 8);
+          const float4 w0 = wr[0], w1 = wr[1];
+          const float u = uu[j], v = vv[j];
+          a0[0] = fmaf(u, w0.x, a0[0]); a0[1] = fmaf(u, w0.y, a0[1]); a0[2] = fmaf(u, w0.z, a0[2]); a0[3] = fmaf(u, w0.w, a0[3]);
+          a0[4] = fmaf(u, w1.x, a0[4]); a0[5] = fmaf(u, w1.y, a0[5]); a0[6] = fmaf(u, w1.z, a0[6]); a0[7] = fmaf(u, w1.w, a0[7]);
+          a1[0] = fmaf(v, w0.x, a1[0]); a1[1] = fmaf(v, w0.y, a1[1]); a1[2] = fmaf(v, w0.z, a1[2]); a1[3] = fmaf(v, w0.w, a1[3]);
+          a1[4] = fmaf(v, w1.x, a1[4]); a1[5] = fmaf(v, w1.y, a1[5]); a1[6] = fmaf(v, w1.z, a1[6]); a1[7] = fmaf(v, w1.w, a1[7]);
+        }
       }
 #pragma unroll
       for (int h2 = 0; h2 < 2; ++h2) {
         const long long pix = base + 2 * q + h2;
         if (pix >= total) continue;
         const float* a = h2 ? a1 : a0;
-        T* y = (T*)p.y + pix * p.Cout + g * 8;
+        T* y = (T*)p.y + pix * COUT + g * 8;
         if (sizeof(T) == 2) {
-          *(uint4*)y = pack8(a);                      // Cout % 8 == 0: 16-byte aligned
+          *(uint4*)y = pack8(a);                      // COUT % 8 == 0: 16-byte aligned
         } else {
 #pragma unroll
           for (int t = 0; t < 8; ++t) y[t] = from_f<T>(a[t]);
@@ -885,12 +895,23 @@ void launch_small_conv_fwd(const SmallConvProb& p, bool w_is_bf16, bool is_bf16,
   long long groups = (total + SCF_PIX - 1) / SCF_PIX;
   const unsigned grid = (unsigned)std::min<long long>(groups, 148LL * 8);
   const size_t smem = ((size_t)9 * p.Cin * p.Cout + (size_t)SCF_PIX * (SC_KP + 4)) * sizeof(float);
-  if (is_bf16) {
-    if (w_is_bf16) small_conv_fwd_kernel<bf16, bf16><<<grid, 256, smem, s>>>(p);
-    else small_conv_fwd_kernel<bf16, float><<<grid, 256, smem, s>>>(p);
-  } else {
-    small_conv_fwd_kernel<float, float><<<grid, 256, smem, s>>>(p);
+#define LP_FWD(CO)                                                                                    \
+  do {                                                                                                \
+    if (is_bf16) {                                                                                    \
+      if (w_is_bf16) small_conv_fwd_kernel<bf16, bf16, CO><<<grid, 256, smem, s>>>(p);                \
+      else small_conv_fwd_kernel<bf16, float, CO><<<grid, 256, smem, s>>>(p);                         \
+    } else {                                                                                          \
+      small_conv_fwd_kernel<float, float, CO><<<grid, 256, smem, s>>>(p);                             \
+    }                                                                                                 \
+  } while (0)
+  switch (p.Cout) {
+    case 8: LP_FWD(8); break;
+    case 16: LP_FWD(16); break;
+    case 32: LP_FWD(32); break;
+    case 64: LP_FWD(64); break;
+    default: break;                                      // the builder chooses these kernels for these widths only
   }
+#undef LP_FWD
 }
 void launch_small_conv_wgrad(const SmallConvProb& p, bool is_bf16, cudaStream_t s) {
   const long long total = (long long)p.N * p.H * p.W;
