@@ -522,6 +522,17 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
         // this CTA's 128 output pixels start at row a_h0 of image a_img (whole rows)
         int a_img = 0, a_h0 = 0;
         if (conv != CONV_WGRAD) { a_img = m0 / cv_hw; a_h0 = (m0 - a_img * cv_hw) / cv_w; }
+        // Filter gradient: 64-row boxes that lie wholly beyond the problem's rows (M = C_out of 64: the second A
+        // box) or beyond the last filter tap are not fetched at all.  What the stage then holds there feeds only
+        // accumulator rows >= M and columns >= N, which the epilogue never stores.
+        uint32_t tx_tile = stage_tx;
+        const int p_m = p.M;
+        if (conv == CONV_WGRAD) {
+          int boxes = 0;
+          for (int i = 0; i < BM / 64; ++i) boxes += (m0 + i * 64 < p_m) ? 1 : 0;
+          for (int i = 0; i < bnl / 64; ++i) boxes += ((n0 + i * 64) / cv_c < cv_taps) ? 1 : 0;
+          tx_tile = (uint32_t)boxes * (BK * 128);
+        }
         for (int kb = 0; kb < kb_n; ++kb) {
           if (!(ok = mbar_wait(&sh->empty[stage], phase ^ 1, sh, status))) break;
           uint8_t* a_dst = tiles + stage * STAGE_BYTES;
@@ -529,8 +540,8 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
           int k0 = kb * BK;
           uint64_t* bar1 = &sh->full[stage];
           uint32_t bar2 = 0;
-          if (CG == 1) mbar_expect_tx(bar1, stage_tx);
-          else { bar2 = map_to_rank(smem_u32(bar1), 0); mbar_expect_tx_cluster(bar2, stage_tx); }
+          if (CG == 1) mbar_expect_tx(bar1, tx_tile);
+          else { bar2 = map_to_rank(smem_u32(bar1), 0); mbar_expect_tx_cluster(bar2, tx_tile); }
           auto ld2 = [&](void* dst, const CUtensorMap* map, int x, int y) {
             if (CG == 1) tma_load_2d(dst, map, x, y, bar1); else tma_load_2d_pair(dst, map, x, y, bar2);
           };
@@ -541,14 +552,14 @@ gemm_tc_kernel(const GemmProb* __restrict__ probs, const CUtensorMap* __restrict
             // A: dy as an ordinary MN-major operand; B: 64 pixels (whole rows) of x per 64-column block, each
             // column block with the shift of its own filter tap
 #pragma unroll
-            for (int i = 0; i < BM / 64; ++i) ld2(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0);
+            for (int i = 0; i < BM / 64; ++i)
+              if (m0 + i * 64 < p_m) ld2(a_dst + i * (BK * 128), mapA, m0 + i * 64, k0);
             const int kp = cv_k0 + k0;
             const int img = kp / cv_hw, h0 = (kp - img * cv_hw) / cv_w;
             for (int i = 0; i < bnl / 64; ++i) {
               const int col = n0 + i * 64;
               const int t = col / cv_c, c0 = col - t * cv_c;
               if (t < cv_taps) ld4(b_dst + i * (BK * 128), mapB, c0, tap_dj(t), h0 * cv_s + tap_di(t), img);
-              else ld4(b_dst + i * (BK * 128), mapB, 0, 0, 0, cv_n);        // beyond the last tap: an all-zero box
             }
           } else {
             // k-slice -> (filter tap, channel block); A: 128 pixels shifted by the tap (mirrored for the input gradient)
