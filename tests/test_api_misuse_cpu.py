@@ -55,6 +55,8 @@ def test_null_handles_and_pointers_are_refused():
                  lambda: L.lp_evaluate(None, None, None, None, 0, None, None, None),
                  lambda: L.lp_reset_pipeline(None),
                  lambda: L.lp_set_ramp(None, 0),
+                 lambda: L.lp_set_drain(None, 0),
+                 lambda: L.lp_set_fused_step(None, 1),
                  lambda: L.lp_set_overlap(None, 1),
                  lambda: L.lp_chunk_output(None, 0, None, 0, None),
                  lambda: L.lp_status_poll(None, None),

@@ -87,6 +87,18 @@ def test_mlp_fp32_single_launch_many_tiles_and_classes(schedule):
     check(cfg, fused=True)
 
 
+@pytest.mark.parametrize("fused", [True, False])
+def test_mlp_fp32_weight_decay_one_chunk_and_many_chunks(fused):
+    """SGD with momentum and weight decay (matrices only); K = 1 is back-propagation (Sec. 3), K = 12 one layer per
+    chunk (greedy local learning) in the pipelined schedule."""
+    one = lp_synth.config("c1", batch=33, d_in=70, chunks=[[96, 64, 80]], classes=11)
+    one["optim"] = dict(kind="sgdm", lr=0.05, momentum=0.9, weight_decay=1e-2)
+    check(one, fused=fused)
+    many = lp_synth.config("c1", batch=40, d_in=48, chunks=[[56]] * 12, classes=5, schedule="pipelined")
+    many["optim"] = dict(kind="sgdm", lr=0.02, momentum=0.8, weight_decay=5e-3)
+    check(many, fused=fused)
+
+
 def test_single_launch_step_is_bit_reproducible_and_refused_where_it_does_not_exist():
     from paper_2012_03837_b200 import binding as lp
     cfg = lp_synth.config("c1", batch=70, d_in=33, chunks=[[65], [40, 50], [31]], classes=7, schedule="pipelined")
