@@ -1,8 +1,12 @@
-// ResNet family (App. B.3): a 3x3 stem convolution + BatchNorm + ReLU in chunk 0, then one stage of
-// BasicBlocks per chunk (conv3x3-BN-ReLU-conv3x3-BN, identity or 1x1-stride-2 conv+BN shortcut, ReLU),
-// BatchNorm with batch statistics, and a global-average-pool + Linear + softmax cross-entropy
-// auxiliary head per chunk (Sec. 3).  Activations are NHWC; a convolution is im2col + GEMM
-// (cols are kept for the weight gradient), its input gradient a GEMM + col2im gather.
+// ResNet family (App. B.3): a 3x3 stem convolution + BatchNorm + ReLU in chunk 0, then one stage of residual
+// blocks per chunk -- BasicBlocks (conv3x3-BN-ReLU-conv3x3-BN) or bottleneck blocks (1x1 - 3x3 - 1x1, expansion
+// 4), identity or 1x1-stride-2 conv+BN shortcut, ReLU -- BatchNorm with batch statistics, and a global-average-
+// pool + Linear + softmax cross-entropy auxiliary head per chunk (Sec. 3).  Activations are NHWC.  In bf16 the
+// 3x3 and 1x1 convolutions with channel counts that are multiples of 64 are implicit GEMMs on the tensor cores
+// (no im2col), 1x1 stride-1 convolutions plain GEMMs over [pixels, C], the few-channel stem a direct FP32-ALU
+// kernel; everything else (fp32, the FP32-ALU backend, other channel counts) is im2col + GEMM with the cols kept
+// for the weight gradient and a GEMM + col2im gather for an input gradient.  BatchNorm is one cooperative launch
+// per layer (forward) and per grouped position (backward) in bf16, three launches otherwise.
 //
 // Backward is truncated at the chunk input (Sec. 3): the first block of a stage k > 0 forms no input
 // gradient (no dgrad for its first convolution and its shortcut convolution), nor does the stem.
