@@ -71,7 +71,7 @@ TRAFFIC = {
     # 256x512 tiles), block products 0.76 GB; every chunk streams its own operands, so a 24-chunk step moves
     # 24 x 2.71 GB = 65 GB over its thirteen GEMM launches
     "c5": dict(bytes_per_launch=5.0e9, chunks=24, kernel_file="paper_2012_03837_b200/csrc/gemm_tc.cu",
-               kernel_sha256="81aead8e0c8b6843a85a1c65735b723708c596eae43919f2823f6cb3ac48cf67"),
+               kernel_sha256="38616d45d63a33ff10b9ee02f9b0c1ba6f1147f3479332c7671486713343fb3b"),
 }
 
 
