@@ -40,6 +40,28 @@ def grad_l2_errors(gm, orc):
     return sorted(out, reverse=True)
 
 
+def oracle_precision_gap(cfg, steps):
+    """Largest distance between the oracle run in fp32 and in fp64 over `steps` steps: relative loss gap, matrix
+    gap ||a-b|| / ||b||, vector gap ||a-b|| / ||b - init||.  CPU only."""
+    from oracle.local_step import LocalUpdateOracle
+    init = lp_synth.init_params(cfg)
+    a, b = LocalUpdateOracle(cfg, init, dtype=np.float32), LocalUpdateOracle(cfg, init, dtype=np.float64)
+    out = {"loss": 0.0, "matrix": 0.0, "vector": 0.0}
+    for t in range(steps):
+        x, y = lp_synth.minibatch(cfg, t)
+        la, lb = a.step(x, y), b.step(x, y)
+        out["loss"] = max(out["loss"], float(np.nanmax(np.abs(la - lb) / np.abs(lb))))
+    for n in a.p:
+        if n in a.buffers:
+            continue
+        d = float(np.linalg.norm(a.p[n].astype(np.float64) - b.p[n]))
+        if a.p[n].ndim >= 2:
+            out["matrix"] = max(out["matrix"], d / float(np.linalg.norm(b.p[n])))
+        else:
+            out["vector"] = max(out["vector"], d / max(float(np.linalg.norm(b.p[n] - np.asarray(init[n], np.float64))), 1e-30))
+    return out
+
+
 def check(cfg, steps=10, gemm_backend=0, grads_first=True, w_tol=None, v_tol=None, loss_tol=None, fused=None):
     from paper_2012_03837_b200 import binding as lp
     dt = cfg["dtype"]
@@ -96,7 +118,14 @@ def test_mlp_fp32_weight_decay_one_chunk_and_many_chunks(fused):
     check(one, fused=fused)
     many = lp_synth.config("c1", batch=40, d_in=48, chunks=[[56]] * 12, classes=5, schedule="pipelined")
     many["optim"] = dict(kind="sgdm", lr=0.02, momentum=0.8, weight_decay=5e-3)
-    check(many, fused=fused)
+    # In this run one ReLU input of chunk 8 comes within fp32 rounding of zero at step 8: the oracle in fp32 and in
+    # fp64 take different sides (loss gap 1.3e-5 at step 8, 8.3e-5 at step 9, a bias vector 6.0e-3 apart after ten
+    # steps, everything else 1e-7), and so do two fp32 summation orders -- the grouped launches land on the fp32
+    # oracle's side, the single launch on the fp64 oracle's.  The bounds are therefore the nominal ones or twice
+    # the oracle's own fp32 / fp64 gap, measured here on the CPU.
+    gap = oracle_precision_gap(many, 10)
+    check(many, fused=fused, loss_tol=max(LOSS_TOL["fp32"], 2 * gap["loss"]), w_tol=max(W_TOL["fp32"], 2 * gap["matrix"]),
+          v_tol=max(V_TOL["fp32"], 2 * gap["vector"]))
 
 
 def test_single_launch_step_is_bit_reproducible_and_refused_where_it_does_not_exist():
