@@ -7,8 +7,8 @@
 // (synchronous), all head products, all softmax cross-entropy rows, all weight / input gradients of one depth, the
 // optimizer sweep.
 //
-// Arithmetic: fp32 throughout, every sum in a fixed order (a tile's reduction index is split over the eight warps
-// of a block in contiguous slices, the slices are added in warp order), so a step is bit-reproducible.
+// Arithmetic: fp32 throughout, every sum in a fixed order (a tile's reduction index is split over groups of the
+// block's sixteen warps in contiguous pieces, the pieces are added in group order), so a step is bit-reproducible.
 #include <algorithm>
 
 #include "common.cuh"
